@@ -1,0 +1,128 @@
+"""Seeded synthetic inputs for one auto-correct decoding step.
+
+Only data generation lives here: shapes, value distributions, ragged lengths
+and planted candidates.  None of the step's arithmetic (no attention, softmax,
+arg-max or acceptance test) is computed in this module, so the same bytes can
+be fed to any implementation of the step.
+
+Every tensor is a numpy array; bf16 tensors are uint16 bit patterns.
+"""
+import numpy as np
+
+# name -> shape parameters.  L is an inclusive range of verified cache lengths,
+# p_accept an inclusive range of the per-sequence probability that a candidate
+# is planted as its target row's strict maximum.
+CONFIGS = {
+    "tiny": dict(B=1, H_q=8, H_kv=8, d=64, L=(128, 128), k=4, V=1000,
+                 logits_dtype="f32", sigma=2.0, p_accept=(0.7, 0.7),
+                 mode="greedy", temperature=1.0, seed=0),
+    "llama7b": dict(B=1, H_q=32, H_kv=32, d=128, L=(2048, 2048), k=5, V=32000,
+                    logits_dtype="bf16", sigma=3.0, p_accept=(0.8, 0.8),
+                    mode="greedy", temperature=1.0, seed=1),
+    "ragged16": dict(B=16, H_q=32, H_kv=32, d=128, L=(512, 4096), k=5, V=32000,
+                     logits_dtype="bf16", sigma=3.0, p_accept=(0.3, 0.9),
+                     mode="greedy", temperature=1.0, seed=2),
+    "gqa70b": dict(B=8, H_q=64, H_kv=8, d=128, L=(8192, 8192), k=6, V=32000,
+                   logits_dtype="bf16", sigma=3.0, p_accept=(0.8, 0.8),
+                   mode="greedy", temperature=1.0, seed=3),
+    "sampling64": dict(B=64, H_q=32, H_kv=8, d=128, L=(1024, 16384), k=4, V=128256,
+                       logits_dtype="bf16", sigma=3.0, p_accept=(0.8, 0.8),
+                       mode="sample", temperature=0.8, seed=4),
+}
+
+# Logit written at a planted candidate.  Greedy: far above any N(0, sigma)
+# draw, so the candidate is the row's unique maximum.  Sampling (T = 0.8,
+# sigma = 3, V = 128256): exp(16/0.8) is about three times the sum of the
+# other terms, so a planted candidate carries roughly 0.75 of the mass.
+PLANT_GREEDY = 30.0
+PLANT_SAMPLE = 16.0
+
+
+def f32_to_bf16_bits(x):
+    """float32 array -> round-to-nearest-even bf16 bit patterns (uint16)."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)
+    return r.astype(np.uint16)
+
+
+def n_block_rows(k):
+    return (k + 1) * (k + 1)
+
+
+def resolve(name, **overrides):
+    cfg = dict(CONFIGS[name])
+    cfg.update(overrides)
+    cfg["name"] = name
+    return cfg
+
+
+def _normal_bf16(rng, shape, sigma=1.0):
+    x = rng.standard_normal(shape, dtype=np.float32)
+    if sigma != 1.0:
+        x *= np.float32(sigma)
+    return f32_to_bf16_bits(x)
+
+
+def make_step_inputs(cfg, set_index=0, s_cap=None, poison_tail=False):
+    """One step's inputs for `cfg` (a dict from `resolve`).
+
+    set_index picks an independent input set under the same configuration
+    (used to rotate distinct sets through the L2 cache in timing runs).
+    s_cap is the cache capacity per sequence (default: max length + block rows,
+    rounded up to 64).  Cache rows at and beyond L_b + n_q are zero, or NaN
+    patterns when poison_tail is set.
+    """
+    B, H_q, H_kv, d, k, V = (cfg[x] for x in ("B", "H_q", "H_kv", "d", "k", "V"))
+    n_q = n_block_rows(k)
+    rng = np.random.Generator(np.random.Philox(key=[cfg["seed"], set_index]))
+    lo, hi = cfg["L"]
+    kv_len = rng.integers(lo, hi + 1, size=B).astype(np.int32)
+    if s_cap is None:
+        s_cap = ((hi + n_q + 63) // 64) * 64
+    fill = np.uint16(0x7FC0) if poison_tail else np.uint16(0)
+    k_cache = np.full((B, H_kv, s_cap, d), fill, dtype=np.uint16)
+    v_cache = np.full((B, H_kv, s_cap, d), fill, dtype=np.uint16)
+    for b in range(B):
+        n = int(kv_len[b]) + n_q
+        k_cache[b, :, :n, :] = _normal_bf16(rng, (H_kv, n, d))
+        v_cache[b, :, :n, :] = _normal_bf16(rng, (H_kv, n, d))
+    q = _normal_bf16(rng, (B, n_q, H_q, d))
+
+    if cfg["logits_dtype"] == "f32":
+        logits = rng.standard_normal((B, n_q, V), dtype=np.float32) * np.float32(cfg["sigma"])
+    else:
+        logits = np.empty((B, n_q, V), dtype=np.uint16)
+        for b in range(B):
+            logits[b] = _normal_bf16(rng, (n_q, V), cfg["sigma"])
+    cand = rng.integers(0, V, size=(B, k)).astype(np.int32)
+    p_lo, p_hi = cfg["p_accept"]
+    p_seq = rng.uniform(p_lo, p_hi, size=B)
+    planted = rng.uniform(size=(B, k)) < p_seq[:, None]
+    plant = PLANT_GREEDY if cfg["mode"] == "greedy" else PLANT_SAMPLE
+    plant_val = np.float32(plant) if logits.dtype == np.float32 \
+        else f32_to_bf16_bits(np.float32(plant))
+    for b in range(B):
+        for i in range(k):
+            if planted[b, i]:
+                logits[b, i * (k + 1), cand[b, i]] = plant_val   # target row of c_{i+1}
+    cand_prob = np.ones((B, k), dtype=np.float32)
+    seq_id = np.arange(B, dtype=np.uint32)
+    return dict(q=q, k_cache=k_cache, v_cache=v_cache, kv_len=kv_len, logits=logits,
+                cand=cand, cand_prob=cand_prob, seq_id=seq_id, planted=planted,
+                s_cap=s_cap, n_q=n_q, scale=float(1.0 / np.sqrt(d)))
+
+
+def algorithmic_bytes(cfg, kv_len, n_accept=None):
+    """Bytes one step has to move at least once: K and V of the cache and block,
+    Q, the attention output (as bf16), 2k+1 logits rows per sequence and the
+    committed rows (read + write).  Used for roofline reporting only."""
+    B, H_q, H_kv, d, k, V = (cfg[x] for x in ("B", "H_q", "H_kv", "d", "k", "V"))
+    n_q = n_block_rows(k)
+    esz = 4 if cfg["logits_dtype"] == "f32" else 2
+    keys = int(np.sum(np.asarray(kv_len, dtype=np.int64) + n_q))
+    kv = keys * H_kv * d * 2 * 2
+    qo = B * n_q * H_q * d * 2 * 2
+    lg = B * (2 * k + 1) * V * esz
+    acc = int(np.sum(n_accept)) if n_accept is not None else 0
+    cm = acc * H_kv * d * 2 * 2 * 2
+    return dict(kv=kv, q_out=qo, logits=lg, commit=cm, total=kv + qo + lg + cm)

@@ -1,0 +1,195 @@
+"""Pins for oracle.verify: greedy invariants (Sec. 3.2 / Table 1 setting),
+acceptance statistics and output marginals of rejection sampling over 10^6
+Philox-driven trials on a 16-token vocabulary."""
+import numpy as np
+import pytest
+
+from oracle import layout
+from oracle.verify import verify_step, softmax_rows, accept_uniform, gumbel_noise
+
+INF = float("inf")
+
+
+def _logits(rng, B, k, V, sigma=2.0):
+    return rng.standard_normal((B, layout.n_block_rows(k), V)) * sigma
+
+
+# ------------------------------------------------------------------ greedy
+@pytest.mark.parametrize("k", [1, 2, 4, 5])
+def test_greedy_accepts_longest_prefix_of_argmax_chain(k):
+    rng = np.random.default_rng(k)
+    B, V = 400, 12
+    z = _logits(rng, B, k, V)
+    chain = np.argmax(z[:, layout.target_rows(k), :], axis=-1)         # [B, k+1]
+    cand = chain[:, :k].copy()
+    # break the chain at a random place for most sequences
+    cut = rng.integers(0, k + 2, size=B)
+    for b in range(B):
+        if cut[b] < k:
+            cand[b, cut[b]] = (cand[b, cut[b]] + 1 + rng.integers(0, V - 1)) % V
+    r = verify_step(z, cand, np.ones((B, k)), k, "greedy")
+    for b in range(B):
+        n = 0
+        while n < k and cand[b, n] == chain[b, n]:
+            n += 1
+        assert r["n_accept"][b] == n == min(cut[b], k)
+        assert r["n_out"][b] == n + 1 and 1 <= r["n_out"][b] <= k + 1       # Sec. 3.2
+        assert list(r["out_tokens"][b, : n + 1]) == list(chain[b, : n + 1])
+        assert all(r["out_tokens"][b, n + 1:] == -1)
+        rows = layout.mask_group_rows(k, n)
+        assert list(r["next_cand"][b]) == [int(np.argmax(z[b, rr])) for rr in rows]
+        p = softmax_rows(z[b, rows[0]])
+        assert np.isclose(r["next_cand_prob"][b, 0], p.max(), rtol=1e-12)
+
+
+def test_greedy_ties_take_lowest_index_and_first_step_emits_one_token():
+    k, V = 3, 8
+    z = np.zeros((1, layout.n_block_rows(k), V))
+    z[0, :, [2, 5]] = 1.0                                   # exact tie everywhere
+    r = verify_step(z, np.array([[5, 5, 5]]), np.full((1, k), INF), k, "greedy")
+    assert r["n_accept"][0] == 0 and r["out_tokens"][0, 0] == 2 and r["n_out"][0] == 1
+    r = verify_step(z, np.array([[2, 2, 5]]), np.ones((1, k)), k, "greedy")
+    assert r["n_accept"][0] == 2 and list(r["out_tokens"][0]) == [2, 2, 2, -1]
+    assert list(r["next_cand"][0]) == [2, 2, 2]
+
+
+def test_out_of_range_candidate_is_rejected():
+    k, V = 2, 6
+    z = _logits(np.random.default_rng(0), 1, k, V)
+    for mode in ("greedy", "sample"):
+        r = verify_step(z, np.array([[V + 3, 1]]), np.ones((1, k)), k, mode, seed=1)
+        assert r["n_accept"][0] == 0
+        r = verify_step(z, np.array([[-1, 1]]), np.ones((1, k)), k, mode, seed=1)
+        assert r["n_accept"][0] == 0
+
+
+def test_eos_truncates():
+    k, V = 3, 10
+    z = np.full((1, layout.n_block_rows(k), V), -5.0)
+    for t, tok in zip(layout.target_rows(k), (4, 7, 9, 1)):
+        z[0, t, tok] = 5.0
+    r = verify_step(z, np.array([[4, 7, 9]]), np.ones((1, k)), k, "greedy", eos_id=9)
+    assert r["n_accept"][0] == 3 and r["n_out"][0] == 2 and r["finished"][0] == 1
+    assert list(r["out_tokens"][0]) == [4, 7, -1, -1]
+    r = verify_step(z, np.array([[4, 7, 9]]), np.ones((1, k)), k, "greedy", eos_id=3)
+    assert r["n_out"][0] == 4 and r["finished"][0] == 0
+
+
+def test_planted_generator_statistics():
+    # With candidates planted as the row maximum with probability p, the expected
+    # accepted count is sum_{i=1..k} p^i (tiny: 1.773, llama7b: 2.689).
+    from paper_2402_11809_b200 import workloads
+    cfg = workloads.resolve("tiny", B=3000, V=64, L=(4, 4), H_q=1, H_kv=1, d=8)
+    x = workloads.make_step_inputs(cfg)
+    r = verify_step(x["logits"], x["cand"], x["cand_prob"], cfg["k"], "greedy")
+    want = sum(0.7 ** i for i in range(1, 5))
+    assert abs(r["n_accept"].mean() - want) < 0.08
+    # accepted count equals the length of the leading run of planted candidates,
+    # except when an unplanted random candidate happens to be the arg-max (1/V)
+    run = np.cumprod(x["planted"], axis=1).sum(axis=1)
+    assert np.mean(r["n_accept"] == run) > 0.95 and np.all(r["n_accept"] >= run)
+
+
+# ---------------------------------------------------------------- sampling
+N = 1_000_000
+V16 = 16
+
+
+def _chi2(counts, probs):
+    n = counts.sum()
+    keep = probs > 0
+    assert counts[~keep].sum() == 0
+    return float((((counts[keep] - n * probs[keep]) ** 2) / (n * probs[keep])).sum()), int(keep.sum()) - 1
+
+
+def _fixed_logits(k, seed):
+    rng = np.random.default_rng(seed)
+    z = rng.standard_normal((1, layout.n_block_rows(k), V16)) * 1.5
+    return np.broadcast_to(z, (N, layout.n_block_rows(k), V16))
+
+
+def test_first_step_rejects_everything():
+    # Algorithm 1 starts with P_c = +inf: nothing can be accepted, one token comes out
+    k = 2
+    z = _fixed_logits(k, 0)[:1000]
+    r = verify_step(z, np.zeros((1000, k), dtype=int), np.full((1000, k), INF), k, "sample",
+                    temperature=0.9, seed=5, seq_id=np.arange(1000))
+    assert np.all(r["n_accept"] == 0) and np.all(r["n_out"] == 1)
+
+
+def test_lossless_variant_reproduces_target_marginals():
+    k, T, seed = 2, 0.8, 20240211
+    z = _fixed_logits(k, 1)
+    q = softmax_rows(z[0, layout.target_rows(k)], T)                   # [k+1, V]
+    c = np.array([int(np.argsort(q[0])[-2]), int(np.argmax(q[1]))])     # fixed drafts
+    cand = np.broadcast_to(c, (N, k))
+    r = verify_step(z, cand, np.ones((N, k)), k, "sample", temperature=T, seed=seed,
+                    seq_id=np.arange(N), kv_len=np.full(N, 11))
+    # acceptance rate of a point-mass draft is q(c)
+    acc1 = (r["n_accept"] >= 1).mean()
+    assert abs(acc1 - q[0, c[0]]) < 5 * np.sqrt(q[0, c[0]] * (1 - q[0, c[0]]) / N)
+    # first emitted token ~ q_0
+    chi, dof = _chi2(np.bincount(r["out_tokens"][:, 0], minlength=V16), q[0])
+    assert chi < 55.0, chi                                              # 15 dof, p ~ 1e-6
+    # second emitted token, given the first candidate was accepted, ~ q_1
+    sel = r["n_accept"] >= 1
+    chi, dof = _chi2(np.bincount(r["out_tokens"][sel, 1], minlength=V16), q[1])
+    assert chi < 55.0, chi
+    sel2 = r["n_accept"] >= 2
+    assert abs(sel2.sum() / sel.sum() - q[1, c[1]]) < 6 * np.sqrt(0.25 / sel.sum())
+    chi, dof = _chi2(np.bincount(r["out_tokens"][sel2, 2], minlength=V16), q[2])
+    assert chi < 55.0, chi
+    # after a rejection the rejected token is never re-drawn
+    rej0 = r["n_accept"] == 0
+    assert not np.any(r["out_tokens"][rej0, 0] == c[0])
+    # new candidates: arg-max of the chosen group's mask rows, probability one
+    for g in range(k + 1):
+        rows = layout.mask_group_rows(k, g)
+        want = [int(np.argmax(z[0, rr])) for rr in rows]
+        assert np.all(r["next_cand"][r["n_accept"] == g] == want)
+    assert np.all(r["next_cand_prob"] == 1.0)
+
+
+def test_literal_variant_matches_its_closed_form():
+    # Algorithm 1 as printed: draft c ~ p, accept w.p. min(1, q/p), extra token a ~ q
+    # also after a rejection.  First-token law: min(p,q)(x) + (1 - sum min(p,q)) q(x).
+    k, T, seed = 1, 1.0, 99
+    z = _fixed_logits(k, 2)
+    q = softmax_rows(z[0, layout.target_rows(k)], T)
+    rng = np.random.default_rng(7)
+    p = softmax_rows(rng.standard_normal(V16) * 1.5)
+    c = rng.choice(V16, size=N, p=p)
+    r = verify_step(z, c[:, None], p[c][:, None], k, "sample", temperature=T, seed=seed,
+                    seq_id=np.arange(N), resample="paper_literal")
+    mn = np.minimum(p, q[0])
+    assert abs((r["n_accept"] == 1).mean() - mn.sum()) < 5 * np.sqrt(0.25 / N)
+    law = mn + (1.0 - mn.sum()) * q[0]
+    chi, _ = _chi2(np.bincount(r["out_tokens"][:, 0], minlength=V16), law)
+    assert chi < 55.0, chi
+    # ... which is measurably not the target law (the lossless variant above is)
+    chi_q, _ = _chi2(np.bincount(r["out_tokens"][:, 0], minlength=V16), q[0])
+    assert chi_q > 500.0
+    # sampled new candidates follow their mask row's distribution and carry its probability
+    for g in (0, 1):
+        sel = r["n_accept"] == g
+        row = layout.mask_group_rows(k, g)[0]
+        pm = softmax_rows(z[0, row], T)
+        chi, _ = _chi2(np.bincount(r["next_cand"][sel, 0], minlength=V16), pm)
+        assert chi < 55.0, chi
+        assert np.allclose(r["next_cand_prob"][sel, 0], pm[r["next_cand"][sel, 0]])
+
+
+def test_draws_are_keyed_by_seed_sequence_and_position():
+    a = accept_uniform(1, np.array([0, 1, 0]), np.array([5, 5, 6]))
+    assert len(set(a.tolist())) == 3
+    assert accept_uniform(2, np.array([0]), np.array([5]))[0] != a[0]
+    g1 = gumbel_noise(1, 1, np.array([3]), np.array([9]), 10)
+    g2 = gumbel_noise(1, 2, np.array([3]), np.array([9]), 10)
+    assert g1.shape == (1, 10) and not np.array_equal(g1, g2)
+    # re-running a step from the same inputs reproduces it exactly (stateless RNG)
+    k = 2
+    z = _fixed_logits(k, 3)[:500]
+    kw = dict(temperature=0.7, seed=11, seq_id=np.arange(500), kv_len=np.arange(500))
+    r1 = verify_step(z, np.ones((500, k), dtype=int), np.ones((500, k)), k, "sample", **kw)
+    r2 = verify_step(z, np.ones((500, k), dtype=int), np.ones((500, k)), k, "sample", **kw)
+    assert all(np.array_equal(r1[x], r2[x]) for x in r1)
