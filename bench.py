@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Benchmark of one auto-correct decoding step (attention + verify + KV commit).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+One step = space_attn_step + space_verify + space_kv_commit for the whole batch
+of one synthetic input set.  Several distinct input sets are rotated so that no
+step finds its inputs in L2.  Prints ONE JSON line (rank 0).
+
+--impl ours       the CUDA library.  `value` is steps/s with inputs resident in
+                  HBM, the K steps replayed from a CUDA graph.  `roofline` comes
+                  from CUDA events recorded around every attention-kernel launch
+                  in a second, stream-launched pass over the same steps; `e2e`
+                  from space_step_host with pinned host buffers; `cpu_baseline`
+                  from the CPU oracle on the host cores.
+--impl reference  the CPU oracle alone on the host cores (rank 0 only).
+With N > 1 (torchrun) every rank runs an independent replica on its own GPU.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+from paper_2402_11809_b200 import workloads  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+METRIC = "auto-correct steps/sec"
+UNIT = "steps/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ---------------------------------------------------------------- clock sampler
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while running."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+            nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------- CPU oracle
+def oracle_step(cfg, x):
+    """One whole step with the CPU oracle (attention, verify, commit)."""
+    from oracle.attention import attention_step
+    from oracle.verify import verify_step
+    from oracle.commit import commit_step
+    k = cfg["k"]
+    attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], k, x["scale"])
+    r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, cfg["mode"],
+                    temperature=cfg["temperature"], seed=cfg["seed"], seq_id=x["seq_id"],
+                    kv_len=x["kv_len"])
+    kc, vc = x["k_cache"].copy(), x["v_cache"].copy()
+    commit_step(kc, vc, x["kv_len"], r["n_accept"], k)
+    return r
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(cfg, x, budget_s, min_reps=3, max_reps=None):
+    oracle_step(cfg, x)                                   # warm-up (imports, BLAS threads)
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        oracle_step(cfg, x)
+        reps += 1
+        el = time.perf_counter() - t0
+        if max_reps is not None and reps >= max_reps:
+            break
+        if max_reps is None and reps >= min_reps and el >= budget_s:
+            break
+    return reps / el, reps, el
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = workloads.resolve(args.config)
+    x = workloads.make_step_inputs(cfg)
+    for _ in range(args.warmup if args.warmup < 3 else 2):
+        oracle_step(cfg, x)
+    # bounded: at most ~150 s of timed work; a "step" stays one whole step of the
+    # workload and the number of timed repetitions is what is bounded
+    t0 = time.perf_counter()
+    oracle_step(cfg, x)
+    one = time.perf_counter() - t0
+    reps = max(1, min(args.steps, int(150.0 / max(one, 1e-6))))
+    sps, reps, el = time_oracle(cfg, x, 0.0, max_reps=reps)
+    cores = blas_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": sps, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / sps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": cfg["name"], "timed_steps": reps,
+                   "note": "CPU oracle (numpy fp64), whole steps; repetitions bounded to ~150 s"},
+        "cpu_baseline": {"value": sps, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{reps} whole step(s) of {cfg['name']} in {el:.1f} s"},
+        "e2e": {"value": sps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------- CUDA arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import gpu_harness as H
+    from paper_2402_11809_b200 import build
+    build.build()
+    from paper_2402_11809_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --impl ours needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    cfg = workloads.resolve(args.config)
+    k, n_q = cfg["k"], workloads.n_block_rows(cfg["k"])
+    sample = cfg["mode"] == "sample"
+    mode = B.MODE_SAMPLE if sample else B.MODE_GREEDY
+
+    # ---- input sets: enough distinct sets that their footprint is twice L2 ----
+    x0 = workloads.make_step_inputs(cfg, set_index=rank * 1000)
+    ab = workloads.algorithmic_bytes(cfg, x0["kv_len"])
+    n_sets = max(2, int(np.ceil(2.0 * L2_BYTES / ab["total"])))
+    n_sets = min(n_sets, 16)
+    sets = [x0] + [workloads.make_step_inputs(cfg, set_index=rank * 1000 + i) for i in range(1, n_sets)]
+
+    s_cap = max(x["s_cap"] for x in sets)
+    ctx = B.Context(device=local, max_batch=cfg["B"], n_q_heads=cfg["H_q"], n_kv_heads=cfg["H_kv"],
+                    head_dim=cfg["d"], k_max=k, vocab=cfg["V"], host_staging=1, s_cap=s_cap)
+    steps_dev = [H.DeviceStep(cfg, x) for x in sets]
+    arg_sets = []
+    for ds in steps_dev:
+        a = ctx.attn_args(ds.q, ds.k_cache, ds.v_cache, ds.kv_len, ds.out, k, ds.scale, status=ds.status)
+        v = ctx.verify_args(ds.logits, ds.cand, ds.cand_prob, ds.kv_len, ds.n_accept, ds.out_tokens,
+                            ds.n_out, ds.next_cand, ds.next_cand_prob, ds.finished, k, mode=mode,
+                            temperature=cfg["temperature"], seed=cfg["seed"], seq_id=ds.seq_id,
+                            status=ds.status)
+        c = ctx.commit_args(ds.k_cache, ds.v_cache, ds.n_accept, ds.kv_len, k, kv_len_out=ds.kv_len_out,
+                            status=ds.status)
+        arg_sets.append((a, v, c))
+
+    def step(i):
+        a, v, c = arg_sets[i % n_sets]
+        ctx.space_attn_step(a)
+        ctx.space_verify(v)
+        ctx.space_kv_commit(c)
+
+    stream = torch.cuda.Stream()
+    K, W = args.steps, max(args.warmup, 3)
+    with torch.cuda.stream(stream):
+        for i in range(n_sets):                           # first launches, descriptor set-up
+            step(i)
+        stream.synchronize()
+        n0 = ctx.launch_count
+        step(0)
+        launches_per_step = ctx.launch_count - n0
+        # one graph holding n_sets consecutive steps, one holding the remainder
+        g_full = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_full, stream=stream):
+            for i in range(n_sets):
+                step(i)
+        rem = K % n_sets
+        g_rem = None
+        if rem:
+            g_rem = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_rem, stream=stream):
+                for i in range(rem):
+                    step(i)
+
+        def run_steps(n):
+            for _ in range(n // n_sets):
+                g_full.replay()
+            if n % n_sets:
+                if n % n_sets == rem and g_rem is not None:
+                    g_rem.replay()
+                else:
+                    for i in range(n % n_sets):
+                        step(i)
+
+        run_steps(W)
+        stream.synchronize()
+        sampler = ClockSampler(local)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        run_steps(K)
+        e1.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms = e0.elapsed_time(e1)
+        # keep the sampler running through the kernel-timing pass as well
+        # ---- second pass: per-kernel CUDA events, stream-launched ------------
+        n_prof = min(K, 2048)
+        ctx.space_profile_enable(1)
+        for i in range(n_prof):
+            step(i)
+        stream.synchronize()
+        ctx.space_profile_enable(0)
+        prof = ctx.space_profile_read()
+        clocks = sampler.stop()
+        status = sum(int(ds.status.abs().sum()) for ds in steps_dev)
+
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    steps_per_s = world * K / (ms * 1e-3)
+
+    # ---- end to end from pinned host buffers (space_step_host) ---------------
+    import ctypes as C
+    x = sets[0]
+    pin = {}
+    for name in ("q", "k_cache", "v_cache", "logits", "cand", "cand_prob", "kv_len"):
+        arr = x[name]
+        t = torch.from_numpy(arr.view(np.int16) if arr.dtype == np.uint16 else arr).clone().pin_memory()
+        pin[name] = t
+    kv_len0 = pin["kv_len"].clone()
+    outs = dict(out=torch.empty((cfg["B"], n_q, cfg["H_q"], cfg["d"]), dtype=torch.float32).pin_memory(),
+                n_accept=torch.empty(cfg["B"], dtype=torch.int32).pin_memory(),
+                out_tokens=torch.empty((cfg["B"], k + 1), dtype=torch.int32).pin_memory(),
+                n_out=torch.empty(cfg["B"], dtype=torch.int32).pin_memory(),
+                next_cand=torch.empty((cfg["B"], k), dtype=torch.int32).pin_memory(),
+                next_cand_prob=torch.empty((cfg["B"], k), dtype=torch.float32).pin_memory(),
+                finished=torch.empty(cfg["B"], dtype=torch.uint8).pin_memory(),
+                status=torch.empty(cfg["B"], dtype=torch.int32).pin_memory())
+    h2d, d2h = C.c_int64(0), C.c_int64(0)
+    hs = B.HostStepArgs(batch=cfg["B"], k=k, vocab=cfg["V"],
+                        logits_dtype=B.DTYPE_F32 if cfg["logits_dtype"] == "f32" else B.DTYPE_BF16,
+                        mode=mode, resample=B.RESAMPLE_RESIDUAL_POINTMASS, eos_id=-1,
+                        mask_variant=B.MASK_SAME_GROUP, scale=x["scale"], temperature=cfg["temperature"],
+                        seed=cfg["seed"],
+                        **{n_: C.c_void_p(t.data_ptr()) for n_, t in pin.items()},
+                        **{n_: C.c_void_p(t.data_ptr()) for n_, t in outs.items()},
+                        h2d_bytes=C.cast(C.pointer(h2d), C.c_void_p), d2h_bytes=C.cast(C.pointer(d2h), C.c_void_p))
+    n_e2e = max(3, min(K, 100))
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            pin["kv_len"].copy_(kv_len0)
+            ctx.space_step_host(hs)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            pin["kv_len"].copy_(kv_len0)
+            ctx.space_step_host(hs)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+    e2e_val = n_e2e / e2e_s
+    if world > 1:
+        t = torch.tensor([e2e_s], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_val = world * n_e2e / float(t.item())
+    e2e_ok = bool((outs["status"] == 0).all()) and \
+        bool(torch.equal(outs["n_accept"], steps_dev[0].n_accept.cpu()))
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (attention) --------------------------
+    peak, peak_src = load_peaks()
+    attn_ms, attn_n = prof["attn"]
+    attn_bytes = np.mean([workloads.algorithmic_bytes(cfg, s["kv_len"])["kv"] +
+                          workloads.algorithmic_bytes(cfg, s["kv_len"])["q_out"] for s in sets])
+    attn_us = 1e3 * attn_ms / max(attn_n, 1)
+    achieved = attn_bytes / (attn_us * 1e-6) / 1e9 if attn_n else None
+    step_bytes = float(np.mean([workloads.algorithmic_bytes(cfg, s["kv_len"],
+                                                            steps_dev[i].n_accept.cpu().numpy())["total"]
+                                for i, s in enumerate(sets)]))
+    per_kernel_us = {name: (1e3 * v[0] / v[1] if v[1] else None) for name, v in prof.items()}
+
+    # ---- CPU oracle on the host cores (bounded: about 10 s) -------------------
+    cpu_sps, cpu_reps, cpu_el = time_oracle(cfg, sets[0], budget_s=10.0)
+
+    line = {
+        "metric": METRIC, "value": steps_per_s, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg["name"], "batch": cfg["B"], "k": k, "heads": [cfg["H_q"], cfg["H_kv"]],
+                   "head_dim": cfg["d"], "kv_len": list(cfg["L"]), "vocab": cfg["V"], "mode": cfg["mode"],
+                   "l2": f"{n_sets} distinct input sets rotated ({n_sets * ab['total'] / 1e6:.0f} MB > 2 x L2)",
+                   "launch": "CUDA graph replay of the three C-ABI calls",
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "gpu_launches": int(launches_per_step * K),
+        "step_algorithmic_bytes": step_bytes,
+        "step_hbm_frac": step_bytes / (ms / K * 1e-3) / 1e9 / peak,
+        "roofline": {"bound": "hbm", "kernel": "attn_tc_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "traffic": None,
+                     "peak_source": peak_src + " (burst copy figure)",
+                     "algorithmic_bytes_per_launch": float(attn_bytes), "avg_launch_us": attn_us,
+                     "launches_timed": int(attn_n),
+                     "timing": "CUDA events around every launch, stream-launched pass after the graph-timed region",
+                     "kernel_us": per_kernel_us},
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d.value),
+                "d2h_bytes_per_step": int(d2h.value), "steps": n_e2e, "matches_device_run": e2e_ok},
+        "cpu_baseline": {"value": cpu_sps, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                         "sample": f"{cpu_reps} whole step(s) of {cfg['name']} in {cpu_el:.1f} s"},
+        "clocks": clocks,
+        "device_status_bits": status,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--config", default="llama7b", choices=sorted(workloads.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

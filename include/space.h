@@ -1,0 +1,226 @@
+/* libspace - one auto-correct decoding step of SPACE (arXiv 2402.11809) on
+ * NVIDIA B200 (sm_100a).
+ *
+ * One step is the single model invocation of Algorithm 1: the block of
+ * (k+1)^2 query rows (last verified token, k candidates, k+1 groups of k mask
+ * tokens, Eq. 4) attends over the verified KV cache under the mask of Eq. 5,
+ * the resulting logits verify the candidates and propose the next ones
+ * (Algorithm 1, Sec. 3.2), and the accepted rows are compacted into the cache.
+ *
+ * Conventions
+ *  - Every pointer named "device" must be device memory of the context's GPU;
+ *    "host" pointers are ordinary host memory.  The library never takes
+ *    ownership of a caller buffer; it borrows it until the work enqueued on
+ *    the given stream has finished.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *    stream).  All entry points except space_step_host are asynchronous and
+ *    perform no allocation and no synchronisation after space_create.
+ *  - Return value: SPACE_OK or a negative SPACE_E_* code; nothing aborts.
+ *    Conditions only the GPU can see are reported per sequence in the
+ *    `status` array (bit set of SPACE_ST_*).
+ *  - Block row order: row g*(k+1)+o, g = 0..k sub-block, o = 0 the real token
+ *    (root for g = 0, candidate c_g otherwise), o = 1..k the o-th mask token.
+ */
+#ifndef SPACE_H
+#define SPACE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPACE_MAX_K     7      /* (k+1)^2 <= 64 block rows                    */
+#define SPACE_MAX_ROWS  64
+
+enum {
+  SPACE_OK            =  0,
+  SPACE_E_INVALID_ARG = -1,    /* NULL pointer, size out of range             */
+  SPACE_E_UNSUPPORTED = -2,    /* shape outside what the kernels implement    */
+  SPACE_E_ALIGNMENT   = -3,    /* base pointer / stride not 16-byte aligned   */
+  SPACE_E_WORKSPACE   = -4,    /* request exceeds what space_create reserved  */
+  SPACE_E_CUDA        = -5,    /* a CUDA runtime or driver call failed        */
+  SPACE_E_NO_DEVICE   = -6     /* no usable sm_100 device                     */
+};
+
+enum { SPACE_MASK_SAME_GROUP = 0, SPACE_MASK_EQ5_LITERAL = 1 };
+enum { SPACE_MODE_GREEDY = 0, SPACE_MODE_SAMPLE = 1 };
+enum { SPACE_RESAMPLE_RESIDUAL_POINTMASS = 0, SPACE_RESAMPLE_PAPER_LITERAL = 1 };
+enum { SPACE_DTYPE_BF16 = 0, SPACE_DTYPE_F32 = 1 };
+enum { SPACE_ATTN_TENSOR = 0, SPACE_ATTN_SIMT = 1 };
+
+/* per-sequence device status bits */
+enum {
+  SPACE_ST_CAPACITY      = 1,  /* kv_len + (k+1)^2 exceeds the cache capacity */
+  SPACE_ST_BAD_CANDIDATE = 2,  /* a candidate id outside [0, vocab): rejected */
+  SPACE_ST_TIMEOUT       = 4   /* a bounded on-chip wait expired              */
+};
+
+typedef struct space_ctx space_ctx;   /* opaque; owns only its own workspace */
+
+typedef struct {
+  int32_t device;        /* CUDA device ordinal                                */
+  int32_t max_batch;     /* largest batch any call will pass                   */
+  int32_t n_q_heads;     /* H_q                                                */
+  int32_t n_kv_heads;    /* H_kv, divides H_q; H_q/H_kv in {1,2,4,8,16}        */
+  int32_t head_dim;      /* d in {64, 128}                                     */
+  int32_t k_max;         /* largest k any call will pass, 1..SPACE_MAX_K       */
+  int32_t vocab;         /* largest vocabulary any verify call will pass       */
+  int32_t host_staging;  /* != 0: also reserve device staging for space_step_host */
+  int64_t s_cap;         /* cache capacity (rows) per sequence and KV head     */
+} space_config;
+
+/* Block layout of Eq. 4 with the visibility rule of Eq. 5 and the position
+ * rule of Sec. 3.2 (position = number of visible keys - 1). */
+typedef struct {
+  int32_t  k;
+  int32_t  n_q;                          /* (k+1)^2                            */
+  uint8_t  kind[SPACE_MAX_ROWS];         /* 0 real token, 1 mask token         */
+  uint8_t  group[SPACE_MAX_ROWS];        /* sub-block g                        */
+  uint8_t  offset[SPACE_MAX_ROWS];       /* o                                  */
+  int32_t  relpos[SPACE_MAX_ROWS];       /* position id minus kv_len           */
+  uint64_t mask[SPACE_MAX_ROWS];         /* bit j: row attends to block row j  */
+  int32_t  target_rows[SPACE_MAX_K + 1]; /* row of the real token of sub-block t */
+} space_layout_t;
+
+/* Attention of the block over cache + block (Algorithm 1 model call restricted
+ * to the attention operator; Eq. 5).  The caller has already written the
+ * block's K/V rows at cache positions kv_len[b] .. kv_len[b]+n_q-1. */
+typedef struct {
+  int32_t batch;            /* B <= max_batch                                  */
+  int32_t k;                /* candidates per sequence                         */
+  int32_t mask_variant;     /* SPACE_MASK_*                                    */
+  int32_t out_dtype;        /* SPACE_DTYPE_F32 or SPACE_DTYPE_BF16             */
+  int32_t impl;             /* SPACE_ATTN_TENSOR (default) or SPACE_ATTN_SIMT  */
+  float   scale;            /* softmax scale, normally 1/sqrt(d)               */
+  const void*    q;         /* device bf16 [B, n_q, H_q, d], contiguous        */
+  const void*    k_cache;   /* device bf16, element (b,h,s,:) at               */
+  const void*    v_cache;   /*   b*stride_b + h*stride_h + s*stride_s (elements), d contiguous */
+  int64_t kv_stride_b, kv_stride_h, kv_stride_s;  /* multiples of 8 elements   */
+  const int32_t* kv_len;    /* device [B] verified lengths L_b                 */
+  void*          out;       /* device [B, n_q, H_q, d] of out_dtype            */
+  float*         lse;       /* device [B, H_q, n_q] natural-log sum-exp, or NULL */
+  int32_t*       status;    /* device [B], OR-ed with SPACE_ST_*, or NULL      */
+} space_attn_args;
+
+/* Verification and emission (Algorithm 1 after the model call; Sec. 3.2). */
+typedef struct {
+  int32_t batch, k, vocab;
+  int32_t logits_dtype;        /* SPACE_DTYPE_BF16 or SPACE_DTYPE_F32          */
+  int32_t mode;                /* SPACE_MODE_*                                 */
+  int32_t resample;            /* SPACE_RESAMPLE_* (sampling mode only)        */
+  int32_t eos_id;              /* -1: no end-of-sequence handling              */
+  float   temperature;         /* > 0 (sampling mode)                          */
+  uint64_t seed;               /* Philox key                                   */
+  const void*     logits;      /* device [B, n_q, V]; row stride below         */
+  int64_t         logits_row_stride;   /* elements between rows; batch stride = n_q * row stride */
+  const int32_t*  cand;        /* device [B, k]  L_c                           */
+  const float*    cand_prob;   /* device [B, k]  P_c (+inf allowed)            */
+  const uint32_t* seq_id;      /* device [B] or NULL (= batch index)           */
+  const int32_t*  kv_len;      /* device [B]: positions for the random counters */
+  int32_t* n_accept;           /* device [B]       i*                          */
+  int32_t* out_tokens;         /* device [B, k+1]  emitted tokens, -1 padded   */
+  int32_t* n_out;              /* device [B]       emitted count               */
+  int32_t* next_cand;          /* device [B, k]                                */
+  float*   next_cand_prob;     /* device [B, k]                                */
+  uint8_t* finished;           /* device [B]       1 once <EOS> was emitted    */
+  int32_t* status;             /* device [B] or NULL                           */
+} space_verify_args;
+
+/* Compaction of the accepted rows (no counterpart in Algorithm 1, which
+ * re-runs the model on the whole sequence; needed by any cached forward). */
+typedef struct {
+  int32_t batch, k;
+  void*   k_cache;             /* device bf16, same addressing as space_attn_args */
+  void*   v_cache;
+  int64_t kv_stride_b, kv_stride_h, kv_stride_s;
+  const int32_t* n_accept;     /* device [B] from space_verify                 */
+  const int32_t* kv_len;       /* device [B] lengths before the step           */
+  int32_t* kv_len_out;         /* device [B] lengths after, may alias kv_len, or NULL */
+  int32_t* commit_src;         /* device [B, k+1] or NULL, -1 padded           */
+  int32_t* commit_dst;         /* device [B, k+1] or NULL                      */
+  int32_t* status;             /* device [B] or NULL                           */
+} space_commit_args;
+
+/* Whole step from host memory (copies in, the three stages, copies out). */
+typedef struct {
+  int32_t batch, k, vocab, logits_dtype, mode, resample, eos_id, mask_variant;
+  float   scale, temperature;
+  uint64_t seed;
+  const void*    q;            /* host bf16 [B, n_q, H_q, d]                   */
+  void*          k_cache;      /* host bf16 [B, H_kv, s_cap, d]; committed rows are written back */
+  void*          v_cache;
+  const void*    logits;       /* host [B, n_q, V] contiguous                  */
+  const int32_t* cand;         /* host [B, k]                                  */
+  const float*   cand_prob;    /* host [B, k]                                  */
+  int32_t*       kv_len;       /* host [B]; updated in place                   */
+  float*    out;               /* host f32 [B, n_q, H_q, d]                    */
+  int32_t*  n_accept;          /* host [B]                                     */
+  int32_t*  out_tokens;        /* host [B, k+1]                                */
+  int32_t*  n_out;             /* host [B]                                     */
+  int32_t*  next_cand;         /* host [B, k]                                  */
+  float*    next_cand_prob;    /* host [B, k]                                  */
+  uint8_t*  finished;          /* host [B]                                     */
+  int32_t*  status;            /* host [B]                                     */
+  int64_t*  h2d_bytes;         /* host, optional: bytes copied to the device   */
+  int64_t*  d2h_bytes;         /* host, optional: bytes copied back            */
+} space_host_step_args;
+
+/* Create a context on cfg->device: validates the shape, reserves the
+ * workspace (split partials, reduction scratch, counters, optional staging).
+ * Errors: INVALID_ARG, UNSUPPORTED, NO_DEVICE, CUDA. */
+int space_create(space_ctx** out, const space_config* cfg);
+void space_destroy(space_ctx* ctx);
+
+/* Device bytes space_create reserves for cfg (0 on invalid cfg). */
+size_t space_workspace_bytes(const space_config* cfg);
+
+/* Host only.  Eq. 4 row kinds, Eq. 5 visibility (mask_variant picks the
+ * same-group reading of Sec. 3.2 / App. A.3 or Eq. 5 as printed), Sec. 3.2
+ * position ids.  Errors: INVALID_ARG for k outside 1..SPACE_MAX_K. */
+int space_layout(int k, int mask_variant, space_layout_t* out);
+
+/* Eq. 5 attention of the (k+1)^2 block rows over cache + block. */
+int space_attn_step(space_ctx* ctx, const space_attn_args* args, void* stream);
+
+/* Algorithm 1 verification loop, extra token and next candidates. */
+int space_verify(space_ctx* ctx, const space_verify_args* args, void* stream);
+
+/* Move accepted rows L+g(k+1) -> L+g, g = 1..i*; lengths grow by i*+1. */
+int space_kv_commit(space_ctx* ctx, const space_commit_args* args, void* stream);
+
+/* The three stages from host buffers; synchronises `stream` before returning.
+ * Needs cfg.host_staging.  Only sequence prefixes in use are copied. */
+int space_step_host(space_ctx* ctx, const space_host_step_args* args, void* stream);
+
+/* Number of kernels this context has launched so far. */
+int64_t space_launch_count(const space_ctx* ctx);
+
+/* Per-kernel timing with CUDA events recorded on the launching stream around
+ * every kernel (attention, merge, verify target rows, verify emit, commit).
+ * space_profile_enable(ctx, 1) starts a fresh recording (at most
+ * SPACE_PROFILE_MAX_STEPS steps are kept; later ones are not recorded);
+ * space_profile_enable(ctx, 0) stops it.  Do not enable during stream capture.
+ * space_profile_read waits for the recorded events, writes the summed
+ * milliseconds per kernel into ms[5] and the number of recorded launches per
+ * kernel into n[5], and clears the recording. */
+#define SPACE_PROFILE_MAX_STEPS 4096
+enum { SPACE_K_ATTN = 0, SPACE_K_MERGE = 1, SPACE_K_VERIFY_TARGET = 2, SPACE_K_VERIFY_EMIT = 3,
+       SPACE_K_COMMIT = 4, SPACE_K_COUNT = 5 };
+int space_profile_enable(space_ctx* ctx, int on);
+int space_profile_read(space_ctx* ctx, float* ms, int64_t* n);
+
+/* Test hook: n Philox4x32-10 blocks (Salmon et al., SC'11) for counters
+ * (c0[i], c1[i], c2[i], c3[i]) and key `seed`; out receives 4 words each.
+ * All pointers device memory. */
+int space_debug_philox(space_ctx* ctx, uint64_t seed, int64_t n, const uint32_t* c0,
+                       const uint32_t* c1, const uint32_t* c2, const uint32_t* c3,
+                       uint32_t* out, void* stream);
+
+const char* space_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPACE_H */

@@ -1,0 +1,239 @@
+"""ctypes binding of libspace.so: the same names as include/space.h, argument
+marshalling only.  Tensors are torch CUDA tensors (device memory and streams
+are torch's); every step of the path runs inside the library's kernels.
+
+Importing this module fails loudly when the compiled library is missing.
+"""
+import ctypes as C
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libspace.so")
+
+SPACE_MAX_K = 7
+SPACE_MAX_ROWS = 64
+OK = 0
+E_INVALID_ARG, E_UNSUPPORTED, E_ALIGNMENT, E_WORKSPACE, E_CUDA, E_NO_DEVICE = -1, -2, -3, -4, -5, -6
+MASK_SAME_GROUP, MASK_EQ5_LITERAL = 0, 1
+MODE_GREEDY, MODE_SAMPLE = 0, 1
+RESAMPLE_RESIDUAL_POINTMASS, RESAMPLE_PAPER_LITERAL = 0, 1
+DTYPE_BF16, DTYPE_F32 = 0, 1
+ATTN_TENSOR, ATTN_SIMT = 0, 1
+ST_CAPACITY, ST_BAD_CANDIDATE, ST_TIMEOUT = 1, 2, 4
+
+EXPORTS = ["space_create", "space_destroy", "space_workspace_bytes", "space_layout",
+           "space_attn_step", "space_verify", "space_kv_commit", "space_step_host",
+           "space_launch_count", "space_profile_enable", "space_profile_read",
+           "space_debug_philox", "space_strerror"]
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2402_11809_b200.build` "
+        "(there is no CPU fallback)")
+lib = C.CDLL(LIB_PATH)
+
+
+class Config(C.Structure):
+    _fields_ = [("device", C.c_int32), ("max_batch", C.c_int32), ("n_q_heads", C.c_int32),
+                ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("k_max", C.c_int32),
+                ("vocab", C.c_int32), ("host_staging", C.c_int32), ("s_cap", C.c_int64)]
+
+
+class Layout(C.Structure):
+    _fields_ = [("k", C.c_int32), ("n_q", C.c_int32),
+                ("kind", C.c_uint8 * SPACE_MAX_ROWS), ("group", C.c_uint8 * SPACE_MAX_ROWS),
+                ("offset", C.c_uint8 * SPACE_MAX_ROWS), ("relpos", C.c_int32 * SPACE_MAX_ROWS),
+                ("mask", C.c_uint64 * SPACE_MAX_ROWS), ("target_rows", C.c_int32 * (SPACE_MAX_K + 1))]
+
+
+class AttnArgs(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("k", C.c_int32), ("mask_variant", C.c_int32),
+                ("out_dtype", C.c_int32), ("impl", C.c_int32), ("scale", C.c_float),
+                ("q", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+                ("kv_stride_b", C.c_int64), ("kv_stride_h", C.c_int64), ("kv_stride_s", C.c_int64),
+                ("kv_len", C.c_void_p), ("out", C.c_void_p), ("lse", C.c_void_p),
+                ("status", C.c_void_p)]
+
+
+class VerifyArgs(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("k", C.c_int32), ("vocab", C.c_int32),
+                ("logits_dtype", C.c_int32), ("mode", C.c_int32), ("resample", C.c_int32),
+                ("eos_id", C.c_int32), ("temperature", C.c_float), ("seed", C.c_uint64),
+                ("logits", C.c_void_p), ("logits_row_stride", C.c_int64),
+                ("cand", C.c_void_p), ("cand_prob", C.c_void_p), ("seq_id", C.c_void_p),
+                ("kv_len", C.c_void_p), ("n_accept", C.c_void_p), ("out_tokens", C.c_void_p),
+                ("n_out", C.c_void_p), ("next_cand", C.c_void_p), ("next_cand_prob", C.c_void_p),
+                ("finished", C.c_void_p), ("status", C.c_void_p)]
+
+
+class CommitArgs(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("k", C.c_int32), ("k_cache", C.c_void_p),
+                ("v_cache", C.c_void_p), ("kv_stride_b", C.c_int64), ("kv_stride_h", C.c_int64),
+                ("kv_stride_s", C.c_int64), ("n_accept", C.c_void_p), ("kv_len", C.c_void_p),
+                ("kv_len_out", C.c_void_p), ("commit_src", C.c_void_p), ("commit_dst", C.c_void_p),
+                ("status", C.c_void_p)]
+
+
+class HostStepArgs(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("k", C.c_int32), ("vocab", C.c_int32),
+                ("logits_dtype", C.c_int32), ("mode", C.c_int32), ("resample", C.c_int32),
+                ("eos_id", C.c_int32), ("mask_variant", C.c_int32), ("scale", C.c_float),
+                ("temperature", C.c_float), ("seed", C.c_uint64),
+                ("q", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+                ("logits", C.c_void_p), ("cand", C.c_void_p), ("cand_prob", C.c_void_p),
+                ("kv_len", C.c_void_p), ("out", C.c_void_p), ("n_accept", C.c_void_p),
+                ("out_tokens", C.c_void_p), ("n_out", C.c_void_p), ("next_cand", C.c_void_p),
+                ("next_cand_prob", C.c_void_p), ("finished", C.c_void_p), ("status", C.c_void_p),
+                ("h2d_bytes", C.c_void_p), ("d2h_bytes", C.c_void_p)]
+
+
+lib.space_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(Config)]
+lib.space_create.restype = C.c_int
+lib.space_destroy.argtypes = [C.c_void_p]
+lib.space_destroy.restype = None
+lib.space_workspace_bytes.argtypes = [C.POINTER(Config)]
+lib.space_workspace_bytes.restype = C.c_size_t
+lib.space_layout.argtypes = [C.c_int, C.c_int, C.POINTER(Layout)]
+lib.space_layout.restype = C.c_int
+for _name, _arg in (("space_attn_step", AttnArgs), ("space_verify", VerifyArgs),
+                    ("space_kv_commit", CommitArgs), ("space_step_host", HostStepArgs)):
+    getattr(lib, _name).argtypes = [C.c_void_p, C.POINTER(_arg), C.c_void_p]
+    getattr(lib, _name).restype = C.c_int
+lib.space_launch_count.argtypes = [C.c_void_p]
+lib.space_launch_count.restype = C.c_int64
+lib.space_profile_enable.argtypes = [C.c_void_p, C.c_int]
+lib.space_profile_enable.restype = C.c_int
+lib.space_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
+lib.space_profile_read.restype = C.c_int
+lib.space_debug_philox.argtypes = [C.c_void_p, C.c_uint64, C.c_int64] + [C.c_void_p] * 6
+lib.space_debug_philox.restype = C.c_int
+lib.space_strerror.argtypes = [C.c_int]
+lib.space_strerror.restype = C.c_char_p
+
+
+class SpaceError(RuntimeError):
+    def __init__(self, code):
+        self.code = code
+        super().__init__(f"libspace error {code}: {lib.space_strerror(code).decode()}")
+
+
+def _check(code):
+    if code != OK:
+        raise SpaceError(code)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def space_layout(k, mask_variant=MASK_SAME_GROUP):
+    lay = Layout()
+    _check(lib.space_layout(k, mask_variant, C.byref(lay)))
+    return lay
+
+
+def space_strerror(code):
+    return lib.space_strerror(code).decode()
+
+
+def space_workspace_bytes(**cfg):
+    return lib.space_workspace_bytes(C.byref(Config(**cfg)))
+
+
+class Context:
+    """space_create / space_destroy plus the per-step entry points."""
+
+    def __init__(self, device=0, max_batch=1, n_q_heads=32, n_kv_heads=32, head_dim=128, k_max=5,
+                 vocab=32000, host_staging=0, s_cap=4096):
+        self.cfg = Config(device=device, max_batch=max_batch, n_q_heads=n_q_heads,
+                          n_kv_heads=n_kv_heads, head_dim=head_dim, k_max=k_max, vocab=vocab,
+                          host_staging=host_staging, s_cap=s_cap)
+        self._h = C.c_void_p()
+        _check(lib.space_create(C.byref(self._h), C.byref(self.cfg)))
+
+    def close(self):
+        if self._h:
+            lib.space_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def launch_count(self):
+        return lib.space_launch_count(self._h)
+
+    KERNELS = ("attn", "merge", "verify_target", "verify_emit", "commit")
+
+    def space_profile_enable(self, on):
+        _check(lib.space_profile_enable(self._h, int(on)))
+
+    def space_profile_read(self):
+        """{kernel: (summed ms, launches)} since profiling was enabled; clears the recording."""
+        ms = (C.c_float * 5)()
+        n = (C.c_int64 * 5)()
+        _check(lib.space_profile_read(self._h, ms, n))
+        return {name: (ms[i], n[i]) for i, name in enumerate(self.KERNELS)}
+
+    # -- space_attn_step --------------------------------------------------
+    def attn_args(self, q, k_cache, v_cache, kv_len, out, k, scale, lse=None, status=None,
+                  mask_variant=MASK_SAME_GROUP, impl=ATTN_TENSOR):
+        import torch
+        assert q.is_contiguous() and out.is_contiguous()
+        assert k_cache.stride() == v_cache.stride() and k_cache.stride(3) == 1
+        return AttnArgs(batch=q.shape[0], k=k, mask_variant=mask_variant,
+                        out_dtype=DTYPE_F32 if out.dtype == torch.float32 else DTYPE_BF16,
+                        impl=impl, scale=scale, q=_ptr(q), k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
+                        kv_stride_b=k_cache.stride(0), kv_stride_h=k_cache.stride(1),
+                        kv_stride_s=k_cache.stride(2), kv_len=_ptr(kv_len), out=_ptr(out),
+                        lse=_ptr(lse), status=_ptr(status))
+
+    def space_attn_step(self, args):
+        _check(lib.space_attn_step(self._h, C.byref(args), _stream()))
+
+    # -- space_verify -----------------------------------------------------
+    def verify_args(self, logits, cand, cand_prob, kv_len, n_accept, out_tokens, n_out, next_cand,
+                    next_cand_prob, finished, k, mode=MODE_GREEDY, temperature=1.0, seed=0,
+                    resample=RESAMPLE_RESIDUAL_POINTMASS, eos_id=-1, seq_id=None, status=None):
+        import torch
+        assert logits.stride(2) == 1 and logits.stride(0) == logits.shape[1] * logits.stride(1)
+        return VerifyArgs(batch=logits.shape[0], k=k, vocab=logits.shape[2],
+                          logits_dtype=DTYPE_F32 if logits.dtype == torch.float32 else DTYPE_BF16,
+                          mode=mode, resample=resample, eos_id=eos_id, temperature=temperature,
+                          seed=seed, logits=_ptr(logits), logits_row_stride=logits.stride(1),
+                          cand=_ptr(cand), cand_prob=_ptr(cand_prob), seq_id=_ptr(seq_id),
+                          kv_len=_ptr(kv_len), n_accept=_ptr(n_accept), out_tokens=_ptr(out_tokens),
+                          n_out=_ptr(n_out), next_cand=_ptr(next_cand),
+                          next_cand_prob=_ptr(next_cand_prob), finished=_ptr(finished),
+                          status=_ptr(status))
+
+    def space_verify(self, args):
+        _check(lib.space_verify(self._h, C.byref(args), _stream()))
+
+    # -- space_kv_commit --------------------------------------------------
+    def commit_args(self, k_cache, v_cache, n_accept, kv_len, k, kv_len_out=None, commit_src=None,
+                    commit_dst=None, status=None):
+        return CommitArgs(batch=k_cache.shape[0], k=k, k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
+                          kv_stride_b=k_cache.stride(0), kv_stride_h=k_cache.stride(1),
+                          kv_stride_s=k_cache.stride(2), n_accept=_ptr(n_accept), kv_len=_ptr(kv_len),
+                          kv_len_out=_ptr(kv_len_out), commit_src=_ptr(commit_src),
+                          commit_dst=_ptr(commit_dst), status=_ptr(status))
+
+    def space_kv_commit(self, args):
+        _check(lib.space_kv_commit(self._h, C.byref(args), _stream()))
+
+    # -- space_step_host --------------------------------------------------
+    def space_step_host(self, args):
+        _check(lib.space_step_host(self._h, C.byref(args), _stream()))
+
+    def space_debug_philox(self, seed, c0, c1, c2, c3, out):
+        _check(lib.space_debug_philox(self._h, seed, c0.numel(), _ptr(c0), _ptr(c1), _ptr(c2),
+                                      _ptr(c3), _ptr(out), _stream()))

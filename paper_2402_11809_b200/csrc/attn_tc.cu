@@ -1,0 +1,725 @@
+// Tensor-core attention of the block rows over cache + block (Eq. 5) for sm_100a.
+//
+// Persistent split-KV flash-decode kernel.  The (sequence, kv head) key ranges
+// are cut into 128-key tiles, the tiles of all sequences form one flat list
+// and every thread-block group takes an equal contiguous share of it, so ragged
+// batches balance without host knowledge of the lengths.  A share that does not
+// cover a whole (sequence, head) leaves an unnormalised partial (running max,
+// sum, accumulator) in scratch memory; attn_merge_kernel combines partials.
+//
+// Inside a block (7 warps):
+//   warp 0  streams K and V tiles with TMA into a ring of shared-memory stages
+//   warp 6  loads the query rows of the current share with TMA
+//   warp 1  issues tcgen05.mma: S = Q K^T into one of two TMEM buffers, then
+//           O += P V with P read back from TMEM
+//   warps 2-5  one thread per query row: read S from TMEM, apply the Eq. 5 mask
+//           on tiles that touch the block or a share boundary, running max with
+//           lazy rescaling of O, P = exp2(...) as bf16 into TMEM
+// The 128 MMA rows are (block row i, head-in-group g) pairs of one kv head, so a
+// GQA group shares each K/V tile.  Every wait is bounded; an expired wait sets
+// SPACE_ST_TIMEOUT and the block drains and exits.
+#include "common.cuh"
+#include <cuda.h>
+#include <math_constants.h>
+
+namespace {
+
+constexpr int TILE_N = 128;            // keys per tile
+constexpr int ROWS = 128;              // MMA M
+constexpr int THREADS = 224;
+constexpr uint64_t WAIT_NS = 1000000000ull;   // one second per wait
+constexpr float RESCALE_THRESHOLD = 8.f;
+
+struct AttnParams {
+  CUtensorMap tm_q, tm_k, tm_v;
+  int B, n_q, H_q, H_kv, G;
+  int n_mblocks, rows_per_mb;          // query-row blocks per kv head; block rows i per block
+  int n_groups;                        // thread-block groups (grid = n_groups * n_mblocks)
+  int out_dtype;
+  int64_t s_cap;
+  float scale_log2;                    // scale * log2(e)
+  const int32_t* kv_len;
+  void* out; float* lse; int32_t* status;
+  float* part;                         // [slots][ROWS*(DH+2)]
+  int* err;                            // one word: first timeout site
+  uint64_t mask[SPACE_MAX_ROWS];
+};
+
+struct Seg { int b, h, t0, t1, T, L; };
+
+// ---------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait (WAIT_NS of wall time).  Returns false when the limit expired or
+// another thread of the block gave up; the first expiry records its site.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* err, int site) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 255u) == 255u) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > WAIT_NS) break;
+    }
+  }
+  *abort_flag = 1;
+  atomicCAS(err, 0, site);
+  return false;
+}
+// Bounded wait without the abort protocol (used while draining before exit).
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try(bar, parity)) return;
+    if ((it & 255u) == 255u) {
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > WAIT_NS) return;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
+                                            int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"((uint64_t)tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after()  { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
+// lbo / sbo in bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> f32, M = 128.
+__host__ __device__ constexpr uint32_t instr_desc(int n, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(ROWS >> 4) << 24);
+}
+
+// ------------------------------------------------------------ work partition
+// Flat tile index space: sequence-major, then kv head, then tile.
+struct Partition {
+  const int* tiles;      // [B]   tiles per (sequence, head)
+  const int* prefix;     // [B+1] flat offset of sequence b
+  int B, H_kv;
+  long long cur, end;
+  int b;
+  __device__ void init(const int* t, const int* pf, int B_, int H, int group, int n_groups) {
+    tiles = t; prefix = pf; B = B_; H_kv = H; b = 0;
+    const long long W = pf[B_];
+    cur = (W * group) / n_groups;
+    end = (W * (group + 1)) / n_groups;
+  }
+  __device__ bool next(Seg& s, const int32_t* kv_len) {
+    if (cur >= end) return false;
+    while (prefix[b + 1] <= cur) ++b;
+    const int T = tiles[b];
+    const int rem = (int)(cur - prefix[b]);
+    s.b = b; s.h = rem / T; s.t0 = rem % T; s.T = T;
+    long long n = T - s.t0;
+    if (n > end - cur) n = end - cur;
+    s.t1 = s.t0 + (int)n;
+    s.L = kv_len[b];
+    cur += n;
+    return true;
+  }
+};
+
+template <int DH>
+struct Smem {
+  static constexpr int HALVES = DH / 64;
+  static constexpr int TILE_BYTES = TILE_N * DH * 2;         // one K or V tile
+  static constexpr int Q_BYTES = ROWS * DH * 2;
+  static constexpr int STAGES = (DH == 128) ? 3 : 4;
+  static constexpr int Q_OFF = 0;
+  static constexpr int KV_OFF = Q_BYTES;
+  static constexpr int BAR_OFF = KV_OFF + STAGES * 2 * TILE_BYTES;
+  // barriers: q_full, q_empty, k_full[S], v_full[S], kv_empty[S], s_full[2], p_ready[2], pv_done[2], drain
+  static constexpr int N_BARS = 2 + 3 * STAGES + 6 + 1;
+  static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;      // tmem base, abort flag
+  static constexpr int TABLE_OFF = MISC_OFF + 16;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_constant__ AttnParams p,
+                                                             int max_batch) {
+  using S = Smem<DH>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* sm = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t sm_base = smem_u32(sm);
+  const uint32_t bar0 = sm_base + S::BAR_OFF;
+  auto BAR = [&](int i) { return bar0 + 8u * i; };
+  const int B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_VFULL = 2 + S::STAGES, B_KVEMPTY = 2 + 2 * S::STAGES,
+            B_SFULL = 2 + 3 * S::STAGES, B_PREADY = B_SFULL + 2, B_PVDONE = B_SFULL + 4, B_DRAIN = B_SFULL + 6;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + S::MISC_OFF);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 4);
+  int* tiles = reinterpret_cast<int*>(sm + S::TABLE_OFF);
+  int* prefix = tiles + max_batch;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int group = blockIdx.x / p.n_mblocks, mb = blockIdx.x % p.n_mblocks;
+  const int i0 = mb * p.rows_per_mb;                       // first block row of this query-row block
+
+  // ---- set-up ------------------------------------------------------------
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    long long acc = 0;
+    for (int b = 0; b < p.B; ++b) {
+      const int L = p.kv_len[b];
+      const bool ok = L >= 0 && (int64_t)L + p.n_q <= p.s_cap;
+      const int T = ok ? (L + p.n_q + TILE_N - 1) / TILE_N : 0;
+      if (!ok && blockIdx.x == 0 && p.status) atomicOr(p.status + b, SPACE_ST_CAPACITY);
+      tiles[b] = T;
+      prefix[b] = (int)acc;
+      acc += (long long)T * p.H_kv;
+    }
+    prefix[p.B] = (int)acc;
+    mbar_init(BAR(B_QFULL), 1);
+    mbar_init(BAR(B_QEMPTY), 1);
+    for (int s = 0; s < S::STAGES; ++s) {
+      mbar_init(BAR(B_KFULL + s), 1);
+      mbar_init(BAR(B_VFULL + s), 1);
+      mbar_init(BAR(B_KVEMPTY + s), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(BAR(B_SFULL + i), 1);
+      mbar_init(BAR(B_PREADY + i), 128);
+      mbar_init(BAR(B_PVDONE + i), 1);
+    }
+    mbar_init(BAR(B_DRAIN), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t TM_S0 = tmem, TM_O = tmem + 2 * TILE_N;    // S buffers at columns 0 and 128, O at 256
+
+  Partition part;
+  part.init(tiles, prefix, p.B, p.H_kv, group, p.n_groups);
+  Seg sg;
+
+  if (warp == 0) {
+    // ================= K/V producer =======================================
+    if (lane == 0) {
+      uint32_t gt = 0;
+      bool ok = true;
+      while (ok && part.next(sg, p.kv_len)) {
+        const int n_keys = sg.L + p.n_q;
+        for (int t = sg.t0; t < sg.t1 && ok; ++t, ++gt) {
+          const int s = gt % S::STAGES;
+          if (gt >= (uint32_t)S::STAGES)
+            ok = mbar_wait(BAR(B_KVEMPTY + s), ((gt / S::STAGES) - 1) & 1, abort_flag, p.err, 1);
+          if (!ok) break;
+          // the last tile of a sequence is shifted back so that it ends at the
+          // last key: rows past the end are never read (they may hold anything)
+          const int kt = ((t + 1) * TILE_N <= n_keys) ? t * TILE_N : n_keys - TILE_N;
+          const uint32_t kdst = sm_base + S::KV_OFF + s * 2 * S::TILE_BYTES;
+          const uint32_t vdst = kdst + S::TILE_BYTES;
+          mbar_expect_tx(BAR(B_KFULL + s), S::TILE_BYTES);
+          for (int hf = 0; hf < S::HALVES; ++hf)
+            tma_load_4d(kdst + hf * (TILE_N * 128), &p.tm_k, BAR(B_KFULL + s), hf * 64, kt, sg.h, sg.b);
+          mbar_expect_tx(BAR(B_VFULL + s), S::TILE_BYTES);
+          for (int hf = 0; hf < S::HALVES; ++hf)
+            tma_load_4d(vdst + hf * (TILE_N * 128), &p.tm_v, BAR(B_VFULL + s), hf * 64, kt, sg.h, sg.b);
+        }
+      }
+      // drain: every issued copy must have landed before the block may exit
+      const uint32_t first = gt > (uint32_t)S::STAGES ? gt - S::STAGES : 0;
+      for (uint32_t g = first; g < gt; ++g) {
+        const int s = g % S::STAGES;
+        const uint32_t par = (g / S::STAGES) & 1;
+        mbar_drain(BAR(B_KFULL + s), par);
+        mbar_drain(BAR(B_VFULL + s), par);
+      }
+    }
+  } else if (warp == 6) {
+    // ================= Q producer =========================================
+    if (lane == 0) {
+      uint32_t seg = 0;
+      bool ok = true;
+      while (ok && part.next(sg, p.kv_len)) {
+        if (seg > 0) ok = mbar_wait(BAR(B_QEMPTY), (seg - 1) & 1, abort_flag, p.err, 2);
+        if (!ok) break;
+        mbar_expect_tx(BAR(B_QFULL), S::Q_BYTES);
+        for (int hf = 0; hf < S::HALVES; ++hf)
+          tma_load_4d(sm_base + S::Q_OFF + hf * (ROWS * 128), &p.tm_q, BAR(B_QFULL), hf * 64,
+                      sg.h * p.G, i0, sg.b);
+        ++seg;
+      }
+      if (seg > 0) mbar_drain(BAR(B_QFULL), (seg - 1) & 1);
+    }
+  } else if (warp == 1) {
+    // ================= MMA issuer =========================================
+    if (lane == 0) {
+      constexpr uint32_t IDESC_QK = instr_desc(TILE_N, 0);
+      constexpr uint32_t IDESC_PV = instr_desc(DH, 1);
+      uint32_t gt = 0, seg = 0;
+      bool ok = true;
+      // O += P V for flat tile g (first_in_seg: overwrite O)
+      auto issue_pv = [&](uint32_t g, bool first_in_seg) -> bool {
+        const int s = g % S::STAGES, buf = g & 1;
+        if (!mbar_wait(BAR(B_VFULL + s), (g / S::STAGES) & 1, abort_flag, p.err, 3)) return false;
+        if (!mbar_wait(BAR(B_PREADY + buf), (g >> 1) & 1, abort_flag, p.err, 4)) return false;
+        tc_fence_after();
+        const uint32_t vsm = sm_base + S::KV_OFF + s * 2 * S::TILE_BYTES + S::TILE_BYTES;
+        const uint32_t ptm = TM_S0 + buf * TILE_N;
+#pragma unroll
+        for (int kk = 0; kk < TILE_N / 16; ++kk) {
+          // V tile is MN-major: 64-wide d blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
+          const uint64_t bd = smem_desc(vsm + kk * 2048, TILE_N * 128, 1024);
+          mma_ts(TM_O, ptm + kk * 8, bd, IDESC_PV, (first_in_seg && kk == 0) ? 0u : 1u);
+        }
+        tc_commit(BAR(B_KVEMPTY + s));
+        tc_commit(BAR(B_PVDONE + buf));
+        return true;
+      };
+      while (ok && part.next(sg, p.kv_len)) {
+        ok = mbar_wait(BAR(B_QFULL), seg & 1, abort_flag, p.err, 5);
+        const int n = sg.t1 - sg.t0;
+        for (int j = 0; j < n && ok; ++j, ++gt) {
+          const int s = gt % S::STAGES, buf = gt & 1;
+          ok = mbar_wait(BAR(B_KFULL + s), (gt / S::STAGES) & 1, abort_flag, p.err, 6);
+          if (ok && gt >= 2) ok = mbar_wait(BAR(B_PVDONE + buf), ((gt >> 1) - 1) & 1, abort_flag, p.err, 7);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t qsm = sm_base + S::Q_OFF;
+          const uint32_t ksm = sm_base + S::KV_OFF + s * 2 * S::TILE_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < DH / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * (ROWS * 128) + (kk & 3) * 32;   // 64-wide half, then 32 B per 16 elements
+            mma_ss(TM_S0 + buf * TILE_N, smem_desc(qsm + off, 16, 1024), smem_desc(ksm + off, 16, 1024),
+                   IDESC_QK, kk > 0 ? 1u : 0u);
+          }
+          tc_commit(BAR(B_SFULL + buf));
+          if (j == n - 1) tc_commit(BAR(B_QEMPTY));
+          if (j > 0) ok = issue_pv(gt - 1, j == 1);
+        }
+        if (ok) ok = issue_pv(gt - 1, n == 1);
+        ++seg;
+      }
+      // all tensor work done before TMEM is released
+      tc_commit(BAR(B_DRAIN));
+      mbar_drain(BAR(B_DRAIN), 0);
+    }
+  } else {
+    // ================= softmax / epilogue: one thread per query row ========
+    const int quarter = warp & 3;                          // TMEM lane quarter this warp may touch
+    const int m = quarter * 32 + lane;                     // MMA row
+    const int il = m / p.G, g = m % p.G;
+    const int i = i0 + il;                                 // block row
+    const bool row_valid = il < p.rows_per_mb && i < p.n_q;
+    const uint64_t mrow = row_valid ? p.mask[i] : 0ull;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const float c = p.scale_log2;
+    uint32_t gt = 0;
+    bool ok = true;
+    while (ok && part.next(sg, p.kv_len)) {
+      const int n_keys = sg.L + p.n_q;
+      float m_ref = -CUDART_INF_F, l_sum = 0.f;
+      for (int t = sg.t0; t < sg.t1 && ok; ++t, ++gt) {
+        const int buf = gt & 1;
+        ok = mbar_wait(BAR(B_SFULL + buf), (gt >> 1) & 1, abort_flag, p.err, 8);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t ts = TM_S0 + buf * TILE_N + lane_addr;
+        uint32_t sreg[TILE_N];
+#pragma unroll
+        for (int cc = 0; cc < TILE_N / 32; ++cc) tmem_ld32(ts + cc * 32, sreg + cc * 32);
+        tmem_wait_ld();
+        const int lo = t * TILE_N;
+        const int kt = ((t + 1) * TILE_N <= n_keys) ? lo : n_keys - TILE_N;
+        const bool masked = (kt + TILE_N > sg.L) || (kt < lo);
+        float tmax = -CUDART_INF_F;
+        if (masked) {
+#pragma unroll
+          for (int cidx = 0; cidx < TILE_N; ++cidx) {
+            const int key = kt + cidx;
+            bool vis = key >= lo;
+            if (key >= sg.L) vis = vis && ((mrow >> ((key - sg.L) & 63)) & 1ull);
+            const float v = vis ? __uint_as_float(sreg[cidx]) : -CUDART_INF_F;
+            sreg[cidx] = __float_as_uint(v);
+            tmax = fmaxf(tmax, v);
+          }
+        } else {
+#pragma unroll
+          for (int cidx = 0; cidx < TILE_N; ++cidx) tmax = fmaxf(tmax, __uint_as_float(sreg[cidx]));
+        }
+        tmax *= c;                                         // c > 0
+        if (!(tmax > -CUDART_INF_F)) tmax = -CUDART_INF_F; // also catches NaN
+        const bool first = (t == sg.t0);
+        bool need = !first && (tmax > m_ref + RESCALE_THRESHOLD);
+        if (first) m_ref = tmax;
+        if (__any_sync(0xFFFFFFFFu, need)) {
+          // lazy rescale of this row's accumulator; PV of the previous tile must be done
+          ok = mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 9);
+          if (!ok) break;
+          tc_fence_after();
+          const float m_new = fmaxf(m_ref, tmax);
+          const float f = (m_ref > -CUDART_INF_F) ? exp2f(m_ref - m_new) : 0.f;
+          l_sum *= f;
+          m_ref = m_new;
+#pragma unroll 1
+          for (int cc = 0; cc < DH / 32; ++cc) {
+            uint32_t o[32];
+            tmem_ld32(TM_O + lane_addr + cc * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * f);
+            tmem_st32(TM_O + lane_addr + cc * 32, o);
+          }
+          tmem_wait_st();
+        }
+        const float m_use = (m_ref > -CUDART_INF_F) ? m_ref : 0.f;
+        uint32_t preg[TILE_N / 2];
+#pragma unroll
+        for (int x = 0; x < TILE_N / 2; ++x) {
+          const float p0 = exp2f(fmaf(__uint_as_float(sreg[2 * x]), c, -m_use));
+          const float p1 = exp2f(fmaf(__uint_as_float(sreg[2 * x + 1]), c, -m_use));
+          l_sum += p0 + p1;
+          const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);   // .x (low half) = even key
+          preg[x] = *reinterpret_cast<const uint32_t*>(&pk);
+        }
+#pragma unroll
+        for (int cc = 0; cc < TILE_N / 64; ++cc) tmem_st32(ts + cc * 32, preg + cc * 32);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(BAR(B_PREADY + buf));
+      }
+      if (!ok) break;
+      // ---- end of share: final output or partial ---------------------------
+      ok = mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 10);
+      if (!ok) break;
+      tc_fence_after();
+      const bool whole = (sg.t0 == 0 && sg.t1 == sg.T);
+      const int hq = sg.h * p.G + g;
+      float* pslot = p.part + ((size_t)((sg.b * p.H_kv + sg.h) + group) * p.n_mblocks + mb) * (ROWS * (DH + 2));
+      const float inv = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
+#pragma unroll 1
+      for (int cc = 0; cc < DH / 32; ++cc) {
+        uint32_t o[32];
+        tmem_ld32(TM_O + lane_addr + cc * 32, o);
+        tmem_wait_ld();
+        if (!row_valid) continue;
+        if (whole) {
+          const size_t off = (((size_t)sg.b * p.n_q + i) * p.H_q + hq) * DH + cc * 32;
+          if (p.out_dtype == SPACE_DTYPE_F32) {
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off);
+#pragma unroll
+            for (int x = 0; x < 8; ++x)
+              dst[x] = make_float4(__uint_as_float(o[4 * x]) * inv, __uint_as_float(o[4 * x + 1]) * inv,
+                                   __uint_as_float(o[4 * x + 2]) * inv, __uint_as_float(o[4 * x + 3]) * inv);
+          } else {
+            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off);
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+              uint32_t w[4];
+#pragma unroll
+              for (int y = 0; y < 4; ++y) {
+                const __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(o[8 * x + 2 * y]) * inv,
+                                                                __uint_as_float(o[8 * x + 2 * y + 1]) * inv);
+                w[y] = *reinterpret_cast<const uint32_t*>(&pk);
+              }
+              dst[x] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        } else {
+          float4* dst = reinterpret_cast<float4*>(pslot + (size_t)m * DH + cc * 32);
+#pragma unroll
+          for (int x = 0; x < 8; ++x)
+            dst[x] = make_float4(__uint_as_float(o[4 * x]), __uint_as_float(o[4 * x + 1]),
+                                 __uint_as_float(o[4 * x + 2]), __uint_as_float(o[4 * x + 3]));
+        }
+      }
+      if (row_valid) {
+        if (whole) {
+          if (p.lse)
+            p.lse[((size_t)sg.b * p.H_q + hq) * p.n_q + i] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+        } else {
+          pslot[ROWS * DH + m] = m_ref;
+          pslot[ROWS * DH + ROWS + m] = l_sum;
+        }
+      }
+      tc_fence_before();
+    }
+  }
+
+  // ---- teardown -----------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+  if (threadIdx.x == 0 && *abort_flag && p.status) {
+    for (int b = 0; b < p.B; ++b) atomicOr(p.status + b, SPACE_ST_TIMEOUT);
+  }
+}
+
+// Combine the partials of every (sequence, kv head, query-row block) that was
+// split over several thread-block groups.  grid = (B*H_kv*n_mblocks, row chunks).
+template <int DH>
+__global__ void __launch_bounds__(DH) attn_merge_kernel(const AttnParams p, int rows_per_block) {
+  const int item = blockIdx.x / p.n_mblocks, mb = blockIdx.x % p.n_mblocks;
+  const int b = item / p.H_kv, h = item % p.H_kv;
+  const int L = p.kv_len[b];
+  if (L < 0 || (int64_t)L + p.n_q > p.s_cap) return;
+  // recompute the partition (same arithmetic as the main kernel)
+  long long f0 = 0, W = 0;
+  for (int bb = 0; bb < p.B; ++bb) {
+    const int LL = p.kv_len[bb];
+    const bool ok = LL >= 0 && (int64_t)LL + p.n_q <= p.s_cap;
+    const long long T = ok ? (LL + p.n_q + TILE_N - 1) / TILE_N : 0;
+    if (bb < b) f0 += T * p.H_kv;
+    W += T * p.H_kv;
+  }
+  const int T = (L + p.n_q + TILE_N - 1) / TILE_N;
+  f0 += (long long)h * T;
+  const long long NG = p.n_groups;
+  const int g_first = (int)(((f0 + 1) * NG - 1) / W);
+  const int g_last = (int)(((f0 + T) * NG - 1) / W);
+  if (g_first == g_last) return;                            // written directly by the main kernel
+  const int c = threadIdx.x;
+  const int i0 = mb * p.rows_per_mb;
+  const int m_begin = blockIdx.y * rows_per_block;
+  for (int m = m_begin; m < m_begin + rows_per_block && m < ROWS; ++m) {
+    const int il = m / p.G, g = m % p.G, i = i0 + il;
+    if (il >= p.rows_per_mb || i >= p.n_q) continue;
+    float mx = -CUDART_INF_F;
+    for (int gi = g_first; gi <= g_last; ++gi) {
+      if ((W * gi) / NG == (W * (gi + 1)) / NG) continue;   // this group holds no tiles
+      const float* ps = p.part + ((size_t)(item + gi) * p.n_mblocks + mb) * (ROWS * (DH + 2));
+      mx = fmaxf(mx, __ldcg(ps + ROWS * DH + m));
+    }
+    float acc = 0.f, den = 0.f;
+    for (int gi = g_first; gi <= g_last; ++gi) {
+      if ((W * gi) / NG == (W * (gi + 1)) / NG) continue;
+      const float* ps = p.part + ((size_t)(item + gi) * p.n_mblocks + mb) * (ROWS * (DH + 2));
+      const float ms = __ldcg(ps + ROWS * DH + m);
+      const float w = (ms > -CUDART_INF_F) ? exp2f(ms - mx) : 0.f;
+      den = fmaf(w, __ldcg(ps + ROWS * DH + ROWS + m), den);
+      acc = fmaf(w, __ldcg(ps + (size_t)m * DH + c), acc);
+    }
+    const int hq = h * p.G + g;
+    const size_t off = (((size_t)b * p.n_q + i) * p.H_q + hq) * DH + c;
+    const float r = acc / den;
+    if (p.out_dtype == SPACE_DTYPE_F32) reinterpret_cast<float*>(p.out)[off] = r;
+    else reinterpret_cast<__nv_bfloat16*>(p.out)[off] = __float2bfloat16_rn(r);
+    if (p.lse && c == 0)
+      p.lse[((size_t)b * p.H_q + hq) * p.n_q + i] = (mx + log2f(den)) * 0.6931471805599453f;
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = (EncodeTiledFn)ptr;
+  }
+  return fn;
+}
+
+int make_map(CUtensorMap* tm, const void* base, const cuuint64_t dims[4], const cuuint64_t strides_bytes[3],
+             const cuuint32_t box[4]) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return SPACE_E_CUDA;
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides_bytes,
+                         box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SPACE_OK : SPACE_E_CUDA;
+}
+
+void plan(const space_config* cfg, int sm_count, int k, AttnPlanHost* pl) {
+  const int G = cfg->n_q_heads / cfg->n_kv_heads;
+  const int n_q = (k + 1) * (k + 1);
+  const int max_rows = ROWS / G;                            // block rows one MMA tile can hold
+  pl->n_mblocks = (n_q + max_rows - 1) / max_rows;
+  pl->rows_per_mblock = (n_q + pl->n_mblocks - 1) / pl->n_mblocks;
+  int groups = sm_count / pl->n_mblocks;
+  if (groups < 1) groups = 1;
+  pl->n_ctas = groups * pl->n_mblocks;
+}
+
+template <int DH>
+size_t smem_bytes(int max_batch) {
+  return 1024 + Smem<DH>::TABLE_OFF + (size_t)(2 * max_batch + 2) * sizeof(int);
+}
+
+}  // namespace
+
+size_t attn_tensor_partial_floats(const space_config* cfg, int sm_count, size_t* slots_out) {
+  AttnPlanHost pl;
+  plan(cfg, sm_count, cfg->k_max, &pl);
+  // the largest slot index is (B*H_kv - 1) + (groups - 1), times the query-row blocks
+  size_t worst_mb = 1;
+  for (int k = 1; k <= cfg->k_max; ++k) {
+    AttnPlanHost q; plan(cfg, sm_count, k, &q);
+    if ((size_t)q.n_mblocks > worst_mb) worst_mb = q.n_mblocks;
+  }
+  const size_t slots = ((size_t)cfg->max_batch * cfg->n_kv_heads + sm_count) * worst_mb;
+  if (slots_out) *slots_out = slots;
+  return slots * (size_t)ROWS * (cfg->head_dim + 2);
+}
+
+int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t* mask_rows,
+                       cudaStream_t st) {
+  const space_config& cfg = ctx->cfg;
+  const int DH = cfg.head_dim;
+  AttnPlanHost pl;
+  plan(&cfg, ctx->sm_count, a->k, &pl);
+  AttnParams p;
+  memset(&p, 0, sizeof(p));
+  p.B = a->batch; p.n_q = (a->k + 1) * (a->k + 1);
+  p.H_q = cfg.n_q_heads; p.H_kv = cfg.n_kv_heads; p.G = p.H_q / p.H_kv;
+  p.n_mblocks = pl.n_mblocks; p.rows_per_mb = pl.rows_per_mblock;
+  p.n_groups = pl.n_ctas / pl.n_mblocks;
+  p.out_dtype = a->out_dtype; p.s_cap = cfg.s_cap;
+  p.scale_log2 = a->scale * 1.4426950408889634f;
+  p.kv_len = a->kv_len; p.out = a->out; p.lse = a->lse; p.status = a->status;
+  p.part = ctx->attn_part; p.err = ctx->counters + 3 * cfg.max_batch;
+  for (int i = 0; i < SPACE_MAX_ROWS; ++i) p.mask[i] = mask_rows[i];
+
+  // TMA descriptors, rebuilt only when a base pointer or a stride changes
+  const int64_t key[8] = {a->kv_stride_b, a->kv_stride_h, a->kv_stride_s, a->batch, p.n_q, 0, 0, 0};
+  if (ctx->tm_q_ptr != a->q || ctx->tm_k_ptr != a->k_cache || ctx->tm_v_ptr != a->v_cache ||
+      memcmp(key, ctx->tm_key, sizeof(key)) != 0) {
+    const cuuint64_t kd[4] = {(cuuint64_t)DH, (cuuint64_t)cfg.s_cap, (cuuint64_t)p.H_kv, (cuuint64_t)a->batch};
+    const cuuint64_t ks[3] = {(cuuint64_t)a->kv_stride_s * 2, (cuuint64_t)a->kv_stride_h * 2,
+                              (cuuint64_t)a->kv_stride_b * 2};
+    const cuuint32_t kb[4] = {64, TILE_N, 1, 1};
+    const cuuint64_t qd[4] = {(cuuint64_t)DH, (cuuint64_t)p.H_q, (cuuint64_t)p.n_q, (cuuint64_t)a->batch};
+    const cuuint64_t qs[3] = {(cuuint64_t)DH * 2, (cuuint64_t)p.H_q * DH * 2, (cuuint64_t)p.n_q * p.H_q * DH * 2};
+    const cuuint32_t qb[4] = {64, (cuuint32_t)p.G, (cuuint32_t)(ROWS / p.G), 1};
+    int rc = make_map((CUtensorMap*)ctx->tm_k, a->k_cache, kd, ks, kb);
+    if (rc == SPACE_OK) rc = make_map((CUtensorMap*)ctx->tm_v, a->v_cache, kd, ks, kb);
+    if (rc == SPACE_OK) rc = make_map((CUtensorMap*)ctx->tm_q, a->q, qd, qs, qb);
+    if (rc != SPACE_OK) { ctx->tm_q_ptr = nullptr; return rc; }
+    ctx->tm_q_ptr = a->q; ctx->tm_k_ptr = a->k_cache; ctx->tm_v_ptr = a->v_cache;
+    memcpy(ctx->tm_key, key, sizeof(key));
+  }
+  memcpy(&p.tm_q, ctx->tm_q, sizeof(CUtensorMap));
+  memcpy(&p.tm_k, ctx->tm_k, sizeof(CUtensorMap));
+  memcpy(&p.tm_v, ctx->tm_v, sizeof(CUtensorMap));
+
+  const int rows_per_block = 8;
+  const dim3 mgrid(a->batch * p.H_kv * p.n_mblocks, (ROWS + rows_per_block - 1) / rows_per_block);
+  if (DH == 128) {
+    const size_t sm = smem_bytes<128>(cfg.max_batch);
+    cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    {
+      ProfScope ps(ctx, SPACE_K_ATTN, st);
+      attn_tc_kernel<128><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
+    }
+    {
+      ProfScope ps(ctx, SPACE_K_MERGE, st);
+      attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(p, rows_per_block);
+    }
+  } else {
+    const size_t sm = smem_bytes<64>(cfg.max_batch);
+    cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    {
+      ProfScope ps(ctx, SPACE_K_ATTN, st);
+      attn_tc_kernel<64><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
+    }
+    {
+      ProfScope ps(ctx, SPACE_K_MERGE, st);
+      attn_merge_kernel<64><<<mgrid, 64, 0, st>>>(p, rows_per_block);
+    }
+  }
+  ctx->launches += 2;
+  return cuda_ok(cudaGetLastError());
+}

@@ -1,0 +1,103 @@
+// Internal declarations shared by the translation units of libspace.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "../../include/space.h"
+
+#define SPACE_VERIFY_MAX_CHUNKS 64
+#define SPACE_VERIFY_THREADS 256
+
+// ---- Philox4x32-10 (Salmon et al., SC'11) ---------------------------------
+struct Philox4 { uint32_t x, y, z, w; };
+
+__host__ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2,
+                                                          uint32_t c3, uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    c1 = (uint32_t)p1;
+    c3 = (uint32_t)p0;
+    c0 = n0;
+    c2 = n2;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return Philox4{c0, c1, c2, c3};
+}
+
+// 32-bit word -> uniform in (0,1), exactly representable in binary32.
+__host__ __device__ __forceinline__ float uniform_open(uint32_t w) {
+  return ((float)(w >> 9) + 0.5f) * 1.1920928955078125e-07f;   // 2^-23
+}
+
+enum { PURPOSE_ACCEPT = 0, PURPOSE_TOKEN = 1, PURPOSE_DRAFT = 2 };
+
+// ---- context ---------------------------------------------------------------
+struct VerifyPartial { float m, s, gs; int idx, gidx, pad0, pad1, pad2; };   // 32 bytes
+struct VerifyRow     { float m, s; int idx, pad; };
+
+struct AttnPlanHost {
+  int n_ctas;         // persistent grid size
+  int n_mblocks;      // query-row blocks per (sequence, kv head)
+  int rows_per_mblock;// block rows (i) per query-row block
+};
+
+struct space_ctx {
+  space_config cfg;
+  int sm_count;
+  int64_t launches;
+  // one allocation, carved up
+  char* ws;
+  size_t ws_bytes;
+  float* attn_part;        // split partials
+  size_t attn_part_slots;
+  int* counters;           // [4][max_batch] self-resetting arrival counters
+  VerifyPartial* vpart;    // [max_batch][k_max+2][SPACE_VERIFY_MAX_CHUNKS]
+  VerifyRow* vrow;         // [max_batch][k_max+1]
+  int32_t* scratch_status; // [max_batch] used when the caller passes no status array
+  // staging for space_step_host
+  char* stage;
+  size_t stage_bytes;
+  // per-kernel event timing (space_profile_*)
+  int prof_on;
+  int prof_n[SPACE_K_COUNT];
+  cudaEvent_t* prof_ev[SPACE_K_COUNT];   // [2 * SPACE_PROFILE_MAX_STEPS] start/stop pairs, lazily created
+  // cached TMA descriptors
+  const void* tm_q_ptr; const void* tm_k_ptr; const void* tm_v_ptr;
+  int64_t tm_key[8];
+  alignas(64) unsigned char tm_q[128];
+  alignas(64) unsigned char tm_k[128];
+  alignas(64) unsigned char tm_v[128];
+};
+
+// ---- per-stage launchers (defined next to their kernels) -------------------
+int launch_verify(space_ctx* ctx, const space_verify_args* a, cudaStream_t st);
+int launch_commit(space_ctx* ctx, const space_commit_args* a, cudaStream_t st);
+int launch_attn_simt(space_ctx* ctx, const space_attn_args* a, const uint64_t* mask_rows,
+                     cudaStream_t st);
+int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t* mask_rows,
+                       cudaStream_t st);
+size_t attn_tensor_partial_floats(const space_config* cfg, int sm_count, size_t* slots);
+int launch_philox_debug(uint64_t seed, int64_t n, const uint32_t* c0, const uint32_t* c1,
+                        const uint32_t* c2, const uint32_t* c3, uint32_t* out, cudaStream_t st);
+
+// Event pair around one kernel launch when profiling is on.
+struct ProfScope {
+  space_ctx* ctx; int which; cudaStream_t st; int slot;
+  ProfScope(space_ctx* c, int w, cudaStream_t s) : ctx(c), which(w), st(s), slot(-1) {
+    if (!c->prof_on || !c->prof_ev[w] || c->prof_n[w] >= SPACE_PROFILE_MAX_STEPS) return;
+    slot = c->prof_n[w];
+    cudaEventRecord(c->prof_ev[w][2 * slot], st);
+  }
+  ~ProfScope() {
+    if (slot < 0) return;
+    cudaEventRecord(ctx->prof_ev[which][2 * slot + 1], st);
+    ctx->prof_n[which] = slot + 1;
+  }
+};
+
+static inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? SPACE_OK : SPACE_E_CUDA; }

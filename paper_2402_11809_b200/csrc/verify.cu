@@ -1,0 +1,424 @@
+// Verification and emission kernels (Algorithm 1 after the model call, Sec. 3.2).
+//
+// Two launches per step.
+//   verify_target_kernel  streams the k+1 target rows (real token of every
+//       sub-block) once: per row the maximum, the lowest-index arg-max and the
+//       sum of exp((z - max)/T).  The last block to finish a sequence runs the
+//       acceptance loop of Algorithm 1 and stores i*.
+//   verify_emit_kernel    streams the k mask rows of group i* (the next
+//       candidates) and, in sampling mode, the target row i* once more for the
+//       extra token a (Gumbel arg-max with Philox noise).  The last block of a
+//       sequence assembles the emitted tokens, the <EOS> cut and the new
+//       candidates with their probabilities.
+// Each row is cut into chunks so that small batches still fill the GPU; chunk
+// results meet in a small scratch array and an arrival counter (reset by the
+// last block) decides who finishes the sequence.
+#include "common.cuh"
+#include <math_constants.h>
+
+namespace {
+
+struct VerifyParams {
+  int B, k, V, n_q, n_chunks, chunk;
+  int mode, resample, eos_id;
+  float c_t;                 // log2(e) / T   (target rows, sampled rows)
+  float inv_t;               // 1 / T
+  uint32_t key0, key1;
+  const void* logits;
+  int64_t row_stride;
+  const int32_t* cand;
+  const float* cand_prob;
+  const uint32_t* seq_id;
+  const int32_t* kv_len;
+  int32_t* n_accept;
+  int32_t* out_tokens;
+  int32_t* n_out;
+  int32_t* next_cand;
+  float* next_cand_prob;
+  uint8_t* finished;
+  int32_t* status;
+  VerifyPartial* part;       // [B][k+2][n_chunks]
+  VerifyRow* rows;           // [B][k+1]
+  int* counter_a;            // [B]
+  int* counter_b;            // [B]
+};
+
+struct Stat {                // running statistics of a set of logits
+  float m, s;  int idx;      // max, sum exp2((z-m)*c), arg-max (lowest index)
+  float gs;    int gidx;     // best Gumbel-perturbed score and its index
+};
+
+__device__ __forceinline__ Stat stat_empty() {
+  return Stat{-CUDART_INF_F, 0.f, 0x7FFFFFFF, -CUDART_INF_F, 0x7FFFFFFF};
+}
+
+__device__ __forceinline__ void stat_merge(Stat& a, const Stat& b, float c) {
+  if (b.m > a.m || (b.m == a.m && b.idx < a.idx)) a.idx = b.idx;
+  const float m = fmaxf(a.m, b.m);
+  if (m > -CUDART_INF_F) {
+    const float sa = (a.m > -CUDART_INF_F) ? a.s * exp2f((a.m - m) * c) : 0.f;
+    const float sb = (b.m > -CUDART_INF_F) ? b.s * exp2f((b.m - m) * c) : 0.f;
+    a.s = sa + sb;
+  }
+  a.m = m;
+  if (b.gs > a.gs || (b.gs == a.gs && b.gidx < a.gidx)) { a.gs = b.gs; a.gidx = b.gidx; }
+}
+
+__device__ __forceinline__ float load_logit(const float* p) { return *p; }
+__device__ __forceinline__ float load_logit(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+template <typename T> struct Vec;
+template <> struct Vec<float> {
+  static constexpr int N = 4;
+  static __device__ __forceinline__ void load(const float* p, float* v) {
+    const float4 x = __ldg(reinterpret_cast<const float4*>(p));
+    v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+  }
+};
+template <> struct Vec<__nv_bfloat16> {
+  static constexpr int N = 8;
+  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float* v) {
+    const uint4 x = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i]     = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+};
+
+// Fold n consecutive logits starting at vocabulary index x0 into st.
+template <int N, bool GUMBEL>
+__device__ __forceinline__ void fold(Stat& st, const float* v, int x0, float c, float inv_t, int exclude,
+                                     uint32_t key0, uint32_t key1, uint32_t purpose,
+                                     uint32_t seq, uint32_t pos) {
+  float vmax = v[0];
+#pragma unroll
+  for (int i = 1; i < N; ++i) vmax = fmaxf(vmax, v[i]);
+  if (vmax > st.m) {
+    st.s = (st.m > -CUDART_INF_F) ? st.s * exp2f((st.m - vmax) * c) : 0.f;
+#pragma unroll
+    for (int i = N - 1; i >= 0; --i) if (v[i] == vmax) st.idx = x0 + i;
+    st.m = vmax;
+  }
+  if (st.m > -CUDART_INF_F) {
+#pragma unroll
+    for (int i = 0; i < N; ++i) st.s += exp2f((v[i] - st.m) * c);
+  }
+  if (GUMBEL) {
+    // noise of token x: lane x&3 of the Philox block with counter word x>>2
+#pragma unroll
+    for (int i0 = 0; i0 < N; i0 += 4) {
+      const int xb = x0 + i0;
+      const Philox4 r = philox4x32_10((uint32_t)(xb >> 2), purpose, seq, pos, key0, key1);
+      const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+      for (int j = 0; j < 4 && i0 + j < N; ++j) {
+        const int lane = (xb + j) & 3;
+        const uint32_t word = (N >= 4) ? w[j] : w[lane];
+        const float u = uniform_open(word);
+        const float sc = v[i0 + j] * inv_t - logf(-logf(u));
+        const int x = xb + j;
+        if (x != exclude && v[i0 + j] > -CUDART_INF_F && (sc > st.gs)) { st.gs = sc; st.gidx = x; }
+      }
+    }
+  }
+}
+
+template <typename T, bool VECTOR, bool GUMBEL>
+__device__ Stat scan_chunk(const T* row, int begin, int end, float c, float inv_t, int exclude,
+                           uint32_t key0, uint32_t key1, uint32_t purpose, uint32_t seq,
+                           uint32_t pos) {
+  Stat st = stat_empty();
+  if (VECTOR) {
+    constexpr int N = Vec<T>::N;
+    // begin is a multiple of N; the tail shorter than N is handled one by one
+    const int full_end = begin + ((end - begin) / N) * N;
+    for (int x = begin + threadIdx.x * N; x < full_end; x += blockDim.x * N) {
+      float v[N];
+      Vec<T>::load(row + x, v);
+      fold<N, GUMBEL>(st, v, x, c, inv_t, exclude, key0, key1, purpose, seq, pos);
+    }
+    for (int x = full_end + threadIdx.x; x < end; x += blockDim.x) {
+      float v[1] = {load_logit(row + x)};
+      Stat one = stat_empty();
+      fold<1, GUMBEL>(one, v, x, c, inv_t, exclude, key0, key1, purpose, seq, pos);
+      stat_merge(st, one, c);
+    }
+  } else {
+    for (int x = begin + threadIdx.x; x < end; x += blockDim.x) {
+      float v[1] = {load_logit(row + x)};
+      fold<1, GUMBEL>(st, v, x, c, inv_t, exclude, key0, key1, purpose, seq, pos);
+    }
+  }
+  return st;
+}
+
+__device__ __forceinline__ Stat warp_reduce(Stat st, float c) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    Stat o;
+    o.m = __shfl_xor_sync(0xFFFFFFFFu, st.m, off);
+    o.s = __shfl_xor_sync(0xFFFFFFFFu, st.s, off);
+    o.idx = __shfl_xor_sync(0xFFFFFFFFu, st.idx, off);
+    o.gs = __shfl_xor_sync(0xFFFFFFFFu, st.gs, off);
+    o.gidx = __shfl_xor_sync(0xFFFFFFFFu, st.gidx, off);
+    stat_merge(st, o, c);
+  }
+  return st;
+}
+
+__device__ Stat block_reduce(Stat st, float c) {
+  __shared__ Stat sh[SPACE_VERIFY_THREADS / 32];
+  st = warp_reduce(st, c);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  if (l == 0) sh[w] = st;
+  __syncthreads();
+  if (w == 0) {
+    st = (l < (int)(blockDim.x >> 5)) ? sh[l] : stat_empty();
+    st = warp_reduce(st, c);
+  }
+  return st;           // valid in warp 0
+}
+
+__device__ __forceinline__ void store_partial(VerifyPartial* p, const Stat& st) {
+  VerifyPartial v;
+  v.m = st.m; v.s = st.s; v.gs = st.gs; v.idx = st.idx; v.gidx = st.gidx;
+  v.pad0 = v.pad1 = v.pad2 = 0;
+  *reinterpret_cast<volatile float*>(&p->m) = v.m;
+  *reinterpret_cast<volatile float*>(&p->s) = v.s;
+  *reinterpret_cast<volatile float*>(&p->gs) = v.gs;
+  *reinterpret_cast<volatile int*>(&p->idx) = v.idx;
+  *reinterpret_cast<volatile int*>(&p->gidx) = v.gidx;
+}
+
+__device__ __forceinline__ Stat load_partial(const VerifyPartial* p) {
+  Stat st;
+  st.m = __ldcg(&p->m); st.s = __ldcg(&p->s); st.gs = __ldcg(&p->gs);
+  st.idx = __ldcg(&p->idx); st.gidx = __ldcg(&p->gidx);
+  return st;
+}
+
+// Combine the chunk partials of one row with a warp; result valid in every lane.
+__device__ Stat gather_row(const VerifyPartial* p, int n_chunks, float c) {
+  Stat st = stat_empty();
+  for (int i = threadIdx.x & 31; i < n_chunks; i += 32) stat_merge(st, load_partial(p + i), c);
+  return warp_reduce(st, c);
+}
+
+// Returns true in exactly one block per sequence: the last one to arrive.
+__device__ bool arrive_last(int* counter, int expected) {
+  __shared__ int last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int prev = atomicAdd(counter, 1);
+    last = (prev == expected - 1);
+    if (last) *counter = 0;            // ready for the next launch
+  }
+  __syncthreads();
+  if (last) __threadfence();
+  return last != 0;
+}
+
+template <typename T, bool VECTOR>
+__global__ void __launch_bounds__(SPACE_VERIFY_THREADS)
+verify_target_kernel(const VerifyParams p) {
+  const int b = blockIdx.z, t = blockIdx.y, ch = blockIdx.x;
+  const int k1 = p.k + 1;
+  const T* row = reinterpret_cast<const T*>(p.logits) + ((int64_t)b * p.n_q + (int64_t)t * k1) * p.row_stride;
+  const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
+  Stat st = scan_chunk<T, VECTOR, false>(row, begin, end, p.c_t, 1.f, -1, 0, 0, 0, 0, 0);
+  st = block_reduce(st, p.c_t);
+  VerifyPartial* part = p.part + ((int64_t)b * (p.k + 2) + t) * p.n_chunks;
+  if (threadIdx.x == 0) store_partial(part + ch, st);
+  if (!arrive_last(p.counter_a + b, k1 * p.n_chunks)) return;
+  if (threadIdx.x >= 32) return;
+
+  // ---- last block of sequence b: acceptance loop of Algorithm 1 ----------
+  const int lane = threadIdx.x;
+  const T* base = reinterpret_cast<const T*>(p.logits) + (int64_t)b * p.n_q * p.row_stride;
+  const uint32_t seq = p.seq_id ? p.seq_id[b] : (uint32_t)b;
+  const int L = p.kv_len ? p.kv_len[b] : 0;
+  int i_star = 0, alive = 1, st_bits = 0;
+  for (int tt = 0; tt < k1; ++tt) {
+    const Stat r = gather_row(p.part + ((int64_t)b * (p.k + 2) + tt) * p.n_chunks, p.n_chunks, p.c_t);
+    if (lane == 0) {
+      VerifyRow vr; vr.m = r.m; vr.s = r.s; vr.idx = r.idx; vr.pad = 0;
+      p.rows[b * k1 + tt] = vr;
+    }
+    if (tt < p.k) {                    // row tt scores candidate c_{tt+1}
+      const int c = p.cand[b * p.k + tt];
+      const bool in_range = (c >= 0 && c < p.V);
+      if (!in_range) st_bits |= SPACE_ST_BAD_CANDIDATE;
+      bool ok;
+      if (p.mode == SPACE_MODE_GREEDY) {
+        ok = in_range && (c == r.idx);
+      } else {
+        float q = 0.f;
+        if (in_range) {
+          const float zc = load_logit(base + (int64_t)tt * k1 * p.row_stride + c);
+          q = exp2f((zc - r.m) * p.c_t) / r.s;
+        }
+        const Philox4 w = philox4x32_10(0u, PURPOSE_ACCEPT, seq, (uint32_t)(L + tt + 1), p.key0, p.key1);
+        const float lhs = uniform_open(w.x) * p.cand_prob[b * p.k + tt];   // r <= Q/P_c  <=>  r*P_c <= Q
+        ok = lhs <= q;
+      }
+      alive = alive && ok;
+      i_star += alive;
+    }
+  }
+  if (lane == 0) {
+    p.n_accept[b] = i_star;
+    if (p.status && st_bits) atomicOr(p.status + b, st_bits);
+  }
+}
+
+template <typename T, bool VECTOR>
+__global__ void __launch_bounds__(SPACE_VERIFY_THREADS)
+verify_emit_kernel(const VerifyParams p) {
+  const int b = blockIdx.z, slot = blockIdx.y, ch = blockIdx.x;
+  const int k1 = p.k + 1;
+  const int i_star = p.n_accept[b];
+  const bool sample = p.mode == SPACE_MODE_SAMPLE;
+  const bool literal = sample && p.resample == SPACE_RESAMPLE_PAPER_LITERAL;
+  const int n_slots = sample ? k1 : p.k;
+  const uint32_t seq = p.seq_id ? p.seq_id[b] : (uint32_t)b;
+  const int L = p.kv_len ? p.kv_len[b] : 0;
+  const T* base = reinterpret_cast<const T*>(p.logits) + (int64_t)b * p.n_q * p.row_stride;
+  // slot o < k: mask row (i*, o+1); slot k: target row i* (extra token, sampling)
+  const int brow = (slot < p.k) ? i_star * k1 + slot + 1 : i_star * k1;
+  const T* row = base + (int64_t)brow * p.row_stride;
+  const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
+  const float c = sample ? p.c_t : 1.4426950408889634f;
+  Stat st;
+  if (slot == p.k) {
+    int exclude = -1;
+    if (!literal && i_star < p.k) exclude = p.cand[b * p.k + i_star];   // residual of a point mass
+    st = scan_chunk<T, VECTOR, true>(row, begin, end, c, p.inv_t, exclude, p.key0, p.key1, PURPOSE_TOKEN,
+                                     seq, (uint32_t)(L + i_star + 1));
+  } else if (literal) {
+    st = scan_chunk<T, VECTOR, true>(row, begin, end, c, p.inv_t, -1, p.key0, p.key1, PURPOSE_DRAFT, seq,
+                                     (uint32_t)(L + i_star + 1 + slot + 1));
+  } else {
+    st = scan_chunk<T, VECTOR, false>(row, begin, end, c, 1.f, -1, 0, 0, 0, 0, 0);
+  }
+  st = block_reduce(st, c);
+  VerifyPartial* part = p.part + ((int64_t)b * (p.k + 2) + slot) * p.n_chunks;
+  if (threadIdx.x == 0) store_partial(part + ch, st);
+  if (!arrive_last(p.counter_b + b, n_slots * p.n_chunks)) return;
+  if (threadIdx.x >= 32) return;
+
+  // ---- last block of sequence b: emitted tokens and new candidates -------
+  const int lane = threadIdx.x;
+  int bonus;
+  if (sample) {
+    const Stat r = gather_row(p.part + ((int64_t)b * (p.k + 2) + p.k) * p.n_chunks, p.n_chunks, c);
+    bonus = r.gidx;
+  } else {
+    bonus = p.rows[b * k1 + i_star].idx;
+  }
+  for (int o = 0; o < p.k; ++o) {
+    const Stat r = gather_row(p.part + ((int64_t)b * (p.k + 2) + o) * p.n_chunks, p.n_chunks, c);
+    if (lane == 0) {
+      int tok; float pr;
+      if (!sample)      { tok = r.idx;  pr = 1.f / r.s; }          // softmax at T = 1 of its own maximum
+      else if (!literal){ tok = r.idx;  pr = 1.f; }                 // point-mass draft
+      else {
+        tok = r.gidx;
+        const float z = load_logit(base + (int64_t)(i_star * k1 + o + 1) * p.row_stride + tok);
+        pr = exp2f((z - r.m) * c) / r.s;
+      }
+      p.next_cand[b * p.k + o] = tok;
+      p.next_cand_prob[b * p.k + o] = pr;
+    }
+  }
+  if (lane == 0) {
+    int n_out = i_star + 1, fin = 0;
+    for (int j = 0; j < k1; ++j) {
+      int tok = (j < i_star) ? p.cand[b * p.k + j] : (j == i_star ? bonus : -1);
+      if (!fin && j <= i_star && p.eos_id >= 0 && tok == p.eos_id) { fin = 1; n_out = j; }
+      if (j >= n_out) tok = -1;
+      p.out_tokens[b * k1 + j] = tok;
+    }
+    p.n_out[b] = n_out;
+    p.finished[b] = (uint8_t)fin;
+  }
+}
+
+template <typename T, bool VECTOR>
+void launch_both(space_ctx* ctx, const VerifyParams& p, int n_slots_b, cudaStream_t st) {
+  dim3 ga(p.n_chunks, p.k + 1, p.B), gb(p.n_chunks, n_slots_b, p.B);
+  {
+    ProfScope ps(ctx, SPACE_K_VERIFY_TARGET, st);
+    verify_target_kernel<T, VECTOR><<<ga, SPACE_VERIFY_THREADS, 0, st>>>(p);
+  }
+  {
+    ProfScope ps(ctx, SPACE_K_VERIFY_EMIT, st);
+    verify_emit_kernel<T, VECTOR><<<gb, SPACE_VERIFY_THREADS, 0, st>>>(p);
+  }
+}
+
+__global__ void philox_debug_kernel(uint32_t k0, uint32_t k1, int64_t n, const uint32_t* c0,
+                                    const uint32_t* c1, const uint32_t* c2, const uint32_t* c3,
+                                    uint32_t* out) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const Philox4 r = philox4x32_10(c0[i], c1[i], c2[i], c3[i], k0, k1);
+  out[4 * i] = r.x; out[4 * i + 1] = r.y; out[4 * i + 2] = r.z; out[4 * i + 3] = r.w;
+}
+
+}  // namespace
+
+int launch_verify(space_ctx* ctx, const space_verify_args* a, cudaStream_t st) {
+  VerifyParams p;
+  p.B = a->batch; p.k = a->k; p.V = a->vocab; p.n_q = (a->k + 1) * (a->k + 1);
+  p.mode = a->mode; p.resample = a->resample; p.eos_id = a->eos_id;
+  const float T = (a->mode == SPACE_MODE_SAMPLE) ? a->temperature : 1.0f;
+  p.c_t = 1.4426950408889634f / T;
+  p.inv_t = 1.0f / T;
+  p.key0 = (uint32_t)(a->seed & 0xFFFFFFFFull); p.key1 = (uint32_t)(a->seed >> 32);
+  p.logits = a->logits; p.row_stride = a->logits_row_stride;
+  p.cand = a->cand; p.cand_prob = a->cand_prob; p.seq_id = a->seq_id; p.kv_len = a->kv_len;
+  p.n_accept = a->n_accept; p.out_tokens = a->out_tokens; p.n_out = a->n_out;
+  p.next_cand = a->next_cand; p.next_cand_prob = a->next_cand_prob; p.finished = a->finished;
+  p.status = a->status;
+  p.part = ctx->vpart; p.rows = ctx->vrow;
+  p.counter_a = ctx->counters; p.counter_b = ctx->counters + ctx->cfg.max_batch;
+
+  const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;
+  const int vec = 16 / esz;
+  const bool vector = ((uintptr_t)a->logits % 16 == 0) && ((a->logits_row_stride * esz) % 16 == 0);
+  // enough chunks to put about two blocks on every SM, but no chunk below two
+  // sweeps of a block
+  const int rows = a->batch * (a->k + 1);
+  int nc = (2 * ctx->sm_count + rows - 1) / rows;
+  const int min_chunk = SPACE_VERIFY_THREADS * vec * 2;
+  const int max_nc = (a->vocab + min_chunk - 1) / min_chunk;
+  if (nc > max_nc) nc = max_nc;
+  if (nc > SPACE_VERIFY_MAX_CHUNKS) nc = SPACE_VERIFY_MAX_CHUNKS;
+  if (nc < 1) nc = 1;
+  int chunk = (a->vocab + nc - 1) / nc;
+  chunk = ((chunk + vec - 1) / vec) * vec;
+  nc = (a->vocab + chunk - 1) / chunk;
+  p.n_chunks = nc; p.chunk = chunk;
+  const int n_slots_b = (a->mode == SPACE_MODE_SAMPLE) ? a->k + 1 : a->k;
+
+  if (a->logits_dtype == SPACE_DTYPE_F32) {
+    if (vector) launch_both<float, true>(ctx, p, n_slots_b, st); else launch_both<float, false>(ctx, p, n_slots_b, st);
+  } else {
+    if (vector) launch_both<__nv_bfloat16, true>(ctx, p, n_slots_b, st);
+    else launch_both<__nv_bfloat16, false>(ctx, p, n_slots_b, st);
+  }
+  ctx->launches += 2;
+  return cuda_ok(cudaGetLastError());
+}
+
+int launch_philox_debug(uint64_t seed, int64_t n, const uint32_t* c0, const uint32_t* c1,
+                        const uint32_t* c2, const uint32_t* c3, uint32_t* out, cudaStream_t st) {
+  if (n <= 0) return SPACE_OK;
+  philox_debug_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
+      (uint32_t)(seed & 0xFFFFFFFFull), (uint32_t)(seed >> 32), n, c0, c1, c2, c3, out);
+  return cuda_ok(cudaGetLastError());
+}

@@ -1,0 +1,347 @@
+"""GPU parity: the CUDA path (through the C-ABI) against the fp64 oracle on the
+same seeded inputs.  Integer results bit-exact; attention within
+max|err| <= min(2e-2, 1e-2 * RMS(oracle output)); probabilities to 1e-4 relative.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import layout as olayout
+from oracle.attention import attention_step, attention_head
+from oracle.verify import verify_step
+from oracle.commit import commit_step
+from oracle.bf16 import bf16_bits_to_f64
+from oracle.philox import philox4x32_10
+from paper_2402_11809_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+ACCEPT_BAND = 1e-4      # relative distance of r*P_c from Q(c) below which an acceptance is a tie
+GUMBEL_BAND = 1e-4      # top-two Gumbel score gap below which a draw is a tie
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2402_11809_b200 import build
+    build.build()
+    from paper_2402_11809_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def H():
+    import gpu_harness
+    return gpu_harness
+
+
+def _check_attention(H, got, ref, what=""):
+    tol, rms = H.attn_tolerance(ref)
+    err = float(np.max(np.abs(got - ref)))
+    assert np.isfinite(got).all(), what
+    assert err <= tol, f"{what}: max|err| {err:.3e} > {tol:.3e} (rms {rms:.3e})"
+    return err / rms
+
+
+def _check_verify(ds, r, k, sample=False):
+    """Compare device verify outputs with oracle dict r; returns excluded sequences."""
+    acc_tie = (r["accept_margin"] <= ACCEPT_BAND).any(axis=1)
+    draw_tie = (r["bonus_gap"] <= GUMBEL_BAND) | (r["draft_gap"] <= GUMBEL_BAND).any(axis=1)
+    excl = acc_tie | draw_tie
+    keep = ~excl
+    n_accept = ds.n_accept.cpu().numpy()
+    assert np.array_equal(n_accept[keep], r["n_accept"][keep])
+    assert np.array_equal(ds.out_tokens.cpu().numpy()[keep], r["out_tokens"][keep])
+    assert np.array_equal(ds.n_out.cpu().numpy()[keep], r["n_out"][keep])
+    assert np.array_equal(ds.next_cand.cpu().numpy()[keep], r["next_cand"][keep])
+    assert np.array_equal(ds.finished.cpu().numpy()[keep], r["finished"][keep])
+    np.testing.assert_allclose(ds.next_cand_prob.cpu().numpy()[keep], r["next_cand_prob"][keep],
+                               rtol=1e-4, atol=1e-30)
+    if excl.any():
+        print(f"excluded {int(excl.sum())} sequence(s) inside the tie band: {np.nonzero(excl)[0].tolist()}")
+    return excl
+
+
+def _small_cfg(k, L, d=128, H_q=2, H_kv=2, Bn=2, V=777, dtype="bf16", seed=0):
+    return workloads.resolve("tiny", B=Bn, H_q=H_q, H_kv=H_kv, d=d, L=L, k=k, V=V,
+                             logits_dtype=dtype, sigma=2.0, p_accept=(0.6, 0.6), seed=seed)
+
+
+# --------------------------------------------------------------------- Philox
+def test_device_philox_matches_oracle(B, H):
+    rng = np.random.default_rng(0)
+    n = 100_000
+    c = rng.integers(0, 2 ** 32, size=(4, n), dtype=np.uint64).astype(np.uint32)
+    c[:, 0] = 0
+    c[:, 1] = 0xFFFFFFFF
+    seed = 0x299F31D0A4093822
+    ctx = B.Context(max_batch=1, s_cap=64)
+    dev = [H.to_dev(x) for x in c]
+    out = torch.zeros(n * 4, dtype=torch.int32, device="cuda")
+    ctx.space_debug_philox(seed, dev[0], dev[1], dev[2], dev[3], out)
+    got = out.cpu().numpy().view(np.uint32).reshape(n, 4)
+    ref = np.stack(philox4x32_10(c[0], c[1], c[2], c[3], seed & 0xFFFFFFFF, seed >> 32), axis=1)
+    assert np.array_equal(got, ref)
+
+
+# ------------------------------------------------------------------ attention
+@pytest.mark.parametrize("impl", ["tensor", "simt"])
+@pytest.mark.parametrize("k,L,d,H_q,H_kv", [
+    (1, (0, 0), 64, 2, 2), (2, (1, 1), 128, 2, 2), (3, (127, 127), 128, 2, 1),
+    (4, (128, 128), 64, 8, 8), (5, (129, 300), 128, 4, 4), (6, (200, 600), 128, 8, 1),
+    (7, (5, 900), 128, 4, 2), (5, (1000, 1400), 64, 16, 1), (2, (250, 260), 128, 16, 1),
+])
+def test_attention_small(B, H, impl, k, L, d, H_q, H_kv):
+    cfg = _small_cfg(k, L, d=d, H_q=H_q, H_kv=H_kv, Bn=3, seed=k)
+    x = workloads.make_step_inputs(cfg, poison_tail=True)
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    ds.attn(ctx, impl=B.ATTN_TENSOR if impl == "tensor" else B.ATTN_SIMT)
+    torch.cuda.synchronize()
+    ref, ref_lse = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], k, x["scale"])
+    _check_attention(H, ds.out.cpu().numpy().astype(np.float64), ref, f"{impl} k={k} L={L}")
+    np.testing.assert_allclose(ds.lse.cpu().numpy(), ref_lse, rtol=0, atol=2e-3)
+    assert int(ds.status.abs().sum()) == 0
+
+
+@pytest.mark.parametrize("k", [3, 5])
+def test_attention_eq5_literal_variant_and_bf16_output(B, H, k):
+    cfg = _small_cfg(k, (100, 200), Bn=2, seed=40 + k)
+    x = workloads.make_step_inputs(cfg)
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    ds.attn(ctx, mask_variant=B.MASK_EQ5_LITERAL)
+    ref, _ = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], k, x["scale"],
+                            olayout.EQ5_LITERAL)
+    _check_attention(H, ds.out.cpu().numpy().astype(np.float64), ref, "literal")
+    same, _ = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], k, x["scale"])
+    assert np.abs(same - ref).max() > 1e-3            # the two readings do differ for k >= 3
+    out16 = torch.zeros_like(ds.out, dtype=torch.bfloat16)
+    ds.attn(ctx, out=out16)
+    got = bf16_bits_to_f64(H.bf16_to_bits(out16))
+    assert np.max(np.abs(got - same)) <= 2.0 ** -8 * np.maximum(np.abs(same), 2.0 ** -126).max()
+
+
+def test_attention_split_invariance_and_determinism(B, H):
+    # A long single sequence is split over many thread blocks; a batch of short
+    # ones is not.  Both must agree with the oracle, and a re-run is bit-identical.
+    cfg = _small_cfg(5, (3000, 3000), H_q=1, H_kv=1, Bn=1, seed=7)
+    x = workloads.make_step_inputs(cfg)
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    ds.attn(ctx)
+    a = ds.out.clone()
+    ds.out.fill_(float("nan"))
+    ds.attn(ctx)
+    assert torch.equal(a, ds.out)
+    ref, _ = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], 5, x["scale"])
+    _check_attention(H, a.cpu().numpy().astype(np.float64), ref, "split")
+
+
+def test_attention_large_scores_rescale_path(B, H):
+    # keys whose scores grow along the sequence force the running maximum to move
+    # by far more than the lazy-rescale threshold in later tiles
+    cfg = _small_cfg(2, (700, 700), H_q=1, H_kv=1, Bn=1, seed=9)
+    x = workloads.make_step_inputs(cfg)
+    kf = bf16_bits_to_f64(x["k_cache"]).astype(np.float32)
+    qf = bf16_bits_to_f64(x["q"]).astype(np.float32)
+    ramp = np.linspace(0.0, 6.0, kf.shape[2], dtype=np.float32)[None, None, :, None]
+    kf = kf + ramp * np.sign(qf[0, 0, 0])[None, None, None, :]
+    x["k_cache"] = workloads.f32_to_bf16_bits(kf)
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    ds.attn(ctx)
+    ref, ref_lse = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], 2, x["scale"])
+    assert ref_lse.max() - ref_lse.min() > 20.0
+    _check_attention(H, ds.out.cpu().numpy().astype(np.float64), ref, "rescale")
+
+
+def test_capacity_overflow_is_flagged_not_computed(B, H):
+    cfg = _small_cfg(3, (50, 50), Bn=2, seed=3)
+    x = workloads.make_step_inputs(cfg)
+    x["kv_len"][1] = x["s_cap"] - 3                       # L + n_q > capacity
+    ctx = H.make_context(cfg, x)
+    for impl in (B.ATTN_TENSOR, B.ATTN_SIMT):
+        ds = H.DeviceStep(cfg, x)
+        ds.attn(ctx, impl=impl)
+        st = ds.status.cpu().numpy()
+        assert st[0] == 0 and st[1] & B.ST_CAPACITY
+        ref, _ = attention_head(x["q"][0, :, 0], x["k_cache"][0, 0], x["v_cache"][0, 0], 50, 3, x["scale"])
+        _check_attention(H, ds.out[0, :, 0].cpu().numpy().astype(np.float64), ref)
+        assert torch.isnan(ds.out[1]).all()               # untouched
+
+
+def test_argument_validation(B, H):
+    cfg = _small_cfg(2, (10, 10), Bn=1)
+    x = workloads.make_step_inputs(cfg)
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    a = ds.attn(ctx)
+    import ctypes as C
+    bad = B.AttnArgs.from_buffer_copy(a); bad.k = 3
+    assert B.lib.space_attn_step(ctx._h, C.byref(bad), None) == B.E_INVALID_ARG
+    bad = B.AttnArgs.from_buffer_copy(a); bad.batch = 2
+    assert B.lib.space_attn_step(ctx._h, C.byref(bad), None) == B.E_WORKSPACE
+    bad = B.AttnArgs.from_buffer_copy(a); bad.q = a.q + 2
+    assert B.lib.space_attn_step(ctx._h, C.byref(bad), None) == B.E_ALIGNMENT
+    bad = B.AttnArgs.from_buffer_copy(a); bad.kv_stride_s = 130
+    assert B.lib.space_attn_step(ctx._h, C.byref(bad), None) == B.E_ALIGNMENT
+    bad = B.AttnArgs.from_buffer_copy(a); bad.scale = 0.0
+    assert B.lib.space_attn_step(ctx._h, C.byref(bad), None) == B.E_INVALID_ARG
+    bad = B.AttnArgs.from_buffer_copy(a); bad.out = None
+    assert B.lib.space_attn_step(ctx._h, C.byref(bad), None) == B.E_INVALID_ARG
+    torch.cuda.synchronize()
+
+
+# --------------------------------------------------------------------- verify
+@pytest.mark.parametrize("k,V,dtype,Bn", [(1, 17, "f32", 5), (2, 1000, "f32", 7), (4, 1003, "bf16", 9),
+                                          (5, 32000, "bf16", 3), (7, 5001, "bf16", 4),
+                                          (3, 128256, "bf16", 2)])
+def test_verify_greedy_small(B, H, k, V, dtype, Bn):
+    cfg = _small_cfg(k, (5, 40), H_q=1, H_kv=1, d=64, Bn=Bn, V=V, dtype=dtype, seed=100 + k)
+    x = workloads.make_step_inputs(cfg)
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    ds.verify(ctx)
+    r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "greedy")
+    excl = _check_verify(ds, r, k)
+    assert not excl.any()
+    # end-of-sequence handling: make the first emitted token of sequence 0 the <EOS>
+    eos = int(r["out_tokens"][0, 0])
+    ds.verify(ctx, eos_id=eos)
+    r2 = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "greedy", eos_id=eos)
+    assert r2["finished"][0] == 1 and r2["n_out"][0] == 0
+    _check_verify(ds, r2, k)
+
+
+def test_verify_greedy_exact_ties_and_bad_candidates(B, H):
+    k, V = 3, 4096
+    cfg = _small_cfg(k, (5, 5), H_q=1, H_kv=1, d=64, Bn=4, V=V, seed=5)
+    x = workloads.make_step_inputs(cfg)
+    # bf16 logits quantised to multiples of 4: thousands of exact ties per row
+    lf = np.round(bf16_bits_to_f64(x["logits"]) / 4.0) * 4.0
+    x["logits"] = workloads.f32_to_bf16_bits(lf.astype(np.float32))
+    x["cand"][1, 0] = V + 5
+    x["cand"][2, 0] = -3
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    ds.verify(ctx)
+    r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "greedy")
+    _check_verify(ds, r, k)
+    st = ds.status.cpu().numpy()
+    assert st[1] & B.ST_BAD_CANDIDATE and st[2] & B.ST_BAD_CANDIDATE and st[0] == 0
+
+
+@pytest.mark.parametrize("resample", ["residual_pointmass", "paper_literal"])
+@pytest.mark.parametrize("k,V,Bn,T", [(2, 16, 64, 1.0), (4, 5000, 16, 0.8), (3, 128256, 4, 0.8)])
+def test_verify_sampling_small(B, H, resample, k, V, Bn, T):
+    cfg = workloads.resolve("sampling64", B=Bn, H_q=1, H_kv=1, d=64, L=(5, 600), k=k, V=V,
+                            temperature=T, seed=200 + k)
+    x = workloads.make_step_inputs(cfg)
+    if resample == "paper_literal":
+        x["cand_prob"] = np.random.default_rng(1).uniform(0.2, 1.0, size=x["cand_prob"].shape).astype(np.float32)
+    x["cand_prob"][0, :] = np.inf                        # Algorithm 1 initial state: nothing accepted
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    code = B.RESAMPLE_RESIDUAL_POINTMASS if resample == "residual_pointmass" else B.RESAMPLE_PAPER_LITERAL
+    for seed in (0, 0xDEADBEEF12345678):
+        ds.verify(ctx, mode=B.MODE_SAMPLE, temperature=T, seed=seed, resample=code)
+        r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "sample", temperature=T, seed=seed,
+                        seq_id=x["seq_id"], kv_len=x["kv_len"], resample=resample)
+        excl = _check_verify(ds, r, k, sample=True)
+        assert excl.mean() < 0.2
+        assert r["n_accept"][0] == 0 and int(ds.n_accept[0]) == 0
+    assert r["n_accept"].max() > 0
+
+
+# --------------------------------------------------------------------- commit
+@pytest.mark.parametrize("k,d,H_kv,Bn", [(1, 64, 1, 3), (5, 128, 32, 2), (7, 128, 8, 5)])
+def test_commit(B, H, k, d, H_kv, Bn):
+    cfg = _small_cfg(k, (3, 90), d=d, H_q=H_kv, H_kv=H_kv, Bn=Bn, seed=300 + k)
+    x = workloads.make_step_inputs(cfg)
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    n_acc = np.random.default_rng(k).integers(0, k + 1, size=Bn).astype(np.int32)
+    n_acc[0] = k
+    ds.n_accept.copy_(torch.from_numpy(n_acc))
+    ds.commit(ctx)
+    Kc, Vc = x["k_cache"].copy(), x["v_cache"].copy()
+    new_len, src, dst = commit_step(Kc, Vc, x["kv_len"], n_acc, k)
+    assert np.array_equal(H.bf16_to_bits(ds.k_cache), Kc)
+    assert np.array_equal(H.bf16_to_bits(ds.v_cache), Vc)
+    assert np.array_equal(ds.kv_len_out.cpu().numpy(), new_len)
+    assert np.array_equal(ds.commit_src.cpu().numpy(), src)
+    assert np.array_equal(ds.commit_dst.cpu().numpy(), dst)
+    # in-place length update
+    a = ctx.commit_args(ds.k_cache, ds.v_cache, ds.n_accept, ds.kv_len, k, kv_len_out=ds.kv_len)
+    ds.n_accept.zero_()
+    ctx.space_kv_commit(a)
+    assert np.array_equal(ds.kv_len.cpu().numpy(), x["kv_len"] + 1)
+
+
+# ------------------------------------------------------------ the five configs
+def _run_config(B, H, name, sample_heads=None, **over):
+    cfg = workloads.resolve(name, **over)
+    x = workloads.make_step_inputs(cfg)
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    k = cfg["k"]
+    sample = cfg["mode"] == "sample"
+    ds.attn(ctx)
+    ds.verify(ctx, mode=B.MODE_SAMPLE if sample else B.MODE_GREEDY, temperature=cfg["temperature"],
+              seed=cfg["seed"])
+    ds.commit(ctx)
+    torch.cuda.synchronize()
+    assert int(ds.status.abs().sum()) == 0
+    out = ds.out.cpu().numpy().astype(np.float64)
+    G = cfg["H_q"] // cfg["H_kv"]
+    if sample_heads is None:
+        ref, _ = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], k, x["scale"])
+        rel = _check_attention(H, out, ref, name)
+    else:
+        rng = np.random.default_rng(cfg["seed"])
+        rel = 0.0
+        for _ in range(sample_heads):
+            b, h = int(rng.integers(cfg["B"])), int(rng.integers(cfg["H_q"]))
+            ref, _ = attention_head(x["q"][b, :, h], x["k_cache"][b, h // G], x["v_cache"][b, h // G],
+                                    int(x["kv_len"][b]), k, x["scale"])
+            rel = max(rel, _check_attention(H, out[b, :, h], ref, f"{name} b={b} h={h}"))
+        assert np.isfinite(out).all()
+    r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, cfg["mode"], temperature=cfg["temperature"],
+                    seed=cfg["seed"], seq_id=x["seq_id"], kv_len=x["kv_len"])
+    excl = _check_verify(ds, r, k, sample)
+    n_acc = ds.n_accept.cpu().numpy()
+    new_len = ds.kv_len_out.cpu().numpy()
+    assert np.array_equal(new_len, x["kv_len"] + n_acc + 1)
+    # committed rows, checked on the device copy against the original input rows
+    kc, vc = H.bf16_to_bits(ds.k_cache), H.bf16_to_bits(ds.v_cache)
+    for b in range(cfg["B"]):
+        L = int(x["kv_len"][b])
+        for g in range(int(n_acc[b]) + 1):
+            assert np.array_equal(kc[b, :, L + g], x["k_cache"][b, :, L + g * (k + 1)])
+            assert np.array_equal(vc[b, :, L + g], x["v_cache"][b, :, L + g * (k + 1)])
+        assert np.array_equal(kc[b, :, :L], x["k_cache"][b, :, :L])
+    print(f"{name}: attention max|err|/rms {rel:.2e}; mean accepted {n_acc.mean():.2f}; "
+          f"excluded {int(excl.sum())}")
+    return n_acc
+
+
+def test_config_tiny(B, H):
+    _run_config(B, H, "tiny")
+
+
+def test_config_llama7b(B, H):
+    n = _run_config(B, H, "llama7b")
+    assert 0 <= n[0] <= 5
+
+
+def test_config_ragged16(B, H):
+    _run_config(B, H, "ragged16", sample_heads=24)
+
+
+def test_config_gqa70b(B, H):
+    _run_config(B, H, "gqa70b", sample_heads=12)
+
+
+def test_config_sampling64(B, H):
+    n = _run_config(B, H, "sampling64", sample_heads=12)
+    assert n.mean() > 0.5
