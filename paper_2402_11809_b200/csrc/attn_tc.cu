@@ -348,10 +348,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         const uint32_t vsm = sm_base + S::KV_OFF + s * 2 * S::TILE_BYTES + S::TILE_BYTES;
         const uint32_t ptm = TM_S0 + buf * TILE_N;
 #pragma unroll
-        for (int kk = 0; kk < TILE_N / 16; ++kk) {
-          // V tile is MN-major: 64-wide d blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
-          const uint64_t bd = smem_desc(vsm + kk * 2048, TILE_N * 128, 1024);
-          mma_ts(TM_O, ptm + kk * 8, bd, IDESC_PV, (first_in_seg && kk == 0) ? 0u : 1u);
+        for (int part_i = 0; part_i < 2; ++part_i) {        // P_hi, then P_lo
+#pragma unroll
+          for (int kk = 0; kk < TILE_N / 16; ++kk) {
+            // V tile is MN-major: 64-wide d blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
+            const uint64_t bd = smem_desc(vsm + kk * 2048, TILE_N * 128, 1024);
+            mma_ts(TM_O, ptm + part_i * (TILE_N / 2) + kk * 8, bd, IDESC_PV,
+                   (first_in_seg && kk == 0 && part_i == 0) ? 0u : 1u);
+          }
         }
         tc_commit(BAR(B_KVEMPTY + s));
         tc_commit(BAR(B_PVDONE + buf));
@@ -454,17 +458,26 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           tmem_wait_st();
         }
         const float m_use = (m_ref > -CUDART_INF_F) ? m_ref : 0.f;
-        uint32_t preg[TILE_N / 2];
+        // P = P_hi + P_lo, two bf16 terms: bf16 alone (8 significant bits) leaves
+        // an output error near 1e-2 of the output RMS.  P_hi goes to columns
+        // 0..63 of the S buffer, P_lo to columns 64..127.
+        uint32_t lreg[TILE_N / 2];
 #pragma unroll
         for (int x = 0; x < TILE_N / 2; ++x) {
           const float p0 = exp2f(fmaf(__uint_as_float(sreg[2 * x]), c, -m_use));
           const float p1 = exp2f(fmaf(__uint_as_float(sreg[2 * x + 1]), c, -m_use));
           l_sum += p0 + p1;
-          const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);   // .x (low half) = even key
-          preg[x] = *reinterpret_cast<const uint32_t*>(&pk);
+          const __nv_bfloat162 hi = __floats2bfloat162_rn(p0, p1);   // .x (low half) = even key
+          const float2 hf = __bfloat1622float2(hi);
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
+          sreg[x] = *reinterpret_cast<const uint32_t*>(&hi);
+          lreg[x] = *reinterpret_cast<const uint32_t*>(&lo);
         }
 #pragma unroll
-        for (int cc = 0; cc < TILE_N / 64; ++cc) tmem_st32(ts + cc * 32, preg + cc * 32);
+        for (int cc = 0; cc < TILE_N / 64; ++cc) {
+          tmem_st32(ts + cc * 32, sreg + cc * 32);
+          tmem_st32(ts + TILE_N / 2 + cc * 32, lreg + cc * 32);
+        }
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(BAR(B_PREADY + buf));
@@ -562,22 +575,31 @@ __global__ void __launch_bounds__(DH) attn_merge_kernel(const AttnParams p, int 
   const int g_first = (int)(((f0 + 1) * NG - 1) / W);
   const int g_last = (int)(((f0 + T) * NG - 1) / W);
   if (g_first == g_last) return;                            // written directly by the main kernel
+  // groups that hold tiles of this (sequence, head): computed once per block
+  __shared__ int list[256];
+  __shared__ int n_list;
+  if (threadIdx.x == 0) {
+    int n = 0;
+    for (int gi = g_first; gi <= g_last && n < 256; ++gi)
+      if ((W * gi) / NG != (W * (gi + 1)) / NG) list[n++] = gi;
+    n_list = n;
+  }
+  __syncthreads();
   const int c = threadIdx.x;
   const int i0 = mb * p.rows_per_mb;
   const int m_begin = blockIdx.y * rows_per_block;
+  const size_t slot_floats = (size_t)ROWS * (DH + 2);
   for (int m = m_begin; m < m_begin + rows_per_block && m < ROWS; ++m) {
     const int il = m / p.G, g = m % p.G, i = i0 + il;
     if (il >= p.rows_per_mb || i >= p.n_q) continue;
     float mx = -CUDART_INF_F;
-    for (int gi = g_first; gi <= g_last; ++gi) {
-      if ((W * gi) / NG == (W * (gi + 1)) / NG) continue;   // this group holds no tiles
-      const float* ps = p.part + ((size_t)(item + gi) * p.n_mblocks + mb) * (ROWS * (DH + 2));
+    for (int x = 0; x < n_list; ++x) {
+      const float* ps = p.part + ((size_t)(item + list[x]) * p.n_mblocks + mb) * slot_floats;
       mx = fmaxf(mx, __ldcg(ps + ROWS * DH + m));
     }
     float acc = 0.f, den = 0.f;
-    for (int gi = g_first; gi <= g_last; ++gi) {
-      if ((W * gi) / NG == (W * (gi + 1)) / NG) continue;
-      const float* ps = p.part + ((size_t)(item + gi) * p.n_mblocks + mb) * (ROWS * (DH + 2));
+    for (int x = 0; x < n_list; ++x) {
+      const float* ps = p.part + ((size_t)(item + list[x]) * p.n_mblocks + mb) * slot_floats;
       const float ms = __ldcg(ps + ROWS * DH + m);
       const float w = (ms > -CUDART_INF_F) ? exp2f(ms - mx) : 0.f;
       den = fmaf(w, __ldcg(ps + ROWS * DH + ROWS + m), den);

@@ -234,44 +234,51 @@ verify_target_kernel(const VerifyParams p) {
   VerifyPartial* part = p.part + ((int64_t)b * (p.k + 2) + t) * p.n_chunks;
   if (threadIdx.x == 0) store_partial(part + ch, st);
   if (!arrive_last(p.counter_a + b, k1 * p.n_chunks)) return;
-  if (threadIdx.x >= 32) return;
 
   // ---- last block of sequence b: acceptance loop of Algorithm 1 ----------
-  const int lane = threadIdx.x;
-  const T* base = reinterpret_cast<const T*>(p.logits) + (int64_t)b * p.n_q * p.row_stride;
-  const uint32_t seq = p.seq_id ? p.seq_id[b] : (uint32_t)b;
-  const int L = p.kv_len ? p.kv_len[b] : 0;
-  int i_star = 0, alive = 1, st_bits = 0;
-  for (int tt = 0; tt < k1; ++tt) {
-    const Stat r = gather_row(p.part + ((int64_t)b * (p.k + 2) + tt) * p.n_chunks, p.n_chunks, p.c_t);
+  // Warp tt combines the chunk results of target row tt and evaluates the
+  // acceptance test of candidate c_{tt+1}; thread 0 then walks the prefix.
+  __shared__ int sh_ok[SPACE_MAX_K + 1];
+  __shared__ int sh_bits;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) sh_bits = 0;
+  __syncthreads();
+  if (warp < k1) {
+    const int tt = warp;
+    const Stat r = gather_row(part - (int64_t)t * p.n_chunks + (int64_t)tt * p.n_chunks, p.n_chunks, p.c_t);
     if (lane == 0) {
       VerifyRow vr; vr.m = r.m; vr.s = r.s; vr.idx = r.idx; vr.pad = 0;
       p.rows[b * k1 + tt] = vr;
-    }
-    if (tt < p.k) {                    // row tt scores candidate c_{tt+1}
-      const int c = p.cand[b * p.k + tt];
-      const bool in_range = (c >= 0 && c < p.V);
-      if (!in_range) st_bits |= SPACE_ST_BAD_CANDIDATE;
-      bool ok;
-      if (p.mode == SPACE_MODE_GREEDY) {
-        ok = in_range && (c == r.idx);
-      } else {
-        float q = 0.f;
-        if (in_range) {
-          const float zc = load_logit(base + (int64_t)tt * k1 * p.row_stride + c);
-          q = exp2f((zc - r.m) * p.c_t) / r.s;
+      bool ok = false;
+      if (tt < p.k) {                  // row tt scores candidate c_{tt+1}
+        const int c = p.cand[b * p.k + tt];
+        const bool in_range = (c >= 0 && c < p.V);
+        if (!in_range) atomicOr(&sh_bits, SPACE_ST_BAD_CANDIDATE);
+        if (p.mode == SPACE_MODE_GREEDY) {
+          ok = in_range && (c == r.idx);
+        } else {
+          const T* base = reinterpret_cast<const T*>(p.logits) + (int64_t)b * p.n_q * p.row_stride;
+          const uint32_t seq = p.seq_id ? p.seq_id[b] : (uint32_t)b;
+          const int L = p.kv_len ? p.kv_len[b] : 0;
+          float q = 0.f;
+          if (in_range) {
+            const float zc = load_logit(base + (int64_t)tt * k1 * p.row_stride + c);
+            q = exp2f((zc - r.m) * p.c_t) / r.s;
+          }
+          const Philox4 w = philox4x32_10(0u, PURPOSE_ACCEPT, seq, (uint32_t)(L + tt + 1), p.key0, p.key1);
+          const float lhs = uniform_open(w.x) * p.cand_prob[b * p.k + tt];   // r <= Q/P_c  <=>  r*P_c <= Q
+          ok = lhs <= q;
         }
-        const Philox4 w = philox4x32_10(0u, PURPOSE_ACCEPT, seq, (uint32_t)(L + tt + 1), p.key0, p.key1);
-        const float lhs = uniform_open(w.x) * p.cand_prob[b * p.k + tt];   // r <= Q/P_c  <=>  r*P_c <= Q
-        ok = lhs <= q;
       }
-      alive = alive && ok;
-      i_star += alive;
+      sh_ok[tt] = ok;
     }
   }
-  if (lane == 0) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int i_star = 0;
+    while (i_star < p.k && sh_ok[i_star]) ++i_star;
     p.n_accept[b] = i_star;
-    if (p.status && st_bits) atomicOr(p.status + b, st_bits);
+    if (p.status && sh_bits) atomicOr(p.status + b, sh_bits);
   }
 }
 
@@ -308,19 +315,15 @@ verify_emit_kernel(const VerifyParams p) {
   VerifyPartial* part = p.part + ((int64_t)b * (p.k + 2) + slot) * p.n_chunks;
   if (threadIdx.x == 0) store_partial(part + ch, st);
   if (!arrive_last(p.counter_b + b, n_slots * p.n_chunks)) return;
-  if (threadIdx.x >= 32) return;
 
   // ---- last block of sequence b: emitted tokens and new candidates -------
-  const int lane = threadIdx.x;
-  int bonus;
-  if (sample) {
-    const Stat r = gather_row(p.part + ((int64_t)b * (p.k + 2) + p.k) * p.n_chunks, p.n_chunks, c);
-    bonus = r.gidx;
-  } else {
-    bonus = p.rows[b * k1 + i_star].idx;
-  }
-  for (int o = 0; o < p.k; ++o) {
-    const Stat r = gather_row(p.part + ((int64_t)b * (p.k + 2) + o) * p.n_chunks, p.n_chunks, c);
+  // Warp o combines mask row o (next candidate o+1); warp k the extra-token row.
+  __shared__ int sh_bonus;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  VerifyPartial* pb = p.part + (int64_t)b * (p.k + 2) * p.n_chunks;
+  if (warp < p.k) {
+    const int o = warp;
+    const Stat r = gather_row(pb + (int64_t)o * p.n_chunks, p.n_chunks, c);
     if (lane == 0) {
       int tok; float pr;
       if (!sample)      { tok = r.idx;  pr = 1.f / r.s; }          // softmax at T = 1 of its own maximum
@@ -333,17 +336,26 @@ verify_emit_kernel(const VerifyParams p) {
       p.next_cand[b * p.k + o] = tok;
       p.next_cand_prob[b * p.k + o] = pr;
     }
+  } else if (warp == p.k) {
+    int bonus;
+    if (sample) bonus = gather_row(pb + (int64_t)p.k * p.n_chunks, p.n_chunks, c).gidx;
+    else bonus = p.rows[b * k1 + i_star].idx;
+    if (lane == 0) sh_bonus = bonus;
   }
-  if (lane == 0) {
-    int n_out = i_star + 1, fin = 0;
-    for (int j = 0; j < k1; ++j) {
-      int tok = (j < i_star) ? p.cand[b * p.k + j] : (j == i_star ? bonus : -1);
-      if (!fin && j <= i_star && p.eos_id >= 0 && tok == p.eos_id) { fin = 1; n_out = j; }
-      if (j >= n_out) tok = -1;
-      p.out_tokens[b * k1 + j] = tok;
+  __syncthreads();
+  if (threadIdx.x < k1) {
+    const int j = threadIdx.x;
+    int tok = (j < i_star) ? p.cand[b * p.k + j] : (j == i_star ? sh_bonus : -1);
+    // <EOS>: keep the tokens before the first one
+    const bool is_eos = p.eos_id >= 0 && j <= i_star && tok == p.eos_id;
+    const unsigned eos_mask = __ballot_sync((1u << k1) - 1u, is_eos);
+    const int first = eos_mask ? __ffs(eos_mask) - 1 : k1;
+    const int n_out = eos_mask ? first : i_star + 1;
+    p.out_tokens[b * k1 + j] = (j < n_out) ? tok : -1;
+    if (j == 0) {
+      p.n_out[b] = n_out;
+      p.finished[b] = (uint8_t)(eos_mask != 0);
     }
-    p.n_out[b] = n_out;
-    p.finished[b] = (uint8_t)fin;
   }
 }
 

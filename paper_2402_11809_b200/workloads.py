@@ -100,11 +100,11 @@ def make_step_inputs(cfg, set_index=0, s_cap=None, poison_tail=False):
     planted = rng.uniform(size=(B, k)) < p_seq[:, None]
     plant = PLANT_GREEDY if cfg["mode"] == "greedy" else PLANT_SAMPLE
     plant_val = np.float32(plant) if logits.dtype == np.float32 \
-        else f32_to_bf16_bits(np.float32(plant))
+        else f32_to_bf16_bits(np.array([plant], dtype=np.float32))[0]
     for b in range(B):
         for i in range(k):
             if planted[b, i]:
-                logits[b, i * (k + 1), cand[b, i]] = plant_val   # target row of c_{i+1}
+                logits[b, i * (k + 1), int(cand[b, i])] = plant_val   # target row of c_{i+1}
     cand_prob = np.ones((B, k), dtype=np.float32)
     seq_id = np.arange(B, dtype=np.uint32)
     return dict(q=q, k_cache=k_cache, v_cache=v_cache, kv_len=kv_len, logits=logits,
