@@ -5,16 +5,19 @@
 // and every thread-block group takes an equal contiguous share of it, so ragged
 // batches balance without host knowledge of the lengths.  A share that does not
 // cover a whole (sequence, head) leaves an unnormalised partial (running max,
-// sum, accumulator) in scratch memory; attn_merge_kernel combines partials.
+// sum, accumulator) in scratch memory; the last group to finish a (sequence,
+// head) combines its partials (arrival counter, reset by the last arriver).
 //
-// Inside a block (7 warps):
-//   warp 0  streams K and V tiles with TMA into a ring of shared-memory stages
-//   warp 6  loads the query rows of the current share with TMA
+// Inside a block (12 warps):
+//   warps 0, 2  stream K and V tiles with TMA into two rings of shared-memory
+//           stages (a K stage is free once Q K^T has read it, a V stage once P V has)
+//   warp 3  loads the query rows of the current share with TMA
 //   warp 1  issues tcgen05.mma: S = Q K^T into one of two TMEM buffers, then
 //           O += P V with P read back from TMEM
-//   warps 2-5  one thread per query row: read S from TMEM, apply the Eq. 5 mask
-//           on tiles that touch the block or a share boundary, running max with
-//           lazy rescaling of O, P = exp2(...) as bf16 into TMEM
+//   warps 4-11  two threads per query row, 64 keys of the tile each: read S
+//           from TMEM, apply the Eq. 5 mask on tiles that touch the block or a
+//           share boundary, running max with lazy rescaling of O, P = exp2(...)
+//           as two bf16 terms into TMEM
 // The 128 MMA rows are (block row i, head-in-group g) pairs of one kv head, so a
 // GQA group shares each K/V tile.  Every wait is bounded; an expired wait sets
 // SPACE_ST_TIMEOUT and the block drains and exits.
@@ -26,7 +29,7 @@ namespace {
 
 constexpr int TILE_N = 128;            // keys per tile
 constexpr int ROWS = 128;              // MMA M
-constexpr int THREADS = 224;
+constexpr int THREADS = 384;            // K, MMA, V, Q warps + 8 softmax warps
 constexpr uint64_t WAIT_NS = 1000000000ull;   // one second per wait
 constexpr float RESCALE_THRESHOLD = 8.f;
 
@@ -42,6 +45,7 @@ struct AttnParams {
   void* out; float* lse; int32_t* status;
   float* part;                         // [slots][ROWS*(DH+2)]
   int* err;                            // one word: first timeout site
+  int* merge_cnt;                      // [B*H_kv*n_mblocks] arrivals per split (sequence, head, row block)
   uint64_t mask[SPACE_MAX_ROWS];
 };
 
@@ -174,104 +178,141 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, int b_mn_major) {
 }
 
 // ------------------------------------------------------------ work partition
-// Flat tile index space: sequence-major, then kv head, then tile.
+// Flat tile index space: sequence-major, then kv head, then tile.  Group g of
+// n_groups owns flat tiles [W*g/n_groups, W*(g+1)/n_groups).
 struct Partition {
-  const int* tiles;      // [B]   tiles per (sequence, head)
+  const int* seq_len;    // [B]   verified length, or -1 for a sequence that does not fit
   const int* prefix;     // [B+1] flat offset of sequence b
-  int B, H_kv;
+  int B, H_kv, n_q;
   long long cur, end;
   int b;
-  __device__ void init(const int* t, const int* pf, int B_, int H, int group, int n_groups) {
-    tiles = t; prefix = pf; B = B_; H_kv = H; b = 0;
+  __device__ void init(const int* sl, const int* pf, int B_, int H, int nq, int group, int n_groups) {
+    seq_len = sl; prefix = pf; B = B_; H_kv = H; n_q = nq; b = 0;
     const long long W = pf[B_];
     cur = (W * group) / n_groups;
     end = (W * (group + 1)) / n_groups;
   }
-  __device__ bool next(Seg& s, const int32_t* kv_len) {
+  __device__ bool next(Seg& s) {
     if (cur >= end) return false;
     while (prefix[b + 1] <= cur) ++b;
-    const int T = tiles[b];
+    const int L = seq_len[b];
+    const int T = (L + n_q + TILE_N - 1) / TILE_N;
     const int rem = (int)(cur - prefix[b]);
-    s.b = b; s.h = rem / T; s.t0 = rem % T; s.T = T;
+    s.b = b; s.h = rem / T; s.t0 = rem % T; s.T = T; s.L = L;
     long long n = T - s.t0;
     if (n > end - cur) n = end - cur;
     s.t1 = s.t0 + (int)n;
-    s.L = kv_len[b];
     cur += n;
     return true;
   }
 };
+
+// group that owns flat tile f (largest g with W*g/NG <= f)
+__device__ __forceinline__ int group_of(long long f, long long W, long long NG) {
+  return (int)(((f + 1) * NG - 1) / W);
+}
 
 template <int DH>
 struct Smem {
   static constexpr int HALVES = DH / 64;
   static constexpr int TILE_BYTES = TILE_N * DH * 2;         // one K or V tile
   static constexpr int Q_BYTES = ROWS * DH * 2;
-  static constexpr int STAGES = (DH == 128) ? 3 : 4;
+  static constexpr int K_STAGES = (DH == 128) ? 2 : 3;
+  static constexpr int V_STAGES = (DH == 128) ? 3 : 4;
   static constexpr int Q_OFF = 0;
-  static constexpr int KV_OFF = Q_BYTES;
-  static constexpr int BAR_OFF = KV_OFF + STAGES * 2 * TILE_BYTES;
-  // barriers: q_full, q_empty, k_full[S], v_full[S], kv_empty[S], s_full[2], p_ready[2], pv_done[2], drain
-  static constexpr int N_BARS = 2 + 3 * STAGES + 6 + 1;
-  static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;      // tmem base, abort flag
-  static constexpr int TABLE_OFF = MISC_OFF + 16;
+  static constexpr int K_OFF = Q_BYTES;
+  static constexpr int V_OFF = K_OFF + K_STAGES * TILE_BYTES;
+  static constexpr int BAR_OFF = V_OFF + V_STAGES * TILE_BYTES;
+  // q_full, q_empty, k_full[], k_empty[], v_full[], v_empty[], s_full[2], p_ready[2], pv_done[2], drain,
+  // pair[4] (the two threads of a row meet), all_soft
+  static constexpr int N_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 6 + 1 + 4 + 1;
+  static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;      // tmem base, abort flag, merge flag, merge count
+  static constexpr int XMAX_OFF = MISC_OFF + 32;             // [2 parities][2 halves][ROWS] float
+  static constexpr int XSUM_OFF = XMAX_OFF + 2 * 2 * ROWS * 4;   // [2 halves][ROWS] float
+  static constexpr int MLIST_OFF = XSUM_OFF + 2 * ROWS * 4;  // [256] short: groups to merge
+  static constexpr int TABLE_OFF = MLIST_OFF + 512;          // seq_len[max_batch], prefix[max_batch+1]
 };
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Warp roles
+constexpr int WARP_K = 0, WARP_MMA = 1, WARP_V = 2, WARP_Q = 3, WARP_SOFTMAX0 = 4;
 
 template <int DH>
 __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_constant__ AttnParams p,
                                                              int max_batch) {
   using S = Smem<DH>;
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char* sm = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) unsigned char sm[];
   const uint32_t sm_base = smem_u32(sm);
   const uint32_t bar0 = sm_base + S::BAR_OFF;
   auto BAR = [&](int i) { return bar0 + 8u * i; };
-  const int B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_VFULL = 2 + S::STAGES, B_KVEMPTY = 2 + 2 * S::STAGES,
-            B_SFULL = 2 + 3 * S::STAGES, B_PREADY = B_SFULL + 2, B_PVDONE = B_SFULL + 4, B_DRAIN = B_SFULL + 6;
+  constexpr int B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = B_KFULL + S::K_STAGES,
+                B_VFULL = B_KEMPTY + S::K_STAGES, B_VEMPTY = B_VFULL + S::V_STAGES,
+                B_SFULL = B_VEMPTY + S::V_STAGES, B_PREADY = B_SFULL + 2, B_PVDONE = B_SFULL + 4,
+                B_DRAIN = B_SFULL + 6, B_PAIR = B_DRAIN + 1, B_ALL = B_PAIR + 4;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + S::MISC_OFF);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 4);
-  int* tiles = reinterpret_cast<int*>(sm + S::TABLE_OFF);
-  int* prefix = tiles + max_batch;
+  volatile int* merge_flag = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 8);
+  volatile int* merge_n = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 12);
+  float* xmax = reinterpret_cast<float*>(sm + S::XMAX_OFF);
+  float* xsum = reinterpret_cast<float*>(sm + S::XSUM_OFF);
+  short* mlist = reinterpret_cast<short*>(sm + S::MLIST_OFF);
+  int* seq_len = reinterpret_cast<int*>(sm + S::TABLE_OFF);
+  int* prefix = seq_len + max_batch;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int group = blockIdx.x / p.n_mblocks, mb = blockIdx.x % p.n_mblocks;
   const int i0 = mb * p.rows_per_mb;                       // first block row of this query-row block
+  // MMA rows that carry a real (block row, head) pair are 0 .. m_valid-1
+  const int m_valid = min(p.rows_per_mb, p.n_q - i0) * p.G;
+  const int n_quarters = (m_valid + 31) >> 5;              // TMEM lane quarters with live rows
+  const int n_soft = 64 * n_quarters;                      // softmax threads that take part
 
   // ---- set-up ------------------------------------------------------------
   if (threadIdx.x == 0) {
-    *abort_flag = 0;
+    *abort_flag = (sm_base & 1023u) ? 1 : 0;               // swizzled tiles need a 1024-byte aligned base
+    if (*abort_flag) atomicCAS(p.err, 0, 99);
+    *merge_flag = 0;
     long long acc = 0;
     for (int b = 0; b < p.B; ++b) {
       const int L = p.kv_len[b];
       const bool ok = L >= 0 && (int64_t)L + p.n_q <= p.s_cap;
-      const int T = ok ? (L + p.n_q + TILE_N - 1) / TILE_N : 0;
       if (!ok && blockIdx.x == 0 && p.status) atomicOr(p.status + b, SPACE_ST_CAPACITY);
-      tiles[b] = T;
+      seq_len[b] = ok ? L : -1;
       prefix[b] = (int)acc;
-      acc += (long long)T * p.H_kv;
+      if (ok) acc += (long long)((L + p.n_q + TILE_N - 1) / TILE_N) * p.H_kv;
     }
     prefix[p.B] = (int)acc;
     mbar_init(BAR(B_QFULL), 1);
     mbar_init(BAR(B_QEMPTY), 1);
-    for (int s = 0; s < S::STAGES; ++s) {
-      mbar_init(BAR(B_KFULL + s), 1);
-      mbar_init(BAR(B_VFULL + s), 1);
-      mbar_init(BAR(B_KVEMPTY + s), 1);
-    }
+    for (int s = 0; s < S::K_STAGES; ++s) { mbar_init(BAR(B_KFULL + s), 1); mbar_init(BAR(B_KEMPTY + s), 1); }
+    for (int s = 0; s < S::V_STAGES; ++s) { mbar_init(BAR(B_VFULL + s), 1); mbar_init(BAR(B_VEMPTY + s), 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(BAR(B_SFULL + i), 1);
-      mbar_init(BAR(B_PREADY + i), 128);
+      mbar_init(BAR(B_PREADY + i), n_soft);
       mbar_init(BAR(B_PVDONE + i), 1);
     }
     mbar_init(BAR(B_DRAIN), 1);
+    for (int q = 0; q < 4; ++q) mbar_init(BAR(B_PAIR + q), 64);
+    mbar_init(BAR(B_ALL), n_soft);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {
+  if (warp == WARP_MMA) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  if (warp == WARP_K && lane == 0)
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_k) : "memory");
+  if (warp == WARP_V && lane == 0)
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_v) : "memory");
+  if (warp == WARP_Q && lane == 0)
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_q) : "memory");
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -279,52 +320,53 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   const uint32_t TM_S0 = tmem, TM_O = tmem + 2 * TILE_N;    // S buffers at columns 0 and 128, O at 256
 
   Partition part;
-  part.init(tiles, prefix, p.B, p.H_kv, group, p.n_groups);
+  part.init(seq_len, prefix, p.B, p.H_kv, p.n_q, group, p.n_groups);
   Seg sg;
+  const bool dead = *abort_flag != 0;
 
-  if (warp == 0) {
-    // ================= K/V producer =======================================
+  if (dead) {
+    // nothing was issued; fall through to the teardown
+  } else if (warp == WARP_K || warp == WARP_V) {
+    // ================= K / V producers ====================================
     if (lane == 0) {
+      const bool is_k = warp == WARP_K;
+      const int n_st = is_k ? S::K_STAGES : S::V_STAGES;
+      const int b_full = is_k ? B_KFULL : B_VFULL, b_empty = is_k ? B_KEMPTY : B_VEMPTY;
+      const uint32_t ring = sm_base + (is_k ? S::K_OFF : S::V_OFF);
+      const CUtensorMap* tm = is_k ? &p.tm_k : &p.tm_v;
       uint32_t gt = 0;
       bool ok = true;
-      while (ok && part.next(sg, p.kv_len)) {
+      while (ok && part.next(sg)) {
         const int n_keys = sg.L + p.n_q;
         for (int t = sg.t0; t < sg.t1 && ok; ++t, ++gt) {
-          const int s = gt % S::STAGES;
-          if (gt >= (uint32_t)S::STAGES)
-            ok = mbar_wait(BAR(B_KVEMPTY + s), ((gt / S::STAGES) - 1) & 1, abort_flag, p.err, 1);
+          const int s = gt % n_st;
+          if (gt >= (uint32_t)n_st)
+            ok = mbar_wait(BAR(b_empty + s), ((gt / n_st) - 1) & 1, abort_flag, p.err, is_k ? 1 : 2);
           if (!ok) break;
           // the last tile of a sequence is shifted back so that it ends at the
           // last key: rows past the end are never read (they may hold anything)
           const int kt = ((t + 1) * TILE_N <= n_keys) ? t * TILE_N : n_keys - TILE_N;
-          const uint32_t kdst = sm_base + S::KV_OFF + s * 2 * S::TILE_BYTES;
-          const uint32_t vdst = kdst + S::TILE_BYTES;
-          mbar_expect_tx(BAR(B_KFULL + s), S::TILE_BYTES);
+          const uint32_t dst = ring + s * S::TILE_BYTES;
+          mbar_expect_tx(BAR(b_full + s), S::TILE_BYTES);
+#pragma unroll
           for (int hf = 0; hf < S::HALVES; ++hf)
-            tma_load_4d(kdst + hf * (TILE_N * 128), &p.tm_k, BAR(B_KFULL + s), hf * 64, kt, sg.h, sg.b);
-          mbar_expect_tx(BAR(B_VFULL + s), S::TILE_BYTES);
-          for (int hf = 0; hf < S::HALVES; ++hf)
-            tma_load_4d(vdst + hf * (TILE_N * 128), &p.tm_v, BAR(B_VFULL + s), hf * 64, kt, sg.h, sg.b);
+            tma_load_4d(dst + hf * (TILE_N * 128), tm, BAR(b_full + s), hf * 64, kt, sg.h, sg.b);
         }
       }
       // drain: every issued copy must have landed before the block may exit
-      const uint32_t first = gt > (uint32_t)S::STAGES ? gt - S::STAGES : 0;
-      for (uint32_t g = first; g < gt; ++g) {
-        const int s = g % S::STAGES;
-        const uint32_t par = (g / S::STAGES) & 1;
-        mbar_drain(BAR(B_KFULL + s), par);
-        mbar_drain(BAR(B_VFULL + s), par);
-      }
+      const uint32_t first = gt > (uint32_t)n_st ? gt - n_st : 0;
+      for (uint32_t g = first; g < gt; ++g) mbar_drain(BAR(b_full + g % n_st), (g / n_st) & 1);
     }
-  } else if (warp == 6) {
+  } else if (warp == WARP_Q) {
     // ================= Q producer =========================================
     if (lane == 0) {
       uint32_t seg = 0;
       bool ok = true;
-      while (ok && part.next(sg, p.kv_len)) {
-        if (seg > 0) ok = mbar_wait(BAR(B_QEMPTY), (seg - 1) & 1, abort_flag, p.err, 2);
+      while (ok && part.next(sg)) {
+        if (seg > 0) ok = mbar_wait(BAR(B_QEMPTY), (seg - 1) & 1, abort_flag, p.err, 3);
         if (!ok) break;
         mbar_expect_tx(BAR(B_QFULL), S::Q_BYTES);
+#pragma unroll
         for (int hf = 0; hf < S::HALVES; ++hf)
           tma_load_4d(sm_base + S::Q_OFF + hf * (ROWS * 128), &p.tm_q, BAR(B_QFULL), hf * 64,
                       sg.h * p.G, i0, sg.b);
@@ -332,20 +374,20 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       }
       if (seg > 0) mbar_drain(BAR(B_QFULL), (seg - 1) & 1);
     }
-  } else if (warp == 1) {
+  } else if (warp == WARP_MMA) {
     // ================= MMA issuer =========================================
     if (lane == 0) {
       constexpr uint32_t IDESC_QK = instr_desc(TILE_N, 0);
       constexpr uint32_t IDESC_PV = instr_desc(DH, 1);
       uint32_t gt = 0, seg = 0;
       bool ok = true;
-      // O += P V for flat tile g (first_in_seg: overwrite O)
+      // O += (P_hi + P_lo) V for flat tile g (first_in_seg: overwrite O)
       auto issue_pv = [&](uint32_t g, bool first_in_seg) -> bool {
-        const int s = g % S::STAGES, buf = g & 1;
-        if (!mbar_wait(BAR(B_VFULL + s), (g / S::STAGES) & 1, abort_flag, p.err, 3)) return false;
-        if (!mbar_wait(BAR(B_PREADY + buf), (g >> 1) & 1, abort_flag, p.err, 4)) return false;
+        const int s = g % S::V_STAGES, buf = g & 1;
+        if (!mbar_wait(BAR(B_VFULL + s), (g / S::V_STAGES) & 1, abort_flag, p.err, 4)) return false;
+        if (!mbar_wait(BAR(B_PREADY + buf), (g >> 1) & 1, abort_flag, p.err, 5)) return false;
         tc_fence_after();
-        const uint32_t vsm = sm_base + S::KV_OFF + s * 2 * S::TILE_BYTES + S::TILE_BYTES;
+        const uint32_t vsm = sm_base + S::V_OFF + s * S::TILE_BYTES;
         const uint32_t ptm = TM_S0 + buf * TILE_N;
 #pragma unroll
         for (int part_i = 0; part_i < 2; ++part_i) {        // P_hi, then P_lo
@@ -357,21 +399,21 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
                    (first_in_seg && kk == 0 && part_i == 0) ? 0u : 1u);
           }
         }
-        tc_commit(BAR(B_KVEMPTY + s));
+        tc_commit(BAR(B_VEMPTY + s));
         tc_commit(BAR(B_PVDONE + buf));
         return true;
       };
-      while (ok && part.next(sg, p.kv_len)) {
-        ok = mbar_wait(BAR(B_QFULL), seg & 1, abort_flag, p.err, 5);
+      while (ok && part.next(sg)) {
+        ok = mbar_wait(BAR(B_QFULL), seg & 1, abort_flag, p.err, 6);
         const int n = sg.t1 - sg.t0;
         for (int j = 0; j < n && ok; ++j, ++gt) {
-          const int s = gt % S::STAGES, buf = gt & 1;
-          ok = mbar_wait(BAR(B_KFULL + s), (gt / S::STAGES) & 1, abort_flag, p.err, 6);
-          if (ok && gt >= 2) ok = mbar_wait(BAR(B_PVDONE + buf), ((gt >> 1) - 1) & 1, abort_flag, p.err, 7);
+          const int s = gt % S::K_STAGES, buf = gt & 1;
+          ok = mbar_wait(BAR(B_KFULL + s), (gt / S::K_STAGES) & 1, abort_flag, p.err, 7);
+          if (ok && gt >= 2) ok = mbar_wait(BAR(B_PVDONE + buf), ((gt >> 1) - 1) & 1, abort_flag, p.err, 8);
           if (!ok) break;
           tc_fence_after();
           const uint32_t qsm = sm_base + S::Q_OFF;
-          const uint32_t ksm = sm_base + S::KV_OFF + s * 2 * S::TILE_BYTES;
+          const uint32_t ksm = sm_base + S::K_OFF + s * S::TILE_BYTES;
 #pragma unroll
           for (int kk = 0; kk < DH / 16; ++kk) {
             const uint32_t off = (kk >> 2) * (ROWS * 128) + (kk & 3) * 32;   // 64-wide half, then 32 B per 16 elements
@@ -379,6 +421,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
                    IDESC_QK, kk > 0 ? 1u : 0u);
           }
           tc_commit(BAR(B_SFULL + buf));
+          tc_commit(BAR(B_KEMPTY + s));
           if (j == n - 1) tc_commit(BAR(B_QEMPTY));
           if (j > 0) ok = issue_pv(gt - 1, j == 1);
         }
@@ -389,30 +432,44 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       tc_commit(BAR(B_DRAIN));
       mbar_drain(BAR(B_DRAIN), 0);
     }
-  } else {
-    // ================= softmax / epilogue: one thread per query row ========
+  } else if ((warp & 3) < n_quarters) {
+    // ================= softmax / epilogue ==================================
+    // Two threads per query row: `half` picks which 64 keys of a tile (and which
+    // half of the head dimension in the epilogue) this thread handles.
     const int quarter = warp & 3;                          // TMEM lane quarter this warp may touch
+    const int half = (warp - WARP_SOFTMAX0) >> 2;
     const int m = quarter * 32 + lane;                     // MMA row
     const int il = m / p.G, g = m % p.G;
     const int i = i0 + il;                                 // block row
-    const bool row_valid = il < p.rows_per_mb && i < p.n_q;
+    const bool row_valid = m < m_valid;
     const uint64_t mrow = row_valid ? p.mask[i] : 0ull;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const int sidx = half * (32 * n_quarters) + m;          // index among the n_soft softmax threads
     const float c = p.scale_log2;
-    uint32_t gt = 0;
+    constexpr int HC = TILE_N / 2;                         // keys per thread and tile
+    constexpr int OC = DH / 2;                             // output columns per thread
+    uint32_t gt = 0, pair_ph = 0, all_ph = 0;
     bool ok = true;
-    while (ok && part.next(sg, p.kv_len)) {
+    // Rendezvous on an mbarrier (bounded, unlike bar.sync): the two threads of a
+    // row, or all softmax threads.  Shared-memory writes before it are visible after.
+    auto meet = [&](int bar, uint32_t& ph, int site) -> bool {
+      mbar_arrive(BAR(bar));
+      const bool r = mbar_wait(BAR(bar), ph & 1, abort_flag, p.err, site);
+      ++ph;
+      return r;
+    };
+    while (ok && part.next(sg)) {
       const int n_keys = sg.L + p.n_q;
       float m_ref = -CUDART_INF_F, l_sum = 0.f;
       for (int t = sg.t0; t < sg.t1 && ok; ++t, ++gt) {
         const int buf = gt & 1;
-        ok = mbar_wait(BAR(B_SFULL + buf), (gt >> 1) & 1, abort_flag, p.err, 8);
+        ok = mbar_wait(BAR(B_SFULL + buf), (gt >> 1) & 1, abort_flag, p.err, 9);
         if (!ok) break;
         tc_fence_after();
         const uint32_t ts = TM_S0 + buf * TILE_N + lane_addr;
-        uint32_t sreg[TILE_N];
+        uint32_t sreg[HC];
 #pragma unroll
-        for (int cc = 0; cc < TILE_N / 32; ++cc) tmem_ld32(ts + cc * 32, sreg + cc * 32);
+        for (int cc = 0; cc < HC / 32; ++cc) tmem_ld32(ts + half * HC + cc * 32, sreg + cc * 32);
         tmem_wait_ld();
         const int lo = t * TILE_N;
         const int kt = ((t + 1) * TILE_N <= n_keys) ? lo : n_keys - TILE_N;
@@ -420,8 +477,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         float tmax = -CUDART_INF_F;
         if (masked) {
 #pragma unroll
-          for (int cidx = 0; cidx < TILE_N; ++cidx) {
-            const int key = kt + cidx;
+          for (int cidx = 0; cidx < HC; ++cidx) {
+            const int key = kt + half * HC + cidx;
             bool vis = key >= lo;
             if (key >= sg.L) vis = vis && ((mrow >> ((key - sg.L) & 63)) & 1ull);
             const float v = vis ? __uint_as_float(sreg[cidx]) : -CUDART_INF_F;
@@ -430,75 +487,86 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           }
         } else {
 #pragma unroll
-          for (int cidx = 0; cidx < TILE_N; ++cidx) tmax = fmaxf(tmax, __uint_as_float(sreg[cidx]));
+          for (int cidx = 0; cidx < HC; ++cidx) tmax = fmaxf(tmax, __uint_as_float(sreg[cidx]));
         }
+        // the row maximum needs the other half's keys; the pair barrier also orders
+        // both threads' reads of S before either overwrites it with P
+        float* xm = xmax + (gt & 1) * (2 * ROWS);
+        xm[half * ROWS + m] = tmax;
+        ok = meet(B_PAIR + quarter, pair_ph, 12);
+        if (!ok) break;
+        tmax = fmaxf(tmax, xm[(half ^ 1) * ROWS + m]);
         tmax *= c;                                         // c > 0
         if (!(tmax > -CUDART_INF_F)) tmax = -CUDART_INF_F; // also catches NaN
         const bool first = (t == sg.t0);
-        bool need = !first && (tmax > m_ref + RESCALE_THRESHOLD);
+        const bool need = !first && (tmax > m_ref + RESCALE_THRESHOLD);
         if (first) m_ref = tmax;
         if (__any_sync(0xFFFFFFFFu, need)) {
           // lazy rescale of this row's accumulator; PV of the previous tile must be done
-          ok = mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 9);
+          ok = mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 10);
           if (!ok) break;
           tc_fence_after();
           const float m_new = fmaxf(m_ref, tmax);
-          const float f = (m_ref > -CUDART_INF_F) ? exp2f(m_ref - m_new) : 0.f;
+          const float f = (m_ref > -CUDART_INF_F) ? fast_exp2(m_ref - m_new) : 0.f;
           l_sum *= f;
           m_ref = m_new;
 #pragma unroll 1
-          for (int cc = 0; cc < DH / 32; ++cc) {
+          for (int cc = 0; cc < OC / 32; ++cc) {
             uint32_t o[32];
-            tmem_ld32(TM_O + lane_addr + cc * 32, o);
+            const uint32_t ta = TM_O + lane_addr + half * OC + cc * 32;
+            tmem_ld32(ta, o);
             tmem_wait_ld();
 #pragma unroll
             for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * f);
-            tmem_st32(TM_O + lane_addr + cc * 32, o);
+            tmem_st32(ta, o);
           }
           tmem_wait_st();
         }
         const float m_use = (m_ref > -CUDART_INF_F) ? m_ref : 0.f;
         // P = P_hi + P_lo, two bf16 terms: bf16 alone (8 significant bits) leaves
-        // an output error near 1e-2 of the output RMS.  P_hi goes to columns
-        // 0..63 of the S buffer, P_lo to columns 64..127.
-        uint32_t lreg[TILE_N / 2];
+        // an output error near 1e-2 of the output RMS.  P_hi occupies columns
+        // 0..63 of the S buffer, P_lo columns 64..127 (two keys per column).
+        uint32_t lreg[HC / 2];
 #pragma unroll
-        for (int x = 0; x < TILE_N / 2; ++x) {
-          const float p0 = exp2f(fmaf(__uint_as_float(sreg[2 * x]), c, -m_use));
-          const float p1 = exp2f(fmaf(__uint_as_float(sreg[2 * x + 1]), c, -m_use));
+        for (int x = 0; x < HC / 2; ++x) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[2 * x]), c, -m_use));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[2 * x + 1]), c, -m_use));
           l_sum += p0 + p1;
           const __nv_bfloat162 hi = __floats2bfloat162_rn(p0, p1);   // .x (low half) = even key
           const float2 hf = __bfloat1622float2(hi);
-          const __nv_bfloat162 lo = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
+          const __nv_bfloat162 lw = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
           sreg[x] = *reinterpret_cast<const uint32_t*>(&hi);
-          lreg[x] = *reinterpret_cast<const uint32_t*>(&lo);
+          lreg[x] = *reinterpret_cast<const uint32_t*>(&lw);
         }
-#pragma unroll
-        for (int cc = 0; cc < TILE_N / 64; ++cc) {
-          tmem_st32(ts + cc * 32, sreg + cc * 32);
-          tmem_st32(ts + TILE_N / 2 + cc * 32, lreg + cc * 32);
-        }
+        tmem_st32(ts + half * (HC / 2), sreg);
+        tmem_st32(ts + TILE_N / 2 + half * (HC / 2), lreg);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(BAR(B_PREADY + buf));
       }
       if (!ok) break;
       // ---- end of share: final output or partial ---------------------------
-      ok = mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 10);
+      ok = mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 11);
       if (!ok) break;
       tc_fence_after();
+      xsum[half * ROWS + m] = l_sum;
+      ok = meet(B_PAIR + quarter, pair_ph, 13);
+      if (!ok) break;
+      const float l_tot = l_sum + xsum[(half ^ 1) * ROWS + m];
       const bool whole = (sg.t0 == 0 && sg.t1 == sg.T);
       const int hq = sg.h * p.G + g;
-      float* pslot = p.part + ((size_t)((sg.b * p.H_kv + sg.h) + group) * p.n_mblocks + mb) * (ROWS * (DH + 2));
-      const float inv = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
+      const int item = sg.b * p.H_kv + sg.h;
+      float* pslot = p.part + ((size_t)(item + group) * p.n_mblocks + mb) * (ROWS * (DH + 2));
+      const float inv = (l_tot > 0.f) ? 1.f / l_tot : 0.f;
 #pragma unroll 1
-      for (int cc = 0; cc < DH / 32; ++cc) {
+      for (int cc = 0; cc < OC / 32; ++cc) {
         uint32_t o[32];
-        tmem_ld32(TM_O + lane_addr + cc * 32, o);
+        const int col = half * OC + cc * 32;
+        tmem_ld32(TM_O + lane_addr + col, o);
         tmem_wait_ld();
         if (!row_valid) continue;
         if (whole) {
-          const size_t off = (((size_t)sg.b * p.n_q + i) * p.H_q + hq) * DH + cc * 32;
+          const size_t off = (((size_t)sg.b * p.n_q + i) * p.H_q + hq) * DH + col;
           if (p.out_dtype == SPACE_DTYPE_F32) {
             float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off);
 #pragma unroll
@@ -520,98 +588,100 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
             }
           }
         } else {
-          float4* dst = reinterpret_cast<float4*>(pslot + (size_t)m * DH + cc * 32);
+          float4* dst = reinterpret_cast<float4*>(pslot + (size_t)m * DH + col);
 #pragma unroll
           for (int x = 0; x < 8; ++x)
-            dst[x] = make_float4(__uint_as_float(o[4 * x]), __uint_as_float(o[4 * x + 1]),
-                                 __uint_as_float(o[4 * x + 2]), __uint_as_float(o[4 * x + 3]));
-        }
-      }
-      if (row_valid) {
-        if (whole) {
-          if (p.lse)
-            p.lse[((size_t)sg.b * p.H_q + hq) * p.n_q + i] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
-        } else {
-          pslot[ROWS * DH + m] = m_ref;
-          pslot[ROWS * DH + ROWS + m] = l_sum;
+            __stcg(dst + x, make_float4(__uint_as_float(o[4 * x]), __uint_as_float(o[4 * x + 1]),
+                                        __uint_as_float(o[4 * x + 2]), __uint_as_float(o[4 * x + 3])));
         }
       }
       tc_fence_before();
+      if (whole) {
+        if (row_valid && half == 0 && p.lse)
+          p.lse[((size_t)sg.b * p.H_q + hq) * p.n_q + i] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
+        continue;
+      }
+      if (row_valid && half == 0) {
+        __stcg(pslot + ROWS * DH + m, m_ref);
+        __stcg(pslot + ROWS * DH + ROWS + m, l_tot);
+      }
+      // ---- partial: the last group to finish a (sequence, head) merges it ----
+      __threadfence();
+      ok = meet(B_ALL, all_ph, 14);
+      if (!ok) break;
+      if (sidx == 0) {
+        const long long W = prefix[p.B], NG = p.n_groups;
+        const long long f0 = (long long)prefix[sg.b] + (long long)sg.h * sg.T;
+        int n = 0;
+        if (W >= NG) {                                     // every group holds tiles
+          const int g0 = group_of(f0, W, NG), g1 = group_of(f0 + sg.T - 1, W, NG);
+          for (int gi = g0; gi <= g1 && n < 256; ++gi) mlist[n++] = (short)gi;
+        } else {                                           // one tile per non-empty group
+          for (int t = 0; t < sg.T && n < 256; ++t) mlist[n++] = (short)group_of(f0 + t, W, NG);
+        }
+        int* cnt = p.merge_cnt + (size_t)item * p.n_mblocks + mb;
+        const int prev = atomicAdd(cnt, 1);
+        const int last = (prev == n - 1);
+        if (last) *cnt = 0;                                // ready for the next launch
+        *merge_n = n;
+        *merge_flag = last;
+      }
+      ok = meet(B_ALL, all_ph, 15);
+      if (!ok) break;
+      if (*merge_flag) {
+        __threadfence();
+        const int n = *merge_n;
+        constexpr int C4 = DH / 4;
+        const size_t slot_floats = (size_t)ROWS * (DH + 2);
+        const float* pbase = p.part + ((size_t)item * p.n_mblocks + mb) * slot_floats;
+        const size_t gstride = (size_t)p.n_mblocks * slot_floats;
+        for (int idx = sidx; idx < m_valid * C4; idx += n_soft) {
+          const int r = idx / C4, c4 = idx % C4;
+          float mx = -CUDART_INF_F;
+#pragma unroll 4
+          for (int x = 0; x < n; ++x) mx = fmaxf(mx, __ldcg(pbase + mlist[x] * gstride + ROWS * DH + r));
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          float den = 0.f;
+#pragma unroll 4
+          for (int x = 0; x < n; ++x) {
+            const float* ps = pbase + mlist[x] * gstride;
+            const float ms = __ldcg(ps + ROWS * DH + r);
+            const float ls = __ldcg(ps + ROWS * DH + ROWS + r);
+            const float4 ov = __ldcg(reinterpret_cast<const float4*>(ps + (size_t)r * DH) + c4);
+            const float w = (ms > -CUDART_INF_F) ? fast_exp2(ms - mx) : 0.f;
+            den = fmaf(w, ls, den);
+            acc.x = fmaf(w, ov.x, acc.x); acc.y = fmaf(w, ov.y, acc.y);
+            acc.z = fmaf(w, ov.z, acc.z); acc.w = fmaf(w, ov.w, acc.w);
+          }
+          const float rinv = 1.f / den;
+          const int ri = i0 + r / p.G, rhq = sg.h * p.G + r % p.G;
+          const size_t off = (((size_t)sg.b * p.n_q + ri) * p.H_q + rhq) * DH + c4 * 4;
+          if (p.out_dtype == SPACE_DTYPE_F32) {
+            *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off) =
+                make_float4(acc.x * rinv, acc.y * rinv, acc.z * rinv, acc.w * rinv);
+          } else {
+            const __nv_bfloat162 a = __floats2bfloat162_rn(acc.x * rinv, acc.y * rinv);
+            const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc.z * rinv, acc.w * rinv);
+            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off) =
+                make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b2));
+          }
+          if (p.lse && c4 == 0)
+            p.lse[((size_t)sg.b * p.H_q + rhq) * p.n_q + ri] = (mx + log2f(den)) * 0.6931471805599453f;
+        }
+        ok = meet(B_ALL, all_ph, 16);                      // merge_flag / mlist are reused by the next share
+      }
     }
   }
 
   // ---- teardown -----------------------------------------------------------
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == WARP_MMA) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
   }
   if (threadIdx.x == 0 && *abort_flag && p.status) {
     for (int b = 0; b < p.B; ++b) atomicOr(p.status + b, SPACE_ST_TIMEOUT);
-  }
-}
-
-// Combine the partials of every (sequence, kv head, query-row block) that was
-// split over several thread-block groups.  grid = (B*H_kv*n_mblocks, row chunks).
-template <int DH>
-__global__ void __launch_bounds__(DH) attn_merge_kernel(const AttnParams p, int rows_per_block) {
-  const int item = blockIdx.x / p.n_mblocks, mb = blockIdx.x % p.n_mblocks;
-  const int b = item / p.H_kv, h = item % p.H_kv;
-  const int L = p.kv_len[b];
-  if (L < 0 || (int64_t)L + p.n_q > p.s_cap) return;
-  // recompute the partition (same arithmetic as the main kernel)
-  long long f0 = 0, W = 0;
-  for (int bb = 0; bb < p.B; ++bb) {
-    const int LL = p.kv_len[bb];
-    const bool ok = LL >= 0 && (int64_t)LL + p.n_q <= p.s_cap;
-    const long long T = ok ? (LL + p.n_q + TILE_N - 1) / TILE_N : 0;
-    if (bb < b) f0 += T * p.H_kv;
-    W += T * p.H_kv;
-  }
-  const int T = (L + p.n_q + TILE_N - 1) / TILE_N;
-  f0 += (long long)h * T;
-  const long long NG = p.n_groups;
-  const int g_first = (int)(((f0 + 1) * NG - 1) / W);
-  const int g_last = (int)(((f0 + T) * NG - 1) / W);
-  if (g_first == g_last) return;                            // written directly by the main kernel
-  // groups that hold tiles of this (sequence, head): computed once per block
-  __shared__ int list[256];
-  __shared__ int n_list;
-  if (threadIdx.x == 0) {
-    int n = 0;
-    for (int gi = g_first; gi <= g_last && n < 256; ++gi)
-      if ((W * gi) / NG != (W * (gi + 1)) / NG) list[n++] = gi;
-    n_list = n;
-  }
-  __syncthreads();
-  const int c = threadIdx.x;
-  const int i0 = mb * p.rows_per_mb;
-  const int m_begin = blockIdx.y * rows_per_block;
-  const size_t slot_floats = (size_t)ROWS * (DH + 2);
-  for (int m = m_begin; m < m_begin + rows_per_block && m < ROWS; ++m) {
-    const int il = m / p.G, g = m % p.G, i = i0 + il;
-    if (il >= p.rows_per_mb || i >= p.n_q) continue;
-    float mx = -CUDART_INF_F;
-    for (int x = 0; x < n_list; ++x) {
-      const float* ps = p.part + ((size_t)(item + list[x]) * p.n_mblocks + mb) * slot_floats;
-      mx = fmaxf(mx, __ldcg(ps + ROWS * DH + m));
-    }
-    float acc = 0.f, den = 0.f;
-    for (int x = 0; x < n_list; ++x) {
-      const float* ps = p.part + ((size_t)(item + list[x]) * p.n_mblocks + mb) * slot_floats;
-      const float ms = __ldcg(ps + ROWS * DH + m);
-      const float w = (ms > -CUDART_INF_F) ? exp2f(ms - mx) : 0.f;
-      den = fmaf(w, __ldcg(ps + ROWS * DH + ROWS + m), den);
-      acc = fmaf(w, __ldcg(ps + (size_t)m * DH + c), acc);
-    }
-    const int hq = h * p.G + g;
-    const size_t off = (((size_t)b * p.n_q + i) * p.H_q + hq) * DH + c;
-    const float r = acc / den;
-    if (p.out_dtype == SPACE_DTYPE_F32) reinterpret_cast<float*>(p.out)[off] = r;
-    else reinterpret_cast<__nv_bfloat16*>(p.out)[off] = __float2bfloat16_rn(r);
-    if (p.lse && c == 0)
-      p.lse[((size_t)b * p.H_q + hq) * p.n_q + i] = (mx + log2f(den)) * 0.6931471805599453f;
   }
 }
 
@@ -658,7 +728,7 @@ void plan(const space_config* cfg, int sm_count, int k, AttnPlanHost* pl) {
 
 template <int DH>
 size_t smem_bytes(int max_batch) {
-  return 1024 + Smem<DH>::TABLE_OFF + (size_t)(2 * max_batch + 2) * sizeof(int);
+  return Smem<DH>::TABLE_OFF + (size_t)(2 * max_batch + 2) * sizeof(int);
 }
 
 }  // namespace
@@ -693,6 +763,7 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   p.scale_log2 = a->scale * 1.4426950408889634f;
   p.kv_len = a->kv_len; p.out = a->out; p.lse = a->lse; p.status = a->status;
   p.part = ctx->attn_part; p.err = ctx->counters + 3 * cfg.max_batch;
+  p.merge_cnt = ctx->merge_cnt;
   for (int i = 0; i < SPACE_MAX_ROWS; ++i) p.mask[i] = mask_rows[i];
 
   // TMA descriptors, rebuilt only when a base pointer or a stride changes
@@ -717,31 +788,17 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   memcpy(&p.tm_k, ctx->tm_k, sizeof(CUtensorMap));
   memcpy(&p.tm_v, ctx->tm_v, sizeof(CUtensorMap));
 
-  const int rows_per_block = 8;
-  const dim3 mgrid(a->batch * p.H_kv * p.n_mblocks, (ROWS + rows_per_block - 1) / rows_per_block);
   if (DH == 128) {
     const size_t sm = smem_bytes<128>(cfg.max_batch);
     cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    {
-      ProfScope ps(ctx, SPACE_K_ATTN, st);
-      attn_tc_kernel<128><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
-    }
-    {
-      ProfScope ps(ctx, SPACE_K_MERGE, st);
-      attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(p, rows_per_block);
-    }
+    ProfScope ps(ctx, SPACE_K_ATTN, st);
+    attn_tc_kernel<128><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
   } else {
     const size_t sm = smem_bytes<64>(cfg.max_batch);
     cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    {
-      ProfScope ps(ctx, SPACE_K_ATTN, st);
-      attn_tc_kernel<64><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
-    }
-    {
-      ProfScope ps(ctx, SPACE_K_MERGE, st);
-      attn_merge_kernel<64><<<mgrid, 64, 0, st>>>(p, rows_per_block);
-    }
+    ProfScope ps(ctx, SPACE_K_ATTN, st);
+    attn_tc_kernel<64><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
   }
-  ctx->launches += 2;
+  ctx->launches += 1;
   return cuda_ok(cudaGetLastError());
 }

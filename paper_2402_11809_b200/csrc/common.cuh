@@ -56,6 +56,7 @@ struct space_ctx {
   float* attn_part;        // split partials
   size_t attn_part_slots;
   int* counters;           // [4][max_batch] self-resetting arrival counters
+  int* merge_cnt;          // attention split arrivals, one per (sequence, kv head, row block)
   VerifyPartial* vpart;    // [max_batch][k_max+2][SPACE_VERIFY_MAX_CHUNKS]
   VerifyRow* vrow;         // [max_batch][k_max+1]
   int32_t* scratch_status; // [max_batch] used when the caller passes no status array

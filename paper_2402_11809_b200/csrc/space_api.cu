@@ -27,7 +27,7 @@ int config_supported(const space_config* c) {
 }
 
 struct Carve {
-  size_t attn_part, counters, vpart, vrow, status, stage, total;
+  size_t attn_part, counters, merge_cnt, vpart, vrow, status, stage, total;
   size_t part_slots;
   // staging sub-offsets (relative to stage)
   size_t st_q, st_k, st_v, st_logits, st_small;
@@ -39,6 +39,8 @@ Carve carve(const space_config* c, int sm_count) {
   v.attn_part = off;
   off += align_up(attn_tensor_partial_floats(c, sm_count, &v.part_slots) * sizeof(float), 256);
   v.counters = off; off += align_up((size_t)(3 * c->max_batch + 4) * sizeof(int), 256);
+  v.merge_cnt = off;
+  off += align_up((size_t)c->max_batch * c->n_kv_heads * 8 * sizeof(int), 256);   // up to 8 row blocks
   v.vpart = off;
   off += align_up((size_t)c->max_batch * (c->k_max + 2) * SPACE_VERIFY_MAX_CHUNKS * sizeof(VerifyPartial), 256);
   v.vrow = off; off += align_up((size_t)c->max_batch * (c->k_max + 1) * sizeof(VerifyRow), 256);
@@ -133,6 +135,7 @@ int space_create(space_ctx** out, const space_config* cfg) {
   ctx->attn_part = (float*)(ctx->ws + cv.attn_part);
   ctx->attn_part_slots = cv.part_slots;
   ctx->counters = (int*)(ctx->ws + cv.counters);
+  ctx->merge_cnt = (int*)(ctx->ws + cv.merge_cnt);
   ctx->vpart = (VerifyPartial*)(ctx->ws + cv.vpart);
   ctx->vrow = (VerifyRow*)(ctx->ws + cv.vrow);
   ctx->scratch_status = (int32_t*)(ctx->ws + cv.status);
