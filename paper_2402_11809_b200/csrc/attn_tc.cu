@@ -5,8 +5,8 @@
 // and every thread-block group takes an equal contiguous share of it, so ragged
 // batches balance without host knowledge of the lengths.  A share that does not
 // cover a whole (sequence, head) leaves an unnormalised partial (running max,
-// sum, accumulator) in scratch memory; the last group to finish a (sequence,
-// head) combines its partials (arrival counter, reset by the last arriver).
+// sum, accumulator) in scratch memory; attn_merge_kernel combines the partials
+// of every (sequence, head) that was cut.
 //
 // Inside a block (12 warps):
 //   warps 0, 2  stream K and V tiles with TMA into two rings of shared-memory
@@ -45,7 +45,7 @@ struct AttnParams {
   void* out; float* lse; int32_t* status;
   float* part;                         // [slots][ROWS*(DH+2)]
   int* err;                            // one word: first timeout site
-  int* merge_cnt;                      // [B*H_kv*n_mblocks] arrivals per split (sequence, head, row block)
+  int2* desc;                          // [B*H_kv*n_mblocks] {first group, number of groups} of each cut
   uint64_t mask[SPACE_MAX_ROWS];
 };
 
@@ -82,6 +82,7 @@ __device__ __forceinline__ uint64_t global_ns() {
 // another thread of the block gave up; the first expiry records its site.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int* err, int site) {
+  if (*abort_flag) return mbar_try(bar, parity);            // draining: never block
   uint64_t t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try(bar, parity)) return true;
@@ -180,17 +181,28 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, int b_mn_major) {
 // ------------------------------------------------------------ work partition
 // Flat tile index space: sequence-major, then kv head, then tile.  Group g of
 // n_groups owns flat tiles [W*g/n_groups, W*(g+1)/n_groups).
+// floor(a * b / c) for a*b that may need 64 bits; 32-bit division when it fits
+__device__ __forceinline__ long long muldiv(long long a, long long b, long long c) {
+  const unsigned long long prod = (unsigned long long)a * (unsigned long long)b;
+  if ((prod >> 32) == 0) return (long long)((unsigned)prod / (unsigned)c);
+  return (long long)(prod / (unsigned long long)c);
+}
+
 struct Partition {
   const int* seq_len;    // [B]   verified length, or -1 for a sequence that does not fit
   const int* prefix;     // [B+1] flat offset of sequence b
   int B, H_kv, n_q;
   long long cur, end;
   int b;
+  // Only min(n_groups, W) groups take part, so every taking-part group owns at
+  // least one tile and the groups of one (sequence, head) are consecutive.
   __device__ void init(const int* sl, const int* pf, int B_, int H, int nq, int group, int n_groups) {
     seq_len = sl; prefix = pf; B = B_; H_kv = H; n_q = nq; b = 0;
     const long long W = pf[B_];
-    cur = (W * group) / n_groups;
-    end = (W * (group + 1)) / n_groups;
+    const long long NG = W < n_groups ? W : n_groups;
+    if (group >= NG) { cur = end = 0; return; }
+    cur = muldiv(W, group, NG);
+    end = muldiv(W, group + 1, NG);
   }
   __device__ bool next(Seg& s) {
     if (cur >= end) return false;
@@ -198,7 +210,7 @@ struct Partition {
     const int L = seq_len[b];
     const int T = (L + n_q + TILE_N - 1) / TILE_N;
     const int rem = (int)(cur - prefix[b]);
-    s.b = b; s.h = rem / T; s.t0 = rem % T; s.T = T; s.L = L;
+    s.b = b; s.h = rem / T; s.t0 = rem - s.h * T; s.T = T; s.L = L;
     long long n = T - s.t0;
     if (n > end - cur) n = end - cur;
     s.t1 = s.t0 + (int)n;
@@ -207,9 +219,11 @@ struct Partition {
   }
 };
 
-// group that owns flat tile f (largest g with W*g/NG <= f)
+// group that owns flat tile f (largest g with floor(W*g/NG) <= f)
 __device__ __forceinline__ int group_of(long long f, long long W, long long NG) {
-  return (int)(((f + 1) * NG - 1) / W);
+  const unsigned long long num = (unsigned long long)(f + 1) * (unsigned long long)NG - 1ull;
+  if ((num >> 32) == 0) return (int)((unsigned)num / (unsigned)W);
+  return (int)(num / (unsigned long long)W);
 }
 
 template <int DH>
@@ -223,20 +237,23 @@ struct Smem {
   static constexpr int K_OFF = Q_BYTES;
   static constexpr int V_OFF = K_OFF + K_STAGES * TILE_BYTES;
   static constexpr int BAR_OFF = V_OFF + V_STAGES * TILE_BYTES;
-  // q_full, q_empty, k_full[], k_empty[], v_full[], v_empty[], s_full[2], p_ready[2], pv_done[2], drain,
-  // pair[4] (the two threads of a row meet), all_soft
-  static constexpr int N_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 6 + 1 + 4 + 1;
-  static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;      // tmem base, abort flag, merge flag, merge count
+  // q_full, q_empty, k_full[], k_empty[], v_full[], v_empty[], s_full[2], p_ready[2], pv_done[2], drain
+  static constexpr int N_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 6 + 1;
+  static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;      // tmem base, abort flag
   static constexpr int XMAX_OFF = MISC_OFF + 32;             // [2 parities][2 halves][ROWS] float
   static constexpr int XSUM_OFF = XMAX_OFF + 2 * 2 * ROWS * 4;   // [2 halves][ROWS] float
-  static constexpr int MLIST_OFF = XSUM_OFF + 2 * ROWS * 4;  // [256] short: groups to merge
-  static constexpr int TABLE_OFF = MLIST_OFF + 512;          // seq_len[max_batch], prefix[max_batch+1]
+  static constexpr int TABLE_OFF = XSUM_OFF + 2 * ROWS * 4;  // seq_len[max_batch], prefix[max_batch+1]
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// The two softmax warps that share a TMEM lane quarter meet here (ids 1..4).
+__device__ __forceinline__ void pair_sync(int quarter) {
+  asm volatile("bar.sync %0, 64;" ::"r"(quarter + 1) : "memory");
 }
 
 // Warp roles
@@ -253,14 +270,11 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   constexpr int B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = B_KFULL + S::K_STAGES,
                 B_VFULL = B_KEMPTY + S::K_STAGES, B_VEMPTY = B_VFULL + S::V_STAGES,
                 B_SFULL = B_VEMPTY + S::V_STAGES, B_PREADY = B_SFULL + 2, B_PVDONE = B_SFULL + 4,
-                B_DRAIN = B_SFULL + 6, B_PAIR = B_DRAIN + 1, B_ALL = B_PAIR + 4;
+                B_DRAIN = B_SFULL + 6;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + S::MISC_OFF);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 4);
-  volatile int* merge_flag = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 8);
-  volatile int* merge_n = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 12);
   float* xmax = reinterpret_cast<float*>(sm + S::XMAX_OFF);
   float* xsum = reinterpret_cast<float*>(sm + S::XSUM_OFF);
-  short* mlist = reinterpret_cast<short*>(sm + S::MLIST_OFF);
   int* seq_len = reinterpret_cast<int*>(sm + S::TABLE_OFF);
   int* prefix = seq_len + max_batch;
 
@@ -276,17 +290,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   if (threadIdx.x == 0) {
     *abort_flag = (sm_base & 1023u) ? 1 : 0;               // swizzled tiles need a 1024-byte aligned base
     if (*abort_flag) atomicCAS(p.err, 0, 99);
-    *merge_flag = 0;
-    long long acc = 0;
-    for (int b = 0; b < p.B; ++b) {
-      const int L = p.kv_len[b];
-      const bool ok = L >= 0 && (int64_t)L + p.n_q <= p.s_cap;
-      if (!ok && blockIdx.x == 0 && p.status) atomicOr(p.status + b, SPACE_ST_CAPACITY);
-      seq_len[b] = ok ? L : -1;
-      prefix[b] = (int)acc;
-      if (ok) acc += (long long)((L + p.n_q + TILE_N - 1) / TILE_N) * p.H_kv;
-    }
-    prefix[p.B] = (int)acc;
     mbar_init(BAR(B_QFULL), 1);
     mbar_init(BAR(B_QEMPTY), 1);
     for (int s = 0; s < S::K_STAGES; ++s) { mbar_init(BAR(B_KFULL + s), 1); mbar_init(BAR(B_KEMPTY + s), 1); }
@@ -297,10 +300,32 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       mbar_init(BAR(B_PVDONE + i), 1);
     }
     mbar_init(BAR(B_DRAIN), 1);
-    for (int q = 0; q < 4; ++q) mbar_init(BAR(B_PAIR + q), 64);
-    mbar_init(BAR(B_ALL), n_soft);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == WARP_SOFTMAX0) {
+    // per-sequence tile counts and their running sum, 32 sequences per round
+    int carry = 0;
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+      const int b = b0 + lane;
+      int L = -1, tiles = 0;
+      if (b < p.B) {
+        L = p.kv_len[b];
+        const bool ok = L >= 0 && (int64_t)L + p.n_q <= p.s_cap;
+        if (!ok && blockIdx.x == 0 && p.status) atomicOr(p.status + b, SPACE_ST_CAPACITY);
+        if (!ok) L = -1;
+        tiles = ok ? ((L + p.n_q + TILE_N - 1) / TILE_N) * p.H_kv : 0;
+      }
+      int incl = tiles;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      if (b < p.B) { seq_len[b] = L; prefix[b] = carry + incl - tiles; }
+      carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+    if (lane == 0) prefix[p.B] = carry;
   }
   if (warp == WARP_MMA) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -448,23 +473,17 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     const float c = p.scale_log2;
     constexpr int HC = TILE_N / 2;                         // keys per thread and tile
     constexpr int OC = DH / 2;                             // output columns per thread
-    uint32_t gt = 0, pair_ph = 0, all_ph = 0;
+    uint32_t gt = 0;
+    // A failed (expired) wait does not leave the loops: every thread keeps the
+    // same control flow so that the pair barriers below always match up; once
+    // the abort flag is set all later waits return at once and the block drains.
     bool ok = true;
-    // Rendezvous on an mbarrier (bounded, unlike bar.sync): the two threads of a
-    // row, or all softmax threads.  Shared-memory writes before it are visible after.
-    auto meet = [&](int bar, uint32_t& ph, int site) -> bool {
-      mbar_arrive(BAR(bar));
-      const bool r = mbar_wait(BAR(bar), ph & 1, abort_flag, p.err, site);
-      ++ph;
-      return r;
-    };
-    while (ok && part.next(sg)) {
+    while (part.next(sg)) {
       const int n_keys = sg.L + p.n_q;
       float m_ref = -CUDART_INF_F, l_sum = 0.f;
-      for (int t = sg.t0; t < sg.t1 && ok; ++t, ++gt) {
+      for (int t = sg.t0; t < sg.t1; ++t, ++gt) {
         const int buf = gt & 1;
-        ok = mbar_wait(BAR(B_SFULL + buf), (gt >> 1) & 1, abort_flag, p.err, 9);
-        if (!ok) break;
+        ok &= mbar_wait(BAR(B_SFULL + buf), (gt >> 1) & 1, abort_flag, p.err, 9);
         tc_fence_after();
         const uint32_t ts = TM_S0 + buf * TILE_N + lane_addr;
         uint32_t sreg[HC];
@@ -493,8 +512,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         // both threads' reads of S before either overwrites it with P
         float* xm = xmax + (gt & 1) * (2 * ROWS);
         xm[half * ROWS + m] = tmax;
-        ok = meet(B_PAIR + quarter, pair_ph, 12);
-        if (!ok) break;
+        pair_sync(quarter);
         tmax = fmaxf(tmax, xm[(half ^ 1) * ROWS + m]);
         tmax *= c;                                         // c > 0
         if (!(tmax > -CUDART_INF_F)) tmax = -CUDART_INF_F; // also catches NaN
@@ -503,8 +521,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         if (first) m_ref = tmax;
         if (__any_sync(0xFFFFFFFFu, need)) {
           // lazy rescale of this row's accumulator; PV of the previous tile must be done
-          ok = mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 10);
-          if (!ok) break;
+          ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 10);
           tc_fence_after();
           const float m_new = fmaxf(m_ref, tmax);
           const float f = (m_ref > -CUDART_INF_F) ? fast_exp2(m_ref - m_new) : 0.f;
@@ -544,27 +561,37 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         tc_fence_before();
         mbar_arrive(BAR(B_PREADY + buf));
       }
-      if (!ok) break;
       // ---- end of share: final output or partial ---------------------------
-      ok = mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 11);
-      if (!ok) break;
+      ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 11);
       tc_fence_after();
       xsum[half * ROWS + m] = l_sum;
-      ok = meet(B_PAIR + quarter, pair_ph, 13);
-      if (!ok) break;
+      pair_sync(quarter);
       const float l_tot = l_sum + xsum[(half ^ 1) * ROWS + m];
       const bool whole = (sg.t0 == 0 && sg.t1 == sg.T);
       const int hq = sg.h * p.G + g;
       const int item = sg.b * p.H_kv + sg.h;
       float* pslot = p.part + ((size_t)(item + group) * p.n_mblocks + mb) * (ROWS * (DH + 2));
       const float inv = (l_tot > 0.f) ? 1.f / l_tot : 0.f;
+      if (sidx == 0 && ok) {
+        // how this (sequence, head) was cut: first group and number of groups,
+        // read by attn_merge_kernel (every group of the cut writes the same pair)
+        int2 d = make_int2(group, 1);
+        if (!whole) {
+          const long long W = prefix[p.B];
+          const long long NG = W < p.n_groups ? W : p.n_groups;
+          const long long f0 = (long long)prefix[sg.b] + (long long)sg.h * sg.T;
+          d.x = group_of(f0, W, NG);
+          d.y = group_of(f0 + sg.T - 1, W, NG) - d.x + 1;
+        }
+        p.desc[(size_t)item * p.n_mblocks + mb] = d;
+      }
 #pragma unroll 1
       for (int cc = 0; cc < OC / 32; ++cc) {
         uint32_t o[32];
         const int col = half * OC + cc * 32;
         tmem_ld32(TM_O + lane_addr + col, o);
         tmem_wait_ld();
-        if (!row_valid) continue;
+        if (!row_valid || !ok) continue;
         if (whole) {
           const size_t off = (((size_t)sg.b * p.n_q + i) * p.H_q + hq) * DH + col;
           if (p.out_dtype == SPACE_DTYPE_F32) {
@@ -591,84 +618,19 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           float4* dst = reinterpret_cast<float4*>(pslot + (size_t)m * DH + col);
 #pragma unroll
           for (int x = 0; x < 8; ++x)
-            __stcg(dst + x, make_float4(__uint_as_float(o[4 * x]), __uint_as_float(o[4 * x + 1]),
-                                        __uint_as_float(o[4 * x + 2]), __uint_as_float(o[4 * x + 3])));
+            dst[x] = make_float4(__uint_as_float(o[4 * x]), __uint_as_float(o[4 * x + 1]),
+                                 __uint_as_float(o[4 * x + 2]), __uint_as_float(o[4 * x + 3]));
         }
       }
       tc_fence_before();
-      if (whole) {
-        if (row_valid && half == 0 && p.lse)
-          p.lse[((size_t)sg.b * p.H_q + hq) * p.n_q + i] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
-        continue;
-      }
-      if (row_valid && half == 0) {
-        __stcg(pslot + ROWS * DH + m, m_ref);
-        __stcg(pslot + ROWS * DH + ROWS + m, l_tot);
-      }
-      // ---- partial: the last group to finish a (sequence, head) merges it ----
-      __threadfence();
-      ok = meet(B_ALL, all_ph, 14);
-      if (!ok) break;
-      if (sidx == 0) {
-        const long long W = prefix[p.B], NG = p.n_groups;
-        const long long f0 = (long long)prefix[sg.b] + (long long)sg.h * sg.T;
-        int n = 0;
-        if (W >= NG) {                                     // every group holds tiles
-          const int g0 = group_of(f0, W, NG), g1 = group_of(f0 + sg.T - 1, W, NG);
-          for (int gi = g0; gi <= g1 && n < 256; ++gi) mlist[n++] = (short)gi;
-        } else {                                           // one tile per non-empty group
-          for (int t = 0; t < sg.T && n < 256; ++t) mlist[n++] = (short)group_of(f0 + t, W, NG);
+      if (row_valid && half == 0 && ok) {
+        if (whole) {
+          if (p.lse)
+            p.lse[((size_t)sg.b * p.H_q + hq) * p.n_q + i] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
+        } else {
+          pslot[ROWS * DH + m] = m_ref;
+          pslot[ROWS * DH + ROWS + m] = l_tot;
         }
-        int* cnt = p.merge_cnt + (size_t)item * p.n_mblocks + mb;
-        const int prev = atomicAdd(cnt, 1);
-        const int last = (prev == n - 1);
-        if (last) *cnt = 0;                                // ready for the next launch
-        *merge_n = n;
-        *merge_flag = last;
-      }
-      ok = meet(B_ALL, all_ph, 15);
-      if (!ok) break;
-      if (*merge_flag) {
-        __threadfence();
-        const int n = *merge_n;
-        constexpr int C4 = DH / 4;
-        const size_t slot_floats = (size_t)ROWS * (DH + 2);
-        const float* pbase = p.part + ((size_t)item * p.n_mblocks + mb) * slot_floats;
-        const size_t gstride = (size_t)p.n_mblocks * slot_floats;
-        for (int idx = sidx; idx < m_valid * C4; idx += n_soft) {
-          const int r = idx / C4, c4 = idx % C4;
-          float mx = -CUDART_INF_F;
-#pragma unroll 4
-          for (int x = 0; x < n; ++x) mx = fmaxf(mx, __ldcg(pbase + mlist[x] * gstride + ROWS * DH + r));
-          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-          float den = 0.f;
-#pragma unroll 4
-          for (int x = 0; x < n; ++x) {
-            const float* ps = pbase + mlist[x] * gstride;
-            const float ms = __ldcg(ps + ROWS * DH + r);
-            const float ls = __ldcg(ps + ROWS * DH + ROWS + r);
-            const float4 ov = __ldcg(reinterpret_cast<const float4*>(ps + (size_t)r * DH) + c4);
-            const float w = (ms > -CUDART_INF_F) ? fast_exp2(ms - mx) : 0.f;
-            den = fmaf(w, ls, den);
-            acc.x = fmaf(w, ov.x, acc.x); acc.y = fmaf(w, ov.y, acc.y);
-            acc.z = fmaf(w, ov.z, acc.z); acc.w = fmaf(w, ov.w, acc.w);
-          }
-          const float rinv = 1.f / den;
-          const int ri = i0 + r / p.G, rhq = sg.h * p.G + r % p.G;
-          const size_t off = (((size_t)sg.b * p.n_q + ri) * p.H_q + rhq) * DH + c4 * 4;
-          if (p.out_dtype == SPACE_DTYPE_F32) {
-            *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off) =
-                make_float4(acc.x * rinv, acc.y * rinv, acc.z * rinv, acc.w * rinv);
-          } else {
-            const __nv_bfloat162 a = __floats2bfloat162_rn(acc.x * rinv, acc.y * rinv);
-            const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc.z * rinv, acc.w * rinv);
-            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off) =
-                make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b2));
-          }
-          if (p.lse && c4 == 0)
-            p.lse[((size_t)sg.b * p.H_q + rhq) * p.n_q + ri] = (mx + log2f(den)) * 0.6931471805599453f;
-        }
-        ok = meet(B_ALL, all_ph, 16);                      // merge_flag / mlist are reused by the next share
       }
     }
   }
@@ -683,6 +645,59 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   if (threadIdx.x == 0 && *abort_flag && p.status) {
     for (int b = 0; b < p.B; ++b) atomicOr(p.status + b, SPACE_ST_TIMEOUT);
   }
+}
+
+// Combine the partials of every (sequence, kv head, query-row block) that was
+// cut over several groups: one thread per 16 output bytes, all loads of a
+// thread independent, running maximum / denominator / accumulator in one pass.
+// grid = (B*H_kv*n_mblocks, ceil(rows*DH/4 / 128)), 128 threads.
+template <int DH>
+__global__ void __launch_bounds__(128) attn_merge_kernel(const AttnParams p) {
+  constexpr int C4 = DH / 4;
+  const int item = blockIdx.x / p.n_mblocks, mb = blockIdx.x % p.n_mblocks;
+  const int b = item / p.H_kv, h = item % p.H_kv;
+  const int L = p.kv_len[b];
+  if (L < 0 || (int64_t)L + p.n_q > p.s_cap) return;
+  const int2 d = p.desc[blockIdx.x];
+  const int n = d.y;
+  if (n <= 1) return;                                       // written directly by the main kernel
+  const int i0 = mb * p.rows_per_mb;
+  const int m_valid = min(p.rows_per_mb, p.n_q - i0) * p.G;
+  const int idx = blockIdx.y * 128 + threadIdx.x;
+  if (idx >= m_valid * C4) return;
+  const int r = idx / C4, c4 = idx % C4;
+  const size_t slot_floats = (size_t)ROWS * (DH + 2);
+  const float* ps = p.part + ((size_t)(item + d.x) * p.n_mblocks + mb) * slot_floats;
+  const size_t gstride = (size_t)p.n_mblocks * slot_floats;
+  float mx = -CUDART_INF_F, den = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+  for (int x = 0; x < n; ++x, ps += gstride) {
+    const float ms = __ldcg(ps + ROWS * DH + r), ls = __ldcg(ps + ROWS * DH + ROWS + r);
+    const float4 ov = __ldcg(reinterpret_cast<const float4*>(ps + (size_t)r * DH) + c4);
+    const float mn = fmaxf(mx, ms);
+    if (mn > -CUDART_INF_F) {
+      const float e0 = fast_exp2(mx - mn), e1 = fast_exp2(ms - mn);
+      den = den * e0 + ls * e1;
+      acc.x = acc.x * e0 + ov.x * e1; acc.y = acc.y * e0 + ov.y * e1;
+      acc.z = acc.z * e0 + ov.z * e1; acc.w = acc.w * e0 + ov.w * e1;
+    }
+    mx = mn;
+  }
+  const float rd = 1.f / den;
+  const int ri = i0 + r / p.G, hq = h * p.G + r % p.G;
+  const size_t off = (((size_t)b * p.n_q + ri) * p.H_q + hq) * DH + c4 * 4;
+  if (p.out_dtype == SPACE_DTYPE_F32) {
+    *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off) =
+        make_float4(acc.x * rd, acc.y * rd, acc.z * rd, acc.w * rd);
+  } else {
+    const __nv_bfloat162 a = __floats2bfloat162_rn(acc.x * rd, acc.y * rd);
+    const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc.z * rd, acc.w * rd);
+    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off) =
+        make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b2));
+  }
+  if (p.lse && c4 == 0)
+    p.lse[((size_t)b * p.H_q + hq) * p.n_q + ri] = (mx + log2f(den)) * 0.6931471805599453f;
 }
 
 // ------------------------------------------------------------------ host side
@@ -763,7 +778,7 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   p.scale_log2 = a->scale * 1.4426950408889634f;
   p.kv_len = a->kv_len; p.out = a->out; p.lse = a->lse; p.status = a->status;
   p.part = ctx->attn_part; p.err = ctx->counters + 3 * cfg.max_batch;
-  p.merge_cnt = ctx->merge_cnt;
+  p.desc = reinterpret_cast<int2*>(ctx->merge_cnt);
   for (int i = 0; i < SPACE_MAX_ROWS; ++i) p.mask[i] = mask_rows[i];
 
   // TMA descriptors, rebuilt only when a base pointer or a stride changes
@@ -788,17 +803,31 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   memcpy(&p.tm_k, ctx->tm_k, sizeof(CUtensorMap));
   memcpy(&p.tm_v, ctx->tm_v, sizeof(CUtensorMap));
 
+  const int m_valid_max = p.rows_per_mb * p.G;
+  const dim3 mgrid(a->batch * p.H_kv * p.n_mblocks, (m_valid_max * (DH / 4) + 127) / 128);
   if (DH == 128) {
     const size_t sm = smem_bytes<128>(cfg.max_batch);
     cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    ProfScope ps(ctx, SPACE_K_ATTN, st);
-    attn_tc_kernel<128><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
+    {
+      ProfScope ps(ctx, SPACE_K_ATTN, st);
+      attn_tc_kernel<128><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
+    }
+    {
+      ProfScope ps(ctx, SPACE_K_MERGE, st);
+      attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(p);
+    }
   } else {
     const size_t sm = smem_bytes<64>(cfg.max_batch);
     cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    ProfScope ps(ctx, SPACE_K_ATTN, st);
-    attn_tc_kernel<64><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
+    {
+      ProfScope ps(ctx, SPACE_K_ATTN, st);
+      attn_tc_kernel<64><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
+    }
+    {
+      ProfScope ps(ctx, SPACE_K_MERGE, st);
+      attn_merge_kernel<64><<<mgrid, 128, 0, st>>>(p);
+    }
   }
-  ctx->launches += 1;
+  ctx->launches += 2;
   return cuda_ok(cudaGetLastError());
 }
