@@ -287,9 +287,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   const int n_soft = 64 * n_quarters;                      // softmax threads that take part
 
   // ---- set-up ------------------------------------------------------------
+  pdl_launch_dependents();
   if (threadIdx.x == 0) {
     *abort_flag = (sm_base & 1023u) ? 1 : 0;               // swizzled tiles need a 1024-byte aligned base
-    if (*abort_flag) atomicCAS(p.err, 0, 99);
     mbar_init(BAR(B_QFULL), 1);
     mbar_init(BAR(B_QEMPTY), 1);
     for (int s = 0; s < S::K_STAGES; ++s) { mbar_init(BAR(B_KFULL + s), 1); mbar_init(BAR(B_KEMPTY + s), 1); }
@@ -303,6 +303,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  pdl_wait();                                              // global memory from here on
   if (warp == WARP_SOFTMAX0) {
     // per-sequence tile counts and their running sum, 32 sequences per round
     int carry = 0;
@@ -653,6 +654,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
 // grid = (B*H_kv*n_mblocks, ceil(rows*DH/4 / 128)), 128 threads.
 template <int DH>
 __global__ void __launch_bounds__(128) attn_merge_kernel(const AttnParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int C4 = DH / 4;
   const int item = blockIdx.x / p.n_mblocks, mb = blockIdx.x % p.n_mblocks;
   const int b = item / p.H_kv, h = item % p.H_kv;
@@ -810,22 +813,22 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
     cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     {
       ProfScope ps(ctx, SPACE_K_ATTN, st);
-      attn_tc_kernel<128><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
+      launch_pdl(attn_tc_kernel<128>, dim3(pl.n_ctas), dim3(THREADS), sm, st, p, cfg.max_batch);
     }
     {
       ProfScope ps(ctx, SPACE_K_MERGE, st);
-      attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(p);
+      launch_pdl(attn_merge_kernel<128>, mgrid, dim3(128), 0, st, p);
     }
   } else {
     const size_t sm = smem_bytes<64>(cfg.max_batch);
     cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     {
       ProfScope ps(ctx, SPACE_K_ATTN, st);
-      attn_tc_kernel<64><<<pl.n_ctas, THREADS, sm, st>>>(p, cfg.max_batch);
+      launch_pdl(attn_tc_kernel<64>, dim3(pl.n_ctas), dim3(THREADS), sm, st, p, cfg.max_batch);
     }
     {
       ProfScope ps(ctx, SPACE_K_MERGE, st);
-      attn_merge_kernel<64><<<mgrid, 128, 0, st>>>(p);
+      launch_pdl(attn_merge_kernel<64>, mgrid, dim3(128), 0, st, p);
     }
   }
   ctx->launches += 2;

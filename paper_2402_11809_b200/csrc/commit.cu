@@ -20,6 +20,8 @@ struct CommitParams {
 };
 
 __global__ void __launch_bounds__(256) kv_commit_kernel(const CommitParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int b = blockIdx.y, part = blockIdx.x;
   const int L = p.kv_len[b];
   int i_star = p.n_accept[b];
@@ -83,7 +85,7 @@ int launch_commit(space_ctx* ctx, const space_commit_args* a, cudaStream_t st) {
   p.blocks_per_seq = blocks;
   {
     ProfScope ps(ctx, SPACE_K_COMMIT, st);
-    kv_commit_kernel<<<dim3(blocks, a->batch), 256, 0, st>>>(p);
+    launch_pdl(kv_commit_kernel, dim3(blocks, a->batch), dim3(256), 0, st, p);
   }
   ctx->launches += 1;
   return cuda_ok(cudaGetLastError());

@@ -59,6 +59,7 @@ struct space_ctx {
   int* merge_cnt;          // attention split arrivals, one per (sequence, kv head, row block)
   VerifyPartial* vpart;    // [max_batch][k_max+2][SPACE_VERIFY_MAX_CHUNKS]
   VerifyRow* vrow;         // [max_batch][k_max+1]
+  VerifyPartial* vfused;   // [max_batch][SPACE_MAX_ROWS][16] single-launch greedy path
   int32_t* scratch_status; // [max_batch] used when the caller passes no status array
   // staging for space_step_host
   char* stage;
@@ -100,5 +101,24 @@ struct ProfScope {
     ctx->prof_n[which] = slot + 1;
   }
 };
+
+// Programmatic dependent launch: the kernel may be scheduled while the previous
+// kernel of the stream is still draining; every kernel calls pdl_wait() before
+// it touches global memory, which blocks until the previous kernel has finished
+// and its writes are visible.  Both are no-ops without the launch attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                     cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 static inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? SPACE_OK : SPACE_E_CUDA; }

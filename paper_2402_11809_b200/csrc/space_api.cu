@@ -27,7 +27,7 @@ int config_supported(const space_config* c) {
 }
 
 struct Carve {
-  size_t attn_part, counters, merge_cnt, vpart, vrow, status, stage, total;
+  size_t attn_part, counters, merge_cnt, vpart, vfused, vrow, status, stage, total;
   size_t part_slots;
   // staging sub-offsets (relative to stage)
   size_t st_q, st_k, st_v, st_logits, st_small;
@@ -43,6 +43,7 @@ Carve carve(const space_config* c, int sm_count) {
   off += align_up((size_t)c->max_batch * c->n_kv_heads * 8 * sizeof(int), 256);   // up to 8 row blocks
   v.vpart = off;
   off += align_up((size_t)c->max_batch * (c->k_max + 2) * SPACE_VERIFY_MAX_CHUNKS * sizeof(VerifyPartial), 256);
+  v.vfused = off; off += align_up((size_t)c->max_batch * SPACE_MAX_ROWS * 16 * sizeof(VerifyPartial), 256);
   v.vrow = off; off += align_up((size_t)c->max_batch * (c->k_max + 1) * sizeof(VerifyRow), 256);
   v.status = off; off += align_up((size_t)c->max_batch * sizeof(int32_t), 256);
   v.stage = off;
@@ -138,6 +139,7 @@ int space_create(space_ctx** out, const space_config* cfg) {
   ctx->merge_cnt = (int*)(ctx->ws + cv.merge_cnt);
   ctx->vpart = (VerifyPartial*)(ctx->ws + cv.vpart);
   ctx->vrow = (VerifyRow*)(ctx->ws + cv.vrow);
+  ctx->vfused = (VerifyPartial*)(ctx->ws + cv.vfused);
   ctx->scratch_status = (int32_t*)(ctx->ws + cv.status);
   ctx->stage = cfg->host_staging ? ctx->ws + cv.stage : nullptr;
   ctx->stage_bytes = cv.total - cv.stage;

@@ -13,10 +13,19 @@
 // Each row is cut into chunks so that small batches still fill the GPU; chunk
 // results meet in a small scratch array and an arrival counter (reset by the
 // last block) decides who finishes the sequence.
+//
+// Small greedy problems (all (k+1)^2 rows of the batch within a few MB) are
+// latency bound, not bandwidth bound: for them verify_fused_kernel streams
+// every row in one launch and the last block of a sequence picks i* and the
+// mask rows of group i* from the per-row results, which removes the second
+// launch and its dependent round trips at the price of reading rows that the
+// two-launch path skips.
 #include "common.cuh"
 #include <math_constants.h>
 
 namespace {
+
+constexpr int64_t SPACE_FUSED_MAX_BYTES = 8ll << 20;
 
 struct VerifyParams {
   int B, k, V, n_q, n_chunks, chunk;
@@ -225,6 +234,8 @@ __device__ bool arrive_last(int* counter, int expected) {
 template <typename T, bool VECTOR>
 __global__ void __launch_bounds__(SPACE_VERIFY_THREADS)
 verify_target_kernel(const VerifyParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int b = blockIdx.z, t = blockIdx.y, ch = blockIdx.x;
   const int k1 = p.k + 1;
   const T* row = reinterpret_cast<const T*>(p.logits) + ((int64_t)b * p.n_q + (int64_t)t * k1) * p.row_stride;
@@ -285,6 +296,8 @@ verify_target_kernel(const VerifyParams p) {
 template <typename T, bool VECTOR>
 __global__ void __launch_bounds__(SPACE_VERIFY_THREADS)
 verify_emit_kernel(const VerifyParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int b = blockIdx.z, slot = blockIdx.y, ch = blockIdx.x;
   const int k1 = p.k + 1;
   const int i_star = p.n_accept[b];
@@ -359,16 +372,94 @@ verify_emit_kernel(const VerifyParams p) {
   }
 }
 
+
+#define SPACE_FUSED_MAX_CHUNKS 16
+
+// One launch for greedy mode on small inputs: statistics of every block row,
+// then acceptance, emission and next candidates by the last block of a sequence.
+template <typename T, bool VECTOR>
+__global__ void __launch_bounds__(SPACE_VERIFY_THREADS)
+verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int b = blockIdx.z, row_i = blockIdx.y, ch = blockIdx.x;
+  const int k1 = p.k + 1;
+  constexpr float C1 = 1.4426950408889634f;                 // T = 1
+  const T* row = reinterpret_cast<const T*>(p.logits) + ((int64_t)b * p.n_q + row_i) * p.row_stride;
+  const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
+  Stat st = scan_chunk<T, VECTOR, false>(row, begin, end, C1, 1.f, -1, 0, 0, 0, 0, 0);
+  st = block_reduce(st, C1);
+  VerifyPartial* pb = fpart + (int64_t)b * SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS;
+  if (threadIdx.x == 0) store_partial(pb + row_i * p.n_chunks + ch, st);
+  if (!arrive_last(p.counter_a + b, p.n_q * p.n_chunks)) return;
+
+  // ---- last block of sequence b -------------------------------------------
+  __shared__ float sh_m[SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS];
+  __shared__ float sh_s[SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS];
+  __shared__ int sh_i[SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS];
+  __shared__ float row_s[SPACE_MAX_ROWS];
+  __shared__ int row_idx[SPACE_MAX_ROWS];
+  __shared__ int sh_cand[SPACE_MAX_K];
+  const int total = p.n_q * p.n_chunks;
+  for (int t = threadIdx.x; t < total; t += blockDim.x) {   // every chunk result, one round trip
+    sh_m[t] = __ldcg(&pb[t].m); sh_s[t] = __ldcg(&pb[t].s); sh_i[t] = __ldcg(&pb[t].idx);
+  }
+  if (threadIdx.x < p.k) sh_cand[threadIdx.x] = p.cand[b * p.k + threadIdx.x];
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int r = warp; r < p.n_q; r += SPACE_VERIFY_THREADS / 32) {
+    Stat a = stat_empty();
+    if (lane < p.n_chunks) { a.m = sh_m[r * p.n_chunks + lane]; a.s = sh_s[r * p.n_chunks + lane]; a.idx = sh_i[r * p.n_chunks + lane]; }
+    a = warp_reduce(a, C1);
+    if (lane == 0) { row_s[r] = a.s; row_idx[r] = a.idx; }
+  }
+  __syncthreads();
+  if (threadIdx.x >= 32) return;
+  // acceptance: longest prefix of candidates equal to the arg-max chain
+  int i_star = 0, bits = 0;
+  for (int t = 0; t < p.k; ++t) {
+    const int c = sh_cand[t];
+    if (c < 0 || c >= p.V) bits |= SPACE_ST_BAD_CANDIDATE;
+  }
+  while (i_star < p.k && sh_cand[i_star] >= 0 && sh_cand[i_star] < p.V &&
+         sh_cand[i_star] == row_idx[i_star * k1]) ++i_star;
+  const int j = lane;
+  if (j < k1) {
+    int tok = (j < i_star) ? sh_cand[j] : (j == i_star ? row_idx[i_star * k1] : -1);
+    const bool is_eos = p.eos_id >= 0 && j <= i_star && tok == p.eos_id;
+    const unsigned eos_mask = __ballot_sync((1u << k1) - 1u, is_eos);
+    const int n_out = eos_mask ? __ffs(eos_mask) - 1 : i_star + 1;
+    p.out_tokens[b * k1 + j] = (j < n_out) ? tok : -1;
+    if (j < p.k) {                                          // next candidate j+1 from mask row (i*, j+1)
+      const int mr = i_star * k1 + j + 1;
+      p.next_cand[b * p.k + j] = row_idx[mr];
+      p.next_cand_prob[b * p.k + j] = 1.f / row_s[mr];      // softmax at T = 1 of its own maximum
+    }
+    if (j == 0) {
+      p.n_accept[b] = i_star;
+      p.n_out[b] = n_out;
+      p.finished[b] = (uint8_t)(eos_mask != 0);
+      if (p.status && bits) atomicOr(p.status + b, bits);
+    }
+  }
+}
+
+template <typename T, bool VECTOR>
+void launch_fused(space_ctx* ctx, const VerifyParams& p, cudaStream_t st) {
+  ProfScope ps(ctx, SPACE_K_VERIFY_TARGET, st);
+  launch_pdl(verify_fused_kernel<T, VECTOR>, dim3(p.n_chunks, p.n_q, p.B), dim3(SPACE_VERIFY_THREADS), 0, st, p, ctx->vfused);
+}
+
 template <typename T, bool VECTOR>
 void launch_both(space_ctx* ctx, const VerifyParams& p, int n_slots_b, cudaStream_t st) {
   dim3 ga(p.n_chunks, p.k + 1, p.B), gb(p.n_chunks, n_slots_b, p.B);
   {
     ProfScope ps(ctx, SPACE_K_VERIFY_TARGET, st);
-    verify_target_kernel<T, VECTOR><<<ga, SPACE_VERIFY_THREADS, 0, st>>>(p);
+    launch_pdl(verify_target_kernel<T, VECTOR>, ga, dim3(SPACE_VERIFY_THREADS), 0, st, p);
   }
   {
     ProfScope ps(ctx, SPACE_K_VERIFY_EMIT, st);
-    verify_emit_kernel<T, VECTOR><<<gb, SPACE_VERIFY_THREADS, 0, st>>>(p);
+    launch_pdl(verify_emit_kernel<T, VECTOR>, gb, dim3(SPACE_VERIFY_THREADS), 0, st, p);
   }
 }
 
@@ -402,6 +493,28 @@ int launch_verify(space_ctx* ctx, const space_verify_args* a, cudaStream_t st) {
   const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;
   const int vec = 16 / esz;
   const bool vector = ((uintptr_t)a->logits % 16 == 0) && ((a->logits_row_stride * esz) % 16 == 0);
+  // small greedy problem: one launch over all block rows (see the file header)
+  const int64_t all_bytes = (int64_t)a->batch * p.n_q * a->vocab * esz;
+  if (a->mode == SPACE_MODE_GREEDY && all_bytes <= SPACE_FUSED_MAX_BYTES) {
+    const int rows_all = a->batch * p.n_q;
+    int nc = (2 * ctx->sm_count + rows_all - 1) / rows_all;
+    const int min_chunk = SPACE_VERIFY_THREADS * vec;
+    const int max_nc = (a->vocab + min_chunk - 1) / min_chunk;
+    if (nc > max_nc) nc = max_nc;
+    if (nc > SPACE_FUSED_MAX_CHUNKS) nc = SPACE_FUSED_MAX_CHUNKS;
+    if (nc < 1) nc = 1;
+    int chunk = (a->vocab + nc - 1) / nc;
+    chunk = ((chunk + vec - 1) / vec) * vec;
+    nc = (a->vocab + chunk - 1) / chunk;
+    p.n_chunks = nc; p.chunk = chunk;
+    if (a->logits_dtype == SPACE_DTYPE_F32) {
+      if (vector) launch_fused<float, true>(ctx, p, st); else launch_fused<float, false>(ctx, p, st);
+    } else {
+      if (vector) launch_fused<__nv_bfloat16, true>(ctx, p, st); else launch_fused<__nv_bfloat16, false>(ctx, p, st);
+    }
+    ctx->launches += 1;
+    return cuda_ok(cudaGetLastError());
+  }
   // enough chunks to put about two blocks on every SM, but no chunk below two
   // sweeps of a block
   const int rows = a->batch * (a->k + 1);
