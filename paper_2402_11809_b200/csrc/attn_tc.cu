@@ -4,23 +4,30 @@
 // are cut into 128-key tiles, the tiles of all sequences form one flat list
 // and every thread-block group takes an equal contiguous share of it, so ragged
 // batches balance without host knowledge of the lengths.  A share that does not
-// cover a whole (sequence, head) leaves an unnormalised partial (running max,
-// sum, accumulator) in scratch memory; attn_merge_kernel combines the partials
-// of every (sequence, head) that was cut.
+// cover a whole (sequence, head) leaves an unnormalised partial (reference
+// maximum, sum, accumulator) in scratch memory; attn_merge_kernel combines the
+// partials of every (sequence, head) that was cut.
+//
+// The query block of one kv head is small (the (k+1)^2 block rows times the GQA
+// group: 25 to 112 rows), so the two tile products are taken transposed: the
+// 128 keys of a tile are the MMA M extent and the query rows the N extent,
+//   S^T = K Q^T   (128 x N),      O^T += V^T (P_hi + P_lo)^T   (head_dim x N),
+// which costs N/128 of a full tile and puts one key on every TMEM lane.
 //
 // Inside a block (12 warps):
 //   warps 0, 2  stream K and V tiles with TMA into two rings of shared-memory
-//           stages (a K stage is free once Q K^T has read it, a V stage once P V has)
+//           stages (a K stage is free once K Q^T has read it, a V stage once V^T P^T has)
 //   warp 3  loads the query rows of the current share with TMA
-//   warp 1  issues tcgen05.mma: S = Q K^T into one of two TMEM buffers, then
-//           O += P V with P read back from TMEM
-//   warps 4-11  two threads per query row, 64 keys of the tile each: read S
-//           from TMEM, apply the Eq. 5 mask on tiles that touch the block or a
-//           share boundary, running max with lazy rescaling of O, P = exp2(...)
-//           as two bf16 terms into TMEM
-// The 128 MMA rows are (block row i, head-in-group g) pairs of one kv head, so a
-// GQA group shares each K/V tile.  Every wait is bounded; an expired wait sets
-// SPACE_ST_TIMEOUT and the block drains and exits.
+//   warp 1  issues tcgen05.mma: S^T into one of two TMEM buffers, then O^T
+//   warps 4-11  two threads per key: read S^T from TMEM, apply the Eq. 5 mask
+//           on tiles that touch the block or a share boundary, P = exp2(score -
+//           reference) as two bf16 terms into shared memory for the second MMA.
+//           The per-row reference is set on a share's first tile and moved only
+//           when a score exceeds it by 2^60 (a block-wide vote per tile), so no
+//           per-tile row maximum is needed; row sums are kept per key and added
+//           across keys once per share.
+// Every wait is bounded; an expired wait sets SPACE_ST_TIMEOUT and the block
+// drains and exits.
 #include "common.cuh"
 #include <cuda.h>
 #include <math_constants.h>
@@ -31,12 +38,12 @@ constexpr int TILE_N = 128;            // keys per tile
 constexpr int ROWS = 128;              // MMA M
 constexpr int THREADS = 384;            // K, MMA, V, Q warps + 8 softmax warps
 constexpr uint64_t WAIT_NS = 1000000000ull;   // one second per wait
-constexpr float RESCALE_THRESHOLD = 8.f;
 
 struct AttnParams {
   CUtensorMap tm_q, tm_k, tm_v;
   int B, n_q, H_q, H_kv, G;
   int n_mblocks, rows_per_mb;          // query-row blocks per kv head; block rows i per block
+  int n_pad;                           // rows_per_mb * G rounded up to 16: N of the MMAs
   int n_groups;                        // thread-block groups (grid = n_groups * n_mblocks)
   int out_dtype;
   int64_t s_cap;
@@ -128,36 +135,6 @@ __device__ __forceinline__ void mma_ss(uint32_t d, uint64_t adesc, uint64_t bdes
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-      ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -172,12 +149,6 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
   d |= (uint64_t)2 << 61;
   return d;
 }
-// Instruction descriptor: bf16 x bf16 -> f32, M = 128.
-__host__ __device__ constexpr uint32_t instr_desc(int n, int b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) |
-         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(ROWS >> 4) << 24);
-}
-
 // ------------------------------------------------------------ work partition
 // Flat tile index space: sequence-major, then kv head, then tile.  Group g of
 // n_groups owns flat tiles [W*g/n_groups, W*(g+1)/n_groups).
@@ -226,23 +197,28 @@ __device__ __forceinline__ int group_of(long long f, long long W, long long NG) 
   return (int)(num / (unsigned long long)W);
 }
 
-template <int DH>
+// Shared-memory plan.  NB = number of 64-query blocks a thread block handles
+// (1: up to 64 query rows, 2: up to 128).
+template <int DH, int NB>
 struct Smem {
   static constexpr int HALVES = DH / 64;
   static constexpr int TILE_BYTES = TILE_N * DH * 2;         // one K or V tile
-  static constexpr int Q_BYTES = ROWS * DH * 2;
+  static constexpr int Q_ROWS = NB == 1 ? 64 : 112;          // query rows (with padding) per thread block
+  static constexpr int Q_BYTES = Q_ROWS * DH * 2;
+  static constexpr int P_PART = NB * TILE_N * 128;           // P_hi or P_lo: [block][key][64 queries] bf16
   static constexpr int K_STAGES = (DH == 128) ? 2 : 3;
-  static constexpr int V_STAGES = (DH == 128) ? 3 : 4;
+  static constexpr int V_STAGES = (DH == 128) ? (NB == 1 ? 3 : 2) : 4;
   static constexpr int Q_OFF = 0;
   static constexpr int K_OFF = Q_BYTES;
   static constexpr int V_OFF = K_OFF + K_STAGES * TILE_BYTES;
-  static constexpr int BAR_OFF = V_OFF + V_STAGES * TILE_BYTES;
-  // q_full, q_empty, k_full[], k_empty[], v_full[], v_empty[], s_full[2], p_ready[2], pv_done[2], drain
-  static constexpr int N_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 6 + 1;
+  static constexpr int P_OFF = V_OFF + V_STAGES * TILE_BYTES;
+  static constexpr int BAR_OFF = P_OFF + 2 * P_PART;
+  // q_full, q_empty, k_full[], k_empty[], v_full[], v_empty[], s_full[2], p_ready[2], pv_done, drain
+  static constexpr int N_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 4 + 1 + 1;
   static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;      // tmem base, abort flag
-  static constexpr int XMAX_OFF = MISC_OFF + 32;             // [2 parities][2 halves][ROWS] float
-  static constexpr int XSUM_OFF = XMAX_OFF + 2 * 2 * ROWS * 4;   // [2 halves][ROWS] float
-  static constexpr int TABLE_OFF = XSUM_OFF + 2 * ROWS * 4;  // seq_len[max_batch], prefix[max_batch+1]
+  static constexpr int MREF_OFF = MISC_OFF + 32;             // [2][128] float: reference maximum per query row
+  static constexpr int XQ_OFF = MREF_OFF + 2 * 128 * 4;          // [4 quarters][128] float: cross-lane reductions
+  static constexpr int TABLE_OFF = XQ_OFF + 4 * 128 * 4;     // seq_len[max_batch], prefix[max_batch+1]
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -250,19 +226,54 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-
-// The two softmax warps that share a TMEM lane quarter meet here (ids 1..4).
-__device__ __forceinline__ void pair_sync(int quarter) {
-  asm volatile("bar.sync %0, 64;" ::"r"(quarter + 1) : "memory");
+// Barrier over the 256 softmax threads (id 1); the second form also ORs a predicate.
+__device__ __forceinline__ void soft_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ bool soft_any(bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\t"
+      "bar.red.or.pred q, 1, 256, p;\n\tselp.b32 %0, 1, 0, q;\n\t}"
+      : "=r"(r) : "r"((uint32_t)pred) : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// Instruction descriptor: bf16 x bf16 -> f32, M = 128, N = n; a_mn / b_mn = operand is MN-major.
+__device__ __forceinline__ uint32_t instr_desc_rt(int n, int a_mn, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(ROWS >> 4) << 24);
 }
 
 // Warp roles
 constexpr int WARP_K = 0, WARP_MMA = 1, WARP_V = 2, WARP_Q = 3, WARP_SOFTMAX0 = 4;
+constexpr float OVER_THRESHOLD = 60.f;   // re-reference a query row when a score exceeds its reference by 2^60
 
-template <int DH>
+// The tile products are taken transposed: S^T = K Q^T (128 keys x N query rows)
+// and O^T += V^T P^T (head_dim x N), so the MMA N extent is the number of
+// query rows rounded up to 16 instead of a full 128-row tile, and one thread
+// owns one key of the tile (all 128 TMEM lanes carry work).
+template <int DH, int NB>
 __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_constant__ AttnParams p,
                                                              int max_batch) {
-  using S = Smem<DH>;
+  using S = Smem<DH, NB>;
   extern __shared__ __align__(1024) unsigned char sm[];
   const uint32_t sm_base = smem_u32(sm);
   const uint32_t bar0 = sm_base + S::BAR_OFF;
@@ -270,21 +281,21 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   constexpr int B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = B_KFULL + S::K_STAGES,
                 B_VFULL = B_KEMPTY + S::K_STAGES, B_VEMPTY = B_VFULL + S::V_STAGES,
                 B_SFULL = B_VEMPTY + S::V_STAGES, B_PREADY = B_SFULL + 2, B_PVDONE = B_SFULL + 4,
-                B_DRAIN = B_SFULL + 6;
+                B_DRAIN = B_SFULL + 5;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + S::MISC_OFF);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 4);
-  float* xmax = reinterpret_cast<float*>(sm + S::XMAX_OFF);
-  float* xsum = reinterpret_cast<float*>(sm + S::XSUM_OFF);
+  float* mref_buf = reinterpret_cast<float*>(sm + S::MREF_OFF);
+  float* xq = reinterpret_cast<float*>(sm + S::XQ_OFF);
   int* seq_len = reinterpret_cast<int*>(sm + S::TABLE_OFF);
   int* prefix = seq_len + max_batch;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int group = blockIdx.x / p.n_mblocks, mb = blockIdx.x % p.n_mblocks;
   const int i0 = mb * p.rows_per_mb;                       // first block row of this query-row block
-  // MMA rows that carry a real (block row, head) pair are 0 .. m_valid-1
+  // query rows (block row, head) handled here: 0 .. m_valid-1; N of the MMAs is n_pad
   const int m_valid = min(p.rows_per_mb, p.n_q - i0) * p.G;
-  const int n_quarters = (m_valid + 31) >> 5;              // TMEM lane quarters with live rows
-  const int n_soft = 64 * n_quarters;                      // softmax threads that take part
+  const int n_pad = p.n_pad;
+  const int n_chunks = n_pad >> 4;                         // 16-query column chunks
 
   // ---- set-up ------------------------------------------------------------
   pdl_launch_dependents();
@@ -296,13 +307,24 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     for (int s = 0; s < S::V_STAGES; ++s) { mbar_init(BAR(B_VFULL + s), 1); mbar_init(BAR(B_VEMPTY + s), 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(BAR(B_SFULL + i), 1);
-      mbar_init(BAR(B_PREADY + i), n_soft);
-      mbar_init(BAR(B_PVDONE + i), 1);
+      mbar_init(BAR(B_PREADY + i), 256);
     }
+    mbar_init(BAR(B_PVDONE), 1);
     mbar_init(BAR(B_DRAIN), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if (warp == WARP_MMA) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (warp == WARP_K && lane == 0)
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_k) : "memory");
+  if (warp == WARP_V && lane == 0)
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_v) : "memory");
+  if (warp == WARP_Q && lane == 0)
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_q) : "memory");
   pdl_wait();                                              // global memory from here on
   if (warp == WARP_SOFTMAX0) {
     // per-sequence tile counts and their running sum, 32 sequences per round
@@ -328,22 +350,12 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     }
     if (lane == 0) prefix[p.B] = carry;
   }
-  if (warp == WARP_MMA) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  if (warp == WARP_K && lane == 0)
-    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_k) : "memory");
-  if (warp == WARP_V && lane == 0)
-    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_v) : "memory");
-  if (warp == WARP_Q && lane == 0)
-    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_q) : "memory");
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t TM_S0 = tmem, TM_O = tmem + 2 * TILE_N;    // S buffers at columns 0 and 128, O at 256
+  // TMEM columns: S^T buffers at 0 and 128, O^T at 256 (n_pad <= 128 columns each)
+  const uint32_t TM_S0 = tmem, TM_O = tmem + 256;
 
   Partition part;
   part.init(seq_len, prefix, p.B, p.H_kv, p.n_q, group, p.n_groups);
@@ -388,13 +400,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     if (lane == 0) {
       uint32_t seg = 0;
       bool ok = true;
+      const uint32_t q_bytes = (uint32_t)n_pad * DH * 2;
       while (ok && part.next(sg)) {
         if (seg > 0) ok = mbar_wait(BAR(B_QEMPTY), (seg - 1) & 1, abort_flag, p.err, 3);
         if (!ok) break;
-        mbar_expect_tx(BAR(B_QFULL), S::Q_BYTES);
+        mbar_expect_tx(BAR(B_QFULL), q_bytes);
 #pragma unroll
         for (int hf = 0; hf < S::HALVES; ++hf)
-          tma_load_4d(sm_base + S::Q_OFF + hf * (ROWS * 128), &p.tm_q, BAR(B_QFULL), hf * 64,
+          tma_load_4d(sm_base + S::Q_OFF + hf * (n_pad * 128), &p.tm_q, BAR(B_QFULL), hf * 64,
                       sg.h * p.G, i0, sg.b);
         ++seg;
       }
@@ -403,30 +416,30 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   } else if (warp == WARP_MMA) {
     // ================= MMA issuer =========================================
     if (lane == 0) {
-      constexpr uint32_t IDESC_QK = instr_desc(TILE_N, 0);
-      constexpr uint32_t IDESC_PV = instr_desc(DH, 1);
+      const uint32_t idesc_qk = instr_desc_rt(n_pad, 0, 0);   // A = K tile (K-major), B = Q (K-major)
+      const uint32_t idesc_pv = instr_desc_rt(n_pad, 1, 1);   // A = V^T (d contiguous), B = P^T (queries contiguous)
       uint32_t gt = 0, seg = 0;
       bool ok = true;
-      // O += (P_hi + P_lo) V for flat tile g (first_in_seg: overwrite O)
+      // O^T += V^T (P_hi + P_lo)^T for flat tile g (first_in_seg: overwrite O^T)
       auto issue_pv = [&](uint32_t g, bool first_in_seg) -> bool {
-        const int s = g % S::V_STAGES, buf = g & 1;
+        const int s = g % S::V_STAGES;
         if (!mbar_wait(BAR(B_VFULL + s), (g / S::V_STAGES) & 1, abort_flag, p.err, 4)) return false;
-        if (!mbar_wait(BAR(B_PREADY + buf), (g >> 1) & 1, abort_flag, p.err, 5)) return false;
+        if (!mbar_wait(BAR(B_PREADY + (g & 1)), (g >> 1) & 1, abort_flag, p.err, 5)) return false;
         tc_fence_after();
         const uint32_t vsm = sm_base + S::V_OFF + s * S::TILE_BYTES;
-        const uint32_t ptm = TM_S0 + buf * TILE_N;
+        const uint32_t psm = sm_base + S::P_OFF;
 #pragma unroll
         for (int part_i = 0; part_i < 2; ++part_i) {        // P_hi, then P_lo
 #pragma unroll
           for (int kk = 0; kk < TILE_N / 16; ++kk) {
-            // V tile is MN-major: 64-wide d blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
-            const uint64_t bd = smem_desc(vsm + kk * 2048, TILE_N * 128, 1024);
-            mma_ts(TM_O, ptm + part_i * (TILE_N / 2) + kk * 8, bd, IDESC_PV,
-                   (first_in_seg && kk == 0 && part_i == 0) ? 0u : 1u);
+            // both operands: 64-wide blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
+            const uint64_t ad = smem_desc(vsm + kk * 2048, TILE_N * 128, 1024);
+            const uint64_t bd = smem_desc(psm + part_i * S::P_PART + kk * 2048, TILE_N * 128, 1024);
+            mma_ss(TM_O, ad, bd, idesc_pv, (first_in_seg && kk == 0 && part_i == 0) ? 0u : 1u);
           }
         }
         tc_commit(BAR(B_VEMPTY + s));
-        tc_commit(BAR(B_PVDONE + buf));
+        tc_commit(BAR(B_PVDONE));
         return true;
       };
       while (ok && part.next(sg)) {
@@ -434,17 +447,20 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         const int n = sg.t1 - sg.t0;
         for (int j = 0; j < n && ok; ++j, ++gt) {
           const int s = gt % S::K_STAGES, buf = gt & 1;
+          // S^T buffer `buf` was last read by the softmax of tile gt-2, whose
+          // p_ready this thread has already waited for when it issued that PV
           ok = mbar_wait(BAR(B_KFULL + s), (gt / S::K_STAGES) & 1, abort_flag, p.err, 7);
-          if (ok && gt >= 2) ok = mbar_wait(BAR(B_PVDONE + buf), ((gt >> 1) - 1) & 1, abort_flag, p.err, 8);
           if (!ok) break;
           tc_fence_after();
           const uint32_t qsm = sm_base + S::Q_OFF;
           const uint32_t ksm = sm_base + S::K_OFF + s * S::TILE_BYTES;
 #pragma unroll
           for (int kk = 0; kk < DH / 16; ++kk) {
-            const uint32_t off = (kk >> 2) * (ROWS * 128) + (kk & 3) * 32;   // 64-wide half, then 32 B per 16 elements
-            mma_ss(TM_S0 + buf * TILE_N, smem_desc(qsm + off, 16, 1024), smem_desc(ksm + off, 16, 1024),
-                   IDESC_QK, kk > 0 ? 1u : 0u);
+            // 64-wide half of d, then 32 bytes per 16 elements inside the swizzled row
+            const uint32_t koff = (kk >> 2) * (TILE_N * 128) + (kk & 3) * 32;
+            const uint32_t qoff = (kk >> 2) * (n_pad * 128) + (kk & 3) * 32;
+            mma_ss(TM_S0 + buf * 128, smem_desc(ksm + koff, 16, 1024), smem_desc(qsm + qoff, 16, 1024),
+                   idesc_qk, kk > 0 ? 1u : 0u);
           }
           tc_commit(BAR(B_SFULL + buf));
           tc_commit(BAR(B_KEMPTY + s));
@@ -458,122 +474,211 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       tc_commit(BAR(B_DRAIN));
       mbar_drain(BAR(B_DRAIN), 0);
     }
-  } else if ((warp & 3) < n_quarters) {
+  } else {
     // ================= softmax / epilogue ==================================
-    // Two threads per query row: `half` picks which 64 keys of a tile (and which
-    // half of the head dimension in the epilogue) this thread handles.
+    // One key of the tile per TMEM lane; two threads per key, which take the
+    // 16-query column chunks alternately (chunk c belongs to half c & 1).
+    constexpr int MAXCH = NB * 2;                          // chunks per thread at most
     const int quarter = warp & 3;                          // TMEM lane quarter this warp may touch
     const int half = (warp - WARP_SOFTMAX0) >> 2;
-    const int m = quarter * 32 + lane;                     // MMA row
-    const int il = m / p.G, g = m % p.G;
-    const int i = i0 + il;                                 // block row
-    const bool row_valid = m < m_valid;
-    const uint64_t mrow = row_valid ? p.mask[i] : 0ull;
+    const int kl = quarter * 32 + lane;                    // key within the tile; head-dim index in the epilogue
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-    const int sidx = half * (32 * n_quarters) + m;          // index among the n_soft softmax threads
     const float c = p.scale_log2;
-    constexpr int HC = TILE_N / 2;                         // keys per thread and tile
-    constexpr int OC = DH / 2;                             // output columns per thread
+    const uint32_t prow = sm_base + S::P_OFF + kl * 128;   // this key's 128-byte row in each P block
+    const uint32_t swz = (uint32_t)(kl & 7);
+    float lsum[MAXCH][16];                                 // this key's share of every row sum
     uint32_t gt = 0;
+    int mpar = 0;                                          // which copy of the references is current
+    const float* mref = mref_buf;
     // A failed (expired) wait does not leave the loops: every thread keeps the
-    // same control flow so that the pair barriers below always match up; once
-    // the abort flag is set all later waits return at once and the block drains.
+    // same control flow so that the block-wide barriers below always match up;
+    // once the abort flag is set all later waits return at once and the block drains.
     bool ok = true;
     while (part.next(sg)) {
       const int n_keys = sg.L + p.n_q;
-      float m_ref = -CUDART_INF_F, l_sum = 0.f;
+#pragma unroll
+      for (int u = 0; u < MAXCH; ++u)
+#pragma unroll
+        for (int e = 0; e < 16; ++e) lsum[u][e] = 0.f;
       for (int t = sg.t0; t < sg.t1; ++t, ++gt) {
         const int buf = gt & 1;
+        const bool first = (t == sg.t0);
         ok &= mbar_wait(BAR(B_SFULL + buf), (gt >> 1) & 1, abort_flag, p.err, 9);
         tc_fence_after();
-        const uint32_t ts = TM_S0 + buf * TILE_N + lane_addr;
-        uint32_t sreg[HC];
-#pragma unroll
-        for (int cc = 0; cc < HC / 32; ++cc) tmem_ld32(ts + half * HC + cc * 32, sreg + cc * 32);
-        tmem_wait_ld();
+        const uint32_t ts = TM_S0 + buf * 128 + lane_addr;
         const int lo = t * TILE_N;
         const int kt = ((t + 1) * TILE_N <= n_keys) ? lo : n_keys - TILE_N;
         const bool masked = (kt + TILE_N > sg.L) || (kt < lo);
-        float tmax = -CUDART_INF_F;
-        if (masked) {
+        const int key = kt + kl;
+        const bool key_ok = key >= lo;                     // keys before `lo` belong to the previous tile
+        const int jb = key - sg.L;                         // block key index when >= 0
+        // visibility of this key for the 16 query rows of chunk ch (bit e)
+        auto chunk_vis = [&](int ch) -> uint32_t {
+          if (!masked) return 0xFFFFu;
+          if (!key_ok) return 0u;
+          if (jb < 0) return 0xFFFFu;
+          uint32_t v = 0;
 #pragma unroll
-          for (int cidx = 0; cidx < HC; ++cidx) {
-            const int key = kt + half * HC + cidx;
-            bool vis = key >= lo;
-            if (key >= sg.L) vis = vis && ((mrow >> ((key - sg.L) & 63)) & 1ull);
-            const float v = vis ? __uint_as_float(sreg[cidx]) : -CUDART_INF_F;
-            sreg[cidx] = __float_as_uint(v);
-            tmax = fmaxf(tmax, v);
+          for (int e = 0; e < 16; ++e) {
+            const int q = ch * 16 + e;
+            const int i = i0 + q / p.G;
+            const uint64_t mr = (q < m_valid) ? p.mask[i] : 0ull;
+            v |= (uint32_t)((mr >> jb) & 1ull) << e;
           }
-        } else {
+          return v;
+        };
+        // ---- pass 0: does any score exceed its row's reference by 2^60? ------
+        bool over = first;
+        if (!first) {
 #pragma unroll
-          for (int cidx = 0; cidx < HC; ++cidx) tmax = fmaxf(tmax, __uint_as_float(sreg[cidx]));
+          for (int u = 0; u < MAXCH; ++u) {
+            const int ch = 2 * u + half;
+            if (ch < n_chunks) {
+              uint32_t sr[16];
+              tmem_ld16(ts + ch * 16, sr);
+              tmem_wait_ld();
+              const uint32_t vis = chunk_vis(ch);
+              const float4* mr4 = reinterpret_cast<const float4*>(mref + ch * 16);
+#pragma unroll
+              for (int e4 = 0; e4 < 4; ++e4) {
+                const float4 mr = mr4[e4];
+                const float mm[4] = {mr.x, mr.y, mr.z, mr.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float v = fmaf(__uint_as_float(sr[e4 * 4 + e]), c, -mm[e]);
+                  over |= ((vis >> (e4 * 4 + e)) & 1u) && !(v <= OVER_THRESHOLD);
+                }
+              }
+            }
+          }
         }
-        // the row maximum needs the other half's keys; the pair barrier also orders
-        // both threads' reads of S before either overwrites it with P
-        float* xm = xmax + (gt & 1) * (2 * ROWS);
-        xm[half * ROWS + m] = tmax;
-        pair_sync(quarter);
-        tmax = fmaxf(tmax, xm[(half ^ 1) * ROWS + m]);
-        tmax *= c;                                         // c > 0
-        if (!(tmax > -CUDART_INF_F)) tmax = -CUDART_INF_F; // also catches NaN
-        const bool first = (t == sg.t0);
-        const bool need = !first && (tmax > m_ref + RESCALE_THRESHOLD);
-        if (first) m_ref = tmax;
-        if (__any_sync(0xFFFFFFFFu, need)) {
-          // lazy rescale of this row's accumulator; PV of the previous tile must be done
-          ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 10);
-          tc_fence_after();
-          const float m_new = fmaxf(m_ref, tmax);
-          const float f = (m_ref > -CUDART_INF_F) ? fast_exp2(m_ref - m_new) : 0.f;
-          l_sum *= f;
-          m_ref = m_new;
-#pragma unroll 1
-          for (int cc = 0; cc < OC / 32; ++cc) {
-            uint32_t o[32];
-            const uint32_t ta = TM_O + lane_addr + half * OC + cc * 32;
-            tmem_ld32(ta, o);
+        if (soft_any(over)) {
+          // ---- re-reference: per query row maximum over the 128 keys of this tile
+#pragma unroll
+          for (int u = 0; u < MAXCH; ++u) {
+            const int ch = 2 * u + half;
+            if (ch < n_chunks) {
+              uint32_t sr[16];
+              tmem_ld16(ts + ch * 16, sr);
+              tmem_wait_ld();
+              const uint32_t vis = chunk_vis(ch);
+#pragma unroll
+              for (int e = 0; e < 16; ++e) {
+                float v = ((vis >> e) & 1u) ? __uint_as_float(sr[e]) : -CUDART_INF_F;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+                if (lane == 0) xq[quarter * 128 + ch * 16 + e] = v;
+              }
+            }
+          }
+          soft_sync();
+          // PV of the previous tile must be done before O^T is rescaled
+          if (!first) {
+            ok &= mbar_wait(BAR(B_PVDONE), (gt - 1) & 1, abort_flag, p.err, 10);
+            tc_fence_after();
+          }
+#pragma unroll
+          for (int u = 0; u < MAXCH; ++u) {
+            const int ch = 2 * u + half;
+            if (ch < n_chunks) {
+              float f[16];
+#pragma unroll
+              for (int e = 0; e < 16; ++e) {
+                const int q = ch * 16 + e;
+                float tm = fmaxf(fmaxf(xq[q], xq[128 + q]), fmaxf(xq[256 + q], xq[384 + q])) * c;
+                if (!(tm > -CUDART_INF_F)) tm = -CUDART_INF_F;      // also catches NaN
+                const float m_old = first ? -CUDART_INF_F : mref[q];
+                const float m_new = fmaxf(m_old, tm);
+                f[e] = (m_old > -CUDART_INF_F) ? fast_exp2(m_old - m_new) : 0.f;
+                lsum[u][e] *= f[e];
+                mref_buf[(mpar ^ 1) * 128 + q] = m_new;     // every thread of the chunk writes the same value
+              }
+              if (!first) {
+                uint32_t o[16];
+                tmem_ld16(TM_O + lane_addr + ch * 16, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f[e]);
+                tmem_st16(TM_O + lane_addr + ch * 16, o);
+              }
+            }
+          }
+          if (!first) tmem_wait_st();
+          mpar ^= 1;
+          mref = mref_buf + mpar * 128;
+          soft_sync();                                      // new references visible to every thread
+        }
+        // the P buffer is free once the PV product of the previous tile has read it
+        if (gt > 0) ok &= mbar_wait(BAR(B_PVDONE), (gt - 1) & 1, abort_flag, p.err, 11);
+        // ---- pass 1: P = exp2(score - reference) as P_hi + P_lo (two bf16 terms:
+        // bf16 alone leaves an output error near 1e-2 of the output RMS)
+#pragma unroll
+        for (int u = 0; u < MAXCH; ++u) {
+          const int ch = 2 * u + half;
+          if (ch < n_chunks) {
+            uint32_t sr[16];
+            tmem_ld16(ts + ch * 16, sr);
             tmem_wait_ld();
+            const uint32_t vis = chunk_vis(ch);
+            const float4* mr4 = reinterpret_cast<const float4*>(mref + ch * 16);
+            uint32_t hi[8], lw[8];
 #pragma unroll
-            for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * f);
-            tmem_st32(ta, o);
+            for (int e4 = 0; e4 < 4; ++e4) {
+              const float4 mr = mr4[e4];
+              const float mm[4] = {mr.x, mr.y, mr.z, mr.w};
+              float pv[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float m_use = (mm[e] > -CUDART_INF_F) ? mm[e] : 0.f;
+                const float x = fast_exp2(fmaf(__uint_as_float(sr[e4 * 4 + e]), c, -m_use));
+                pv[e] = ((vis >> (e4 * 4 + e)) & 1u) ? x : 0.f;
+                lsum[u][e4 * 4 + e] += pv[e];
+              }
+#pragma unroll
+              for (int e2 = 0; e2 < 2; ++e2) {
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(pv[2 * e2], pv[2 * e2 + 1]);   // .x = lower query row
+                const float2 hf = __bfloat1622float2(h2);
+                const __nv_bfloat162 l2 = __floats2bfloat162_rn(pv[2 * e2] - hf.x, pv[2 * e2 + 1] - hf.y);
+                hi[e4 * 2 + e2] = *reinterpret_cast<const uint32_t*>(&h2);
+                lw[e4 * 2 + e2] = *reinterpret_cast<const uint32_t*>(&l2);
+              }
+            }
+            // P^T rows are keys; a row holds 64 query rows as eight 16-byte pieces,
+            // piece j stored at j ^ (key & 7) (128-byte swizzle)
+            const uint32_t blk = prow + (uint32_t)(ch >> 2) * (TILE_N * 128);
+            const uint32_t j0 = (uint32_t)(ch & 3) * 2;
+            st_shared_v4(blk + (((j0) ^ swz) << 4), hi[0], hi[1], hi[2], hi[3]);
+            st_shared_v4(blk + (((j0 + 1) ^ swz) << 4), hi[4], hi[5], hi[6], hi[7]);
+            st_shared_v4(blk + S::P_PART + (((j0) ^ swz) << 4), lw[0], lw[1], lw[2], lw[3]);
+            st_shared_v4(blk + S::P_PART + (((j0 + 1) ^ swz) << 4), lw[4], lw[5], lw[6], lw[7]);
           }
-          tmem_wait_st();
         }
-        const float m_use = (m_ref > -CUDART_INF_F) ? m_ref : 0.f;
-        // P = P_hi + P_lo, two bf16 terms: bf16 alone (8 significant bits) leaves
-        // an output error near 1e-2 of the output RMS.  P_hi occupies columns
-        // 0..63 of the S buffer, P_lo columns 64..127 (two keys per column).
-        uint32_t lreg[HC / 2];
-#pragma unroll
-        for (int x = 0; x < HC / 2; ++x) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[2 * x]), c, -m_use));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[2 * x + 1]), c, -m_use));
-          l_sum += p0 + p1;
-          const __nv_bfloat162 hi = __floats2bfloat162_rn(p0, p1);   // .x (low half) = even key
-          const float2 hf = __bfloat1622float2(hi);
-          const __nv_bfloat162 lw = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
-          sreg[x] = *reinterpret_cast<const uint32_t*>(&hi);
-          lreg[x] = *reinterpret_cast<const uint32_t*>(&lw);
-        }
-        tmem_st32(ts + half * (HC / 2), sreg);
-        tmem_st32(ts + TILE_N / 2 + half * (HC / 2), lreg);
-        tmem_wait_st();
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core
         tc_fence_before();
         mbar_arrive(BAR(B_PREADY + buf));
       }
       // ---- end of share: final output or partial ---------------------------
-      ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 11);
+      // row sums: add this key's share over the 128 keys (lanes, then quarters)
+#pragma unroll
+      for (int u = 0; u < MAXCH; ++u) {
+        const int ch = 2 * u + half;
+        if (ch < n_chunks) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            float v = lsum[u][e];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+            if (lane == 0) xq[quarter * 128 + ch * 16 + e] = v;
+          }
+        }
+      }
+      soft_sync();
+      ok &= mbar_wait(BAR(B_PVDONE), (gt - 1) & 1, abort_flag, p.err, 12);
       tc_fence_after();
-      xsum[half * ROWS + m] = l_sum;
-      pair_sync(quarter);
-      const float l_tot = l_sum + xsum[(half ^ 1) * ROWS + m];
       const bool whole = (sg.t0 == 0 && sg.t1 == sg.T);
-      const int hq = sg.h * p.G + g;
       const int item = sg.b * p.H_kv + sg.h;
       float* pslot = p.part + ((size_t)(item + group) * p.n_mblocks + mb) * (ROWS * (DH + 2));
-      const float inv = (l_tot > 0.f) ? 1.f / l_tot : 0.f;
-      if (sidx == 0 && ok) {
+      if (threadIdx.x == WARP_SOFTMAX0 * 32 && ok) {
         // how this (sequence, head) was cut: first group and number of groups,
         // read by attn_merge_kernel (every group of the cut writes the same pair)
         int2 d = make_int2(group, 1);
@@ -586,53 +691,43 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         }
         p.desc[(size_t)item * p.n_mblocks + mb] = d;
       }
-#pragma unroll 1
-      for (int cc = 0; cc < OC / 32; ++cc) {
-        uint32_t o[32];
-        const int col = half * OC + cc * 32;
-        tmem_ld32(TM_O + lane_addr + col, o);
-        tmem_wait_ld();
-        if (!row_valid || !ok) continue;
-        if (whole) {
-          const size_t off = (((size_t)sg.b * p.n_q + i) * p.H_q + hq) * DH + col;
-          if (p.out_dtype == SPACE_DTYPE_F32) {
-            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off);
+      // O^T: lane = head-dim index, column = query row.  A warp writes 32
+      // consecutive floats of one output row per store.
+      const bool d_ok = kl < DH;                            // lanes 64..127 repeat 0..63 when head_dim is 64
 #pragma unroll
-            for (int x = 0; x < 8; ++x)
-              dst[x] = make_float4(__uint_as_float(o[4 * x]) * inv, __uint_as_float(o[4 * x + 1]) * inv,
-                                   __uint_as_float(o[4 * x + 2]) * inv, __uint_as_float(o[4 * x + 3]) * inv);
-          } else {
-            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off);
+      for (int u = 0; u < MAXCH; ++u) {
+        const int ch = 2 * u + half;
+        if (ch < n_chunks) {
+          uint32_t o[16];
+          tmem_ld16(TM_O + lane_addr + ch * 16, o);
+          tmem_wait_ld();
 #pragma unroll
-            for (int x = 0; x < 4; ++x) {
-              uint32_t w[4];
-#pragma unroll
-              for (int y = 0; y < 4; ++y) {
-                const __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(o[8 * x + 2 * y]) * inv,
-                                                                __uint_as_float(o[8 * x + 2 * y + 1]) * inv);
-                w[y] = *reinterpret_cast<const uint32_t*>(&pk);
+          for (int e = 0; e < 16; ++e) {
+            const int q = ch * 16 + e;
+            if (q < m_valid && d_ok && ok) {
+              const float l_tot = (xq[q] + xq[128 + q]) + (xq[256 + q] + xq[384 + q]);
+              const float val = __uint_as_float(o[e]);
+              if (whole) {
+                const int i = i0 + q / p.G, hq = sg.h * p.G + q % p.G;
+                const size_t off = (((size_t)sg.b * p.n_q + i) * p.H_q + hq) * DH + kl;
+                const float r = val / l_tot;
+                if (p.out_dtype == SPACE_DTYPE_F32) reinterpret_cast<float*>(p.out)[off] = r;
+                else reinterpret_cast<__nv_bfloat16*>(p.out)[off] = __float2bfloat16_rn(r);
+                if (kl == 0 && p.lse)
+                  p.lse[((size_t)sg.b * p.H_q + hq) * p.n_q + i] = (mref[q] + log2f(l_tot)) * 0.6931471805599453f;
+              } else {
+                pslot[(size_t)q * DH + kl] = val;
+                if (kl == 0) {
+                  pslot[ROWS * DH + q] = mref[q];
+                  pslot[ROWS * DH + ROWS + q] = l_tot;
+                }
               }
-              dst[x] = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }
-        } else {
-          float4* dst = reinterpret_cast<float4*>(pslot + (size_t)m * DH + col);
-#pragma unroll
-          for (int x = 0; x < 8; ++x)
-            dst[x] = make_float4(__uint_as_float(o[4 * x]), __uint_as_float(o[4 * x + 1]),
-                                 __uint_as_float(o[4 * x + 2]), __uint_as_float(o[4 * x + 3]));
         }
       }
       tc_fence_before();
-      if (row_valid && half == 0 && ok) {
-        if (whole) {
-          if (p.lse)
-            p.lse[((size_t)sg.b * p.H_q + hq) * p.n_q + i] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
-        } else {
-          pslot[ROWS * DH + m] = m_ref;
-          pslot[ROWS * DH + ROWS + m] = l_tot;
-        }
-      }
+      soft_sync();                                          // xq and mref are reused by the next share
     }
   }
 
@@ -736,7 +831,7 @@ int make_map(CUtensorMap* tm, const void* base, const cuuint64_t dims[4], const 
 void plan(const space_config* cfg, int sm_count, int k, AttnPlanHost* pl) {
   const int G = cfg->n_q_heads / cfg->n_kv_heads;
   const int n_q = (k + 1) * (k + 1);
-  const int max_rows = ROWS / G;                            // block rows one MMA tile can hold
+  const int max_rows = 112 / G;                             // (block row, head) pairs per thread block: at most 112
   pl->n_mblocks = (n_q + max_rows - 1) / max_rows;
   pl->rows_per_mblock = (n_q + pl->n_mblocks - 1) / pl->n_mblocks;
   int groups = sm_count / pl->n_mblocks;
@@ -744,9 +839,16 @@ void plan(const space_config* cfg, int sm_count, int k, AttnPlanHost* pl) {
   pl->n_ctas = groups * pl->n_mblocks;
 }
 
-template <int DH>
+template <int DH, int NB>
 size_t smem_bytes(int max_batch) {
-  return Smem<DH>::TABLE_OFF + (size_t)(2 * max_batch + 2) * sizeof(int);
+  return Smem<DH, NB>::TABLE_OFF + (size_t)(2 * max_batch + 2) * sizeof(int);
+}
+
+template <int DH, int NB>
+cudaError_t launch_main(const AttnParams& p, int n_ctas, int max_batch, cudaStream_t st) {
+  const size_t sm = smem_bytes<DH, NB>(max_batch);
+  cudaFuncSetAttribute(attn_tc_kernel<DH, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+  return launch_pdl(attn_tc_kernel<DH, NB>, dim3(n_ctas), dim3(THREADS), sm, st, p, max_batch);
 }
 
 }  // namespace
@@ -777,6 +879,7 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   p.H_q = cfg.n_q_heads; p.H_kv = cfg.n_kv_heads; p.G = p.H_q / p.H_kv;
   p.n_mblocks = pl.n_mblocks; p.rows_per_mb = pl.rows_per_mblock;
   p.n_groups = pl.n_ctas / pl.n_mblocks;
+  p.n_pad = ((pl.rows_per_mblock * p.G + 15) / 16) * 16;
   p.out_dtype = a->out_dtype; p.s_cap = cfg.s_cap;
   p.scale_log2 = a->scale * 1.4426950408889634f;
   p.kv_len = a->kv_len; p.out = a->out; p.lse = a->lse; p.status = a->status;
@@ -785,7 +888,7 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   for (int i = 0; i < SPACE_MAX_ROWS; ++i) p.mask[i] = mask_rows[i];
 
   // TMA descriptors, rebuilt only when a base pointer or a stride changes
-  const int64_t key[8] = {a->kv_stride_b, a->kv_stride_h, a->kv_stride_s, a->batch, p.n_q, 0, 0, 0};
+  const int64_t key[8] = {a->kv_stride_b, a->kv_stride_h, a->kv_stride_s, a->batch, p.n_q, p.n_pad, 0, 0};
   if (ctx->tm_q_ptr != a->q || ctx->tm_k_ptr != a->k_cache || ctx->tm_v_ptr != a->v_cache ||
       memcmp(key, ctx->tm_key, sizeof(key)) != 0) {
     const cuuint64_t kd[4] = {(cuuint64_t)DH, (cuuint64_t)cfg.s_cap, (cuuint64_t)p.H_kv, (cuuint64_t)a->batch};
@@ -794,7 +897,7 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
     const cuuint32_t kb[4] = {64, TILE_N, 1, 1};
     const cuuint64_t qd[4] = {(cuuint64_t)DH, (cuuint64_t)p.H_q, (cuuint64_t)p.n_q, (cuuint64_t)a->batch};
     const cuuint64_t qs[3] = {(cuuint64_t)DH * 2, (cuuint64_t)p.H_q * DH * 2, (cuuint64_t)p.n_q * p.H_q * DH * 2};
-    const cuuint32_t qb[4] = {64, (cuuint32_t)p.G, (cuuint32_t)(ROWS / p.G), 1};
+    const cuuint32_t qb[4] = {64, (cuuint32_t)p.G, (cuuint32_t)(p.n_pad / p.G), 1};
     int rc = make_map((CUtensorMap*)ctx->tm_k, a->k_cache, kd, ks, kb);
     if (rc == SPACE_OK) rc = make_map((CUtensorMap*)ctx->tm_v, a->v_cache, kd, ks, kb);
     if (rc == SPACE_OK) rc = make_map((CUtensorMap*)ctx->tm_q, a->q, qd, qs, qb);
@@ -808,28 +911,19 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
 
   const int m_valid_max = p.rows_per_mb * p.G;
   const dim3 mgrid(a->batch * p.H_kv * p.n_mblocks, (m_valid_max * (DH / 4) + 127) / 128);
-  if (DH == 128) {
-    const size_t sm = smem_bytes<128>(cfg.max_batch);
-    cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    {
-      ProfScope ps(ctx, SPACE_K_ATTN, st);
-      launch_pdl(attn_tc_kernel<128>, dim3(pl.n_ctas), dim3(THREADS), sm, st, p, cfg.max_batch);
+  {
+    ProfScope ps(ctx, SPACE_K_ATTN, st);
+    const bool wide = p.n_pad > 64;
+    if (DH == 128) {
+      if (wide) launch_main<128, 2>(p, pl.n_ctas, cfg.max_batch, st); else launch_main<128, 1>(p, pl.n_ctas, cfg.max_batch, st);
+    } else {
+      if (wide) launch_main<64, 2>(p, pl.n_ctas, cfg.max_batch, st); else launch_main<64, 1>(p, pl.n_ctas, cfg.max_batch, st);
     }
-    {
-      ProfScope ps(ctx, SPACE_K_MERGE, st);
-      launch_pdl(attn_merge_kernel<128>, mgrid, dim3(128), 0, st, p);
-    }
-  } else {
-    const size_t sm = smem_bytes<64>(cfg.max_batch);
-    cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    {
-      ProfScope ps(ctx, SPACE_K_ATTN, st);
-      launch_pdl(attn_tc_kernel<64>, dim3(pl.n_ctas), dim3(THREADS), sm, st, p, cfg.max_batch);
-    }
-    {
-      ProfScope ps(ctx, SPACE_K_MERGE, st);
-      launch_pdl(attn_merge_kernel<64>, mgrid, dim3(128), 0, st, p);
-    }
+  }
+  {
+    ProfScope ps(ctx, SPACE_K_MERGE, st);
+    if (DH == 128) launch_pdl(attn_merge_kernel<128>, mgrid, dim3(128), 0, st, p);
+    else launch_pdl(attn_merge_kernel<64>, mgrid, dim3(128), 0, st, p);
   }
   ctx->launches += 2;
   return cuda_ok(cudaGetLastError());

@@ -142,9 +142,20 @@ __device__ Stat scan_chunk(const T* row, int begin, int end, float c, float inv_
   Stat st = stat_empty();
   if (VECTOR) {
     constexpr int N = Vec<T>::N;
+    constexpr int U = 4;                                    // independent 16-byte loads in flight per thread
     // begin is a multiple of N; the tail shorter than N is handled one by one
     const int full_end = begin + ((end - begin) / N) * N;
-    for (int x = begin + threadIdx.x * N; x < full_end; x += blockDim.x * N) {
+    const int stride = blockDim.x * N;
+    int x = begin + threadIdx.x * N;
+    for (; x + (U - 1) * stride < full_end; x += U * stride) {
+      float v[U][N];
+#pragma unroll
+      for (int u = 0; u < U; ++u) Vec<T>::load(row + x + u * stride, v[u]);
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        fold<N, GUMBEL>(st, v[u], x + u * stride, c, inv_t, exclude, key0, key1, purpose, seq, pos);
+    }
+    for (; x < full_end; x += stride) {
       float v[N];
       Vec<T>::load(row + x, v);
       fold<N, GUMBEL>(st, v, x, c, inv_t, exclude, key0, key1, purpose, seq, pos);
@@ -497,7 +508,7 @@ int launch_verify(space_ctx* ctx, const space_verify_args* a, cudaStream_t st) {
   const int64_t all_bytes = (int64_t)a->batch * p.n_q * a->vocab * esz;
   if (a->mode == SPACE_MODE_GREEDY && all_bytes <= SPACE_FUSED_MAX_BYTES) {
     const int rows_all = a->batch * p.n_q;
-    int nc = (2 * ctx->sm_count + rows_all - 1) / rows_all;
+    int nc = ctx->sm_count / rows_all;                      // about one block per SM: few arrivals, four loads in flight
     const int min_chunk = SPACE_VERIFY_THREADS * vec;
     const int max_nc = (a->vocab + min_chunk - 1) / min_chunk;
     if (nc > max_nc) nc = max_nc;
@@ -515,11 +526,12 @@ int launch_verify(space_ctx* ctx, const space_verify_args* a, cudaStream_t st) {
     ctx->launches += 1;
     return cuda_ok(cudaGetLastError());
   }
-  // enough chunks to put about two blocks on every SM, but no chunk below two
-  // sweeps of a block
+  // enough chunks to put about eight blocks on every SM (many loads in flight, and
+  // the Gumbel rows of sampling mode spread over the GPU), but no chunk below
+  // four sweeps of a block
   const int rows = a->batch * (a->k + 1);
-  int nc = (2 * ctx->sm_count + rows - 1) / rows;
-  const int min_chunk = SPACE_VERIFY_THREADS * vec * 2;
+  int nc = (8 * ctx->sm_count + rows - 1) / rows;
+  const int min_chunk = SPACE_VERIFY_THREADS * vec * 4;
   const int max_nc = (a->vocab + min_chunk - 1) / min_chunk;
   if (nc > max_nc) nc = max_nc;
   if (nc > SPACE_VERIFY_MAX_CHUNKS) nc = SPACE_VERIFY_MAX_CHUNKS;
