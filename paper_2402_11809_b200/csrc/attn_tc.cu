@@ -87,7 +87,7 @@ __device__ __forceinline__ uint64_t global_ns() {
 }
 // Bounded wait (WAIT_NS of wall time).  Returns false when the limit expired or
 // another thread of the block gave up; the first expiry records its site.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int* err, int site) {
   if (*abort_flag) return mbar_try(bar, parity);            // draining: never block
   uint64_t t0 = 0;
@@ -105,7 +105,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 // Bounded wait without the abort protocol (used while draining before exit).
-__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+__device__ __noinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
   uint64_t t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try(bar, parity)) return;
@@ -218,7 +218,8 @@ struct Smem {
   static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;      // tmem base, abort flag
   static constexpr int MREF_OFF = MISC_OFF + 32;             // [2][128] float: reference maximum per query row
   static constexpr int XQ_OFF = MREF_OFF + 2 * 128 * 4;          // [4 quarters][128] float: cross-lane reductions
-  static constexpr int TABLE_OFF = XQ_OFF + 4 * 128 * 4;     // seq_len[max_batch], prefix[max_batch+1]
+  static constexpr int FQ_OFF = XQ_OFF + 4 * 128 * 4;        // [128] float: rescale factors / final row sums
+  static constexpr int TABLE_OFF = FQ_OFF + 128 * 4;         // seq_len[max_batch], prefix[max_batch+1]
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -262,6 +263,64 @@ __device__ __forceinline__ uint32_t instr_desc_rt(int n, int a_mn, int b_mn) {
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(ROWS >> 4) << 24);
 }
 
+// ---- pieces of the softmax threads that are off the hot path; kept out of line
+// so that the per-tile loop stays small enough for the instruction cache ----
+
+// Which of the 16 query rows of chunk `ch` see block key `jb` (bit e = row ch*16+e).
+__device__ __noinline__ uint32_t block_key_visibility(const uint64_t* mask, int ch, int jb, int i0, int G,
+                                                      int m_valid) {
+  uint32_t v = 0;
+#pragma unroll 1
+  for (int e = 0; e < 16; ++e) {
+    const int q = ch * 16 + e;
+    if (q < m_valid) v |= (uint32_t)((mask[i0 + q / G] >> jb) & 1ull) << e;
+  }
+  return v;
+}
+
+// Maximum over the 32 keys of this warp for each of the 16 query rows of a chunk
+// (visible entries only); lane 0 stores them at dst[0..15].
+__device__ __noinline__ void chunk_key_max(uint32_t taddr, uint32_t vis, float* dst) {
+  uint32_t sr[16];
+  tmem_ld16(taddr, sr);
+  tmem_wait_ld();
+#pragma unroll
+  for (int e = 0; e < 16; ++e) {
+    // order-preserving map float -> int so that one integer warp reduction does it
+    const int bits = ((vis >> e) & 1u) ? (int)sr[e] : (int)0xFF800000u;      // -inf when not visible
+    const int key = bits ^ ((bits >> 31) & 0x7FFFFFFF);
+    const int mx = __reduce_max_sync(0xFFFFFFFFu, key);
+    if ((threadIdx.x & 31) == 0) dst[e] = __int_as_float(mx ^ ((mx >> 31) & 0x7FFFFFFF));
+  }
+}
+
+// New reference for the 16 query rows of a chunk from the four quarter maxima in
+// xq; writes the reference to mnew[0..15] and the factor old -> new to fq[0..15].
+// Every thread of the chunk computes the same values (identical writes).
+__device__ __noinline__ void chunk_new_reference(const float* xq, const float* mold, float* mnew, float* fq,
+                                                 float c, bool first) {
+#pragma unroll 1
+  for (int e = 0; e < 16; ++e) {
+    float tm = fmaxf(fmaxf(xq[e], xq[128 + e]), fmaxf(xq[256 + e], xq[384 + e])) * c;
+    if (!(tm > -CUDART_INF_F)) tm = -CUDART_INF_F;          // also catches NaN
+    const float m_old = first ? -CUDART_INF_F : mold[e];
+    const float m_new = fmaxf(m_old, tm);
+    mnew[e] = m_new;
+    fq[e] = (m_old > -CUDART_INF_F) ? fast_exp2(m_old - m_new) : 0.f;
+  }
+}
+
+// O^T[lane][16 columns] *= fq[0..15]
+__device__ __noinline__ void chunk_rescale(uint32_t taddr, const float* fq) {
+  uint32_t o[16];
+  tmem_ld16(taddr, o);
+  tmem_wait_ld();
+#pragma unroll
+  for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * fq[e]);
+  tmem_st16(taddr, o);
+  tmem_wait_st();
+}
+
 // Warp roles
 constexpr int WARP_K = 0, WARP_MMA = 1, WARP_V = 2, WARP_Q = 3, WARP_SOFTMAX0 = 4;
 constexpr float OVER_THRESHOLD = 60.f;   // re-reference a query row when a score exceeds its reference by 2^60
@@ -286,6 +345,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 4);
   float* mref_buf = reinterpret_cast<float*>(sm + S::MREF_OFF);
   float* xq = reinterpret_cast<float*>(sm + S::XQ_OFF);
+  float* fq = reinterpret_cast<float*>(sm + S::FQ_OFF);
   int* seq_len = reinterpret_cast<int*>(sm + S::TABLE_OFF);
   int* prefix = seq_len + max_batch;
 
@@ -478,15 +538,18 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     // ================= softmax / epilogue ==================================
     // One key of the tile per TMEM lane; two threads per key, which take the
     // 16-query column chunks alternately (chunk c belongs to half c & 1).
-    constexpr int MAXCH = NB * 2;                          // chunks per thread at most
+    constexpr int MAXCH = NB == 1 ? 2 : 4;                 // chunks per thread at most
     const int quarter = warp & 3;                          // TMEM lane quarter this warp may touch
     const int half = (warp - WARP_SOFTMAX0) >> 2;
     const int kl = quarter * 32 + lane;                    // key within the tile; head-dim index in the epilogue
+    const int sidx = half * 128 + kl;                      // index among the 256 softmax threads
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const float c = p.scale_log2;
     const uint32_t prow = sm_base + S::P_OFF + kl * 128;   // this key's 128-byte row in each P block
     const uint32_t swz = (uint32_t)(kl & 7);
+    float* xs = reinterpret_cast<float*>(sm + S::P_OFF);   // end-of-share scratch over the idle P buffer
     float lsum[MAXCH][16];                                 // this key's share of every row sum
+    uint32_t visb[MAXCH];                                  // per chunk: which of its 16 query rows see this key
     uint32_t gt = 0;
     int mpar = 0;                                          // which copy of the references is current
     const float* mref = mref_buf;
@@ -508,25 +571,18 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         const uint32_t ts = TM_S0 + buf * 128 + lane_addr;
         const int lo = t * TILE_N;
         const int kt = ((t + 1) * TILE_N <= n_keys) ? lo : n_keys - TILE_N;
-        const bool masked = (kt + TILE_N > sg.L) || (kt < lo);
         const int key = kt + kl;
-        const bool key_ok = key >= lo;                     // keys before `lo` belong to the previous tile
         const int jb = key - sg.L;                         // block key index when >= 0
-        // visibility of this key for the 16 query rows of chunk ch (bit e)
-        auto chunk_vis = [&](int ch) -> uint32_t {
-          if (!masked) return 0xFFFFu;
-          if (!key_ok) return 0u;
-          if (jb < 0) return 0xFFFFu;
-          uint32_t v = 0;
+        // visibility of this thread's key: keys before `lo` belong to the previous
+        // tile; cached keys are seen by every row; block keys by the Eq. 5 mask
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const int q = ch * 16 + e;
-            const int i = i0 + q / p.G;
-            const uint64_t mr = (q < m_valid) ? p.mask[i] : 0ull;
-            v |= (uint32_t)((mr >> jb) & 1ull) << e;
-          }
-          return v;
-        };
+        for (int u = 0; u < MAXCH; ++u) {
+          const int ch = 2 * u + half;
+          uint32_t v = 0xFFFFu;
+          if (key < lo) v = 0u;
+          else if (jb >= 0 && ch < n_chunks) v = block_key_visibility(p.mask, ch, jb, i0, p.G, m_valid);
+          visb[u] = v;
+        }
         // ---- pass 0: does any score exceed its row's reference by 2^60? ------
         bool over = first;
         if (!first) {
@@ -537,8 +593,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
               uint32_t sr[16];
               tmem_ld16(ts + ch * 16, sr);
               tmem_wait_ld();
-              const uint32_t vis = chunk_vis(ch);
               const float4* mr4 = reinterpret_cast<const float4*>(mref + ch * 16);
+              float worst = -CUDART_INF_F;
 #pragma unroll
               for (int e4 = 0; e4 < 4; ++e4) {
                 const float4 mr = mr4[e4];
@@ -546,9 +602,12 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                   const float v = fmaf(__uint_as_float(sr[e4 * 4 + e]), c, -mm[e]);
-                  over |= ((vis >> (e4 * 4 + e)) & 1u) && !(v <= OVER_THRESHOLD);
+                  const bool seen = (visb[u] >> (e4 * 4 + e)) & 1u;
+                  worst = fmaxf(worst, seen ? v : -CUDART_INF_F);
+                  over |= seen && (v != v);                 // NaN
                 }
               }
+              over |= worst > OVER_THRESHOLD;
             }
           }
         }
@@ -557,19 +616,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
 #pragma unroll
           for (int u = 0; u < MAXCH; ++u) {
             const int ch = 2 * u + half;
-            if (ch < n_chunks) {
-              uint32_t sr[16];
-              tmem_ld16(ts + ch * 16, sr);
-              tmem_wait_ld();
-              const uint32_t vis = chunk_vis(ch);
-#pragma unroll
-              for (int e = 0; e < 16; ++e) {
-                float v = ((vis >> e) & 1u) ? __uint_as_float(sr[e]) : -CUDART_INF_F;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
-                if (lane == 0) xq[quarter * 128 + ch * 16 + e] = v;
-              }
-            }
+            if (ch < n_chunks) chunk_key_max(ts + ch * 16, visb[u], xq + quarter * 128 + ch * 16);
           }
           soft_sync();
           // PV of the previous tile must be done before O^T is rescaled
@@ -581,29 +628,18 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           for (int u = 0; u < MAXCH; ++u) {
             const int ch = 2 * u + half;
             if (ch < n_chunks) {
-              float f[16];
-#pragma unroll
-              for (int e = 0; e < 16; ++e) {
-                const int q = ch * 16 + e;
-                float tm = fmaxf(fmaxf(xq[q], xq[128 + q]), fmaxf(xq[256 + q], xq[384 + q])) * c;
-                if (!(tm > -CUDART_INF_F)) tm = -CUDART_INF_F;      // also catches NaN
-                const float m_old = first ? -CUDART_INF_F : mref[q];
-                const float m_new = fmaxf(m_old, tm);
-                f[e] = (m_old > -CUDART_INF_F) ? fast_exp2(m_old - m_new) : 0.f;
-                lsum[u][e] *= f[e];
-                mref_buf[(mpar ^ 1) * 128 + q] = m_new;     // every thread of the chunk writes the same value
-              }
+              // every thread keeps its own copy of the factors: fq is written and
+              // read back by the same thread with identical values from its peers
+              chunk_new_reference(xq + ch * 16, mref + ch * 16, mref_buf + (mpar ^ 1) * 128 + ch * 16,
+                                  fq + ch * 16, c, first);
+              __syncwarp();
               if (!first) {
-                uint32_t o[16];
-                tmem_ld16(TM_O + lane_addr + ch * 16, o);
-                tmem_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f[e]);
-                tmem_st16(TM_O + lane_addr + ch * 16, o);
+                for (int e = 0; e < 16; ++e) lsum[u][e] *= fq[ch * 16 + e];
+                chunk_rescale(TM_O + lane_addr + ch * 16, fq + ch * 16);
               }
             }
           }
-          if (!first) tmem_wait_st();
           mpar ^= 1;
           mref = mref_buf + mpar * 128;
           soft_sync();                                      // new references visible to every thread
@@ -619,7 +655,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
             uint32_t sr[16];
             tmem_ld16(ts + ch * 16, sr);
             tmem_wait_ld();
-            const uint32_t vis = chunk_vis(ch);
+            const uint32_t vis = visb[u];
             const float4* mr4 = reinterpret_cast<const float4*>(mref + ch * 16);
             uint32_t hi[8], lw[8];
 #pragma unroll
@@ -629,8 +665,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
               float pv[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const float m_use = (mm[e] > -CUDART_INF_F) ? mm[e] : 0.f;
-                const float x = fast_exp2(fmaf(__uint_as_float(sr[e4 * 4 + e]), c, -m_use));
+                // a row without any visible key so far has reference -inf and only
+                // invisible entries: the select below keeps those at zero
+                const float x = fast_exp2(fmaf(__uint_as_float(sr[e4 * 4 + e]), c, -mm[e]));
                 pv[e] = ((vis >> (e4 * 4 + e)) & 1u) ? x : 0.f;
                 lsum[u][e4 * 4 + e] += pv[e];
               }
@@ -658,27 +695,38 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         mbar_arrive(BAR(B_PREADY + buf));
       }
       // ---- end of share: final output or partial ---------------------------
-      // row sums: add this key's share over the 128 keys (lanes, then quarters)
+      ok &= mbar_wait(BAR(B_PVDONE), (gt - 1) & 1, abort_flag, p.err, 12);   // P buffer idle from here
+      tc_fence_after();
+      // row sums: every key's share goes to scratch as xs[query row][key]; then
+      // thread (row r, piece j) adds 16 keys and an 8-lane shuffle finishes the row
 #pragma unroll
       for (int u = 0; u < MAXCH; ++u) {
         const int ch = 2 * u + half;
         if (ch < n_chunks) {
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            float v = lsum[u][e];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-            if (lane == 0) xq[quarter * 128 + ch * 16 + e] = v;
-          }
+          for (int e = 0; e < 16; ++e) xs[(ch * 16 + e) * TILE_N + kl] = lsum[u][e];
         }
       }
       soft_sync();
-      ok &= mbar_wait(BAR(B_PVDONE), (gt - 1) & 1, abort_flag, p.err, 12);
-      tc_fence_after();
+      for (int base = 0; base < n_pad; base += 32) {
+        const int r = base + (sidx >> 3), j = sidx & 7;
+        float v = 0.f;
+        if (r < n_pad) {
+          const float4* src = reinterpret_cast<const float4*>(xs + r * TILE_N + j * 16);
+          const float4 a = src[0], b = src[1], cc = src[2], d = src[3];
+          v = ((a.x + a.y) + (a.z + a.w)) + ((b.x + b.y) + (b.z + b.w)) +
+              ((cc.x + cc.y) + (cc.z + cc.w)) + ((d.x + d.y) + (d.z + d.w));
+        }
+        v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+        v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+        v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
+        if (j == 0 && r < n_pad) fq[r] = v;                 // fq now holds the row sums
+      }
+      soft_sync();
       const bool whole = (sg.t0 == 0 && sg.t1 == sg.T);
       const int item = sg.b * p.H_kv + sg.h;
       float* pslot = p.part + ((size_t)(item + group) * p.n_mblocks + mb) * (ROWS * (DH + 2));
-      if (threadIdx.x == WARP_SOFTMAX0 * 32 && ok) {
+      if (sidx == 0 && ok) {
         // how this (sequence, head) was cut: first group and number of groups,
         // read by attn_merge_kernel (every group of the cut writes the same pair)
         int2 d = make_int2(group, 1);
@@ -691,43 +739,47 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         }
         p.desc[(size_t)item * p.n_mblocks + mb] = d;
       }
+      if (sidx < m_valid && ok) {                           // per-row scalars
+        const int q = sidx;
+        if (whole) {
+          if (p.lse) {
+            const int i = i0 + q / p.G, hq = sg.h * p.G + q % p.G;
+            p.lse[((size_t)sg.b * p.H_q + hq) * p.n_q + i] = (mref[q] + log2f(fq[q])) * 0.6931471805599453f;
+          }
+        } else {
+          pslot[ROWS * DH + q] = mref[q];
+          pslot[ROWS * DH + ROWS + q] = fq[q];
+        }
+      }
       // O^T: lane = head-dim index, column = query row.  A warp writes 32
       // consecutive floats of one output row per store.
-      const bool d_ok = kl < DH;                            // lanes 64..127 repeat 0..63 when head_dim is 64
-#pragma unroll
-      for (int u = 0; u < MAXCH; ++u) {
-        const int ch = 2 * u + half;
-        if (ch < n_chunks) {
-          uint32_t o[16];
-          tmem_ld16(TM_O + lane_addr + ch * 16, o);
-          tmem_wait_ld();
+      const bool d_ok = kl < DH && ok;                      // lanes 64..127 repeat 0..63 when head_dim is 64
+#pragma unroll 1
+      for (int ch = half; ch < n_chunks; ch += 2) {
+        uint32_t o[16];
+        tmem_ld16(TM_O + lane_addr + ch * 16, o);
+        tmem_wait_ld();
+        const int q0 = ch * 16;
+        if (whole) {
+          int i = i0 + q0 / p.G, g = q0 % p.G;
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            const int q = ch * 16 + e;
-            if (q < m_valid && d_ok && ok) {
-              const float l_tot = (xq[q] + xq[128 + q]) + (xq[256 + q] + xq[384 + q]);
-              const float val = __uint_as_float(o[e]);
-              if (whole) {
-                const int i = i0 + q / p.G, hq = sg.h * p.G + q % p.G;
-                const size_t off = (((size_t)sg.b * p.n_q + i) * p.H_q + hq) * DH + kl;
-                const float r = val / l_tot;
-                if (p.out_dtype == SPACE_DTYPE_F32) reinterpret_cast<float*>(p.out)[off] = r;
-                else reinterpret_cast<__nv_bfloat16*>(p.out)[off] = __float2bfloat16_rn(r);
-                if (kl == 0 && p.lse)
-                  p.lse[((size_t)sg.b * p.H_q + hq) * p.n_q + i] = (mref[q] + log2f(l_tot)) * 0.6931471805599453f;
-              } else {
-                pslot[(size_t)q * DH + kl] = val;
-                if (kl == 0) {
-                  pslot[ROWS * DH + q] = mref[q];
-                  pslot[ROWS * DH + ROWS + q] = l_tot;
-                }
-              }
+            if (q0 + e < m_valid && d_ok) {
+              const size_t off = (((size_t)sg.b * p.n_q + i) * p.H_q + sg.h * p.G + g) * DH + kl;
+              const float r = __uint_as_float(o[e]) / fq[q0 + e];
+              if (p.out_dtype == SPACE_DTYPE_F32) reinterpret_cast<float*>(p.out)[off] = r;
+              else reinterpret_cast<__nv_bfloat16*>(p.out)[off] = __float2bfloat16_rn(r);
             }
+            if (++g == p.G) { g = 0; ++i; }
           }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 16; ++e)
+            if (q0 + e < m_valid && d_ok) pslot[(size_t)(q0 + e) * DH + kl] = __uint_as_float(o[e]);
         }
       }
       tc_fence_before();
-      soft_sync();                                          // xq and mref are reused by the next share
+      soft_sync();                                          // scratch, fq and mref are reused by the next share
     }
   }
 
