@@ -478,6 +478,13 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     if (lane == 0) {
       const uint32_t idesc_qk = instr_desc_rt(n_pad, 0, 0);   // A = K tile (K-major), B = Q (K-major)
       const uint32_t idesc_pv = instr_desc_rt(n_pad, 1, 1);   // A = V^T (d contiguous), B = P^T (queries contiguous)
+      // descriptors of the first stage of every operand; a later stage or k-step
+      // only adds to the 14-bit address field (16-byte units, no carry possible)
+      const uint64_t kdesc0 = smem_desc(sm_base + S::K_OFF, 16, 1024);           // K-major rows of 128 bytes
+      const uint64_t qdesc0 = smem_desc(sm_base + S::Q_OFF, 16, 1024);
+      // V^T and P^T: 64-wide blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
+      const uint64_t vdesc0 = smem_desc(sm_base + S::V_OFF, TILE_N * 128, 1024);
+      const uint64_t pdesc0 = smem_desc(sm_base + S::P_OFF, TILE_N * 128, 1024);
       uint32_t gt = 0, seg = 0;
       bool ok = true;
       // O^T += V^T (P_hi + P_lo)^T for flat tile g (first_in_seg: overwrite O^T)
@@ -486,16 +493,15 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         if (!mbar_wait(BAR(B_VFULL + s), (g / S::V_STAGES) & 1, abort_flag, p.err, 4)) return false;
         if (!mbar_wait(BAR(B_PREADY + (g & 1)), (g >> 1) & 1, abort_flag, p.err, 5)) return false;
         tc_fence_after();
-        const uint32_t vsm = sm_base + S::V_OFF + s * S::TILE_BYTES;
-        const uint32_t psm = sm_base + S::P_OFF;
+        const uint64_t ad0 = vdesc0 + (uint64_t)((s * S::TILE_BYTES) >> 4);
 #pragma unroll
         for (int part_i = 0; part_i < 2; ++part_i) {        // P_hi, then P_lo
 #pragma unroll
           for (int kk = 0; kk < TILE_N / 16; ++kk) {
-            // both operands: 64-wide blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
-            const uint64_t ad = smem_desc(vsm + kk * 2048, TILE_N * 128, 1024);
-            const uint64_t bd = smem_desc(psm + part_i * S::P_PART + kk * 2048, TILE_N * 128, 1024);
-            mma_ss(TM_O, ad, bd, idesc_pv, (first_in_seg && kk == 0 && part_i == 0) ? 0u : 1u);
+            // 16 keys further = 2048 bytes further in both operands
+            mma_ss(TM_O, ad0 + (uint64_t)((kk * 2048) >> 4),
+                   pdesc0 + (uint64_t)((part_i * S::P_PART + kk * 2048) >> 4), idesc_pv,
+                   (first_in_seg && kk == 0 && part_i == 0) ? 0u : 1u);
           }
         }
         tc_commit(BAR(B_VEMPTY + s));
@@ -512,15 +518,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           ok = mbar_wait(BAR(B_KFULL + s), (gt / S::K_STAGES) & 1, abort_flag, p.err, 7);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t qsm = sm_base + S::Q_OFF;
-          const uint32_t ksm = sm_base + S::K_OFF + s * S::TILE_BYTES;
+          const uint64_t kd = kdesc0 + (uint64_t)((s * S::TILE_BYTES) >> 4);
 #pragma unroll
           for (int kk = 0; kk < DH / 16; ++kk) {
             // 64-wide half of d, then 32 bytes per 16 elements inside the swizzled row
             const uint32_t koff = (kk >> 2) * (TILE_N * 128) + (kk & 3) * 32;
             const uint32_t qoff = (kk >> 2) * (n_pad * 128) + (kk & 3) * 32;
-            mma_ss(TM_S0 + buf * 128, smem_desc(ksm + koff, 16, 1024), smem_desc(qsm + qoff, 16, 1024),
-                   idesc_qk, kk > 0 ? 1u : 0u);
+            mma_ss(TM_S0 + buf * 128, kd + (uint64_t)(koff >> 4), qdesc0 + (uint64_t)(qoff >> 4), idesc_qk,
+                   kk > 0 ? 1u : 0u);
           }
           tc_commit(BAR(B_SFULL + buf));
           tc_commit(BAR(B_KEMPTY + s));
