@@ -32,6 +32,9 @@ sys.path.insert(0, os.path.join(ROOT, "tests"))
 from paper_2402_11809_b200 import workloads  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum per attn_tc_kernel launch from the ncu capture summarised
+# in profiles/attn_tc_kernel_llama7b.txt (bytes); None for workloads without a capture of the current kernel
+ATTN_TRAFFIC = {"llama7b": None}
 METRIC = "auto-correct steps/sec"
 UNIT = "steps/s"
 
@@ -359,7 +362,7 @@ def run_ours(args):
         "step_algorithmic_bytes": step_bytes,
         "step_hbm_frac": step_bytes / (ms / K * 1e-3) / 1e9 / peak,
         "roofline": {"bound": "hbm", "kernel": "attn_tc_kernel", "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "traffic": None,
+                     "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "traffic": ATTN_TRAFFIC.get(cfg["name"]),
                      "peak_source": peak_src + " (burst copy figure)",
                      "algorithmic_bytes_per_launch": float(attn_bytes), "avg_launch_us": attn_us,
                      "launches_timed": int(attn_n),
