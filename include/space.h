@@ -41,7 +41,8 @@ enum {
   SPACE_E_ALIGNMENT   = -3,    /* base pointer / stride not 16-byte aligned   */
   SPACE_E_WORKSPACE   = -4,    /* request exceeds what space_create reserved  */
   SPACE_E_CUDA        = -5,    /* a CUDA runtime or driver call failed        */
-  SPACE_E_NO_DEVICE   = -6     /* no usable sm_100 device                     */
+  SPACE_E_NO_DEVICE   = -6,    /* no usable sm_100 device                     */
+  SPACE_E_STATIC_LIMIT = -7    /* size beyond the fixed scratch of space_verify_greedy_noalloc */
 };
 
 enum { SPACE_MASK_SAME_GROUP = 0, SPACE_MASK_EQ5_LITERAL = 1 };
@@ -186,6 +187,32 @@ int space_attn_step(space_ctx* ctx, const space_attn_args* args, void* stream);
 
 /* Algorithm 1 verification loop, extra token and next candidates. */
 int space_verify(space_ctx* ctx, const space_verify_args* args, void* stream);
+
+/* Greedy verification without any allocation.  (The paper has no counterpart:
+ * this entry point exists for how the library is embedded, not for the method.)
+ *
+ * Some hosts of this library may not allocate device memory once they are
+ * running: a serving process that hands all of the GPU's memory to its own pool
+ * at start-up leaves nothing for cudaMalloc, and a latency-critical decode loop
+ * cannot afford the implicit device-wide synchronisation an allocation can
+ * cause.  Such callers cannot use space_create, which reserves a workspace.
+ * This call needs no context: its scratch (chunk results and per-sequence
+ * arrival counters, SPACE_NOALLOC_MAX_BATCH * 32 KiB + 256 bytes) is a fixed
+ * array inside the library image, resident on every GPU that loads the library
+ * until the process exits.  It calls no cudaMalloc / cudaFree and no allocating
+ * library routine.
+ *
+ * Same arguments, outputs and results as space_verify in SPACE_MODE_GREEDY
+ * (args->mode must be SPACE_MODE_GREEDY; temperature, seed, resample ignored);
+ * all (k+1)^2 logits rows are read in one kernel.  Runs on the current device.
+ * Limits: batch <= SPACE_NOALLOC_MAX_BATCH, else SPACE_E_STATIC_LIMIT; k in
+ * 1..SPACE_MAX_K.  The first call on a device looks up the array's device
+ * address (cudaGetSymbolAddress); make that first call outside any stream
+ * capture.  All calls share the one array: the counters are cleared at the start
+ * of every call, and two calls whose kernels overlap on the GPU (different
+ * streams, or several host threads) race on it - serialise them. */
+#define SPACE_NOALLOC_MAX_BATCH 8
+int space_verify_greedy_noalloc(const space_verify_args* args, void* stream);
 
 /* Move accepted rows L+g(k+1) -> L+g, g = 1..i*; lengths grow by i*+1. */
 int space_kv_commit(space_ctx* ctx, const space_commit_args* args, void* stream);

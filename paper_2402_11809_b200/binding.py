@@ -14,6 +14,8 @@ SPACE_MAX_K = 7
 SPACE_MAX_ROWS = 64
 OK = 0
 E_INVALID_ARG, E_UNSUPPORTED, E_ALIGNMENT, E_WORKSPACE, E_CUDA, E_NO_DEVICE = -1, -2, -3, -4, -5, -6
+E_STATIC_LIMIT = -7
+NOALLOC_MAX_BATCH = 8
 MASK_SAME_GROUP, MASK_EQ5_LITERAL = 0, 1
 MODE_GREEDY, MODE_SAMPLE = 0, 1
 RESAMPLE_RESIDUAL_POINTMASS, RESAMPLE_PAPER_LITERAL = 0, 1
@@ -22,7 +24,8 @@ ATTN_TENSOR, ATTN_SIMT = 0, 1
 ST_CAPACITY, ST_BAD_CANDIDATE, ST_TIMEOUT = 1, 2, 4
 
 EXPORTS = ["space_create", "space_destroy", "space_workspace_bytes", "space_layout",
-           "space_attn_step", "space_verify", "space_kv_commit", "space_step_host",
+           "space_attn_step", "space_verify", "space_verify_greedy_noalloc", "space_kv_commit",
+           "space_step_host",
            "space_launch_count", "space_profile_enable", "space_profile_read",
            "space_debug_philox", "space_strerror"]
 
@@ -99,6 +102,8 @@ for _name, _arg in (("space_attn_step", AttnArgs), ("space_verify", VerifyArgs),
                     ("space_kv_commit", CommitArgs), ("space_step_host", HostStepArgs)):
     getattr(lib, _name).argtypes = [C.c_void_p, C.POINTER(_arg), C.c_void_p]
     getattr(lib, _name).restype = C.c_int
+lib.space_verify_greedy_noalloc.argtypes = [C.POINTER(VerifyArgs), C.c_void_p]
+lib.space_verify_greedy_noalloc.restype = C.c_int
 lib.space_launch_count.argtypes = [C.c_void_p]
 lib.space_launch_count.restype = C.c_int64
 lib.space_profile_enable.argtypes = [C.c_void_p, C.c_int]
@@ -135,6 +140,11 @@ def space_layout(k, mask_variant=MASK_SAME_GROUP):
     lay = Layout()
     _check(lib.space_layout(k, mask_variant, C.byref(lay)))
     return lay
+
+
+def space_verify_greedy_noalloc(args):
+    """Greedy verification with no context and no allocation (see include/space.h)."""
+    _check(lib.space_verify_greedy_noalloc(C.byref(args), _stream()))
 
 
 def space_strerror(code):

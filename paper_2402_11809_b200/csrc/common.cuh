@@ -7,6 +7,7 @@
 
 #define SPACE_VERIFY_MAX_CHUNKS 64
 #define SPACE_VERIFY_THREADS 256
+#define SPACE_FUSED_MAX_CHUNKS 16
 
 // ---- Philox4x32-10 (Salmon et al., SC'11) ---------------------------------
 struct Philox4 { uint32_t x, y, z, w; };
@@ -78,6 +79,7 @@ struct space_ctx {
 
 // ---- per-stage launchers (defined next to their kernels) -------------------
 int launch_verify(space_ctx* ctx, const space_verify_args* a, cudaStream_t st);
+int launch_verify_noalloc(const space_verify_args* a, cudaStream_t st);
 int launch_commit(space_ctx* ctx, const space_commit_args* a, cudaStream_t st);
 int launch_attn_simt(space_ctx* ctx, const space_attn_args* a, const uint64_t* mask_rows,
                      cudaStream_t st);

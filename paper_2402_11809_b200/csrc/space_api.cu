@@ -215,6 +215,22 @@ int space_verify(space_ctx* ctx, const space_verify_args* a, void* stream) {
   return launch_verify(ctx, a, (cudaStream_t)stream);
 }
 
+int space_verify_greedy_noalloc(const space_verify_args* a, void* stream) {
+  if (!a) return SPACE_E_INVALID_ARG;
+  if (a->batch < 0 || a->k < 1 || a->k > SPACE_MAX_K || a->vocab < 1) return SPACE_E_INVALID_ARG;
+  if (a->batch > SPACE_NOALLOC_MAX_BATCH) return SPACE_E_STATIC_LIMIT;
+  if (a->batch == 0) return SPACE_OK;
+  if (a->mode != SPACE_MODE_GREEDY) return SPACE_E_INVALID_ARG;
+  if (!a->logits || !a->cand || !a->cand_prob || !a->n_accept || !a->out_tokens || !a->n_out ||
+      !a->next_cand || !a->next_cand_prob || !a->finished)
+    return SPACE_E_INVALID_ARG;
+  if (a->logits_dtype != SPACE_DTYPE_F32 && a->logits_dtype != SPACE_DTYPE_BF16) return SPACE_E_INVALID_ARG;
+  if (a->logits_row_stride < a->vocab) return SPACE_E_INVALID_ARG;
+  const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;
+  if ((uintptr_t)a->logits % esz) return SPACE_E_ALIGNMENT;
+  return launch_verify_noalloc(a, (cudaStream_t)stream);
+}
+
 int space_kv_commit(space_ctx* ctx, const space_commit_args* a, void* stream) {
   if (!ctx || !a) return SPACE_E_INVALID_ARG;
   if (a->batch < 0 || a->batch > ctx->cfg.max_batch) return SPACE_E_WORKSPACE;
@@ -393,6 +409,7 @@ const char* space_strerror(int code) {
     case SPACE_E_WORKSPACE: return "request exceeds the workspace reserved by space_create";
     case SPACE_E_CUDA: return "CUDA call failed";
     case SPACE_E_NO_DEVICE: return "no usable sm_100 device";
+    case SPACE_E_STATIC_LIMIT: return "batch exceeds the fixed scratch of space_verify_greedy_noalloc (SPACE_NOALLOC_MAX_BATCH)";
     default: return "unknown error";
   }
 }

@@ -384,7 +384,6 @@ verify_emit_kernel(const VerifyParams p) {
 }
 
 
-#define SPACE_FUSED_MAX_CHUNKS 16
 
 // One launch for greedy mode on small inputs: statistics of every block row,
 // then acceptance, emission and next candidates by the last block of a sequence.
@@ -558,4 +557,87 @@ int launch_philox_debug(uint64_t seed, int64_t n, const uint32_t* c0, const uint
   philox_debug_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
       (uint32_t)(seed & 0xFFFFFFFFull), (uint32_t)(seed >> 32), n, c0, c1, c2, c3, out);
   return cuda_ok(cudaGetLastError());
+}
+
+// ---------------------------------------------------------------------------
+// Allocation-free greedy verification (space_verify_greedy_noalloc).
+//
+// The scratch that verify_fused_kernel needs (chunk results and one arrival
+// counter per sequence) lives in this file-scope device array instead of a
+// context workspace, so the entry point never calls cudaMalloc.  Every GPU that
+// loads the library holds the array until the process exits.
+#define SPACE_NOALLOC_COUNTER_BYTES 256
+#define SPACE_NOALLOC_SCRATCH_BYTES \
+  (SPACE_NOALLOC_COUNTER_BYTES +      \
+   SPACE_NOALLOC_MAX_BATCH * SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS * (int)sizeof(VerifyPartial))
+static __device__ __align__(256) unsigned char g_noalloc_scratch[SPACE_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int NOALLOC_MAX_DEVICES = 64;
+// The array's name is only a host-side handle; the address kernels can use is
+// looked up once per device (with that device current) and kept here.
+void* g_noalloc_ptr[NOALLOC_MAX_DEVICES];
+int g_noalloc_sms[NOALLOC_MAX_DEVICES];
+}  // namespace
+
+int launch_verify_noalloc(const space_verify_args* a, cudaStream_t st) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return SPACE_E_NO_DEVICE;
+  if (!g_noalloc_ptr[dev]) {
+    // first call on this device: resolve the device address of the scratch array
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return SPACE_E_CUDA;
+    }
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+      cudaGetLastError();
+      return SPACE_E_CUDA;
+    }
+    g_noalloc_sms[dev] = sms;
+    g_noalloc_ptr[dev] = ptr;
+  }
+  unsigned char* base = static_cast<unsigned char*>(g_noalloc_ptr[dev]);
+  // the arrival counters must start at zero whatever an earlier call left behind
+  if (cudaMemsetAsync(base, 0, SPACE_NOALLOC_COUNTER_BYTES, st) != cudaSuccess) return SPACE_E_CUDA;
+
+  VerifyParams p;
+  p.B = a->batch; p.k = a->k; p.V = a->vocab; p.n_q = (a->k + 1) * (a->k + 1);
+  p.mode = SPACE_MODE_GREEDY; p.resample = SPACE_RESAMPLE_RESIDUAL_POINTMASS; p.eos_id = a->eos_id;
+  p.c_t = 1.4426950408889634f; p.inv_t = 1.0f;
+  p.key0 = 0; p.key1 = 0;
+  p.logits = a->logits; p.row_stride = a->logits_row_stride;
+  p.cand = a->cand; p.cand_prob = a->cand_prob; p.seq_id = a->seq_id; p.kv_len = a->kv_len;
+  p.n_accept = a->n_accept; p.out_tokens = a->out_tokens; p.n_out = a->n_out;
+  p.next_cand = a->next_cand; p.next_cand_prob = a->next_cand_prob; p.finished = a->finished;
+  p.status = a->status;
+  p.part = nullptr; p.rows = nullptr;
+  p.counter_a = reinterpret_cast<int*>(base); p.counter_b = nullptr;
+  VerifyPartial* fpart = reinterpret_cast<VerifyPartial*>(base + SPACE_NOALLOC_COUNTER_BYTES);
+
+  const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;
+  const int vec = 16 / esz;
+  const bool vector = ((uintptr_t)a->logits % 16 == 0) && ((a->logits_row_stride * esz) % 16 == 0);
+  const int rows_all = a->batch * p.n_q;
+  int nc = g_noalloc_sms[dev] / rows_all;
+  const int min_chunk = SPACE_VERIFY_THREADS * vec;
+  const int max_nc = (a->vocab + min_chunk - 1) / min_chunk;
+  if (nc > max_nc) nc = max_nc;
+  if (nc > SPACE_FUSED_MAX_CHUNKS) nc = SPACE_FUSED_MAX_CHUNKS;
+  if (nc < 1) nc = 1;
+  int chunk = (a->vocab + nc - 1) / nc;
+  chunk = ((chunk + vec - 1) / vec) * vec;
+  nc = (a->vocab + chunk - 1) / chunk;
+  p.n_chunks = nc; p.chunk = chunk;
+  const dim3 grid(nc, p.n_q, a->batch), block(SPACE_VERIFY_THREADS);
+  cudaError_t e;
+  if (a->logits_dtype == SPACE_DTYPE_F32) {
+    e = vector ? launch_pdl(verify_fused_kernel<float, true>, grid, block, 0, st, p, fpart)
+               : launch_pdl(verify_fused_kernel<float, false>, grid, block, 0, st, p, fpart);
+  } else {
+    e = vector ? launch_pdl(verify_fused_kernel<__nv_bfloat16, true>, grid, block, 0, st, p, fpart)
+               : launch_pdl(verify_fused_kernel<__nv_bfloat16, false>, grid, block, 0, st, p, fpart);
+  }
+  return cuda_ok(e);
 }
