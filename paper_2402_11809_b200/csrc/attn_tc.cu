@@ -826,18 +826,32 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(const AttnParams p) {
   const size_t gstride = (size_t)p.n_mblocks * slot_floats;
   float mx = -CUDART_INF_F, den = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 8
-  for (int x = 0; x < n; ++x, ps += gstride) {
-    const float ms = __ldcg(ps + ROWS * DH + r), ls = __ldcg(ps + ROWS * DH + ROWS + r);
-    const float4 ov = __ldcg(reinterpret_cast<const float4*>(ps + (size_t)r * DH) + c4);
-    const float mn = fmaxf(mx, ms);
-    if (mn > -CUDART_INF_F) {
-      const float e0 = fast_exp2(mx - mn), e1 = fast_exp2(ms - mn);
-      den = den * e0 + ls * e1;
-      acc.x = acc.x * e0 + ov.x * e1; acc.y = acc.y * e0 + ov.y * e1;
-      acc.z = acc.z * e0 + ov.z * e1; acc.w = acc.w * e0 + ov.w * e1;
+  // batches of eight partials: all loads of a batch are issued before any is used
+  for (int x0 = 0; x0 < n; x0 += 8) {
+    float ms[8], ls[8];
+    float4 ov[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (x0 + j < n) {
+        const float* pj = ps + (size_t)(x0 + j) * gstride;
+        ms[j] = __ldcg(pj + ROWS * DH + r);
+        ls[j] = __ldcg(pj + ROWS * DH + ROWS + r);
+        ov[j] = __ldcg(reinterpret_cast<const float4*>(pj + (size_t)r * DH) + c4);
+      }
     }
-    mx = mn;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (x0 + j < n) {
+        const float mn = fmaxf(mx, ms[j]);
+        if (mn > -CUDART_INF_F) {
+          const float e0 = fast_exp2(mx - mn), e1 = fast_exp2(ms[j] - mn);
+          den = den * e0 + ls[j] * e1;
+          acc.x = acc.x * e0 + ov[j].x * e1; acc.y = acc.y * e0 + ov[j].y * e1;
+          acc.z = acc.z * e0 + ov[j].z * e1; acc.w = acc.w * e0 + ov[j].w * e1;
+        }
+        mx = mn;
+      }
+    }
   }
   const float rd = 1.f / den;
   const int ri = i0 + r / p.G, hq = h * p.G + r % p.G;

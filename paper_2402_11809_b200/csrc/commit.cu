@@ -10,7 +10,7 @@
 namespace {
 
 struct CommitParams {
-  int B, k, H_kv, d, blocks_per_seq;
+  int B, k, H_kv, d, blocks_per_seq, in_place;
   int64_t s_cap;
   __nv_bfloat16* kc; __nv_bfloat16* vc;
   int64_t sb, sh, ss;
@@ -43,17 +43,25 @@ __global__ void __launch_bounds__(256) kv_commit_kernel(const CommitParams p) {
       *dd = *s;
     }
   }
-  // the last block of the sequence publishes the new length and the index tables
-  __shared__ int last;
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const int prev = atomicAdd(p.counter + b, 1);
-    last = (prev == p.blocks_per_seq - 1);
-    if (last) p.counter[b] = 0;
+  // New length and index tables.  When the new length goes to its own array no
+  // block depends on another and block 0 writes them at once; when it overwrites
+  // kv_len itself the other blocks must have read the old value first, so the
+  // last block to arrive (counter, reset for the next launch) writes them.
+  if (p.in_place) {
+    __shared__ int last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const int prev = atomicAdd(p.counter + b, 1);
+      last = (prev == p.blocks_per_seq - 1);
+      if (last) p.counter[b] = 0;
+    }
+    __syncthreads();
+    if (!last) return;
+  } else if (part != 0) {
+    return;
   }
-  __syncthreads();
-  if (!last || threadIdx.x != 0) return;
+  if (threadIdx.x != 0) return;
   if (!fits) {
     if (p.status) atomicOr(p.status + b, SPACE_ST_CAPACITY);
     i_star = -1;                                        // nothing committed, length unchanged
@@ -76,6 +84,7 @@ int launch_commit(space_ctx* ctx, const space_commit_args* a, cudaStream_t st) {
   p.n_accept = a->n_accept; p.kv_len = a->kv_len; p.kv_len_out = a->kv_len_out;
   p.src = a->commit_src; p.dst = a->commit_dst; p.status = a->status;
   p.counter = ctx->counters + 2 * ctx->cfg.max_batch;
+  p.in_place = (a->kv_len_out == a->kv_len);
   // worst case k rows x H_kv heads x K,V x d/8 pieces; one piece per thread, 256 threads
   const int worst = a->k * p.H_kv * 2 * (p.d / 8);
   int blocks = (worst + 255) / 256;

@@ -146,19 +146,17 @@ __device__ Stat scan_chunk(const T* row, int begin, int end, float c, float inv_
     // begin is a multiple of N; the tail shorter than N is handled one by one
     const int full_end = begin + ((end - begin) / N) * N;
     const int stride = blockDim.x * N;
-    int x = begin + threadIdx.x * N;
-    for (; x + (U - 1) * stride < full_end; x += U * stride) {
+    // U loads are issued together (predicated at the end of the chunk) so that a
+    // short chunk costs one memory round trip, not one per sweep
+    for (int x = begin + threadIdx.x * N; x < full_end; x += U * stride) {
       float v[U][N];
 #pragma unroll
-      for (int u = 0; u < U; ++u) Vec<T>::load(row + x + u * stride, v[u]);
+      for (int u = 0; u < U; ++u)
+        if (x + u * stride < full_end) Vec<T>::load(row + x + u * stride, v[u]);
 #pragma unroll
       for (int u = 0; u < U; ++u)
-        fold<N, GUMBEL>(st, v[u], x + u * stride, c, inv_t, exclude, key0, key1, purpose, seq, pos);
-    }
-    for (; x < full_end; x += stride) {
-      float v[N];
-      Vec<T>::load(row + x, v);
-      fold<N, GUMBEL>(st, v, x, c, inv_t, exclude, key0, key1, purpose, seq, pos);
+        if (x + u * stride < full_end)
+          fold<N, GUMBEL>(st, v[u], x + u * stride, c, inv_t, exclude, key0, key1, purpose, seq, pos);
     }
     for (int x = full_end + threadIdx.x; x < end; x += blockDim.x) {
       float v[1] = {load_logit(row + x)};
@@ -200,6 +198,57 @@ __device__ Stat block_reduce(Stat st, float c) {
     st = warp_reduce(st, c);
   }
   return st;           // valid in warp 0
+}
+
+
+// Reductions for (max, sum, arg-max) only: the maximum (lowest index on ties)
+// first, then every contributor rescales its sum once and the sums are added.
+// Far fewer exponentials than merging pairwise.
+__device__ __forceinline__ void warp_max_idx(float& m, int& idx, int width = 32) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    if (off < width) {
+      const float om = __shfl_xor_sync(0xFFFFFFFFu, m, off);
+      const int oi = __shfl_xor_sync(0xFFFFFFFFu, idx, off);
+      if (om > m || (om == m && oi < idx)) { m = om; idx = oi; }
+    }
+  }
+}
+__device__ __forceinline__ float warp_sum(float v, int width = 32) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1)
+    if (off < width) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+  return v;
+}
+// Block-wide (m, s, idx); result valid in thread 0.  gs/gidx are not touched.
+__device__ Stat block_reduce_plain(Stat st, float c) {
+  __shared__ float sh_m[SPACE_VERIFY_THREADS / 32];
+  __shared__ int sh_i[SPACE_VERIFY_THREADS / 32];
+  __shared__ float sh_s[SPACE_VERIFY_THREADS / 32];
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  constexpr int NW = SPACE_VERIFY_THREADS / 32;
+  float m = st.m; int idx = st.idx;
+  warp_max_idx(m, idx);
+  if (l == 0) { sh_m[w] = m; sh_i[w] = idx; }
+  __syncthreads();
+  float bm = sh_m[0]; int bi = sh_i[0];
+#pragma unroll
+  for (int i = 1; i < NW; ++i) {
+    const float om = sh_m[i]; const int oi = sh_i[i];
+    if (om > bm || (om == bm && oi < bi)) { bm = om; bi = oi; }
+  }
+  float sv = (st.m > -CUDART_INF_F) ? st.s * exp2f((st.m - bm) * c) : 0.f;
+  sv = warp_sum(sv);
+  if (l == 0) sh_s[w] = sv;
+  __syncthreads();
+  Stat r = stat_empty();
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < NW; ++i) tot += sh_s[i];
+    r.m = bm; r.idx = bi; r.s = tot;
+  }
+  return r;
 }
 
 __device__ __forceinline__ void store_partial(VerifyPartial* p, const Stat& st) {
@@ -252,7 +301,7 @@ verify_target_kernel(const VerifyParams p) {
   const T* row = reinterpret_cast<const T*>(p.logits) + ((int64_t)b * p.n_q + (int64_t)t * k1) * p.row_stride;
   const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
   Stat st = scan_chunk<T, VECTOR, false>(row, begin, end, p.c_t, 1.f, -1, 0, 0, 0, 0, 0);
-  st = block_reduce(st, p.c_t);
+  st = block_reduce_plain(st, p.c_t);
   VerifyPartial* part = p.part + ((int64_t)b * (p.k + 2) + t) * p.n_chunks;
   if (threadIdx.x == 0) store_partial(part + ch, st);
   if (!arrive_last(p.counter_a + b, k1 * p.n_chunks)) return;
@@ -398,7 +447,7 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   const T* row = reinterpret_cast<const T*>(p.logits) + ((int64_t)b * p.n_q + row_i) * p.row_stride;
   const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
   Stat st = scan_chunk<T, VECTOR, false>(row, begin, end, C1, 1.f, -1, 0, 0, 0, 0, 0);
-  st = block_reduce(st, C1);
+  st = block_reduce_plain(st, C1);
   VerifyPartial* pb = fpart + (int64_t)b * SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS;
   if (threadIdx.x == 0) store_partial(pb + row_i * p.n_chunks + ch, st);
   if (!arrive_last(p.counter_a + b, p.n_q * p.n_chunks)) return;
@@ -417,11 +466,16 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   if (threadIdx.x < p.k) sh_cand[threadIdx.x] = p.cand[b * p.k + threadIdx.x];
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int r = warp; r < p.n_q; r += SPACE_VERIFY_THREADS / 32) {
-    Stat a = stat_empty();
-    if (lane < p.n_chunks) { a.m = sh_m[r * p.n_chunks + lane]; a.s = sh_s[r * p.n_chunks + lane]; a.idx = sh_i[r * p.n_chunks + lane]; }
-    a = warp_reduce(a, C1);
-    if (lane == 0) { row_s[r] = a.s; row_idx[r] = a.idx; }
+  // two rows per warp at a time: lanes 0..15 and 16..31 each reduce one row's chunks
+  for (int r0 = warp * 2; r0 < p.n_q; r0 += 2 * (SPACE_VERIFY_THREADS / 32)) {
+    const int r = r0 + (lane >> 4), cl = lane & 15;
+    float m = -CUDART_INF_F, sv = 0.f; int idx = 0x7FFFFFFF;
+    if (r < p.n_q && cl < p.n_chunks) { m = sh_m[r * p.n_chunks + cl]; sv = sh_s[r * p.n_chunks + cl]; idx = sh_i[r * p.n_chunks + cl]; }
+    float bm = m; int bi = idx;
+    warp_max_idx(bm, bi, 16);
+    sv = (m > -CUDART_INF_F) ? sv * exp2f((m - bm) * C1) : 0.f;
+    sv = warp_sum(sv, 16);
+    if (cl == 0 && r < p.n_q) { row_s[r] = sv; row_idx[r] = bi; }
   }
   __syncthreads();
   if (threadIdx.x >= 32) return;
