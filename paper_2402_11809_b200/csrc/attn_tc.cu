@@ -295,18 +295,31 @@ __device__ __noinline__ void chunk_key_max(uint32_t taddr, uint32_t vis, float* 
 }
 
 // New reference for the 16 query rows of a chunk from the four quarter maxima in
-// xq; writes the reference to mnew[0..15] and the factor old -> new to fq[0..15].
-// Every thread of the chunk computes the same values (identical writes).
+// xq; writes the reference to mnew[0..15] and (unless this is a share's first
+// tile) the factor old -> new to fq[0..15].  Every thread of the chunk computes
+// the same values (identical writes).  All pointers are 16-byte aligned.
 __device__ __noinline__ void chunk_new_reference(const float* xq, const float* mold, float* mnew, float* fq,
                                                  float c, bool first) {
-#pragma unroll 1
-  for (int e = 0; e < 16; ++e) {
-    float tm = fmaxf(fmaxf(xq[e], xq[128 + e]), fmaxf(xq[256 + e], xq[384 + e])) * c;
-    if (!(tm > -CUDART_INF_F)) tm = -CUDART_INF_F;          // also catches NaN
-    const float m_old = first ? -CUDART_INF_F : mold[e];
-    const float m_new = fmaxf(m_old, tm);
-    mnew[e] = m_new;
-    fq[e] = (m_old > -CUDART_INF_F) ? fast_exp2(m_old - m_new) : 0.f;
+#pragma unroll
+  for (int v = 0; v < 4; ++v) {
+    const float4 a = reinterpret_cast<const float4*>(xq)[v], b = reinterpret_cast<const float4*>(xq + 128)[v];
+    const float4 d = reinterpret_cast<const float4*>(xq + 256)[v], e = reinterpret_cast<const float4*>(xq + 384)[v];
+    float tm[4] = {fmaxf(fmaxf(a.x, b.x), fmaxf(d.x, e.x)) * c, fmaxf(fmaxf(a.y, b.y), fmaxf(d.y, e.y)) * c,
+                   fmaxf(fmaxf(a.z, b.z), fmaxf(d.z, e.z)) * c, fmaxf(fmaxf(a.w, b.w), fmaxf(d.w, e.w)) * c};
+    float mo[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+    if (!first) {
+      const float4 o = reinterpret_cast<const float4*>(mold)[v];
+      mo[0] = o.x; mo[1] = o.y; mo[2] = o.z; mo[3] = o.w;
+    }
+    float mn[4], f[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (!(tm[j] > -CUDART_INF_F)) tm[j] = -CUDART_INF_F;  // also catches NaN
+      mn[j] = fmaxf(mo[j], tm[j]);
+      f[j] = (mo[j] > -CUDART_INF_F) ? fast_exp2(mo[j] - mn[j]) : 0.f;
+    }
+    reinterpret_cast<float4*>(mnew)[v] = make_float4(mn[0], mn[1], mn[2], mn[3]);
+    if (!first) reinterpret_cast<float4*>(fq)[v] = make_float4(f[0], f[1], f[2], f[3]);
   }
 }
 
@@ -725,7 +738,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
         v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
         v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
-        if (j == 0 && r < n_pad) fq[r] = v;                 // fq now holds the row sums
+        if (j == 0 && r < n_pad) { fq[r] = v; xq[r] = 1.f / v; }   // row sums and their reciprocals
       }
       soft_sync();
       const bool whole = (sg.t0 == 0 && sg.t1 == sg.T);
@@ -766,21 +779,31 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         tmem_wait_ld();
         const int q0 = ch * 16;
         if (whole) {
-          int i = i0 + q0 / p.G, g = q0 % p.G;
+          // consecutive query rows are consecutive heads of one block row, then the next block row
+          int g = q0 % p.G;
+          size_t off = (((size_t)sg.b * p.n_q + (i0 + q0 / p.G)) * p.H_q + sg.h * p.G + g) * DH + kl;
+          const size_t row_jump = (size_t)(p.H_q - p.G) * DH;
+          const float4* rv = reinterpret_cast<const float4*>(xq + q0);
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            if (q0 + e < m_valid && d_ok) {
-              const size_t off = (((size_t)sg.b * p.n_q + i) * p.H_q + sg.h * p.G + g) * DH + kl;
-              const float r = __uint_as_float(o[e]) / fq[q0 + e];
-              if (p.out_dtype == SPACE_DTYPE_F32) reinterpret_cast<float*>(p.out)[off] = r;
-              else reinterpret_cast<__nv_bfloat16*>(p.out)[off] = __float2bfloat16_rn(r);
+          for (int e4 = 0; e4 < 4; ++e4) {
+            const float4 r4 = rv[e4];
+            const float rr[4] = {r4.x, r4.y, r4.z, r4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              if (q0 + e4 * 4 + e < m_valid && d_ok) {
+                const float r = __uint_as_float(o[e4 * 4 + e]) * rr[e];
+                if (p.out_dtype == SPACE_DTYPE_F32) reinterpret_cast<float*>(p.out)[off] = r;
+                else reinterpret_cast<__nv_bfloat16*>(p.out)[off] = __float2bfloat16_rn(r);
+              }
+              off += DH;
+              if (++g == p.G) { g = 0; off += row_jump; }
             }
-            if (++g == p.G) { g = 0; ++i; }
           }
         } else {
+          float* dst = pslot + (size_t)q0 * DH + kl;
 #pragma unroll
           for (int e = 0; e < 16; ++e)
-            if (q0 + e < m_valid && d_ok) pslot[(size_t)(q0 + e) * DH + kl] = __uint_as_float(o[e]);
+            if (q0 + e < m_valid && d_ok) dst[e * DH] = __uint_as_float(o[e]);
         }
       }
       tc_fence_before();
