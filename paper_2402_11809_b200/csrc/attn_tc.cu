@@ -52,11 +52,11 @@ struct AttnParams {
   void* out; float* lse; int32_t* status;
   float* part;                         // [slots][ROWS*(DH+2)]
   int* err;                            // one word: first timeout site
-  int2* desc;                          // [B*H_kv*n_mblocks] {first group, number of groups} of each cut
+  int2* desc;                          // [B*H_kv*n_mblocks] {first partial slot, number of partials} of each cut
   uint64_t mask[SPACE_MAX_ROWS];
 };
 
-struct Seg { int b, h, t0, t1, T, L; };
+struct Seg { int b, h, t0, t1, T, L, slot, dfirst, dn; };   // slot: partial slot; dfirst/dn: cut (aligned mode)
 
 // ---------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -93,6 +93,7 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
   uint64_t t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try(bar, parity)) return true;
+    __nanosleep(64);                                        // leave the issue slots to the working warps
     if ((it & 255u) == 255u) {
       if (*abort_flag) return false;
       const uint64_t now = global_ns();
@@ -162,21 +163,44 @@ __device__ __forceinline__ long long muldiv(long long a, long long b, long long 
 struct Partition {
   const int* seq_len;    // [B]   verified length, or -1 for a sequence that does not fit
   const int* prefix;     // [B+1] flat offset of sequence b
-  int B, H_kv, n_q;
+  const int* aprefix;    // [B+1] first group of sequence b in aligned mode; aprefix[B] < 0: flat mode
+  int B, H_kv, n_q, group, ngroups;
   long long cur, end;
   int b;
-  // Only min(n_groups, W) groups take part, so every taking-part group owns at
-  // least one tile and the groups of one (sequence, head) are consecutive.
-  __device__ void init(const int* sl, const int* pf, int B_, int H, int nq, int group, int n_groups) {
-    seq_len = sl; prefix = pf; B = B_; H_kv = H; n_q = nq; b = 0;
+  // Flat mode: only min(n_groups, W) groups take part, so every taking-part group
+  // owns at least one tile and the groups of one (sequence, head) are consecutive.
+  // Aligned mode (few tiles per group): every (sequence, head) gets a whole number
+  // of groups and is cut evenly among them, so no group straddles two of them and
+  // pays the per-share set-up and epilogue twice.
+  __device__ void init(const int* sl, const int* pf, const int* apf, int B_, int H, int nq, int group_,
+                       int n_groups) {
+    seq_len = sl; prefix = pf; aprefix = apf; B = B_; H_kv = H; n_q = nq; b = 0;
+    group = group_; ngroups = n_groups;
     const long long W = pf[B_];
+    if (apf[B_] >= 0) {                                     // aligned
+      cur = (group_ < apf[B_]) ? 0 : 1; end = 1;
+      return;
+    }
     const long long NG = W < n_groups ? W : n_groups;
-    if (group >= NG) { cur = end = 0; return; }
-    cur = muldiv(W, group, NG);
-    end = muldiv(W, group + 1, NG);
+    if (group_ >= NG) { cur = end = 0; return; }
+    cur = muldiv(W, group_, NG);
+    end = muldiv(W, group_ + 1, NG);
   }
   __device__ bool next(Seg& s) {
     if (cur >= end) return false;
+    if (aprefix[B] >= 0) {                                  // aligned: exactly one share
+      while (aprefix[b + 1] <= group) ++b;
+      const int L = seq_len[b];
+      const int T = (L + n_q + TILE_N - 1) / TILE_N;
+      const int a = (aprefix[b + 1] - aprefix[b]) / H_kv;   // groups per (sequence, head)
+      const int local = group - aprefix[b];
+      const int h = local / a, piece = local - h * a;
+      s.b = b; s.h = h; s.T = T; s.L = L;
+      s.t0 = (T * piece) / a; s.t1 = (T * (piece + 1)) / a;
+      s.slot = group; s.dfirst = aprefix[b] + h * a; s.dn = a;
+      cur = end;
+      return true;
+    }
     while (prefix[b + 1] <= cur) ++b;
     const int L = seq_len[b];
     const int T = (L + n_q + TILE_N - 1) / TILE_N;
@@ -185,6 +209,7 @@ struct Partition {
     long long n = T - s.t0;
     if (n > end - cur) n = end - cur;
     s.t1 = s.t0 + (int)n;
+    s.slot = b * H_kv + s.h + group; s.dfirst = -1; s.dn = 0;
     cur += n;
     return true;
   }
@@ -207,17 +232,19 @@ struct Smem {
   static constexpr int Q_BYTES = Q_ROWS * DH * 2;
   static constexpr int P_PART = NB * TILE_N * 128;           // P_hi or P_lo: [block][key][64 queries] bf16
   static constexpr int K_STAGES = (DH == 128) ? 2 : 3;
-  static constexpr int V_STAGES = (DH == 128) ? (NB == 1 ? 3 : 2) : 4;
+  static constexpr int V_STAGES = (DH == 128) ? 2 : 4;
+  static constexpr int P_BUFS = NB == 1 ? 2 : 1;             // P^T buffers (each P_hi + P_lo)
   static constexpr int Q_OFF = 0;
   static constexpr int K_OFF = Q_BYTES;
   static constexpr int V_OFF = K_OFF + K_STAGES * TILE_BYTES;
   static constexpr int P_OFF = V_OFF + V_STAGES * TILE_BYTES;
-  static constexpr int BAR_OFF = P_OFF + 2 * P_PART;
-  // q_full, q_empty, k_full[], k_empty[], v_full[], v_empty[], s_full[2], p_ready[2], pv_done, drain
-  static constexpr int N_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 4 + 1 + 1;
-  static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;      // tmem base, abort flag
+  static constexpr int BAR_OFF = P_OFF + P_BUFS * 2 * P_PART;
+  // q_full, q_empty, k_full[], k_empty[], v_full[], v_empty[], s_full[2], p_ready[2], pv_done[2], drain
+  static constexpr int N_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 6 + 1;
+  static constexpr int MISC_OFF = BAR_OFF + (N_BARS * 8 + 15) / 16 * 16;   // tmem base, abort flag (16-byte aligned:
+                                                                           // the float arrays below are read as float4)
   static constexpr int MREF_OFF = MISC_OFF + 32;             // [2][128] float: reference maximum per query row
-  static constexpr int XQ_OFF = MREF_OFF + 2 * 128 * 4;          // [4 quarters][128] float: cross-lane reductions
+  static constexpr int XQ_OFF = MREF_OFF + 2 * 128 * 4;      // [4 quarters][128] float: cross-lane reductions
   static constexpr int FQ_OFF = XQ_OFF + 4 * 128 * 4;        // [128] float: rescale factors / final row sums
   static constexpr int TABLE_OFF = FQ_OFF + 128 * 4;         // seq_len[max_batch], prefix[max_batch+1]
 };
@@ -237,23 +264,6 @@ __device__ __forceinline__ bool soft_any(bool pred) {
       : "=r"(r) : "r"((uint32_t)pred) : "memory");
   return r != 0;
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-      ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -263,45 +273,60 @@ __device__ __forceinline__ uint32_t instr_desc_rt(int n, int a_mn, int b_mn) {
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(ROWS >> 4) << 24);
 }
 
-// ---- pieces of the softmax threads that are off the hot path; kept out of line
+// ---- parts of the softmax threads that are off the hot path; kept out of line
 // so that the per-tile loop stays small enough for the instruction cache ----
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
 
-// Which of the 16 query rows of chunk `ch` see block key `jb` (bit e = row ch*16+e).
-__device__ __noinline__ uint32_t block_key_visibility(const uint64_t* mask, int ch, int jb, int i0, int G,
-                                                      int m_valid) {
-  uint32_t v = 0;
+// Which of the query rows col0 .. col0+ncol-1 see block key `jb` (bit = row - col0).
+__device__ __noinline__ uint64_t block_key_visibility(const uint64_t* mask, int col0, int ncol, int jb, int i0,
+                                                      int G, int m_valid) {
+  uint64_t v = 0;
 #pragma unroll 1
-  for (int e = 0; e < 16; ++e) {
-    const int q = ch * 16 + e;
-    if (q < m_valid) v |= (uint32_t)((mask[i0 + q / G] >> jb) & 1ull) << e;
+  for (int e = 0; e < ncol; ++e) {
+    const int q = col0 + e;
+    if (q < m_valid) v |= ((mask[i0 + q / G] >> jb) & 1ull) << e;
   }
   return v;
 }
 
-// Maximum over the 32 keys of this warp for each of the 16 query rows of a chunk
-// (visible entries only); lane 0 stores them at dst[0..15].
-__device__ __noinline__ void chunk_key_max(uint32_t taddr, uint32_t vis, float* dst) {
-  uint32_t sr[16];
-  tmem_ld16(taddr, sr);
+// Maximum over the 32 keys of this warp for each of 8 query rows (visible
+// entries only); lane 0 stores them at dst[0..7].
+__device__ __noinline__ void piece_key_max(uint32_t taddr, uint32_t vis, float* dst) {
+  uint32_t sr[8];
+  tmem_ld8(taddr, sr);
   tmem_wait_ld();
+  float out[8];
 #pragma unroll
-  for (int e = 0; e < 16; ++e) {
+  for (int e = 0; e < 8; ++e) {
     // order-preserving map float -> int so that one integer warp reduction does it
     const int bits = ((vis >> e) & 1u) ? (int)sr[e] : (int)0xFF800000u;      // -inf when not visible
     const int key = bits ^ ((bits >> 31) & 0x7FFFFFFF);
     const int mx = __reduce_max_sync(0xFFFFFFFFu, key);
-    if ((threadIdx.x & 31) == 0) dst[e] = __int_as_float(mx ^ ((mx >> 31) & 0x7FFFFFFF));
+    out[e] = __int_as_float(mx ^ ((mx >> 31) & 0x7FFFFFFF));
+  }
+  if ((threadIdx.x & 31) == 0) {
+    reinterpret_cast<float4*>(dst)[0] = make_float4(out[0], out[1], out[2], out[3]);
+    reinterpret_cast<float4*>(dst)[1] = make_float4(out[4], out[5], out[6], out[7]);
   }
 }
 
-// New reference for the 16 query rows of a chunk from the four quarter maxima in
-// xq; writes the reference to mnew[0..15] and (unless this is a share's first
-// tile) the factor old -> new to fq[0..15].  Every thread of the chunk computes
-// the same values (identical writes).  All pointers are 16-byte aligned.
-__device__ __noinline__ void chunk_new_reference(const float* xq, const float* mold, float* mnew, float* fq,
+// New reference for 8 query rows from the four quarter maxima in xq; writes the
+// reference to mnew[0..7] and (unless this is a share's first tile) the factor
+// old -> new to fq[0..7].  Every thread that owns the rows computes the same
+// values (identical writes).  All pointers are 16-byte aligned.
+__device__ __noinline__ void piece_new_reference(const float* xq, const float* mold, float* mnew, float* fq,
                                                  float c, bool first) {
 #pragma unroll
-  for (int v = 0; v < 4; ++v) {
+  for (int v = 0; v < 2; ++v) {
     const float4 a = reinterpret_cast<const float4*>(xq)[v], b = reinterpret_cast<const float4*>(xq + 128)[v];
     const float4 d = reinterpret_cast<const float4*>(xq + 256)[v], e = reinterpret_cast<const float4*>(xq + 384)[v];
     float tm[4] = {fmaxf(fmaxf(a.x, b.x), fmaxf(d.x, e.x)) * c, fmaxf(fmaxf(a.y, b.y), fmaxf(d.y, e.y)) * c,
@@ -323,14 +348,14 @@ __device__ __noinline__ void chunk_new_reference(const float* xq, const float* m
   }
 }
 
-// O^T[lane][16 columns] *= fq[0..15]
-__device__ __noinline__ void chunk_rescale(uint32_t taddr, const float* fq) {
-  uint32_t o[16];
-  tmem_ld16(taddr, o);
+// O^T[lane][8 columns] *= fq[0..7]
+__device__ __noinline__ void piece_rescale(uint32_t taddr, const float* fq) {
+  uint32_t o[8];
+  tmem_ld8(taddr, o);
   tmem_wait_ld();
 #pragma unroll
-  for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * fq[e]);
-  tmem_st16(taddr, o);
+  for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * fq[e]);
+  tmem_st8(taddr, o);
   tmem_wait_st();
 }
 
@@ -353,7 +378,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   constexpr int B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = B_KFULL + S::K_STAGES,
                 B_VFULL = B_KEMPTY + S::K_STAGES, B_VEMPTY = B_VFULL + S::V_STAGES,
                 B_SFULL = B_VEMPTY + S::V_STAGES, B_PREADY = B_SFULL + 2, B_PVDONE = B_SFULL + 4,
-                B_DRAIN = B_SFULL + 5;
+                B_DRAIN = B_SFULL + 6;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + S::MISC_OFF);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 4);
   float* mref_buf = reinterpret_cast<float*>(sm + S::MREF_OFF);
@@ -361,6 +386,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   float* fq = reinterpret_cast<float*>(sm + S::FQ_OFF);
   int* seq_len = reinterpret_cast<int*>(sm + S::TABLE_OFF);
   int* prefix = seq_len + max_batch;
+  int* aprefix = prefix + max_batch + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int group = blockIdx.x / p.n_mblocks, mb = blockIdx.x % p.n_mblocks;
@@ -368,7 +394,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   // query rows (block row, head) handled here: 0 .. m_valid-1; N of the MMAs is n_pad
   const int m_valid = min(p.rows_per_mb, p.n_q - i0) * p.G;
   const int n_pad = p.n_pad;
-  const int n_chunks = n_pad >> 4;                         // 16-query column chunks
 
   // ---- set-up ------------------------------------------------------------
   pdl_launch_dependents();
@@ -383,6 +408,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       mbar_init(BAR(B_PREADY + i), 256);
     }
     mbar_init(BAR(B_PVDONE), 1);
+    mbar_init(BAR(B_PVDONE + 1), 1);
     mbar_init(BAR(B_DRAIN), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -421,7 +447,34 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       if (b < p.B) { seq_len[b] = L; prefix[b] = carry + incl - tiles; }
       carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
-    if (lane == 0) prefix[p.B] = carry;
+    // aligned mode when a group would get fewer than 8 tiles: groups per (sequence,
+    // head) a_b = floor(groups * T_b / W), at least 1 tile each; fall back to the flat
+    // cut if that needs more groups than there are
+    const int W = carry;
+    __syncwarp();
+    int acarry = 0;
+    bool fits = W > 0 && W < 8 * p.n_groups;
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+      const int b = b0 + lane;
+      int a = 0;
+      if (b < p.B && seq_len[b] >= 0) {
+        const int T = (seq_len[b] + p.n_q + TILE_N - 1) / TILE_N;
+        a = (int)(((long long)p.n_groups * T) / (W > 0 ? W : 1));
+        a = max(1, min(a, T));
+      }
+      int incl = a * p.H_kv;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      if (b < p.B) aprefix[b] = acarry + incl - a * p.H_kv;
+      acarry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+    if (lane == 0) {
+      prefix[p.B] = W;
+      aprefix[p.B] = (fits && acarry <= p.n_groups) ? acarry : -1;
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -431,7 +484,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   const uint32_t TM_S0 = tmem, TM_O = tmem + 256;
 
   Partition part;
-  part.init(seq_len, prefix, p.B, p.H_kv, p.n_q, group, p.n_groups);
+  part.init(seq_len, prefix, aprefix, p.B, p.H_kv, p.n_q, group, p.n_groups);
   Seg sg;
   const bool dead = *abort_flag != 0;
 
@@ -507,18 +560,19 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         if (!mbar_wait(BAR(B_PREADY + (g & 1)), (g >> 1) & 1, abort_flag, p.err, 5)) return false;
         tc_fence_after();
         const uint64_t ad0 = vdesc0 + (uint64_t)((s * S::TILE_BYTES) >> 4);
+        const uint64_t pd0 = pdesc0 + (uint64_t)(((g % S::P_BUFS) * 2 * S::P_PART) >> 4);
 #pragma unroll
         for (int part_i = 0; part_i < 2; ++part_i) {        // P_hi, then P_lo
 #pragma unroll
           for (int kk = 0; kk < TILE_N / 16; ++kk) {
             // 16 keys further = 2048 bytes further in both operands
             mma_ss(TM_O, ad0 + (uint64_t)((kk * 2048) >> 4),
-                   pdesc0 + (uint64_t)((part_i * S::P_PART + kk * 2048) >> 4), idesc_pv,
+                   pd0 + (uint64_t)((part_i * S::P_PART + kk * 2048) >> 4), idesc_pv,
                    (first_in_seg && kk == 0 && part_i == 0) ? 0u : 1u);
           }
         }
         tc_commit(BAR(B_VEMPTY + s));
-        tc_commit(BAR(B_PVDONE));
+        tc_commit(BAR(B_PVDONE + (g & 1)));
         return true;
       };
       while (ok && part.next(sg)) {
@@ -554,20 +608,20 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     }
   } else {
     // ================= softmax / epilogue ==================================
-    // One key of the tile per TMEM lane; two threads per key, which take the
-    // 16-query column chunks alternately (chunk c belongs to half c & 1).
-    constexpr int MAXCH = NB == 1 ? 2 : 4;                 // chunks per thread at most
+    // One key of the tile per TMEM lane; two threads per key, each with one half
+    // of the query-row columns, handled in pieces of 8 columns.
+    constexpr int MAXP = NB == 1 ? 4 : 7;                  // pieces per thread at most
     const int quarter = warp & 3;                          // TMEM lane quarter this warp may touch
     const int half = (warp - WARP_SOFTMAX0) >> 2;
     const int kl = quarter * 32 + lane;                    // key within the tile; head-dim index in the epilogue
     const int sidx = half * 128 + kl;                      // index among the 256 softmax threads
+    const int ncol = n_pad >> 1, col0 = half * ncol, np = ncol >> 3;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const float c = p.scale_log2;
     const uint32_t prow = sm_base + S::P_OFF + kl * 128;   // this key's 128-byte row in each P block
     const uint32_t swz = (uint32_t)(kl & 7);
-    float* xs = reinterpret_cast<float*>(sm + S::P_OFF);   // end-of-share scratch over the idle P buffer
-    float lsum[MAXCH][16];                                 // this key's share of every row sum
-    uint32_t visb[MAXCH];                                  // per chunk: which of its 16 query rows see this key
+    float lsum[MAXP][8];                                   // this key's share of every row sum
+    float sv[MAXP][8];                                     // scores, then score - reference (log2 units)
     uint32_t gt = 0;
     int mpar = 0;                                          // which copy of the references is current
     const float* mref = mref_buf;
@@ -578,134 +632,134 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     while (part.next(sg)) {
       const int n_keys = sg.L + p.n_q;
 #pragma unroll
-      for (int u = 0; u < MAXCH; ++u)
+      for (int j = 0; j < MAXP; ++j)
 #pragma unroll
-        for (int e = 0; e < 16; ++e) lsum[u][e] = 0.f;
+        for (int e = 0; e < 8; ++e) lsum[j][e] = 0.f;
       for (int t = sg.t0; t < sg.t1; ++t, ++gt) {
         const int buf = gt & 1;
         const bool first = (t == sg.t0);
         ok &= mbar_wait(BAR(B_SFULL + buf), (gt >> 1) & 1, abort_flag, p.err, 9);
         tc_fence_after();
-        const uint32_t ts = TM_S0 + buf * 128 + lane_addr;
+        const uint32_t ts = TM_S0 + buf * 128 + lane_addr + col0;
+        // this key's scores for its columns, all loads in flight together
+#pragma unroll
+        for (int j = 0; j < MAXP; ++j)
+          if (j < np) tmem_ld8(ts + j * 8, reinterpret_cast<uint32_t*>(sv[j]));
+        tmem_wait_ld();
         const int lo = t * TILE_N;
         const int kt = ((t + 1) * TILE_N <= n_keys) ? lo : n_keys - TILE_N;
         const int key = kt + kl;
         const int jb = key - sg.L;                         // block key index when >= 0
-        // visibility of this thread's key: keys before `lo` belong to the previous
-        // tile; cached keys are seen by every row; block keys by the Eq. 5 mask
-#pragma unroll
-        for (int u = 0; u < MAXCH; ++u) {
-          const int ch = 2 * u + half;
-          uint32_t v = 0xFFFFu;
-          if (key < lo) v = 0u;
-          else if (jb >= 0 && ch < n_chunks) v = block_key_visibility(p.mask, ch, jb, i0, p.G, m_valid);
-          visb[u] = v;
+        // Visibility of this thread's key: keys before `lo` belong to the previous
+        // tile; cached keys are seen by every row; block keys by the Eq. 5 mask.
+        const bool masked = (kt + TILE_N > sg.L) || (kt < lo);   // same for the whole block
+        uint64_t vis = ~0ull;
+        if (masked) {
+          if (key < lo) vis = 0ull;
+          else if (jb >= 0) vis = block_key_visibility(p.mask, col0, ncol, jb, i0, p.G, m_valid);
         }
-        // ---- pass 0: does any score exceed its row's reference by 2^60? ------
+        // ---- pass 0: score - reference; does any exceed 2^60? -----------------
         bool over = first;
         if (!first) {
+          // (independent maxima per piece: a single running flag would chain every element)
+          float worst[MAXP];
 #pragma unroll
-          for (int u = 0; u < MAXCH; ++u) {
-            const int ch = 2 * u + half;
-            if (ch < n_chunks) {
-              uint32_t sr[16];
-              tmem_ld16(ts + ch * 16, sr);
-              tmem_wait_ld();
-              const float4* mr4 = reinterpret_cast<const float4*>(mref + ch * 16);
-              float worst = -CUDART_INF_F;
+          for (int j = 0; j < MAXP; ++j) {
+            worst[j] = -CUDART_INF_F;
+            if (j < np) {
+              const float4 m0 = reinterpret_cast<const float4*>(mref + col0 + j * 8)[0];
+              const float4 m1 = reinterpret_cast<const float4*>(mref + col0 + j * 8)[1];
+              const float mm[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
 #pragma unroll
-              for (int e4 = 0; e4 < 4; ++e4) {
-                const float4 mr = mr4[e4];
-                const float mm[4] = {mr.x, mr.y, mr.z, mr.w};
+              for (int e = 0; e < 8; ++e) sv[j][e] = fmaf(sv[j][e], c, -mm[e]);
+              if (!masked) {
+                worst[j] = fmaxf(fmaxf(fmaxf(sv[j][0], sv[j][1]), fmaxf(sv[j][2], sv[j][3])),
+                                 fmaxf(fmaxf(sv[j][4], sv[j][5]), fmaxf(sv[j][6], sv[j][7])));
+              } else {
+                const uint32_t vb = (uint32_t)(vis >> (j * 8)) & 0xFFu;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  const float v = fmaf(__uint_as_float(sr[e4 * 4 + e]), c, -mm[e]);
-                  const bool seen = (visb[u] >> (e4 * 4 + e)) & 1u;
-                  worst = fmaxf(worst, seen ? v : -CUDART_INF_F);
-                  over |= seen && (v != v);                 // NaN
-                }
+                for (int e = 0; e < 8; ++e)
+                  worst[j] = fmaxf(worst[j], ((vb >> e) & 1u) ? sv[j][e] : -CUDART_INF_F);
               }
-              over |= worst > OVER_THRESHOLD;
             }
           }
+          float w = worst[0];
+#pragma unroll
+          for (int j = 1; j < MAXP; ++j) w = fmaxf(w, worst[j]);
+          over = !(w <= OVER_THRESHOLD);                    // also true for NaN
         }
         if (soft_any(over)) {
           // ---- re-reference: per query row maximum over the 128 keys of this tile
 #pragma unroll
-          for (int u = 0; u < MAXCH; ++u) {
-            const int ch = 2 * u + half;
-            if (ch < n_chunks) chunk_key_max(ts + ch * 16, visb[u], xq + quarter * 128 + ch * 16);
-          }
+          for (int j = 0; j < MAXP; ++j)
+            if (j < np) piece_key_max(ts + j * 8, (uint32_t)(vis >> (j * 8)) & 0xFFu, xq + quarter * 128 + col0 + j * 8);
           soft_sync();
           // PV of the previous tile must be done before O^T is rescaled
           if (!first) {
-            ok &= mbar_wait(BAR(B_PVDONE), (gt - 1) & 1, abort_flag, p.err, 10);
+            ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 10);
             tc_fence_after();
           }
+          float* mnew = mref_buf + (mpar ^ 1) * 128;
 #pragma unroll
-          for (int u = 0; u < MAXCH; ++u) {
-            const int ch = 2 * u + half;
-            if (ch < n_chunks) {
-              // every thread keeps its own copy of the factors: fq is written and
-              // read back by the same thread with identical values from its peers
-              chunk_new_reference(xq + ch * 16, mref + ch * 16, mref_buf + (mpar ^ 1) * 128 + ch * 16,
-                                  fq + ch * 16, c, first);
+          for (int j = 0; j < MAXP; ++j) {
+            if (j < np) {
+              const int q0 = col0 + j * 8;
+              // fq is written and read back by the same thread (its peers write identical values)
+              piece_new_reference(xq + q0, mref + q0, mnew + q0, fq + q0, c, first);
               __syncwarp();
               if (!first) {
 #pragma unroll
-                for (int e = 0; e < 16; ++e) lsum[u][e] *= fq[ch * 16 + e];
-                chunk_rescale(TM_O + lane_addr + ch * 16, fq + ch * 16);
+                for (int e = 0; e < 8; ++e) lsum[j][e] *= fq[q0 + e];
+                piece_rescale(TM_O + lane_addr + q0, fq + q0);
               }
+              // scores again, now against the new reference
+              uint32_t sr[8];
+              tmem_ld8(ts + j * 8, sr);
+              tmem_wait_ld();
+#pragma unroll
+              for (int e = 0; e < 8; ++e) sv[j][e] = fmaf(__uint_as_float(sr[e]), c, -mnew[q0 + e]);
             }
           }
           mpar ^= 1;
           mref = mref_buf + mpar * 128;
           soft_sync();                                      // new references visible to every thread
         }
-        // the P buffer is free once the PV product of the previous tile has read it
-        if (gt > 0) ok &= mbar_wait(BAR(B_PVDONE), (gt - 1) & 1, abort_flag, p.err, 11);
+        // the P buffer is free once the PV product that last read it has finished
+        {
+          const uint32_t prev = gt - S::P_BUFS;             // tile that used this P buffer before
+          if (gt >= (uint32_t)S::P_BUFS)
+            ok &= mbar_wait(BAR(B_PVDONE + (prev & 1)), (prev >> 1) & 1, abort_flag, p.err, 11);
+        }
+        const uint32_t pbuf = prow + (gt % S::P_BUFS) * (2 * S::P_PART);
         // ---- pass 1: P = exp2(score - reference) as P_hi + P_lo (two bf16 terms:
         // bf16 alone leaves an output error near 1e-2 of the output RMS)
 #pragma unroll
-        for (int u = 0; u < MAXCH; ++u) {
-          const int ch = 2 * u + half;
-          if (ch < n_chunks) {
-            uint32_t sr[16];
-            tmem_ld16(ts + ch * 16, sr);
-            tmem_wait_ld();
-            const uint32_t vis = visb[u];
-            const float4* mr4 = reinterpret_cast<const float4*>(mref + ch * 16);
-            uint32_t hi[8], lw[8];
+        for (int j = 0; j < MAXP; ++j) {
+          if (j < np) {
+            uint32_t hi[4], lw[4];
 #pragma unroll
-            for (int e4 = 0; e4 < 4; ++e4) {
-              const float4 mr = mr4[e4];
-              const float mm[4] = {mr.x, mr.y, mr.z, mr.w};
-              float pv[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
+            for (int e2 = 0; e2 < 4; ++e2) {
+              float p0 = fast_exp2(sv[j][2 * e2]), p1 = fast_exp2(sv[j][2 * e2 + 1]);
+              if (masked) {
                 // a row without any visible key so far has reference -inf and only
-                // invisible entries: the select below keeps those at zero
-                const float x = fast_exp2(fmaf(__uint_as_float(sr[e4 * 4 + e]), c, -mm[e]));
-                pv[e] = ((vis >> (e4 * 4 + e)) & 1u) ? x : 0.f;
-                lsum[u][e4 * 4 + e] += pv[e];
+                // invisible entries: the select keeps those at zero
+                p0 = ((vis >> (j * 8 + 2 * e2)) & 1ull) ? p0 : 0.f;
+                p1 = ((vis >> (j * 8 + 2 * e2 + 1)) & 1ull) ? p1 : 0.f;
               }
-#pragma unroll
-              for (int e2 = 0; e2 < 2; ++e2) {
-                const __nv_bfloat162 h2 = __floats2bfloat162_rn(pv[2 * e2], pv[2 * e2 + 1]);   // .x = lower query row
-                const float2 hf = __bfloat1622float2(h2);
-                const __nv_bfloat162 l2 = __floats2bfloat162_rn(pv[2 * e2] - hf.x, pv[2 * e2 + 1] - hf.y);
-                hi[e4 * 2 + e2] = *reinterpret_cast<const uint32_t*>(&h2);
-                lw[e4 * 2 + e2] = *reinterpret_cast<const uint32_t*>(&l2);
-              }
+              lsum[j][2 * e2] += p0;
+              lsum[j][2 * e2 + 1] += p1;
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);        // .x = lower query row
+              const float2 hf = __bfloat1622float2(h2);
+              const __nv_bfloat162 l2 = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
+              hi[e2] = *reinterpret_cast<const uint32_t*>(&h2);
+              lw[e2] = *reinterpret_cast<const uint32_t*>(&l2);
             }
             // P^T rows are keys; a row holds 64 query rows as eight 16-byte pieces,
             // piece j stored at j ^ (key & 7) (128-byte swizzle)
-            const uint32_t blk = prow + (uint32_t)(ch >> 2) * (TILE_N * 128);
-            const uint32_t j0 = (uint32_t)(ch & 3) * 2;
-            st_shared_v4(blk + (((j0) ^ swz) << 4), hi[0], hi[1], hi[2], hi[3]);
-            st_shared_v4(blk + (((j0 + 1) ^ swz) << 4), hi[4], hi[5], hi[6], hi[7]);
-            st_shared_v4(blk + S::P_PART + (((j0) ^ swz) << 4), lw[0], lw[1], lw[2], lw[3]);
-            st_shared_v4(blk + S::P_PART + (((j0 + 1) ^ swz) << 4), lw[4], lw[5], lw[6], lw[7]);
+            const int q0 = col0 + j * 8;
+            const uint32_t dst = pbuf + (uint32_t)(q0 >> 6) * (TILE_N * 128) + ((((uint32_t)(q0 & 63) >> 3) ^ swz) << 4);
+            st_shared_v4(dst, hi[0], hi[1], hi[2], hi[3]);
+            st_shared_v4(dst + S::P_PART, lw[0], lw[1], lw[2], lw[3]);
           }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core
@@ -713,16 +767,18 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         mbar_arrive(BAR(B_PREADY + buf));
       }
       // ---- end of share: final output or partial ---------------------------
-      ok &= mbar_wait(BAR(B_PVDONE), (gt - 1) & 1, abort_flag, p.err, 12);   // P buffer idle from here
+      ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 12);
+      if (S::P_BUFS == 2 && gt >= 2)                       // both P buffers idle: they become scratch
+        ok &= mbar_wait(BAR(B_PVDONE + (gt & 1)), ((gt - 2) >> 1) & 1, abort_flag, p.err, 13);
       tc_fence_after();
-      // row sums: every key's share goes to scratch as xs[query row][key]; then
-      // thread (row r, piece j) adds 16 keys and an 8-lane shuffle finishes the row
+      float* xs = reinterpret_cast<float*>(sm + S::P_OFF);  // [query row][key] over the idle P buffers
+      // row sums: every key's share goes to scratch; then thread (row r, piece j)
+      // adds 16 keys and an 8-lane shuffle finishes the row
 #pragma unroll
-      for (int u = 0; u < MAXCH; ++u) {
-        const int ch = 2 * u + half;
-        if (ch < n_chunks) {
+      for (int j = 0; j < MAXP; ++j) {
+        if (j < np) {
 #pragma unroll
-          for (int e = 0; e < 16; ++e) xs[(ch * 16 + e) * TILE_N + kl] = lsum[u][e];
+          for (int e = 0; e < 8; ++e) xs[(col0 + j * 8 + e) * TILE_N + kl] = lsum[j][e];
         }
       }
       soft_sync();
@@ -743,17 +799,21 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       soft_sync();
       const bool whole = (sg.t0 == 0 && sg.t1 == sg.T);
       const int item = sg.b * p.H_kv + sg.h;
-      float* pslot = p.part + ((size_t)(item + group) * p.n_mblocks + mb) * (ROWS * (DH + 2));
+      float* pslot = p.part + ((size_t)sg.slot * p.n_mblocks + mb) * (ROWS * (DH + 2));
       if (sidx == 0 && ok) {
-        // how this (sequence, head) was cut: first group and number of groups,
-        // read by attn_merge_kernel (every group of the cut writes the same pair)
-        int2 d = make_int2(group, 1);
-        if (!whole) {
+        // how this (sequence, head) was cut, read by attn_merge_kernel (every group of
+        // the cut writes the same pair)
+        // {first partial slot, number of partials}
+        int2 d = make_int2(sg.slot, 1);
+        if (sg.dfirst >= 0) {
+          d = make_int2(sg.dfirst, sg.dn);
+        } else if (!whole) {
           const long long W = prefix[p.B];
           const long long NG = W < p.n_groups ? W : p.n_groups;
           const long long f0 = (long long)prefix[sg.b] + (long long)sg.h * sg.T;
-          d.x = group_of(f0, W, NG);
-          d.y = group_of(f0 + sg.T - 1, W, NG) - d.x + 1;
+          const int g0 = group_of(f0, W, NG);
+          d.x = item + g0;
+          d.y = group_of(f0 + sg.T - 1, W, NG) - g0 + 1;
         }
         p.desc[(size_t)item * p.n_mblocks + mb] = d;
       }
@@ -773,36 +833,32 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       // consecutive floats of one output row per store.
       const bool d_ok = kl < DH && ok;                      // lanes 64..127 repeat 0..63 when head_dim is 64
 #pragma unroll 1
-      for (int ch = half; ch < n_chunks; ch += 2) {
-        uint32_t o[16];
-        tmem_ld16(TM_O + lane_addr + ch * 16, o);
+      for (int j = 0; j < np; ++j) {
+        uint32_t o[8];
+        const int q0 = col0 + j * 8;
+        tmem_ld8(TM_O + lane_addr + q0, o);
         tmem_wait_ld();
-        const int q0 = ch * 16;
         if (whole) {
           // consecutive query rows are consecutive heads of one block row, then the next block row
           int g = q0 % p.G;
           size_t off = (((size_t)sg.b * p.n_q + (i0 + q0 / p.G)) * p.H_q + sg.h * p.G + g) * DH + kl;
           const size_t row_jump = (size_t)(p.H_q - p.G) * DH;
-          const float4* rv = reinterpret_cast<const float4*>(xq + q0);
+          const float4 r0 = reinterpret_cast<const float4*>(xq + q0)[0], r1 = reinterpret_cast<const float4*>(xq + q0)[1];
+          const float rr[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
 #pragma unroll
-          for (int e4 = 0; e4 < 4; ++e4) {
-            const float4 r4 = rv[e4];
-            const float rr[4] = {r4.x, r4.y, r4.z, r4.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              if (q0 + e4 * 4 + e < m_valid && d_ok) {
-                const float r = __uint_as_float(o[e4 * 4 + e]) * rr[e];
-                if (p.out_dtype == SPACE_DTYPE_F32) reinterpret_cast<float*>(p.out)[off] = r;
-                else reinterpret_cast<__nv_bfloat16*>(p.out)[off] = __float2bfloat16_rn(r);
-              }
-              off += DH;
-              if (++g == p.G) { g = 0; off += row_jump; }
+          for (int e = 0; e < 8; ++e) {
+            if (q0 + e < m_valid && d_ok) {
+              const float r = __uint_as_float(o[e]) * rr[e];
+              if (p.out_dtype == SPACE_DTYPE_F32) reinterpret_cast<float*>(p.out)[off] = r;
+              else reinterpret_cast<__nv_bfloat16*>(p.out)[off] = __float2bfloat16_rn(r);
             }
+            off += DH;
+            if (++g == p.G) { g = 0; off += row_jump; }
           }
         } else {
           float* dst = pslot + (size_t)q0 * DH + kl;
 #pragma unroll
-          for (int e = 0; e < 16; ++e)
+          for (int e = 0; e < 8; ++e)
             if (q0 + e < m_valid && d_ok) dst[e * DH] = __uint_as_float(o[e]);
         }
       }
@@ -845,7 +901,7 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(const AttnParams p) {
   if (idx >= m_valid * C4) return;
   const int r = idx / C4, c4 = idx % C4;
   const size_t slot_floats = (size_t)ROWS * (DH + 2);
-  const float* ps = p.part + ((size_t)(item + d.x) * p.n_mblocks + mb) * slot_floats;
+  const float* ps = p.part + ((size_t)d.x * p.n_mblocks + mb) * slot_floats;
   const size_t gstride = (size_t)p.n_mblocks * slot_floats;
   float mx = -CUDART_INF_F, den = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -935,7 +991,7 @@ void plan(const space_config* cfg, int sm_count, int k, AttnPlanHost* pl) {
 
 template <int DH, int NB>
 size_t smem_bytes(int max_batch) {
-  return Smem<DH, NB>::TABLE_OFF + (size_t)(2 * max_batch + 2) * sizeof(int);
+  return Smem<DH, NB>::TABLE_OFF + (size_t)(3 * max_batch + 3) * sizeof(int);
 }
 
 template <int DH, int NB>
