@@ -17,8 +17,9 @@
 // Inside a block (12 warps):
 //   warps 0, 2  stream K and V tiles with TMA into two rings of shared-memory
 //           stages (a K stage is free once K Q^T has read it, a V stage once V^T P^T has)
-//   warp 3  loads the query rows of the current share with TMA
-//   warp 1  issues tcgen05.mma: S^T into one of two TMEM buffers, then O^T
+//   warp 1  loads the query rows of the current share with TMA and issues the
+//           S^T products (tcgen05.mma) into one of two TMEM buffers
+//   warp 3  issues the O^T products
 //   warps 4-11  two threads per key: read S^T from TMEM, apply the Eq. 5 mask
 //           on tiles that touch the block or a share boundary, P = exp2(score -
 //           reference) as two bf16 terms into shared memory for the second MMA.
@@ -360,7 +361,7 @@ __device__ __noinline__ void piece_rescale(uint32_t taddr, const float* fq) {
 }
 
 // Warp roles
-constexpr int WARP_K = 0, WARP_MMA = 1, WARP_V = 2, WARP_Q = 3, WARP_SOFTMAX0 = 4;
+constexpr int WARP_K = 0, WARP_MMA = 1, WARP_V = 2, WARP_PV = 3, WARP_SOFTMAX0 = 4;
 constexpr float OVER_THRESHOLD = 60.f;   // re-reference a query row when a score exceeds its reference by 2^60
 
 // The tile products are taken transposed: S^T = K Q^T (128 keys x N query rows)
@@ -422,7 +423,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_k) : "memory");
   if (warp == WARP_V && lane == 0)
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_v) : "memory");
-  if (warp == WARP_Q && lane == 0)
+  if (warp == WARP_MMA && lane == 0)
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_q) : "memory");
   pdl_wait();                                              // global memory from here on
   if (warp == WARP_SOFTMAX0) {
@@ -521,13 +522,19 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       const uint32_t first = gt > (uint32_t)n_st ? gt - n_st : 0;
       for (uint32_t g = first; g < gt; ++g) mbar_drain(BAR(b_full + g % n_st), (g / n_st) & 1);
     }
-  } else if (warp == WARP_Q) {
-    // ================= Q producer =========================================
+  } else if (warp == WARP_MMA) {
+    // ================= S^T issuer (also loads the query rows) ================
     if (lane == 0) {
-      uint32_t seg = 0;
-      bool ok = true;
+      const uint32_t idesc_qk = instr_desc_rt(n_pad, 0, 0);   // A = K tile (K-major), B = Q (K-major)
+      // descriptors of the first stage of every operand; a later stage or k-step
+      // only adds to the 14-bit address field (16-byte units, no carry possible)
+      const uint64_t kdesc0 = smem_desc(sm_base + S::K_OFF, 16, 1024);           // K-major rows of 128 bytes
+      const uint64_t qdesc0 = smem_desc(sm_base + S::Q_OFF, 16, 1024);
       const uint32_t q_bytes = (uint32_t)n_pad * DH * 2;
+      uint32_t gt = 0, seg = 0;
+      bool ok = true;
       while (ok && part.next(sg)) {
+        // the previous share's products must have finished reading Q
         if (seg > 0) ok = mbar_wait(BAR(B_QEMPTY), (seg - 1) & 1, abort_flag, p.err, 3);
         if (!ok) break;
         mbar_expect_tx(BAR(B_QFULL), q_bytes);
@@ -535,54 +542,13 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         for (int hf = 0; hf < S::HALVES; ++hf)
           tma_load_4d(sm_base + S::Q_OFF + hf * (n_pad * 128), &p.tm_q, BAR(B_QFULL), hf * 64,
                       sg.h * p.G, i0, sg.b);
-        ++seg;
-      }
-      if (seg > 0) mbar_drain(BAR(B_QFULL), (seg - 1) & 1);
-    }
-  } else if (warp == WARP_MMA) {
-    // ================= MMA issuer =========================================
-    if (lane == 0) {
-      const uint32_t idesc_qk = instr_desc_rt(n_pad, 0, 0);   // A = K tile (K-major), B = Q (K-major)
-      const uint32_t idesc_pv = instr_desc_rt(n_pad, 1, 1);   // A = V^T (d contiguous), B = P^T (queries contiguous)
-      // descriptors of the first stage of every operand; a later stage or k-step
-      // only adds to the 14-bit address field (16-byte units, no carry possible)
-      const uint64_t kdesc0 = smem_desc(sm_base + S::K_OFF, 16, 1024);           // K-major rows of 128 bytes
-      const uint64_t qdesc0 = smem_desc(sm_base + S::Q_OFF, 16, 1024);
-      // V^T and P^T: 64-wide blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
-      const uint64_t vdesc0 = smem_desc(sm_base + S::V_OFF, TILE_N * 128, 1024);
-      const uint64_t pdesc0 = smem_desc(sm_base + S::P_OFF, TILE_N * 128, 1024);
-      uint32_t gt = 0, seg = 0;
-      bool ok = true;
-      // O^T += V^T (P_hi + P_lo)^T for flat tile g (first_in_seg: overwrite O^T)
-      auto issue_pv = [&](uint32_t g, bool first_in_seg) -> bool {
-        const int s = g % S::V_STAGES;
-        if (!mbar_wait(BAR(B_VFULL + s), (g / S::V_STAGES) & 1, abort_flag, p.err, 4)) return false;
-        if (!mbar_wait(BAR(B_PREADY + (g & 1)), (g >> 1) & 1, abort_flag, p.err, 5)) return false;
-        tc_fence_after();
-        const uint64_t ad0 = vdesc0 + (uint64_t)((s * S::TILE_BYTES) >> 4);
-        const uint64_t pd0 = pdesc0 + (uint64_t)(((g % S::P_BUFS) * 2 * S::P_PART) >> 4);
-#pragma unroll
-        for (int part_i = 0; part_i < 2; ++part_i) {        // P_hi, then P_lo
-#pragma unroll
-          for (int kk = 0; kk < TILE_N / 16; ++kk) {
-            // 16 keys further = 2048 bytes further in both operands
-            mma_ss(TM_O, ad0 + (uint64_t)((kk * 2048) >> 4),
-                   pd0 + (uint64_t)((part_i * S::P_PART + kk * 2048) >> 4), idesc_pv,
-                   (first_in_seg && kk == 0 && part_i == 0) ? 0u : 1u);
-          }
-        }
-        tc_commit(BAR(B_VEMPTY + s));
-        tc_commit(BAR(B_PVDONE + (g & 1)));
-        return true;
-      };
-      while (ok && part.next(sg)) {
         ok = mbar_wait(BAR(B_QFULL), seg & 1, abort_flag, p.err, 6);
         const int n = sg.t1 - sg.t0;
         for (int j = 0; j < n && ok; ++j, ++gt) {
           const int s = gt % S::K_STAGES, buf = gt & 1;
-          // S^T buffer `buf` was last read by the softmax of tile gt-2, whose
-          // p_ready this thread has already waited for when it issued that PV
           ok = mbar_wait(BAR(B_KFULL + s), (gt / S::K_STAGES) & 1, abort_flag, p.err, 7);
+          // S^T buffer `buf` was last read by the softmax of tile gt-2
+          if (ok && gt >= 2) ok = mbar_wait(BAR(B_PREADY + buf), ((gt - 2) >> 1) & 1, abort_flag, p.err, 8);
           if (!ok) break;
           tc_fence_after();
           const uint64_t kd = kdesc0 + (uint64_t)((s * S::TILE_BYTES) >> 4);
@@ -597,12 +563,48 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           tc_commit(BAR(B_SFULL + buf));
           tc_commit(BAR(B_KEMPTY + s));
           if (j == n - 1) tc_commit(BAR(B_QEMPTY));
-          if (j > 0) ok = issue_pv(gt - 1, j == 1);
         }
-        if (ok) ok = issue_pv(gt - 1, n == 1);
         ++seg;
       }
-      // all tensor work done before TMEM is released
+      if (seg > 0) mbar_drain(BAR(B_QFULL), (seg - 1) & 1);
+    }
+  } else if (warp == WARP_PV) {
+    // ================= O^T issuer ===========================================
+    // A thread of its own: the S^T products of the next tile need not queue
+    // behind the sixteen instructions of this one.
+    if (lane == 0) {
+      const uint32_t idesc_pv = instr_desc_rt(n_pad, 1, 1);   // A = V^T (d contiguous), B = P^T (queries contiguous)
+      // V^T and P^T: 64-wide blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
+      const uint64_t vdesc0 = smem_desc(sm_base + S::V_OFF, TILE_N * 128, 1024);
+      const uint64_t pdesc0 = smem_desc(sm_base + S::P_OFF, TILE_N * 128, 1024);
+      uint32_t g = 0;
+      bool ok = true;
+      while (ok && part.next(sg)) {
+        for (int t = sg.t0; t < sg.t1 && ok; ++t, ++g) {
+          const int s = g % S::V_STAGES;
+          ok = mbar_wait(BAR(B_VFULL + s), (g / S::V_STAGES) & 1, abort_flag, p.err, 4);
+          if (ok) ok = mbar_wait(BAR(B_PREADY + (g & 1)), (g >> 1) & 1, abort_flag, p.err, 5);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t ad0 = vdesc0 + (uint64_t)((s * S::TILE_BYTES) >> 4);
+          const uint64_t pd0 = pdesc0 + (uint64_t)(((g % S::P_BUFS) * 2 * S::P_PART) >> 4);
+#pragma unroll
+          for (int part_i = 0; part_i < 2; ++part_i) {      // P_hi, then P_lo
+#pragma unroll
+            for (int kk = 0; kk < TILE_N / 16; ++kk) {
+              // 16 keys further = 2048 bytes further in both operands; the first
+              // product of a share overwrites O^T
+              mma_ss(TM_O, ad0 + (uint64_t)((kk * 2048) >> 4),
+                     pd0 + (uint64_t)((part_i * S::P_PART + kk * 2048) >> 4), idesc_pv,
+                     (t == sg.t0 && kk == 0 && part_i == 0) ? 0u : 1u);
+            }
+          }
+          tc_commit(BAR(B_VEMPTY + s));
+          tc_commit(BAR(B_PVDONE + (g & 1)));
+        }
+      }
+      // all tensor work done before TMEM is released (every S^T product was
+      // consumed by the softmax before the O^T product that follows it)
       tc_commit(BAR(B_DRAIN));
       mbar_drain(BAR(B_DRAIN), 0);
     }
