@@ -17,8 +17,8 @@
 // Inside a block (12 warps):
 //   warps 0, 2  stream K and V tiles with TMA into two rings of shared-memory
 //           stages (a K stage is free once K Q^T has read it, a V stage once V^T P^T has)
-//   warp 1  loads the query rows of the current share with TMA and issues the
-//           S^T products (tcgen05.mma) into one of two TMEM buffers
+//           (warp 0 also loads the query rows of each share, one share ahead)
+//   warp 1  issues the S^T products (tcgen05.mma) into one of two TMEM buffers
 //   warp 3  issues the O^T products
 //   warps 4-11  two threads per key: read S^T from TMEM, apply the Eq. 5 mask
 //           on tiles that touch the block or a share boundary, P = exp2(score -
@@ -36,6 +36,7 @@
 namespace {
 
 constexpr int TILE_N = 128;            // keys per tile
+constexpr int SHARE_COST = 3;          // fixed cost of a share (query load, first-tile reference, epilogue) in tiles
 constexpr int ROWS = 128;              // MMA M
 constexpr int THREADS = 384;            // K, MMA, V, Q warps + 8 softmax warps
 constexpr uint64_t WAIT_NS = 1000000000ull;   // one second per wait
@@ -188,8 +189,8 @@ struct Partition {
     end = muldiv(W, group_ + 1, NG);
   }
   __device__ bool next(Seg& s) {
-    if (cur >= end) return false;
-    if (aprefix[B] >= 0) {                                  // aligned: exactly one share
+    if (aprefix[B] >= 0) {
+      if (cur >= end) return false;                                  // aligned: exactly one share
       while (aprefix[b + 1] <= group) ++b;
       const int L = seq_len[b];
       const int T = (L + n_q + TILE_N - 1) / TILE_N;
@@ -202,17 +203,26 @@ struct Partition {
       cur = end;
       return true;
     }
-    while (prefix[b + 1] <= cur) ++b;
-    const int L = seq_len[b];
-    const int T = (L + n_q + TILE_N - 1) / TILE_N;
-    const int rem = (int)(cur - prefix[b]);
-    s.b = b; s.h = rem / T; s.t0 = rem - s.h * T; s.T = T; s.L = L;
-    long long n = T - s.t0;
-    if (n > end - cur) n = end - cur;
-    s.t1 = s.t0 + (int)n;
-    s.slot = b * H_kv + s.h + group; s.dfirst = -1; s.dn = 0;
-    cur += n;
-    return true;
+    // Flat mode: the list holds T + SHARE_COST entries per (sequence, head); the
+    // first SHARE_COST stand for the fixed cost of starting a share there, so
+    // that equal list shares are shares of about equal time.
+    for (;;) {
+      if (cur >= end) return false;
+      while (prefix[b + 1] <= cur) ++b;
+      const int L = seq_len[b];
+      const int T = (L + n_q + TILE_N - 1) / TILE_N;
+      const int Tv = T + SHARE_COST;
+      const int rem = (int)(cur - prefix[b]);
+      const int h = rem / Tv, r0 = rem - h * Tv;
+      long long n = Tv - r0;
+      if (n > end - cur) n = end - cur;
+      cur += n;
+      const int t0 = max(r0 - SHARE_COST, 0), t1 = max(r0 + (int)n - SHARE_COST, 0);
+      if (t1 <= t0) continue;                               // only the cost entries: no tiles here
+      s.b = b; s.h = h; s.t0 = t0; s.t1 = t1; s.T = T; s.L = L;
+      s.slot = b * H_kv + h + group; s.dfirst = -1; s.dn = 0;
+      return true;
+    }
   }
 };
 
@@ -234,14 +244,15 @@ struct Smem {
   static constexpr int P_PART = NB * TILE_N * 128;           // P_hi or P_lo: [block][key][64 queries] bf16
   static constexpr int K_STAGES = (DH == 128) ? 2 : 3;
   static constexpr int V_STAGES = (DH == 128) ? 2 : 4;
-  static constexpr int P_BUFS = NB == 1 ? 2 : 1;             // P^T buffers (each P_hi + P_lo)
+  static constexpr int P_BUFS = 1;                           // P^T buffers (each P_hi + P_lo)
+  static constexpr int Q_BUFS = NB == 1 ? 2 : 1;             // query buffers: the next share's rows load early
   static constexpr int Q_OFF = 0;
-  static constexpr int K_OFF = Q_BYTES;
+  static constexpr int K_OFF = Q_BUFS * Q_BYTES;
   static constexpr int V_OFF = K_OFF + K_STAGES * TILE_BYTES;
   static constexpr int P_OFF = V_OFF + V_STAGES * TILE_BYTES;
   static constexpr int BAR_OFF = P_OFF + P_BUFS * 2 * P_PART;
-  // q_full, q_empty, k_full[], k_empty[], v_full[], v_empty[], s_full[2], p_ready[2], pv_done[2], drain
-  static constexpr int N_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 6 + 1;
+  // q_full[2], q_empty[2], k_full[], k_empty[], v_full[], v_empty[], s_full[2], p_ready[2], pv_done[2], drain
+  static constexpr int N_BARS = 4 + 2 * K_STAGES + 2 * V_STAGES + 6 + 1;
   static constexpr int MISC_OFF = BAR_OFF + (N_BARS * 8 + 15) / 16 * 16;   // tmem base, abort flag (16-byte aligned:
                                                                            // the float arrays below are read as float4)
   static constexpr int MREF_OFF = MISC_OFF + 32;             // [2][128] float: reference maximum per query row
@@ -376,7 +387,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   const uint32_t sm_base = smem_u32(sm);
   const uint32_t bar0 = sm_base + S::BAR_OFF;
   auto BAR = [&](int i) { return bar0 + 8u * i; };
-  constexpr int B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = B_KFULL + S::K_STAGES,
+  constexpr int B_QFULL = 0, B_QEMPTY = 2, B_KFULL = 4, B_KEMPTY = B_KFULL + S::K_STAGES,
                 B_VFULL = B_KEMPTY + S::K_STAGES, B_VEMPTY = B_VFULL + S::V_STAGES,
                 B_SFULL = B_VEMPTY + S::V_STAGES, B_PREADY = B_SFULL + 2, B_PVDONE = B_SFULL + 4,
                 B_DRAIN = B_SFULL + 6;
@@ -400,8 +411,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   pdl_launch_dependents();
   if (threadIdx.x == 0) {
     *abort_flag = (sm_base & 1023u) ? 1 : 0;               // swizzled tiles need a 1024-byte aligned base
-    mbar_init(BAR(B_QFULL), 1);
-    mbar_init(BAR(B_QEMPTY), 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(BAR(B_QFULL + i), 1); mbar_init(BAR(B_QEMPTY + i), 1); }
     for (int s = 0; s < S::K_STAGES; ++s) { mbar_init(BAR(B_KFULL + s), 1); mbar_init(BAR(B_KEMPTY + s), 1); }
     for (int s = 0; s < S::V_STAGES; ++s) { mbar_init(BAR(B_VFULL + s), 1); mbar_init(BAR(B_VEMPTY + s), 1); }
     for (int i = 0; i < 2; ++i) {
@@ -437,7 +447,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         const bool ok = L >= 0 && (int64_t)L + p.n_q <= p.s_cap;
         if (!ok && blockIdx.x == 0 && p.status) atomicOr(p.status + b, SPACE_ST_CAPACITY);
         if (!ok) L = -1;
-        tiles = ok ? ((L + p.n_q + TILE_N - 1) / TILE_N) * p.H_kv : 0;
+        tiles = ok ? ((L + p.n_q + TILE_N - 1) / TILE_N + SHARE_COST) * p.H_kv : 0;
       }
       int incl = tiles;
 #pragma unroll
@@ -451,8 +461,16 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     // aligned mode when a group would get fewer than 8 tiles: groups per (sequence,
     // head) a_b = floor(groups * T_b / W), at least 1 tile each; fall back to the flat
     // cut if that needs more groups than there are
-    const int W = carry;
+    const int Wv = carry;                                  // list entries (tiles + share costs)
     __syncwarp();
+    int W = 0;                                             // real tiles
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+      const int b = b0 + lane;
+      int t = (b < p.B && seq_len[b] >= 0) ? ((seq_len[b] + p.n_q + TILE_N - 1) / TILE_N) * p.H_kv : 0;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+      W += t;
+    }
     int acarry = 0;
     bool fits = W > 0 && W < 8 * p.n_groups;
     for (int b0 = 0; b0 < p.B; b0 += 32) {
@@ -473,7 +491,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       acarry += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
     if (lane == 0) {
-      prefix[p.B] = W;
+      prefix[p.B] = Wv;
       aprefix[p.B] = (fits && acarry <= p.n_groups) ? acarry : -1;
     }
   }
@@ -499,10 +517,24 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       const int b_full = is_k ? B_KFULL : B_VFULL, b_empty = is_k ? B_KEMPTY : B_VEMPTY;
       const uint32_t ring = sm_base + (is_k ? S::K_OFF : S::V_OFF);
       const CUtensorMap* tm = is_k ? &p.tm_k : &p.tm_v;
-      uint32_t gt = 0;
+      uint32_t gt = 0, seg = 0;
       bool ok = true;
+      const uint32_t q_bytes = (uint32_t)n_pad * DH * 2;
       while (ok && part.next(sg)) {
         const int n_keys = sg.L + p.n_q;
+        if (is_k) {
+          // the K producer also loads this share's query rows, into the buffer that
+          // the share before the previous one used (with one buffer: the previous one)
+          const uint32_t qb = seg % S::Q_BUFS, use = seg / S::Q_BUFS;
+          if (use > 0) ok = mbar_wait(BAR(B_QEMPTY + qb), (use - 1) & 1, abort_flag, p.err, 3);
+          if (!ok) break;
+          mbar_expect_tx(BAR(B_QFULL + qb), q_bytes);
+#pragma unroll
+          for (int hf = 0; hf < S::HALVES; ++hf)
+            tma_load_4d(sm_base + S::Q_OFF + qb * S::Q_BYTES + hf * (n_pad * 128), &p.tm_q, BAR(B_QFULL + qb),
+                        hf * 64, sg.h * p.G, i0, sg.b);
+          ++seg;
+        }
         for (int t = sg.t0; t < sg.t1 && ok; ++t, ++gt) {
           const int s = gt % n_st;
           if (gt >= (uint32_t)n_st)
@@ -521,28 +553,25 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       // drain: every issued copy must have landed before the block may exit
       const uint32_t first = gt > (uint32_t)n_st ? gt - n_st : 0;
       for (uint32_t g = first; g < gt; ++g) mbar_drain(BAR(b_full + g % n_st), (g / n_st) & 1);
+      if (is_k && seg > 0) {
+        mbar_drain(BAR(B_QFULL + (seg - 1) % S::Q_BUFS), ((seg - 1) / S::Q_BUFS) & 1);
+        if (S::Q_BUFS == 2 && seg > 1) mbar_drain(BAR(B_QFULL + (seg - 2) % 2), ((seg - 2) / 2) & 1);
+      }
     }
   } else if (warp == WARP_MMA) {
-    // ================= S^T issuer (also loads the query rows) ================
+    // ================= S^T issuer ==========================================
     if (lane == 0) {
       const uint32_t idesc_qk = instr_desc_rt(n_pad, 0, 0);   // A = K tile (K-major), B = Q (K-major)
       // descriptors of the first stage of every operand; a later stage or k-step
       // only adds to the 14-bit address field (16-byte units, no carry possible)
       const uint64_t kdesc0 = smem_desc(sm_base + S::K_OFF, 16, 1024);           // K-major rows of 128 bytes
       const uint64_t qdesc0 = smem_desc(sm_base + S::Q_OFF, 16, 1024);
-      const uint32_t q_bytes = (uint32_t)n_pad * DH * 2;
       uint32_t gt = 0, seg = 0;
       bool ok = true;
       while (ok && part.next(sg)) {
-        // the previous share's products must have finished reading Q
-        if (seg > 0) ok = mbar_wait(BAR(B_QEMPTY), (seg - 1) & 1, abort_flag, p.err, 3);
-        if (!ok) break;
-        mbar_expect_tx(BAR(B_QFULL), q_bytes);
-#pragma unroll
-        for (int hf = 0; hf < S::HALVES; ++hf)
-          tma_load_4d(sm_base + S::Q_OFF + hf * (n_pad * 128), &p.tm_q, BAR(B_QFULL), hf * 64,
-                      sg.h * p.G, i0, sg.b);
-        ok = mbar_wait(BAR(B_QFULL), seg & 1, abort_flag, p.err, 6);
+        const uint32_t qb = seg % S::Q_BUFS, use = seg / S::Q_BUFS;
+        ok = mbar_wait(BAR(B_QFULL + qb), use & 1, abort_flag, p.err, 6);
+        const uint64_t qd = qdesc0 + (uint64_t)((qb * S::Q_BYTES) >> 4);
         const int n = sg.t1 - sg.t0;
         for (int j = 0; j < n && ok; ++j, ++gt) {
           const int s = gt % S::K_STAGES, buf = gt & 1;
@@ -557,16 +586,15 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
             // 64-wide half of d, then 32 bytes per 16 elements inside the swizzled row
             const uint32_t koff = (kk >> 2) * (TILE_N * 128) + (kk & 3) * 32;
             const uint32_t qoff = (kk >> 2) * (n_pad * 128) + (kk & 3) * 32;
-            mma_ss(TM_S0 + buf * 128, kd + (uint64_t)(koff >> 4), qdesc0 + (uint64_t)(qoff >> 4), idesc_qk,
+            mma_ss(TM_S0 + buf * 128, kd + (uint64_t)(koff >> 4), qd + (uint64_t)(qoff >> 4), idesc_qk,
                    kk > 0 ? 1u : 0u);
           }
           tc_commit(BAR(B_SFULL + buf));
           tc_commit(BAR(B_KEMPTY + s));
-          if (j == n - 1) tc_commit(BAR(B_QEMPTY));
+          if (j == n - 1) tc_commit(BAR(B_QEMPTY + qb));
         }
         ++seg;
       }
-      if (seg > 0) mbar_drain(BAR(B_QFULL), (seg - 1) & 1);
     }
   } else if (warp == WARP_PV) {
     // ================= O^T issuer ===========================================
@@ -812,10 +840,10 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         } else if (!whole) {
           const long long W = prefix[p.B];
           const long long NG = W < p.n_groups ? W : p.n_groups;
-          const long long f0 = (long long)prefix[sg.b] + (long long)sg.h * sg.T;
-          const int g0 = group_of(f0, W, NG);
+          const long long f0 = (long long)prefix[sg.b] + (long long)sg.h * (sg.T + SHARE_COST);
+          const int g0 = group_of(f0 + SHARE_COST, W, NG);  // group of the first tile
           d.x = item + g0;
-          d.y = group_of(f0 + sg.T - 1, W, NG) - g0 + 1;
+          d.y = group_of(f0 + SHARE_COST + sg.T - 1, W, NG) - g0 + 1;
         }
         p.desc[(size_t)item * p.n_mblocks + mb] = d;
       }
