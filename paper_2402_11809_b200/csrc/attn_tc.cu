@@ -1053,6 +1053,10 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   const int DH = cfg.head_dim;
   AttnPlanHost pl;
   plan(&cfg, ctx->sm_count, a->k, &pl);
+  // wide query blocks (more than 64 rows per kv head) are better served by the
+  // row-orientation kernel
+  if (((pl.rows_per_mblock * (cfg.n_q_heads / cfg.n_kv_heads) + 15) / 16) * 16 > 64)
+    return launch_attn_rows(ctx, a, mask_rows, st);
   AttnParams p;
   memset(&p, 0, sizeof(p));
   p.B = a->batch; p.n_q = (a->k + 1) * (a->k + 1);
@@ -1093,12 +1097,8 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   const dim3 mgrid(a->batch * p.H_kv * p.n_mblocks, (m_valid_max * (DH / 4) + 127) / 128);
   {
     ProfScope ps(ctx, SPACE_K_ATTN, st);
-    const bool wide = p.n_pad > 64;
-    if (DH == 128) {
-      if (wide) launch_main<128, 2>(p, pl.n_ctas, cfg.max_batch, st); else launch_main<128, 1>(p, pl.n_ctas, cfg.max_batch, st);
-    } else {
-      if (wide) launch_main<64, 2>(p, pl.n_ctas, cfg.max_batch, st); else launch_main<64, 1>(p, pl.n_ctas, cfg.max_batch, st);
-    }
+    if (DH == 128) launch_main<128, 1>(p, pl.n_ctas, cfg.max_batch, st);
+    else launch_main<64, 1>(p, pl.n_ctas, cfg.max_batch, st);
   }
   {
     ProfScope ps(ctx, SPACE_K_MERGE, st);

@@ -85,6 +85,7 @@ int launch_attn_simt(space_ctx* ctx, const space_attn_args* a, const uint64_t* m
                      cudaStream_t st);
 int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t* mask_rows,
                        cudaStream_t st);
+int launch_attn_rows(space_ctx* ctx, const space_attn_args* a, const uint64_t* mask_rows, cudaStream_t st);
 size_t attn_tensor_partial_floats(const space_config* cfg, int sm_count, size_t* slots);
 int launch_philox_debug(uint64_t seed, int64_t n, const uint32_t* c0, const uint32_t* c1,
                         const uint32_t* c2, const uint32_t* c3, uint32_t* out, cudaStream_t st);
