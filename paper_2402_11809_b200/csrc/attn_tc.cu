@@ -55,7 +55,8 @@ struct AttnParams {
   float* part;                         // [slots][ROWS*(DH+2)]
   int* err;                            // one word: first timeout site
   int2* desc;                          // [B*H_kv*n_mblocks] {first partial slot, number of partials} of each cut
-  uint64_t mask[SPACE_MAX_ROWS];
+  uint64_t mask[SPACE_MAX_ROWS];       // bit j of mask[i]: block row i sees block key j
+  uint64_t mask_t[SPACE_MAX_ROWS];     // transposed: bit i of mask_t[j]
 };
 
 struct Seg { int b, h, t0, t1, T, L, slot, dfirst, dn; };   // slot: partial slot; dfirst/dn: cut (aligned mode)
@@ -198,7 +199,10 @@ struct Partition {
       const int local = group - aprefix[b];
       const int h = local / a, piece = local - h * a;
       s.b = b; s.h = h; s.T = T; s.L = L;
-      s.t0 = (T * piece) / a; s.t1 = (T * (piece + 1)) / a;
+      // T = a*q + r: the first r pieces get q+1 tiles, so the last piece, which also
+      // has the tile with the Eq. 5 mask, is never longer than the others
+      const int q = T / a, r = T - q * a;
+      s.t0 = piece * q + min(piece, r); s.t1 = s.t0 + q + (piece < r ? 1 : 0);
       s.slot = group; s.dfirst = aprefix[b] + h * a; s.dn = a;
       cur = end;
       return true;
@@ -299,13 +303,17 @@ __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
 }
 
 // Which of the query rows col0 .. col0+ncol-1 see block key `jb` (bit = row - col0).
-__device__ __noinline__ uint64_t block_key_visibility(const uint64_t* mask, int col0, int ncol, int jb, int i0,
-                                                      int G, int m_valid) {
+// rows_t = mask_t[jb]: bit i set when block row i sees the key; query row q is
+// block row i0 + q / G.
+__device__ __noinline__ uint64_t block_key_visibility(uint64_t rows_t, int col0, int ncol, int i0, int G,
+                                                      int m_valid) {
+  const uint64_t rel = rows_t >> i0;
   uint64_t v = 0;
+  int r = col0 / G, g = col0 - r * G;
 #pragma unroll 1
   for (int e = 0; e < ncol; ++e) {
-    const int q = col0 + e;
-    if (q < m_valid) v |= ((mask[i0 + q / G] >> jb) & 1ull) << e;
+    if (col0 + e < m_valid) v |= ((rel >> r) & 1ull) << e;
+    if (++g == G) { g = 0; ++r; }
   }
   return v;
 }
@@ -520,6 +528,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       uint32_t gt = 0, seg = 0;
       bool ok = true;
       const uint32_t q_bytes = (uint32_t)n_pad * DH * 2;
+      // The very first S^T product needs only Q and the first K tile: V holds back
+      // until that K tile has landed, so that it does not share the opening burst.
+      bool v_hold = !is_k;
       while (ok && part.next(sg)) {
         const int n_keys = sg.L + p.n_q;
         if (is_k) {
@@ -540,6 +551,11 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           if (gt >= (uint32_t)n_st)
             ok = mbar_wait(BAR(b_empty + s), ((gt / n_st) - 1) & 1, abort_flag, p.err, is_k ? 1 : 2);
           if (!ok) break;
+          if (v_hold) {
+            ok = mbar_wait(BAR(B_KFULL), 0, abort_flag, p.err, 14);
+            v_hold = false;
+            if (!ok) break;
+          }
           // the last tile of a sequence is shifted back so that it ends at the
           // last key: rows past the end are never read (they may hold anything)
           const int kt = ((t + 1) * TILE_N <= n_keys) ? t * TILE_N : n_keys - TILE_N;
@@ -686,7 +702,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         uint64_t vis = ~0ull;
         if (masked) {
           if (key < lo) vis = 0ull;
-          else if (jb >= 0) vis = block_key_visibility(p.mask, col0, ncol, jb, i0, p.G, m_valid);
+          else if (jb >= 0) vis = block_key_visibility(p.mask_t[jb], col0, ncol, i0, p.G, m_valid);
         }
         // ---- pass 0: score - reference; does any exceed 2^60? -----------------
         bool over = first;
@@ -1070,6 +1086,11 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   p.part = ctx->attn_part; p.err = ctx->counters + 3 * cfg.max_batch;
   p.desc = reinterpret_cast<int2*>(ctx->merge_cnt);
   for (int i = 0; i < SPACE_MAX_ROWS; ++i) p.mask[i] = mask_rows[i];
+  for (int j = 0; j < SPACE_MAX_ROWS; ++j) {
+    uint64_t t = 0;
+    for (int i = 0; i < SPACE_MAX_ROWS; ++i) t |= ((mask_rows[i] >> j) & 1ull) << i;
+    p.mask_t[j] = t;
+  }
 
   // TMA descriptors, rebuilt only when a base pointer or a stride changes
   const int64_t key[8] = {a->kv_stride_b, a->kv_stride_h, a->kv_stride_s, a->batch, p.n_q, p.n_pad, 0, 0};
