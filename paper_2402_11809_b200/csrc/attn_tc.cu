@@ -704,9 +704,29 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           if (key < lo) vis = 0ull;
           else if (jb >= 0) vis = block_key_visibility(p.mask_t[jb], col0, ncol, i0, p.G, m_valid);
         }
+        // ---- first tile of a share, every key visible: the scores of the tile's
+        // first key serve as references.  Any reference within 2^60 of the row
+        // maximum is as good as the maximum itself (P keeps its relative precision
+        // as P_hi + P_lo, sums are fp32); pass 0 below checks exactly that bound.
+        if (first && !masked) {
+          float* mnew = mref_buf + (mpar ^ 1) * 128;
+          if (kl == 0) {
+#pragma unroll
+            for (int j = 0; j < MAXP; ++j) {
+              if (j < np) {
+                float4* dst = reinterpret_cast<float4*>(mnew + col0 + j * 8);
+                dst[0] = make_float4(sv[j][0] * c, sv[j][1] * c, sv[j][2] * c, sv[j][3] * c);
+                dst[1] = make_float4(sv[j][4] * c, sv[j][5] * c, sv[j][6] * c, sv[j][7] * c);
+              }
+            }
+          }
+          soft_sync();
+          mpar ^= 1;
+          mref = mref_buf + mpar * 128;
+        }
         // ---- pass 0: score - reference; does any exceed 2^60? -----------------
-        bool over = first;
-        if (!first) {
+        bool over = first && masked;
+        if (!over) {
           // (independent maxima per piece: a single running flag would chain every element)
           float worst[MAXP];
 #pragma unroll
