@@ -167,43 +167,38 @@ struct Partition {
   const int* seq_len;    // [B]   verified length, or -1 for a sequence that does not fit
   const int* prefix;     // [B+1] flat offset of sequence b
   const int* aprefix;    // [B+1] first group of sequence b in aligned mode; aprefix[B] < 0: flat mode
+  const int* seg0;       // aligned mode: {b, h, t0, t1, T, L, first group of the cut, groups in the cut}
   int B, H_kv, n_q, group, ngroups;
   long long cur, end;
   int b;
+  bool aligned;
   // Flat mode: only min(n_groups, W) groups take part, so every taking-part group
   // owns at least one tile and the groups of one (sequence, head) are consecutive.
   // Aligned mode (few tiles per group): every (sequence, head) gets a whole number
   // of groups and is cut evenly among them, so no group straddles two of them and
   // pays the per-share set-up and epilogue twice.
-  __device__ void init(const int* sl, const int* pf, const int* apf, int B_, int H, int nq, int group_,
-                       int n_groups) {
-    seq_len = sl; prefix = pf; aprefix = apf; B = B_; H_kv = H; n_q = nq; b = 0;
+  __device__ void init(const int* sl, const int* pf, const int* apf, const int* seg0_, int B_, int H, int nq,
+                       int group_, int n_groups) {
+    seq_len = sl; prefix = pf; aprefix = apf; seg0 = seg0_; B = B_; H_kv = H; n_q = nq; b = 0;
     group = group_; ngroups = n_groups;
-    const long long W = pf[B_];
-    if (apf[B_] >= 0) {                                     // aligned
+    aligned = apf[B_] >= 0;
+    if (aligned) {
       cur = (group_ < apf[B_]) ? 0 : 1; end = 1;
       return;
     }
+    const long long W = pf[B_];
     const long long NG = W < n_groups ? W : n_groups;
     if (group_ >= NG) { cur = end = 0; return; }
     cur = muldiv(W, group_, NG);
     end = muldiv(W, group_ + 1, NG);
   }
   __device__ bool next(Seg& s) {
-    if (aprefix[B] >= 0) {
-      if (cur >= end) return false;                                  // aligned: exactly one share
-      while (aprefix[b + 1] <= group) ++b;
-      const int L = seq_len[b];
-      const int T = (L + n_q + TILE_N - 1) / TILE_N;
-      const int a = (aprefix[b + 1] - aprefix[b]) / H_kv;   // groups per (sequence, head)
-      const int local = group - aprefix[b];
-      const int h = local / a, piece = local - h * a;
-      s.b = b; s.h = h; s.T = T; s.L = L;
-      // T = a*q + r: the first r pieces get q+1 tiles, so the last piece, which also
-      // has the tile with the Eq. 5 mask, is never longer than the others
-      const int q = T / a, r = T - q * a;
-      s.t0 = piece * q + min(piece, r); s.t1 = s.t0 + q + (piece < r ? 1 : 0);
-      s.slot = group; s.dfirst = aprefix[b] + h * a; s.dn = a;
+    if (aligned) {
+      // exactly one share, worked out once per thread block during the set-up
+      if (cur >= end) return false;
+      const int4 u = reinterpret_cast<const int4*>(seg0)[0], v = reinterpret_cast<const int4*>(seg0)[1];
+      s.b = u.x; s.h = u.y; s.t0 = u.z; s.t1 = u.w; s.T = v.x; s.L = v.y; s.dfirst = v.z; s.dn = v.w;
+      s.slot = group;
       cur = end;
       return true;
     }
@@ -259,7 +254,8 @@ struct Smem {
   static constexpr int N_BARS = 4 + 2 * K_STAGES + 2 * V_STAGES + 6 + 1;
   static constexpr int MISC_OFF = BAR_OFF + (N_BARS * 8 + 15) / 16 * 16;   // tmem base, abort flag (16-byte aligned:
                                                                            // the float arrays below are read as float4)
-  static constexpr int MREF_OFF = MISC_OFF + 32;             // [2][128] float: reference maximum per query row
+  static constexpr int SEG0_OFF = MISC_OFF + 16;             // Seg of this group's only share (aligned mode)
+  static constexpr int MREF_OFF = MISC_OFF + 64;             // [2][128] float: reference maximum per query row
   static constexpr int XQ_OFF = MREF_OFF + 2 * 128 * 4;      // [4 quarters][128] float: cross-lane reductions
   static constexpr int FQ_OFF = XQ_OFF + 4 * 128 * 4;        // [128] float: rescale factors / final row sums
   static constexpr int TABLE_OFF = FQ_OFF + 128 * 4;         // seq_len[max_batch], prefix[max_batch+1]
@@ -407,6 +403,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   int* seq_len = reinterpret_cast<int*>(sm + S::TABLE_OFF);
   int* prefix = seq_len + max_batch;
   int* aprefix = prefix + max_batch + 1;
+  int* seg0 = reinterpret_cast<int*>(sm + S::SEG0_OFF);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int group = blockIdx.x / p.n_mblocks, mb = blockIdx.x % p.n_mblocks;
@@ -446,13 +443,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   pdl_wait();                                              // global memory from here on
   if (warp == WARP_SOFTMAX0) {
     // per-sequence tile counts and their running sum, 32 sequences per round
-    int carry = 0;
+    int carry = 0, nvalid = 0;
     for (int b0 = 0; b0 < p.B; b0 += 32) {
       const int b = b0 + lane;
       int L = -1, tiles = 0;
+      bool ok = false;
       if (b < p.B) {
         L = p.kv_len[b];
-        const bool ok = L >= 0 && (int64_t)L + p.n_q <= p.s_cap;
+        ok = L >= 0 && (int64_t)L + p.n_q <= p.s_cap;
         if (!ok && blockIdx.x == 0 && p.status) atomicOr(p.status + b, SPACE_ST_CAPACITY);
         if (!ok) L = -1;
         tiles = ok ? ((L + p.n_q + TILE_N - 1) / TILE_N + SHARE_COST) * p.H_kv : 0;
@@ -465,42 +463,51 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       }
       if (b < p.B) { seq_len[b] = L; prefix[b] = carry + incl - tiles; }
       carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+      nvalid += __popc(__ballot_sync(0xFFFFFFFFu, ok));
     }
     // aligned mode when a group would get fewer than 8 tiles: groups per (sequence,
     // head) a_b = floor(groups * T_b / W), at least 1 tile each; fall back to the flat
     // cut if that needs more groups than there are
     const int Wv = carry;                                  // list entries (tiles + share costs)
-    __syncwarp();
-    int W = 0;                                             // real tiles
-    for (int b0 = 0; b0 < p.B; b0 += 32) {
-      const int b = b0 + lane;
-      int t = (b < p.B && seq_len[b] >= 0) ? ((seq_len[b] + p.n_q + TILE_N - 1) / TILE_N) * p.H_kv : 0;
+    const int W = Wv - SHARE_COST * p.H_kv * nvalid;       // real tiles
+    int acarry = -1;
+    if (W > 0 && W < 8 * p.n_groups) {
+      acarry = 0;
+      for (int b0 = 0; b0 < p.B; b0 += 32) {
+        const int b = b0 + lane;
+        int a = 0, T = 0, L = -1;
+        if (b < p.B) L = seq_len[b];                         // written by this lane above
+        if (L >= 0) {
+          T = (L + p.n_q + TILE_N - 1) / TILE_N;
+          a = (int)muldiv(p.n_groups, T, W);
+          a = max(1, min(a, T));
+        }
+        int incl = a * p.H_kv;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
-      W += t;
-    }
-    int acarry = 0;
-    bool fits = W > 0 && W < 8 * p.n_groups;
-    for (int b0 = 0; b0 < p.B; b0 += 32) {
-      const int b = b0 + lane;
-      int a = 0;
-      if (b < p.B && seq_len[b] >= 0) {
-        const int T = (seq_len[b] + p.n_q + TILE_N - 1) / TILE_N;
-        a = (int)(((long long)p.n_groups * T) / (W > 0 ? W : 1));
-        a = max(1, min(a, T));
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+          if (lane >= o) incl += v;
+        }
+        const int first = acarry + incl - a * p.H_kv;        // first group of sequence b
+        if (b < p.B) aprefix[b] = first;
+        if (a > 0 && group >= first && group < first + a * p.H_kv) {
+          // this group's share: head h, piece `piece` of a.  T = a*q + r: the first r
+          // pieces get q+1 tiles, so the last piece, which also has the tile with
+          // the Eq. 5 mask, is never longer than the others
+          const int local = group - first;
+          const int h = local / a, piece = local - h * a;
+          const int q = T / a, r = T - q * a;
+          const int t0 = piece * q + min(piece, r);
+          reinterpret_cast<int4*>(seg0)[0] = make_int4(b, h, t0, t0 + q + (piece < r ? 1 : 0));
+          reinterpret_cast<int4*>(seg0)[1] = make_int4(T, L, first + h * a, a);
+        }
+        acarry += __shfl_sync(0xFFFFFFFFu, incl, 31);
       }
-      int incl = a * p.H_kv;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += v;
-      }
-      if (b < p.B) aprefix[b] = acarry + incl - a * p.H_kv;
-      acarry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+      if (acarry > p.n_groups) acarry = -1;
     }
     if (lane == 0) {
       prefix[p.B] = Wv;
-      aprefix[p.B] = (fits && acarry <= p.n_groups) ? acarry : -1;
+      aprefix[p.B] = acarry;
     }
   }
   tc_fence_before();
@@ -511,7 +518,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   const uint32_t TM_S0 = tmem, TM_O = tmem + 256;
 
   Partition part;
-  part.init(seq_len, prefix, aprefix, p.B, p.H_kv, p.n_q, group, p.n_groups);
+  part.init(seq_len, prefix, aprefix, seg0, p.B, p.H_kv, p.n_q, group, p.n_groups);
   Seg sg;
   const bool dead = *abort_flag != 0;
 
@@ -617,8 +624,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     // A thread of its own: the S^T products of the next tile need not queue
     // behind the sixteen instructions of this one.
     if (lane == 0) {
-      const uint32_t idesc_pv = instr_desc_rt(n_pad, 1, 1);   // A = V^T (d contiguous), B = P^T (queries contiguous)
+      // B = [P_hi | P_lo]: the two 64-column blocks lie one leading-dimension stride
+      // apart, so a single product of N = 128 gives O_hi^T in columns 0..63 and
+      // O_lo^T in columns 64..127 (an instruction costs the same at every N here);
+      // the epilogue adds the two.  Columns past the padded query rows hold whatever
+      // the shared memory held; they only reach output columns nobody reads.
+      const uint32_t idesc_pv = instr_desc_rt(128, 1, 1);     // A = V^T (d contiguous), B = P^T (queries contiguous)
       // V^T and P^T: 64-wide blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
+      static_assert(S::P_PART == TILE_N * 128, "P_lo must follow P_hi at the block stride");
       const uint64_t vdesc0 = smem_desc(sm_base + S::V_OFF, TILE_N * 128, 1024);
       const uint64_t pdesc0 = smem_desc(sm_base + S::P_OFF, TILE_N * 128, 1024);
       uint32_t g = 0;
@@ -633,15 +646,11 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           const uint64_t ad0 = vdesc0 + (uint64_t)((s * S::TILE_BYTES) >> 4);
           const uint64_t pd0 = pdesc0 + (uint64_t)(((g % S::P_BUFS) * 2 * S::P_PART) >> 4);
 #pragma unroll
-          for (int part_i = 0; part_i < 2; ++part_i) {      // P_hi, then P_lo
-#pragma unroll
-            for (int kk = 0; kk < TILE_N / 16; ++kk) {
-              // 16 keys further = 2048 bytes further in both operands; the first
-              // product of a share overwrites O^T
-              mma_ss(TM_O, ad0 + (uint64_t)((kk * 2048) >> 4),
-                     pd0 + (uint64_t)((part_i * S::P_PART + kk * 2048) >> 4), idesc_pv,
-                     (t == sg.t0 && kk == 0 && part_i == 0) ? 0u : 1u);
-            }
+          for (int kk = 0; kk < TILE_N / 16; ++kk) {
+            // 16 keys further = 2048 bytes further in both operands; the first
+            // product of a share overwrites O^T
+            mma_ss(TM_O, ad0 + (uint64_t)((kk * 2048) >> 4), pd0 + (uint64_t)((kk * 2048) >> 4), idesc_pv,
+                   (t == sg.t0 && kk == 0) ? 0u : 1u);
           }
           tc_commit(BAR(B_VEMPTY + s));
           tc_commit(BAR(B_PVDONE + (g & 1)));
@@ -777,6 +786,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
 #pragma unroll
                 for (int e = 0; e < 8; ++e) lsum[j][e] *= fq[q0 + e];
                 piece_rescale(TM_O + lane_addr + q0, fq + q0);
+                piece_rescale(TM_O + lane_addr + 64 + q0, fq + q0);
               }
               // scores again, now against the new reference
               uint32_t sr[8];
@@ -833,35 +843,37 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         mbar_arrive(BAR(B_PREADY + buf));
       }
       // ---- end of share: final output or partial ---------------------------
-      ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 12);
-      if (S::P_BUFS == 2 && gt >= 2)                       // both P buffers idle: they become scratch
-        ok &= mbar_wait(BAR(B_PVDONE + (gt & 1)), ((gt - 2) >> 1) & 1, abort_flag, p.err, 13);
-      tc_fence_after();
-      float* xs = reinterpret_cast<float*>(sm + S::P_OFF);  // [query row][key] over the idle P buffers
-      // row sums: every key's share goes to scratch; then thread (row r, piece j)
-      // adds 16 keys and an 8-lane shuffle finishes the row
+      // Row sums first, while the last O^T product still runs.  Every thread holds
+      // its key's share of up to 32 rows; a halving butterfly over the warp leaves
+      // lane r with the sum over the warp's 32 keys for row col0 + r.
+      static_assert(MAXP * 8 == 32, "the butterfly below folds 32 values over 32 lanes");
+      {
+        float red[32];
 #pragma unroll
-      for (int j = 0; j < MAXP; ++j) {
-        if (j < np) {
+        for (int j = 0; j < MAXP; ++j)
 #pragma unroll
-          for (int e = 0; e < 8; ++e) xs[(col0 + j * 8 + e) * TILE_N + kl] = lsum[j][e];
+          for (int e = 0; e < 8; ++e) red[j * 8 + e] = (j < np) ? lsum[j][e] : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const bool up = (lane & o) != 0;
+#pragma unroll
+          for (int i = 0; i < o; ++i) {
+            const float send = up ? red[i] : red[i + o];
+            const float keep = up ? red[i + o] : red[i];
+            red[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, o);
+          }
         }
+        if (lane < ncol) xq[quarter * 128 + col0 + lane] = red[0];
       }
       soft_sync();
-      for (int base = 0; base < n_pad; base += 32) {
-        const int r = base + (sidx >> 3), j = sidx & 7;
-        float v = 0.f;
-        if (r < n_pad) {
-          const float4* src = reinterpret_cast<const float4*>(xs + r * TILE_N + j * 16);
-          const float4 a = src[0], b = src[1], cc = src[2], d = src[3];
-          v = ((a.x + a.y) + (a.z + a.w)) + ((b.x + b.y) + (b.z + b.w)) +
-              ((cc.x + cc.y) + (cc.z + cc.w)) + ((d.x + d.y) + (d.z + d.w));
-        }
-        v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-        v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
-        v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
-        if (j == 0 && r < n_pad) { fq[r] = v; xq[r] = 1.f / v; }   // row sums and their reciprocals
+      float* rcp = mref_buf + (mpar ^ 1) * 128;             // the idle copy of the references
+      if (sidx < n_pad) {
+        const float v = (xq[sidx] + xq[128 + sidx]) + (xq[256 + sidx] + xq[384 + sidx]);
+        fq[sidx] = v;                                        // row sums and their reciprocals
+        rcp[sidx] = 1.f / v;
       }
+      ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 12);
+      tc_fence_after();
       soft_sync();
       const bool whole = (sg.t0 == 0 && sg.t1 == sg.T);
       const int item = sg.b * p.H_kv + sg.h;
@@ -898,18 +910,21 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       // O^T: lane = head-dim index, column = query row.  A warp writes 32
       // consecutive floats of one output row per store.
       const bool d_ok = kl < DH && ok;                      // lanes 64..127 repeat 0..63 when head_dim is 64
-#pragma unroll 1
+#pragma unroll 2
       for (int j = 0; j < np; ++j) {
-        uint32_t o[8];
+        uint32_t o[8], o2[8];
         const int q0 = col0 + j * 8;
         tmem_ld8(TM_O + lane_addr + q0, o);
+        tmem_ld8(TM_O + lane_addr + 64 + q0, o2);
         tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) + __uint_as_float(o2[e]));
         if (whole) {
           // consecutive query rows are consecutive heads of one block row, then the next block row
           int g = q0 % p.G;
           size_t off = (((size_t)sg.b * p.n_q + (i0 + q0 / p.G)) * p.H_q + sg.h * p.G + g) * DH + kl;
           const size_t row_jump = (size_t)(p.H_q - p.G) * DH;
-          const float4 r0 = reinterpret_cast<const float4*>(xq + q0)[0], r1 = reinterpret_cast<const float4*>(xq + q0)[1];
+          const float4 r0 = reinterpret_cast<const float4*>(rcp + q0)[0], r1 = reinterpret_cast<const float4*>(rcp + q0)[1];
           const float rr[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
