@@ -27,9 +27,8 @@ import numpy as np
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
-sys.path.insert(0, os.path.join(ROOT, "tests"))
 
-from paper_2402_11809_b200 import workloads  # noqa: E402
+from paper_2402_11809_b200 import replicas, workloads  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per attn_tc_kernel launch from the ncu capture summarised
@@ -137,8 +136,8 @@ def time_oracle(cfg, x, budget_s, min_reps=3, max_reps=None):
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    rank, _, _ = replicas.rank_env()
+    if rank != 0:                                         # rank 0 alone times the oracle
         return
     cfg = workloads.resolve(args.config)
     x = workloads.make_step_inputs(cfg)
@@ -169,20 +168,16 @@ def run_reference(args):
 # --------------------------------------------------------------------- CUDA arm
 def run_ours(args):
     import torch
-    import torch.distributed as dist
-    import gpu_harness as H
+    from paper_2402_11809_b200 import device as H
     from paper_2402_11809_b200 import build
     build.build()
     from paper_2402_11809_b200 import binding as B
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = replicas.rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py --impl ours needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    replicas.init("nccl", local)
 
     cfg = workloads.resolve(args.config)
     k, n_q = cfg["k"], workloads.n_block_rows(cfg["k"])
@@ -190,11 +185,11 @@ def run_ours(args):
     mode = B.MODE_SAMPLE if sample else B.MODE_GREEDY
 
     # ---- input sets: enough distinct sets that their footprint is twice L2 ----
-    x0 = workloads.make_step_inputs(cfg, set_index=rank * 1000)
+    x0 = workloads.make_step_inputs(cfg, set_index=replicas.set_index(rank, 0))
     ab = workloads.algorithmic_bytes(cfg, x0["kv_len"])
     n_sets = max(2, int(np.ceil(2.0 * L2_BYTES / ab["total"])))
     n_sets = min(n_sets, 16)
-    sets = [x0] + [workloads.make_step_inputs(cfg, set_index=rank * 1000 + i) for i in range(1, n_sets)]
+    sets = [x0] + [workloads.make_step_inputs(cfg, set_index=replicas.set_index(rank, i)) for i in range(1, n_sets)]
 
     s_cap = max(x["s_cap"] for x in sets)
     ctx = B.Context(device=local, max_batch=cfg["B"], n_q_heads=cfg["H_q"], n_kv_heads=cfg["H_kv"],
@@ -252,8 +247,7 @@ def run_ours(args):
         run_steps(W)
         stream.synchronize()
         sampler = ClockSampler(local)
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
         sampler.start()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -262,8 +256,7 @@ def run_ours(args):
         e1.record(stream)
         stream.synchronize()
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         ms = e0.elapsed_time(e1)
         # keep the sampler running through the kernel-timing pass as well
         # ---- second pass: per-kernel CUDA events, stream-launched ------------
@@ -277,11 +270,8 @@ def run_ours(args):
         clocks = sampler.stop()
         status = sum(int(ds.status.abs().sum()) for ds in steps_dev)
 
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    steps_per_s = world * K / (ms * 1e-3)
+    steps_per_s, sec = replicas.job_throughput(K, ms * 1e-3, device="cuda")
+    ms = sec * 1e3
 
     # ---- end to end from pinned host buffers (space_step_host) ---------------
     import ctypes as C
@@ -321,17 +311,12 @@ def run_ours(args):
             ctx.space_step_host(hs)
         torch.cuda.synchronize()
         e2e_s = time.perf_counter() - t0
-    e2e_val = n_e2e / e2e_s
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_val = world * n_e2e / float(t.item())
+    e2e_val, _ = replicas.job_throughput(n_e2e, e2e_s, device="cuda")
     e2e_ok = bool((outs["status"] == 0).all()) and \
         bool(torch.equal(outs["n_accept"], steps_dev[0].n_accept.cpu()))
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        replicas.shutdown()
         return
 
     # ---- roofline of the dominant kernel (attention) --------------------------
@@ -376,8 +361,7 @@ def run_ours(args):
         "device_status_bits": status,
     }
     print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.shutdown()
 
 
 def main():
