@@ -33,7 +33,7 @@ from paper_2402_11809_b200 import replicas, workloads  # noqa: E402
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per attn_tc_kernel launch from the ncu capture summarised
 # in profiles/attn_tc_kernel_llama7b.txt (bytes); None for workloads without a capture of the current kernel
-ATTN_TRAFFIC = {"llama7b": None}
+ATTN_TRAFFIC = {"llama7b": 34517760}
 METRIC = "auto-correct steps/sec"
 UNIT = "steps/s"
 
