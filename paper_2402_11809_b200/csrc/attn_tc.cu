@@ -166,7 +166,6 @@ __device__ __forceinline__ long long muldiv(long long a, long long b, long long 
 struct Partition {
   const int* seq_len;    // [B]   verified length, or -1 for a sequence that does not fit
   const int* prefix;     // [B+1] flat offset of sequence b
-  const int* aprefix;    // [B+1] first group of sequence b in aligned mode; aprefix[B] < 0: flat mode
   const int* seg0;       // aligned mode: {b, h, t0, t1, T, L, first group of the cut, groups in the cut}
   int B, H_kv, n_q, group, ngroups;
   long long cur, end;
@@ -177,13 +176,14 @@ struct Partition {
   // Aligned mode (few tiles per group): every (sequence, head) gets a whole number
   // of groups and is cut evenly among them, so no group straddles two of them and
   // pays the per-share set-up and epilogue twice.
-  __device__ void init(const int* sl, const int* pf, const int* apf, const int* seg0_, int B_, int H, int nq,
+  // agroups: groups that have a share in aligned mode, or < 0 for flat mode
+  __device__ void init(const int* sl, const int* pf, int agroups, const int* seg0_, int B_, int H, int nq,
                        int group_, int n_groups) {
-    seq_len = sl; prefix = pf; aprefix = apf; seg0 = seg0_; B = B_; H_kv = H; n_q = nq; b = 0;
+    seq_len = sl; prefix = pf; seg0 = seg0_; B = B_; H_kv = H; n_q = nq; b = 0;
     group = group_; ngroups = n_groups;
-    aligned = apf[B_] >= 0;
+    aligned = agroups >= 0;
     if (aligned) {
-      cur = (group_ < apf[B_]) ? 0 : 1; end = 1;
+      cur = (group_ < agroups) ? 0 : 1; end = 1;
       return;
     }
     const long long W = pf[B_];
@@ -243,7 +243,9 @@ struct Smem {
   static constexpr int P_PART = NB * TILE_N * 128;           // P_hi or P_lo: [block][key][64 queries] bf16
   static constexpr int K_STAGES = (DH == 128) ? 2 : 3;
   static constexpr int V_STAGES = (DH == 128) ? 2 : 4;
-  static constexpr int P_BUFS = 1;                           // P^T buffers (each P_hi + P_lo)
+  static constexpr int P_BUFS = 1;                           // P^T buffers (each P_hi + P_lo); a second one, so that the exponentials of a tile
+                                                             // overlap the O^T product of the tile before, measured no faster
+  static constexpr int RS = 64 * NB;                         // query rows (padded) per thread block at most
   static constexpr int Q_BUFS = NB == 1 ? 2 : 1;             // query buffers: the next share's rows load early
   static constexpr int Q_OFF = 0;
   static constexpr int K_OFF = Q_BUFS * Q_BYTES;
@@ -255,10 +257,12 @@ struct Smem {
   static constexpr int MISC_OFF = BAR_OFF + (N_BARS * 8 + 15) / 16 * 16;   // tmem base, abort flag (16-byte aligned:
                                                                            // the float arrays below are read as float4)
   static constexpr int SEG0_OFF = MISC_OFF + 16;             // Seg of this group's only share (aligned mode)
-  static constexpr int MREF_OFF = MISC_OFF + 64;             // [2][128] float: reference maximum per query row
-  static constexpr int XQ_OFF = MREF_OFF + 2 * 128 * 4;      // [4 quarters][128] float: cross-lane reductions
-  static constexpr int FQ_OFF = XQ_OFF + 4 * 128 * 4;        // [128] float: rescale factors / final row sums
-  static constexpr int TABLE_OFF = FQ_OFF + 128 * 4;         // seq_len[max_batch], prefix[max_batch+1]
+  static constexpr int MREF_OFF = MISC_OFF + 64;             // [2][RS] float: reference maximum per query row
+  static constexpr int XQ_OFF = MREF_OFF + 2 * RS * 4;       // [4 quarters][RS] float: cross-lane reductions
+  static constexpr int FQ_OFF = XQ_OFF + 4 * RS * 4;         // [RS] float: rescale factors / final row sums
+  static constexpr int TABLE_OFF = FQ_OFF + RS * 4;          // seq_len[max_batch], prefix[max_batch+1]
+  // with the tables of the largest batch (128 sequences) the plan must fit the 227 KB a block may have
+  static_assert(TABLE_OFF + (2 * 128 + 1) * 4 <= 227 * 1024, "shared-memory plan too large");
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -335,16 +339,16 @@ __device__ __noinline__ void piece_key_max(uint32_t taddr, uint32_t vis, float* 
   }
 }
 
-// New reference for 8 query rows from the four quarter maxima in xq; writes the
+// New reference for 8 query rows from the four quarter maxima in xq (rs floats apart); writes the
 // reference to mnew[0..7] and (unless this is a share's first tile) the factor
 // old -> new to fq[0..7].  Every thread that owns the rows computes the same
 // values (identical writes).  All pointers are 16-byte aligned.
-__device__ __noinline__ void piece_new_reference(const float* xq, const float* mold, float* mnew, float* fq,
+__device__ __noinline__ void piece_new_reference(const float* xq, int rs, const float* mold, float* mnew, float* fq,
                                                  float c, bool first) {
 #pragma unroll
   for (int v = 0; v < 2; ++v) {
-    const float4 a = reinterpret_cast<const float4*>(xq)[v], b = reinterpret_cast<const float4*>(xq + 128)[v];
-    const float4 d = reinterpret_cast<const float4*>(xq + 256)[v], e = reinterpret_cast<const float4*>(xq + 384)[v];
+    const float4 a = reinterpret_cast<const float4*>(xq)[v], b = reinterpret_cast<const float4*>(xq + rs)[v];
+    const float4 d = reinterpret_cast<const float4*>(xq + 2 * rs)[v], e = reinterpret_cast<const float4*>(xq + 3 * rs)[v];
     float tm[4] = {fmaxf(fmaxf(a.x, b.x), fmaxf(d.x, e.x)) * c, fmaxf(fmaxf(a.y, b.y), fmaxf(d.y, e.y)) * c,
                    fmaxf(fmaxf(a.z, b.z), fmaxf(d.z, e.z)) * c, fmaxf(fmaxf(a.w, b.w), fmaxf(d.w, e.w)) * c};
     float mo[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
@@ -402,7 +406,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   float* fq = reinterpret_cast<float*>(sm + S::FQ_OFF);
   int* seq_len = reinterpret_cast<int*>(sm + S::TABLE_OFF);
   int* prefix = seq_len + max_batch;
-  int* aprefix = prefix + max_batch + 1;
+  volatile int* agroups = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 8);
   int* seg0 = reinterpret_cast<int*>(sm + S::SEG0_OFF);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -489,7 +493,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           if (lane >= o) incl += v;
         }
         const int first = acarry + incl - a * p.H_kv;        // first group of sequence b
-        if (b < p.B) aprefix[b] = first;
         if (a > 0 && group >= first && group < first + a * p.H_kv) {
           // this group's share: head h, piece `piece` of a.  T = a*q + r: the first r
           // pieces get q+1 tiles, so the last piece, which also has the tile with
@@ -507,7 +510,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     }
     if (lane == 0) {
       prefix[p.B] = Wv;
-      aprefix[p.B] = acarry;
+      *agroups = acarry;
     }
   }
   tc_fence_before();
@@ -518,7 +521,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   const uint32_t TM_S0 = tmem, TM_O = tmem + 256;
 
   Partition part;
-  part.init(seq_len, prefix, aprefix, seg0, p.B, p.H_kv, p.n_q, group, p.n_groups);
+  part.init(seq_len, prefix, *agroups, seg0, p.B, p.H_kv, p.n_q, group, p.n_groups);
   Seg sg;
   const bool dead = *abort_flag != 0;
 
@@ -718,7 +721,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         // maximum is as good as the maximum itself (P keeps its relative precision
         // as P_hi + P_lo, sums are fp32); pass 0 below checks exactly that bound.
         if (first && !masked) {
-          float* mnew = mref_buf + (mpar ^ 1) * 128;
+          float* mnew = mref_buf + (mpar ^ 1) * S::RS;
           if (kl == 0) {
 #pragma unroll
             for (int j = 0; j < MAXP; ++j) {
@@ -731,7 +734,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           }
           soft_sync();
           mpar ^= 1;
-          mref = mref_buf + mpar * 128;
+          mref = mref_buf + mpar * S::RS;
         }
         // ---- pass 0: score - reference; does any exceed 2^60? -----------------
         bool over = first && masked;
@@ -767,20 +770,20 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           // ---- re-reference: per query row maximum over the 128 keys of this tile
 #pragma unroll
           for (int j = 0; j < MAXP; ++j)
-            if (j < np) piece_key_max(ts + j * 8, (uint32_t)(vis >> (j * 8)) & 0xFFu, xq + quarter * 128 + col0 + j * 8);
+            if (j < np) piece_key_max(ts + j * 8, (uint32_t)(vis >> (j * 8)) & 0xFFu, xq + quarter * S::RS + col0 + j * 8);
           soft_sync();
           // PV of the previous tile must be done before O^T is rescaled
           if (!first) {
             ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 10);
             tc_fence_after();
           }
-          float* mnew = mref_buf + (mpar ^ 1) * 128;
+          float* mnew = mref_buf + (mpar ^ 1) * S::RS;
 #pragma unroll
           for (int j = 0; j < MAXP; ++j) {
             if (j < np) {
               const int q0 = col0 + j * 8;
               // fq is written and read back by the same thread (its peers write identical values)
-              piece_new_reference(xq + q0, mref + q0, mnew + q0, fq + q0, c, first);
+              piece_new_reference(xq + q0, S::RS, mref + q0, mnew + q0, fq + q0, c, first);
               __syncwarp();
               if (!first) {
 #pragma unroll
@@ -797,7 +800,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
             }
           }
           mpar ^= 1;
-          mref = mref_buf + mpar * 128;
+          mref = mref_buf + mpar * S::RS;
           soft_sync();                                      // new references visible to every thread
         }
         // the P buffer is free once the PV product that last read it has finished
@@ -863,12 +866,12 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
             red[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, o);
           }
         }
-        if (lane < ncol) xq[quarter * 128 + col0 + lane] = red[0];
+        if (lane < ncol) xq[quarter * S::RS + col0 + lane] = red[0];
       }
       soft_sync();
-      float* rcp = mref_buf + (mpar ^ 1) * 128;             // the idle copy of the references
+      float* rcp = mref_buf + (mpar ^ 1) * S::RS;            // the idle copy of the references
       if (sidx < n_pad) {
-        const float v = (xq[sidx] + xq[128 + sidx]) + (xq[256 + sidx] + xq[384 + sidx]);
+        const float v = (xq[sidx] + xq[S::RS + sidx]) + (xq[2 * S::RS + sidx] + xq[3 * S::RS + sidx]);
         fq[sidx] = v;                                        // row sums and their reciprocals
         rcp[sidx] = 1.f / v;
       }
@@ -1072,7 +1075,7 @@ void plan(const space_config* cfg, int sm_count, int k, AttnPlanHost* pl) {
 
 template <int DH, int NB>
 size_t smem_bytes(int max_batch) {
-  return Smem<DH, NB>::TABLE_OFF + (size_t)(3 * max_batch + 3) * sizeof(int);
+  return Smem<DH, NB>::TABLE_OFF + (size_t)(2 * max_batch + 1) * sizeof(int);
 }
 
 template <int DH, int NB>
