@@ -197,7 +197,8 @@ def run_ours(args):
     steps_dev = [H.DeviceStep(cfg, x) for x in sets]
     arg_sets = []
     for ds in steps_dev:
-        a = ctx.attn_args(ds.q, ds.k_cache, ds.v_cache, ds.kv_len, ds.out, k, ds.scale, status=ds.status)
+        a = ctx.attn_args(ds.q, ds.k_cache, ds.v_cache, ds.kv_len, ds.out, k, ds.scale, status=ds.status,
+                          impl=B.ATTN_TENSOR_ROWS if args.attn_impl == "rows" else B.ATTN_TENSOR)
         v = ctx.verify_args(ds.logits, ds.cand, ds.cand_prob, ds.kv_len, ds.n_accept, ds.out_tokens,
                             ds.n_out, ds.next_cand, ds.next_cand_prob, ds.finished, k, mode=mode,
                             temperature=cfg["temperature"], seed=cfg["seed"], seq_id=ds.seq_id,
@@ -371,6 +372,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--config", default="llama7b", choices=sorted(workloads.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--attn-impl", default="tensor", choices=["tensor", "rows"],
+                    help="tensor: keys on the MMA M extent (default); rows: query rows on M")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -49,7 +49,7 @@ enum { SPACE_MASK_SAME_GROUP = 0, SPACE_MASK_EQ5_LITERAL = 1 };
 enum { SPACE_MODE_GREEDY = 0, SPACE_MODE_SAMPLE = 1 };
 enum { SPACE_RESAMPLE_RESIDUAL_POINTMASS = 0, SPACE_RESAMPLE_PAPER_LITERAL = 1 };
 enum { SPACE_DTYPE_BF16 = 0, SPACE_DTYPE_F32 = 1 };
-enum { SPACE_ATTN_TENSOR = 0, SPACE_ATTN_SIMT = 1 };
+enum { SPACE_ATTN_TENSOR = 0, SPACE_ATTN_SIMT = 1, SPACE_ATTN_TENSOR_ROWS = 2 };
 
 /* per-sequence device status bits */
 enum {
@@ -93,7 +93,8 @@ typedef struct {
   int32_t k;                /* candidates per sequence                         */
   int32_t mask_variant;     /* SPACE_MASK_*                                    */
   int32_t out_dtype;        /* SPACE_DTYPE_F32 or SPACE_DTYPE_BF16             */
-  int32_t impl;             /* SPACE_ATTN_TENSOR (default) or SPACE_ATTN_SIMT  */
+  int32_t impl;             /* SPACE_ATTN_TENSOR (default: keys on the MMA M extent),
+                               SPACE_ATTN_TENSOR_ROWS (query rows on M) or SPACE_ATTN_SIMT */
   float   scale;            /* softmax scale, normally 1/sqrt(d)               */
   const void*    q;         /* device bf16 [B, n_q, H_q, d], contiguous        */
   const void*    k_cache;   /* device bf16, element (b,h,s,:) at               */

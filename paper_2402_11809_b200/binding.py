@@ -20,7 +20,7 @@ MASK_SAME_GROUP, MASK_EQ5_LITERAL = 0, 1
 MODE_GREEDY, MODE_SAMPLE = 0, 1
 RESAMPLE_RESIDUAL_POINTMASS, RESAMPLE_PAPER_LITERAL = 0, 1
 DTYPE_BF16, DTYPE_F32 = 0, 1
-ATTN_TENSOR, ATTN_SIMT = 0, 1
+ATTN_TENSOR, ATTN_SIMT, ATTN_TENSOR_ROWS = 0, 1, 2
 ST_CAPACITY, ST_BAD_CANDIDATE, ST_TIMEOUT = 1, 2, 4
 
 EXPORTS = ["space_create", "space_destroy", "space_workspace_bytes", "space_layout",

@@ -20,9 +20,12 @@ namespace {
 
 constexpr int TILE_N = 128;            // keys per tile
 constexpr int ROWS = 128;              // MMA M
-constexpr int THREADS = 384;            // K, MMA, V, Q warps + 8 softmax warps
+constexpr int THREADS = 384;            // K (+Q), S-issuer, V, O-issuer warps + 8 softmax warps
 constexpr uint64_t WAIT_NS = 1000000000ull;   // one second per wait
 constexpr float RESCALE_THRESHOLD = 8.f;
+// Starting a share (query load, pipeline refill, epilogue) costs about as much as
+// this many tiles; the flat list carries that many extra entries per (sequence, head).
+constexpr int SHARE_COST = 4;
 
 struct AttnParams {
   CUtensorMap tm_q, tm_k, tm_v;
@@ -196,17 +199,25 @@ struct Partition {
     end = muldiv(W, group + 1, NG);
   }
   __device__ bool next(Seg& s) {
-    if (cur >= end) return false;
-    while (prefix[b + 1] <= cur) ++b;
-    const int L = seq_len[b];
-    const int T = (L + n_q + TILE_N - 1) / TILE_N;
-    const int rem = (int)(cur - prefix[b]);
-    s.b = b; s.h = rem / T; s.t0 = rem - s.h * T; s.T = T; s.L = L;
-    long long n = T - s.t0;
-    if (n > end - cur) n = end - cur;
-    s.t1 = s.t0 + (int)n;
-    cur += n;
-    return true;
+    // The list holds T + SHARE_COST entries per (sequence, head); the first
+    // SHARE_COST stand for the fixed cost of starting a share there, so that
+    // equal list shares are shares of about equal time.
+    for (;;) {
+      if (cur >= end) return false;
+      while (prefix[b + 1] <= cur) ++b;
+      const int L = seq_len[b];
+      const int T = (L + n_q + TILE_N - 1) / TILE_N;
+      const int Tv = T + SHARE_COST;
+      const int rem = (int)(cur - prefix[b]);
+      const int h = rem / Tv, r0 = rem - h * Tv;
+      long long n = Tv - r0;
+      if (n > end - cur) n = end - cur;
+      cur += n;
+      const int t0 = max(r0 - SHARE_COST, 0), t1 = max(r0 + (int)n - SHARE_COST, 0);
+      if (t1 <= t0) continue;                               // only cost entries here: no tiles
+      s.b = b; s.h = h; s.t0 = t0; s.t1 = t1; s.T = T; s.L = L;
+      return true;
+    }
   }
 };
 
@@ -228,9 +239,10 @@ struct Smem {
   static constexpr int K_OFF = Q_BYTES;
   static constexpr int V_OFF = K_OFF + K_STAGES * TILE_BYTES;
   static constexpr int BAR_OFF = V_OFF + V_STAGES * TILE_BYTES;
-  // q_full, q_empty, k_full[], k_empty[], v_full[], v_empty[], s_full[2], p_ready[2], pv_done[2], drain
-  static constexpr int N_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 6 + 1;
-  static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;      // tmem base, abort flag
+  static constexpr int S_BUFS = 3;                           // S / P buffers in TMEM (3 x 128 columns, O at 384)
+  // q_full, q_empty, k_full[], k_empty[], v_full[], v_empty[], s_full[3], p_ready[3], pv_done[3], drain
+  static constexpr int N_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 3 * S_BUFS + 1;
+  static constexpr int MISC_OFF = BAR_OFF + (N_BARS * 8 + 15) / 16 * 16;   // tmem base, abort flag
   static constexpr int XMAX_OFF = MISC_OFF + 32;             // [2 parities][2 halves][ROWS] float
   static constexpr int XSUM_OFF = XMAX_OFF + 2 * 2 * ROWS * 4;   // [2 halves][ROWS] float
   static constexpr int TABLE_OFF = XSUM_OFF + 2 * ROWS * 4;  // seq_len[max_batch], prefix[max_batch+1]
@@ -248,7 +260,7 @@ __device__ __forceinline__ void pair_sync(int quarter) {
 }
 
 // Warp roles
-constexpr int WARP_K = 0, WARP_MMA = 1, WARP_V = 2, WARP_Q = 3, WARP_SOFTMAX0 = 4;
+constexpr int WARP_K = 0, WARP_MMA = 1, WARP_V = 2, WARP_PV = 3, WARP_SOFTMAX0 = 4;
 
 template <int DH>
 __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_constant__ AttnParams p,
@@ -260,8 +272,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
   auto BAR = [&](int i) { return bar0 + 8u * i; };
   constexpr int B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = B_KFULL + S::K_STAGES,
                 B_VFULL = B_KEMPTY + S::K_STAGES, B_VEMPTY = B_VFULL + S::V_STAGES,
-                B_SFULL = B_VEMPTY + S::V_STAGES, B_PREADY = B_SFULL + 2, B_PVDONE = B_SFULL + 4,
-                B_DRAIN = B_SFULL + 6;
+                B_SFULL = B_VEMPTY + S::V_STAGES, B_PREADY = B_SFULL + S::S_BUFS,
+                B_PVDONE = B_SFULL + 2 * S::S_BUFS, B_DRAIN = B_SFULL + 3 * S::S_BUFS;
+  constexpr uint32_t NS = S::S_BUFS;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + S::MISC_OFF);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 4);
   float* xmax = reinterpret_cast<float*>(sm + S::XMAX_OFF);
@@ -285,7 +298,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
     mbar_init(BAR(B_QEMPTY), 1);
     for (int s = 0; s < S::K_STAGES; ++s) { mbar_init(BAR(B_KFULL + s), 1); mbar_init(BAR(B_KEMPTY + s), 1); }
     for (int s = 0; s < S::V_STAGES; ++s) { mbar_init(BAR(B_VFULL + s), 1); mbar_init(BAR(B_VEMPTY + s), 1); }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < S::S_BUFS; ++i) {
       mbar_init(BAR(B_SFULL + i), 1);
       mbar_init(BAR(B_PREADY + i), n_soft);
       mbar_init(BAR(B_PVDONE + i), 1);
@@ -306,7 +319,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
         const bool ok = L >= 0 && (int64_t)L + p.n_q <= p.s_cap;
         if (!ok && blockIdx.x == 0 && p.status) atomicOr(p.status + b, SPACE_ST_CAPACITY);
         if (!ok) L = -1;
-        tiles = ok ? ((L + p.n_q + TILE_N - 1) / TILE_N) * p.H_kv : 0;
+        tiles = ok ? ((L + p.n_q + TILE_N - 1) / TILE_N + SHARE_COST) * p.H_kv : 0;
       }
       int incl = tiles;
 #pragma unroll
@@ -328,13 +341,13 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_k) : "memory");
   if (warp == WARP_V && lane == 0)
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_v) : "memory");
-  if (warp == WARP_Q && lane == 0)
+  if (warp == WARP_MMA && lane == 0)
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_q) : "memory");
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t TM_S0 = tmem, TM_O = tmem + 2 * TILE_N;    // S buffers at columns 0 and 128, O at 256
+  const uint32_t TM_S0 = tmem, TM_O = tmem + S::S_BUFS * TILE_N;   // S buffers at columns 0, 128, 256; O at 384
 
   Partition part;
   part.init(seq_len, prefix, p.B, p.H_kv, p.n_q, group, p.n_groups);
@@ -351,10 +364,22 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
       const int b_full = is_k ? B_KFULL : B_VFULL, b_empty = is_k ? B_KEMPTY : B_VEMPTY;
       const uint32_t ring = sm_base + (is_k ? S::K_OFF : S::V_OFF);
       const CUtensorMap* tm = is_k ? &p.tm_k : &p.tm_v;
-      uint32_t gt = 0;
+      uint32_t gt = 0, seg = 0;
       bool ok = true;
       while (ok && part.next(sg)) {
         const int n_keys = sg.L + p.n_q;
+        if (is_k) {
+          // the K producer also loads this share's query rows, once the last S
+          // product of the share before has read the buffer
+          if (seg > 0) ok = mbar_wait(BAR(B_QEMPTY), (seg - 1) & 1, abort_flag, p.err, 3);
+          if (!ok) break;
+          mbar_expect_tx(BAR(B_QFULL), S::Q_BYTES);
+#pragma unroll
+          for (int hf = 0; hf < S::HALVES; ++hf)
+            tma_load_4d(sm_base + S::Q_OFF + hf * (ROWS * 128), &p.tm_q, BAR(B_QFULL), hf * 64,
+                        sg.h * p.G, i0, sg.b);
+          ++seg;
+        }
         for (int t = sg.t0; t < sg.t1 && ok; ++t, ++gt) {
           const int s = gt % n_st;
           if (gt >= (uint32_t)n_st)
@@ -373,60 +398,23 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
       // drain: every issued copy must have landed before the block may exit
       const uint32_t first = gt > (uint32_t)n_st ? gt - n_st : 0;
       for (uint32_t g = first; g < gt; ++g) mbar_drain(BAR(b_full + g % n_st), (g / n_st) & 1);
-    }
-  } else if (warp == WARP_Q) {
-    // ================= Q producer =========================================
-    if (lane == 0) {
-      uint32_t seg = 0;
-      bool ok = true;
-      while (ok && part.next(sg)) {
-        if (seg > 0) ok = mbar_wait(BAR(B_QEMPTY), (seg - 1) & 1, abort_flag, p.err, 3);
-        if (!ok) break;
-        mbar_expect_tx(BAR(B_QFULL), S::Q_BYTES);
-#pragma unroll
-        for (int hf = 0; hf < S::HALVES; ++hf)
-          tma_load_4d(sm_base + S::Q_OFF + hf * (ROWS * 128), &p.tm_q, BAR(B_QFULL), hf * 64,
-                      sg.h * p.G, i0, sg.b);
-        ++seg;
-      }
-      if (seg > 0) mbar_drain(BAR(B_QFULL), (seg - 1) & 1);
+      if (is_k && seg > 0) mbar_drain(BAR(B_QFULL), (seg - 1) & 1);
     }
   } else if (warp == WARP_MMA) {
-    // ================= MMA issuer =========================================
+    // ================= S issuer ============================================
     if (lane == 0) {
       constexpr uint32_t IDESC_QK = instr_desc(TILE_N, 0);
-      constexpr uint32_t IDESC_PV = instr_desc(DH, 1);
       uint32_t gt = 0, seg = 0;
       bool ok = true;
-      // O += (P_hi + P_lo) V for flat tile g (first_in_seg: overwrite O)
-      auto issue_pv = [&](uint32_t g, bool first_in_seg) -> bool {
-        const int s = g % S::V_STAGES, buf = g & 1;
-        if (!mbar_wait(BAR(B_VFULL + s), (g / S::V_STAGES) & 1, abort_flag, p.err, 4)) return false;
-        if (!mbar_wait(BAR(B_PREADY + buf), (g >> 1) & 1, abort_flag, p.err, 5)) return false;
-        tc_fence_after();
-        const uint32_t vsm = sm_base + S::V_OFF + s * S::TILE_BYTES;
-        const uint32_t ptm = TM_S0 + buf * TILE_N;
-#pragma unroll
-        for (int part_i = 0; part_i < 2; ++part_i) {        // P_hi, then P_lo
-#pragma unroll
-          for (int kk = 0; kk < TILE_N / 16; ++kk) {
-            // V tile is MN-major: 64-wide d blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
-            const uint64_t bd = smem_desc(vsm + kk * 2048, TILE_N * 128, 1024);
-            mma_ts(TM_O, ptm + part_i * (TILE_N / 2) + kk * 8, bd, IDESC_PV,
-                   (first_in_seg && kk == 0 && part_i == 0) ? 0u : 1u);
-          }
-        }
-        tc_commit(BAR(B_VEMPTY + s));
-        tc_commit(BAR(B_PVDONE + buf));
-        return true;
-      };
       while (ok && part.next(sg)) {
         ok = mbar_wait(BAR(B_QFULL), seg & 1, abort_flag, p.err, 6);
         const int n = sg.t1 - sg.t0;
         for (int j = 0; j < n && ok; ++j, ++gt) {
-          const int s = gt % S::K_STAGES, buf = gt & 1;
+          const int s = gt % S::K_STAGES;
+          const uint32_t buf = gt % NS;
           ok = mbar_wait(BAR(B_KFULL + s), (gt / S::K_STAGES) & 1, abort_flag, p.err, 7);
-          if (ok && gt >= 2) ok = mbar_wait(BAR(B_PVDONE + buf), ((gt >> 1) - 1) & 1, abort_flag, p.err, 8);
+          // S buffer `buf` held the P of tile gt - 3, read by that tile's O product
+          if (ok && gt >= NS) ok = mbar_wait(BAR(B_PVDONE + buf), ((gt / NS) - 1) & 1, abort_flag, p.err, 8);
           if (!ok) break;
           tc_fence_after();
           const uint32_t qsm = sm_base + S::Q_OFF;
@@ -440,12 +428,45 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
           tc_commit(BAR(B_SFULL + buf));
           tc_commit(BAR(B_KEMPTY + s));
           if (j == n - 1) tc_commit(BAR(B_QEMPTY));
-          if (j > 0) ok = issue_pv(gt - 1, j == 1);
         }
-        if (ok) ok = issue_pv(gt - 1, n == 1);
         ++seg;
       }
-      // all tensor work done before TMEM is released
+    }
+  } else if (warp == WARP_PV) {
+    // ================= O issuer ============================================
+    // A thread of its own: the S products of later tiles need not queue behind
+    // the sixteen instructions of an O product or wait for its operands.
+    if (lane == 0) {
+      constexpr uint32_t IDESC_PV = instr_desc(DH, 1);
+      uint32_t g = 0;
+      bool ok = true;
+      while (ok && part.next(sg)) {
+        for (int t = sg.t0; t < sg.t1 && ok; ++t, ++g) {
+          // O += (P_hi + P_lo) V; the first product of a share overwrites O
+          const int s = g % S::V_STAGES;
+          const uint32_t buf = g % NS;
+          ok = mbar_wait(BAR(B_VFULL + s), (g / S::V_STAGES) & 1, abort_flag, p.err, 4);
+          if (ok) ok = mbar_wait(BAR(B_PREADY + buf), (g / NS) & 1, abort_flag, p.err, 5);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t vsm = sm_base + S::V_OFF + s * S::TILE_BYTES;
+          const uint32_t ptm = TM_S0 + buf * TILE_N;
+#pragma unroll
+          for (int part_i = 0; part_i < 2; ++part_i) {        // P_hi, then P_lo
+#pragma unroll
+            for (int kk = 0; kk < TILE_N / 16; ++kk) {
+              // V tile is MN-major: 64-wide d blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
+              const uint64_t bd = smem_desc(vsm + kk * 2048, TILE_N * 128, 1024);
+              mma_ts(TM_O, ptm + part_i * (TILE_N / 2) + kk * 8, bd, IDESC_PV,
+                     (t == sg.t0 && kk == 0 && part_i == 0) ? 0u : 1u);
+            }
+          }
+          tc_commit(BAR(B_VEMPTY + s));
+          tc_commit(BAR(B_PVDONE + buf));
+        }
+      }
+      // all tensor work done before TMEM is released (every S product was read by
+      // the softmax before the O product that follows it was issued)
       tc_commit(BAR(B_DRAIN));
       mbar_drain(BAR(B_DRAIN), 0);
     }
@@ -474,8 +495,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
       const int n_keys = sg.L + p.n_q;
       float m_ref = -CUDART_INF_F, l_sum = 0.f;
       for (int t = sg.t0; t < sg.t1; ++t, ++gt) {
-        const int buf = gt & 1;
-        ok &= mbar_wait(BAR(B_SFULL + buf), (gt >> 1) & 1, abort_flag, p.err, 9);
+        const uint32_t buf = gt % NS;
+        ok &= mbar_wait(BAR(B_SFULL + buf), (gt / NS) & 1, abort_flag, p.err, 9);
         tc_fence_after();
         const uint32_t ts = TM_S0 + buf * TILE_N + lane_addr;
         uint32_t sreg[HC];
@@ -513,7 +534,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
         if (first) m_ref = tmax;
         if (__any_sync(0xFFFFFFFFu, need)) {
           // lazy rescale of this row's accumulator; PV of the previous tile must be done
-          ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 10);
+          ok &= mbar_wait(BAR(B_PVDONE + (gt - 1) % NS), ((gt - 1) / NS) & 1, abort_flag, p.err, 10);
           tc_fence_after();
           const float m_new = fmaxf(m_ref, tmax);
           const float f = (m_ref > -CUDART_INF_F) ? fast_exp2(m_ref - m_new) : 0.f;
@@ -554,7 +575,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
         mbar_arrive(BAR(B_PREADY + buf));
       }
       // ---- end of share: final output or partial ---------------------------
-      ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 11);
+      ok &= mbar_wait(BAR(B_PVDONE + (gt - 1) % NS), ((gt - 1) / NS) & 1, abort_flag, p.err, 11);
       tc_fence_after();
       xsum[half * ROWS + m] = l_sum;
       pair_sync(quarter);
@@ -571,8 +592,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
         if (!whole) {
           const long long W = prefix[p.B];
           const long long NG = W < p.n_groups ? W : p.n_groups;
-          const long long f0 = (long long)prefix[sg.b] + (long long)sg.h * sg.T;
-          d.x = group_of(f0, W, NG);
+          const long long f0 = (long long)prefix[sg.b] + (long long)sg.h * (sg.T + SHARE_COST) + SHARE_COST;
+          d.x = group_of(f0, W, NG);                        // group of the first tile
           d.y = group_of(f0 + sg.T - 1, W, NG) - d.x + 1;
         }
         p.desc[(size_t)item * p.n_mblocks + mb] = d;

@@ -517,7 +517,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  // TMEM columns: S^T buffers at 0 and 128, O^T at 256 (n_pad <= 128 columns each)
+  // TMEM columns: S^T buffers at 0 and 128 (n_pad <= 128 columns each), [O_hi^T | O_lo^T] at 256
+  // (64*NB columns each)
   const uint32_t TM_S0 = tmem, TM_O = tmem + 256;
 
   Partition part;
@@ -632,9 +633,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       // O_lo^T in columns 64..127 (an instruction costs the same at every N here);
       // the epilogue adds the two.  Columns past the padded query rows hold whatever
       // the shared memory held; they only reach output columns nobody reads.
-      const uint32_t idesc_pv = instr_desc_rt(128, 1, 1);     // A = V^T (d contiguous), B = P^T (queries contiguous)
+      const uint32_t idesc_pv = instr_desc_rt(128 * NB, 1, 1);   // A = V^T (d contiguous), B = P^T (queries contiguous)
       // V^T and P^T: 64-wide blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
-      static_assert(S::P_PART == TILE_N * 128, "P_lo must follow P_hi at the block stride");
+      static_assert(S::P_PART == NB * TILE_N * 128, "P_lo must follow the NB blocks of P_hi at the block stride");
       const uint64_t vdesc0 = smem_desc(sm_base + S::V_OFF, TILE_N * 128, 1024);
       const uint64_t pdesc0 = smem_desc(sm_base + S::P_OFF, TILE_N * 128, 1024);
       uint32_t g = 0;
@@ -789,7 +790,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
 #pragma unroll
                 for (int e = 0; e < 8; ++e) lsum[j][e] *= fq[q0 + e];
                 piece_rescale(TM_O + lane_addr + q0, fq + q0);
-                piece_rescale(TM_O + lane_addr + 64 + q0, fq + q0);
+                piece_rescale(TM_O + lane_addr + 64 * NB + q0, fq + q0);
               }
               // scores again, now against the new reference
               uint32_t sr[8];
@@ -848,14 +849,16 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       // ---- end of share: final output or partial ---------------------------
       // Row sums first, while the last O^T product still runs.  Every thread holds
       // its key's share of up to 32 rows; a halving butterfly over the warp leaves
-      // lane r with the sum over the warp's 32 keys for row col0 + r.
-      static_assert(MAXP * 8 == 32, "the butterfly below folds 32 values over 32 lanes");
-      {
+      // lane r with the sum over the warp's 32 keys for row col0 + r
+      // (with two 64-row blocks: two such folds, rows col0 + r and col0 + 32 + r)
+#pragma unroll
+      for (int f0 = 0; f0 < MAXP * 8; f0 += 32) {
         float red[32];
 #pragma unroll
-        for (int j = 0; j < MAXP; ++j)
-#pragma unroll
-          for (int e = 0; e < 8; ++e) red[j * 8 + e] = (j < np) ? lsum[j][e] : 0.f;
+        for (int x = 0; x < 32; ++x) {
+          const int j = (f0 + x) >> 3, e = (f0 + x) & 7;     // piece and element, compile-time after unrolling
+          red[x] = (j < MAXP && j < np) ? lsum[j < MAXP ? j : 0][e] : 0.f;
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
           const bool up = (lane & o) != 0;
@@ -866,7 +869,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
             red[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, o);
           }
         }
-        if (lane < ncol) xq[quarter * S::RS + col0 + lane] = red[0];
+        if (f0 + lane < ncol) xq[quarter * S::RS + col0 + f0 + lane] = red[0];
       }
       soft_sync();
       float* rcp = mref_buf + (mpar ^ 1) * S::RS;            // the idle copy of the references
@@ -918,7 +921,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         uint32_t o[8], o2[8];
         const int q0 = col0 + j * 8;
         tmem_ld8(TM_O + lane_addr + q0, o);
-        tmem_ld8(TM_O + lane_addr + 64 + q0, o2);
+        tmem_ld8(TM_O + lane_addr + 64 * NB + q0, o2);
         tmem_wait_ld();
 #pragma unroll
         for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) + __uint_as_float(o2[e]));
@@ -1107,9 +1110,10 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   const int DH = cfg.head_dim;
   AttnPlanHost pl;
   plan(&cfg, ctx->sm_count, a->k, &pl);
-  // wide query blocks (more than 64 rows per kv head) are better served by the
-  // row-orientation kernel
-  if (((pl.rows_per_mblock * (cfg.n_q_heads / cfg.n_kv_heads) + 15) / 16) * 16 > 64)
+  // Query blocks wider than 64 rows per kv head are better served by the kernel
+  // with the query rows on the M extent (measured), which can also be asked for.
+  if (a->impl == SPACE_ATTN_TENSOR_ROWS ||
+      ((pl.rows_per_mblock * (cfg.n_q_heads / cfg.n_kv_heads) + 15) / 16) * 16 > 64)
     return launch_attn_rows(ctx, a, mask_rows, st);
   AttnParams p;
   memset(&p, 0, sizeof(p));
@@ -1156,6 +1160,8 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   const dim3 mgrid(a->batch * p.H_kv * p.n_mblocks, (m_valid_max * (DH / 4) + 127) / 128);
   {
     ProfScope ps(ctx, SPACE_K_ATTN, st);
+    // (the two-block form NB = 2 of this kernel works but measured slower than the
+    // row-orientation kernel on every wide workload, so it is not instantiated)
     if (DH == 128) launch_main<128, 1>(p, pl.n_ctas, cfg.max_batch, st);
     else launch_main<64, 1>(p, pl.n_ctas, cfg.max_batch, st);
   }

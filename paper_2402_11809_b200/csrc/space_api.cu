@@ -191,7 +191,7 @@ int space_attn_step(space_ctx* ctx, const space_attn_args* a, void* stream) {
   build_layout(a->k, a->mask_variant, &lay);
   cudaStream_t st = (cudaStream_t)stream;
   if (a->impl == SPACE_ATTN_SIMT) return launch_attn_simt(ctx, a, lay.mask, st);
-  if (a->impl != SPACE_ATTN_TENSOR) return SPACE_E_INVALID_ARG;
+  if (a->impl != SPACE_ATTN_TENSOR && a->impl != SPACE_ATTN_TENSOR_ROWS) return SPACE_E_INVALID_ARG;
   return launch_attn_tensor(ctx, a, lay.mask, st);
 }
 

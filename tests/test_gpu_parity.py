@@ -82,7 +82,7 @@ def test_device_philox_matches_oracle(B, H):
 
 
 # ------------------------------------------------------------------ attention
-@pytest.mark.parametrize("impl", ["tensor", "simt"])
+@pytest.mark.parametrize("impl", ["tensor", "rows", "simt"])
 @pytest.mark.parametrize("k,L,d,H_q,H_kv", [
     (1, (0, 0), 64, 2, 2), (2, (1, 1), 128, 2, 2), (3, (127, 127), 128, 2, 1),
     (4, (128, 128), 64, 8, 8), (5, (129, 300), 128, 4, 4), (6, (200, 600), 128, 8, 1),
@@ -93,7 +93,7 @@ def test_attention_small(B, H, impl, k, L, d, H_q, H_kv):
     x = workloads.make_step_inputs(cfg, poison_tail=True)
     ctx = H.make_context(cfg, x)
     ds = H.DeviceStep(cfg, x)
-    ds.attn(ctx, impl=B.ATTN_TENSOR if impl == "tensor" else B.ATTN_SIMT)
+    ds.attn(ctx, impl={"tensor": B.ATTN_TENSOR, "rows": B.ATTN_TENSOR_ROWS, "simt": B.ATTN_SIMT}[impl])
     torch.cuda.synchronize()
     ref, ref_lse = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], k, x["scale"])
     _check_attention(H, ds.out.cpu().numpy().astype(np.float64), ref, f"{impl} k={k} L={L}")
@@ -119,23 +119,26 @@ def test_attention_eq5_literal_variant_and_bf16_output(B, H, k):
     assert np.max(np.abs(got - same)) <= 2.0 ** -8 * np.maximum(np.abs(same), 2.0 ** -126).max()
 
 
-def test_attention_split_invariance_and_determinism(B, H):
+@pytest.mark.parametrize("impl", ["tensor", "rows"])
+def test_attention_split_invariance_and_determinism(B, H, impl):
+    impl = {"tensor": B.ATTN_TENSOR, "rows": B.ATTN_TENSOR_ROWS}[impl]
     # A long single sequence is split over many thread blocks; a batch of short
     # ones is not.  Both must agree with the oracle, and a re-run is bit-identical.
     cfg = _small_cfg(5, (3000, 3000), H_q=1, H_kv=1, Bn=1, seed=7)
     x = workloads.make_step_inputs(cfg)
     ctx = H.make_context(cfg, x)
     ds = H.DeviceStep(cfg, x)
-    ds.attn(ctx)
+    ds.attn(ctx, impl=impl)
     a = ds.out.clone()
     ds.out.fill_(float("nan"))
-    ds.attn(ctx)
+    ds.attn(ctx, impl=impl)
     assert torch.equal(a, ds.out)
     ref, _ = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], 5, x["scale"])
     _check_attention(H, a.cpu().numpy().astype(np.float64), ref, "split")
 
 
-def test_attention_large_scores_rescale_path(B, H):
+@pytest.mark.parametrize("impl", ["tensor", "rows"])
+def test_attention_large_scores_rescale_path(B, H, impl):
     # keys whose scores grow along the sequence force the running maximum to move
     # by far more than the lazy-rescale threshold in later tiles
     cfg = _small_cfg(2, (700, 700), H_q=1, H_kv=1, Bn=1, seed=9)
@@ -147,7 +150,7 @@ def test_attention_large_scores_rescale_path(B, H):
     x["k_cache"] = workloads.f32_to_bf16_bits(kf)
     ctx = H.make_context(cfg, x)
     ds = H.DeviceStep(cfg, x)
-    ds.attn(ctx)
+    ds.attn(ctx, impl={"tensor": B.ATTN_TENSOR, "rows": B.ATTN_TENSOR_ROWS}[impl])
     ref, ref_lse = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], 2, x["scale"])
     assert ref_lse.max() - ref_lse.min() > 20.0
     _check_attention(H, ds.out.cpu().numpy().astype(np.float64), ref, "rescale")
@@ -158,7 +161,7 @@ def test_capacity_overflow_is_flagged_not_computed(B, H):
     x = workloads.make_step_inputs(cfg)
     x["kv_len"][1] = x["s_cap"] - 3                       # L + n_q > capacity
     ctx = H.make_context(cfg, x)
-    for impl in (B.ATTN_TENSOR, B.ATTN_SIMT):
+    for impl in (B.ATTN_TENSOR, B.ATTN_TENSOR_ROWS, B.ATTN_SIMT):
         ds = H.DeviceStep(cfg, x)
         ds.attn(ctx, impl=impl)
         st = ds.status.cpu().numpy()
