@@ -60,14 +60,22 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-// Gumbel noise -log(-log u) for u = (m + 1/2) 2^-23.  Near u = 1 the inner
-// logarithm is taken from its series in d = 1 - u (exact in binary32), elsewhere
-// from the hardware log2; the error of the result stays below 3e-5, inside the
-// 1e-4 band within which two scores count as tied.
-__device__ __forceinline__ float gumbel_from_uniform(float u) {
+// Gumbel noise in units of log 2:  -log2(-log2 u)  for u = (m + 1/2) 2^-23.
+// arg-max_x (z_x/T - log(-log u_x)) = arg-max_x (z_x*log2(e)/T - log2(-log2 u_x)):
+// the two scores differ by the factor log 2 and a constant, so the hardware
+// base-2 logarithm serves without rescaling.  Near u = 1 the inner logarithm is
+// taken from its series in d = 1 - u (exact in binary32); the error of the result
+// stays below 3e-5, inside the 1e-4 band within which two scores count as tied.
+__device__ __forceinline__ float fast_log2(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float gumbel2_from_uniform(float u) {
   const float d = 1.0f - u;
-  const float t = (d < 0.0078125f) ? d * (1.0f + d * (0.5f + d * 0.33333334f)) : -__logf(u);
-  return -__logf(t);
+  const float t = (d < 0.0078125f) ? d * (1.0f + d * (0.5f + d * 0.33333334f)) * 1.4426950408889634f
+                                   : -fast_log2(u);
+  return -fast_log2(t);
 }
 
 struct Stat {                // running statistics of a set of logits
@@ -97,15 +105,16 @@ __device__ __forceinline__ float load_logit(const __nv_bfloat16* p) { return __b
 template <typename T> struct Vec;
 template <> struct Vec<float> {
   static constexpr int N = 4;
-  static __device__ __forceinline__ void load(const float* p, float* v) {
-    const float4 x = __ldg(reinterpret_cast<const float4*>(p));
-    v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+  static constexpr uint32_t NEG_INF = 0xFF800000u;          // raw word that converts to -inf
+  static __device__ __forceinline__ void convert(const uint4& x, float* v) {
+    v[0] = __uint_as_float(x.x); v[1] = __uint_as_float(x.y);
+    v[2] = __uint_as_float(x.z); v[3] = __uint_as_float(x.w);
   }
 };
 template <> struct Vec<__nv_bfloat16> {
   static constexpr int N = 8;
-  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float* v) {
-    const uint4 x = __ldg(reinterpret_cast<const uint4*>(p));
+  static constexpr uint32_t NEG_INF = 0xFF80FF80u;
+  static __device__ __forceinline__ void convert(const uint4& x, float* v) {
     const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -115,78 +124,159 @@ template <> struct Vec<__nv_bfloat16> {
   }
 };
 
-// Fold n consecutive logits starting at vocabulary index x0 into st.
-template <int N, bool GUMBEL>
-__device__ __forceinline__ void fold(Stat& st, const float* v, int x0, float c, float inv_t, int exclude,
-                                     uint32_t key0, uint32_t key1, uint32_t purpose,
-                                     uint32_t seq, uint32_t pos) {
-  float vmax = v[0];
-#pragma unroll
-  for (int i = 1; i < N; ++i) vmax = fmaxf(vmax, v[i]);
-  if (vmax > st.m) {
-    st.s = (st.m > -CUDART_INF_F) ? st.s * fast_exp2((st.m - vmax) * c) : 0.f;
-#pragma unroll
-    for (int i = N - 1; i >= 0; --i) if (v[i] == vmax) st.idx = x0 + i;
-    st.m = vmax;
-  }
-  if (st.m > -CUDART_INF_F) {
-#pragma unroll
-    for (int i = 0; i < N; ++i) st.s += fast_exp2((v[i] - st.m) * c);
+// One logit (the ragged ends of a chunk and unaligned rows).
+template <bool GUMBEL, bool STATS>
+__device__ __forceinline__ void fold_one(Stat& st, float v, int x, float c, int exclude,
+                                         uint32_t key0, uint32_t key1, uint32_t purpose,
+                                         uint32_t seq, uint32_t pos) {
+  if (STATS) {
+    if (v > st.m) {
+      st.s = (st.m > -CUDART_INF_F) ? st.s * fast_exp2((st.m - v) * c) : 0.f;
+      st.idx = x;
+      st.m = v;
+    }
+    if (st.m > -CUDART_INF_F) st.s += fast_exp2(fmaf(v, c, -st.m * c));
   }
   if (GUMBEL) {
     // noise of token x: lane x&3 of the Philox block with counter word x>>2
-#pragma unroll
-    for (int i0 = 0; i0 < N; i0 += 4) {
-      const int xb = x0 + i0;
-      const Philox4 r = philox4x32_10((uint32_t)(xb >> 2), purpose, seq, pos, key0, key1);
-      const uint32_t w[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-      for (int j = 0; j < 4 && i0 + j < N; ++j) {
-        const int lane = (xb + j) & 3;
-        const uint32_t word = (N >= 4) ? w[j] : w[lane];
-        const float u = uniform_open(word);
-        const float sc = v[i0 + j] * inv_t + gumbel_from_uniform(u);
-        const int x = xb + j;
-        if (x != exclude && v[i0 + j] > -CUDART_INF_F && (sc > st.gs)) { st.gs = sc; st.gidx = x; }
-      }
-    }
+    const Philox4 r = philox4x32_10((uint32_t)(x >> 2), purpose, seq, pos, key0, key1);
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+    const float sc = (x == exclude) ? -CUDART_INF_F : fmaf(v, c, gumbel2_from_uniform(uniform_open(w[x & 3])));
+    if (sc > st.gs) { st.gs = sc; st.gidx = x; }
   }
 }
 
-template <typename T, bool VECTOR, bool GUMBEL>
-__device__ Stat scan_chunk(const T* row, int begin, int end, float c, float inv_t, int exclude,
+// (max, lowest arg-max, sum of exp2((z - max) c)) of U vectors of N logits, the
+// first at index x0, the u-th `stride` further: one maximum and one rescale per
+// call, then independent exponentials and tree sums.  -inf entries (slots past the
+// end of the chunk) change neither the maximum nor the sum.
+template <int U, int N>
+__device__ __forceinline__ void fold_stats(Stat& st, const float (&v)[U][N], int x0, int stride, float c) {
+  float vm[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    float a[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) a[i] = v[u][i];
+#pragma unroll
+    for (int w = N / 2; w > 0; w >>= 1)
+#pragma unroll
+      for (int i = 0; i < w; ++i) a[i] = fmaxf(a[i], a[i + w]);
+    vm[u] = a[0];
+  }
+  float vmax = vm[0];
+#pragma unroll
+  for (int u = 1; u < U; ++u) vmax = fmaxf(vmax, vm[u]);
+  if (vmax > st.m) {
+    st.s = (st.m > -CUDART_INF_F) ? st.s * fast_exp2((st.m - vmax) * c) : 0.f;
+    // lowest index that holds the new maximum: walk backwards, the last hit wins
+#pragma unroll
+    for (int u = U - 1; u >= 0; --u) {
+      if (vm[u] == vmax) {
+#pragma unroll
+        for (int i = N - 1; i >= 0; --i) if (v[u][i] == vmax) st.idx = x0 + u * stride + i;
+      }
+    }
+    st.m = vmax;
+  }
+  if (st.m > -CUDART_INF_F) {
+    const float nmc = -st.m * c;                            // exp2(z*c - m*c): exponent error below 1e-5
+    float su[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      float e[N];
+#pragma unroll
+      for (int i = 0; i < N; ++i) e[i] = fast_exp2(fmaf(v[u][i], c, nmc));
+#pragma unroll
+      for (int w = N / 2; w > 0; w >>= 1)
+#pragma unroll
+        for (int i = 0; i < w; ++i) e[i] += e[i + w];
+      su[u] = e[0];
+    }
+    float tot = su[0];
+#pragma unroll
+    for (int u = 1; u < U; ++u) tot += su[u];
+    st.s += tot;
+  }
+}
+
+// Best Gumbel-perturbed score of N logits starting at index x0 (a multiple of 4).
+// A -inf logit (also the excluded token, set to -inf by the caller) never wins.
+template <int N>
+__device__ __forceinline__ void fold_gumbel(Stat& st, const float* v, int x0, float c,
+                                            uint32_t key0, uint32_t key1, uint32_t purpose,
+                                            uint32_t seq, uint32_t pos) {
+#pragma unroll
+  for (int i0 = 0; i0 < N; i0 += 4) {
+    const Philox4 r = philox4x32_10((uint32_t)((x0 + i0) >> 2), purpose, seq, pos, key0, key1);
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+    float sc[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) sc[j] = fmaf(v[i0 + j], c, gumbel2_from_uniform(uniform_open(w[j])));
+    // best of the four (lowest index on ties), then one update of the running best
+    float b01 = sc[0]; int i01 = 0;
+    if (sc[1] > b01) { b01 = sc[1]; i01 = 1; }
+    float b23 = sc[2]; int i23 = 2;
+    if (sc[3] > b23) { b23 = sc[3]; i23 = 3; }
+    if (b23 > b01) { b01 = b23; i01 = i23; }
+    if (b01 > st.gs) { st.gs = b01; st.gidx = x0 + i0 + i01; }
+  }
+}
+
+// Statistics of logits [begin, end) of one row.  STATS: maximum, arg-max and sum;
+// GUMBEL: the best noisy score (token `exclude` left out).  With VECTOR, `begin`
+// is a multiple of the vector length and the row is 16-byte aligned.
+template <typename T, bool VECTOR, bool GUMBEL, bool STATS>
+__device__ Stat scan_chunk(const T* row, int begin, int end, float c, int exclude,
                            uint32_t key0, uint32_t key1, uint32_t purpose, uint32_t seq,
                            uint32_t pos) {
   Stat st = stat_empty();
   if (VECTOR) {
     constexpr int N = Vec<T>::N;
     constexpr int U = 4;                                    // independent 16-byte loads in flight per thread
-    // begin is a multiple of N; the tail shorter than N is handled one by one
+    // the tail shorter than N is handled one by one
     const int full_end = begin + ((end - begin) / N) * N;
     const int stride = blockDim.x * N;
-    // U loads are issued together (predicated at the end of the chunk) so that a
-    // short chunk costs one memory round trip, not one per sweep
-    for (int x = begin + threadIdx.x * N; x < full_end; x += U * stride) {
+    const uint4 ninf = make_uint4(Vec<T>::NEG_INF, Vec<T>::NEG_INF, Vec<T>::NEG_INF, Vec<T>::NEG_INF);
+    // The U loads of the next sweep are issued before the current one is folded,
+    // so a thread always has loads in flight; slots past the end read as -inf.
+    uint4 cur[U], nxt[U];
+    int x = begin + threadIdx.x * N;
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      cur[u] = (x + u * stride < full_end) ? __ldg(reinterpret_cast<const uint4*>(row + x + u * stride)) : ninf;
+    while (x < full_end) {
+      const int xn = x + U * stride;
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        nxt[u] = (xn + u * stride < full_end) ? __ldg(reinterpret_cast<const uint4*>(row + xn + u * stride)) : ninf;
       float v[U][N];
 #pragma unroll
-      for (int u = 0; u < U; ++u)
-        if (x + u * stride < full_end) Vec<T>::load(row + x + u * stride, v[u]);
+      for (int u = 0; u < U; ++u) Vec<T>::convert(cur[u], v[u]);
+      if (STATS) fold_stats<U, N>(st, v, x, stride, c);
+      if (GUMBEL) {
 #pragma unroll
-      for (int u = 0; u < U; ++u)
-        if (x + u * stride < full_end)
-          fold<N, GUMBEL>(st, v[u], x + u * stride, c, inv_t, exclude, key0, key1, purpose, seq, pos);
+        for (int u = 0; u < U; ++u) {
+          const int xu = x + u * stride;
+          if ((unsigned)(exclude - xu) < (unsigned)N) {     // the one token left out of the draw
+#pragma unroll
+            for (int i = 0; i < N; ++i) if (xu + i == exclude) v[u][i] = -CUDART_INF_F;
+          }
+          if (xu < full_end) fold_gumbel<N>(st, v[u], xu, c, key0, key1, purpose, seq, pos);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) cur[u] = nxt[u];
+      x = xn;
     }
-    for (int x = full_end + threadIdx.x; x < end; x += blockDim.x) {
-      float v[1] = {load_logit(row + x)};
+    for (int xt = full_end + threadIdx.x; xt < end; xt += blockDim.x) {
       Stat one = stat_empty();
-      fold<1, GUMBEL>(one, v, x, c, inv_t, exclude, key0, key1, purpose, seq, pos);
+      fold_one<GUMBEL, STATS>(one, load_logit(row + xt), xt, c, exclude, key0, key1, purpose, seq, pos);
       stat_merge(st, one, c);
     }
   } else {
-    for (int x = begin + threadIdx.x; x < end; x += blockDim.x) {
-      float v[1] = {load_logit(row + x)};
-      fold<1, GUMBEL>(st, v, x, c, inv_t, exclude, key0, key1, purpose, seq, pos);
-    }
+    for (int xt = begin + threadIdx.x; xt < end; xt += blockDim.x)
+      fold_one<GUMBEL, STATS>(st, load_logit(row + xt), xt, c, exclude, key0, key1, purpose, seq, pos);
   }
   return st;
 }
@@ -318,7 +408,7 @@ verify_target_kernel(const VerifyParams p) {
   const int k1 = p.k + 1;
   const T* row = reinterpret_cast<const T*>(p.logits) + ((int64_t)b * p.n_q + (int64_t)t * k1) * p.row_stride;
   const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
-  Stat st = scan_chunk<T, VECTOR, false>(row, begin, end, p.c_t, 1.f, -1, 0, 0, 0, 0, 0);
+  Stat st = scan_chunk<T, VECTOR, false, true>(row, begin, end, p.c_t, -1, 0, 0, 0, 0, 0);
   st = block_reduce_plain(st, p.c_t);
   VerifyPartial* part = p.part + ((int64_t)b * (p.k + 2) + t) * p.n_chunks;
   if (threadIdx.x == 0) store_partial(part + ch, st);
@@ -394,13 +484,14 @@ verify_emit_kernel(const VerifyParams p) {
   if (slot == p.k) {
     int exclude = -1;
     if (!literal && i_star < p.k) exclude = p.cand[b * p.k + i_star];   // residual of a point mass
-    st = scan_chunk<T, VECTOR, true>(row, begin, end, c, p.inv_t, exclude, p.key0, p.key1, PURPOSE_TOKEN,
-                                     seq, (uint32_t)(L + i_star + 1));
+    // the extra token needs the noisy arg-max alone: the row's sums are known
+    st = scan_chunk<T, VECTOR, true, false>(row, begin, end, c, exclude, p.key0, p.key1, PURPOSE_TOKEN,
+                                            seq, (uint32_t)(L + i_star + 1));
   } else if (literal) {
-    st = scan_chunk<T, VECTOR, true>(row, begin, end, c, p.inv_t, -1, p.key0, p.key1, PURPOSE_DRAFT, seq,
-                                     (uint32_t)(L + i_star + 1 + slot + 1));
+    st = scan_chunk<T, VECTOR, true, true>(row, begin, end, c, -1, p.key0, p.key1, PURPOSE_DRAFT, seq,
+                                           (uint32_t)(L + i_star + 1 + slot + 1));
   } else {
-    st = scan_chunk<T, VECTOR, false>(row, begin, end, c, 1.f, -1, 0, 0, 0, 0, 0);
+    st = scan_chunk<T, VECTOR, false, true>(row, begin, end, c, -1, 0, 0, 0, 0, 0);
   }
   st = block_reduce(st, c);
   VerifyPartial* part = p.part + ((int64_t)b * (p.k + 2) + slot) * p.n_chunks;
@@ -464,7 +555,7 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   constexpr float C1 = 1.4426950408889634f;                 // T = 1
   const T* row = reinterpret_cast<const T*>(p.logits) + ((int64_t)b * p.n_q + row_i) * p.row_stride;
   const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
-  Stat st = scan_chunk<T, VECTOR, false>(row, begin, end, C1, 1.f, -1, 0, 0, 0, 0, 0);
+  Stat st = scan_chunk<T, VECTOR, false, true>(row, begin, end, C1, -1, 0, 0, 0, 0, 0);
   st = block_reduce_plain(st, C1);
   VerifyPartial* pb = fpart + (int64_t)b * SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS;
   if (threadIdx.x == 0) store_partial(pb + row_i * p.n_chunks + ch, st);
