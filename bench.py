@@ -31,9 +31,10 @@ sys.path.insert(0, ROOT)
 from paper_2402_11809_b200 import replicas, workloads  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum per attn_tc_kernel launch from the ncu capture summarised
-# in profiles/attn_tc_kernel_llama7b.txt (bytes); None for workloads without a capture of the current kernel
-ATTN_TRAFFIC = {"llama7b": 34517760}
+# dram__bytes_read.sum + dram__bytes_write.sum per attention launch from the ncu captures summarised in
+# profiles/attn_tc_kernel_llama7b.txt and profiles/attn_rows_kernel_gqa70b.txt (bytes); None for workloads
+# without a capture of the current kernel
+ATTN_TRAFFIC = {"llama7b": 34517760, "gqa70b": 292199680}
 METRIC = "auto-correct steps/sec"
 UNIT = "steps/s"
 
@@ -41,8 +42,9 @@ UNIT = "steps/s"
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
-        return float(json.load(open(path))["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops", 1590.0)), "measured"
+    return 6650.0, 1590.0, "fallback"
 
 
 # ---------------------------------------------------------------- clock sampler
@@ -321,7 +323,7 @@ def run_ours(args):
         return
 
     # ---- roofline of the dominant kernel (attention) --------------------------
-    peak, peak_src = load_peaks()
+    peak, peak_tf, peak_src = load_peaks()
     attn_ms, attn_n = prof["attn"]
     attn_bytes = np.mean([workloads.algorithmic_bytes(cfg, s["kv_len"])["kv"] +
                           workloads.algorithmic_bytes(cfg, s["kv_len"])["q_out"] for s in sets])
@@ -331,6 +333,20 @@ def run_ours(args):
                                                             steps_dev[i].n_accept.cpu().numpy())["total"]
                                 for i, s in enumerate(sets)]))
     per_kernel_us = {name: (1e3 * v[0] / v[1] if v[1] else None) for name, v in prof.items()}
+    # Which roof binds the attention launch: the three tile products (S, P_hi V, P_lo V) over every
+    # (query row, key) pair against the K, V, Q and output bytes.
+    rows = n_q * (cfg["H_q"] // cfg["H_kv"])
+    attn_flops = float(np.mean([sum(6.0 * rows * cfg["d"] * (int(L) + n_q) * cfg["H_kv"] for L in s_["kv_len"])
+                                for s_ in sets]))
+    tensor_bound = attn_flops / (peak_tf * 1e12) > attn_bytes / (peak * 1e9)
+    if tensor_bound and attn_n:
+        roof = {"bound": "tensor", "achieved": attn_flops / (attn_us * 1e-6) / 1e12, "peak": peak_tf,
+                "unit": "TFLOP/s", "algorithmic_flops_per_launch": attn_flops,
+                "peak_source": peak_src + " (burst bf16 GEMM figure)"}
+    else:
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "peak_source": peak_src + " (burst copy figure)"}
+    roof["frac"] = (roof["achieved"] / roof["peak"]) if roof["achieved"] else None
 
     # ---- CPU oracle on the host cores (bounded: about 10 s) -------------------
     cpu_sps, cpu_reps, cpu_el = time_oracle(cfg, sets[0], budget_s=10.0)
@@ -347,9 +363,8 @@ def run_ours(args):
         "gpu_launches": int(launches_per_step * K),
         "step_algorithmic_bytes": step_bytes,
         "step_hbm_frac": step_bytes / (ms / K * 1e-3) / 1e9 / peak,
-        "roofline": {"bound": "hbm", "kernel": "attn_tc_kernel", "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "traffic": ATTN_TRAFFIC.get(cfg["name"]),
-                     "peak_source": peak_src + " (burst copy figure)",
+        "roofline": {**roof, "kernel": "attn_tc_kernel" if rows <= 64 else "attn_rows_kernel",
+                     "traffic": ATTN_TRAFFIC.get(cfg["name"]),
                      "algorithmic_bytes_per_launch": float(attn_bytes), "avg_launch_us": attn_us,
                      "launches_timed": int(attn_n),
                      "timing": "CUDA events around every launch, stream-launched pass after the graph-timed region",
