@@ -40,6 +40,8 @@ struct AttnParams {
   float* part;                         // [slots][ROWS*(DH+2)]
   int* err;                            // one word: first timeout site
   int2* desc;                          // [B*H_kv*n_mblocks] {first group, number of groups} of each cut
+  int* owner;                          // [grid] (sequence, kv head) whose last piece this thread block computed, or -1
+  int merge_by_owner;                  // the merge grid is indexed by attention thread block, not by (sequence, head)
   uint64_t mask[SPACE_MAX_ROWS];
 };
 
@@ -491,6 +493,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
     // same control flow so that the pair barriers below always match up; once
     // the abort flag is set all later waits return at once and the block drains.
     bool ok = true;
+    int own = -1;                                          // item whose last piece of a cut this block holds
     while (part.next(sg)) {
       const int n_keys = sg.L + p.n_q;
       float m_ref = -CUDART_INF_F, l_sum = 0.f;
@@ -597,6 +600,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
           d.y = group_of(f0 + sg.T - 1, W, NG) - d.x + 1;
         }
         p.desc[(size_t)item * p.n_mblocks + mb] = d;
+        if (sg.t0 > 0 && sg.t1 == sg.T) own = item;        // at most one per block: only its first share can start late
       }
 #pragma unroll 1
       for (int cc = 0; cc < OC / 32; ++cc) {
@@ -646,6 +650,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
         }
       }
     }
+    if (sidx == 0) p.owner[blockIdx.x] = own;
   }
 
   // ---- teardown -----------------------------------------------------------
@@ -669,11 +674,18 @@ __global__ void __launch_bounds__(128) attn_rows_merge_kernel(const AttnParams p
   pdl_launch_dependents();
   pdl_wait();
   constexpr int C4 = DH / 4;
-  const int item = blockIdx.x / p.n_mblocks, mb = blockIdx.x % p.n_mblocks;
+  // Large batches: one grid column per attention thread block (each holds the last
+  // piece of at most one cut); small ones: one per (sequence, head, row block).
+  int item = blockIdx.x / p.n_mblocks;
+  const int mb = blockIdx.x % p.n_mblocks;
+  if (p.merge_by_owner) {
+    item = p.owner[blockIdx.x];
+    if (item < 0) return;
+  }
   const int b = item / p.H_kv, h = item % p.H_kv;
   const int L = p.kv_len[b];
   if (L < 0 || (int64_t)L + p.n_q > p.s_cap) return;
-  const int2 d = p.desc[blockIdx.x];
+  const int2 d = p.desc[(size_t)item * p.n_mblocks + mb];
   const int n = d.y;
   if (n <= 1) return;                                       // written directly by the main kernel
   const int i0 = mb * p.rows_per_mb;
@@ -780,6 +792,8 @@ int launch_attn_rows(space_ctx* ctx, const space_attn_args* a, const uint64_t* m
   p.kv_len = a->kv_len; p.out = a->out; p.lse = a->lse; p.status = a->status;
   p.part = ctx->attn_part; p.err = ctx->counters + 3 * cfg.max_batch;
   p.desc = reinterpret_cast<int2*>(ctx->merge_cnt);
+  p.owner = ctx->merge_cnt + (size_t)cfg.max_batch * cfg.n_kv_heads * 8 * 2;
+  p.merge_by_owner = (a->batch * p.H_kv * p.n_mblocks > pl.n_ctas) ? 1 : 0;
   for (int i = 0; i < SPACE_MAX_ROWS; ++i) p.mask[i] = mask_rows[i];
 
   // TMA descriptors, rebuilt only when a base pointer or a stride changes
@@ -805,7 +819,7 @@ int launch_attn_rows(space_ctx* ctx, const space_attn_args* a, const uint64_t* m
   memcpy(&p.tm_v, ctx->tm_v, sizeof(CUtensorMap));
 
   const int m_valid_max = p.rows_per_mb * p.G;
-  const dim3 mgrid(a->batch * p.H_kv * p.n_mblocks, (m_valid_max * (DH / 4) + 127) / 128);
+  const dim3 mgrid(p.merge_by_owner ? pl.n_ctas : a->batch * p.H_kv * p.n_mblocks, (m_valid_max * (DH / 4) + 127) / 128);
   if (DH == 128) {
     const size_t sm = smem_bytes<128>(cfg.max_batch);
     cudaFuncSetAttribute(attn_rows_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);

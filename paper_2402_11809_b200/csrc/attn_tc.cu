@@ -55,6 +55,8 @@ struct AttnParams {
   float* part;                         // [slots][ROWS*(DH+2)]
   int* err;                            // one word: first timeout site
   int2* desc;                          // [B*H_kv*n_mblocks] {first partial slot, number of partials} of each cut
+  int* owner;                          // [grid] (sequence, kv head) whose last piece this thread block computed, or -1
+  int merge_by_owner;                  // the merge grid is indexed by attention thread block, not by (sequence, head)
   uint64_t mask[SPACE_MAX_ROWS];       // bit j of mask[i]: block row i sees block key j
   uint64_t mask_t[SPACE_MAX_ROWS];     // transposed: bit i of mask_t[j]
 };
@@ -688,6 +690,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     // same control flow so that the block-wide barriers below always match up;
     // once the abort flag is set all later waits return at once and the block drains.
     bool ok = true;
+    int own = -1;                                          // item whose last piece of a cut this block holds
     while (part.next(sg)) {
       const int n_keys = sg.L + p.n_q;
 #pragma unroll
@@ -900,6 +903,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           d.y = group_of(f0 + SHARE_COST + sg.T - 1, W, NG) - g0 + 1;
         }
         p.desc[(size_t)item * p.n_mblocks + mb] = d;
+        if (sg.t0 > 0 && sg.t1 == sg.T) own = item;        // at most one per block: only its first share can start late
       }
       if (sidx < m_valid && ok) {                           // per-row scalars
         const int q = sidx;
@@ -952,6 +956,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       tc_fence_before();
       soft_sync();                                          // scratch, fq and mref are reused by the next share
     }
+    if (sidx == 0) p.owner[blockIdx.x] = own;
   }
 
   // ---- teardown -----------------------------------------------------------
@@ -975,11 +980,18 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(const AttnParams p) {
   pdl_launch_dependents();
   pdl_wait();
   constexpr int C4 = DH / 4;
-  const int item = blockIdx.x / p.n_mblocks, mb = blockIdx.x % p.n_mblocks;
+  // Large batches: one grid column per attention thread block (each holds the last
+  // piece of at most one cut); small ones: one per (sequence, head, row block).
+  int item = blockIdx.x / p.n_mblocks;
+  const int mb = blockIdx.x % p.n_mblocks;
+  if (p.merge_by_owner) {
+    item = p.owner[blockIdx.x];
+    if (item < 0) return;
+  }
   const int b = item / p.H_kv, h = item % p.H_kv;
   const int L = p.kv_len[b];
   if (L < 0 || (int64_t)L + p.n_q > p.s_cap) return;
-  const int2 d = p.desc[blockIdx.x];
+  const int2 d = p.desc[(size_t)item * p.n_mblocks + mb];
   const int n = d.y;
   if (n <= 1) return;                                       // written directly by the main kernel
   const int i0 = mb * p.rows_per_mb;
@@ -1127,6 +1139,8 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   p.kv_len = a->kv_len; p.out = a->out; p.lse = a->lse; p.status = a->status;
   p.part = ctx->attn_part; p.err = ctx->counters + 3 * cfg.max_batch;
   p.desc = reinterpret_cast<int2*>(ctx->merge_cnt);
+  p.owner = ctx->merge_cnt + (size_t)cfg.max_batch * cfg.n_kv_heads * 8 * 2;
+  p.merge_by_owner = (a->batch * p.H_kv * p.n_mblocks > pl.n_ctas) ? 1 : 0;
   for (int i = 0; i < SPACE_MAX_ROWS; ++i) p.mask[i] = mask_rows[i];
   for (int j = 0; j < SPACE_MAX_ROWS; ++j) {
     uint64_t t = 0;
@@ -1157,7 +1171,7 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   memcpy(&p.tm_v, ctx->tm_v, sizeof(CUtensorMap));
 
   const int m_valid_max = p.rows_per_mb * p.G;
-  const dim3 mgrid(a->batch * p.H_kv * p.n_mblocks, (m_valid_max * (DH / 4) + 127) / 128);
+  const dim3 mgrid(p.merge_by_owner ? pl.n_ctas : a->batch * p.H_kv * p.n_mblocks, (m_valid_max * (DH / 4) + 127) / 128);
   {
     ProfScope ps(ctx, SPACE_K_ATTN, st);
     // (the two-block form NB = 2 of this kernel works but measured slower than the

@@ -40,7 +40,8 @@ Carve carve(const space_config* c, int sm_count) {
   off += align_up(attn_tensor_partial_floats(c, sm_count, &v.part_slots) * sizeof(float), 256);
   v.counters = off; off += align_up((size_t)(3 * c->max_batch + 4) * sizeof(int), 256);
   v.merge_cnt = off;
-  off += align_up((size_t)c->max_batch * c->n_kv_heads * 8 * sizeof(int2), 256);   // up to 8 row blocks, one {first, count} pair each
+  // up to 8 row blocks, one {first, count} pair each; then one word per thread block of the attention grid
+  off += align_up((size_t)c->max_batch * c->n_kv_heads * 8 * sizeof(int2) + (size_t)(sm_count + 8) * sizeof(int), 256);
   v.vpart = off;
   off += align_up((size_t)c->max_batch * (c->k_max + 2) * SPACE_VERIFY_MAX_CHUNKS * sizeof(VerifyPartial), 256);
   v.vfused = off; off += align_up((size_t)c->max_batch * SPACE_MAX_ROWS * 16 * sizeof(VerifyPartial), 256);

@@ -87,6 +87,9 @@ def test_device_philox_matches_oracle(B, H):
     (1, (0, 0), 64, 2, 2), (2, (1, 1), 128, 2, 2), (3, (127, 127), 128, 2, 1),
     (4, (128, 128), 64, 8, 8), (5, (129, 300), 128, 4, 4), (6, (200, 600), 128, 8, 1),
     (7, (5, 900), 128, 4, 2), (5, (1000, 1400), 64, 16, 1), (2, (250, 260), 128, 16, 1),
+    # more (sequence, head) pairs than thread blocks, one or two tiles each: the even cut per pair
+    # does not fit and the flat cut takes over; the merge grid goes by thread block
+    (2, (10, 200), 64, 64, 64),
 ])
 def test_attention_small(B, H, impl, k, L, d, H_q, H_kv):
     cfg = _small_cfg(k, L, d=d, H_q=H_q, H_kv=H_kv, Bn=3, seed=k)
