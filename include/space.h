@@ -167,6 +167,12 @@ typedef struct {
   int32_t*  status;            /* host [B]                                     */
   int64_t*  h2d_bytes;         /* host, optional: bytes copied to the device   */
   int64_t*  d2h_bytes;         /* host, optional: bytes copied back            */
+  int32_t   cache_resident;    /* 0: upload rows 0 .. kv_len+n_q-1 of every sequence's K and V.
+                                  1: the KV cache is the decoder's state and already sits in the context's
+                                  staging copy from an earlier call (rows 0 .. kv_len-1 of every sequence,
+                                  as that call's commit left them); only the block's own rows
+                                  kv_len .. kv_len+n_q-1 are uploaded                               */
+  int32_t   reserved;          /* 0                                                              */
 } space_host_step_args;
 
 /* Create a context on cfg->device: validates the shape, reserves the
@@ -219,7 +225,8 @@ int space_verify_greedy_noalloc(const space_verify_args* args, void* stream);
 int space_kv_commit(space_ctx* ctx, const space_commit_args* args, void* stream);
 
 /* The three stages from host buffers; synchronises `stream` before returning.
- * Needs cfg.host_staging.  Only sequence prefixes in use are copied. */
+ * Needs cfg.host_staging.  Only sequence prefixes in use are copied (with
+ * cache_resident: only the block's rows, see the field). */
 int space_step_host(space_ctx* ctx, const space_host_step_args* args, void* stream);
 
 /* Number of kernels this context has launched so far. */

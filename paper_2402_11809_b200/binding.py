@@ -87,7 +87,8 @@ class HostStepArgs(C.Structure):
                 ("kv_len", C.c_void_p), ("out", C.c_void_p), ("n_accept", C.c_void_p),
                 ("out_tokens", C.c_void_p), ("n_out", C.c_void_p), ("next_cand", C.c_void_p),
                 ("next_cand_prob", C.c_void_p), ("finished", C.c_void_p), ("status", C.c_void_p),
-                ("h2d_bytes", C.c_void_p), ("d2h_bytes", C.c_void_p)]
+                ("h2d_bytes", C.c_void_p), ("d2h_bytes", C.c_void_p),
+                ("cache_resident", C.c_int32), ("reserved", C.c_int32)]
 
 
 lib.space_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(Config)]

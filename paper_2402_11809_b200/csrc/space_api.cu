@@ -298,11 +298,13 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* a, void* stream)
   for (int b = 0; b < B && ok; ++b) {
     const int64_t L = a->kv_len[b];
     if (L < 0 || L + n_q > c.s_cap) continue;            // flagged by the kernels
-    const size_t w = (size_t)(L + n_q) * row_b;
-    ok = ok && cudaMemcpy2DAsync(d_k + b * seq_b, head_pitch, (const char*)a->k_cache + b * seq_b, head_pitch,
-                                 w, c.n_kv_heads, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpy2DAsync(d_v + b * seq_b, head_pitch, (const char*)a->v_cache + b * seq_b, head_pitch,
-                                 w, c.n_kv_heads, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    // everything in use, or (cache kept from an earlier call) the block's own rows only
+    const size_t first = a->cache_resident ? (size_t)L * row_b : 0;
+    const size_t w = (size_t)(L + n_q) * row_b - first;
+    ok = ok && cudaMemcpy2DAsync(d_k + b * seq_b + first, head_pitch, (const char*)a->k_cache + b * seq_b + first,
+                                 head_pitch, w, c.n_kv_heads, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpy2DAsync(d_v + b * seq_b + first, head_pitch, (const char*)a->v_cache + b * seq_b + first,
+                                 head_pitch, w, c.n_kv_heads, cudaMemcpyHostToDevice, st) == cudaSuccess;
     h2d += 2 * (int64_t)w * c.n_kv_heads;
   }
   ok = ok && cudaMemsetAsync(d_status, 0, (size_t)B * 4, st) == cudaSuccess;
