@@ -64,6 +64,7 @@ struct space_ctx {
   int32_t* scratch_status; // [max_batch] used when the caller passes no status array
   // staging for space_step_host
   char* stage;
+  char* host_small;        // pinned host mirror of the staging area's small per-sequence arrays (host_staging only)
   size_t stage_bytes;
   // per-kernel event timing (space_profile_*)
   int prof_on;

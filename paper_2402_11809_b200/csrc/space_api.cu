@@ -144,8 +144,17 @@ int space_create(space_ctx** out, const space_config* cfg) {
   ctx->scratch_status = (int32_t*)(ctx->ws + cv.status);
   ctx->stage = cfg->host_staging ? ctx->ws + cv.stage : nullptr;
   ctx->stage_bytes = cv.total - cv.stage;
+  ctx->host_small = nullptr;
+  if (cfg->host_staging &&
+      cudaHostAlloc((void**)&ctx->host_small, (size_t)cfg->max_batch * 64 * 11, cudaHostAllocDefault) != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(ctx->ws);
+    delete ctx;
+    return SPACE_E_CUDA;
+  }
   // counters and status start at zero; the kernels restore them after use
   if (cudaMemset(ctx->ws + cv.counters, 0, cv.stage - cv.counters) != cudaSuccess) {
+    if (ctx->host_small) cudaFreeHost(ctx->host_small);
     cudaFree(ctx->ws);
     delete ctx;
     return SPACE_E_CUDA;
@@ -162,6 +171,7 @@ void space_destroy(space_ctx* ctx) {
     for (int i = 0; i < 2 * SPACE_PROFILE_MAX_STEPS; ++i) cudaEventDestroy(ctx->prof_ev[w][i]);
     free(ctx->prof_ev[w]);
   }
+  if (ctx->host_small) cudaFreeHost(ctx->host_small);
   cudaFree(ctx->ws);
   delete ctx;
 }
@@ -292,9 +302,13 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* a, void* stream)
   const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;
   ok = ok && up(d_q, a->q, (size_t)B * n_q * c.n_q_heads * d * 2);
   ok = ok && up(d_logits, a->logits, (size_t)B * n_q * a->vocab * esz);
-  ok = ok && up(d_kvlen, a->kv_len, (size_t)B * 4);
-  ok = ok && up(d_cand, a->cand, (size_t)B * k * 4);
-  ok = ok && up(d_cprob, a->cand_prob, (size_t)B * k * 4);
+  // the small per-sequence arrays travel as one block each way through a pinned mirror of their slots
+  char* hsm = ctx->host_small;
+  memcpy(hsm, a->kv_len, (size_t)B * 4);
+  memcpy(hsm + slot, a->cand, (size_t)B * k * 4);
+  memcpy(hsm + 2 * slot, a->cand_prob, (size_t)B * k * 4);
+  ok = ok && cudaMemcpyAsync(d_small, hsm, 3 * slot, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  h2d += (int64_t)B * 4 * (1 + 2 * k);
   for (int b = 0; b < B && ok; ++b) {
     const int64_t L = a->kv_len[b];
     if (L < 0 || L + n_q > c.s_cap) continue;            // flagged by the kernels
@@ -334,13 +348,8 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* a, void* stream)
   if (rc != SPACE_OK) return rc;
 
   ok = ok && down(a->out, d_out, (size_t)B * n_q * c.n_q_heads * d * 4);
-  ok = ok && down(a->n_accept, d_nacc, (size_t)B * 4);
-  ok = ok && down(a->out_tokens, d_tok, (size_t)B * k1 * 4);
-  ok = ok && down(a->n_out, d_nout, (size_t)B * 4);
-  ok = ok && down(a->next_cand, d_ncand, (size_t)B * k * 4);
-  ok = ok && down(a->next_cand_prob, d_nprob, (size_t)B * k * 4);
-  ok = ok && down(a->finished, d_fin, (size_t)B);
-  ok = ok && down(a->status, d_status, (size_t)B * 4);
+  ok = ok && cudaMemcpyAsync(hsm + 3 * slot, d_small + 3 * slot, 8 * slot, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  d2h += (int64_t)B * (4 + k1 * 4 + 4 + k * 4 + k * 4 + 1 + 4 + 4);
   for (int b = 0; b < B && ok; ++b) {                    // rows L .. L+k: the compacted rows
     const int64_t L = a->kv_len[b];
     if (L < 0 || L + n_q > c.s_cap) continue;
@@ -351,9 +360,16 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* a, void* stream)
                                  cudaMemcpyDeviceToHost, st) == cudaSuccess;
     d2h += 2 * (int64_t)w * c.n_kv_heads;
   }
-  ok = ok && down(a->kv_len, d_kvlen_out, (size_t)B * 4);
   if (!ok) { cudaGetLastError(); return SPACE_E_CUDA; }
   if (cudaStreamSynchronize(st) != cudaSuccess) return SPACE_E_CUDA;
+  memcpy(a->n_accept, hsm + 3 * slot, (size_t)B * 4);
+  memcpy(a->out_tokens, hsm + 4 * slot, (size_t)B * k1 * 4);
+  memcpy(a->n_out, hsm + 5 * slot, (size_t)B * 4);
+  memcpy(a->next_cand, hsm + 6 * slot, (size_t)B * k * 4);
+  memcpy(a->next_cand_prob, hsm + 7 * slot, (size_t)B * k * 4);
+  memcpy(a->finished, hsm + 8 * slot, (size_t)B);
+  memcpy(a->status, hsm + 9 * slot, (size_t)B * 4);
+  memcpy(a->kv_len, hsm + 10 * slot, (size_t)B * 4);
   if (a->h2d_bytes) *a->h2d_bytes = h2d;
   if (a->d2h_bytes) *a->d2h_bytes = d2h;
   return SPACE_OK;
