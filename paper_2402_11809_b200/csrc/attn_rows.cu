@@ -511,18 +511,33 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
         const bool masked = (kt + TILE_N > sg.L) || (kt < lo);
         float tmax = -CUDART_INF_F;
         if (masked) {
+          // Visibility of this thread's 64 keys as one 64-bit word (bit c: key k0 + c):
+          // keys before `lo` belong to the previous tile; cached keys (< L) are seen by
+          // every row; block keys by the Eq. 5 mask row of this query row.
+          const int k0 = kt + half * HC;
+          const int sh = sg.L - k0;                         // first block key sits at bit `sh`
+          uint64_t vis;
+          if (sh >= 64) vis = ~0ull;
+          else if (sh > 0) vis = ((1ull << sh) - 1ull) | (mrow << sh);
+          else if (sh > -64) vis = mrow >> (-sh);
+          else vis = 0ull;
+          const int below = lo - k0;                        // keys k0 .. lo-1 are not this tile's
+          if (below >= 64) vis = 0ull;
+          else if (below > 0) vis &= ~0ull << below;
+          const uint32_t v0 = (uint32_t)vis, v1 = (uint32_t)(vis >> 32);
 #pragma unroll
           for (int cidx = 0; cidx < HC; ++cidx) {
-            const int key = kt + half * HC + cidx;
-            bool vis = key >= lo;
-            if (key >= sg.L) vis = vis && ((mrow >> ((key - sg.L) & 63)) & 1ull);
-            const float v = vis ? __uint_as_float(sreg[cidx]) : -CUDART_INF_F;
+            const uint32_t w = cidx < 32 ? v0 : v1;
+            const float v = ((w >> (cidx & 31)) & 1u) ? __uint_as_float(sreg[cidx]) : -CUDART_INF_F;
             sreg[cidx] = __float_as_uint(v);
-            tmax = fmaxf(tmax, v);
           }
-        } else {
+        }
+        {
+          // four independent running maxima: one chain over 64 values would cost 64 dependent steps
+          float t4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-          for (int cidx = 0; cidx < HC; ++cidx) tmax = fmaxf(tmax, __uint_as_float(sreg[cidx]));
+          for (int cidx = 0; cidx < HC; ++cidx) t4[cidx & 3] = fmaxf(t4[cidx & 3], __uint_as_float(sreg[cidx]));
+          tmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
         }
         // the row maximum needs the other half's keys; the pair barrier also orders
         // both threads' reads of S before either overwrites it with P
