@@ -236,7 +236,7 @@ struct Smem {
   static constexpr int TILE_BYTES = TILE_N * DH * 2;         // one K or V tile
   static constexpr int Q_BYTES = ROWS * DH * 2;
   static constexpr int K_STAGES = (DH == 128) ? 2 : 3;
-  static constexpr int V_STAGES = (DH == 128) ? 3 : 4;
+  static constexpr int V_STAGES = (DH == 128) ? 2 : 4;
   static constexpr int Q_OFF = 0;
   static constexpr int K_OFF = Q_BYTES;
   static constexpr int V_OFF = K_OFF + K_STAGES * TILE_BYTES;
@@ -247,7 +247,9 @@ struct Smem {
   static constexpr int MISC_OFF = BAR_OFF + (N_BARS * 8 + 15) / 16 * 16;   // tmem base, abort flag
   static constexpr int XMAX_OFF = MISC_OFF + 32;             // [2 parities][2 halves][ROWS] float
   static constexpr int XSUM_OFF = XMAX_OFF + 2 * 2 * ROWS * 4;   // [2 halves][ROWS] float
-  static constexpr int TABLE_OFF = XSUM_OFF + 2 * ROWS * 4;  // seq_len[max_batch], prefix[max_batch+1]
+  static constexpr int EPI_PITCH = 36;                       // floats per staged row: 32 columns + 4 (16-byte aligned, conflict-free)
+  static constexpr int EPI_OFF = XSUM_OFF + 2 * ROWS * 4;    // [8 warps][32 rows][EPI_PITCH] float: epilogue transpose
+  static constexpr int TABLE_OFF = EPI_OFF + 8 * 32 * EPI_PITCH * 4;   // seq_len[max_batch], prefix[max_batch+1]
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -617,42 +619,45 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
         p.desc[(size_t)item * p.n_mblocks + mb] = d;
         if (sg.t0 > 0 && sg.t1 == sg.T) own = item;        // at most one per block: only its first share can start late
       }
+      // O leaves TMEM with one row per lane; written like that, a store instruction
+      // would touch 32 different lines.  Each warp turns its 32 x 32 block through
+      // shared memory so that eight lanes write 128 contiguous bytes of one row.
+      float* stg = reinterpret_cast<float*>(sm + S::EPI_OFF) + (warp - WARP_SOFTMAX0) * (32 * S::EPI_PITCH);
+      const int gsh = __ffs(p.G) - 1;                       // G is a power of two
+      const float scale_o = whole ? inv : 1.f;
 #pragma unroll 1
       for (int cc = 0; cc < OC / 32; ++cc) {
         uint32_t o[32];
         const int col = half * OC + cc * 32;
         tmem_ld32(TM_O + lane_addr + col, o);
         tmem_wait_ld();
-        if (!row_valid || !ok) continue;
-        if (whole) {
-          const size_t off = (((size_t)sg.b * p.n_q + i) * p.H_q + hq) * DH + col;
-          if (p.out_dtype == SPACE_DTYPE_F32) {
-            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off);
 #pragma unroll
-            for (int x = 0; x < 8; ++x)
-              dst[x] = make_float4(__uint_as_float(o[4 * x]) * inv, __uint_as_float(o[4 * x + 1]) * inv,
-                                   __uint_as_float(o[4 * x + 2]) * inv, __uint_as_float(o[4 * x + 3]) * inv);
-          } else {
-            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off);
+        for (int x = 0; x < 8; ++x)
+          *reinterpret_cast<float4*>(stg + lane * S::EPI_PITCH + 4 * x) =
+              make_float4(__uint_as_float(o[4 * x]) * scale_o, __uint_as_float(o[4 * x + 1]) * scale_o,
+                          __uint_as_float(o[4 * x + 2]) * scale_o, __uint_as_float(o[4 * x + 3]) * scale_o);
+        __syncwarp();
 #pragma unroll
-            for (int x = 0; x < 4; ++x) {
-              uint32_t w[4];
-#pragma unroll
-              for (int y = 0; y < 4; ++y) {
-                const __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(o[8 * x + 2 * y]) * inv,
-                                                                __uint_as_float(o[8 * x + 2 * y + 1]) * inv);
-                w[y] = *reinterpret_cast<const uint32_t*>(&pk);
-              }
-              dst[x] = make_uint4(w[0], w[1], w[2], w[3]);
+        for (int it = 0; it < 8; ++it) {
+          const int rl = it * 4 + (lane >> 3), c4 = (lane & 7) * 4;   // row within the warp's block, first of 4 columns
+          const int mr = quarter * 32 + rl;
+          const float4 v = *reinterpret_cast<const float4*>(stg + rl * S::EPI_PITCH + c4);
+          if (mr >= m_valid || !ok) continue;
+          if (whole) {
+            const int ir = i0 + (mr >> gsh), hr = sg.h * p.G + (mr & (p.G - 1));
+            const size_t off = (((size_t)sg.b * p.n_q + ir) * p.H_q + hr) * DH + col + c4;
+            if (p.out_dtype == SPACE_DTYPE_F32) {
+              *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off) = v;
+            } else {
+              const __nv_bfloat162 a0 = __floats2bfloat162_rn(v.x, v.y), a1 = __floats2bfloat162_rn(v.z, v.w);
+              *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off) =
+                  make_uint2(*reinterpret_cast<const uint32_t*>(&a0), *reinterpret_cast<const uint32_t*>(&a1));
             }
+          } else {
+            *reinterpret_cast<float4*>(pslot + (size_t)mr * DH + col + c4) = v;
           }
-        } else {
-          float4* dst = reinterpret_cast<float4*>(pslot + (size_t)m * DH + col);
-#pragma unroll
-          for (int x = 0; x < 8; ++x)
-            dst[x] = make_float4(__uint_as_float(o[4 * x]), __uint_as_float(o[4 * x + 1]),
-                                 __uint_as_float(o[4 * x + 2]), __uint_as_float(o[4 * x + 3]));
         }
+        __syncwarp();                                       // the block is rewritten by the next chunk
       }
       tc_fence_before();
       if (row_valid && half == 0 && ok) {
