@@ -920,6 +920,11 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       // O^T: lane = head-dim index, column = query row.  A warp writes 32
       // consecutive floats of one output row per store.
       const bool d_ok = kl < DH && ok;                      // lanes 64..127 repeat 0..63 when head_dim is 64
+      const int gsh = __ffs(p.G) - 1;
+      const bool out_f32 = p.out_dtype == SPACE_DTYPE_F32;
+      // element (block row i0, head h*G, dim kl) of this sequence; one block row further = H_q*DH
+      const size_t out_base = (((size_t)sg.b * p.n_q + i0) * p.H_q + (size_t)sg.h * p.G) * DH + kl;
+      const size_t out_row = (size_t)p.H_q * DH;
 #pragma unroll 2
       for (int j = 0; j < np; ++j) {
         uint32_t o[8], o2[8];
@@ -930,21 +935,24 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
 #pragma unroll
         for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) + __uint_as_float(o2[e]));
         if (whole) {
-          // consecutive query rows are consecutive heads of one block row, then the next block row
-          int g = q0 % p.G;
-          size_t off = (((size_t)sg.b * p.n_q + (i0 + q0 / p.G)) * p.H_q + sg.h * p.G + g) * DH + kl;
-          const size_t row_jump = (size_t)(p.H_q - p.G) * DH;
+          // query row q of the block is head q mod G of block row q / G (G is a power of two)
           const float4 r0 = reinterpret_cast<const float4*>(rcp + q0)[0], r1 = reinterpret_cast<const float4*>(rcp + q0)[1];
           const float rr[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+          size_t off[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
-            if (q0 + e < m_valid && d_ok) {
-              const float r = __uint_as_float(o[e]) * rr[e];
-              if (p.out_dtype == SPACE_DTYPE_F32) reinterpret_cast<float*>(p.out)[off] = r;
-              else reinterpret_cast<__nv_bfloat16*>(p.out)[off] = __float2bfloat16_rn(r);
-            }
-            off += DH;
-            if (++g == p.G) { g = 0; off += row_jump; }
+            const int q = q0 + e;
+            off[e] = out_base + (size_t)(q >> gsh) * out_row + (size_t)(q & (p.G - 1)) * DH;
+          }
+          if (out_f32) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              if (q0 + e < m_valid && d_ok) reinterpret_cast<float*>(p.out)[off[e]] = __uint_as_float(o[e]) * rr[e];
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              if (q0 + e < m_valid && d_ok)
+                reinterpret_cast<__nv_bfloat16*>(p.out)[off[e]] = __float2bfloat16_rn(__uint_as_float(o[e]) * rr[e]);
           }
         } else {
           float* dst = pslot + (size_t)q0 * DH + kl;
