@@ -446,8 +446,40 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_v) : "memory");
   if (warp == WARP_MMA && lane == 0)
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_q) : "memory");
+  // barriers and the TMEM allocation are visible to every warp before the first
+  // global access (with a programmatic launch this part runs under the previous kernel)
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
   pdl_wait();                                              // global memory from here on
-  if (warp == WARP_SOFTMAX0) {
+  const bool single = p.B == 1;
+  if (single) {
+    // One sequence (the usual decoding case): the tables have a closed form, so every
+    // thread works them out for itself from the one length (identical values, each
+    // thread reads back what it wrote) and no warp has to hand them over.
+    const int L0 = p.kv_len[0];
+    const bool okL = L0 >= 0 && (int64_t)L0 + p.n_q <= p.s_cap;
+    if (!okL && blockIdx.x == 0 && threadIdx.x == 0 && p.status) atomicOr(p.status, SPACE_ST_CAPACITY);
+    const int L = okL ? L0 : -1;
+    const int T = okL ? (L + p.n_q + TILE_N - 1) / TILE_N : 0;
+    seq_len[0] = L; prefix[0] = 0; prefix[1] = okL ? (T + SHARE_COST) * p.H_kv : 0;
+    int ag = -1;
+    const int W = T * p.H_kv;
+    if (W > 0 && W < 8 * p.n_groups) {
+      const int a = max(1, min(p.n_groups / p.H_kv, T));   // = floor(groups * T / W)
+      if (a * p.H_kv <= p.n_groups) {
+        ag = a * p.H_kv;
+        if (group < ag) {
+          const int h = group / a, piece = group - h * a;
+          const int q = T / a, r = T - q * a;
+          const int t0 = piece * q + min(piece, r);
+          reinterpret_cast<int4*>(seg0)[0] = make_int4(0, h, t0, t0 + q + (piece < r ? 1 : 0));
+          reinterpret_cast<int4*>(seg0)[1] = make_int4(T, L, h * a, a);
+        }
+      }
+    }
+    *agroups = ag;
+  } else if (warp == WARP_SOFTMAX0) {
     // per-sequence tile counts and their running sum, 32 sequences per round
     int carry = 0, nvalid = 0;
     for (int b0 = 0; b0 < p.B; b0 += 32) {
@@ -515,9 +547,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       *agroups = acarry;
     }
   }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
+  if (!single) __syncthreads();                            // the tables of warp 4 reach every warp
   const uint32_t tmem = *tmem_slot;
   // TMEM columns: S^T buffers at 0 and 128 (n_pad <= 128 columns each), [O_hi^T | O_lo^T] at 256
   // (64*NB columns each)
