@@ -34,7 +34,7 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per attention launch from the ncu captures summarised in
 # profiles/attn_tc_kernel_llama7b.txt and profiles/attn_rows_kernel_gqa70b.txt (bytes); None for workloads
 # without a capture of the current kernel
-ATTN_TRAFFIC = {"llama7b": 34517760, "gqa70b": 292199680}
+ATTN_TRAFFIC = {"llama7b": 34518272, "gqa70b": 293366272}
 METRIC = "auto-correct steps/sec"
 UNIT = "steps/s"
 
