@@ -1027,9 +1027,10 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(const AttnParams p) {
     if (item < 0) return;
   }
   const int b = item / p.H_kv, h = item % p.H_kv;
-  const int L = p.kv_len[b];
+  // both loads are issued before either is tested: one round trip, not two
+  const int L = __ldcg(p.kv_len + b);
+  const int2 d = __ldcg(p.desc + (size_t)item * p.n_mblocks + mb);
   if (L < 0 || (int64_t)L + p.n_q > p.s_cap) return;
-  const int2 d = p.desc[(size_t)item * p.n_mblocks + mb];
   const int n = d.y;
   if (n <= 1) return;                                       // written directly by the main kernel
   const int i0 = mb * p.rows_per_mb;
