@@ -150,7 +150,8 @@ __device__ __forceinline__ void fold_one(Stat& st, float v, int x, float c, int 
 // (max, lowest arg-max, sum of exp2((z - max) c)) of U vectors of N logits, the
 // first at index x0, the u-th `stride` further: one maximum and one rescale per
 // call, then independent exponentials and tree sums.  -inf entries (slots past the
-// end of the chunk) change neither the maximum nor the sum.
+// end of the chunk) change neither the maximum nor the sum.  st.idx is left at the first
+// index of the vector that holds the maximum (see scan_chunk).
 template <int U, int N>
 __device__ __forceinline__ void fold_stats(Stat& st, const float (&v)[U][N], int x0, int stride, float c) {
   float vm[U];
@@ -170,14 +171,12 @@ __device__ __forceinline__ void fold_stats(Stat& st, const float (&v)[U][N], int
   for (int u = 1; u < U; ++u) vmax = fmaxf(vmax, vm[u]);
   if (vmax > st.m) {
     st.s = (st.m > -CUDART_INF_F) ? st.s * fast_exp2((st.m - vmax) * c) : 0.f;
-    // lowest index that holds the new maximum: walk backwards, the last hit wins
+    // first vector that holds the new maximum (walk backwards, the last hit wins); which of
+    // its N logits it is gets settled once, at the end of the chunk (this branch is taken in
+    // almost every sweep of a short chunk, so it stays small)
 #pragma unroll
-    for (int u = U - 1; u >= 0; --u) {
-      if (vm[u] == vmax) {
-#pragma unroll
-        for (int i = N - 1; i >= 0; --i) if (v[u][i] == vmax) st.idx = x0 + u * stride + i;
-      }
-    }
+    for (int u = U - 1; u >= 0; --u)
+      if (vm[u] == vmax) st.idx = x0 + u * stride;
     st.m = vmax;
   }
   if (st.m > -CUDART_INF_F) {
@@ -269,6 +268,15 @@ __device__ Stat scan_chunk(const T* row, int begin, int end, float c, int exclud
 #pragma unroll
       for (int u = 0; u < U; ++u) cur[u] = nxt[u];
       x = xn;
+    }
+    if (STATS && st.m > -CUDART_INF_F) {
+      // settle the arg-max inside its vector: lowest index equal to the maximum
+      float vv[N];
+      Vec<T>::convert(__ldg(reinterpret_cast<const uint4*>(row + st.idx)), vv);
+      int off = 0;
+#pragma unroll
+      for (int i = N - 1; i >= 0; --i) if (vv[i] == st.m) off = i;
+      st.idx += off;
     }
     for (int xt = full_end + threadIdx.x; xt < end; xt += blockDim.x) {
       Stat one = stat_empty();
