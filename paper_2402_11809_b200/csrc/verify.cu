@@ -475,10 +475,14 @@ __global__ void __launch_bounds__(SPACE_VERIFY_THREADS)
 verify_emit_kernel(const VerifyParams p) {
   pdl_launch_dependents();
   pdl_wait();
-  const int b = blockIdx.z, slot = blockIdx.y, ch = blockIdx.x;
+  const int b = blockIdx.y, ch = blockIdx.x;
   const int k1 = p.k + 1;
   const int i_star = p.n_accept[b];
   const bool sample = p.mode == SPACE_MODE_SAMPLE;
+  // Slot is the slowest grid dimension and the rows with Gumbel noise (several times
+  // the work of a plain row) come first in it: the long blocks of every sequence
+  // start before any short one, so none is left for the tail of the launch.
+  const int slot = sample ? (blockIdx.z == 0 ? p.k : (int)blockIdx.z - 1) : (int)blockIdx.z;
   const bool literal = sample && p.resample == SPACE_RESAMPLE_PAPER_LITERAL;
   const int n_slots = sample ? k1 : p.k;
   const uint32_t seq = p.seq_id ? p.seq_id[b] : (uint32_t)b;
@@ -634,7 +638,7 @@ void launch_fused(space_ctx* ctx, const VerifyParams& p, cudaStream_t st) {
 
 template <typename T, bool VECTOR>
 void launch_both(space_ctx* ctx, const VerifyParams& p, int n_slots_b, cudaStream_t st) {
-  dim3 ga(p.n_chunks, p.k + 1, p.B), gb(p.n_chunks, n_slots_b, p.B);
+  dim3 ga(p.n_chunks, p.k + 1, p.B), gb(p.n_chunks, p.B, n_slots_b);
   {
     ProfScope ps(ctx, SPACE_K_VERIFY_TARGET, st);
     launch_pdl(verify_target_kernel<T, VECTOR>, ga, dim3(SPACE_VERIFY_THREADS), 0, st, p);
