@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include "../../include/space.h"
+#include <cstring>
 
 #define SPACE_VERIFY_MAX_CHUNKS 64
 #define SPACE_VERIFY_THREADS 256
@@ -31,8 +32,18 @@ __host__ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t 
 }
 
 // 32-bit word -> uniform in (0,1), exactly representable in binary32.
+// ((w >> 9) + 1/2) 2^-23, built without an integer-to-float conversion: the 23 bits
+// become the mantissa of a float in [1, 2), and subtracting 1 - 2^-24 (the largest
+// float below 1) leaves (2m + 1) 2^-24 exactly.
 __host__ __device__ __forceinline__ float uniform_open(uint32_t w) {
-  return ((float)(w >> 9) + 0.5f) * 1.1920928955078125e-07f;   // 2^-23
+  const uint32_t bits = 0x3F800000u | (w >> 9);
+  float f;
+#ifdef __CUDA_ARCH__
+  f = __uint_as_float(bits);
+#else
+  memcpy(&f, &bits, sizeof(f));
+#endif
+  return f - 0.99999994f;
 }
 
 enum { PURPOSE_ACCEPT = 0, PURPOSE_TOKEN = 1, PURPOSE_DRAFT = 2 };
