@@ -226,7 +226,10 @@ int space_kv_commit(space_ctx* ctx, const space_commit_args* args, void* stream)
 
 /* The three stages from host buffers; synchronises `stream` before returning.
  * Needs cfg.host_staging.  Only sequence prefixes in use are copied (with
- * cache_resident: only the block's rows, see the field). */
+ * cache_resident: only the block's rows, see the field).  The call stages the
+ * small per-sequence arrays in a pinned buffer of the context: one call at a
+ * time per context.  Errors: INVALID_ARG (NULL pointer), WORKSPACE (no staging,
+ * or sizes beyond cfg), CUDA. */
 int space_step_host(space_ctx* ctx, const space_host_step_args* args, void* stream);
 
 /* Number of kernels this context has launched so far. */
