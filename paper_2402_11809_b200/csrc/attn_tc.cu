@@ -36,7 +36,7 @@
 namespace {
 
 constexpr int TILE_N = 128;            // keys per tile
-constexpr int SHARE_COST = 3;          // fixed cost of a share (query load, first-tile reference, epilogue) in tiles
+constexpr int SHARE_COST = 4;          // fixed cost of a share (query load, first tile, last product, epilogue) in tiles; swept 2..8
 constexpr int ROWS = 128;              // MMA M
 constexpr int THREADS = 384;            // K, MMA, V, Q warps + 8 softmax warps
 constexpr uint64_t WAIT_NS = 1000000000ull;   // one second per wait
