@@ -701,11 +701,11 @@ int launch_verify(space_ctx* ctx, const space_verify_args* a, cudaStream_t st) {
     ctx->launches += 1;
     return cuda_ok(cudaGetLastError());
   }
-  // enough chunks to put about eight blocks on every SM (many loads in flight, and
-  // the Gumbel rows of sampling mode spread over the GPU), but no chunk below
-  // four sweeps of a block
+  // enough chunks to put about four blocks on every SM: little more than one resident
+  // wave (measured on the 64-sequence sampling workload: 4 per SM 29 / 39 us, 8 per SM
+  // 31 / 43 us, 16 per SM 38 / 54 us), but no chunk below four sweeps of a block
   const int rows = a->batch * (a->k + 1);
-  int nc = (8 * ctx->sm_count + rows - 1) / rows;
+  int nc = (4 * ctx->sm_count + rows - 1) / rows;
   const int min_chunk = SPACE_VERIFY_THREADS * vec * 4;
   const int max_nc = (a->vocab + min_chunk - 1) / min_chunk;
   if (nc > max_nc) nc = max_nc;
