@@ -471,7 +471,7 @@ verify_target_kernel(const VerifyParams p) {
 }
 
 template <typename T, bool VECTOR>
-__global__ void __launch_bounds__(SPACE_VERIFY_THREADS)
+__global__ void __launch_bounds__(SPACE_VERIFY_THREADS, 3)   // 80 registers, no spills: three blocks per SM
 verify_emit_kernel(const VerifyParams p) {
   pdl_launch_dependents();
   pdl_wait();
