@@ -14,6 +14,8 @@ attention  block-over-cache attention in fp64
 philox     Philox4x32-10 counter-based generator (Salmon et al., SC'11)
 verify     Algorithm 1 verification: greedy and rejection sampling
 commit     compaction of accepted rows into the verified cache
+lmhead     output projection (hidden states x output embedding) followed by greedy
+           verification: the end of the model call of Algorithm 1 and the loop after it
 bf16       exact bf16 <-> float conversion helpers
 
 Parity pins: every function here is pinned by a CPU test (tests/test_oracle_*.py);

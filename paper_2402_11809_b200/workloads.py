@@ -126,3 +126,60 @@ def algorithmic_bytes(cfg, kv_len, n_accept=None):
     acc = int(np.sum(n_accept)) if n_accept is not None else 0
     cm = acc * H_kv * d * 2 * 2 * 2
     return dict(kv=kv, q_out=qo, logits=lg, commit=cm, total=kv + qo + lg + cm)
+
+
+# Output-projection workloads: the step starts from the block rows' final hidden
+# states and the output embedding instead of ready logits.  D is the hidden size.
+LMHEAD_CONFIGS = {
+    "lmhead_tiny": dict(B=1, k=4, V=1000, D=256, sigma=2.0, p_accept=(0.7, 0.7), seed=10),
+    "lmhead_llama7b": dict(B=1, k=5, V=32000, D=4096, sigma=3.0, p_accept=(0.8, 0.8), seed=11),
+    "lmhead_batch4": dict(B=4, k=5, V=32000, D=4096, sigma=3.0, p_accept=(0.3, 0.9), seed=12),
+}
+
+
+def resolve_lmhead(name, **overrides):
+    cfg = dict(LMHEAD_CONFIGS[name])
+    cfg.update(overrides)
+    cfg["name"] = name
+    return cfg
+
+
+def make_lmhead_inputs(cfg, set_index=0):
+    """hidden [B, n_q, D] and weight [V, D] as bf16 bit patterns, candidates [B, k].
+
+    weight ~ N(0, sigma^2 / D) and hidden ~ N(0, 1), so a logit is ~ N(0, sigma).
+    With probability p per position the candidate is planted: the hidden row that
+    scores it is replaced by a multiple of the candidate's own embedding row (plus
+    a little noise), which makes that token the row's maximum by a wide margin
+    (its logit is near PLANT_GREEDY, every other one near N(0, PLANT_GREEDY / sqrt(D)))."""
+    B, k, V, D = (cfg[x] for x in ("B", "k", "V", "D"))
+    n_q = n_block_rows(k)
+    rng = np.random.Generator(np.random.Philox(key=[cfg["seed"], set_index]))
+    w_sigma = cfg["sigma"] / np.sqrt(D)
+    weight = np.empty((V, D), dtype=np.uint16)
+    step = max(1, (1 << 24) // D)
+    for r0 in range(0, V, step):                              # in slabs: bounded temporaries
+        r1 = min(V, r0 + step)
+        weight[r0:r1] = _normal_bf16(rng, (r1 - r0, D), w_sigma)
+    hidden_f = rng.standard_normal((B, n_q, D), dtype=np.float32)
+    cand = rng.integers(0, V, size=(B, k)).astype(np.int32)
+    p_lo, p_hi = cfg["p_accept"]
+    p_seq = rng.uniform(p_lo, p_hi, size=B)
+    planted = rng.uniform(size=(B, k)) < p_seq[:, None]
+    gain = np.float32(PLANT_GREEDY / cfg["sigma"] ** 2)
+    for b in range(B):
+        for i in range(k):
+            if planted[b, i]:
+                w_row = (weight[int(cand[b, i])].astype(np.uint32) << np.uint32(16)).view(np.float32)
+                hidden_f[b, i * (k + 1)] = gain * w_row + np.float32(0.05) * hidden_f[b, i * (k + 1)]
+    hidden = f32_to_bf16_bits(hidden_f)
+    cand_prob = np.ones((B, k), dtype=np.float32)
+    return dict(hidden=hidden, weight=weight, cand=cand, cand_prob=cand_prob, planted=planted, n_q=n_q)
+
+
+def lmhead_algorithmic_bytes(cfg):
+    """Bytes the projection step has to move at least once: the output embedding
+    read once and the block rows' hidden states."""
+    B, k, V, D = (cfg[x] for x in ("B", "k", "V", "D"))
+    return dict(weight=V * D * 2, hidden=B * n_block_rows(k) * D * 2,
+                total=V * D * 2 + B * n_block_rows(k) * D * 2)
