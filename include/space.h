@@ -130,6 +130,35 @@ typedef struct {
   int32_t* status;             /* device [B] or NULL                           */
 } space_verify_args;
 
+/* Output projection fused with greedy verification: the end of the model call
+ * P = M(I) of Algorithm 1 (logits[r, x] = <h_r, W_x> for every block row r and
+ * vocabulary token x; the rows of P are their softmax) and the loop after it
+ * (acceptance of the candidates against the arg-max chain, extra token, <EOS>,
+ * next candidates from the mask rows of group i*; Sec. 3.2).  The logits are
+ * never written: only (max, lowest arg-max, sum exp) of every row leave the chip. */
+#define SPACE_LMHEAD_MAX_ROWS 256   /* batch * (k+1)^2 block rows per call     */
+typedef struct {
+  int32_t batch, k, vocab;
+  int32_t hidden_dim;          /* D, a multiple of 8                           */
+  int32_t eos_id;              /* -1: no end-of-sequence handling              */
+  int32_t reserved;            /* 0                                            */
+  const void* hidden;          /* device bf16 [B * n_q, D]: final hidden state of every block row,
+                                  sequence-major, block row order               */
+  int64_t hidden_row_stride;   /* elements between rows, a multiple of 8       */
+  const void* weight;          /* device bf16 [V, D]: output embedding, one row per token */
+  int64_t weight_row_stride;   /* elements between rows, a multiple of 8       */
+  const int32_t* cand;         /* device [B, k]  L_c                           */
+  int32_t* n_accept;           /* device [B]       i*                          */
+  int32_t* out_tokens;         /* device [B, k+1]  emitted tokens, -1 padded   */
+  int32_t* n_out;              /* device [B]                                   */
+  int32_t* next_cand;          /* device [B, k]                                */
+  float*   next_cand_prob;     /* device [B, k]  softmax (T = 1) of the token's own row */
+  uint8_t* finished;           /* device [B]                                   */
+  int32_t* status;             /* device [B] or NULL                           */
+  float*   row_max;            /* device [B * n_q] or NULL: largest logit of every block row */
+  int32_t* row_argmax;         /* device [B * n_q] or NULL: its token (lowest on ties) */
+} space_lmhead_args;
+
 /* Compaction of the accepted rows (no counterpart in Algorithm 1, which
  * re-runs the model on the whole sequence; needed by any cached forward). */
 typedef struct {
@@ -221,6 +250,17 @@ int space_verify(space_ctx* ctx, const space_verify_args* args, void* stream);
 #define SPACE_NOALLOC_MAX_BATCH 8
 int space_verify_greedy_noalloc(const space_verify_args* args, void* stream);
 
+/* Greedy step from hidden states (see space_lmhead_args): one kernel, the output
+ * embedding is read once, products on the tensor cores in bf16 with fp32
+ * accumulation, arg-max decided on the fp32 accumulators (lowest token on exact
+ * ties).  Same outputs as space_verify in SPACE_MODE_GREEDY on the logits the
+ * projection defines.  Asynchronous on `stream`, no allocation.  One call at a
+ * time per context (the calls share the context's reduction scratch).
+ * Errors: INVALID_ARG (NULL pointer, sizes), WORKSPACE (batch or k beyond the
+ * context's), ALIGNMENT (16-byte base, strides and D multiples of 8),
+ * UNSUPPORTED (more than SPACE_LMHEAD_MAX_ROWS block rows), CUDA. */
+int space_lmhead_verify(space_ctx* ctx, const space_lmhead_args* args, void* stream);
+
 /* Move accepted rows L+g(k+1) -> L+g, g = 1..i*; lengths grow by i*+1. */
 int space_kv_commit(space_ctx* ctx, const space_commit_args* args, void* stream);
 
@@ -236,16 +276,17 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* args, void* stre
 int64_t space_launch_count(const space_ctx* ctx);
 
 /* Per-kernel timing with CUDA events recorded on the launching stream around
- * every kernel (attention, merge, verify target rows, verify emit, commit).
+ * every kernel (attention, merge, verify target rows, verify emit, commit,
+ * projection + verify).
  * space_profile_enable(ctx, 1) starts a fresh recording (at most
  * SPACE_PROFILE_MAX_STEPS steps are kept; later ones are not recorded);
  * space_profile_enable(ctx, 0) stops it.  Do not enable during stream capture.
  * space_profile_read waits for the recorded events, writes the summed
- * milliseconds per kernel into ms[5] and the number of recorded launches per
- * kernel into n[5], and clears the recording. */
+ * milliseconds per kernel into ms[SPACE_K_COUNT] and the number of recorded launches
+ * per kernel into n[SPACE_K_COUNT], and clears the recording. */
 #define SPACE_PROFILE_MAX_STEPS 4096
 enum { SPACE_K_ATTN = 0, SPACE_K_MERGE = 1, SPACE_K_VERIFY_TARGET = 2, SPACE_K_VERIFY_EMIT = 3,
-       SPACE_K_COMMIT = 4, SPACE_K_COUNT = 5 };
+       SPACE_K_COMMIT = 4, SPACE_K_LMHEAD = 5, SPACE_K_COUNT = 6 };
 int space_profile_enable(space_ctx* ctx, int on);
 int space_profile_read(space_ctx* ctx, float* ms, int64_t* n);
 

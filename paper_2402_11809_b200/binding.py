@@ -16,6 +16,7 @@ OK = 0
 E_INVALID_ARG, E_UNSUPPORTED, E_ALIGNMENT, E_WORKSPACE, E_CUDA, E_NO_DEVICE = -1, -2, -3, -4, -5, -6
 E_STATIC_LIMIT = -7
 NOALLOC_MAX_BATCH = 8
+LMHEAD_MAX_ROWS = 256
 MASK_SAME_GROUP, MASK_EQ5_LITERAL = 0, 1
 MODE_GREEDY, MODE_SAMPLE = 0, 1
 RESAMPLE_RESIDUAL_POINTMASS, RESAMPLE_PAPER_LITERAL = 0, 1
@@ -25,6 +26,7 @@ ST_CAPACITY, ST_BAD_CANDIDATE, ST_TIMEOUT = 1, 2, 4
 
 EXPORTS = ["space_create", "space_destroy", "space_workspace_bytes", "space_layout",
            "space_attn_step", "space_verify", "space_verify_greedy_noalloc", "space_kv_commit",
+           "space_lmhead_verify",
            "space_step_host",
            "space_launch_count", "space_profile_enable", "space_profile_read",
            "space_debug_philox", "space_strerror"]
@@ -77,6 +79,17 @@ class CommitArgs(C.Structure):
                 ("status", C.c_void_p)]
 
 
+class LmHeadArgs(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("k", C.c_int32), ("vocab", C.c_int32),
+                ("hidden_dim", C.c_int32), ("eos_id", C.c_int32), ("reserved", C.c_int32),
+                ("hidden", C.c_void_p), ("hidden_row_stride", C.c_int64),
+                ("weight", C.c_void_p), ("weight_row_stride", C.c_int64),
+                ("cand", C.c_void_p), ("n_accept", C.c_void_p), ("out_tokens", C.c_void_p),
+                ("n_out", C.c_void_p), ("next_cand", C.c_void_p), ("next_cand_prob", C.c_void_p),
+                ("finished", C.c_void_p), ("status", C.c_void_p), ("row_max", C.c_void_p),
+                ("row_argmax", C.c_void_p)]
+
+
 class HostStepArgs(C.Structure):
     _fields_ = [("batch", C.c_int32), ("k", C.c_int32), ("vocab", C.c_int32),
                 ("logits_dtype", C.c_int32), ("mode", C.c_int32), ("resample", C.c_int32),
@@ -100,7 +113,8 @@ lib.space_workspace_bytes.restype = C.c_size_t
 lib.space_layout.argtypes = [C.c_int, C.c_int, C.POINTER(Layout)]
 lib.space_layout.restype = C.c_int
 for _name, _arg in (("space_attn_step", AttnArgs), ("space_verify", VerifyArgs),
-                    ("space_kv_commit", CommitArgs), ("space_step_host", HostStepArgs)):
+                    ("space_kv_commit", CommitArgs), ("space_step_host", HostStepArgs),
+                    ("space_lmhead_verify", LmHeadArgs)):
     getattr(lib, _name).argtypes = [C.c_void_p, C.POINTER(_arg), C.c_void_p]
     getattr(lib, _name).restype = C.c_int
 lib.space_verify_greedy_noalloc.argtypes = [C.POINTER(VerifyArgs), C.c_void_p]
@@ -182,15 +196,15 @@ class Context:
     def launch_count(self):
         return lib.space_launch_count(self._h)
 
-    KERNELS = ("attn", "merge", "verify_target", "verify_emit", "commit")
+    KERNELS = ("attn", "merge", "verify_target", "verify_emit", "commit", "lmhead")
 
     def space_profile_enable(self, on):
         _check(lib.space_profile_enable(self._h, int(on)))
 
     def space_profile_read(self):
         """{kernel: (summed ms, launches)} since profiling was enabled; clears the recording."""
-        ms = (C.c_float * 5)()
-        n = (C.c_int64 * 5)()
+        ms = (C.c_float * len(self.KERNELS))()
+        n = (C.c_int64 * len(self.KERNELS))()
         _check(lib.space_profile_read(self._h, ms, n))
         return {name: (ms[i], n[i]) for i, name in enumerate(self.KERNELS)}
 
@@ -228,6 +242,23 @@ class Context:
 
     def space_verify(self, args):
         _check(lib.space_verify(self._h, C.byref(args), _stream()))
+
+    # -- space_lmhead_verify ----------------------------------------------
+    def lmhead_args(self, hidden, weight, cand, n_accept, out_tokens, n_out, next_cand, next_cand_prob,
+                    finished, k, eos_id=-1, status=None, row_max=None, row_argmax=None):
+        """hidden [B, n_q, D] and weight [V, D] bf16 CUDA tensors with contiguous last dimension."""
+        assert hidden.stride(2) == 1 and weight.stride(1) == 1
+        assert hidden.stride(0) == hidden.shape[1] * hidden.stride(1)
+        return LmHeadArgs(batch=hidden.shape[0], k=k, vocab=weight.shape[0], hidden_dim=weight.shape[1],
+                          eos_id=eos_id, reserved=0, hidden=_ptr(hidden), hidden_row_stride=hidden.stride(1),
+                          weight=_ptr(weight), weight_row_stride=weight.stride(0), cand=_ptr(cand),
+                          n_accept=_ptr(n_accept), out_tokens=_ptr(out_tokens), n_out=_ptr(n_out),
+                          next_cand=_ptr(next_cand), next_cand_prob=_ptr(next_cand_prob),
+                          finished=_ptr(finished), status=_ptr(status), row_max=_ptr(row_max),
+                          row_argmax=_ptr(row_argmax))
+
+    def space_lmhead_verify(self, args):
+        _check(lib.space_lmhead_verify(self._h, C.byref(args), _stream()))
 
     # -- space_kv_commit --------------------------------------------------
     def commit_args(self, k_cache, v_cache, n_accept, kv_len, k, kv_len_out=None, commit_src=None,

@@ -73,6 +73,8 @@ struct space_ctx {
   VerifyRow* vrow;         // [max_batch][k_max+1]
   VerifyPartial* vfused;   // [max_batch][SPACE_MAX_ROWS][16] single-launch greedy path
   int32_t* scratch_status; // [max_batch] used when the caller passes no status array
+  char* lm_part;           // output-projection statistics [256 block rows][sm_count] x 16 bytes
+  int* lm_counter;         // {arrival counter, first timeout site}
   // staging for space_step_host
   char* stage;
   char* host_small;        // pinned host mirror of the staging area's small per-sequence arrays (host_staging only)
@@ -93,6 +95,8 @@ struct space_ctx {
 int launch_verify(space_ctx* ctx, const space_verify_args* a, cudaStream_t st);
 int launch_verify_noalloc(const space_verify_args* a, cudaStream_t st);
 int launch_commit(space_ctx* ctx, const space_commit_args* a, cudaStream_t st);
+int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_t st);
+size_t lmhead_partial_bytes(int sm_count);
 int launch_attn_simt(space_ctx* ctx, const space_attn_args* a, const uint64_t* mask_rows,
                      cudaStream_t st);
 int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t* mask_rows,

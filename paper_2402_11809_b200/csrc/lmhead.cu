@@ -1,0 +1,493 @@
+// Output projection fused with greedy verification (Algorithm 1: the end of the
+// model call P = M(I) and the loop after it).
+//
+// logits[r, x] = <h_r, W_x> for the (k+1)^2 block rows of every sequence and the
+// whole vocabulary, but the logits never reach memory: the product runs on the
+// tensor cores with the vocabulary on the MMA M extent (A = 128 rows of W,
+// K-major; B = all block rows of the batch, K-major; fp32 accumulators in TMEM),
+// and the epilogue reduces every accumulator column (= one block row) to
+// (max, lowest arg-max, sum exp(z - max)) over the thread block's vocabulary
+// range.  The last thread block to finish combines the ranges and runs the
+// acceptance scan, the extra token, the <EOS> cut and the next candidates.
+//
+// The output embedding is streamed exactly once (the step's HBM roof); the
+// hidden rows are re-read from L2 by every thread block.
+//
+// Vocabulary ranges: thread block c owns rows [V*c/G, V*(c+1)/G) and covers them
+// with boxes of 128 rows; the last box is shifted back so that it ends at the
+// range's end (rows it shares with the previous box are masked in the epilogue),
+// so no box reads past the range and the only rows read twice come from L2.
+//
+// Warps: 0 TMA producer, 1 TMEM owner and MMA issuer, 2..5 epilogue (one TMEM
+// lane quarter each).  Two accumulators alternate between boxes so that the
+// epilogue of one box runs under the products of the next.  Every wait is
+// bounded; an expired wait sets SPACE_ST_TIMEOUT, the block drains and exits.
+#include "common.cuh"
+#include <cuda.h>
+#include <math_constants.h>
+
+namespace {
+
+constexpr int LM_THREADS = 192;
+constexpr int LM_BOX = 128;                 // vocabulary rows per box (MMA M)
+constexpr int LM_KB = 64;                   // hidden elements per stage (128 bytes: one swizzle row)
+constexpr int LM_A_BYTES = LM_BOX * LM_KB * 2;
+constexpr int LM_MAX_STAGES = 10;
+constexpr int LM_MAX_N = 256;               // block rows of the whole batch, padded to 16
+constexpr uint64_t LM_WAIT_NS = 1000000000ull;
+constexpr float LOG2E = 1.4426950408889634f;
+
+struct LmPartial { float m, s; int idx, pad; };   // 16 bytes
+
+struct LmParams {
+  CUtensorMap tm_w, tm_h;
+  int B, k, V, D, n_q;
+  int n_rows;                 // B * n_q
+  int n_pad;                  // n_rows rounded up to 16: N of the MMAs
+  int stages;
+  int eos_id;
+  const int32_t* cand;
+  int32_t* n_accept; int32_t* out_tokens; int32_t* n_out; int32_t* next_cand;
+  float* next_cand_prob; uint8_t* finished; int32_t* status;
+  float* row_max; int32_t* row_argmax;
+  LmPartial* part;            // [n_rows][gridDim.x]
+  int* counter;               // arrival counter (self-resetting)
+  int* err;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false when the limit expired or another thread gave up.
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err, int site) {
+  if (*abort_flag) return mbar_try(bar, parity);
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 255u) == 255u) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > LM_WAIT_NS) break;
+    }
+  }
+  *abort_flag = 1;
+  atomicCAS(err, 0, site);
+  return false;
+}
+__device__ __noinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try(bar, parity)) return;
+    if ((it & 255u) == 255u) {
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > LM_WAIT_NS) return;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
+                                            int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"((uint64_t)tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after()  { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Shared-memory matrix descriptor: K-major rows of 128 bytes, 128-byte swizzle
+// (groups of 8 rows 1024 bytes apart), descriptor version of sm_100.
+__device__ __forceinline__ uint64_t smem_desc_k128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);
+  d |= (uint64_t)((16u >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((1024u >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> f32, M = 128, N = n, both operands K-major.
+__device__ __forceinline__ uint32_t instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(LM_BOX >> 4) << 24);
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// (max, lowest arg-max) over the warp, result in every lane
+__device__ __forceinline__ void warp_max_idx(float& m, int& idx) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float om = __shfl_xor_sync(0xFFFFFFFFu, m, off);
+    const int oi = __shfl_xor_sync(0xFFFFFFFFu, idx, off);
+    if (om > m || (om == m && oi < idx)) { m = om; idx = oi; }
+  }
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+  return v;
+}
+// fold (m2, s2, i2) into (m, s, i): sums are relative to their own maximum
+__device__ __forceinline__ void stat_fold(float& m, float& s, int& i, float m2, float s2, int i2) {
+  if (m2 > m || (m2 == m && i2 < i)) i = i2;
+  const float mm = fmaxf(m, m2);
+  if (mm > -CUDART_INF_F) {
+    const float a = (m > -CUDART_INF_F) ? s * fast_exp2((m - mm) * LOG2E) : 0.f;
+    const float b = (m2 > -CUDART_INF_F) ? s2 * fast_exp2((m2 - mm) * LOG2E) : 0.f;
+    s = a + b;
+  }
+  m = mm;
+}
+
+// Shared-memory plan (dynamic, 1024-byte aligned base):
+//   [stages][A 16 KB] [stages][B n_pad*128] | barriers | running statistics [4][n_pad] x 3 | row results [n_pad] x 2
+struct LmSmem {
+  uint32_t a_off, b_off, bar_off, stat_off, row_off, misc_off, total;
+  int b_bytes;
+  __host__ __device__ LmSmem(int n_pad, int stages) {
+    b_bytes = n_pad * LM_KB * 2;
+    a_off = 0;
+    b_off = a_off + (uint32_t)stages * LM_A_BYTES;
+    bar_off = b_off + (uint32_t)stages * b_bytes;
+    stat_off = bar_off + 8u * (2 * LM_MAX_STAGES + 4);
+    row_off = stat_off + 4u * 3u * 4u * (uint32_t)n_pad;
+    misc_off = row_off + 2u * 4u * (uint32_t)n_pad;
+    total = misc_off + 64u;
+  }
+};
+
+__global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __grid_constant__ LmParams p) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const uint32_t sm_base = smem_u32(smem_raw);
+  const LmSmem L(p.n_pad, p.stages);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int S = p.stages;
+  const uint32_t bar0 = sm_base + L.bar_off;
+#define LBAR(i) (bar0 + 8u * (uint32_t)(i))
+  const int B_FULL = 0, B_EMPTY = LM_MAX_STAGES, B_ACCFULL = 2 * LM_MAX_STAGES, B_ACCEMPTY = 2 * LM_MAX_STAGES + 2;
+  float* run_m = reinterpret_cast<float*>(smem_raw + L.stat_off);          // [4][n_pad]
+  float* run_s = run_m + 4 * p.n_pad;
+  int* run_i = reinterpret_cast<int*>(run_s + 4 * p.n_pad);
+  float* row_s = reinterpret_cast<float*>(smem_raw + L.row_off);           // [n_pad]
+  int* row_i = reinterpret_cast<int*>(row_s + p.n_pad);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_raw + L.misc_off);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + L.misc_off + 4);
+  int* last_flag = reinterpret_cast<int*>(smem_raw + L.misc_off + 8);
+
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) {
+    *abort_flag = (sm_base & 1023u) ? 1 : 0;
+    for (int s = 0; s < S; ++s) { mbar_init(LBAR(B_FULL + s), 1); mbar_init(LBAR(B_EMPTY + s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(LBAR(B_ACCFULL + a), 1); mbar_init(LBAR(B_ACCEMPTY + a), 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (warp == 0 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_w) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_h) : "memory");
+  }
+  for (int t = threadIdx.x; t < 4 * p.n_pad; t += LM_THREADS) { run_m[t] = -CUDART_INF_F; run_s[t] = 0.f; run_i[t] = 0x7FFFFFFF; }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  pdl_wait();                                              // global memory from here on
+
+  // this thread block's vocabulary range and its boxes
+  const int G = gridDim.x, c = blockIdx.x;
+  const int r0 = (int)(((long long)p.V * c) / G), r1 = (int)(((long long)p.V * (c + 1)) / G);
+  const int nb = (r1 - r0 + LM_BOX - 1) / LM_BOX;
+  const int KB = (p.D + LM_KB - 1) / LM_KB;
+  const uint32_t stage_tx = (uint32_t)(LM_A_BYTES + L.b_bytes);
+
+  if (warp == 0) {
+    // ================= producer ==============================================
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = !*abort_flag;
+      for (int box = 0; box < nb && ok; ++box) {
+        const int row0 = (box == nb - 1) ? r1 - LM_BOX : r0 + box * LM_BOX;   // may be negative: zero-filled
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % S;
+          if (it >= (uint32_t)S) ok = mbar_wait(LBAR(B_EMPTY + s), ((it / S) - 1) & 1, abort_flag, p.err, 1);
+          if (!ok) break;
+          mbar_expect_tx(LBAR(B_FULL + s), stage_tx);
+          tma_load_4d(sm_base + L.a_off + s * LM_A_BYTES, &p.tm_w, LBAR(B_FULL + s), kb * LM_KB, row0, 0, 0);
+          tma_load_4d(sm_base + L.b_off + s * L.b_bytes, &p.tm_h, LBAR(B_FULL + s), kb * LM_KB, 0, 0, 0);
+        }
+      }
+      if (!ok) {
+        // copies already requested still land: wait for them (bounded) before the block exits
+        const uint32_t first = it > (uint32_t)S ? it - S : 0;
+        for (uint32_t j = first; j < it; ++j) mbar_drain(LBAR(B_FULL + j % S), (j / S) & 1);
+      }
+    }
+  } else if (warp == 1) {
+    // ================= MMA issuer =============================================
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(p.n_pad);
+      const uint64_t adesc0 = smem_desc_k128(sm_base + L.a_off);
+      const uint64_t bdesc0 = smem_desc_k128(sm_base + L.b_off);
+      uint32_t it = 0;
+      bool ok = !*abort_flag;
+      for (int box = 0; box < nb && ok; ++box) {
+        const int a = box & 1;
+        if (box >= 2) ok = mbar_wait(LBAR(B_ACCEMPTY + a), ((box >> 1) - 1) & 1, abort_flag, p.err, 2);
+        if (!ok) break;
+        tc_fence_after();
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % S;
+          ok = mbar_wait(LBAR(B_FULL + s), (it / S) & 1, abort_flag, p.err, 3);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t ad = adesc0 + (uint64_t)((s * LM_A_BYTES) >> 4);
+          const uint64_t bd = bdesc0 + (uint64_t)((s * L.b_bytes) >> 4);
+#pragma unroll
+          for (int kk = 0; kk < LM_KB / 16; ++kk)          // 32 bytes per 16 elements inside the swizzled row
+            mma_ss(tmem + a * LM_MAX_N, ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 2), idesc, (kb | kk) ? 1u : 0u);
+          tc_commit(LBAR(B_EMPTY + s));
+        }
+        if (ok) tc_commit(LBAR(B_ACCFULL + a));
+      }
+    }
+  } else {
+    // ================= epilogue ================================================
+    const int quarter = warp & 3;                          // TMEM lanes 32*quarter .. +31
+    const int ew = warp - 2;                               // 0..3: row of the running statistics
+    bool ok = true;
+    for (int box = 0; box < nb; ++box) {
+      const int a = box & 1;
+      ok = ok && mbar_wait(LBAR(B_ACCFULL + a), (box >> 1) & 1, abort_flag, p.err, 4);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const bool last_box = box == nb - 1;
+      const int row0 = last_box ? r1 - LM_BOX : r0 + box * LM_BOX;
+      const int own_lo = r0 + box * LM_BOX;                // rows below belong to the previous box (shifted last box)
+      const int x = row0 + quarter * 32 + lane;            // this lane's token
+      const bool valid = x >= own_lo && x < r1 && x >= 0;
+      for (int c0 = 0; c0 < p.n_rows; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * LM_MAX_N + c0), v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float z = valid ? __uint_as_float(v[j]) : -CUDART_INF_F;
+          float m = z; int idx = valid ? x : 0x7FFFFFFF;
+          warp_max_idx(m, idx);
+          const float e = (valid && m > -CUDART_INF_F) ? fast_exp2((z - m) * LOG2E) : 0.f;
+          const float sum = warp_sum(e);
+          if (lane == j && c0 + j < p.n_rows) {
+            const int col = ew * p.n_pad + c0 + j;
+            float rm = run_m[col], rs = run_s[col]; int ri = run_i[col];
+            stat_fold(rm, rs, ri, m, sum, idx);
+            run_m[col] = rm; run_s[col] = rs; run_i[col] = ri;
+          }
+        }
+      }
+      // accumulator `a` may be overwritten by the products of box + 2
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(LBAR(B_ACCEMPTY + a));
+    }
+    epi_sync();
+    const int et = threadIdx.x - 64;                       // 0..127
+    // combine the four lane quarters and publish this block's statistics
+    for (int col = et; col < p.n_rows; col += 128) {
+      float m = run_m[col], s = run_s[col]; int i = run_i[col];
+#pragma unroll
+      for (int w = 1; w < 4; ++w) stat_fold(m, s, i, run_m[w * p.n_pad + col], run_s[w * p.n_pad + col], run_i[w * p.n_pad + col]);
+      LmPartial out; out.m = m; out.s = s; out.idx = i; out.pad = 0;
+      *reinterpret_cast<int4*>(p.part + (size_t)col * G + c) = *reinterpret_cast<const int4*>(&out);
+    }
+    __threadfence();
+    epi_sync();
+    if (et == 0) {
+      const int prev = atomicAdd(p.counter, 1);
+      const int last = prev == G - 1;
+      if (last) *p.counter = 0;                            // ready for the next launch
+      *last_flag = last;
+    }
+    epi_sync();
+    if (*last_flag) {
+      __threadfence();
+      // ---- last thread block: combine the ranges, one warp per block row at a time
+      for (int col = ew; col < p.n_rows; col += 4) {
+        float m = -CUDART_INF_F, s = 0.f; int i = 0x7FFFFFFF;
+        const LmPartial* pc = p.part + (size_t)col * G;
+        for (int g = lane; g < G; g += 32) {
+          const int4 raw = __ldcg(reinterpret_cast<const int4*>(pc + g));
+          stat_fold(m, s, i, __int_as_float(raw.x), __int_as_float(raw.y), raw.z);
+        }
+        float bm = m; int bi = i;
+        warp_max_idx(bm, bi);
+        float sv = (m > -CUDART_INF_F) ? s * fast_exp2((m - bm) * LOG2E) : 0.f;
+        sv = warp_sum(sv);
+        if (lane == 0) {
+          row_s[col] = sv; row_i[col] = bi;
+          if (p.row_max) p.row_max[col] = bm;
+          if (p.row_argmax) p.row_argmax[col] = bi;
+        }
+      }
+      epi_sync();
+      // ---- acceptance scan, emitted tokens, next candidates: one warp per sequence
+      const int k1 = p.k + 1;
+      for (int b = ew; b < p.B; b += 4) {
+        const int* ri = row_i + b * p.n_q;
+        const float* rs = row_s + b * p.n_q;
+        const int* cd = p.cand + b * p.k;
+        int i_star = 0, bits = 0;
+        for (int t = 0; t < p.k; ++t) {
+          const int cc = cd[t];
+          if (cc < 0 || cc >= p.V) bits |= SPACE_ST_BAD_CANDIDATE;
+        }
+        while (i_star < p.k && cd[i_star] >= 0 && cd[i_star] < p.V && cd[i_star] == ri[i_star * k1]) ++i_star;
+        const int j = lane;
+        const int tok = (j < i_star) ? cd[min(j, p.k - 1)] : (j == i_star ? ri[i_star * k1] : -1);
+        const bool is_eos = p.eos_id >= 0 && j <= i_star && tok == p.eos_id;
+        const unsigned eos_mask = __ballot_sync(0xFFFFFFFFu, is_eos && j < k1);
+        const int n_out = eos_mask ? __ffs(eos_mask) - 1 : i_star + 1;
+        if (j < k1) p.out_tokens[b * k1 + j] = (j < n_out) ? tok : -1;
+        if (j < p.k) {                                     // next candidate j+1 from mask row (i*, j+1)
+          const int mr = i_star * k1 + j + 1;
+          p.next_cand[b * p.k + j] = ri[mr];
+          p.next_cand_prob[b * p.k + j] = 1.f / rs[mr];    // softmax at T = 1 of its own maximum
+        }
+        if (j == 0) {
+          p.n_accept[b] = i_star;
+          p.n_out[b] = n_out;
+          p.finished[b] = (uint8_t)(eos_mask != 0);
+          if (p.status && bits) atomicOr(p.status + b, bits);
+        }
+      }
+    }
+  }
+#undef LBAR
+  // ---- exit: every role is done (or has given up); free TMEM
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (*abort_flag && threadIdx.x == 0 && p.status) atomicOr(p.status, SPACE_ST_TIMEOUT);
+  if (warp == 1)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+EncodeTiledFn lm_get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = (EncodeTiledFn)ptr;
+  }
+  return fn;
+}
+// [rows, D] bf16 matrix with `ld` elements between rows, boxes of box_rows x 64
+int lm_make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t D, int64_t ld, int box_rows) {
+  EncodeTiledFn enc = lm_get_encode();
+  if (!enc) return SPACE_E_CUDA;
+  const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)rows, 1, 1};
+  const cuuint64_t strides[3] = {(cuuint64_t)ld * 2, (cuuint64_t)ld * 2 * (cuuint64_t)rows, (cuuint64_t)ld * 2 * (cuuint64_t)rows};
+  const cuuint32_t box[4] = {(cuuint32_t)LM_KB, (cuuint32_t)box_rows, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SPACE_OK : SPACE_E_CUDA;
+}
+
+}  // namespace
+
+size_t lmhead_partial_bytes(int sm_count) { return (size_t)LM_MAX_N * sm_count * sizeof(LmPartial); }
+
+int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_t st) {
+  LmParams p;
+  memset(&p, 0, sizeof(p));
+  p.B = a->batch; p.k = a->k; p.V = a->vocab; p.D = a->hidden_dim;
+  p.n_q = (a->k + 1) * (a->k + 1);
+  p.n_rows = p.B * p.n_q;
+  p.n_pad = (p.n_rows + 15) / 16 * 16;
+  if (p.n_pad > LM_MAX_N) return SPACE_E_UNSUPPORTED;
+  // stages: as many as fit beside the statistics, at most LM_MAX_STAGES
+  int stages = LM_MAX_STAGES;
+  const size_t budget = 220 * 1024;
+  while (stages > 2 && LmSmem(p.n_pad, stages).total + 1024 > budget) --stages;
+  p.stages = stages;
+  const LmSmem L(p.n_pad, stages);
+  p.eos_id = a->eos_id;
+  p.cand = a->cand;
+  p.n_accept = a->n_accept; p.out_tokens = a->out_tokens; p.n_out = a->n_out; p.next_cand = a->next_cand;
+  p.next_cand_prob = a->next_cand_prob; p.finished = a->finished; p.status = a->status;
+  p.row_max = a->row_max; p.row_argmax = a->row_argmax;
+  p.part = reinterpret_cast<LmPartial*>(ctx->lm_part);
+  p.counter = ctx->lm_counter;
+  p.err = ctx->lm_counter + 1;
+  int rc = lm_make_map(&p.tm_w, a->weight, a->vocab, a->hidden_dim, a->weight_row_stride, LM_BOX);
+  if (rc == SPACE_OK) rc = lm_make_map(&p.tm_h, a->hidden, p.n_rows, a->hidden_dim, a->hidden_row_stride, p.n_pad);
+  if (rc != SPACE_OK) return rc;
+  int grid = ctx->sm_count;
+  const int max_useful = (a->vocab + 31) / 32;             // at least 32 tokens per thread block
+  if (grid > max_useful) grid = max_useful;
+  if (grid < 1) grid = 1;
+  const size_t sm = L.total + 1024;                        // room to align the base to 1024 bytes
+  cudaFuncSetAttribute(lmhead_verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+  {
+    ProfScope ps(ctx, SPACE_K_LMHEAD, st);
+    launch_pdl(lmhead_verify_kernel, dim3(grid), dim3(LM_THREADS), sm, st, p);
+  }
+  ctx->launches += 1;
+  return cuda_ok(cudaGetLastError());
+}

@@ -27,7 +27,7 @@ int config_supported(const space_config* c) {
 }
 
 struct Carve {
-  size_t attn_part, counters, merge_cnt, vpart, vfused, vrow, status, stage, total;
+  size_t attn_part, counters, merge_cnt, vpart, vfused, vrow, status, lm_part, lm_counter, stage, total;
   size_t part_slots;
   // staging sub-offsets (relative to stage)
   size_t st_q, st_k, st_v, st_logits, st_small;
@@ -47,6 +47,8 @@ Carve carve(const space_config* c, int sm_count) {
   v.vfused = off; off += align_up((size_t)c->max_batch * SPACE_MAX_ROWS * 16 * sizeof(VerifyPartial), 256);
   v.vrow = off; off += align_up((size_t)c->max_batch * (c->k_max + 1) * sizeof(VerifyRow), 256);
   v.status = off; off += align_up((size_t)c->max_batch * sizeof(int32_t), 256);
+  v.lm_part = off; off += align_up(lmhead_partial_bytes(sm_count), 256);
+  v.lm_counter = off; off += 256;
   v.stage = off;
   if (c->host_staging) {
     const size_t n_q = (size_t)(c->k_max + 1) * (c->k_max + 1);
@@ -142,6 +144,8 @@ int space_create(space_ctx** out, const space_config* cfg) {
   ctx->vrow = (VerifyRow*)(ctx->ws + cv.vrow);
   ctx->vfused = (VerifyPartial*)(ctx->ws + cv.vfused);
   ctx->scratch_status = (int32_t*)(ctx->ws + cv.status);
+  ctx->lm_part = ctx->ws + cv.lm_part;
+  ctx->lm_counter = (int*)(ctx->ws + cv.lm_counter);
   ctx->stage = cfg->host_staging ? ctx->ws + cv.stage : nullptr;
   ctx->stage_bytes = cv.total - cv.stage;
   ctx->host_small = nullptr;
@@ -240,6 +244,22 @@ int space_verify_greedy_noalloc(const space_verify_args* a, void* stream) {
   const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;
   if ((uintptr_t)a->logits % esz) return SPACE_E_ALIGNMENT;
   return launch_verify_noalloc(a, (cudaStream_t)stream);
+}
+
+int space_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, void* stream) {
+  if (!ctx || !a) return SPACE_E_INVALID_ARG;
+  if (a->batch < 1 || a->batch > ctx->cfg.max_batch || a->k < 1 || a->k > ctx->cfg.k_max) return SPACE_E_WORKSPACE;
+  if (a->vocab < 1 || a->hidden_dim < 8) return SPACE_E_INVALID_ARG;
+  if (!a->hidden || !a->weight || !a->cand || !a->n_accept || !a->out_tokens || !a->n_out || !a->next_cand ||
+      !a->next_cand_prob || !a->finished)
+    return SPACE_E_INVALID_ARG;
+  if (a->hidden_dim % 8 || a->hidden_row_stride % 8 || a->weight_row_stride % 8 ||
+      ((uintptr_t)a->hidden & 15) || ((uintptr_t)a->weight & 15))
+    return SPACE_E_ALIGNMENT;
+  if (a->hidden_row_stride < a->hidden_dim || a->weight_row_stride < a->hidden_dim) return SPACE_E_INVALID_ARG;
+  if (a->batch * (a->k + 1) * (a->k + 1) > SPACE_LMHEAD_MAX_ROWS) return SPACE_E_UNSUPPORTED;
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return SPACE_E_CUDA;
+  return launch_lmhead_verify(ctx, a, (cudaStream_t)stream);
 }
 
 int space_kv_commit(space_ctx* ctx, const space_commit_args* a, void* stream) {
