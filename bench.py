@@ -3,6 +3,9 @@
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
 
+--config lmhead_* times space_lmhead_verify (output projection fused with greedy
+verification, one kernel per step) on a projection workload instead.
+
 One step = space_attn_step + space_verify + space_kv_commit for the whole batch
 of one synthetic input set.  Several distinct input sets are rotated so that no
 step finds its inputs in L2.  Prints ONE JSON line (rank 0).
@@ -35,6 +38,8 @@ L2_BYTES = 126 * 1024 * 1024
 # profiles/attn_tc_kernel_llama7b.txt and profiles/attn_rows_kernel_gqa70b.txt (bytes); None for workloads
 # without a capture of the current kernel
 ATTN_TRAFFIC = {"llama7b": 34518272, "gqa70b": 293366272}
+# the same for the projection kernel (profiles/lmhead_verify_kernel_*.txt)
+LMHEAD_TRAFFIC = {}
 METRIC = "auto-correct steps/sec"
 UNIT = "steps/s"
 
@@ -405,16 +410,210 @@ def run_ours(args):
     replicas.shutdown()
 
 
+# ------------------------------------------------- projection + verify workloads
+def oracle_lmhead_step(cfg, x):
+    from oracle.lmhead import lmhead_verify_step
+    return lmhead_verify_step(x["hidden"], x["weight"], x["cand"], x["cand_prob"], cfg["k"])
+
+
+def run_lmhead(args):
+    """space_lmhead_verify on a projection workload: one step = one call (one kernel)."""
+    import torch
+    from paper_2402_11809_b200 import device as H
+    from paper_2402_11809_b200 import build
+    build.build()
+    from paper_2402_11809_b200 import binding as B
+
+    rank, world, local = replicas.rank_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --impl ours needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    replicas.init("nccl", local)
+    cfg = workloads.resolve_lmhead(args.config)
+    Bn, k, V, D = cfg["B"], cfg["k"], cfg["V"], cfg["D"]
+    n_q = workloads.n_block_rows(k)
+    ab = workloads.lmhead_algorithmic_bytes(cfg)
+    n_sets = min(8, max(2, int(np.ceil(2.0 * L2_BYTES / ab["total"]))))
+    sets = [workloads.make_lmhead_inputs(cfg, set_index=replicas.set_index(rank, i)) for i in range(n_sets)]
+    ctx = B.Context(device=local, max_batch=Bn, n_q_heads=8, n_kv_heads=8, head_dim=64, k_max=k, vocab=V, s_cap=256)
+    dev = "cuda"
+    bufs, arg_sets = [], []
+    for x in sets:
+        d = dict(hidden=H.to_dev(x["hidden"]), weight=H.to_dev(x["weight"]), cand=H.to_dev(x["cand"]),
+                 n_accept=torch.zeros(Bn, dtype=torch.int32, device=dev),
+                 out_tokens=torch.zeros((Bn, k + 1), dtype=torch.int32, device=dev),
+                 n_out=torch.zeros(Bn, dtype=torch.int32, device=dev),
+                 next_cand=torch.zeros((Bn, k), dtype=torch.int32, device=dev),
+                 next_cand_prob=torch.zeros((Bn, k), device=dev),
+                 finished=torch.zeros(Bn, dtype=torch.uint8, device=dev),
+                 status=torch.zeros(Bn, dtype=torch.int32, device=dev))
+        bufs.append(d)
+        arg_sets.append(ctx.lmhead_args(d["hidden"], d["weight"], d["cand"], d["n_accept"], d["out_tokens"],
+                                        d["n_out"], d["next_cand"], d["next_cand_prob"], d["finished"], k,
+                                        status=d["status"]))
+
+    def step(i):
+        ctx.space_lmhead_verify(arg_sets[i % n_sets])
+
+    stream = torch.cuda.Stream()
+    K, W = args.steps, max(args.warmup, 3)
+    with torch.cuda.stream(stream):
+        for i in range(n_sets):
+            step(i)
+        stream.synchronize()
+        g_full = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_full, stream=stream):
+            for i in range(n_sets):
+                step(i)
+
+        def run_steps(n):
+            for _ in range(n // n_sets):
+                g_full.replay()
+            for i in range(n % n_sets):
+                step(i)
+
+        run_steps(W)
+        stream.synchronize()
+        sampler = ClockSampler(local)
+        replicas.barrier()
+        torch.cuda.synchronize()
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        run_steps(K)
+        e1.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        replicas.barrier()
+        ms = e0.elapsed_time(e1)
+        n_prof = min(K, 2048)
+        ctx.space_profile_enable(1)
+        for i in range(n_prof):
+            step(i)
+        stream.synchronize()
+        ctx.space_profile_enable(0)
+        prof = ctx.space_profile_read()
+        clocks = sampler.stop()
+        status = sum(int(d["status"].abs().sum()) for d in bufs)
+    steps_per_s, sec = replicas.job_throughput(K, ms * 1e-3, device="cuda")
+    ms = sec * 1e3
+
+    # ---- end to end: the step's own inputs (hidden states, candidates) come from pinned host
+    # memory every step and its results are read back; the output embedding is model state and
+    # stays on the device
+    x, d = sets[0], bufs[0]
+    pin_h = torch.from_numpy(x["hidden"].view(np.int16)).clone().pin_memory()
+    pin_c = torch.from_numpy(x["cand"]).clone().pin_memory()
+    res_names = ("n_accept", "out_tokens", "n_out", "next_cand", "next_cand_prob", "finished", "status")
+    pin_o = {n_: torch.empty_like(d[n_], device="cpu").pin_memory() for n_ in res_names}
+    h2d = pin_h.numel() * 2 + pin_c.numel() * 4
+    d2h = sum(t.numel() * t.element_size() for t in pin_o.values())
+    n_e2e = max(3, min(K, 1000))
+    with torch.cuda.stream(stream):
+        def host_step():
+            d["hidden"].view(torch.int16).copy_(pin_h, non_blocking=True)
+            d["cand"].copy_(pin_c, non_blocking=True)
+            ctx.space_lmhead_verify(arg_sets[0])
+            for n_ in res_names:
+                pin_o[n_].copy_(d[n_], non_blocking=True)
+            stream.synchronize()
+        for _ in range(3):
+            host_step()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            host_step()
+        e2e_s = time.perf_counter() - t0
+    e2e_val, _ = replicas.job_throughput(n_e2e, e2e_s, device="cuda")
+    if rank != 0:
+        replicas.shutdown()
+        return
+    peak, peak_tf, peak_src = load_peaks()
+    k_ms, k_n = prof["lmhead"]
+    k_us = 1e3 * k_ms / max(k_n, 1)
+    achieved = ab["total"] / (k_us * 1e-6) / 1e9 if k_n else None
+    ref = oracle_lmhead_step(cfg, sets[0])
+    matches = bool(np.array_equal(pin_o["n_accept"].numpy(), ref["n_accept"]) and
+                   np.array_equal(pin_o["out_tokens"].numpy(), ref["out_tokens"]) and
+                   np.array_equal(pin_o["next_cand"].numpy(), ref["next_cand"]))
+    t0 = time.perf_counter()
+    reps = 0
+    while reps < 2 or time.perf_counter() - t0 < 10.0:
+        oracle_lmhead_step(cfg, sets[0])
+        reps += 1
+    cpu_el = time.perf_counter() - t0
+    line = {
+        "metric": "projection+verify steps/sec", "value": steps_per_s, "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg["name"], "batch": Bn, "k": k, "vocab": V, "hidden_dim": D,
+                   "l2": f"{n_sets} distinct weight sets rotated ({n_sets * ab['total'] / 1e6:.0f} MB > 2 x L2)",
+                   "launch": "CUDA graph replay of the C-ABI call",
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "gpu_launches": int(K),
+        "step_algorithmic_bytes": float(ab["total"]),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "peak_source": peak_src + " (burst copy figure)",
+                     "frac": (achieved / peak) if achieved else None, "kernel": "lmhead_verify_kernel",
+                     "traffic": LMHEAD_TRAFFIC.get(cfg["name"]),
+                     "algorithmic_bytes_per_launch": float(ab["total"]), "avg_launch_us": k_us,
+                     "launches_timed": int(k_n),
+                     "timing": "CUDA events around every launch, stream-launched pass after the graph-timed region"},
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "steps": n_e2e, "matches_oracle": matches,
+                "note": "hidden states and candidates uploaded from pinned host memory and results read back "
+                        "every step; the output embedding is model state resident on the device"},
+        "cpu_baseline": {"value": reps / cpu_el, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                         "sample": f"{reps} whole step(s) of {cfg['name']} in {cpu_el:.1f} s"},
+        "clocks": clocks,
+        "device_status_bits": status,
+    }
+    print(json.dumps(line), flush=True)
+    replicas.shutdown()
+
+
+def run_lmhead_reference(args):
+    rank, _, _ = replicas.rank_env()
+    if rank != 0:
+        return
+    cfg = workloads.resolve_lmhead(args.config)
+    x = workloads.make_lmhead_inputs(cfg)
+    oracle_lmhead_step(cfg, x)
+    t0 = time.perf_counter()
+    oracle_lmhead_step(cfg, x)
+    one = time.perf_counter() - t0
+    reps = max(1, min(args.steps, int(150.0 / max(one, 1e-6))))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle_lmhead_step(cfg, x)
+    el = time.perf_counter() - t0
+    sps = reps / el
+    print(json.dumps({
+        "impl": "reference", "metric": "projection+verify steps/sec", "value": sps, "unit": UNIT,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / sps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg["name"], "timed_steps": reps,
+                   "note": "CPU oracle (numpy fp64), whole steps; repetitions bounded to ~150 s"},
+        "cpu_baseline": {"value": sps, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                         "sample": f"{reps} whole step(s) of {cfg['name']} in {el:.1f} s"},
+        "e2e": {"value": sps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=50)
-    ap.add_argument("--config", default="llama7b", choices=sorted(workloads.CONFIGS))
+    ap.add_argument("--config", default="llama7b",
+                    choices=sorted(workloads.CONFIGS) + sorted(workloads.LMHEAD_CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--attn-impl", default="tensor", choices=["tensor", "rows"],
                     help="tensor: keys on the MMA M extent (default); rows: query rows on M")
     args = ap.parse_args()
+    if args.config in workloads.LMHEAD_CONFIGS:
+        if args.steps == 20000:
+            args.steps = 4000
+        (run_lmhead_reference if args.impl == "reference" else run_lmhead)(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -3,25 +3,31 @@
 //
 // logits[r, x] = <h_r, W_x> for the (k+1)^2 block rows of every sequence and the
 // whole vocabulary, but the logits never reach memory: the product runs on the
-// tensor cores with the vocabulary on the MMA M extent (A = 128 rows of W,
-// K-major; B = all block rows of the batch, K-major; fp32 accumulators in TMEM),
-// and the epilogue reduces every accumulator column (= one block row) to
-// (max, lowest arg-max, sum exp(z - max)) over the thread block's vocabulary
-// range.  The last thread block to finish combines the ranges and runs the
-// acceptance scan, the extra token, the <EOS> cut and the next candidates.
+// tensor cores with the block rows on the MMA M extent (A = hidden rows, K-major)
+// and up to 256 tokens on the N extent (B = rows of W, K-major; fp32 accumulators
+// in TMEM: lane = block row, column = token).  An instruction of this kind costs
+// about the same whatever its N, so the tokens go on N: measured with the tokens
+// on M (128 per instruction) the 512 instructions of a thread block took longer
+// than its share of W takes to arrive.  Every epilogue thread owns one block row
+// and folds its accumulator columns into (max, lowest arg-max, sum exp(z - max))
+// in registers, without any exchange between threads.  The last thread block to
+// finish combines the vocabulary ranges and runs the acceptance scan, the extra
+// token, the <EOS> cut and the next candidates.
 //
 // The output embedding is streamed exactly once (the step's HBM roof); the
 // hidden rows are re-read from L2 by every thread block.
 //
 // Vocabulary ranges: thread block c owns rows [V*c/G, V*(c+1)/G) and covers them
-// with boxes of 128 rows; the last box is shifted back so that it ends at the
-// range's end (rows it shares with the previous box are masked in the epilogue),
-// so no box reads past the range and the only rows read twice come from L2.
+// with boxes of n_box rows (256, or the longest range rounded up to 16 when that
+// is shorter); the last box of a range is loaded through a second tensor map
+// whose box holds only the rows a range's tail can have, so a range reads at
+// most 15 rows of its neighbour.
 //
 // Warps: 0 TMA producer, 1 TMEM owner and MMA issuer, 2..5 epilogue (one TMEM
-// lane quarter each).  Two accumulators alternate between boxes so that the
-// epilogue of one box runs under the products of the next.  Every wait is
-// bounded; an expired wait sets SPACE_ST_TIMEOUT, the block drains and exits.
+// lane quarter each).  With at most 128 block rows two accumulators alternate
+// between boxes so that the epilogue of one box runs under the products of the
+// next.  Every wait is bounded; an expired wait sets SPACE_ST_TIMEOUT, the block
+// drains and exits.
 #include "common.cuh"
 #include <cuda.h>
 #include <math_constants.h>
@@ -29,10 +35,11 @@
 namespace {
 
 constexpr int LM_THREADS = 192;
-constexpr int LM_BOX = 128;                 // vocabulary rows per box (MMA M)
-constexpr int LM_KB = 64;                   // hidden elements per stage (128 bytes: one swizzle row)
-constexpr int LM_A_BYTES = LM_BOX * LM_KB * 2;
+constexpr int LM_M = 128;                   // block rows per accumulator (MMA M)
+constexpr int LM_MAX_BOX = 256;             // vocabulary rows per box (MMA N), at most
+constexpr int LM_KB = 64;                   // hidden elements per slice (128 bytes: one swizzle row)
 constexpr int LM_MAX_STAGES = 10;
+constexpr float LM_NEG = -3.0e38f;          // "no logit yet": finite, so that differences never give NaN
 constexpr int LM_MAX_N = 256;               // block rows of the whole batch, padded to 16
 constexpr uint64_t LM_WAIT_NS = 1000000000ull;
 constexpr float LOG2E = 1.4426950408889634f;
@@ -40,11 +47,15 @@ constexpr float LOG2E = 1.4426950408889634f;
 struct LmPartial { float m, s; int idx, pad; };   // 16 bytes
 
 struct LmParams {
-  CUtensorMap tm_w, tm_h;
+  CUtensorMap tm_w, tm_wt, tm_h;   // W in boxes of n_box rows, W in boxes of tail_rows rows, hidden rows
   int B, k, V, D, n_q;
   int n_rows;                 // B * n_q
-  int n_pad;                  // n_rows rounded up to 16: N of the MMAs
+  int n_pad;                  // n_rows rounded up to 16: rows of the hidden-state tile
+  int n_mt;                   // accumulators of 128 block rows (1 or 2)
   int stages;
+  int n_box;                  // rows of the first tensor map's box (N of its products)
+  int tail_rows;              // rows of the second tensor map's box
+  int kbs;                    // 64-element slices of the hidden dimension per stage
   int eos_id;
   const int32_t* cand;
   int32_t* n_accept; int32_t* out_tokens; int32_t* n_out; int32_t* next_cand;
@@ -80,11 +91,14 @@ __device__ __forceinline__ uint64_t global_ns() {
   return t;
 }
 // Bounded wait.  Returns false when the limit expired or another thread gave up.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err, int site) {
+// `backoff`: sleep between polls (the epilogue warps, which wait for a whole group of products).
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err, int site,
+                                       bool backoff = false) {
   if (*abort_flag) return mbar_try(bar, parity);
   uint64_t t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try(bar, parity)) return true;
+    if (backoff) __nanosleep(128);
     if ((it & 255u) == 255u) {
       if (*abort_flag) return false;
       const uint64_t now = global_ns();
@@ -139,7 +153,7 @@ __device__ __forceinline__ uint64_t smem_desc_k128(uint32_t addr) {
 }
 // Instruction descriptor: bf16 x bf16 -> f32, M = 128, N = n, both operands K-major.
 __device__ __forceinline__ uint32_t instr_desc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(LM_BOX >> 4) << 24);
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(LM_M >> 4) << 24);
 }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
   asm volatile(
@@ -155,6 +169,44 @@ __device__ __forceinline__ float fast_exp2(float x) {
 }
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
+// Statistics of a set of logits: (m, s, i) = (max, sum of exp(z - m), lowest arg-max);
+// the empty set is (LM_NEG, 0, INT_MAX).  fold: union of two sets.  One of the two
+// exponentials is exp(0), so a single ex2 serves.
+__device__ __forceinline__ void stat_fold(float& m, float& s, int& i, float m2, float s2, int i2) {
+  if (m2 > m || (m2 == m && i2 < i)) i = i2;
+  const float e = fast_exp2(-fabsf(m - m2) * LOG2E);
+  s = (m >= m2) ? fmaf(s2, e, s) : fmaf(s, e, s2);
+  m = fmaxf(m, m2);
+}
+
+// Fold 16 consecutive tokens x0 .. x0+15 (the first nv of them valid) into a row's statistics.
+__device__ __forceinline__ void fold16(float& m, float& s, int& idx, const uint32_t* v, int x0, int nv) {
+  float z[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) z[j] = (j < nv) ? __uint_as_float(v[j]) : LM_NEG;
+  float cm = z[0];
+#pragma unroll
+  for (int j = 1; j < 16; ++j) cm = fmaxf(cm, z[j]);
+  if (cm > m) {                                           // strictly larger: an earlier token keeps a tie
+    int at = 15;
+#pragma unroll
+    for (int j = 14; j >= 0; --j) at = (z[j] == cm) ? j : at;
+    idx = x0 + at;
+    s *= fast_exp2((m - cm) * LOG2E);
+    m = cm;
+  }
+  const float ms = -m * LOG2E;
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+  for (int j = 0; j < 16; j += 4) {
+    a0 += fast_exp2(fmaf(z[j], LOG2E, ms));
+    a1 += fast_exp2(fmaf(z[j + 1], LOG2E, ms));
+    a2 += fast_exp2(fmaf(z[j + 2], LOG2E, ms));
+    a3 += fast_exp2(fmaf(z[j + 3], LOG2E, ms));
+  }
+  s += (a0 + a1) + (a2 + a3);
+}
+
 // (max, lowest arg-max) over the warp, result in every lane
 __device__ __forceinline__ void warp_max_idx(float& m, int& idx) {
 #pragma unroll
@@ -169,30 +221,25 @@ __device__ __forceinline__ float warp_sum(float v) {
   for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
   return v;
 }
-// fold (m2, s2, i2) into (m, s, i): sums are relative to their own maximum
-__device__ __forceinline__ void stat_fold(float& m, float& s, int& i, float m2, float s2, int i2) {
-  if (m2 > m || (m2 == m && i2 < i)) i = i2;
-  const float mm = fmaxf(m, m2);
-  if (mm > -CUDART_INF_F) {
-    const float a = (m > -CUDART_INF_F) ? s * fast_exp2((m - mm) * LOG2E) : 0.f;
-    const float b = (m2 > -CUDART_INF_F) ? s2 * fast_exp2((m2 - mm) * LOG2E) : 0.f;
-    s = a + b;
-  }
-  m = mm;
-}
 
 // Shared-memory plan (dynamic, 1024-byte aligned base):
-//   [stages][A 16 KB] [stages][B n_pad*128] | barriers | running statistics [4][n_pad] x 3 | row results [n_pad] x 2
+//   [stages]{ [kbs] hidden tiles of n_pad*128 bytes, [kbs] W tiles of n_box*128 bytes } | pad |
+//   barriers | row results [n_pad] x 2 | misc
+// A product reads 128 rows from a hidden tile's address whatever n_pad is: the rows past the
+// tile are whatever follows in shared memory (the stage's W tiles, then `pad`) and only reach
+// accumulator lanes nobody reads.  `pad` keeps that read inside the allocation.
 struct LmSmem {
-  uint32_t a_off, b_off, bar_off, stat_off, row_off, misc_off, total;
-  int b_bytes;
-  __host__ __device__ LmSmem(int n_pad, int stages) {
-    b_bytes = n_pad * LM_KB * 2;
-    a_off = 0;
-    b_off = a_off + (uint32_t)stages * LM_A_BYTES;
-    bar_off = b_off + (uint32_t)stages * b_bytes;
-    stat_off = bar_off + 8u * (2 * LM_MAX_STAGES + 4);
-    row_off = stat_off + 4u * 3u * 4u * (uint32_t)n_pad;
+  uint32_t a_bytes, b_bytes, b_in_stage, stage_bytes, bar_off, row_off, misc_off, total;
+  __host__ __device__ LmSmem(int n_pad, int n_box, int stages, int kbs) {
+    a_bytes = (uint32_t)n_pad * LM_KB * 2;
+    b_bytes = (uint32_t)n_box * LM_KB * 2;
+    b_in_stage = (uint32_t)kbs * a_bytes;
+    stage_bytes = b_in_stage + (uint32_t)kbs * b_bytes;
+    const uint32_t reach = 16384u * (n_pad > LM_M ? 2u : 1u);            // bytes a product reads from a hidden tile
+    const uint32_t have = a_bytes + (uint32_t)kbs * b_bytes;             // bytes that follow the last hidden tile's start
+    const uint32_t pad = reach > have ? (reach - have + 1023u) / 1024u * 1024u : 0u;
+    bar_off = (uint32_t)stages * stage_bytes + pad;
+    row_off = bar_off + 8u * (2 * LM_MAX_STAGES + 4);
     misc_off = row_off + 2u * 4u * (uint32_t)n_pad;
     total = misc_off + 64u;
   }
@@ -201,15 +248,12 @@ struct LmSmem {
 __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __grid_constant__ LmParams p) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t sm_base = smem_u32(smem_raw);
-  const LmSmem L(p.n_pad, p.stages);
+  const LmSmem L(p.n_pad, p.n_box, p.stages, p.kbs);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int S = p.stages;
   const uint32_t bar0 = sm_base + L.bar_off;
 #define LBAR(i) (bar0 + 8u * (uint32_t)(i))
   const int B_FULL = 0, B_EMPTY = LM_MAX_STAGES, B_ACCFULL = 2 * LM_MAX_STAGES, B_ACCEMPTY = 2 * LM_MAX_STAGES + 2;
-  float* run_m = reinterpret_cast<float*>(smem_raw + L.stat_off);          // [4][n_pad]
-  float* run_s = run_m + 4 * p.n_pad;
-  int* run_i = reinterpret_cast<int*>(run_s + 4 * p.n_pad);
   float* row_s = reinterpret_cast<float*>(smem_raw + L.row_off);           // [n_pad]
   int* row_i = reinterpret_cast<int*>(row_s + p.n_pad);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_raw + L.misc_off);
@@ -218,7 +262,7 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
 
   pdl_launch_dependents();
   if (threadIdx.x == 0) {
-    *abort_flag = (sm_base & 1023u) ? 1 : 0;
+    *abort_flag = (sm_base & 1023u) ? 1 : 0;               // swizzled tiles need a 1024-byte aligned base
     for (int s = 0; s < S; ++s) { mbar_init(LBAR(B_FULL + s), 1); mbar_init(LBAR(B_EMPTY + s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(LBAR(B_ACCFULL + a), 1); mbar_init(LBAR(B_ACCEMPTY + a), 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -231,9 +275,9 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
   }
   if (warp == 0 && lane == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_w) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_wt) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_h) : "memory");
   }
-  for (int t = threadIdx.x; t < 4 * p.n_pad; t += LM_THREADS) { run_m[t] = -CUDART_INF_F; run_s[t] = 0.f; run_i[t] = 0x7FFFFFFF; }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -243,9 +287,10 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
   // this thread block's vocabulary range and its boxes
   const int G = gridDim.x, c = blockIdx.x;
   const int r0 = (int)(((long long)p.V * c) / G), r1 = (int)(((long long)p.V * (c + 1)) / G);
-  const int nb = (r1 - r0 + LM_BOX - 1) / LM_BOX;
+  const int nb = (r1 - r0 + p.n_box - 1) / p.n_box;
   const int KB = (p.D + LM_KB - 1) / LM_KB;
-  const uint32_t stage_tx = (uint32_t)(LM_A_BYTES + L.b_bytes);
+  const int kbs = p.kbs;
+  const int n_bufs = p.n_mt == 1 ? 2 : 1;                  // accumulator buffers of n_mt x 256 columns
 
   if (warp == 0) {
     // ================= producer ==============================================
@@ -253,14 +298,21 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
       uint32_t it = 0;
       bool ok = !*abort_flag;
       for (int box = 0; box < nb && ok; ++box) {
-        const int row0 = (box == nb - 1) ? r1 - LM_BOX : r0 + box * LM_BOX;   // may be negative: zero-filled
-        for (int kb = 0; kb < KB; ++kb, ++it) {
+        const int row0 = r0 + box * p.n_box;
+        const bool tail = r1 - row0 <= p.tail_rows;        // the remaining rows fit the small box
+        const CUtensorMap* tm = tail ? &p.tm_wt : &p.tm_w;
+        const uint32_t w_bytes = (uint32_t)(tail ? p.tail_rows : p.n_box) * LM_KB * 2;
+        for (int kb0 = 0; kb0 < KB; kb0 += kbs, ++it) {
           const int s = it % S;
+          const int nk = min(kbs, KB - kb0);
           if (it >= (uint32_t)S) ok = mbar_wait(LBAR(B_EMPTY + s), ((it / S) - 1) & 1, abort_flag, p.err, 1);
           if (!ok) break;
-          mbar_expect_tx(LBAR(B_FULL + s), stage_tx);
-          tma_load_4d(sm_base + L.a_off + s * LM_A_BYTES, &p.tm_w, LBAR(B_FULL + s), kb * LM_KB, row0, 0, 0);
-          tma_load_4d(sm_base + L.b_off + s * L.b_bytes, &p.tm_h, LBAR(B_FULL + s), kb * LM_KB, 0, 0, 0);
+          mbar_expect_tx(LBAR(B_FULL + s), (uint32_t)nk * (w_bytes + L.a_bytes));
+          const uint32_t st_base = sm_base + (uint32_t)s * L.stage_bytes;
+          for (int j = 0; j < nk; ++j)
+            tma_load_4d(st_base + L.b_in_stage + (uint32_t)j * L.b_bytes, tm, LBAR(B_FULL + s), (kb0 + j) * LM_KB, row0, 0, 0);
+          for (int j = 0; j < nk; ++j)
+            tma_load_4d(st_base + (uint32_t)j * L.a_bytes, &p.tm_h, LBAR(B_FULL + s), (kb0 + j) * LM_KB, 0, 0, 0);
         }
       }
       if (!ok) {
@@ -272,83 +324,91 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
   } else if (warp == 1) {
     // ================= MMA issuer =============================================
     if (lane == 0) {
-      const uint32_t idesc = instr_desc(p.n_pad);
-      const uint64_t adesc0 = smem_desc_k128(sm_base + L.a_off);
-      const uint64_t bdesc0 = smem_desc_k128(sm_base + L.b_off);
+      const uint64_t desc0 = smem_desc_k128(sm_base);
       uint32_t it = 0;
       bool ok = !*abort_flag;
       for (int box = 0; box < nb && ok; ++box) {
-        const int a = box & 1;
-        if (box >= 2) ok = mbar_wait(LBAR(B_ACCEMPTY + a), ((box >> 1) - 1) & 1, abort_flag, p.err, 2);
+        const int buf = box % n_bufs;
+        const int row0 = r0 + box * p.n_box;
+        const uint32_t idesc = instr_desc((r1 - row0 <= p.tail_rows) ? p.tail_rows : p.n_box);
+        if (box >= n_bufs) ok = mbar_wait(LBAR(B_ACCEMPTY + buf), ((box / n_bufs) - 1) & 1, abort_flag, p.err, 2);
         if (!ok) break;
         tc_fence_after();
-        for (int kb = 0; kb < KB; ++kb, ++it) {
+        for (int kb0 = 0; kb0 < KB; kb0 += kbs, ++it) {
           const int s = it % S;
+          const int nk = min(kbs, KB - kb0);
           ok = mbar_wait(LBAR(B_FULL + s), (it / S) & 1, abort_flag, p.err, 3);
           if (!ok) break;
           tc_fence_after();
-          const uint64_t ad = adesc0 + (uint64_t)((s * LM_A_BYTES) >> 4);
-          const uint64_t bd = bdesc0 + (uint64_t)((s * L.b_bytes) >> 4);
+          const uint32_t st_off = (uint32_t)s * L.stage_bytes;
+          for (int j = 0; j < nk; ++j) {
+            const uint64_t wd = desc0 + (uint64_t)((st_off + L.b_in_stage + (uint32_t)j * L.b_bytes) >> 4);
+            for (int mt = 0; mt < p.n_mt; ++mt) {
+              // block rows 128*mt .. of the hidden tile (8-row groups are contiguous: 16 KB further on)
+              const uint64_t hd = desc0 + (uint64_t)((st_off + (uint32_t)j * L.a_bytes + (uint32_t)mt * 16384u) >> 4);
+              const uint32_t acc = tmem + (uint32_t)((buf * p.n_mt + mt) * LM_MAX_BOX);
 #pragma unroll
-          for (int kk = 0; kk < LM_KB / 16; ++kk)          // 32 bytes per 16 elements inside the swizzled row
-            mma_ss(tmem + a * LM_MAX_N, ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 2), idesc, (kb | kk) ? 1u : 0u);
+              for (int kk = 0; kk < LM_KB / 16; ++kk)      // 32 bytes per 16 elements inside the swizzled row
+                mma_ss(acc, hd + (uint64_t)(kk * 2), wd + (uint64_t)(kk * 2), idesc, (kb0 | j | kk) ? 1u : 0u);
+            }
+          }
           tc_commit(LBAR(B_EMPTY + s));
         }
-        if (ok) tc_commit(LBAR(B_ACCFULL + a));
+        if (ok) tc_commit(LBAR(B_ACCFULL + buf));
       }
     }
   } else {
     // ================= epilogue ================================================
     const int quarter = warp & 3;                          // TMEM lanes 32*quarter .. +31
-    const int ew = warp - 2;                               // 0..3: row of the running statistics
+    const int ew = warp - 2;
+    const int row_a = quarter * 32 + lane;                 // this thread's block rows: row_a and row_a + 128
+    float m0 = LM_NEG, s0 = 0.f, m1 = LM_NEG, s1 = 0.f;
+    int i0 = 0x7FFFFFFF, i1 = 0x7FFFFFFF;
+    // a warp whose 32 lanes hold no block row only takes part in the hand-shakes
+    const bool warp_a = quarter * 32 < p.n_rows, warp_b = p.n_mt == 2 && LM_M + quarter * 32 < p.n_rows;
     bool ok = true;
     for (int box = 0; box < nb; ++box) {
-      const int a = box & 1;
-      ok = ok && mbar_wait(LBAR(B_ACCFULL + a), (box >> 1) & 1, abort_flag, p.err, 4);
+      const int buf = box % n_bufs;
+      ok = ok && mbar_wait(LBAR(B_ACCFULL + buf), (box / n_bufs) & 1, abort_flag, p.err, 4, true);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
-      const bool last_box = box == nb - 1;
-      const int row0 = last_box ? r1 - LM_BOX : r0 + box * LM_BOX;
-      const int own_lo = r0 + box * LM_BOX;                // rows below belong to the previous box (shifted last box)
-      const int x = row0 + quarter * 32 + lane;            // this lane's token
-      const bool valid = x >= own_lo && x < r1 && x >= 0;
-      for (int c0 = 0; c0 < p.n_rows; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * LM_MAX_N + c0), v);
-        tmem_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float z = valid ? __uint_as_float(v[j]) : -CUDART_INF_F;
-          float m = z; int idx = valid ? x : 0x7FFFFFFF;
-          warp_max_idx(m, idx);
-          const float e = (valid && m > -CUDART_INF_F) ? fast_exp2((z - m) * LOG2E) : 0.f;
-          const float sum = warp_sum(e);
-          if (lane == j && c0 + j < p.n_rows) {
-            const int col = ew * p.n_pad + c0 + j;
-            float rm = run_m[col], rs = run_s[col]; int ri = run_i[col];
-            stat_fold(rm, rs, ri, m, sum, idx);
-            run_m[col] = rm; run_s[col] = rs; run_i[col] = ri;
-          }
+      const int row0 = r0 + box * p.n_box;
+      const int n_valid = min(r1 - row0, (r1 - row0 <= p.tail_rows) ? p.tail_rows : p.n_box);
+      const uint32_t acc = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.n_mt * LM_MAX_BOX);
+      if (warp_a) {
+        for (int c0 = 0; c0 < n_valid; c0 += 16) {
+          uint32_t v[16];
+          tmem_ld16(acc + (uint32_t)c0, v);
+          tmem_wait_ld();
+          fold16(m0, s0, i0, v, row0 + c0, n_valid - c0);
         }
       }
-      // accumulator `a` may be overwritten by the products of box + 2
+      if (warp_b) {
+        for (int c0 = 0; c0 < n_valid; c0 += 16) {
+          uint32_t v[16];
+          tmem_ld16(acc + (uint32_t)(LM_MAX_BOX + c0), v);
+          tmem_wait_ld();
+          fold16(m1, s1, i1, v, row0 + c0, n_valid - c0);
+        }
+      }
+      // this accumulator buffer may be overwritten by the products of the next box that uses it
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(LBAR(B_ACCEMPTY + a));
+      if (lane == 0) mbar_arrive(LBAR(B_ACCEMPTY + buf));
     }
-    epi_sync();
-    const int et = threadIdx.x - 64;                       // 0..127
-    // combine the four lane quarters and publish this block's statistics
-    for (int col = et; col < p.n_rows; col += 128) {
-      float m = run_m[col], s = run_s[col]; int i = run_i[col];
-#pragma unroll
-      for (int w = 1; w < 4; ++w) stat_fold(m, s, i, run_m[w * p.n_pad + col], run_s[w * p.n_pad + col], run_i[w * p.n_pad + col]);
-      LmPartial out; out.m = m; out.s = s; out.idx = i; out.pad = 0;
-      *reinterpret_cast<int4*>(p.part + (size_t)col * G + c) = *reinterpret_cast<const int4*>(&out);
+    // publish this block's statistics of every block row
+    if (row_a < p.n_rows) {
+      LmPartial out; out.m = m0; out.s = s0; out.idx = i0; out.pad = 0;
+      *reinterpret_cast<int4*>(p.part + (size_t)row_a * G + c) = *reinterpret_cast<const int4*>(&out);
+    }
+    if (p.n_mt == 2 && LM_M + row_a < p.n_rows) {
+      LmPartial out; out.m = m1; out.s = s1; out.idx = i1; out.pad = 0;
+      *reinterpret_cast<int4*>(p.part + (size_t)(LM_M + row_a) * G + c) = *reinterpret_cast<const int4*>(&out);
     }
     __threadfence();
     epi_sync();
+    const int et = threadIdx.x - 64;                       // 0..127
     if (et == 0) {
       const int prev = atomicAdd(p.counter, 1);
       const int last = prev == G - 1;
@@ -360,7 +420,7 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
       __threadfence();
       // ---- last thread block: combine the ranges, one warp per block row at a time
       for (int col = ew; col < p.n_rows; col += 4) {
-        float m = -CUDART_INF_F, s = 0.f; int i = 0x7FFFFFFF;
+        float m = LM_NEG, s = 0.f; int i = 0x7FFFFFFF;
         const LmPartial* pc = p.part + (size_t)col * G;
         for (int g = lane; g < G; g += 32) {
           const int4 raw = __ldcg(reinterpret_cast<const int4*>(pc + g));
@@ -368,7 +428,7 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
         }
         float bm = m; int bi = i;
         warp_max_idx(bm, bi);
-        float sv = (m > -CUDART_INF_F) ? s * fast_exp2((m - bm) * LOG2E) : 0.f;
+        float sv = s * fast_exp2((m - bm) * LOG2E);
         sv = warp_sum(sv);
         if (lane == 0) {
           row_s[col] = sv; row_i[col] = bi;
@@ -461,12 +521,27 @@ int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_
   p.n_rows = p.B * p.n_q;
   p.n_pad = (p.n_rows + 15) / 16 * 16;
   if (p.n_pad > LM_MAX_N) return SPACE_E_UNSUPPORTED;
-  // stages: as many as fit beside the statistics, at most LM_MAX_STAGES
-  int stages = LM_MAX_STAGES;
+  p.n_mt = p.n_pad > LM_M ? 2 : 1;
+  int grid = ctx->sm_count;
+  const int max_useful = (a->vocab + 31) / 32;             // at least 32 tokens per thread block
+  if (grid > max_useful) grid = max_useful;
+  if (grid < 1) grid = 1;
+  const int max_len = (a->vocab + grid - 1) / grid;        // the longest vocabulary range
+  p.n_box = max_len >= LM_MAX_BOX ? LM_MAX_BOX : (max_len + 15) / 16 * 16;
+  p.tail_rows = (((max_len - 1) % p.n_box) + 1 + 15) / 16 * 16;
+  p.kbs = 2;                                               // measured 1..4 on V = 32000, D = 4096: within 3 %
+  // stages: as many as fit, at most LM_MAX_STAGES; one slice per stage when two leave no room for two stages
   const size_t budget = 220 * 1024;
-  while (stages > 2 && LmSmem(p.n_pad, stages).total + 1024 > budget) --stages;
+  int stages = 0;
+  for (; p.kbs >= 1; --p.kbs) {
+    stages = LM_MAX_STAGES;
+    while (stages > 1 && LmSmem(p.n_pad, p.n_box, stages, p.kbs).total + 1024 > budget) --stages;
+    if (stages >= 2) break;
+  }
+  if (stages < 2) return SPACE_E_UNSUPPORTED;
   p.stages = stages;
-  const LmSmem L(p.n_pad, stages);
+  const LmSmem L(p.n_pad, p.n_box, stages, p.kbs);
+  if (L.total + 1024 > 227 * 1024) return SPACE_E_UNSUPPORTED;
   p.eos_id = a->eos_id;
   p.cand = a->cand;
   p.n_accept = a->n_accept; p.out_tokens = a->out_tokens; p.n_out = a->n_out; p.next_cand = a->next_cand;
@@ -475,14 +550,11 @@ int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_
   p.part = reinterpret_cast<LmPartial*>(ctx->lm_part);
   p.counter = ctx->lm_counter;
   p.err = ctx->lm_counter + 1;
-  int rc = lm_make_map(&p.tm_w, a->weight, a->vocab, a->hidden_dim, a->weight_row_stride, LM_BOX);
+  int rc = lm_make_map(&p.tm_w, a->weight, a->vocab, a->hidden_dim, a->weight_row_stride, p.n_box);
+  if (rc == SPACE_OK) rc = lm_make_map(&p.tm_wt, a->weight, a->vocab, a->hidden_dim, a->weight_row_stride, p.tail_rows);
   if (rc == SPACE_OK) rc = lm_make_map(&p.tm_h, a->hidden, p.n_rows, a->hidden_dim, a->hidden_row_stride, p.n_pad);
   if (rc != SPACE_OK) return rc;
-  int grid = ctx->sm_count;
-  const int max_useful = (a->vocab + 31) / 32;             // at least 32 tokens per thread block
-  if (grid > max_useful) grid = max_useful;
-  if (grid < 1) grid = 1;
-  const size_t sm = L.total + 1024;                        // room to align the base to 1024 bytes
+  const size_t sm = L.total + 1024;
   cudaFuncSetAttribute(lmhead_verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
   {
     ProfScope ps(ctx, SPACE_K_LMHEAD, st);

@@ -99,12 +99,14 @@ def _compare(cfg, x, got, eos_id=-1, what=""):
 
 
 @pytest.mark.parametrize("V,D,k,Bn", [
-    (1000, 256, 4, 1),        # ranges shorter than one box: shifted, partly negative starts
+    (1000, 256, 4, 1),        # ranges shorter than 16 tokens
     (4736, 512, 5, 1),        # exactly 32 tokens per thread block
     (5000, 320, 3, 2),        # two sequences, ragged ranges
-    (40000, 192, 2, 3),       # three boxes per range, the last one shifted back
+    (40000, 192, 2, 3),       # two boxes per range: a full one and a tail
+    (130000, 128, 4, 2),      # four boxes per range, alternating accumulators
     (257, 72, 1, 4),          # tiny vocabulary (fewer thread blocks than SMs), D not a multiple of 64
-    (33000, 128, 7, 4),       # 256 block rows: the widest product
+    (33000, 128, 7, 4),       # 256 block rows: two accumulators of 128 rows, one buffer
+    (100000, 64, 5, 4),       # 144 block rows and three boxes per range
 ])
 def test_lmhead_small_shapes(H, V, D, k, Bn):
     cfg = workloads.resolve_lmhead("lmhead_tiny", V=V, D=D, k=k, B=Bn, p_accept=(0.5, 0.9))
