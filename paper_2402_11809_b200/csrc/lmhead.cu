@@ -62,6 +62,7 @@ struct LmParams {
   float* next_cand_prob; uint8_t* finished; int32_t* status;
   float* row_max; int32_t* row_argmax;
   LmPartial* part;            // [n_rows][gridDim.x]
+  unsigned long long* keys;   // [n_rows] arg-max keys, combined with atomicMax; zero between launches
   int* counter;               // arrival counter (self-resetting)
   int* err;
 };
@@ -177,6 +178,21 @@ __device__ __forceinline__ void stat_fold(float& m, float& s, int& i, float m2, 
   const float e = fast_exp2(-fabsf(m - m2) * LOG2E);
   s = (m >= m2) ? fmaf(s2, e, s) : fmaf(s, e, s2);
   m = fmaxf(m, m2);
+}
+
+// (maximum, lowest token) of a row as one 64-bit key whose unsigned order is "larger logit
+// first, then lower token": the ranges of all thread blocks combine with one atomicMax each.
+// 0 is below every key of a real logit.
+__device__ __forceinline__ unsigned long long argmax_key(float m, int idx) {
+  uint32_t u = __float_as_uint(m);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)idx);
+}
+__device__ __forceinline__ void argmax_unkey(unsigned long long key, float& m, int& idx) {
+  uint32_t u = (uint32_t)(key >> 32);
+  u = (u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u;
+  m = __uint_as_float(u);
+  idx = (int)(0xFFFFFFFFu - (uint32_t)key);
 }
 
 // Fold 16 consecutive tokens x0 .. x0+15 (the first nv of them valid) into a row's statistics.
@@ -401,10 +417,12 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
     if (row_a < p.n_rows) {
       LmPartial out; out.m = m0; out.s = s0; out.idx = i0; out.pad = 0;
       *reinterpret_cast<int4*>(p.part + (size_t)row_a * G + c) = *reinterpret_cast<const int4*>(&out);
+      atomicMax(p.keys + row_a, argmax_key(m0, i0));
     }
     if (p.n_mt == 2 && LM_M + row_a < p.n_rows) {
       LmPartial out; out.m = m1; out.s = s1; out.idx = i1; out.pad = 0;
       *reinterpret_cast<int4*>(p.part + (size_t)(LM_M + row_a) * G + c) = *reinterpret_cast<const int4*>(&out);
+      atomicMax(p.keys + LM_M + row_a, argmax_key(m1, i1));
     }
     __threadfence();
     epi_sync();
@@ -418,54 +436,77 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
     epi_sync();
     if (*last_flag) {
       __threadfence();
-      // ---- last thread block: combine the ranges, one warp per block row at a time
-      for (int col = ew; col < p.n_rows; col += 4) {
-        float m = LM_NEG, s = 0.f; int i = 0x7FFFFFFF;
-        const LmPartial* pc = p.part + (size_t)col * G;
-        for (int g = lane; g < G; g += 32) {
-          const int4 raw = __ldcg(reinterpret_cast<const int4*>(pc + g));
-          stat_fold(m, s, i, __int_as_float(raw.x), __int_as_float(raw.y), raw.z);
-        }
-        float bm = m; int bi = i;
-        warp_max_idx(bm, bi);
-        float sv = s * fast_exp2((m - bm) * LOG2E);
-        sv = warp_sum(sv);
-        if (lane == 0) {
-          row_s[col] = sv; row_i[col] = bi;
-          if (p.row_max) p.row_max[col] = bm;
-          if (p.row_argmax) p.row_argmax[col] = bi;
-        }
+      // ---- last thread block.  Every row's (maximum, arg-max) is already combined in its key;
+      // only the k mask rows of group i* of every sequence need their sums, so only those rows'
+      // per-range partials are read, all of them at once over the 128 threads.
+      const int k1 = p.k + 1;
+      float* row_m = row_s;                                // [n_rows] maxima (row_s is reused: sums come later)
+      int* istar = reinterpret_cast<int*>(smem_raw);       // [B] (the pipeline stages are idle now)
+      float* terms = reinterpret_cast<float*>(smem_raw) + LM_MAX_N;   // [B * k][G] scaled sums of the ranges
+      for (int r = et; r < p.n_rows; r += 128) {
+        const unsigned long long key = atomicExch(p.keys + r, 0ull);      // read, and ready for the next launch
+        float m; int idx;
+        argmax_unkey(key, m, idx);
+        row_m[r] = m; row_i[r] = idx;
+        if (p.row_max) p.row_max[r] = m;
+        if (p.row_argmax) p.row_argmax[r] = idx;
       }
       epi_sync();
-      // ---- acceptance scan, emitted tokens, next candidates: one warp per sequence
-      const int k1 = p.k + 1;
+      // acceptance scan and emitted tokens: one warp per sequence
       for (int b = ew; b < p.B; b += 4) {
         const int* ri = row_i + b * p.n_q;
-        const float* rs = row_s + b * p.n_q;
-        const int* cd = p.cand + b * p.k;
-        int i_star = 0, bits = 0;
-        for (int t = 0; t < p.k; ++t) {
-          const int cc = cd[t];
-          if (cc < 0 || cc >= p.V) bits |= SPACE_ST_BAD_CANDIDATE;
-        }
-        while (i_star < p.k && cd[i_star] >= 0 && cd[i_star] < p.V && cd[i_star] == ri[i_star * k1]) ++i_star;
+        const int cv = (lane < p.k) ? p.cand[b * p.k + lane] : -1;        // one load per lane
+        const bool in_range = cv >= 0 && cv < p.V;
+        const unsigned bad = __ballot_sync(0xFFFFFFFFu, lane < p.k && !in_range);
+        const bool match = lane < p.k && in_range && cv == ri[lane * k1];
+        const unsigned acc_mask = __ballot_sync(0xFFFFFFFFu, match);
+        const int i_star = __ffs(~acc_mask) - 1;            // first candidate that does not match (k when all do)
         const int j = lane;
-        const int tok = (j < i_star) ? cd[min(j, p.k - 1)] : (j == i_star ? ri[i_star * k1] : -1);
+        const int c_j = __shfl_sync(0xFFFFFFFFu, cv, min(j, p.k - 1));
+        const int tok = (j < i_star) ? c_j : (j == i_star ? ri[i_star * k1] : -1);
         const bool is_eos = p.eos_id >= 0 && j <= i_star && tok == p.eos_id;
         const unsigned eos_mask = __ballot_sync(0xFFFFFFFFu, is_eos && j < k1);
         const int n_out = eos_mask ? __ffs(eos_mask) - 1 : i_star + 1;
         if (j < k1) p.out_tokens[b * k1 + j] = (j < n_out) ? tok : -1;
-        if (j < p.k) {                                     // next candidate j+1 from mask row (i*, j+1)
-          const int mr = i_star * k1 + j + 1;
-          p.next_cand[b * p.k + j] = ri[mr];
-          p.next_cand_prob[b * p.k + j] = 1.f / rs[mr];    // softmax at T = 1 of its own maximum
-        }
+        if (j < p.k) p.next_cand[b * p.k + j] = ri[i_star * k1 + j + 1];  // mask row (i*, j+1)
         if (j == 0) {
+          istar[b] = i_star;
           p.n_accept[b] = i_star;
           p.n_out[b] = n_out;
           p.finished[b] = (uint8_t)(eos_mask != 0);
-          if (p.status && bits) atomicOr(p.status + b, bits);
+          if (p.status && bad) atomicOr(p.status + b, SPACE_ST_BAD_CANDIDATE);
         }
+      }
+      epi_sync();
+      // sums of the mask rows of group i*: (sequence, mask row, range) triples spread over the threads
+      const int total = p.B * p.k * G;
+      for (int i0 = et; i0 < total; i0 += 128 * 8) {
+        int4 v[8]; float mx[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int at = i0 + u * 128;
+          v[u] = make_int4(0, 0, 0, 0); mx[u] = 0.f;
+          if (at < total) {
+            const int g = at % G, bj = at / G;
+            const int b = bj / p.k, jj = bj - b * p.k;
+            const int row = b * p.n_q + istar[b] * k1 + jj + 1;
+            mx[u] = row_m[row];
+            v[u] = __ldcg(reinterpret_cast<const int4*>(p.part + (size_t)row * G + g));
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int at = i0 + u * 128;
+          if (at < total) terms[at] = __int_as_float(v[u].y) * fast_exp2((__int_as_float(v[u].x) - mx[u]) * LOG2E);
+        }
+      }
+      epi_sync();
+      // fixed summation order: the result does not depend on which block came last or on timing
+      for (int bj = ew; bj < p.B * p.k; bj += 4) {
+        float sv = 0.f;
+        for (int g = lane; g < G; g += 32) sv += terms[bj * G + g];
+        sv = warp_sum(sv);
+        if (lane == 0) p.next_cand_prob[bj] = 1.f / sv;    // softmax at T = 1 of its own maximum
       }
     }
   }
@@ -549,6 +590,7 @@ int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_
   p.row_max = a->row_max; p.row_argmax = a->row_argmax;
   p.part = reinterpret_cast<LmPartial*>(ctx->lm_part);
   p.counter = ctx->lm_counter;
+  p.keys = reinterpret_cast<unsigned long long*>(ctx->lm_counter + 64);
   p.err = ctx->lm_counter + 1;
   int rc = lm_make_map(&p.tm_w, a->weight, a->vocab, a->hidden_dim, a->weight_row_stride, p.n_box);
   if (rc == SPACE_OK) rc = lm_make_map(&p.tm_wt, a->weight, a->vocab, a->hidden_dim, a->weight_row_stride, p.tail_rows);

@@ -48,7 +48,7 @@ Carve carve(const space_config* c, int sm_count) {
   v.vrow = off; off += align_up((size_t)c->max_batch * (c->k_max + 1) * sizeof(VerifyRow), 256);
   v.status = off; off += align_up((size_t)c->max_batch * sizeof(int32_t), 256);
   v.lm_part = off; off += align_up(lmhead_partial_bytes(sm_count), 256);
-  v.lm_counter = off; off += 256;
+  v.lm_counter = off; off += 256 + 256 * sizeof(unsigned long long);   // counter, error word; one arg-max key per block row
   v.stage = off;
   if (c->host_staging) {
     const size_t n_q = (size_t)(c->k_max + 1) * (c->k_max + 1);
