@@ -570,14 +570,14 @@ int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_
   const int max_len = (a->vocab + grid - 1) / grid;        // the longest vocabulary range
   p.n_box = max_len >= LM_MAX_BOX ? LM_MAX_BOX : (max_len + 15) / 16 * 16;
   p.tail_rows = (((max_len - 1) % p.n_box) + 1 + 15) / 16 * 16;
-  p.kbs = 2;                                               // measured 1..4 on V = 32000, D = 4096: within 3 %
-  // stages: as many as fit, at most LM_MAX_STAGES; one slice per stage when two leave no room for two stages
+  // Slices per stage and stages: two slices when that leaves at least three stages (measured 1..4
+  // slices on V = 32000, D = 4096: within 3 %), else one; as many stages as fit, at most LM_MAX_STAGES.
   const size_t budget = 220 * 1024;
   int stages = 0;
-  for (; p.kbs >= 1; --p.kbs) {
+  for (p.kbs = 2; p.kbs >= 1; --p.kbs) {
     stages = LM_MAX_STAGES;
     while (stages > 1 && LmSmem(p.n_pad, p.n_box, stages, p.kbs).total + 1024 > budget) --stages;
-    if (stages >= 2) break;
+    if (stages >= (p.kbs == 2 ? 3 : 2)) break;
   }
   if (stages < 2) return SPACE_E_UNSUPPORTED;
   p.stages = stages;
