@@ -311,25 +311,32 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
   if (warp == 0) {
     // ================= producer ==============================================
     if (lane == 0) {
-      uint32_t it = 0;
+      const int ipb = (KB + kbs - 1) / kbs;                // stages per box
+      const uint32_t n_it = (uint32_t)(nb * ipb);
       bool ok = !*abort_flag;
-      for (int box = 0; box < nb && ok; ++box) {
+      // stage `it`: the W tiles and the hidden tiles of its slices
+      auto issue = [&](uint32_t it) {
+        const int box = (int)it / ipb, kb0 = ((int)it - box * ipb) * kbs;
+        const int s = it % S;
+        const int nk = min(kbs, KB - kb0);
         const int row0 = r0 + box * p.n_box;
         const bool tail = r1 - row0 <= p.tail_rows;        // the remaining rows fit the small box
+        const uint32_t st_base = sm_base + (uint32_t)s * L.stage_bytes;
         const CUtensorMap* tm = tail ? &p.tm_wt : &p.tm_w;
         const uint32_t w_bytes = (uint32_t)(tail ? p.tail_rows : p.n_box) * LM_KB * 2;
-        for (int kb0 = 0; kb0 < KB; kb0 += kbs, ++it) {
-          const int s = it % S;
-          const int nk = min(kbs, KB - kb0);
-          if (it >= (uint32_t)S) ok = mbar_wait(LBAR(B_EMPTY + s), ((it / S) - 1) & 1, abort_flag, p.err, 1);
-          if (!ok) break;
-          mbar_expect_tx(LBAR(B_FULL + s), (uint32_t)nk * (w_bytes + L.a_bytes));
-          const uint32_t st_base = sm_base + (uint32_t)s * L.stage_bytes;
-          for (int j = 0; j < nk; ++j)
-            tma_load_4d(st_base + L.b_in_stage + (uint32_t)j * L.b_bytes, tm, LBAR(B_FULL + s), (kb0 + j) * LM_KB, row0, 0, 0);
-          for (int j = 0; j < nk; ++j)
-            tma_load_4d(st_base + (uint32_t)j * L.a_bytes, &p.tm_h, LBAR(B_FULL + s), (kb0 + j) * LM_KB, 0, 0, 0);
-        }
+        mbar_expect_tx(LBAR(B_FULL + s), (uint32_t)nk * (w_bytes + L.a_bytes));
+        for (int j = 0; j < nk; ++j)
+          tma_load_4d(st_base + L.b_in_stage + (uint32_t)j * L.b_bytes, tm, LBAR(B_FULL + s), (kb0 + j) * LM_KB, row0, 0, 0);
+        for (int j = 0; j < nk; ++j)
+          tma_load_4d(st_base + (uint32_t)j * L.a_bytes, &p.tm_h, LBAR(B_FULL + s), (kb0 + j) * LM_KB, 0, 0, 0);
+      };
+      // (requesting the first stages' W tiles before the dependency wait, so that they stream under the
+      // previous kernel's tail, measured 0.8 us slower per step in graph replay and was left out)
+      uint32_t it = 0;
+      for (; it < n_it && ok; ++it) {
+        if (it >= (uint32_t)S) ok = mbar_wait(LBAR(B_EMPTY + it % S), ((it / S) - 1) & 1, abort_flag, p.err, 1);
+        if (!ok) break;
+        issue(it);
       }
       if (!ok) {
         // copies already requested still land: wait for them (bounded) before the block exits
