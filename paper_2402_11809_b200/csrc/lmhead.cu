@@ -240,12 +240,12 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // Shared-memory plan (dynamic, 1024-byte aligned base):
 //   [stages]{ [kbs] hidden tiles of n_pad*128 bytes, [kbs] W tiles of n_box*128 bytes } | pad |
-//   barriers | row results [n_pad] x 2 | misc
+//   barriers | row results [n_pad] x 2 | candidates | misc
 // A product reads 128 rows from a hidden tile's address whatever n_pad is: the rows past the
 // tile are whatever follows in shared memory (the stage's W tiles, then `pad`) and only reach
 // accumulator lanes nobody reads.  `pad` keeps that read inside the allocation.
 struct LmSmem {
-  uint32_t a_bytes, b_bytes, b_in_stage, stage_bytes, bar_off, row_off, misc_off, total;
+  uint32_t a_bytes, b_bytes, b_in_stage, stage_bytes, bar_off, row_off, cand_off, misc_off, total;
   __host__ __device__ LmSmem(int n_pad, int n_box, int stages, int kbs) {
     a_bytes = (uint32_t)n_pad * LM_KB * 2;
     b_bytes = (uint32_t)n_box * LM_KB * 2;
@@ -256,7 +256,8 @@ struct LmSmem {
     const uint32_t pad = reach > have ? (reach - have + 1023u) / 1024u * 1024u : 0u;
     bar_off = (uint32_t)stages * stage_bytes + pad;
     row_off = bar_off + 8u * (2 * LM_MAX_STAGES + 4);
-    misc_off = row_off + 2u * 4u * (uint32_t)n_pad;
+    cand_off = row_off + 2u * 4u * (uint32_t)n_pad;                      // candidates of the batch: fewer than n_pad
+    misc_off = cand_off + 4u * (uint32_t)n_pad;
     total = misc_off + 64u;
   }
 };
@@ -272,6 +273,7 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
   const int B_FULL = 0, B_EMPTY = LM_MAX_STAGES, B_ACCFULL = 2 * LM_MAX_STAGES, B_ACCEMPTY = 2 * LM_MAX_STAGES + 2;
   float* row_s = reinterpret_cast<float*>(smem_raw + L.row_off);           // [n_pad]
   int* row_i = reinterpret_cast<int*>(row_s + p.n_pad);
+  int* cand_s = reinterpret_cast<int*>(smem_raw + L.cand_off);            // [B * k]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_raw + L.misc_off);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + L.misc_off + 4);
   int* last_flag = reinterpret_cast<int*>(smem_raw + L.misc_off + 8);
@@ -385,6 +387,8 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
     const int quarter = warp & 3;                          // TMEM lanes 32*quarter .. +31
     const int ew = warp - 2;
     const int row_a = quarter * 32 + lane;                 // this thread's block rows: row_a and row_a + 128
+    // the candidates are an input: fetched now, so that the last block's scan does not wait for them
+    for (int t = threadIdx.x - 64; t < p.B * p.k; t += 128) cand_s[t] = p.cand[t];
     float m0 = LM_NEG, s0 = 0.f, m1 = LM_NEG, s1 = 0.f;
     int i0 = 0x7FFFFFFF, i1 = 0x7FFFFFFF;
     // a warp whose 32 lanes hold no block row only takes part in the hand-shakes
@@ -462,7 +466,7 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
       // acceptance scan and emitted tokens: one warp per sequence
       for (int b = ew; b < p.B; b += 4) {
         const int* ri = row_i + b * p.n_q;
-        const int cv = (lane < p.k) ? p.cand[b * p.k + lane] : -1;        // one load per lane
+        const int cv = (lane < p.k) ? cand_s[b * p.k + lane] : -1;
         const bool in_range = cv >= 0 && cv < p.V;
         const unsigned bad = __ballot_sync(0xFFFFFFFFu, lane < p.k && !in_range);
         const bool match = lane < p.k && in_range && cv == ri[lane * k1];
