@@ -113,3 +113,15 @@ def test_reference_arm_runs_on_rank_zero_only():
     assert line["impl"] == "reference" and line["n_gpus"] == 2
     assert line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+
+
+def test_projection_reference_arm_runs_on_rank_zero_only():
+    argv = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "lmhead_tiny",
+            "--gpus", "2", "--steps", "2", "--warmup", "1"]
+    (rc0, o0, e0), (rc1, o1, e1) = spawn(argv, 2)
+    assert rc0 == 0, e0[-2000:]
+    assert rc1 == 0, e1[-2000:]
+    assert o1.strip() == ""
+    line = json.loads(o0.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["config"]["workload"] == "lmhead_tiny"
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
