@@ -134,6 +134,7 @@ LMHEAD_CONFIGS = {
     "lmhead_tiny": dict(B=1, k=4, V=1000, D=256, sigma=2.0, p_accept=(0.7, 0.7), seed=10),
     "lmhead_llama7b": dict(B=1, k=5, V=32000, D=4096, sigma=3.0, p_accept=(0.8, 0.8), seed=11),
     "lmhead_batch4": dict(B=4, k=5, V=32000, D=4096, sigma=3.0, p_accept=(0.3, 0.9), seed=12),
+    "lmhead_vocab128k": dict(B=1, k=4, V=128256, D=4096, sigma=3.0, p_accept=(0.8, 0.8), seed=13),
 }
 
 

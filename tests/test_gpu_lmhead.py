@@ -188,7 +188,7 @@ def test_lmhead_repeated_calls_and_argument_checks(H):
     big.close()
 
 
-@pytest.mark.parametrize("name", ["lmhead_llama7b", "lmhead_batch4"])
+@pytest.mark.parametrize("name", ["lmhead_llama7b", "lmhead_batch4", "lmhead_vocab128k"])
 def test_lmhead_full_size(H, name):
     cfg = workloads.resolve_lmhead(name)
     x = workloads.make_lmhead_inputs(cfg)
