@@ -38,8 +38,8 @@ L2_BYTES = 126 * 1024 * 1024
 # profiles/attn_tc_kernel_llama7b.txt and profiles/attn_rows_kernel_gqa70b.txt (bytes); None for workloads
 # without a capture of the current kernel
 ATTN_TRAFFIC = {"llama7b": 34518272, "gqa70b": 293366272}
-# the same for the projection kernel (profiles/lmhead_verify_kernel_lmhead_llama7b.txt, mean of two launches)
-LMHEAD_TRAFFIC = {"lmhead_llama7b": 266427264}
+# the same for the projection kernel (profiles/lmhead_verify_kernel_lmhead_*.txt, mean of two launches)
+LMHEAD_TRAFFIC = {"lmhead_llama7b": 266427264, "lmhead_vocab128k": 1071626000}
 METRIC = "auto-correct steps/sec"
 UNIT = "steps/s"
 
