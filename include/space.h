@@ -15,6 +15,8 @@
  *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *    stream).  All entry points except space_step_host are asynchronous and
  *    perform no allocation and no synchronisation after space_create.
+ *  - Every entry point that takes a context makes the context's device the
+ *    calling thread's current device (cudaSetDevice) and leaves it current.
  *  - Return value: SPACE_OK or a negative SPACE_E_* code; nothing aborts.
  *    Conditions only the GPU can see are reported per sequence in the
  *    `status` array (bit set of SPACE_ST_*).
@@ -118,7 +120,14 @@ typedef struct {
   const void*     logits;      /* device [B, n_q, V]; row stride below         */
   int64_t         logits_row_stride;   /* elements between rows; batch stride = n_q * row stride */
   const int32_t*  cand;        /* device [B, k]  L_c                           */
-  const float*    cand_prob;   /* device [B, k]  P_c (+inf allowed)            */
+  const float*    cand_prob;   /* device [B, k]  P_c: probability the candidate was drafted with
+                                  (sampling mode; ignored in greedy mode).  +inf is Algorithm 1's
+                                  initial state and is always rejected; a candidate is accepted only
+                                  if its id is in range, P_c > 0 and r * P_c <= Q(c) (NaN, zero and
+                                  negative values are rejected).  With SPACE_RESAMPLE_RESIDUAL_POINTMASS
+                                  a rejected candidate is removed from the extra token's distribution
+                                  only when its P_c is exactly 1 (a point-mass draft); after the
+                                  rejection of any other P_c the extra token is drawn from Q itself */
   const uint32_t* seq_id;      /* device [B] or NULL (= batch index)           */
   const int32_t*  kv_len;      /* device [B]: positions for the random counters */
   int32_t* n_accept;           /* device [B]       i*                          */
@@ -224,6 +233,22 @@ int space_attn_step(space_ctx* ctx, const space_attn_args* args, void* stream);
 /* Algorithm 1 verification loop, extra token and next candidates. */
 int space_verify(space_ctx* ctx, const space_verify_args* args, void* stream);
 
+/* space_verify followed by space_kv_commit with one kernel launch less: the
+ * verification kernels also move the accepted cache rows (Algorithm 1's loop
+ * body after the model call, then the compaction any cached forward needs).
+ * Results are those of the two separate calls, with one freedom: cache rows
+ * L+i*+1 .. L+k, which lie beyond the new length and held mask-token rows of
+ * the step's block that nothing reads again, are left with unspecified block
+ * rows (the single-launch greedy path moves all k candidate rows while the
+ * logits still stream, before i* is known).  Rows below the new length and
+ * rows from L+k+1 on are exactly as space_kv_commit leaves them.
+ * commit->n_accept must be
+ * verify->n_accept, and batch and k must agree (INVALID_ARG otherwise); every
+ * other rule of the two calls applies.  The attention that reads the cache rows
+ * of this step must have been enqueued on `stream` before this call. */
+int space_verify_commit(space_ctx* ctx, const space_verify_args* verify, const space_commit_args* commit,
+                        void* stream);
+
 /* Greedy verification without any allocation.  (The paper has no counterpart:
  * this entry point exists for how the library is embedded, not for the method.)
  *
@@ -242,11 +267,17 @@ int space_verify(space_ctx* ctx, const space_verify_args* args, void* stream);
  * (args->mode must be SPACE_MODE_GREEDY; temperature, seed, resample ignored);
  * all (k+1)^2 logits rows are read in one kernel.  Runs on the current device.
  * Limits: batch <= SPACE_NOALLOC_MAX_BATCH, else SPACE_E_STATIC_LIMIT; k in
- * 1..SPACE_MAX_K.  The first call on a device looks up the array's device
- * address (cudaGetSymbolAddress); make that first call outside any stream
- * capture.  All calls share the one array: the counters are cleared at the start
- * of every call, and two calls whose kernels overlap on the GPU (different
- * streams, or several host threads) race on it - serialise them. */
+ * 1..SPACE_MAX_K.
+ * The first call on a device is a set-up call: it looks up the array's device
+ * address (cudaGetSymbolAddress) and makes the CUDA runtime load the library's
+ * device code, which is when the array and the kernels take their (fixed) share
+ * of device memory.  Make that call once at start-up as a warm-up - before the
+ * host's own pool takes the rest of the memory, and outside any stream capture.
+ * Later calls on that device load nothing and reserve nothing.
+ * All calls share the one array, which keeps the last call's contents: the
+ * arrival counters are cleared at the start of every call, and two calls whose
+ * kernels overlap on the GPU (different streams, or several host threads) race
+ * on it - serialise them. */
 #define SPACE_NOALLOC_MAX_BATCH 8
 int space_verify_greedy_noalloc(const space_verify_args* args, void* stream);
 

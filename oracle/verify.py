@@ -24,6 +24,15 @@ resample:
         mask row and carry P_c = 1 (a point-mass draft).  c_i is accepted with
         probability Q(c_i); after a rejection the extra token is drawn from Q
         with the rejected token removed (the residual of a point mass).
+        The removal applies only to a candidate that really is a point mass
+        (P_c = 1).  Algorithm 1 starts from L_c = [0]*k, P_c = [+inf]*k: such a
+        candidate is rejected with certainty, its rejection says nothing about
+        the token, and the extra token is drawn from Q unchanged (so token 0
+        can be emitted at the first step).  Any other P_c is not a point-mass
+        draft either and is treated the same way (a ~ Q, Algorithm 1 as printed).
+An acceptance needs an in-range candidate and P_c > 0 (a drafted token cannot
+have had probability zero; this also keeps NaN and negative values from passing
+the test r*P_c <= Q by accident).
   "paper_literal"       Algorithm 1 as printed: a ~ Q also after a rejection,
         new candidates are sampled from their mask rows and P_c is the sampled
         token's probability.
@@ -117,7 +126,7 @@ def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed
             r = accept_uniform(seed, seq_id, L + i)
             with np.errstate(invalid="ignore"):
                 lhs = r * P_c[:, i - 1]                      # r <= Q/P_c  <=>  r*P_c <= Q
-                ok = lhs <= Q_ci
+                ok = in_range[:, i - 1] & (P_c[:, i - 1] > 0) & (lhs <= Q_ci)
                 marg = np.abs(lhs - Q_ci) / np.maximum(Q_ci, 1e-300)
             accept_margin[:, i - 1] = np.where(alive & np.isfinite(lhs), marg, np.inf)
         alive = alive & ok
@@ -133,6 +142,7 @@ def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed
             rej = i_star < k
             c_rej = c_safe[bi, np.minimum(i_star, k - 1)]
             rej = rej & in_range[bi, np.minimum(i_star, k - 1)]
+            rej = rej & (P_c[bi, np.minimum(i_star, k - 1)] == 1.0)   # a point-mass draft only
             w[bi[rej], c_rej[rej]] = 0.0
         with np.errstate(divide="ignore"):
             score = np.log(w) + gumbel_noise(seed, PURPOSE_TOKEN, seq_id, L + i_star + 1, V)

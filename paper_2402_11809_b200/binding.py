@@ -25,7 +25,8 @@ ATTN_TENSOR, ATTN_SIMT, ATTN_TENSOR_ROWS = 0, 1, 2
 ST_CAPACITY, ST_BAD_CANDIDATE, ST_TIMEOUT = 1, 2, 4
 
 EXPORTS = ["space_create", "space_destroy", "space_workspace_bytes", "space_layout",
-           "space_attn_step", "space_verify", "space_verify_greedy_noalloc", "space_kv_commit",
+           "space_attn_step", "space_verify", "space_verify_commit", "space_verify_greedy_noalloc",
+           "space_kv_commit",
            "space_lmhead_verify",
            "space_step_host",
            "space_launch_count", "space_profile_enable", "space_profile_read",
@@ -117,6 +118,8 @@ for _name, _arg in (("space_attn_step", AttnArgs), ("space_verify", VerifyArgs),
                     ("space_lmhead_verify", LmHeadArgs)):
     getattr(lib, _name).argtypes = [C.c_void_p, C.POINTER(_arg), C.c_void_p]
     getattr(lib, _name).restype = C.c_int
+lib.space_verify_commit.argtypes = [C.c_void_p, C.POINTER(VerifyArgs), C.POINTER(CommitArgs), C.c_void_p]
+lib.space_verify_commit.restype = C.c_int
 lib.space_verify_greedy_noalloc.argtypes = [C.POINTER(VerifyArgs), C.c_void_p]
 lib.space_verify_greedy_noalloc.restype = C.c_int
 lib.space_launch_count.argtypes = [C.c_void_p]
@@ -242,6 +245,10 @@ class Context:
 
     def space_verify(self, args):
         _check(lib.space_verify(self._h, C.byref(args), _stream()))
+
+    def space_verify_commit(self, vargs, cargs):
+        """space_verify + space_kv_commit in one launch less (see include/space.h)."""
+        _check(lib.space_verify_commit(self._h, C.byref(vargs), C.byref(cargs), _stream()))
 
     # -- space_lmhead_verify ----------------------------------------------
     def lmhead_args(self, hidden, weight, cand, n_accept, out_tokens, n_out, next_cand, next_cand_prob,

@@ -61,7 +61,18 @@ struct AttnParams {
   uint64_t mask_t[SPACE_MAX_ROWS];     // transposed: bit i of mask_t[j]
 };
 
-struct Seg { int b, h, t0, t1, T, L, slot, dfirst, dn; };   // slot: partial slot; dfirst/dn: cut (aligned mode)
+struct Seg { int b, h, t0, t1, T, L, slot, dfirst, dn; };
+
+// Optional per-block timeline (compiled in with -DSPACE_TIMELINE): one %globaltimer stamp
+// per named point and thread block, read back with space_debug_timeline_read.
+#ifdef SPACE_TIMELINE
+#define TL_POINTS 16
+__device__ unsigned long long g_timeline[256 * TL_POINTS];
+#define TL(i) do { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); \
+                   g_timeline[blockIdx.x * TL_POINTS + (i)] = t_; } while (0)
+#else
+#define TL(i) do { } while (0)
+#endif   // slot: partial slot; dfirst/dn: cut (aligned mode)
 
 // ---------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -420,6 +431,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
 
   // ---- set-up ------------------------------------------------------------
   pdl_launch_dependents();
+  if (threadIdx.x == 0) TL(0);
   if (threadIdx.x == 0) {
     *abort_flag = (sm_base & 1023u) ? 1 : 0;               // swizzled tiles need a 1024-byte aligned base
     for (int i = 0; i < 2; ++i) { mbar_init(BAR(B_QFULL + i), 1); mbar_init(BAR(B_QEMPTY + i), 1); }
@@ -451,7 +463,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (threadIdx.x == 0) TL(1);
   pdl_wait();                                              // global memory from here on
+  if (threadIdx.x == 0) TL(2);
   const bool single = p.B == 1;
   if (single) {
     // One sequence (the usual decoding case): the tables have a closed form, so every
@@ -582,6 +596,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           const uint32_t qb = seg % S::Q_BUFS, use = seg / S::Q_BUFS;
           if (use > 0) ok = mbar_wait(BAR(B_QEMPTY + qb), (use - 1) & 1, abort_flag, p.err, 3);
           if (!ok) break;
+          if (seg == 0) TL(3);
           mbar_expect_tx(BAR(B_QFULL + qb), q_bytes);
 #pragma unroll
           for (int hf = 0; hf < S::HALVES; ++hf)
@@ -607,6 +622,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
 #pragma unroll
           for (int hf = 0; hf < S::HALVES; ++hf)
             tma_load_4d(dst + hf * (TILE_N * 128), tm, BAR(b_full + s), hf * 64, kt, sg.h, sg.b);
+          if (is_k) TL(7);
         }
       }
       // drain: every issued copy must have landed before the block may exit
@@ -635,6 +651,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         for (int j = 0; j < n && ok; ++j, ++gt) {
           const int s = gt % S::K_STAGES, buf = gt & 1;
           ok = mbar_wait(BAR(B_KFULL + s), (gt / S::K_STAGES) & 1, abort_flag, p.err, 7);
+          if (gt == 0) TL(4);
           // S^T buffer `buf` was last read by the softmax of tile gt-2
           if (ok && gt >= 2) ok = mbar_wait(BAR(B_PREADY + buf), ((gt - 2) >> 1) & 1, abort_flag, p.err, 8);
           if (!ok) break;
@@ -732,6 +749,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         const bool first = (t == sg.t0);
         ok &= mbar_wait(BAR(B_SFULL + buf), (gt >> 1) & 1, abort_flag, p.err, 9);
         tc_fence_after();
+        if (sidx == 0) { if (gt == 0) TL(5); TL(8); }
         const uint32_t ts = TM_S0 + buf * 128 + lane_addr + col0;
         // this key's scores for its columns, all loads in flight together
 #pragma unroll
@@ -878,6 +896,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core
         tc_fence_before();
         mbar_arrive(BAR(B_PREADY + buf));
+        if (sidx == 0) { if (gt == 0) TL(6); TL(9); }
       }
       // ---- end of share: final output or partial ---------------------------
       // Row sums first, while the last O^T product still runs.  Every thread holds
@@ -914,6 +933,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       ok &= mbar_wait(BAR(B_PVDONE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1, abort_flag, p.err, 12);
       tc_fence_after();
       soft_sync();
+      if (sidx == 0) TL(10);
       const bool whole = (sg.t0 == 0 && sg.t1 == sg.T);
       const int item = sg.b * p.H_kv + sg.h;
       float* pslot = p.part + ((size_t)sg.slot * p.n_mblocks + mb) * (ROWS * (DH + 2));
@@ -993,6 +1013,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       }
       tc_fence_before();
       soft_sync();                                          // scratch, fq and mref are reused by the next share
+      if (sidx == 0) TL(11);
     }
     if (sidx == 0) p.owner[blockIdx.x] = own;
   }
@@ -1000,6 +1021,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   // ---- teardown -----------------------------------------------------------
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) TL(12);
   if (warp == WARP_MMA) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
@@ -1007,6 +1029,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   if (threadIdx.x == 0 && *abort_flag && p.status) {
     for (int b = 0; b < p.B; ++b) atomicOr(p.status + b, SPACE_ST_TIMEOUT);
   }
+  if (threadIdx.x == 32) TL(13);                          // after the TMEM release
 }
 
 // Combine the partials of every (sequence, kv head, query-row block) that was
@@ -1154,6 +1177,12 @@ size_t attn_tensor_partial_floats(const space_config* cfg, int sm_count, size_t*
   if (slots_out) *slots_out = slots;
   return slots * (size_t)ROWS * (cfg->head_dim + 2);
 }
+
+#ifdef SPACE_TIMELINE
+extern "C" int space_debug_timeline_read(unsigned long long* host_dst, int n_blocks) {
+  return cuda_ok(cudaMemcpyFromSymbol(host_dst, g_timeline, sizeof(unsigned long long) * TL_POINTS * n_blocks));
+}
+#endif
 
 int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t* mask_rows,
                        cudaStream_t st) {

@@ -91,8 +91,73 @@ struct space_ctx {
   alignas(64) unsigned char tm_v[128];
 };
 
+// ---- KV commit: shared by kv_commit_kernel and the verify kernels that carry the commit ----
+// Rows L + g(k+1) -> L + g, g = 1..i*, of K and V for every kv head (16-byte pieces).
+struct CommitParams {
+  int B, k, H_kv, d, blocks_per_seq, in_place;
+  int64_t s_cap;
+  __nv_bfloat16* kc; __nv_bfloat16* vc;
+  int64_t sb, sh, ss;
+  const int32_t* n_accept; const int32_t* kv_len;
+  int32_t* kv_len_out; int32_t* src; int32_t* dst; int32_t* status;
+  int* counter;
+};
+
+__device__ __forceinline__ bool commit_fits(const CommitParams& p, int L) {
+  return L >= 0 && (int64_t)L + (int64_t)(p.k + 1) * (p.k + 1) <= p.s_cap;
+}
+
+// Slice `part` of `nparts` of sequence b's move, by `nthreads` threads (this one is `tid`).
+// All loads of a batch are issued before its stores.
+__device__ __forceinline__ void commit_rows(const CommitParams& p, int b, int L, int i_star, int part, int nparts,
+                                            int tid, int nthreads) {
+  const int k1 = p.k + 1;
+  const int vec_per_row = p.d / 8;                      // 16-byte pieces per row
+  const int total = i_star * p.H_kv * 2 * vec_per_row;
+  const int stride = nparts * nthreads;
+  constexpr int U = 8;
+  for (int t0 = part * nthreads + tid; t0 < total; t0 += U * stride) {
+    uint4 val[U];
+    uint4* dd[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int t = t0 + u * stride;
+      dd[u] = nullptr;
+      if (t < total) {
+        int r = t;
+        const int v = r % vec_per_row; r /= vec_per_row;
+        const int which = r % 2;       r /= 2;
+        const int h = r % p.H_kv;      r /= p.H_kv;
+        const int g = r + 1;                            // accepted candidate g = 1..i*
+        __nv_bfloat16* base = (which ? p.vc : p.kc) + (int64_t)b * p.sb + (int64_t)h * p.sh;
+        val[u] = *(reinterpret_cast<const uint4*>(base + (int64_t)(L + g * k1) * p.ss) + v);
+        dd[u] = reinterpret_cast<uint4*>(base + (int64_t)(L + g) * p.ss) + v;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (dd[u]) *dd[u] = val[u];
+  }
+}
+
+// New length and index tables of sequence b (one thread).
+__device__ __forceinline__ void commit_tables(const CommitParams& p, int b, int L, int i_star, bool fits) {
+  const int k1 = p.k + 1;
+  if (!fits) {
+    if (p.status) atomicOr(p.status + b, SPACE_ST_CAPACITY);
+    i_star = -1;                                        // nothing committed, length unchanged
+  }
+  if (p.kv_len_out) p.kv_len_out[b] = L + i_star + 1;
+  for (int g = 0; g < k1; ++g) {
+    if (p.src) p.src[b * k1 + g] = (g <= i_star) ? L + g * k1 : -1;
+    if (p.dst) p.dst[b * k1 + g] = (g <= i_star) ? L + g : -1;
+  }
+}
+
 // ---- per-stage launchers (defined next to their kernels) -------------------
-int launch_verify(space_ctx* ctx, const space_verify_args* a, cudaStream_t st);
+// cm != nullptr: the verify kernels also carry out the commit described by cm (one launch less)
+int launch_verify(space_ctx* ctx, const space_verify_args* a, const space_commit_args* cm, cudaStream_t st);
+void fill_commit_params(const space_ctx* ctx, const space_commit_args* a, CommitParams* p);
 int launch_verify_noalloc(const space_verify_args* a, cudaStream_t st);
 int launch_commit(space_ctx* ctx, const space_commit_args* a, cudaStream_t st);
 int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_t st);

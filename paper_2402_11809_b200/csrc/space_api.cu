@@ -44,7 +44,8 @@ Carve carve(const space_config* c, int sm_count) {
   off += align_up((size_t)c->max_batch * c->n_kv_heads * 8 * sizeof(int2) + (size_t)(sm_count + 8) * sizeof(int), 256);
   v.vpart = off;
   off += align_up((size_t)c->max_batch * (c->k_max + 2) * SPACE_VERIFY_MAX_CHUNKS * sizeof(VerifyPartial), 256);
-  v.vfused = off; off += align_up((size_t)c->max_batch * SPACE_MAX_ROWS * 16 * sizeof(VerifyPartial), 256);
+  static_assert(SPACE_FUSED_MAX_CHUNKS <= 16, "the single-launch verify reduces a row's chunks with 16 lanes");
+  v.vfused = off; off += align_up((size_t)c->max_batch * SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS * sizeof(VerifyPartial), 256);
   v.vrow = off; off += align_up((size_t)c->max_batch * (c->k_max + 1) * sizeof(VerifyRow), 256);
   v.status = off; off += align_up((size_t)c->max_batch * sizeof(int32_t), 256);
   v.lm_part = off; off += align_up(lmhead_partial_bytes(sm_count), 256);
@@ -98,6 +99,39 @@ void build_layout(int k, int variant, space_layout_t* out) {
     out->relpos[i] = __builtin_popcountll(m) - 1;      // Sec. 3.2: visible keys - 1, relative to L
   }
   for (int t = 0; t <= k; ++t) out->target_rows[t] = t * k1;
+}
+
+// Every entry point that takes a context makes the context's device current.
+bool use_device(const space_ctx* ctx) { return cudaSetDevice(ctx->cfg.device) == cudaSuccess; }
+
+int check_verify_args(const space_ctx* ctx, const space_verify_args* a) {
+  if (a->batch < 0 || a->batch > ctx->cfg.max_batch) return SPACE_E_WORKSPACE;
+  if (a->k < 1 || a->k > ctx->cfg.k_max) return SPACE_E_INVALID_ARG;
+  if (a->vocab < 1 || a->vocab > ctx->cfg.vocab) return SPACE_E_WORKSPACE;
+  if (a->batch == 0) return SPACE_OK;
+  if (!a->logits || !a->cand || !a->cand_prob || !a->n_accept || !a->out_tokens || !a->n_out ||
+      !a->next_cand || !a->next_cand_prob || !a->finished)
+    return SPACE_E_INVALID_ARG;
+  if (a->logits_dtype != SPACE_DTYPE_F32 && a->logits_dtype != SPACE_DTYPE_BF16) return SPACE_E_INVALID_ARG;
+  if (a->mode != SPACE_MODE_GREEDY && a->mode != SPACE_MODE_SAMPLE) return SPACE_E_INVALID_ARG;
+  if (a->resample != SPACE_RESAMPLE_RESIDUAL_POINTMASS && a->resample != SPACE_RESAMPLE_PAPER_LITERAL)
+    return SPACE_E_INVALID_ARG;
+  if (a->mode == SPACE_MODE_SAMPLE && !(a->temperature > 0.f)) return SPACE_E_INVALID_ARG;
+  if (a->logits_row_stride < a->vocab) return SPACE_E_INVALID_ARG;
+  const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;
+  if ((uintptr_t)a->logits % esz) return SPACE_E_ALIGNMENT;
+  return SPACE_OK;
+}
+
+int check_commit_args(const space_ctx* ctx, const space_commit_args* a) {
+  if (a->batch < 0 || a->batch > ctx->cfg.max_batch) return SPACE_E_WORKSPACE;
+  if (a->k < 1 || a->k > ctx->cfg.k_max) return SPACE_E_INVALID_ARG;
+  if (a->batch == 0) return SPACE_OK;
+  if (!a->k_cache || !a->v_cache || !a->n_accept || !a->kv_len) return SPACE_E_INVALID_ARG;
+  if (!aligned16(a->k_cache) || !aligned16(a->v_cache)) return SPACE_E_ALIGNMENT;
+  if (a->kv_stride_b % 8 || a->kv_stride_h % 8 || a->kv_stride_s % 8) return SPACE_E_ALIGNMENT;
+  if (a->kv_stride_s < ctx->cfg.head_dim) return SPACE_E_INVALID_ARG;
+  return SPACE_OK;
 }
 
 }  // namespace
@@ -202,6 +236,7 @@ int space_attn_step(space_ctx* ctx, const space_attn_args* a, void* stream) {
     return SPACE_E_ALIGNMENT;
   if (a->kv_stride_s < ctx->cfg.head_dim || a->kv_stride_b < 1 || a->kv_stride_h < 1) return SPACE_E_INVALID_ARG;
   if (a->kv_stride_b % 8 || a->kv_stride_h % 8 || a->kv_stride_s % 8) return SPACE_E_ALIGNMENT;
+  if (!use_device(ctx)) return SPACE_E_CUDA;
   space_layout_t lay;
   build_layout(a->k, a->mask_variant, &lay);
   cudaStream_t st = (cudaStream_t)stream;
@@ -212,22 +247,22 @@ int space_attn_step(space_ctx* ctx, const space_attn_args* a, void* stream) {
 
 int space_verify(space_ctx* ctx, const space_verify_args* a, void* stream) {
   if (!ctx || !a) return SPACE_E_INVALID_ARG;
-  if (a->batch < 0 || a->batch > ctx->cfg.max_batch) return SPACE_E_WORKSPACE;
-  if (a->k < 1 || a->k > ctx->cfg.k_max) return SPACE_E_INVALID_ARG;
-  if (a->vocab < 1 || a->vocab > ctx->cfg.vocab) return SPACE_E_WORKSPACE;
+  const int rc = check_verify_args(ctx, a);
+  if (rc != SPACE_OK || a->batch == 0) return rc;
+  if (!use_device(ctx)) return SPACE_E_CUDA;
+  return launch_verify(ctx, a, nullptr, (cudaStream_t)stream);
+}
+
+int space_verify_commit(space_ctx* ctx, const space_verify_args* a, const space_commit_args* c, void* stream) {
+  if (!ctx || !a || !c) return SPACE_E_INVALID_ARG;
+  int rc = check_verify_args(ctx, a);
+  if (rc != SPACE_OK) return rc;
+  rc = check_commit_args(ctx, c);
+  if (rc != SPACE_OK) return rc;
+  if (c->batch != a->batch || c->k != a->k || c->n_accept != a->n_accept) return SPACE_E_INVALID_ARG;
   if (a->batch == 0) return SPACE_OK;
-  if (!a->logits || !a->cand || !a->cand_prob || !a->n_accept || !a->out_tokens || !a->n_out ||
-      !a->next_cand || !a->next_cand_prob || !a->finished)
-    return SPACE_E_INVALID_ARG;
-  if (a->logits_dtype != SPACE_DTYPE_F32 && a->logits_dtype != SPACE_DTYPE_BF16) return SPACE_E_INVALID_ARG;
-  if (a->mode != SPACE_MODE_GREEDY && a->mode != SPACE_MODE_SAMPLE) return SPACE_E_INVALID_ARG;
-  if (a->resample != SPACE_RESAMPLE_RESIDUAL_POINTMASS && a->resample != SPACE_RESAMPLE_PAPER_LITERAL)
-    return SPACE_E_INVALID_ARG;
-  if (a->mode == SPACE_MODE_SAMPLE && !(a->temperature > 0.f)) return SPACE_E_INVALID_ARG;
-  if (a->logits_row_stride < a->vocab) return SPACE_E_INVALID_ARG;
-  const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;
-  if ((uintptr_t)a->logits % esz) return SPACE_E_ALIGNMENT;
-  return launch_verify(ctx, a, (cudaStream_t)stream);
+  if (!use_device(ctx)) return SPACE_E_CUDA;
+  return launch_verify(ctx, a, c, (cudaStream_t)stream);
 }
 
 int space_verify_greedy_noalloc(const space_verify_args* a, void* stream) {
@@ -258,19 +293,15 @@ int space_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, void* stream
     return SPACE_E_ALIGNMENT;
   if (a->hidden_row_stride < a->hidden_dim || a->weight_row_stride < a->hidden_dim) return SPACE_E_INVALID_ARG;
   if (a->batch * (a->k + 1) * (a->k + 1) > SPACE_LMHEAD_MAX_ROWS) return SPACE_E_UNSUPPORTED;
-  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return SPACE_E_CUDA;
+  if (!use_device(ctx)) return SPACE_E_CUDA;
   return launch_lmhead_verify(ctx, a, (cudaStream_t)stream);
 }
 
 int space_kv_commit(space_ctx* ctx, const space_commit_args* a, void* stream) {
   if (!ctx || !a) return SPACE_E_INVALID_ARG;
-  if (a->batch < 0 || a->batch > ctx->cfg.max_batch) return SPACE_E_WORKSPACE;
-  if (a->k < 1 || a->k > ctx->cfg.k_max) return SPACE_E_INVALID_ARG;
-  if (a->batch == 0) return SPACE_OK;
-  if (!a->k_cache || !a->v_cache || !a->n_accept || !a->kv_len) return SPACE_E_INVALID_ARG;
-  if (!aligned16(a->k_cache) || !aligned16(a->v_cache)) return SPACE_E_ALIGNMENT;
-  if (a->kv_stride_b % 8 || a->kv_stride_h % 8 || a->kv_stride_s % 8) return SPACE_E_ALIGNMENT;
-  if (a->kv_stride_s < ctx->cfg.head_dim) return SPACE_E_INVALID_ARG;
+  const int rc = check_commit_args(ctx, a);
+  if (rc != SPACE_OK || a->batch == 0) return rc;
+  if (!use_device(ctx)) return SPACE_E_CUDA;
   return launch_commit(ctx, a, (cudaStream_t)stream);
 }
 
@@ -285,6 +316,7 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* a, void* stream)
       !a->out || !a->n_accept || !a->out_tokens || !a->n_out || !a->next_cand || !a->next_cand_prob ||
       !a->finished || !a->status)
     return SPACE_E_INVALID_ARG;
+  if (!use_device(ctx)) return SPACE_E_CUDA;
   cudaStream_t st = (cudaStream_t)stream;
   const int B = a->batch, k = a->k, k1 = k + 1, n_q = k1 * k1, d = c.head_dim;
   const Carve cv = carve(&c, ctx->sm_count);
@@ -358,13 +390,11 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* a, void* stream)
   ve.logits = d_logits; ve.logits_row_stride = a->vocab; ve.cand = d_cand; ve.cand_prob = d_cprob;
   ve.seq_id = nullptr; ve.kv_len = d_kvlen; ve.n_accept = d_nacc; ve.out_tokens = d_tok; ve.n_out = d_nout;
   ve.next_cand = d_ncand; ve.next_cand_prob = d_nprob; ve.finished = d_fin; ve.status = d_status;
-  rc = space_verify(ctx, &ve, stream);
-  if (rc != SPACE_OK) return rc;
   space_commit_args cm{};
   cm.batch = B; cm.k = k; cm.k_cache = d_k; cm.v_cache = d_v;
   cm.kv_stride_b = at.kv_stride_b; cm.kv_stride_h = at.kv_stride_h; cm.kv_stride_s = at.kv_stride_s;
   cm.n_accept = d_nacc; cm.kv_len = d_kvlen; cm.kv_len_out = d_kvlen_out; cm.status = d_status;
-  rc = space_kv_commit(ctx, &cm, stream);
+  rc = space_verify_commit(ctx, &ve, &cm, stream);
   if (rc != SPACE_OK) return rc;
 
   ok = ok && down(a->out, d_out, (size_t)B * n_q * c.n_q_heads * d * 4);
@@ -436,6 +466,7 @@ int space_profile_read(space_ctx* ctx, float* ms, int64_t* n) {
 int space_debug_philox(space_ctx* ctx, uint64_t seed, int64_t n, const uint32_t* c0, const uint32_t* c1,
                        const uint32_t* c2, const uint32_t* c3, uint32_t* out, void* stream) {
   if (!ctx || n < 0 || (n > 0 && (!c0 || !c1 || !c2 || !c3 || !out))) return SPACE_E_INVALID_ARG;
+  if (!use_device(ctx)) return SPACE_E_CUDA;
   return launch_philox_debug(seed, n, c0, c1, c2, c3, out, (cudaStream_t)stream);
 }
 

@@ -51,6 +51,8 @@ struct VerifyParams {
   VerifyRow* rows;           // [B][k+1]
   int* counter_a;            // [B]
   int* counter_b;            // [B]
+  int do_commit;             // the kernels also move the accepted cache rows (space_verify_commit)
+  CommitParams cm;
 };
 
 // 2^x by the hardware approximation (relative error about 2^-22: far inside the
@@ -454,8 +456,9 @@ verify_target_kernel(const VerifyParams p) {
             q = fast_exp2((zc - r.m) * p.c_t) / r.s;
           }
           const Philox4 w = philox4x32_10(0u, PURPOSE_ACCEPT, seq, (uint32_t)(L + tt + 1), p.key0, p.key1);
-          const float lhs = uniform_open(w.x) * p.cand_prob[b * p.k + tt];   // r <= Q/P_c  <=>  r*P_c <= Q
-          ok = lhs <= q;
+          const float pc = p.cand_prob[b * p.k + tt];
+          const float lhs = uniform_open(w.x) * pc;                          // r <= Q/P_c  <=>  r*P_c <= Q
+          ok = in_range && pc > 0.f && lhs <= q;                             // NaN, zero or negative P_c: rejected
         }
       }
       sh_ok[tt] = ok;
@@ -488,6 +491,15 @@ verify_emit_kernel(const VerifyParams p) {
   const uint32_t seq = p.seq_id ? p.seq_id[b] : (uint32_t)b;
   const int L = p.kv_len ? p.kv_len[b] : 0;
   const T* base = reinterpret_cast<const T*>(p.logits) + (int64_t)b * p.n_q * p.row_stride;
+  // With the commit on board every block of the sequence moves its slice of the accepted
+  // rows (i* is known to all of them); the last block writes the new length and the tables.
+  int Lc = 0;
+  if (p.do_commit) {
+    Lc = p.cm.kv_len[b];
+    if (commit_fits(p.cm, Lc))
+      commit_rows(p.cm, b, Lc, max(0, min(i_star, p.k)), slot * p.n_chunks + ch, n_slots * p.n_chunks,
+                  threadIdx.x, blockDim.x);
+  }
   // slot o < k: mask row (i*, o+1); slot k: target row i* (extra token, sampling)
   const int brow = (slot < p.k) ? i_star * k1 + slot + 1 : i_star * k1;
   const T* row = base + (int64_t)brow * p.row_stride;
@@ -496,7 +508,9 @@ verify_emit_kernel(const VerifyParams p) {
   Stat st;
   if (slot == p.k) {
     int exclude = -1;
-    if (!literal && i_star < p.k) exclude = p.cand[b * p.k + i_star];   // residual of a point mass
+    // residual of a point-mass draft (P_c = 1): the rejected token is removed.  A candidate
+    // with any other P_c (Algorithm 1 starts from P_c = +inf) was no point mass: a ~ Q.
+    if (!literal && i_star < p.k && p.cand_prob[b * p.k + i_star] == 1.0f) exclude = p.cand[b * p.k + i_star];
     // the extra token needs the noisy arg-max alone: the row's sums are known
     st = scan_chunk<T, VECTOR, true, false>(row, begin, end, c, exclude, p.key0, p.key1, PURPOSE_TOKEN,
                                             seq, (uint32_t)(L + i_star + 1));
@@ -550,6 +564,8 @@ verify_emit_kernel(const VerifyParams p) {
     if (j == 0) {
       p.n_out[b] = n_out;
       p.finished[b] = (uint8_t)(eos_mask != 0);
+      // every block of the sequence has read the old length by now (arrival counter)
+      if (p.do_commit) commit_tables(p.cm, b, Lc, max(0, min(i_star, p.k)), commit_fits(p.cm, Lc));
     }
   }
 }
@@ -568,7 +584,16 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   constexpr float C1 = 1.4426950408889634f;                 // T = 1
   const T* row = reinterpret_cast<const T*>(p.logits) + ((int64_t)b * p.n_q + row_i) * p.row_stride;
   const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
+  int Lc = 0;
+  if (p.do_commit) Lc = p.cm.kv_len[b];                     // in flight during the scan
   Stat st = scan_chunk<T, VECTOR, false, true>(row, begin, end, C1, -1, 0, 0, 0, 0, 0);
+  // KV commit on board: which candidates are accepted is known only to the last block, at the very
+  // end, so every block moves its slice of ALL k candidate rows now, while the logits stream.
+  // Rows L+1 .. L+i* end up exactly as the plain commit leaves them; rows L+i*+1 .. L+k, which lie
+  // beyond the new length and held mask-token rows nobody reads again, receive the rejected
+  // candidates' rows instead.
+  if (p.do_commit && commit_fits(p.cm, Lc))
+    commit_rows(p.cm, b, Lc, p.k, row_i * p.n_chunks + ch, p.n_q * p.n_chunks, threadIdx.x, blockDim.x);
   st = block_reduce_plain(st, C1);
   VerifyPartial* pb = fpart + (int64_t)b * SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS;
   if (threadIdx.x == 0) store_partial(pb + row_i * p.n_chunks + ch, st);
@@ -626,6 +651,8 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
       p.n_out[b] = n_out;
       p.finished[b] = (uint8_t)(eos_mask != 0);
       if (p.status && bits) atomicOr(p.status + b, bits);
+      // new length and index tables; every block of the sequence read the old length before it arrived
+      if (p.do_commit) commit_tables(p.cm, b, Lc, i_star, commit_fits(p.cm, Lc));
     }
   }
 }
@@ -660,8 +687,10 @@ __global__ void philox_debug_kernel(uint32_t k0, uint32_t k1, int64_t n, const u
 
 }  // namespace
 
-int launch_verify(space_ctx* ctx, const space_verify_args* a, cudaStream_t st) {
+int launch_verify(space_ctx* ctx, const space_verify_args* a, const space_commit_args* cm, cudaStream_t st) {
   VerifyParams p;
+  p.do_commit = cm != nullptr;
+  if (cm) fill_commit_params(ctx, cm, &p.cm); else memset(&p.cm, 0, sizeof(p.cm));
   p.B = a->batch; p.k = a->k; p.V = a->vocab; p.n_q = (a->k + 1) * (a->k + 1);
   p.mode = a->mode; p.resample = a->resample; p.eos_id = a->eos_id;
   const float T = (a->mode == SPACE_MODE_SAMPLE) ? a->temperature : 1.0f;
@@ -771,6 +800,16 @@ int launch_verify_noalloc(const space_verify_args* a, cudaStream_t st) {
       cudaGetLastError();
       return SPACE_E_CUDA;
     }
+    // With lazy module loading a kernel's code reaches the device at its first use: ask for the
+    // attributes of all four variants now, so that no later call is the one that loads anything.
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, verify_fused_kernel<float, true>) != cudaSuccess ||
+        cudaFuncGetAttributes(&fa, verify_fused_kernel<float, false>) != cudaSuccess ||
+        cudaFuncGetAttributes(&fa, verify_fused_kernel<__nv_bfloat16, true>) != cudaSuccess ||
+        cudaFuncGetAttributes(&fa, verify_fused_kernel<__nv_bfloat16, false>) != cudaSuccess) {
+      cudaGetLastError();
+      return SPACE_E_CUDA;
+    }
     g_noalloc_sms[dev] = sms;
     g_noalloc_ptr[dev] = ptr;
   }
@@ -790,6 +829,7 @@ int launch_verify_noalloc(const space_verify_args* a, cudaStream_t st) {
   p.status = a->status;
   p.part = nullptr; p.rows = nullptr;
   p.counter_a = reinterpret_cast<int*>(base); p.counter_b = nullptr;
+  p.do_commit = 0; memset(&p.cm, 0, sizeof(p.cm));
   VerifyPartial* fpart = reinterpret_cast<VerifyPartial*>(base + SPACE_NOALLOC_COUNTER_BYTES);
 
   const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;

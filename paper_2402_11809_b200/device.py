@@ -69,6 +69,18 @@ class DeviceStep:
         ctx.space_verify(a)
         return a
 
+    def verify_commit(self, ctx, mode=B.MODE_GREEDY, temperature=1.0, seed=0,
+                      resample=B.RESAMPLE_RESIDUAL_POINTMASS, eos_id=-1, in_place=False):
+        v = ctx.verify_args(self.logits, self.cand, self.cand_prob, self.kv_len, self.n_accept,
+                            self.out_tokens, self.n_out, self.next_cand, self.next_cand_prob,
+                            self.finished, self.k, mode=mode, temperature=temperature, seed=seed,
+                            resample=resample, eos_id=eos_id, seq_id=self.seq_id, status=self.status)
+        c = ctx.commit_args(self.k_cache, self.v_cache, self.n_accept, self.kv_len, self.k,
+                            kv_len_out=self.kv_len if in_place else self.kv_len_out,
+                            commit_src=self.commit_src, commit_dst=self.commit_dst, status=self.status)
+        ctx.space_verify_commit(v, c)
+        return v, c
+
     def commit(self, ctx):
         a = ctx.commit_args(self.k_cache, self.v_cache, self.n_accept, self.kv_len, self.k,
                             kv_len_out=self.kv_len_out, commit_src=self.commit_src,

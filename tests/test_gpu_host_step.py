@@ -78,13 +78,16 @@ def test_host_step_matches_oracle_full_and_resident(B, k, L, H_q, H_kv):
         assert np.array_equal(outs["n_out"].numpy(), r["n_out"])
         assert np.array_equal(outs["next_cand"].numpy(), r["next_cand"])
         assert np.array_equal(pin["kv_len"].numpy(), new_len)
-        # the rows the commit moved come back to the host cache: rows L .. L+k of every head
+        # the rows the commit moved come back to the host cache: rows L .. new length - 1 of every
+        # head (rows from the new length up to L+k come back too, but lie beyond the verified prefix
+        # and are unspecified)
         got_k = pin["k_cache"].numpy().view(np.uint16)
         got_v = pin["v_cache"].numpy().view(np.uint16)
         for b in range(cfg["B"]):
-            Lb = int(x["kv_len"][b])
-            assert np.array_equal(got_k[b, :, Lb:Lb + k + 1], Kc[b, :, Lb:Lb + k + 1])
-            assert np.array_equal(got_v[b, :, Lb:Lb + k + 1], Vc[b, :, Lb:Lb + k + 1])
+            Lb, nb = int(x["kv_len"][b]), int(new_len[b])
+            assert np.array_equal(got_k[b, :, Lb:nb], Kc[b, :, Lb:nb])
+            assert np.array_equal(got_v[b, :, Lb:nb], Vc[b, :, Lb:nb])
+            assert np.array_equal(got_k[b, :, Lb + k + 1:], Kc[b, :, Lb + k + 1:])
 
     pin = fresh_pins()
     outs, h2d_full, _ = _run(B, ctx, cfg, x, pin, resident=False)

@@ -56,6 +56,10 @@ def _check_verify(ds, r, k, sample=False):
                                rtol=1e-4, atol=1e-30)
     if excl.any():
         print(f"excluded {int(excl.sum())} sequence(s) inside the tie band: {np.nonzero(excl)[0].tolist()}")
+    # The bands are 1e-4 wide: about one floating-point decision in 10^4 falls inside one.  More than
+    # one excluded sequence per call means the diagnostics (or the comparison) are broken, and greedy
+    # mode takes no floating-point decision at all.
+    assert int(excl.sum()) <= (1 if sample else 0), f"{int(excl.sum())} sequences excluded"
     return excl
 
 
@@ -233,6 +237,19 @@ def test_verify_greedy_exact_ties_and_bad_candidates(B, H):
     _check_verify(ds, r, k)
     st = ds.status.cpu().numpy()
     assert st[1] & B.ST_BAD_CANDIDATE and st[2] & B.ST_BAD_CANDIDATE and st[0] == 0
+    # sampling mode: an out-of-range id is rejected whatever P_c says (0, negative, NaN), and so is
+    # an in-range one whose P_c is not positive
+    x["cand_prob"][1, 0] = 0.0
+    x["cand_prob"][2, 0] = -2.0
+    x["cand_prob"][3, :] = np.array([0.0, -1.0, np.nan], dtype=np.float32)
+    ds = H.DeviceStep(cfg, x)
+    ds.verify(ctx, mode=B.MODE_SAMPLE, temperature=1.0, seed=3)
+    r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "sample", temperature=1.0, seed=3,
+                    seq_id=x["seq_id"], kv_len=x["kv_len"])
+    _check_verify(ds, r, k, sample=True)
+    assert r["n_accept"][1] == 0 and r["n_accept"][2] == 0 and r["n_accept"][3] == 0
+    st = ds.status.cpu().numpy()
+    assert st[1] & B.ST_BAD_CANDIDATE and st[2] & B.ST_BAD_CANDIDATE
 
 
 @pytest.mark.parametrize("resample", ["residual_pointmass", "paper_literal"])
@@ -251,10 +268,29 @@ def test_verify_sampling_small(B, H, resample, k, V, Bn, T):
         ds.verify(ctx, mode=B.MODE_SAMPLE, temperature=T, seed=seed, resample=code)
         r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "sample", temperature=T, seed=seed,
                         seq_id=x["seq_id"], kv_len=x["kv_len"], resample=resample)
-        excl = _check_verify(ds, r, k, sample=True)
-        assert excl.mean() < 0.2
+        _check_verify(ds, r, k, sample=True)                # at most one sequence inside a tie band
         assert r["n_accept"][0] == 0 and int(ds.n_accept[0]) == 0
     assert r["n_accept"].max() > 0
+
+
+def test_verify_sampling_initial_state_can_emit_token_zero(B, H):
+    # Algorithm 1 starts from L_c = [0]*k, P_c = [+inf]*k: the rejected "candidate" 0 stays in
+    # the extra token's distribution.  Token 0 carries almost all of the mass here.
+    k, V, Bn = 2, 64, 32
+    cfg = workloads.resolve("sampling64", B=Bn, H_q=1, H_kv=1, d=64, L=(5, 50), k=k, V=V, seed=77)
+    x = workloads.make_step_inputs(cfg)
+    lf = bf16_bits_to_f64(x["logits"]).astype(np.float32)
+    lf[:, :, 0] = 25.0
+    x["logits"] = workloads.f32_to_bf16_bits(lf)
+    x["cand"][:] = 0
+    x["cand_prob"][:] = np.inf
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    ds.verify(ctx, mode=B.MODE_SAMPLE, temperature=1.0, seed=9)
+    r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "sample", temperature=1.0, seed=9,
+                    seq_id=x["seq_id"], kv_len=x["kv_len"])
+    _check_verify(ds, r, k, sample=True)
+    assert np.all(r["n_accept"] == 0) and (r["out_tokens"][:, 0] == 0).sum() >= Bn - 2
 
 
 # --------------------------------------------------------------------- commit
@@ -275,41 +311,110 @@ def test_commit(B, H, k, d, H_kv, Bn):
     assert np.array_equal(ds.kv_len_out.cpu().numpy(), new_len)
     assert np.array_equal(ds.commit_src.cpu().numpy(), src)
     assert np.array_equal(ds.commit_dst.cpu().numpy(), dst)
-    # in-place length update
-    a = ctx.commit_args(ds.k_cache, ds.v_cache, ds.n_accept, ds.kv_len, k, kv_len_out=ds.kv_len)
-    ds.n_accept.zero_()
+    # in-place length update, with rows to move: a fresh copy of the inputs
+    ds = H.DeviceStep(cfg, x)
+    ds.n_accept.copy_(torch.from_numpy(n_acc))
+    a = ctx.commit_args(ds.k_cache, ds.v_cache, ds.n_accept, ds.kv_len, k, kv_len_out=ds.kv_len,
+                        commit_src=ds.commit_src, commit_dst=ds.commit_dst)
     ctx.space_kv_commit(a)
-    assert np.array_equal(ds.kv_len.cpu().numpy(), x["kv_len"] + 1)
+    assert np.array_equal(H.bf16_to_bits(ds.k_cache), Kc)
+    assert np.array_equal(H.bf16_to_bits(ds.v_cache), Vc)
+    assert np.array_equal(ds.kv_len.cpu().numpy(), new_len)
+    assert np.array_equal(ds.commit_src.cpu().numpy(), src)
+    assert np.array_equal(ds.commit_dst.cpu().numpy(), dst)
+
+
+@pytest.mark.parametrize("in_place", [False, True])
+@pytest.mark.parametrize("case", ["greedy_one_launch", "greedy_two_launches", "sample", "sample_literal"])
+def test_verify_commit_in_one_call(B, H, case, in_place):
+    # space_verify_commit against the oracle's verify_step followed by commit_step
+    sample = case.startswith("sample")
+    if case == "greedy_two_launches":          # more than 64 MB of logits rows: target + emit kernels
+        cfg = _small_cfg(3, (3, 90), d=64, H_q=4, H_kv=2, Bn=17, V=128256, seed=31)
+    elif sample:
+        cfg = workloads.resolve("sampling64", B=6, H_q=4, H_kv=2, d=128, L=(5, 300), k=4, V=5000, seed=32)
+    else:
+        cfg = _small_cfg(5, (3, 90), d=128, H_q=8, H_kv=8, Bn=3, V=32000, seed=33)
+    k = cfg["k"]
+    x = workloads.make_step_inputs(cfg)
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    resample = "paper_literal" if case == "sample_literal" else "residual_pointmass"
+    n0 = ctx.launch_count
+    ds.verify_commit(ctx, mode=B.MODE_SAMPLE if sample else B.MODE_GREEDY, temperature=0.8, seed=5,
+                     resample=B.RESAMPLE_PAPER_LITERAL if case == "sample_literal" else B.RESAMPLE_RESIDUAL_POINTMASS,
+                     in_place=in_place)
+    assert ctx.launch_count - n0 == (1 if case == "greedy_one_launch" else 2)
+    r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "sample" if sample else "greedy",
+                    temperature=0.8, seed=5, seq_id=x["seq_id"], kv_len=x["kv_len"], resample=resample)
+    excl = _check_verify(ds, r, k, sample)
+    assert not excl.any()
+    assert r["n_accept"].max() > 0
+    Kc, Vc = x["k_cache"].copy(), x["v_cache"].copy()
+    new_len, src, dst = commit_step(Kc, Vc, x["kv_len"], r["n_accept"], k)
+    kc, vc = H.bf16_to_bits(ds.k_cache), H.bf16_to_bits(ds.v_cache)
+    if case == "greedy_one_launch":
+        # the single-launch path moves all k candidate rows before i* is known: the verified prefix
+        # (rows below the new length) and everything from row L+k+1 on must equal the oracle's cache;
+        # rows new_len .. L+k lie beyond the new length (dead mask-token rows) and are unspecified
+        for b in range(cfg["B"]):
+            n, hi = int(new_len[b]), int(x["kv_len"][b]) + k + 1
+            assert np.array_equal(kc[b, :, :n], Kc[b, :, :n]) and np.array_equal(vc[b, :, :n], Vc[b, :, :n])
+            assert np.array_equal(kc[b, :, hi:], Kc[b, :, hi:]) and np.array_equal(vc[b, :, hi:], Vc[b, :, hi:])
+    else:
+        assert np.array_equal(kc, Kc)
+        assert np.array_equal(vc, Vc)
+    assert np.array_equal((ds.kv_len if in_place else ds.kv_len_out).cpu().numpy(), new_len)
+    assert np.array_equal(ds.commit_src.cpu().numpy(), src)
+    assert np.array_equal(ds.commit_dst.cpu().numpy(), dst)
+    assert int(ds.status.abs().sum()) == 0
 
 
 # ------------------------------------------------------------ the five configs
-def _run_config(B, H, name, sample_heads=None, **over):
+def _run_config(B, H, name, heads_per_seq=None, fused=False, **over):
+    """One whole step of a BASELINE configuration at full size against the oracle.
+
+    heads_per_seq None: every (sequence, query head) is compared; an integer: that many
+    seeded query heads of every sequence (the oracle needs too long for all of them)."""
     cfg = workloads.resolve(name, **over)
     x = workloads.make_step_inputs(cfg)
     ctx = H.make_context(cfg, x)
     ds = H.DeviceStep(cfg, x)
     k = cfg["k"]
     sample = cfg["mode"] == "sample"
+    mode = B.MODE_SAMPLE if sample else B.MODE_GREEDY
     ds.attn(ctx)
-    ds.verify(ctx, mode=B.MODE_SAMPLE if sample else B.MODE_GREEDY, temperature=cfg["temperature"],
-              seed=cfg["seed"])
-    ds.commit(ctx)
+    if fused:
+        ds.verify_commit(ctx, mode=mode, temperature=cfg["temperature"], seed=cfg["seed"])
+    else:
+        ds.verify(ctx, mode=mode, temperature=cfg["temperature"], seed=cfg["seed"])
+        ds.commit(ctx)
     torch.cuda.synchronize()
     assert int(ds.status.abs().sum()) == 0
     out = ds.out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(out).all()
     G = cfg["H_q"] // cfg["H_kv"]
-    if sample_heads is None:
-        ref, _ = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], k, x["scale"])
-        rel = _check_attention(H, out, ref, name)
-    else:
-        rng = np.random.default_rng(cfg["seed"])
-        rel = 0.0
-        for _ in range(sample_heads):
-            b, h = int(rng.integers(cfg["B"])), int(rng.integers(cfg["H_q"]))
+    rng = np.random.default_rng(cfg["seed"])
+    rel, n_cmp = 0.0, 0
+    batch_sq, batch_n, errs = 0.0, 0, []
+    for b in range(cfg["B"]):
+        heads = range(cfg["H_q"]) if heads_per_seq is None else \
+            sorted(rng.choice(cfg["H_q"], size=heads_per_seq, replace=False).tolist())
+        L = int(x["kv_len"][b])
+        refs, gots = [], []
+        for h in heads:
             ref, _ = attention_head(x["q"][b, :, h], x["k_cache"][b, h // G], x["v_cache"][b, h // G],
-                                    int(x["kv_len"][b]), k, x["scale"])
-            rel = max(rel, _check_attention(H, out[b, :, h], ref, f"{name} b={b} h={h}"))
-        assert np.isfinite(out).all()
+                                    L, k, x["scale"])
+            refs.append(ref); gots.append(out[b, :, h])
+            n_cmp += 1
+        refs, gots = np.stack(refs), np.stack(gots)
+        # per-sequence reading of the tolerance: this sequence's heads against their own RMS
+        rel = max(rel, _check_attention(H, gots[None], refs[None], f"{name} b={b}"))
+        batch_sq += float(np.sum(np.square(refs))); batch_n += refs.size
+        errs.append(float(np.max(np.abs(gots - refs))))
+    # whole-batch reading: one RMS over everything compared
+    rms_all = float(np.sqrt(batch_sq / batch_n))
+    assert max(errs) <= min(2e-2, 1e-2 * rms_all), (max(errs), rms_all)
     r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, cfg["mode"], temperature=cfg["temperature"],
                     seed=cfg["seed"], seq_id=x["seq_id"], kv_len=x["kv_len"])
     excl = _check_verify(ds, r, k, sample)
@@ -324,28 +429,30 @@ def _run_config(B, H, name, sample_heads=None, **over):
             assert np.array_equal(kc[b, :, L + g], x["k_cache"][b, :, L + g * (k + 1)])
             assert np.array_equal(vc[b, :, L + g], x["v_cache"][b, :, L + g * (k + 1)])
         assert np.array_equal(kc[b, :, :L], x["k_cache"][b, :, :L])
-    print(f"{name}: attention max|err|/rms {rel:.2e}; mean accepted {n_acc.mean():.2f}; "
-          f"excluded {int(excl.sum())}")
+    print(f"{name}: attention max|err|/rms {rel:.2e} over {n_cmp} (sequence, head) pairs; "
+          f"mean accepted {n_acc.mean():.2f}; excluded {int(excl.sum())}")
     return n_acc
 
 
 def test_config_tiny(B, H):
     _run_config(B, H, "tiny")
+    _run_config(B, H, "tiny", fused=True)
 
 
 def test_config_llama7b(B, H):
     n = _run_config(B, H, "llama7b")
     assert 0 <= n[0] <= 5
+    assert np.array_equal(n, _run_config(B, H, "llama7b", fused=True))
 
 
 def test_config_ragged16(B, H):
-    _run_config(B, H, "ragged16", sample_heads=24)
+    _run_config(B, H, "ragged16", fused=True)
 
 
 def test_config_gqa70b(B, H):
-    _run_config(B, H, "gqa70b", sample_heads=12)
+    _run_config(B, H, "gqa70b")
 
 
 def test_config_sampling64(B, H):
-    n = _run_config(B, H, "sampling64", sample_heads=12)
+    n = _run_config(B, H, "sampling64", heads_per_seq=1, fused=True)
     assert n.mean() > 0.5

@@ -193,3 +193,101 @@ def test_draws_are_keyed_by_seed_sequence_and_position():
     r1 = verify_step(z, np.ones((500, k), dtype=int), np.ones((500, k)), k, "sample", **kw)
     r2 = verify_step(z, np.ones((500, k), dtype=int), np.ones((500, k)), k, "sample", **kw)
     assert all(np.array_equal(r1[x], r2[x]) for x in r1)
+
+
+# ------------------------------------------------- tie diagnostics (parity bands)
+def test_top2_gap_on_hand_written_rows():
+    # The GPU parity tests drop a sequence whose decision sits inside a tie band; these
+    # are the numbers that decide it, so they are fixed here on rows written by hand.
+    from oracle.verify import _top2_gap
+    s = np.array([[0.0, 3.0, 1.0, 2.5],          # clear winner: index 1, gap 0.5
+                  [7.0, 7.0, 1.0, 7.0],          # exact three-way tie: lowest index, gap 0
+                  [-np.inf, -2.0, -np.inf, -5.0],  # -inf entries never win: gap 3
+                  [4.0, -np.inf, -np.inf, -np.inf]])  # a single finite score: gap inf
+    best, gap = _top2_gap(s)
+    assert best.tolist() == [1, 0, 1, 0]
+    assert gap.tolist() == [0.5, 0.0, 3.0, np.inf]
+    # the input is left as it was
+    assert s[0, 1] == 3.0 and s[1, 0] == 7.0
+
+
+def _uniform_by_hand(seed, seq, pos):
+    # r of Algorithm 1 for (sequence, position): first Philox word of counter
+    # (0, ACCEPT = 0, seq, pos), mapped to ((w >> 9) + 1/2) 2^-23 -- written out here,
+    # Philox itself is pinned by its known-answer vectors
+    from oracle.philox import philox4x32_10
+    w = philox4x32_10(0, 0, seq, pos, seed & 0xFFFFFFFF, seed >> 32)[0]
+    return (float(int(w) >> 9) + 0.5) * 2.0 ** -23
+
+
+def test_accept_margin_on_hand_written_cases():
+    k, V, T, seed, L = 2, 2, 1.0, 77, 9
+    z = np.zeros((4, layout.n_block_rows(k), V))
+    z[:, 0, 1] = np.log(3.0)                      # row 0: Q = (1/4, 3/4)
+    z[:, layout.target_rows(k)[1], 0] = np.log(4.0)   # row of c_1: Q = (4/5, 1/5)
+    cand = np.array([[1, 0]] * 4)
+    seq = np.arange(4)
+    r1 = np.array([_uniform_by_hand(seed, s, L + 1) for s in seq])
+    r2 = np.array([_uniform_by_hand(seed, s, L + 2) for s in seq])
+    P = np.ones((4, k))
+    P[0, 0] = 0.75 / r1[0]                        # r*P_c == Q exactly: margin 0 (accepted, "<=")
+    P[0, 1] = 2 * 0.8 / r2[0]                     # r*P_c = 2Q: margin 1, rejected
+    P[1, 0] = 0.5 * 0.75 / r1[1]                  # r*P_c = Q/2: margin 1/2, accepted
+    P[1, 1] = INF                                 # cannot be accepted; no floating-point decision
+    P[2, 0] = 3 * 0.75 / r1[2]                    # rejected at i = 1: margin 2 ...
+    P[2, 1] = 0.8 / r2[2]                         # ... and position 2 is never tested: inf
+    P[3, :] = 1e-9                                # both accepted, margins ~ 1
+    r = verify_step(z, cand, P, k, "sample", temperature=T, seed=seed, seq_id=seq,
+                    kv_len=np.full(4, L))
+    am = r["accept_margin"]
+    assert r["n_accept"].tolist() == [1, 1, 0, 2]
+    assert am[0, 0] < 1e-15 and abs(am[0, 1] - 1.0) < 1e-12
+    assert abs(am[1, 0] - 0.5) < 1e-12 and am[1, 1] == INF
+    assert abs(am[2, 0] - 2.0) < 1e-12 and am[2, 1] == INF
+    assert np.all(np.abs(am[3] - 1.0) < 1e-6)
+    # greedy mode takes no floating-point acceptance decision
+    g = verify_step(z, cand, np.ones((4, k)), k, "greedy")
+    assert np.all(g["accept_margin"] == INF) and np.all(g["bonus_gap"] == INF)
+
+
+def test_bonus_gap_matches_scores_written_by_hand():
+    # one sequence, three tokens: the extra token's top-two gap recomputed from
+    # log Q + Gumbel noise written out explicitly
+    from oracle.philox import philox4x32_10
+    k, V, T, seed, L = 1, 3, 0.5, 5, 4
+    z = np.zeros((1, layout.n_block_rows(k), V))
+    z[0, 0] = [0.2, -0.1, 0.4]
+    r = verify_step(z, np.array([[1]]), np.full((1, k), INF), k, "sample", temperature=T,
+                    seed=seed, kv_len=np.array([L]), resample="paper_literal")
+    assert r["n_accept"][0] == 0
+    w = philox4x32_10(0, 1, 0, L + 1, seed, 0)       # tokens 0..2 share counter word 0, purpose TOKEN = 1
+    u = [(float(int(w[j]) >> 9) + 0.5) * 2.0 ** -23 for j in range(3)]
+    q = np.exp(z[0, 0] / T); q /= q.sum()
+    score = sorted(np.log(q[j]) - np.log(-np.log(u[j])) for j in range(3))
+    assert abs(r["bonus_gap"][0] - (score[2] - score[1])) < 1e-12
+
+
+# --------------------------------------- Algorithm 1's initial state, odd P_c values
+def test_initial_state_draws_the_first_token_from_Q_including_token_zero():
+    # L_c = [0]*k, P_c = [+inf]*k (Algorithm 1): everything is rejected and the one
+    # emitted token must follow Q -- token 0, the "rejected candidate", included.
+    k, T, seed = 2, 0.8, 424242
+    z = _fixed_logits(k, 4)
+    q0 = softmax_rows(z[0, 0], T)
+    r = verify_step(z, np.zeros((N, k), dtype=int), np.full((N, k), INF), k, "sample",
+                    temperature=T, seed=seed, seq_id=np.arange(N), kv_len=np.full(N, 3))
+    assert np.all(r["n_accept"] == 0)
+    counts = np.bincount(r["out_tokens"][:, 0], minlength=V16)
+    assert counts[0] > 0
+    chi, _ = _chi2(counts, q0)
+    assert chi < 55.0, chi
+
+
+def test_acceptance_needs_a_positive_probability_and_an_in_range_token():
+    k, V = 2, 6
+    z = _logits(np.random.default_rng(3), 8, k, V)
+    for bad_p in (0.0, -1.0, np.nan):
+        for c0 in (1, V + 2, -4):
+            r = verify_step(z, np.full((8, k), c0), np.full((8, k), bad_p), k, "sample",
+                            seed=3, seq_id=np.arange(8))
+            assert np.all(r["n_accept"] == 0), (bad_p, c0)
