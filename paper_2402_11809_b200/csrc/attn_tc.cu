@@ -48,6 +48,7 @@ struct AttnParams {
   int n_pad;                           // rows_per_mb * G rounded up to 16: N of the MMAs
   int n_groups;                        // thread-block groups (grid = n_groups * n_mblocks)
   int out_dtype;
+  int spec;                            // one sequence: every group requests its first K tile before the length is read
   int64_t s_cap;
   float scale_log2;                    // scale * log2(e)
   const int32_t* kv_len;
@@ -57,11 +58,17 @@ struct AttnParams {
   int2* desc;                          // [B*H_kv*n_mblocks] {first partial slot, number of partials} of each cut
   int* owner;                          // [grid] (sequence, kv head) whose last piece this thread block computed, or -1
   int merge_by_owner;                  // the merge grid is indexed by attention thread block, not by (sequence, head)
-  uint64_t mask[SPACE_MAX_ROWS];       // bit j of mask[i]: block row i sees block key j
-  uint64_t mask_t[SPACE_MAX_ROWS];     // transposed: bit i of mask_t[j]
+  // Eq. 5 per (query column, block key), worked out by the host once per call: bit q of
+  // visq[mb][j] says that query column q of query-row block mb (block row mb * rows_per_mb + q / G,
+  // any of its G heads) sees block key j
+  uint64_t visq[2][SPACE_MAX_ROWS];
 };
 
-struct Seg { int b, h, t0, t1, T, L, slot, dfirst, dn; };
+// One share: tiles t0, t0 + step, ... (n of them) of the T tiles of (sequence b, kv head h).
+struct Seg {
+  int b, h, t0, n, step, T, L, slot, dfirst, dn;   // slot: partial slot; dfirst/dn: cut (aligned mode)
+  __device__ __forceinline__ int tile_at(int j) const { return t0 + j * step; }
+};
 
 // Optional per-block timeline (compiled in with -DSPACE_TIMELINE): one %globaltimer stamp
 // per named point and thread block, read back with space_debug_timeline_read.
@@ -140,6 +147,20 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm,
       " [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(dst), "l"((uint64_t)tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+// The same load with an L2 policy: K and V tiles are read once per step, so their lines are marked
+// to be evicted first and leave the cache to what is read again (code, lengths, partials).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
+                                                 int c0, int c1, int c2, int c3, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+      ::"r"(dst), "l"((uint64_t)tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after()  { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -176,10 +197,26 @@ __device__ __forceinline__ long long muldiv(long long a, long long b, long long 
   return (long long)(prod / (unsigned long long)c);
 }
 
+// Piece `piece` of `a` of a (sequence, head) with T tiles: tiles [t0, t1).  When the last tile is a
+// partial one and there are at least `a` full tiles, the full tiles are cut evenly (the first pieces
+// take the remainder) and the partial tile goes to the last piece on top; otherwise all T tiles are
+// cut evenly.
+__device__ __forceinline__ void even_cut(int T, int n_keys, int a, int piece, int& t0, int& t1) {
+  const int Tf = (n_keys % TILE_N) ? T - 1 : T;
+  const int Tc = (Tf < T && a <= Tf) ? Tf : T;
+  const int q = Tc / a, r = Tc - q * a;
+  t0 = piece * q + min(piece, r);
+  t1 = t0 + q + (piece < r ? 1 : 0);
+  if (piece == a - 1) t1 = T;
+}
+
 struct Partition {
   const int* seq_len;    // [B]   verified length, or -1 for a sequence that does not fit
   const int* prefix;     // [B+1] flat offset of sequence b
-  const int* seg0;       // aligned mode: {b, h, t0, t1, T, L, first group of the cut, groups in the cut}
+  // aligned mode: {b, h, t0, n, T, L, first slot of the cut, pieces in the cut, step, early requests
+  // serve the first share, head stride from share to share, slot (slots per head when the stride is
+  // not 0), number of shares}
+  const int* seg0;
   int B, H_kv, n_q, group, ngroups;
   long long cur, end;
   int b;
@@ -196,7 +233,7 @@ struct Partition {
     group = group_; ngroups = n_groups;
     aligned = agroups >= 0;
     if (aligned) {
-      cur = (group_ < agroups) ? 0 : 1; end = 1;
+      cur = 0; end = seg0_[12];
       return;
     }
     const long long W = pf[B_];
@@ -207,12 +244,20 @@ struct Partition {
   }
   __device__ bool next(Seg& s) {
     if (aligned) {
-      // exactly one share, worked out once per thread block during the set-up
+      // the shares were worked out once per thread block during the set-up: one, or (one
+      // sequence, groups left over after every head got its pieces) the last tile of several heads
       if (cur >= end) return false;
       const int4 u = reinterpret_cast<const int4*>(seg0)[0], v = reinterpret_cast<const int4*>(seg0)[1];
-      s.b = u.x; s.h = u.y; s.t0 = u.z; s.t1 = u.w; s.T = v.x; s.L = v.y; s.dfirst = v.z; s.dn = v.w;
-      s.slot = group;
-      cur = end;
+      s.b = u.x; s.h = u.y; s.t0 = u.z; s.n = u.w; s.T = v.x; s.L = v.y; s.dfirst = v.z; s.dn = v.w;
+      s.step = seg0[8];
+      s.slot = seg0[11];
+      const int hstep = seg0[10];
+      if (hstep > 0) {
+        s.h = u.y + (int)cur * hstep;
+        s.dfirst = s.h * seg0[11];
+        s.slot = s.dfirst + seg0[11] - 1;
+      }
+      ++cur;
       return true;
     }
     // Flat mode: the list holds T + SHARE_COST entries per (sequence, head); the
@@ -231,7 +276,7 @@ struct Partition {
       cur += n;
       const int t0 = max(r0 - SHARE_COST, 0), t1 = max(r0 + (int)n - SHARE_COST, 0);
       if (t1 <= t0) continue;                               // only the cost entries: no tiles here
-      s.b = b; s.h = h; s.t0 = t0; s.t1 = t1; s.T = T; s.L = L;
+      s.b = b; s.h = h; s.t0 = t0; s.n = t1 - t0; s.step = 1; s.T = T; s.L = L;
       s.slot = b * H_kv + h + group; s.dfirst = -1; s.dn = 0;
       return true;
     }
@@ -270,10 +315,11 @@ struct Smem {
   static constexpr int MISC_OFF = BAR_OFF + (N_BARS * 8 + 15) / 16 * 16;   // tmem base, abort flag (16-byte aligned:
                                                                            // the float arrays below are read as float4)
   static constexpr int SEG0_OFF = MISC_OFF + 16;             // Seg of this group's only share (aligned mode)
-  static constexpr int MREF_OFF = MISC_OFF + 64;             // [2][RS] float: reference maximum per query row
+  static constexpr int MREF_OFF = MISC_OFF + 96;             // [2][RS] float: reference maximum per query row
   static constexpr int XQ_OFF = MREF_OFF + 2 * RS * 4;       // [4 quarters][RS] float: cross-lane reductions
   static constexpr int FQ_OFF = XQ_OFF + 4 * RS * 4;         // [RS] float: rescale factors / final row sums
-  static constexpr int TABLE_OFF = FQ_OFF + RS * 4;          // seq_len[max_batch], prefix[max_batch+1]
+  static constexpr int VISQ_OFF = FQ_OFF + RS * 4;           // [64] uint64: query columns that see block key j (bit = column)
+  static constexpr int TABLE_OFF = VISQ_OFF + SPACE_MAX_ROWS * 8;   // seq_len[max_batch], prefix[max_batch+1]
   // with the tables of the largest batch (128 sequences) the plan must fit the 227 KB a block may have
   static_assert(TABLE_OFF + (2 * 128 + 1) * 4 <= 227 * 1024, "shared-memory plan too large");
 };
@@ -313,22 +359,6 @@ __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
                ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
                : "memory");
-}
-
-// Which of the query rows col0 .. col0+ncol-1 see block key `jb` (bit = row - col0).
-// rows_t = mask_t[jb]: bit i set when block row i sees the key; query row q is
-// block row i0 + q / G.
-__device__ __noinline__ uint64_t block_key_visibility(uint64_t rows_t, int col0, int ncol, int i0, int G,
-                                                      int m_valid) {
-  const uint64_t rel = rows_t >> i0;
-  uint64_t v = 0;
-  int r = col0 / G, g = col0 - r * G;
-#pragma unroll 1
-  for (int e = 0; e < ncol; ++e) {
-    if (col0 + e < m_valid) v |= ((rel >> r) & 1ull) << e;
-    if (++g == G) { g = 0; ++r; }
-  }
-  return v;
 }
 
 // Maximum over the 32 keys of this warp for each of 8 query rows (visible
@@ -417,6 +447,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   float* mref_buf = reinterpret_cast<float*>(sm + S::MREF_OFF);
   float* xq = reinterpret_cast<float*>(sm + S::XQ_OFF);
   float* fq = reinterpret_cast<float*>(sm + S::FQ_OFF);
+  uint64_t* visq = reinterpret_cast<uint64_t*>(sm + S::VISQ_OFF);
   int* seq_len = reinterpret_cast<int*>(sm + S::TABLE_OFF);
   int* prefix = seq_len + max_batch;
   volatile int* agroups = reinterpret_cast<volatile int*>(sm + S::MISC_OFF + 8);
@@ -452,6 +483,12 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
                  ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  if (warp >= WARP_SOFTMAX0 && threadIdx.x - WARP_SOFTMAX0 * 32 < SPACE_MAX_ROWS) {
+    // this block's visibility words into shared memory (the softmax threads index them by key)
+    static_assert(NB == 1, "one 64-bit word covers the query columns of a block");
+    const int j = threadIdx.x - WARP_SOFTMAX0 * 32;
+    visq[j] = p.visq[mb][j];
+  }
   if (warp == WARP_K && lane == 0)
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_k) : "memory");
   if (warp == WARP_V && lane == 0)
@@ -467,6 +504,32 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   pdl_wait();                                              // global memory from here on
   if (threadIdx.x == 0) TL(2);
   const bool single = p.B == 1;
+  // One sequence, no more kv heads than groups: every head gets `base` groups (piece i of a head
+  // takes tiles i, i + base, ...: its first tile does not depend on the length), and the groups
+  // left over are helpers that each take the last tile of some heads -- the one with the block's
+  // own keys, whose Eq. 5 mask makes it the slowest -- so that no regular piece carries it on top
+  // of its share of the full tiles.
+  const int sp_base = max(p.n_groups / p.H_kv, 1), sp_extra = p.n_groups - sp_base * p.H_kv;
+  const bool sp_helper = group >= sp_base * p.H_kv;
+  const int sp_h = sp_helper ? group - sp_base * p.H_kv : group / sp_base;
+  const int sp_piece = sp_helper ? 0 : group - sp_h * sp_base;
+  const bool early = p.spec && !sp_helper;                 // this group requests Q and its first K tile at once
+  if (early && warp == WARP_K && lane == 0 && !*abort_flag) {
+    // Which head and which first tile a regular group works on does not depend on the length,
+    // so its query rows and its first K tile are requested before the length is even read (one
+    // memory round trip earlier).  Should the length turn out too short for that tile, the S^T
+    // issuer lets both buffers go unused.
+    mbar_expect_tx(BAR(B_QFULL), (uint32_t)n_pad * DH * 2);
+#pragma unroll
+    for (int hf = 0; hf < S::HALVES; ++hf)
+      tma_load_4d(sm_base + S::Q_OFF + hf * (n_pad * 128), &p.tm_q, BAR(B_QFULL), hf * 64, sp_h * p.G, i0, 0);
+    mbar_expect_tx(BAR(B_KFULL), S::TILE_BYTES);
+#pragma unroll
+    for (int hf = 0; hf < S::HALVES; ++hf)
+      tma_load_4d_hint(sm_base + S::K_OFF + hf * (TILE_N * 128), &p.tm_k, BAR(B_KFULL), hf * 64, sp_piece * TILE_N, sp_h, 0,
+                       l2_evict_first_policy());
+    TL(3);
+  }
   if (single) {
     // One sequence (the usual decoding case): the tables have a closed form, so every
     // thread works them out for itself from the one length (identical values, each
@@ -477,21 +540,28 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     const int L = okL ? L0 : -1;
     const int T = okL ? (L + p.n_q + TILE_N - 1) / TILE_N : 0;
     seq_len[0] = L; prefix[0] = 0; prefix[1] = okL ? (T + SHARE_COST) * p.H_kv : 0;
-    int ag = -1;
+    int ag = -1, spec_ok = 0;
     const int W = T * p.H_kv;
-    if (W > 0 && W < 8 * p.n_groups) {
-      const int a = max(1, min(p.n_groups / p.H_kv, T));   // = floor(groups * T / W)
-      if (a * p.H_kv <= p.n_groups) {
-        ag = a * p.H_kv;
-        if (group < ag) {
-          const int h = group / a, piece = group - h * a;
-          const int q = T / a, r = T - q * a;
-          const int t0 = piece * q + min(piece, r);
-          reinterpret_cast<int4*>(seg0)[0] = make_int4(0, h, t0, t0 + q + (piece < r ? 1 : 0));
-          reinterpret_cast<int4*>(seg0)[1] = make_int4(T, L, h * a, a);
-        }
+    if (W > 0 && W < 8 * p.n_groups && p.H_kv <= p.n_groups) {
+      ag = p.n_groups;
+      const bool helpers = sp_extra > 0 && T > sp_base;    // the last tile goes to a helper group
+      const int Treg = helpers ? T - 1 : T;                // tiles cut among the regular pieces
+      const int dn = helpers ? sp_base + 1 : min(sp_base, T);
+      if (!sp_helper) {
+        const int n_mine = sp_piece < Treg ? (Treg - sp_piece + sp_base - 1) / sp_base : 0;
+        spec_ok = (n_mine > 0 && (sp_piece + 1) * TILE_N <= L + p.n_q) ? 1 : 0;   // the requested tile is this share's first
+        reinterpret_cast<int4*>(seg0)[0] = make_int4(0, sp_h, sp_piece, n_mine);
+        reinterpret_cast<int4*>(seg0)[1] = make_int4(T, L, sp_h * (sp_base + 1), dn);
+        seg0[8] = sp_base; seg0[10] = 0; seg0[11] = sp_h * (sp_base + 1) + sp_piece; seg0[12] = n_mine > 0 ? 1 : 0;
+      } else {
+        // helper e: the last tile of heads e, e + extra, e + 2 extra, ...
+        reinterpret_cast<int4*>(seg0)[0] = make_int4(0, sp_h, T - 1, 1);
+        reinterpret_cast<int4*>(seg0)[1] = make_int4(T, L, 0, dn);
+        seg0[8] = 1; seg0[10] = sp_extra; seg0[11] = sp_base + 1;
+        seg0[12] = helpers ? (p.H_kv - sp_h + sp_extra - 1) / sp_extra : 0;
       }
     }
+    seg0[9] = spec_ok;
     *agroups = ag;
   } else if (warp == WARP_SOFTMAX0) {
     // per-sequence tile counts and their running sum, 32 sequences per round
@@ -520,6 +590,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     // aligned mode when a group would get fewer than 8 tiles: groups per (sequence,
     // head) a_b = floor(groups * T_b / W), at least 1 tile each; fall back to the flat
     // cut if that needs more groups than there are
+    if (lane == 0) { seg0[8] = 1; seg0[9] = 0; seg0[10] = 0; seg0[11] = group; seg0[12] = 0; }   // no share yet
+    __syncwarp();
     const int Wv = carry;                                  // list entries (tiles + share costs)
     const int W = Wv - SHARE_COST * p.H_kv * nvalid;       // real tiles
     int acarry = -1;
@@ -542,15 +614,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         }
         const int first = acarry + incl - a * p.H_kv;        // first group of sequence b
         if (a > 0 && group >= first && group < first + a * p.H_kv) {
-          // this group's share: head h, piece `piece` of a.  T = a*q + r: the first r
-          // pieces get q+1 tiles, so the last piece, which also has the tile with
-          // the Eq. 5 mask, is never longer than the others
+          // this group's share: head h, piece `piece` of a (see even_cut)
           const int local = group - first;
           const int h = local / a, piece = local - h * a;
-          const int q = T / a, r = T - q * a;
-          const int t0 = piece * q + min(piece, r);
-          reinterpret_cast<int4*>(seg0)[0] = make_int4(b, h, t0, t0 + q + (piece < r ? 1 : 0));
+          int t0, t1;
+          even_cut(T, L + p.n_q, a, piece, t0, t1);
+          reinterpret_cast<int4*>(seg0)[0] = make_int4(b, h, t0, t1 - t0);
           reinterpret_cast<int4*>(seg0)[1] = make_int4(T, L, first + h * a, a);
+          seg0[12] = 1;
         }
         acarry += __shfl_sync(0xFFFFFFFFu, incl, 31);
       }
@@ -582,7 +653,13 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       const int b_full = is_k ? B_KFULL : B_VFULL, b_empty = is_k ? B_KEMPTY : B_VEMPTY;
       const uint32_t ring = sm_base + (is_k ? S::K_OFF : S::V_OFF);
       const CUtensorMap* tm = is_k ? &p.tm_k : &p.tm_v;
-      uint32_t gt = 0, seg = 0;
+      // Early requests (one sequence): when this share's first tile is the requested one, the K
+      // producer skips the query rows and that tile; when it is not, the two buffers are given
+      // back by the S^T issuer and the rings start one slot further.
+      const uint64_t kv_policy = l2_evict_first_policy();
+      bool pre = early && is_k && seg0[9] != 0;
+      const uint32_t koff = (early && is_k && !pre) ? 1u : 0u;
+      uint32_t gt = 0, seg = koff;
       bool ok = true;
       const uint32_t q_bytes = (uint32_t)n_pad * DH * 2;
       // The very first S^T product needs only Q and the first K tile: V holds back
@@ -594,20 +671,25 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           // the K producer also loads this share's query rows, into the buffer that
           // the share before the previous one used (with one buffer: the previous one)
           const uint32_t qb = seg % S::Q_BUFS, use = seg / S::Q_BUFS;
-          if (use > 0) ok = mbar_wait(BAR(B_QEMPTY + qb), (use - 1) & 1, abort_flag, p.err, 3);
-          if (!ok) break;
-          if (seg == 0) TL(3);
-          mbar_expect_tx(BAR(B_QFULL + qb), q_bytes);
+          if (!pre) {
+            if (use > 0) ok = mbar_wait(BAR(B_QEMPTY + qb), (use - 1) & 1, abort_flag, p.err, 3);
+            if (!ok) break;
+            if (seg == 0) TL(3);
+            mbar_expect_tx(BAR(B_QFULL + qb), q_bytes);
 #pragma unroll
-          for (int hf = 0; hf < S::HALVES; ++hf)
-            tma_load_4d(sm_base + S::Q_OFF + qb * S::Q_BYTES + hf * (n_pad * 128), &p.tm_q, BAR(B_QFULL + qb),
-                        hf * 64, sg.h * p.G, i0, sg.b);
+            for (int hf = 0; hf < S::HALVES; ++hf)
+              tma_load_4d(sm_base + S::Q_OFF + qb * S::Q_BYTES + hf * (n_pad * 128), &p.tm_q, BAR(B_QFULL + qb),
+                          hf * 64, sg.h * p.G, i0, sg.b);
+          }
           ++seg;
         }
-        for (int t = sg.t0; t < sg.t1 && ok; ++t, ++gt) {
-          const int s = gt % n_st;
-          if (gt >= (uint32_t)n_st)
-            ok = mbar_wait(BAR(b_empty + s), ((gt / n_st) - 1) & 1, abort_flag, p.err, is_k ? 1 : 2);
+        for (int j = 0; j < sg.n && ok; ++j, ++gt) {
+          if (pre) { pre = false; continue; }                 // requested before the length was known
+          const int t = sg.tile_at(j);
+          const uint32_t g = gt + koff;
+          const int s = g % n_st;
+          if (g >= (uint32_t)n_st)
+            ok = mbar_wait(BAR(b_empty + s), ((g / n_st) - 1) & 1, abort_flag, p.err, is_k ? 1 : 2);
           if (!ok) break;
           if (v_hold) {
             ok = mbar_wait(BAR(B_KFULL), 0, abort_flag, p.err, 14);
@@ -621,13 +703,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           mbar_expect_tx(BAR(b_full + s), S::TILE_BYTES);
 #pragma unroll
           for (int hf = 0; hf < S::HALVES; ++hf)
-            tma_load_4d(dst + hf * (TILE_N * 128), tm, BAR(b_full + s), hf * 64, kt, sg.h, sg.b);
+            tma_load_4d_hint(dst + hf * (TILE_N * 128), tm, BAR(b_full + s), hf * 64, kt, sg.h, sg.b, kv_policy);
           if (is_k) TL(7);
         }
       }
       // drain: every issued copy must have landed before the block may exit
-      const uint32_t first = gt > (uint32_t)n_st ? gt - n_st : 0;
-      for (uint32_t g = first; g < gt; ++g) mbar_drain(BAR(b_full + g % n_st), (g / n_st) & 1);
+      const uint32_t issued = gt + koff;
+      const uint32_t first = issued > (uint32_t)n_st ? issued - n_st : 0;
+      for (uint32_t g = first; g < issued; ++g) mbar_drain(BAR(b_full + g % n_st), (g / n_st) & 1);
       if (is_k && seg > 0) {
         mbar_drain(BAR(B_QFULL + (seg - 1) % S::Q_BUFS), ((seg - 1) / S::Q_BUFS) & 1);
         if (S::Q_BUFS == 2 && seg > 1) mbar_drain(BAR(B_QFULL + (seg - 2) % 2), ((seg - 2) / 2) & 1);
@@ -641,16 +724,25 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       // only adds to the 14-bit address field (16-byte units, no carry possible)
       const uint64_t kdesc0 = smem_desc(sm_base + S::K_OFF, 16, 1024);           // K-major rows of 128 bytes
       const uint64_t qdesc0 = smem_desc(sm_base + S::Q_OFF, 16, 1024);
-      uint32_t gt = 0, seg = 0;
+      uint32_t gt = 0, seg = 0, koff = 0;
       bool ok = true;
+      if (early && seg0[9] == 0) {
+        // the early requests do not serve this group's first share: once they have landed their
+        // buffers go back to the producer unused
+        ok = mbar_wait(BAR(B_QFULL), 0, abort_flag, p.err, 15);
+        if (ok) ok = mbar_wait(BAR(B_KFULL), 0, abort_flag, p.err, 16);
+        mbar_arrive(BAR(B_QEMPTY));
+        mbar_arrive(BAR(B_KEMPTY));
+        seg = 1; koff = 1;
+      }
       while (ok && part.next(sg)) {
         const uint32_t qb = seg % S::Q_BUFS, use = seg / S::Q_BUFS;
         ok = mbar_wait(BAR(B_QFULL + qb), use & 1, abort_flag, p.err, 6);
         const uint64_t qd = qdesc0 + (uint64_t)((qb * S::Q_BYTES) >> 4);
-        const int n = sg.t1 - sg.t0;
+        const int n = sg.n;
         for (int j = 0; j < n && ok; ++j, ++gt) {
-          const int s = gt % S::K_STAGES, buf = gt & 1;
-          ok = mbar_wait(BAR(B_KFULL + s), (gt / S::K_STAGES) & 1, abort_flag, p.err, 7);
+          const int s = (gt + koff) % S::K_STAGES, buf = gt & 1;
+          ok = mbar_wait(BAR(B_KFULL + s), ((gt + koff) / S::K_STAGES) & 1, abort_flag, p.err, 7);
           if (gt == 0) TL(4);
           // S^T buffer `buf` was last read by the softmax of tile gt-2
           if (ok && gt >= 2) ok = mbar_wait(BAR(B_PREADY + buf), ((gt - 2) >> 1) & 1, abort_flag, p.err, 8);
@@ -690,7 +782,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       uint32_t g = 0;
       bool ok = true;
       while (ok && part.next(sg)) {
-        for (int t = sg.t0; t < sg.t1 && ok; ++t, ++g) {
+        for (int j = 0; j < sg.n && ok; ++j, ++g) {
           const int s = g % S::V_STAGES;
           ok = mbar_wait(BAR(B_VFULL + s), (g / S::V_STAGES) & 1, abort_flag, p.err, 4);
           if (ok) ok = mbar_wait(BAR(B_PREADY + (g & 1)), (g >> 1) & 1, abort_flag, p.err, 5);
@@ -703,7 +795,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
             // 16 keys further = 2048 bytes further in both operands; the first
             // product of a share overwrites O^T
             mma_ss(TM_O, ad0 + (uint64_t)((kk * 2048) >> 4), pd0 + (uint64_t)((kk * 2048) >> 4), idesc_pv,
-                   (t == sg.t0 && kk == 0) ? 0u : 1u);
+                   (j == 0 && kk == 0) ? 0u : 1u);
           }
           tc_commit(BAR(B_VEMPTY + s));
           tc_commit(BAR(B_PVDONE + (g & 1)));
@@ -744,9 +836,10 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       for (int j = 0; j < MAXP; ++j)
 #pragma unroll
         for (int e = 0; e < 8; ++e) lsum[j][e] = 0.f;
-      for (int t = sg.t0; t < sg.t1; ++t, ++gt) {
+      for (int jt = 0; jt < sg.n; ++jt, ++gt) {
+        const int t = sg.tile_at(jt);
         const int buf = gt & 1;
-        const bool first = (t == sg.t0);
+        const bool first = (jt == 0);
         ok &= mbar_wait(BAR(B_SFULL + buf), (gt >> 1) & 1, abort_flag, p.err, 9);
         tc_fence_after();
         if (sidx == 0) { if (gt == 0) TL(5); TL(8); }
@@ -766,22 +859,47 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         uint64_t vis = ~0ull;
         if (masked) {
           if (key < lo) vis = 0ull;
-          else if (jb >= 0) vis = block_key_visibility(p.mask_t[jb], col0, ncol, i0, p.G, m_valid);
+          else if (jb >= 0) vis = visq[jb] >> col0;         // (bits past this thread's columns are never looked at)
         }
-        // ---- first tile of a share, every key visible: the scores of the tile's
-        // first key serve as references.  Any reference within 2^60 of the row
-        // maximum is as good as the maximum itself (P keeps its relative precision
-        // as P_hi + P_lo, sums are fp32); pass 0 below checks exactly that bound.
-        if (first && !masked) {
+        // ---- first tile of a share: references from scores at hand.  Any reference within
+        // 2^60 of the row maximum is as good as the maximum itself (P keeps its relative
+        // precision as P_hi + P_lo, sums are fp32); pass 0 below checks exactly that bound.
+        // Every row sees every cached key, so the scores of the tile's first cached key that
+        // counts serve all rows.  A tile without one holds block keys only (it is then the last
+        // tile of its sequence): a row's own key is always visible to it (Eq. 5) and gives its
+        // reference; rows before the tile's first block key see nothing here and get -inf.
+        if (first) {
           float* mnew = mref_buf + (mpar ^ 1) * S::RS;
-          if (kl == 0) {
+          const int vstart = max(kt, lo);                    // first key of the tile that counts
+          if (vstart < sg.L) {
+            if (key == vstart) {
+#pragma unroll
+              for (int j = 0; j < MAXP; ++j) {
+                if (j < np) {
+                  float4* dst = reinterpret_cast<float4*>(mnew + col0 + j * 8);
+                  dst[0] = make_float4(sv[j][0] * c, sv[j][1] * c, sv[j][2] * c, sv[j][3] * c);
+                  dst[1] = make_float4(sv[j][4] * c, sv[j][5] * c, sv[j][6] * c, sv[j][7] * c);
+                }
+              }
+            }
+          } else {
+            // block keys only: every thread parks its raw scores in the P buffer (idle until pass 1
+            // of this very tile), then one thread per query column fetches the score of that
+            // row's own key
+            float* stage = reinterpret_cast<float*>(sm + S::P_OFF) + kl * 64 + col0;
 #pragma unroll
             for (int j = 0; j < MAXP; ++j) {
               if (j < np) {
-                float4* dst = reinterpret_cast<float4*>(mnew + col0 + j * 8);
-                dst[0] = make_float4(sv[j][0] * c, sv[j][1] * c, sv[j][2] * c, sv[j][3] * c);
-                dst[1] = make_float4(sv[j][4] * c, sv[j][5] * c, sv[j][6] * c, sv[j][7] * c);
+                reinterpret_cast<float4*>(stage + j * 8)[0] = make_float4(sv[j][0], sv[j][1], sv[j][2], sv[j][3]);
+                reinterpret_cast<float4*>(stage + j * 8)[1] = make_float4(sv[j][4], sv[j][5], sv[j][6], sv[j][7]);
               }
+            }
+            soft_sync();
+            if (sidx < n_pad) {
+              const int i = i0 + (sidx >> (__ffs(p.G) - 1));  // block row of query column sidx
+              const int krow = sg.L + i - kt;                  // its own key's place in the tile
+              const bool seen = sidx < m_valid && sg.L + i >= vstart;
+              mnew[sidx] = seen ? reinterpret_cast<const float*>(sm + S::P_OFF)[krow * 64 + sidx] * c : -CUDART_INF_F;
             }
           }
           soft_sync();
@@ -789,7 +907,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           mref = mref_buf + mpar * S::RS;
         }
         // ---- pass 0: score - reference; does any exceed 2^60? -----------------
-        bool over = first && masked;
+        bool over = false;
         if (!over) {
           // (independent maxima per piece: a single running flag would chain every element)
           float worst[MAXP];
@@ -934,7 +1052,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       tc_fence_after();
       soft_sync();
       if (sidx == 0) TL(10);
-      const bool whole = (sg.t0 == 0 && sg.t1 == sg.T);
+      const bool whole = sg.n == sg.T;
       const int item = sg.b * p.H_kv + sg.h;
       float* pslot = p.part + ((size_t)sg.slot * p.n_mblocks + mb) * (ROWS * (DH + 2));
       if (sidx == 0 && ok) {
@@ -953,7 +1071,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           d.y = group_of(f0 + SHARE_COST + sg.T - 1, W, NG) - g0 + 1;
         }
         p.desc[(size_t)item * p.n_mblocks + mb] = d;
-        if (sg.t0 > 0 && sg.t1 == sg.T) own = item;        // at most one per block: only its first share can start late
+        if (!whole && sg.tile_at(sg.n - 1) == sg.T - 1) own = item;   // the piece with the pair's last tile; at most one per block
       }
       if (sidx < m_valid && ok) {                           // per-row scalars
         const int q = sidx;
@@ -1158,7 +1276,15 @@ size_t smem_bytes(int max_batch) {
 template <int DH, int NB>
 cudaError_t launch_main(const AttnParams& p, int n_ctas, int max_batch, cudaStream_t st) {
   const size_t sm = smem_bytes<DH, NB>(max_batch);
-  cudaFuncSetAttribute(attn_tc_kernel<DH, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+  // the shared-memory limit of the kernel is raised once per device (to the most any batch needs)
+  static unsigned long long done_mask = 0;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 64 || !((done_mask >> dev) & 1ull)) {
+    cudaFuncSetAttribute(attn_tc_kernel<DH, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)smem_bytes<DH, NB>(128));
+    if (dev < 64) done_mask |= 1ull << dev;
+  }
   return launch_pdl(attn_tc_kernel<DH, NB>, dim3(n_ctas), dim3(THREADS), sm, st, p, max_batch);
 }
 
@@ -1209,12 +1335,22 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   p.desc = reinterpret_cast<int2*>(ctx->merge_cnt);
   p.owner = ctx->merge_cnt + (size_t)cfg.max_batch * cfg.n_kv_heads * 8 * 2;
   p.merge_by_owner = (a->batch * p.H_kv * p.n_mblocks > pl.n_ctas) ? 1 : 0;
-  for (int i = 0; i < SPACE_MAX_ROWS; ++i) p.mask[i] = mask_rows[i];
-  for (int j = 0; j < SPACE_MAX_ROWS; ++j) {
-    uint64_t t = 0;
-    for (int i = 0; i < SPACE_MAX_ROWS; ++i) t |= ((mask_rows[i] >> j) & 1ull) << i;
-    p.mask_t[j] = t;
+  p.spec = (a->batch == 1 && p.H_kv <= p.n_groups) ? 1 : 0;
+  if (p.n_mblocks > 2) return SPACE_E_UNSUPPORTED;         // (cannot happen: at most 64 block rows, at least 32 per block)
+  if (ctx->visq_k != a->k || ctx->visq_variant != a->mask_variant) {
+    memset(ctx->visq, 0, sizeof(ctx->visq));
+    for (int m = 0; m < p.n_mblocks; ++m) {
+      const int i0 = m * p.rows_per_mb;
+      const int rows = (p.n_q - i0 < p.rows_per_mb ? p.n_q - i0 : p.rows_per_mb);
+      for (int j = 0; j < SPACE_MAX_ROWS; ++j) {
+        uint64_t v = 0;
+        for (int q = 0; q < rows * p.G; ++q) v |= ((mask_rows[i0 + q / p.G] >> j) & 1ull) << q;
+        ctx->visq[m][j] = v;
+      }
+    }
+    ctx->visq_k = a->k; ctx->visq_variant = a->mask_variant;
   }
+  memcpy(p.visq, ctx->visq, sizeof(p.visq));
 
   // TMA descriptors, rebuilt only when a base pointer or a stride changes
   const int64_t key[8] = {a->kv_stride_b, a->kv_stride_h, a->kv_stride_s, a->batch, p.n_q, p.n_pad, 0, 0};

@@ -83,6 +83,11 @@ struct space_ctx {
   int prof_on;
   int prof_n[SPACE_K_COUNT];
   cudaEvent_t* prof_ev[SPACE_K_COUNT];   // [2 * SPACE_PROFILE_MAX_STEPS] start/stop pairs, lazily created
+  // cached block layout (Eq. 5 mask rows) and the attention kernel's visibility words, per (k, mask variant)
+  int lay_k, lay_variant;                // lay_k = 0: nothing cached
+  uint64_t lay_mask[SPACE_MAX_ROWS];
+  int visq_k, visq_variant;
+  uint64_t visq[2][SPACE_MAX_ROWS];
   // cached TMA descriptors
   const void* tm_q_ptr; const void* tm_k_ptr; const void* tm_v_ptr;
   int64_t tm_key[8];

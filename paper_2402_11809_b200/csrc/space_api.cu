@@ -237,12 +237,16 @@ int space_attn_step(space_ctx* ctx, const space_attn_args* a, void* stream) {
   if (a->kv_stride_s < ctx->cfg.head_dim || a->kv_stride_b < 1 || a->kv_stride_h < 1) return SPACE_E_INVALID_ARG;
   if (a->kv_stride_b % 8 || a->kv_stride_h % 8 || a->kv_stride_s % 8) return SPACE_E_ALIGNMENT;
   if (!use_device(ctx)) return SPACE_E_CUDA;
-  space_layout_t lay;
-  build_layout(a->k, a->mask_variant, &lay);
+  if (ctx->lay_k != a->k || ctx->lay_variant != a->mask_variant) {   // the layout is rebuilt only when k or the reading changes
+    space_layout_t lay;
+    build_layout(a->k, a->mask_variant, &lay);
+    memcpy(ctx->lay_mask, lay.mask, sizeof(ctx->lay_mask));
+    ctx->lay_k = a->k; ctx->lay_variant = a->mask_variant;
+  }
   cudaStream_t st = (cudaStream_t)stream;
-  if (a->impl == SPACE_ATTN_SIMT) return launch_attn_simt(ctx, a, lay.mask, st);
+  if (a->impl == SPACE_ATTN_SIMT) return launch_attn_simt(ctx, a, ctx->lay_mask, st);
   if (a->impl != SPACE_ATTN_TENSOR && a->impl != SPACE_ATTN_TENSOR_ROWS) return SPACE_E_INVALID_ARG;
-  return launch_attn_tensor(ctx, a, lay.mask, st);
+  return launch_attn_tensor(ctx, a, ctx->lay_mask, st);
 }
 
 int space_verify(space_ctx* ctx, const space_verify_args* a, void* stream) {
