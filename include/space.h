@@ -328,6 +328,18 @@ int space_debug_philox(space_ctx* ctx, uint64_t seed, int64_t n, const uint32_t*
                        const uint32_t* c1, const uint32_t* c2, const uint32_t* c3,
                        uint32_t* out, void* stream);
 
+/* Test hook for the bounded on-chip waits (every mbarrier wait of the tensor-core
+ * kernels gives up after one second, sets SPACE_ST_TIMEOUT and lets the block drain;
+ * no wait in the library is unbounded).  Launches one small kernel that waits, with that
+ * same wait routine and a limit of limit_ns (1 .. 10^8 ns), on a barrier nothing ever
+ * arrives on.  The kernel returns normally; the context stays usable.
+ * out4: device int32[4], written as {status bits: SPACE_ST_TIMEOUT when the wait expired,
+ * 8 if a later wait did not also give up, 16 when the block's abort flag was set;
+ * the recorded site (77); microseconds the expired wait took; microseconds a second
+ * wait took (about 0: a block that has given up never blocks again)}.
+ * Errors: INVALID_ARG (NULL, limit out of range), CUDA. */
+int space_debug_wait_timeout(space_ctx* ctx, uint64_t limit_ns, int32_t* out4, void* stream);
+
 const char* space_strerror(int code);
 
 #ifdef __cplusplus

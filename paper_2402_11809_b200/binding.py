@@ -30,7 +30,7 @@ EXPORTS = ["space_create", "space_destroy", "space_workspace_bytes", "space_layo
            "space_lmhead_verify",
            "space_step_host",
            "space_launch_count", "space_profile_enable", "space_profile_read",
-           "space_debug_philox", "space_strerror"]
+           "space_debug_philox", "space_debug_wait_timeout", "space_strerror"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -130,6 +130,8 @@ lib.space_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C
 lib.space_profile_read.restype = C.c_int
 lib.space_debug_philox.argtypes = [C.c_void_p, C.c_uint64, C.c_int64] + [C.c_void_p] * 6
 lib.space_debug_philox.restype = C.c_int
+lib.space_debug_wait_timeout.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p]
+lib.space_debug_wait_timeout.restype = C.c_int
 lib.space_strerror.argtypes = [C.c_int]
 lib.space_strerror.restype = C.c_char_p
 
@@ -282,6 +284,10 @@ class Context:
     # -- space_step_host --------------------------------------------------
     def space_step_host(self, args):
         _check(lib.space_step_host(self._h, C.byref(args), _stream()))
+
+    def space_debug_wait_timeout(self, limit_ns, out4):
+        """Let a bounded on-chip wait run out (see include/space.h); out4: int32 CUDA tensor of 4."""
+        _check(lib.space_debug_wait_timeout(self._h, int(limit_ns), _ptr(out4), _stream()))
 
     def space_debug_philox(self, seed, c0, c1, c2, c3, out):
         _check(lib.space_debug_philox(self._h, seed, c0.numel(), _ptr(c0), _ptr(c1), _ptr(c2),

@@ -8,8 +8,8 @@
 // maximum, sum, accumulator) in scratch memory; attn_merge_kernel combines the
 // partials of every (sequence, head) that was cut.
 //
-// The query block of one kv head is small (the (k+1)^2 block rows times the GQA
-// group: 25 to 112 rows), so the two tile products are taken transposed: the
+// The query block of one kv head is small here (the (k+1)^2 block rows times the GQA
+// group, at most 64 rows; wider blocks go to attn_rows.cu), so the two tile products are taken transposed: the
 // 128 keys of a tile are the MMA M extent and the query rows the N extent,
 //   S^T = K Q^T   (128 x N),      O^T += V^T (P_hi + P_lo)^T   (head_dim x N),
 // which costs N/128 of a full tile and puts one key on every TMEM lane.
@@ -29,7 +29,14 @@
 //           across keys once per share.
 // Every wait is bounded; an expired wait sets SPACE_ST_TIMEOUT and the block
 // drains and exits.
+//
+// One sequence (the usual decoding case) takes a partition of its own: every kv head gets the
+// same number of groups, piece i of a head takes tiles i, i + pieces, ... (so a group's first
+// tile does not depend on the length and is requested, with the query rows, before the length
+// is read), and the groups left over take the heads' last tiles, the ones with the block's own
+// keys and the Eq. 5 mask.
 #include "common.cuh"
+#include "tc_common.cuh"
 #include <cuda.h>
 #include <math_constants.h>
 
@@ -81,112 +88,13 @@ __device__ unsigned long long g_timeline[256 * TL_POINTS];
 #define TL(i) do { } while (0)
 #endif   // slot: partial slot; dfirst/dn: cut (aligned mode)
 
-// ---------------------------------------------------------------- PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
+// PTX helpers: tc_common.cuh.  Every wait of this kernel is bounded by WAIT_NS.
+using namespace tc;
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err, int site) {
+  return mbar_wait_bounded(bar, parity, abort_flag, err, site, WAIT_NS, 64);   // sleeps between polls
 }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.b32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait (WAIT_NS of wall time).  Returns false when the limit expired or
-// another thread of the block gave up; the first expiry records its site.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* err, int site) {
-  if (*abort_flag) return mbar_try(bar, parity);            // draining: never block
-  uint64_t t0 = 0;
-  for (uint32_t it = 0;; ++it) {
-    if (mbar_try(bar, parity)) return true;
-    __nanosleep(64);                                        // leave the issue slots to the working warps
-    if ((it & 255u) == 255u) {
-      if (*abort_flag) return false;
-      const uint64_t now = global_ns();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > WAIT_NS) break;
-    }
-  }
-  *abort_flag = 1;
-  atomicCAS(err, 0, site);
-  return false;
-}
-// Bounded wait without the abort protocol (used while draining before exit).
-__device__ __noinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
-  uint64_t t0 = 0;
-  for (uint32_t it = 0;; ++it) {
-    if (mbar_try(bar, parity)) return;
-    if ((it & 255u) == 255u) {
-      const uint64_t now = global_ns();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > WAIT_NS) return;
-    }
-  }
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
-                                            int c0, int c1, int c2, int c3) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"((uint64_t)tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-// The same load with an L2 policy: K and V tiles are read once per step, so their lines are marked
-// to be evicted first and leave the cache to what is read again (code, lengths, partials).
-__device__ __forceinline__ uint64_t l2_evict_first_policy() {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-  return pol;
-}
-__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
-                                                 int c0, int c1, int c2, int c3, uint64_t pol) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
-      " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
-      ::"r"(dst), "l"((uint64_t)tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after()  { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __noinline__ void mbar_drain(uint32_t bar, uint32_t parity) { mbar_drain_bounded(bar, parity, WAIT_NS); }
 
-// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
-// lbo / sbo in bytes.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr >> 4) & 0x3FFF);
-  d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
-  d |= (uint64_t)((sbo >> 4) & 0x3FFF) << 32;
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)2 << 61;
-  return d;
-}
 // ------------------------------------------------------------ work partition
 // Flat tile index space: sequence-major, then kv head, then tile.  Group g of
 // n_groups owns flat tiles [W*g/n_groups, W*(g+1)/n_groups).
@@ -290,21 +198,20 @@ __device__ __forceinline__ int group_of(long long f, long long W, long long NG) 
   return (int)(num / (unsigned long long)W);
 }
 
-// Shared-memory plan.  NB = number of 64-query blocks a thread block handles
-// (1: up to 64 query rows, 2: up to 128).
-template <int DH, int NB>
+// Shared-memory plan (up to 64 query rows per thread block).
+template <int DH>
 struct Smem {
   static constexpr int HALVES = DH / 64;
   static constexpr int TILE_BYTES = TILE_N * DH * 2;         // one K or V tile
-  static constexpr int Q_ROWS = NB == 1 ? 64 : 112;          // query rows (with padding) per thread block
+  static constexpr int Q_ROWS = 64;                          // query rows (with padding) per thread block
   static constexpr int Q_BYTES = Q_ROWS * DH * 2;
-  static constexpr int P_PART = NB * TILE_N * 128;           // P_hi or P_lo: [block][key][64 queries] bf16
+  static constexpr int P_PART = TILE_N * 128;                // P_hi or P_lo: [key][64 queries] bf16
   static constexpr int K_STAGES = (DH == 128) ? 2 : 3;
   static constexpr int V_STAGES = (DH == 128) ? 2 : 4;
   static constexpr int P_BUFS = 1;                           // P^T buffers (each P_hi + P_lo); a second one, so that the exponentials of a tile
                                                              // overlap the O^T product of the tile before, measured no faster
-  static constexpr int RS = 64 * NB;                         // query rows (padded) per thread block at most
-  static constexpr int Q_BUFS = NB == 1 ? 2 : 1;             // query buffers: the next share's rows load early
+  static constexpr int RS = 64;                              // query rows (padded) per thread block at most
+  static constexpr int Q_BUFS = 2;                           // query buffers: the next share's rows load early
   static constexpr int Q_OFF = 0;
   static constexpr int K_OFF = Q_BUFS * Q_BYTES;
   static constexpr int V_OFF = K_OFF + K_STAGES * TILE_BYTES;
@@ -324,11 +231,6 @@ struct Smem {
   static_assert(TABLE_OFF + (2 * 128 + 1) * 4 <= 227 * 1024, "shared-memory plan too large");
 };
 
-__device__ __forceinline__ float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 // Barrier over the 256 softmax threads (id 1); the second form also ORs a predicate.
 __device__ __forceinline__ void soft_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ bool soft_any(bool pred) {
@@ -430,10 +332,10 @@ constexpr float OVER_THRESHOLD = 60.f;   // re-reference a query row when a scor
 // and O^T += V^T P^T (head_dim x N), so the MMA N extent is the number of
 // query rows rounded up to 16 instead of a full 128-row tile, and one thread
 // owns one key of the tile (all 128 TMEM lanes carry work).
-template <int DH, int NB>
+template <int DH>
 __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_constant__ AttnParams p,
                                                              int max_batch) {
-  using S = Smem<DH, NB>;
+  using S = Smem<DH>;
   extern __shared__ __align__(1024) unsigned char sm[];
   const uint32_t sm_base = smem_u32(sm);
   const uint32_t bar0 = sm_base + S::BAR_OFF;
@@ -485,7 +387,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   }
   if (warp >= WARP_SOFTMAX0 && threadIdx.x - WARP_SOFTMAX0 * 32 < SPACE_MAX_ROWS) {
     // this block's visibility words into shared memory (the softmax threads index them by key)
-    static_assert(NB == 1, "one 64-bit word covers the query columns of a block");
     const int j = threadIdx.x - WARP_SOFTMAX0 * 32;
     visq[j] = p.visq[mb][j];
   }
@@ -635,7 +536,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   if (!single) __syncthreads();                            // the tables of warp 4 reach every warp
   const uint32_t tmem = *tmem_slot;
   // TMEM columns: S^T buffers at 0 and 128 (n_pad <= 128 columns each), [O_hi^T | O_lo^T] at 256
-  // (64*NB columns each)
+  // (64 columns each)
   const uint32_t TM_S0 = tmem, TM_O = tmem + 256;
 
   Partition part;
@@ -774,9 +675,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       // O_lo^T in columns 64..127 (an instruction costs the same at every N here);
       // the epilogue adds the two.  Columns past the padded query rows hold whatever
       // the shared memory held; they only reach output columns nobody reads.
-      const uint32_t idesc_pv = instr_desc_rt(128 * NB, 1, 1);   // A = V^T (d contiguous), B = P^T (queries contiguous)
+      const uint32_t idesc_pv = instr_desc_rt(128, 1, 1);   // A = V^T (d contiguous), B = P^T (queries contiguous)
       // V^T and P^T: 64-wide blocks TILE_N*128 bytes apart, 8-key groups 1024 bytes apart
-      static_assert(S::P_PART == NB * TILE_N * 128, "P_lo must follow the NB blocks of P_hi at the block stride");
+      static_assert(S::P_PART == TILE_N * 128, "P_lo must follow P_hi at the block stride");
       const uint64_t vdesc0 = smem_desc(sm_base + S::V_OFF, TILE_N * 128, 1024);
       const uint64_t pdesc0 = smem_desc(sm_base + S::P_OFF, TILE_N * 128, 1024);
       uint32_t g = 0;
@@ -810,7 +711,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     // ================= softmax / epilogue ==================================
     // One key of the tile per TMEM lane; two threads per key, each with one half
     // of the query-row columns, handled in pieces of 8 columns.
-    constexpr int MAXP = NB == 1 ? 4 : 7;                  // pieces per thread at most
+    constexpr int MAXP = 4;                                // pieces per thread at most
     const int quarter = warp & 3;                          // TMEM lane quarter this warp may touch
     const int half = (warp - WARP_SOFTMAX0) >> 2;
     const int kl = quarter * 32 + lane;                    // key within the tile; head-dim index in the epilogue
@@ -959,7 +860,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
 #pragma unroll
                 for (int e = 0; e < 8; ++e) lsum[j][e] *= fq[q0 + e];
                 piece_rescale(TM_O + lane_addr + q0, fq + q0);
-                piece_rescale(TM_O + lane_addr + 64 * NB + q0, fq + q0);
+                piece_rescale(TM_O + lane_addr + 64 + q0, fq + q0);
               }
               // scores again, now against the new reference
               uint32_t sr[8];
@@ -1098,7 +999,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         uint32_t o[8], o2[8];
         const int q0 = col0 + j * 8;
         tmem_ld8(TM_O + lane_addr + q0, o);
-        tmem_ld8(TM_O + lane_addr + 64 * NB + q0, o2);
+        tmem_ld8(TM_O + lane_addr + 64 + q0, o2);
         tmem_wait_ld();
 #pragma unroll
         for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) + __uint_as_float(o2[e]));
@@ -1268,24 +1169,24 @@ void plan(const space_config* cfg, int sm_count, int k, AttnPlanHost* pl) {
   pl->n_ctas = groups * pl->n_mblocks;
 }
 
-template <int DH, int NB>
+template <int DH>
 size_t smem_bytes(int max_batch) {
-  return Smem<DH, NB>::TABLE_OFF + (size_t)(2 * max_batch + 1) * sizeof(int);
+  return Smem<DH>::TABLE_OFF + (size_t)(2 * max_batch + 1) * sizeof(int);
 }
 
-template <int DH, int NB>
+template <int DH>
 cudaError_t launch_main(const AttnParams& p, int n_ctas, int max_batch, cudaStream_t st) {
-  const size_t sm = smem_bytes<DH, NB>(max_batch);
+  const size_t sm = smem_bytes<DH>(max_batch);
   // the shared-memory limit of the kernel is raised once per device (to the most any batch needs)
   static unsigned long long done_mask = 0;
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 64 || !((done_mask >> dev) & 1ull)) {
-    cudaFuncSetAttribute(attn_tc_kernel<DH, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         (int)smem_bytes<DH, NB>(128));
+    cudaFuncSetAttribute(attn_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)smem_bytes<DH>(128));
     if (dev < 64) done_mask |= 1ull << dev;
   }
-  return launch_pdl(attn_tc_kernel<DH, NB>, dim3(n_ctas), dim3(THREADS), sm, st, p, max_batch);
+  return launch_pdl(attn_tc_kernel<DH>, dim3(n_ctas), dim3(THREADS), sm, st, p, max_batch);
 }
 
 }  // namespace
@@ -1378,10 +1279,8 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   const dim3 mgrid(p.merge_by_owner ? pl.n_ctas : a->batch * p.H_kv * p.n_mblocks, (m_valid_max * (DH / 4) + 127) / 128);
   {
     ProfScope ps(ctx, SPACE_K_ATTN, st);
-    // (the two-block form NB = 2 of this kernel works but measured slower than the
-    // row-orientation kernel on every wide workload, so it is not instantiated)
-    if (DH == 128) launch_main<128, 1>(p, pl.n_ctas, cfg.max_batch, st);
-    else launch_main<64, 1>(p, pl.n_ctas, cfg.max_batch, st);
+    if (DH == 128) launch_main<128>(p, pl.n_ctas, cfg.max_batch, st);
+    else launch_main<64>(p, pl.n_ctas, cfg.max_batch, st);
   }
   {
     ProfScope ps(ctx, SPACE_K_MERGE, st);

@@ -1,6 +1,7 @@
 // Host side of libspace: context, argument validation, block layout, and the
 // exported entry points declared in include/space.h.
 #include "common.cuh"
+#include "tc_common.cuh"
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -132,6 +133,28 @@ int check_commit_args(const space_ctx* ctx, const space_commit_args* a) {
   if (a->kv_stride_b % 8 || a->kv_stride_h % 8 || a->kv_stride_s % 8) return SPACE_E_ALIGNMENT;
   if (a->kv_stride_s < ctx->cfg.head_dim) return SPACE_E_INVALID_ARG;
   return SPACE_OK;
+}
+
+// Test hook kernel: one mbarrier that nothing ever arrives on, waited for with the bounded wait
+// every tensor-core kernel of the library uses.  The wait gives up after limit_ns, the kernel
+// reports what it saw and returns normally: nothing faults, traps or spins without a bound.
+__global__ void wait_timeout_kernel(unsigned long long limit_ns, int32_t* out) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x != 0) return;
+  abort_flag = 0;
+  const uint32_t b = tc::smem_u32(&bar);
+  tc::mbar_init(b, 1);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  int* err = out + 1;                                       // first time-out site (zeroed by the host)
+  const unsigned long long t0 = tc::global_ns();
+  const bool ok = tc::mbar_wait_bounded(b, 0, &abort_flag, err, 77, limit_ns, 64);
+  const unsigned long long t1 = tc::global_ns();
+  const bool again = tc::mbar_wait_bounded(b, 0, &abort_flag, err, 78, limit_ns, 64);   // draining: returns at once
+  const unsigned long long t2 = tc::global_ns();
+  out[0] = (ok ? 0 : SPACE_ST_TIMEOUT) | (again ? 8 : 0) | (abort_flag ? 16 : 0);
+  out[2] = (int32_t)((t1 - t0) / 1000ull);                  // microseconds the first wait took
+  out[3] = (int32_t)((t2 - t1) / 1000ull);                  // and the second
 }
 
 }  // namespace
@@ -472,6 +495,15 @@ int space_debug_philox(space_ctx* ctx, uint64_t seed, int64_t n, const uint32_t*
   if (!ctx || n < 0 || (n > 0 && (!c0 || !c1 || !c2 || !c3 || !out))) return SPACE_E_INVALID_ARG;
   if (!use_device(ctx)) return SPACE_E_CUDA;
   return launch_philox_debug(seed, n, c0, c1, c2, c3, out, (cudaStream_t)stream);
+}
+
+int space_debug_wait_timeout(space_ctx* ctx, uint64_t limit_ns, int32_t* out4, void* stream) {
+  if (!ctx || !out4 || limit_ns == 0 || limit_ns > 100000000ull) return SPACE_E_INVALID_ARG;   // at most 0.1 s
+  if (!use_device(ctx)) return SPACE_E_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemsetAsync(out4, 0, 4 * sizeof(int32_t), st) != cudaSuccess) return SPACE_E_CUDA;
+  wait_timeout_kernel<<<1, 32, 0, st>>>((unsigned long long)limit_ns, out4);
+  return cuda_ok(cudaGetLastError());
 }
 
 const char* space_strerror(int code) {

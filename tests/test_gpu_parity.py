@@ -456,3 +456,30 @@ def test_config_gqa70b(B, H):
 def test_config_sampling64(B, H):
     n = _run_config(B, H, "sampling64", heads_per_seq=1, fused=True)
     assert n.mean() > 0.5
+
+
+# ------------------------------------------------------------- bounded waits
+def test_bounded_wait_runs_out_and_the_context_stays_usable(B, H):
+    # The wait routine of the tensor-core kernels on a barrier nothing arrives on: it must give up
+    # after its limit, report SPACE_ST_TIMEOUT with the recorded site, never block again, and leave
+    # the context fit for an ordinary call.  Nothing faults or hangs: the kernel waits, gives up
+    # and returns.
+    cfg = _small_cfg(3, (100, 200), Bn=2, seed=55)
+    x = workloads.make_step_inputs(cfg)
+    ctx = H.make_context(cfg, x)
+    out4 = torch.full((4,), -1, dtype=torch.int32, device="cuda")
+    ctx.space_debug_wait_timeout(200_000, out4)             # 200 microseconds
+    torch.cuda.synchronize()
+    st, site, us_first, us_second = out4.cpu().tolist()
+    assert st & B.ST_TIMEOUT and st & 16 and not st & 8
+    assert site == 77
+    assert 150 <= us_first <= 5000 and us_second <= 50
+    import ctypes as C
+    assert B.lib.space_debug_wait_timeout(ctx._h, 0, C.c_void_p(out4.data_ptr()), None) == B.E_INVALID_ARG
+    assert B.lib.space_debug_wait_timeout(ctx._h, 10 ** 9, C.c_void_p(out4.data_ptr()), None) == B.E_INVALID_ARG
+    ds = H.DeviceStep(cfg, x)
+    ds.attn(ctx)
+    torch.cuda.synchronize()
+    ref, _ = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], 3, x["scale"])
+    _check_attention(H, ds.out.cpu().numpy().astype(np.float64), ref, "after a time-out")
+    assert int(ds.status.abs().sum()) == 0
