@@ -303,6 +303,51 @@ int space_kv_commit(space_ctx* ctx, const space_commit_args* args, void* stream)
  * or sizes beyond cfg), CUDA. */
 int space_step_host(space_ctx* ctx, const space_host_step_args* args, void* stream);
 
+/* Device-resident state of the decoding loop (Algorithm 1 in full): the generated
+ * tokens O, the candidates L_c with their probabilities P_c, the verified length, the
+ * <EOS> latch, and the token and position ids of the block rows the next model call
+ * evaluates (Eq. 4: the last verified token, then every candidate followed by k mask
+ * tokens; Sec. 3.2: position = visible keys - 1).  All arrays are device memory owned
+ * by the caller; the library only reads and writes them in the two calls below. */
+typedef struct {
+  int32_t batch, k;
+  int32_t max_tokens;       /* capacity of `tokens` per sequence; a full buffer ends the sequence */
+  int32_t mask_token_id;    /* id of the mask token [M]                                       */
+  int32_t mask_variant;     /* SPACE_MASK_*: the reading of Eq. 5 the position ids follow     */
+  int32_t reserved;         /* 0                                                              */
+  int32_t* tokens;          /* [B, max_tokens] generated tokens (the prompt is not stored)    */
+  int32_t* n_tokens;        /* [B]   how many of them                                         */
+  int32_t* last_token;      /* [B]   x_l: the last verified token, whose KV is not cached yet */
+  int32_t* cand;            /* [B, k] L_c                                                     */
+  float*   cand_prob;       /* [B, k] P_c                                                     */
+  int32_t* kv_len;          /* [B]   verified cache length L_b (set by the caller's prefill)  */
+  uint8_t* finished;        /* [B]   1 once <EOS> was met or the token buffer is full; latched */
+  int32_t* block_tokens;    /* [B, (k+1)^2] token ids of the next call's block rows           */
+  int32_t* block_pos;       /* [B, (k+1)^2] their position ids                                */
+} space_decode_state;
+
+/* Initial state of Algorithm 1: no generated token, L_c = [0]*k, P_c = [+inf]*k (so
+ * that the first step accepts nothing in sampling mode), finished = 0, and the block
+ * rows of the first step.  last_prompt_token: device [B], the last token of every
+ * prompt (the cache already holds the tokens before it and state->kv_len says how many).
+ * Asynchronous on `stream`.  Errors: INVALID_ARG, WORKSPACE (batch beyond the context's), CUDA. */
+int space_decode_begin(space_ctx* ctx, const space_decode_state* state, const int32_t* last_prompt_token,
+                       void* stream);
+
+/* End of one loop iteration of Algorithm 1, after space_verify (+ space_kv_commit) of
+ * the step: appends the step's out_tokens[b, 0 .. n_out[b]-1] to O, latches finished
+ * when the step met <EOS> (step_finished, from space_verify) or the buffer is full,
+ * and otherwise carries next_cand / next_cand_prob into L_c / P_c, takes kv_len_next
+ * (the commit's kv_len_out; must not alias state->kv_len) as the new length and writes
+ * the next call's block rows.  A sequence that is already finished is left untouched:
+ * the step's results for it are dropped and its length no longer grows.  All pointers
+ * device memory, shapes as in space_verify_args / space_commit_args.
+ * Asynchronous on `stream`, no host synchronisation: model, attention, verification,
+ * commit and this call can be enqueued step after step, or captured in one CUDA graph. */
+int space_decode_advance(space_ctx* ctx, const space_decode_state* state, const int32_t* out_tokens,
+                         const int32_t* n_out, const int32_t* next_cand, const float* next_cand_prob,
+                         const uint8_t* step_finished, const int32_t* kv_len_next, void* stream);
+
 /* Number of kernels this context has launched so far. */
 int64_t space_launch_count(const space_ctx* ctx);
 

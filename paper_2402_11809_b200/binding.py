@@ -27,7 +27,7 @@ ST_CAPACITY, ST_BAD_CANDIDATE, ST_TIMEOUT = 1, 2, 4
 EXPORTS = ["space_create", "space_destroy", "space_workspace_bytes", "space_layout",
            "space_attn_step", "space_verify", "space_verify_commit", "space_verify_greedy_noalloc",
            "space_kv_commit",
-           "space_lmhead_verify",
+           "space_lmhead_verify", "space_decode_begin", "space_decode_advance",
            "space_step_host",
            "space_launch_count", "space_profile_enable", "space_profile_read",
            "space_debug_philox", "space_debug_wait_timeout", "space_strerror"]
@@ -91,6 +91,14 @@ class LmHeadArgs(C.Structure):
                 ("row_argmax", C.c_void_p)]
 
 
+class DecodeState(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("k", C.c_int32), ("max_tokens", C.c_int32),
+                ("mask_token_id", C.c_int32), ("mask_variant", C.c_int32), ("reserved", C.c_int32),
+                ("tokens", C.c_void_p), ("n_tokens", C.c_void_p), ("last_token", C.c_void_p),
+                ("cand", C.c_void_p), ("cand_prob", C.c_void_p), ("kv_len", C.c_void_p),
+                ("finished", C.c_void_p), ("block_tokens", C.c_void_p), ("block_pos", C.c_void_p)]
+
+
 class HostStepArgs(C.Structure):
     _fields_ = [("batch", C.c_int32), ("k", C.c_int32), ("vocab", C.c_int32),
                 ("logits_dtype", C.c_int32), ("mode", C.c_int32), ("resample", C.c_int32),
@@ -118,6 +126,10 @@ for _name, _arg in (("space_attn_step", AttnArgs), ("space_verify", VerifyArgs),
                     ("space_lmhead_verify", LmHeadArgs)):
     getattr(lib, _name).argtypes = [C.c_void_p, C.POINTER(_arg), C.c_void_p]
     getattr(lib, _name).restype = C.c_int
+lib.space_decode_begin.argtypes = [C.c_void_p, C.POINTER(DecodeState), C.c_void_p, C.c_void_p]
+lib.space_decode_begin.restype = C.c_int
+lib.space_decode_advance.argtypes = [C.c_void_p, C.POINTER(DecodeState)] + [C.c_void_p] * 7
+lib.space_decode_advance.restype = C.c_int
 lib.space_verify_commit.argtypes = [C.c_void_p, C.POINTER(VerifyArgs), C.POINTER(CommitArgs), C.c_void_p]
 lib.space_verify_commit.restype = C.c_int
 lib.space_verify_greedy_noalloc.argtypes = [C.POINTER(VerifyArgs), C.c_void_p]
@@ -280,6 +292,22 @@ class Context:
 
     def space_kv_commit(self, args):
         _check(lib.space_kv_commit(self._h, C.byref(args), _stream()))
+
+    # -- decoding loop state (Algorithm 1) ---------------------------------
+    def decode_state(self, tokens, n_tokens, last_token, cand, cand_prob, kv_len, finished, block_tokens,
+                     block_pos, k, mask_token_id, mask_variant=MASK_SAME_GROUP):
+        return DecodeState(batch=tokens.shape[0], k=k, max_tokens=tokens.shape[1], mask_token_id=mask_token_id,
+                           mask_variant=mask_variant, reserved=0, tokens=_ptr(tokens), n_tokens=_ptr(n_tokens),
+                           last_token=_ptr(last_token), cand=_ptr(cand), cand_prob=_ptr(cand_prob),
+                           kv_len=_ptr(kv_len), finished=_ptr(finished), block_tokens=_ptr(block_tokens),
+                           block_pos=_ptr(block_pos))
+
+    def space_decode_begin(self, state, last_prompt_token):
+        _check(lib.space_decode_begin(self._h, C.byref(state), _ptr(last_prompt_token), _stream()))
+
+    def space_decode_advance(self, state, out_tokens, n_out, next_cand, next_cand_prob, step_finished, kv_len_next):
+        _check(lib.space_decode_advance(self._h, C.byref(state), _ptr(out_tokens), _ptr(n_out), _ptr(next_cand),
+                                        _ptr(next_cand_prob), _ptr(step_finished), _ptr(kv_len_next), _stream()))
 
     # -- space_step_host --------------------------------------------------
     def space_step_host(self, args):
