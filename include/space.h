@@ -139,29 +139,40 @@ typedef struct {
   int32_t* status;             /* device [B] or NULL                           */
 } space_verify_args;
 
-/* Output projection fused with greedy verification: the end of the model call
- * P = M(I) of Algorithm 1 (logits[r, x] = <h_r, W_x> for every block row r and
- * vocabulary token x; the rows of P are their softmax) and the loop after it
- * (acceptance of the candidates against the arg-max chain, extra token, <EOS>,
- * next candidates from the mask rows of group i*; Sec. 3.2).  The logits are
- * never written: only (max, lowest arg-max, sum exp) of every row leave the chip. */
-#define SPACE_LMHEAD_MAX_ROWS 256   /* batch * (k+1)^2 block rows per call     */
+/* Output projection fused with verification: the end of the model call P = M(I) of
+ * Algorithm 1 (logits[r, x] = <h_r, W_x> for every block row r and vocabulary token
+ * x; the rows of P are softmax(logits / T)) and the loop after it (acceptance of the
+ * candidates -- against the arg-max chain in greedy mode, by r <= Q/P_c with Philox
+ * draws in sampling mode --, extra token, <EOS>, next candidates from the mask rows of
+ * group i*; Sec. 3.2).  The logits are never written: only per-row statistics
+ * (maximum, lowest arg-max, sum of exponentials, best noisy score) leave the chip. */
+#define SPACE_LMHEAD_MAX_ROWS 256   /* block rows one kernel launch covers; a larger batch is
+                                       split into groups of sequences, one launch (and one pass
+                                       over the output embedding) per group                   */
 typedef struct {
   int32_t batch, k, vocab;
   int32_t hidden_dim;          /* D, a multiple of 8                           */
   int32_t eos_id;              /* -1: no end-of-sequence handling              */
-  int32_t reserved;            /* 0                                            */
+  int32_t mode;                /* SPACE_MODE_GREEDY or SPACE_MODE_SAMPLE       */
+  int32_t resample;            /* SPACE_RESAMPLE_* (sampling mode)             */
+  float   temperature;         /* > 0 (sampling mode)                          */
+  uint64_t seed;               /* Philox key (sampling mode), keyed as in space_verify */
   const void* hidden;          /* device bf16 [B * n_q, D]: final hidden state of every block row,
                                   sequence-major, block row order               */
   int64_t hidden_row_stride;   /* elements between rows, a multiple of 8       */
   const void* weight;          /* device bf16 [V, D]: output embedding, one row per token */
   int64_t weight_row_stride;   /* elements between rows, a multiple of 8       */
   const int32_t* cand;         /* device [B, k]  L_c                           */
+  const float*   cand_prob;    /* device [B, k]  P_c (sampling mode; may be NULL in greedy mode);
+                                  same rules as space_verify_args.cand_prob    */
+  const uint32_t* seq_id;      /* device [B] or NULL (= batch index): sequence ids of the random counters */
+  const int32_t*  kv_len;      /* device [B] or NULL (= 0): positions of the random counters */
   int32_t* n_accept;           /* device [B]       i*                          */
   int32_t* out_tokens;         /* device [B, k+1]  emitted tokens, -1 padded   */
   int32_t* n_out;              /* device [B]                                   */
   int32_t* next_cand;          /* device [B, k]                                */
-  float*   next_cand_prob;     /* device [B, k]  softmax (T = 1) of the token's own row */
+  float*   next_cand_prob;     /* device [B, k]  greedy: softmax (T = 1) of the token's own row;
+                                  sampling: as space_verify                    */
   uint8_t* finished;           /* device [B]                                   */
   int32_t* status;             /* device [B] or NULL                           */
   float*   row_max;            /* device [B * n_q] or NULL: largest logit of every block row */
@@ -281,15 +292,16 @@ int space_verify_commit(space_ctx* ctx, const space_verify_args* verify, const s
 #define SPACE_NOALLOC_MAX_BATCH 8
 int space_verify_greedy_noalloc(const space_verify_args* args, void* stream);
 
-/* Greedy step from hidden states (see space_lmhead_args): one kernel, the output
- * embedding is read once, products on the tensor cores in bf16 with fp32
- * accumulation, arg-max decided on the fp32 accumulators (lowest token on exact
- * ties).  Same outputs as space_verify in SPACE_MODE_GREEDY on the logits the
- * projection defines.  Asynchronous on `stream`, no allocation.  One call at a
- * time per context (the calls share the context's reduction scratch).
- * Errors: INVALID_ARG (NULL pointer, sizes), WORKSPACE (batch or k beyond the
- * context's), ALIGNMENT (16-byte base, strides and D multiples of 8),
- * UNSUPPORTED (more than SPACE_LMHEAD_MAX_ROWS block rows), CUDA. */
+/* One step from hidden states (see space_lmhead_args): the output embedding is read
+ * once per group of at most SPACE_LMHEAD_MAX_ROWS block rows, products on the tensor cores
+ * in bf16 with fp32 accumulation, every decision taken on the fp32 accumulators (arg-max:
+ * lowest token on exact ties; sampling: the same tests and Gumbel arg-maxes as
+ * space_verify, with the same Philox counters).  Same outputs as space_verify on the
+ * logits the projection defines.  Asynchronous on `stream`, no allocation.  One call at
+ * a time per context (the calls share the context's reduction scratch).
+ * Errors: INVALID_ARG (NULL pointer, sizes, mode, temperature), WORKSPACE (batch or k
+ * beyond the context's), ALIGNMENT (16-byte base, strides and D multiples of 8),
+ * UNSUPPORTED (one sequence alone exceeds the rows of a launch: cannot happen for k <= 7), CUDA. */
 int space_lmhead_verify(space_ctx* ctx, const space_lmhead_args* args, void* stream);
 
 /* Move accepted rows L+g(k+1) -> L+g, g = 1..i*; lengths grow by i*+1. */
@@ -347,6 +359,32 @@ int space_decode_begin(space_ctx* ctx, const space_decode_state* state, const in
 int space_decode_advance(space_ctx* ctx, const space_decode_state* state, const int32_t* out_tokens,
                          const int32_t* n_out, const int32_t* next_cand, const float* next_cand_prob,
                          const uint8_t* step_finished, const int32_t* kv_len_next, void* stream);
+
+/* Data-loader transform of semi-autoregressive fine-tuning (Sec. 3.1, App. A.1) on a
+ * padded batch of training samples, in place.  A sample (prompt of prompt_len tokens, then
+ * an answer y_1..y_N of answer_len tokens, in the first slots of its row) stays as it is
+ * with probability p_ar; otherwise a position m is drawn from {0..N-k}, the k answer tokens
+ * from there on become mask_token_id in input_ids (labels keep their tokens), and both rows
+ * are cut after the first m+k answer tokens (input_ids padded with pad_token_id, labels set
+ * to ignore_index).  An answer shorter than k stays autoregressive.
+ * Randomness is the caller's: two 32-bit words per sample; the sample stays autoregressive
+ * when the first is below ar_threshold (= p_ar * 2^32), and m = (second * (N-k+1)) >> 32.
+ * Needs no context; runs on the current device, asynchronous on `stream`.
+ * Errors: INVALID_ARG (NULL pointer, sizes), CUDA. */
+typedef struct {
+  int32_t batch, seq_cap, k;
+  int32_t mask_token_id, pad_token_id, ignore_index;
+  uint32_t ar_threshold;
+  int32_t reserved;            /* 0                                                   */
+  int32_t* input_ids;          /* device [B, seq_cap], in place                       */
+  int32_t* labels;             /* device [B, seq_cap], in place                       */
+  const int32_t* prompt_len;   /* device [B]                                          */
+  const int32_t* answer_len;   /* device [B]  N                                       */
+  const uint32_t* rand_words;  /* device [B, 2]                                       */
+  int32_t* new_len;            /* device [B] or NULL: tokens kept (prompt + answer part) */
+  int32_t* mask_start;         /* device [B] or NULL: m, or -1 for an unchanged sample */
+} space_sar_args;
+int space_sar_sft_transform(const space_sar_args* args, void* stream);
 
 /* Number of kernels this context has launched so far. */
 int64_t space_launch_count(const space_ctx* ctx);

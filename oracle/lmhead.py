@@ -1,4 +1,4 @@
-"""Output projection followed by greedy verification, in float64.
+"""Output projection followed by verification (greedy or sampling), in float64.
 
 Test infrastructure.  In Algorithm 1 the model call P = M(I) ends with the
 language-model head: every block row's final hidden state h is multiplied with
@@ -36,12 +36,15 @@ def top_two_gap(logits):
     return top - rest.max(axis=-1)
 
 
-def lmhead_verify_step(hidden, weight, cand, cand_prob, k, eos_id=-1):
-    """Greedy step of Algorithm 1 from hidden states: projection, then verification.
+def lmhead_verify_step(hidden, weight, cand, cand_prob, k, eos_id=-1, mode="greedy", temperature=1.0,
+                       seed=0, seq_id=None, kv_len=None, resample="residual_pointmass"):
+    """One step of Algorithm 1 from hidden states: projection, then verification (greedy, or
+    rejection sampling with the same Philox keying as verify.verify_step).
 
     Returns verify_step's dict plus `logits` (float64) and `row_gap` [B, n_q]."""
     logits = lm_head_logits(hidden, weight)
-    r = verify_step(logits, cand, cand_prob, k, "greedy", eos_id=eos_id)
+    r = verify_step(logits, cand, cand_prob, k, mode, temperature=temperature, seed=seed, seq_id=seq_id,
+                    kv_len=kv_len, resample=resample, eos_id=eos_id)
     r["logits"] = logits
     r["row_gap"] = top_two_gap(logits)
     return r

@@ -27,7 +27,7 @@ ST_CAPACITY, ST_BAD_CANDIDATE, ST_TIMEOUT = 1, 2, 4
 EXPORTS = ["space_create", "space_destroy", "space_workspace_bytes", "space_layout",
            "space_attn_step", "space_verify", "space_verify_commit", "space_verify_greedy_noalloc",
            "space_kv_commit",
-           "space_lmhead_verify", "space_decode_begin", "space_decode_advance",
+           "space_lmhead_verify", "space_sar_sft_transform", "space_decode_begin", "space_decode_advance",
            "space_step_host",
            "space_launch_count", "space_profile_enable", "space_profile_read",
            "space_debug_philox", "space_debug_wait_timeout", "space_strerror"]
@@ -82,10 +82,12 @@ class CommitArgs(C.Structure):
 
 class LmHeadArgs(C.Structure):
     _fields_ = [("batch", C.c_int32), ("k", C.c_int32), ("vocab", C.c_int32),
-                ("hidden_dim", C.c_int32), ("eos_id", C.c_int32), ("reserved", C.c_int32),
+                ("hidden_dim", C.c_int32), ("eos_id", C.c_int32), ("mode", C.c_int32),
+                ("resample", C.c_int32), ("temperature", C.c_float), ("seed", C.c_uint64),
                 ("hidden", C.c_void_p), ("hidden_row_stride", C.c_int64),
                 ("weight", C.c_void_p), ("weight_row_stride", C.c_int64),
-                ("cand", C.c_void_p), ("n_accept", C.c_void_p), ("out_tokens", C.c_void_p),
+                ("cand", C.c_void_p), ("cand_prob", C.c_void_p), ("seq_id", C.c_void_p),
+                ("kv_len", C.c_void_p), ("n_accept", C.c_void_p), ("out_tokens", C.c_void_p),
                 ("n_out", C.c_void_p), ("next_cand", C.c_void_p), ("next_cand_prob", C.c_void_p),
                 ("finished", C.c_void_p), ("status", C.c_void_p), ("row_max", C.c_void_p),
                 ("row_argmax", C.c_void_p)]
@@ -97,6 +99,15 @@ class DecodeState(C.Structure):
                 ("tokens", C.c_void_p), ("n_tokens", C.c_void_p), ("last_token", C.c_void_p),
                 ("cand", C.c_void_p), ("cand_prob", C.c_void_p), ("kv_len", C.c_void_p),
                 ("finished", C.c_void_p), ("block_tokens", C.c_void_p), ("block_pos", C.c_void_p)]
+
+
+class SarArgs(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("seq_cap", C.c_int32), ("k", C.c_int32),
+                ("mask_token_id", C.c_int32), ("pad_token_id", C.c_int32), ("ignore_index", C.c_int32),
+                ("ar_threshold", C.c_uint32), ("reserved", C.c_int32),
+                ("input_ids", C.c_void_p), ("labels", C.c_void_p), ("prompt_len", C.c_void_p),
+                ("answer_len", C.c_void_p), ("rand_words", C.c_void_p), ("new_len", C.c_void_p),
+                ("mask_start", C.c_void_p)]
 
 
 class HostStepArgs(C.Structure):
@@ -126,6 +137,8 @@ for _name, _arg in (("space_attn_step", AttnArgs), ("space_verify", VerifyArgs),
                     ("space_lmhead_verify", LmHeadArgs)):
     getattr(lib, _name).argtypes = [C.c_void_p, C.POINTER(_arg), C.c_void_p]
     getattr(lib, _name).restype = C.c_int
+lib.space_sar_sft_transform.argtypes = [C.POINTER(SarArgs), C.c_void_p]
+lib.space_sar_sft_transform.restype = C.c_int
 lib.space_decode_begin.argtypes = [C.c_void_p, C.POINTER(DecodeState), C.c_void_p, C.c_void_p]
 lib.space_decode_begin.restype = C.c_int
 lib.space_decode_advance.argtypes = [C.c_void_p, C.POINTER(DecodeState)] + [C.c_void_p] * 7
@@ -177,6 +190,17 @@ def space_layout(k, mask_variant=MASK_SAME_GROUP):
 def space_verify_greedy_noalloc(args):
     """Greedy verification with no context and no allocation (see include/space.h)."""
     _check(lib.space_verify_greedy_noalloc(C.byref(args), _stream()))
+
+
+def space_sar_sft_transform(input_ids, labels, prompt_len, answer_len, rand_words, k, mask_token_id,
+                            ar_threshold, pad_token_id=0, ignore_index=-100, new_len=None, mask_start=None):
+    """SAR-SFT sample transform on int32 CUDA tensors, in place (see include/space.h)."""
+    a = SarArgs(batch=input_ids.shape[0], seq_cap=input_ids.shape[1], k=k, mask_token_id=mask_token_id,
+                pad_token_id=pad_token_id, ignore_index=ignore_index, ar_threshold=ar_threshold, reserved=0,
+                input_ids=_ptr(input_ids), labels=_ptr(labels), prompt_len=_ptr(prompt_len),
+                answer_len=_ptr(answer_len), rand_words=_ptr(rand_words), new_len=_ptr(new_len),
+                mask_start=_ptr(mask_start))
+    _check(lib.space_sar_sft_transform(C.byref(a), _stream()))
 
 
 def space_strerror(code):
@@ -266,13 +290,17 @@ class Context:
 
     # -- space_lmhead_verify ----------------------------------------------
     def lmhead_args(self, hidden, weight, cand, n_accept, out_tokens, n_out, next_cand, next_cand_prob,
-                    finished, k, eos_id=-1, status=None, row_max=None, row_argmax=None):
+                    finished, k, eos_id=-1, status=None, row_max=None, row_argmax=None, mode=MODE_GREEDY,
+                    temperature=1.0, seed=0, resample=RESAMPLE_RESIDUAL_POINTMASS, cand_prob=None,
+                    seq_id=None, kv_len=None):
         """hidden [B, n_q, D] and weight [V, D] bf16 CUDA tensors with contiguous last dimension."""
         assert hidden.stride(2) == 1 and weight.stride(1) == 1
         assert hidden.stride(0) == hidden.shape[1] * hidden.stride(1)
         return LmHeadArgs(batch=hidden.shape[0], k=k, vocab=weight.shape[0], hidden_dim=weight.shape[1],
-                          eos_id=eos_id, reserved=0, hidden=_ptr(hidden), hidden_row_stride=hidden.stride(1),
+                          eos_id=eos_id, mode=mode, resample=resample, temperature=temperature, seed=seed,
+                          hidden=_ptr(hidden), hidden_row_stride=hidden.stride(1),
                           weight=_ptr(weight), weight_row_stride=weight.stride(0), cand=_ptr(cand),
+                          cand_prob=_ptr(cand_prob), seq_id=_ptr(seq_id), kv_len=_ptr(kv_len),
                           n_accept=_ptr(n_accept), out_tokens=_ptr(out_tokens), n_out=_ptr(n_out),
                           next_cand=_ptr(next_cand), next_cand_prob=_ptr(next_cand_prob),
                           finished=_ptr(finished), status=_ptr(status), row_max=_ptr(row_max),

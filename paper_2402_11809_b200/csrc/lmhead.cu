@@ -46,6 +46,7 @@ constexpr uint64_t LM_WAIT_NS = 1000000000ull;
 constexpr float LOG2E = 1.4426950408889634f;
 
 struct LmPartial { float m, s; int idx, pad; };   // 16 bytes
+struct LmNoisy { float gs, gz; int gidx, pad; };   // best noisy score of a range, the logit that has it, its token
 
 struct LmParams {
   CUtensorMap tm_w, tm_wt, tm_h;   // W in boxes of n_box rows, W in boxes of tail_rows rows, hidden rows
@@ -58,6 +59,13 @@ struct LmParams {
   int tail_rows;              // rows of the second tensor map's box
   int kbs;                    // 64-element slices of the hidden dimension per stage
   int eos_id;
+  int mode, resample;         // SPACE_MODE_*, SPACE_RESAMPLE_*
+  float c_t;                  // log2(e) / T: exponent scale of the sums and of the noisy scores (sampling)
+  uint32_t key0, key1;        // Philox key
+  uint32_t seq_base;          // sequence id of the group's first sequence when seq_id is NULL
+  const float* cand_prob; const uint32_t* seq_id; const int32_t* kv_len;
+  LmNoisy* gpart;             // [n_rows][gridDim.x] (sampling)
+  float* zc;                  // [n_rows] logit of the candidate a target row scores, written by the block that owns the token
   const int32_t* cand;
   int32_t* n_accept; int32_t* out_tokens; int32_t* n_out; int32_t* next_cand;
   float* next_cand_prob; uint8_t* finished; int32_t* status;
@@ -153,6 +161,90 @@ __device__ __forceinline__ void fold16(float& m, float& s, int& idx, const uint3
   s += (a0 + a1) + (a2 + a3);
 }
 
+// What an epilogue thread keeps of one block row in sampling mode.
+struct RowNoisy {
+  float gs, gz; int gidx;     // best noisy score so far, the logit that has it, its token
+  float zc;                   // logit of the candidate this (target) row scores
+  int cand_tok;               // that candidate, or -1
+  int exclude;                // token left out of the draw (the rejected point-mass candidate), or -1
+  uint32_t purpose, seq, pos; // Philox counter words of this row's noise
+  bool noisy;                 // this row draws a token at all
+};
+
+// Sampling-mode fold of 16 consecutive tokens x0 .. x0+15 (x0 a multiple of 16, the first nv valid):
+// (max, lowest arg-max, sum of exp2((z - max) c)), the candidate's own logit when it lies here, and
+// the best Gumbel-perturbed score z c + noise(token) -- the noise of token x is lane x & 3 of the
+// Philox block with counter word x >> 2, as in the verification kernels.
+__device__ __forceinline__ void fold16_noisy(float& m, float& s, int& idx, RowNoisy& r, const uint32_t* v, int x0,
+                                             int nv, float c, uint32_t key0, uint32_t key1) {
+  float z[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) z[j] = (j < nv) ? __uint_as_float(v[j]) : LM_NEG;
+  float cm = z[0];
+#pragma unroll
+  for (int j = 1; j < 16; ++j) cm = fmaxf(cm, z[j]);
+  if (cm > m) {
+    int at = 15;
+#pragma unroll
+    for (int j = 14; j >= 0; --j) at = (z[j] == cm) ? j : at;
+    idx = x0 + at;
+    s *= fast_exp2((m - cm) * c);
+    m = cm;
+  }
+  const float ms = -m * c;
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+  for (int j = 0; j < 16; j += 4) {
+    a0 += fast_exp2(fmaf(z[j], c, ms));
+    a1 += fast_exp2(fmaf(z[j + 1], c, ms));
+    a2 += fast_exp2(fmaf(z[j + 2], c, ms));
+    a3 += fast_exp2(fmaf(z[j + 3], c, ms));
+  }
+  s += (a0 + a1) + (a2 + a3);
+  if ((unsigned)(r.cand_tok - x0) < 16u) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) if (x0 + j == r.cand_tok) r.zc = z[j];
+  }
+  if (r.noisy) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const Philox4 ph = philox4x32_10((uint32_t)((x0 >> 2) + i), r.purpose, r.seq, r.pos, key0, key1);
+      const uint32_t w[4] = {ph.x, ph.y, ph.z, ph.w};
+#pragma unroll
+      for (int l = 0; l < 4; ++l) {
+        const int j = 4 * i + l;
+        const float sc = fmaf(z[j], c, gumbel2_from_uniform(uniform_open(w[l])));
+        if (j < nv && x0 + j != r.exclude && sc > r.gs) { r.gs = sc; r.gidx = x0 + j; r.gz = z[j]; }
+      }
+    }
+  }
+}
+
+// Per-row constants of the sampling mode: block row `row` of the batch is row i = row mod n_q of
+// sequence b; target rows (i = t(k+1)) score candidate c_{t+1} and draw the extra token of the
+// case i* = t at position L+t+1; mask rows (t, o) draw candidate o of that case at position
+// L+t+1+o when candidates are sampled (Algorithm 1 as printed).
+__device__ __forceinline__ void row_noisy_init(RowNoisy& r, const LmParams& p, int row) {
+  r.gs = -CUDART_INF_F; r.gz = 0.f; r.gidx = 0x7FFFFFFF; r.zc = LM_NEG;
+  r.cand_tok = -1; r.exclude = -1; r.purpose = 0; r.seq = 0; r.pos = 0; r.noisy = false;
+  if (row >= p.n_rows) return;
+  const int k1 = p.k + 1;
+  const int b = row / p.n_q, i = row - b * p.n_q;
+  const int t = i / k1, o = i - t * k1;
+  const bool literal = p.resample == SPACE_RESAMPLE_PAPER_LITERAL;
+  r.seq = p.seq_id ? p.seq_id[b] : p.seq_base + (uint32_t)b;
+  const int L = p.kv_len ? p.kv_len[b] : 0;
+  if (o == 0) {
+    r.noisy = true; r.purpose = PURPOSE_TOKEN; r.pos = (uint32_t)(L + t + 1);
+    if (t < p.k) {
+      r.cand_tok = p.cand[b * p.k + t];
+      if (!literal && p.cand_prob[b * p.k + t] == 1.0f) r.exclude = r.cand_tok;   // residual of a point mass
+    }
+  } else if (literal) {
+    r.noisy = true; r.purpose = PURPOSE_DRAFT; r.pos = (uint32_t)(L + t + 1 + o);
+  }
+}
+
 // (max, lowest arg-max) over the warp, result in every lane
 __device__ __forceinline__ void warp_max_idx(float& m, int& idx) {
 #pragma unroll
@@ -234,7 +326,10 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
 
   // this thread block's vocabulary range and its boxes
   const int G = gridDim.x, c = blockIdx.x;
-  const int r0 = (int)(((long long)p.V * c) / G), r1 = (int)(((long long)p.V * (c + 1)) / G);
+  // (range boundaries are multiples of 16 tokens, so that a group of 16 accumulator columns
+  // always starts on a Philox block)
+  const int r0 = (int)(((long long)p.V * c) / G) & ~15;
+  const int r1 = (c == G - 1) ? p.V : ((int)(((long long)p.V * (c + 1)) / G) & ~15);
   const int nb = (r1 - r0 + p.n_box - 1) / p.n_box;
   const int KB = (p.D + LM_KB - 1) / LM_KB;
   const int kbs = p.kbs;
@@ -321,6 +416,9 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
     for (int t = threadIdx.x - 64; t < p.B * p.k; t += 128) cand_s[t] = p.cand[t];
     float m0 = LM_NEG, s0 = 0.f, m1 = LM_NEG, s1 = 0.f;
     int i0 = 0x7FFFFFFF, i1 = 0x7FFFFFFF;
+    const bool sample = p.mode == SPACE_MODE_SAMPLE;
+    RowNoisy n0, n1;
+    if (sample) { row_noisy_init(n0, p, row_a); row_noisy_init(n1, p, p.n_mt == 2 ? LM_M + row_a : p.n_rows); }
     // a warp whose 32 lanes hold no block row only takes part in the hand-shakes
     const bool warp_a = quarter * 32 < p.n_rows, warp_b = p.n_mt == 2 && LM_M + quarter * 32 < p.n_rows;
     bool ok = true;
@@ -338,7 +436,8 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
           uint32_t v[16];
           tmem_ld16(acc + (uint32_t)c0, v);
           tmem_wait_ld();
-          fold16(m0, s0, i0, v, row0 + c0, n_valid - c0);
+          if (sample) fold16_noisy(m0, s0, i0, n0, v, row0 + c0, n_valid - c0, p.c_t, p.key0, p.key1);
+          else fold16(m0, s0, i0, v, row0 + c0, n_valid - c0);
         }
       }
       if (warp_b) {
@@ -346,7 +445,8 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
           uint32_t v[16];
           tmem_ld16(acc + (uint32_t)(LM_MAX_BOX + c0), v);
           tmem_wait_ld();
-          fold16(m1, s1, i1, v, row0 + c0, n_valid - c0);
+          if (sample) fold16_noisy(m1, s1, i1, n1, v, row0 + c0, n_valid - c0, p.c_t, p.key0, p.key1);
+          else fold16(m1, s1, i1, v, row0 + c0, n_valid - c0);
         }
       }
       // this accumulator buffer may be overwritten by the products of the next box that uses it
@@ -359,11 +459,21 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
       LmPartial out; out.m = m0; out.s = s0; out.idx = i0; out.pad = 0;
       *reinterpret_cast<int4*>(p.part + (size_t)row_a * G + c) = *reinterpret_cast<const int4*>(&out);
       atomicMax(p.keys + row_a, argmax_key(m0, i0));
+      if (sample) {
+        LmNoisy g; g.gs = n0.gs; g.gz = n0.gz; g.gidx = n0.gidx; g.pad = 0;
+        *reinterpret_cast<int4*>(p.gpart + (size_t)row_a * G + c) = *reinterpret_cast<const int4*>(&g);
+        if ((unsigned)(n0.cand_tok - r0) < (unsigned)(r1 - r0)) p.zc[row_a] = n0.zc;   // this block owns the candidate's token
+      }
     }
     if (p.n_mt == 2 && LM_M + row_a < p.n_rows) {
       LmPartial out; out.m = m1; out.s = s1; out.idx = i1; out.pad = 0;
       *reinterpret_cast<int4*>(p.part + (size_t)(LM_M + row_a) * G + c) = *reinterpret_cast<const int4*>(&out);
       atomicMax(p.keys + LM_M + row_a, argmax_key(m1, i1));
+      if (sample) {
+        LmNoisy g; g.gs = n1.gs; g.gz = n1.gz; g.gidx = n1.gidx; g.pad = 0;
+        *reinterpret_cast<int4*>(p.gpart + (size_t)(LM_M + row_a) * G + c) = *reinterpret_cast<const int4*>(&g);
+        if ((unsigned)(n1.cand_tok - r0) < (unsigned)(r1 - r0)) p.zc[LM_M + row_a] = n1.zc;
+      }
     }
     __threadfence();
     epi_sync();
@@ -393,6 +503,120 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
         if (p.row_argmax) p.row_argmax[r] = idx;
       }
       epi_sync();
+      if (sample) {
+        // ---- sampling mode (Algorithm 1 with r <= Q/P_c; see verify.cu for the same steps on
+        // stored logits).  tsum: sums of exp2((z - max) c) of the rows named by row_of(b, j),
+        // j = 0..k-1, combined from the ranges' partials in a fixed order.
+        const float cT = p.c_t;
+        float* tsum = reinterpret_cast<float*>(smem_raw) + LM_MAX_N;        // [B * k]
+        float* terms2 = tsum + LM_MAX_N;                                    // [B * k][G]
+        const bool literal = p.resample == SPACE_RESAMPLE_PAPER_LITERAL;
+        auto sum_rows = [&](bool mask_rows) {
+          const int total = p.B * p.k * G;
+          for (int i0 = et; i0 < total; i0 += 128 * 8) {
+            int4 v[8]; float mx[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int at = i0 + u * 128;
+              v[u] = make_int4(0, 0, 0, 0); mx[u] = 0.f;
+              if (at < total) {
+                const int g = at % G, bj = at / G;
+                const int b = bj / p.k, jj = bj - b * p.k;
+                const int row = b * p.n_q + (mask_rows ? istar[b] * k1 + jj + 1 : jj * k1);
+                mx[u] = row_m[row];
+                v[u] = __ldcg(reinterpret_cast<const int4*>(p.part + (size_t)row * G + g));
+              }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int at = i0 + u * 128;
+              if (at < total) terms2[at] = __int_as_float(v[u].y) * fast_exp2((__int_as_float(v[u].x) - mx[u]) * cT);
+            }
+          }
+          epi_sync();
+          for (int bj = ew; bj < p.B * p.k; bj += 4) {
+            float sv = 0.f;
+            for (int g = lane; g < G; g += 32) sv += terms2[bj * G + g];
+            sv = warp_sum(sv);
+            if (lane == 0) tsum[bj] = sv;
+          }
+          epi_sync();
+        };
+        // best noisy score of a row over the ranges: larger score, then lower token; every lane gets it
+        auto best_noisy = [&](int row, float& gz_out) -> int {
+          float gs = -CUDART_INF_F, gz = 0.f; int gi = 0x7FFFFFFF;
+          for (int g = lane; g < G; g += 32) {
+            const int4 v = __ldcg(reinterpret_cast<const int4*>(p.gpart + (size_t)row * G + g));
+            const float s2 = __int_as_float(v.x);
+            if (s2 > gs || (s2 == gs && v.z < gi)) { gs = s2; gz = __int_as_float(v.y); gi = v.z; }
+          }
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) {
+            const float os = __shfl_xor_sync(0xFFFFFFFFu, gs, off);
+            const float oz = __shfl_xor_sync(0xFFFFFFFFu, gz, off);
+            const int oi = __shfl_xor_sync(0xFFFFFFFFu, gi, off);
+            if (os > gs || (os == gs && oi < gi)) { gs = os; gz = oz; gi = oi; }
+          }
+          gz_out = gz;
+          return gi;
+        };
+        sum_rows(false);                                   // target rows t = 0..k-1 of every sequence
+        for (int b = ew; b < p.B; b += 4) {
+          const int* ri = row_i + b * p.n_q;
+          const int t = lane;
+          const int cv = (t < p.k) ? cand_s[b * p.k + t] : -1;
+          const bool in_range = cv >= 0 && cv < p.V;
+          const unsigned bad = __ballot_sync(0xFFFFFFFFu, t < p.k && !in_range);
+          bool okc = false;
+          const uint32_t seq = p.seq_id ? p.seq_id[b] : p.seq_base + (uint32_t)b;
+          const int Lb = p.kv_len ? p.kv_len[b] : 0;
+          if (t < p.k && in_range) {
+            const int row = b * p.n_q + t * k1;
+            const float zc = __ldcg(p.zc + row);
+            const float q = fast_exp2((zc - row_m[row]) * cT) / tsum[b * p.k + t];
+            const Philox4 w = philox4x32_10(0u, PURPOSE_ACCEPT, seq, (uint32_t)(Lb + t + 1), p.key0, p.key1);
+            const float pc = p.cand_prob[b * p.k + t];
+            okc = pc > 0.f && uniform_open(w.x) * pc <= q;  // r <= Q/P_c  <=>  r P_c <= Q
+          }
+          const unsigned acc_mask = __ballot_sync(0xFFFFFFFFu, okc);
+          const int i_star = __ffs(~acc_mask) - 1;          // first candidate that is not accepted (k when all are)
+          float gz_unused;
+          const int bonus = best_noisy(b * p.n_q + i_star * k1, gz_unused);   // a: the draw of the case i* (row i*)
+          const int j = lane;
+          const int c_j = __shfl_sync(0xFFFFFFFFu, cv, min(j, p.k - 1));
+          const int tok = (j < i_star) ? c_j : (j == i_star ? bonus : -1);
+          const bool is_eos = p.eos_id >= 0 && j <= i_star && tok == p.eos_id;
+          const unsigned eos_mask = __ballot_sync(0xFFFFFFFFu, is_eos && j < k1);
+          const int n_out = eos_mask ? __ffs(eos_mask) - 1 : i_star + 1;
+          if (j < k1) p.out_tokens[b * k1 + j] = (j < n_out) ? tok : -1;
+          if (j < p.k && !literal) {                        // point-mass drafts: arg-max of mask row (i*, j+1), P_c = 1
+            p.next_cand[b * p.k + j] = ri[i_star * k1 + j + 1];
+            p.next_cand_prob[b * p.k + j] = 1.f;
+          }
+          if (j == 0) {
+            istar[b] = i_star;
+            p.n_accept[b] = i_star;
+            p.n_out[b] = n_out;
+            p.finished[b] = (uint8_t)(eos_mask != 0);
+            if (p.status && bad) atomicOr(p.status + b, SPACE_ST_BAD_CANDIDATE);
+          }
+        }
+        epi_sync();
+        if (literal) {
+          // candidates sampled from the mask rows of group i*, with their probabilities
+          sum_rows(true);
+          for (int bj = ew; bj < p.B * p.k; bj += 4) {
+            const int b = bj / p.k, jj = bj - b * p.k;
+            const int row = b * p.n_q + istar[b] * k1 + jj + 1;
+            float gz;
+            const int tok = best_noisy(row, gz);
+            if (lane == 0) {
+              p.next_cand[bj] = tok;
+              p.next_cand_prob[bj] = fast_exp2((gz - row_m[row]) * cT) / tsum[bj];
+            }
+          }
+        }
+      } else {
       // acceptance scan and emitted tokens: one warp per sequence
       for (int b = ew; b < p.B; b += 4) {
         const int* ri = row_i + b * p.n_q;
@@ -449,6 +673,7 @@ __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_verify_kernel(const __gr
         sv = warp_sum(sv);
         if (lane == 0) p.next_cand_prob[bj] = 1.f / sv;    // softmax at T = 1 of its own maximum
       }
+      }
     }
   }
 #undef LBAR
@@ -494,9 +719,15 @@ int lm_make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t D, int6
 
 }  // namespace
 
-size_t lmhead_partial_bytes(int sm_count) { return (size_t)LM_MAX_N * sm_count * sizeof(LmPartial); }
+size_t lmhead_partial_bytes(int sm_count) {
+  return (size_t)LM_MAX_N * sm_count * (sizeof(LmPartial) + sizeof(LmNoisy));
+}
 
-int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_t st) {
+namespace {
+
+// One launch: the sequences of `a` (at most LM_MAX_N block rows); seq_base = index of the first
+// of them in the caller's batch.
+int launch_group(space_ctx* ctx, const space_lmhead_args* a, uint32_t seq_base, cudaStream_t st) {
   LmParams p;
   memset(&p, 0, sizeof(p));
   p.B = a->batch; p.k = a->k; p.V = a->vocab; p.D = a->hidden_dim;
@@ -509,7 +740,7 @@ int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_
   const int max_useful = (a->vocab + 31) / 32;             // at least 32 tokens per thread block
   if (grid > max_useful) grid = max_useful;
   if (grid < 1) grid = 1;
-  const int max_len = (a->vocab + grid - 1) / grid;        // the longest vocabulary range
+  const int max_len = (a->vocab + grid - 1) / grid + 15;   // the longest vocabulary range (boundaries are multiples of 16)
   p.n_box = max_len >= LM_MAX_BOX ? LM_MAX_BOX : (max_len + 15) / 16 * 16;
   p.tail_rows = (((max_len - 1) % p.n_box) + 1 + 15) / 16 * 16;
   // Slices per stage and stages: two slices when that leaves at least three stages (measured 1..4
@@ -526,6 +757,13 @@ int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_
   const LmSmem L(p.n_pad, p.n_box, stages, p.kbs);
   if (L.total + 1024 > 227 * 1024) return SPACE_E_UNSUPPORTED;
   p.eos_id = a->eos_id;
+  p.mode = a->mode; p.resample = a->resample;
+  p.c_t = LOG2E / (a->mode == SPACE_MODE_SAMPLE ? a->temperature : 1.0f);
+  p.key0 = (uint32_t)(a->seed & 0xFFFFFFFFull); p.key1 = (uint32_t)(a->seed >> 32);
+  p.seq_base = seq_base;
+  p.cand_prob = a->cand_prob; p.seq_id = a->seq_id; p.kv_len = a->kv_len;
+  p.gpart = reinterpret_cast<LmNoisy*>(ctx->lm_part + (size_t)LM_MAX_N * ctx->sm_count * sizeof(LmPartial));
+  p.zc = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->lm_counter) + 256 + LM_MAX_N * sizeof(unsigned long long));
   p.cand = a->cand;
   p.n_accept = a->n_accept; p.out_tokens = a->out_tokens; p.n_out = a->n_out; p.next_cand = a->next_cand;
   p.next_cand_prob = a->next_cand_prob; p.finished = a->finished; p.status = a->status;
@@ -546,4 +784,33 @@ int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_
   }
   ctx->launches += 1;
   return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace
+
+// A batch of more block rows than one launch covers goes group of sequences by group of
+// sequences: every group streams the output embedding once and is complete in itself (the
+// results are per sequence).  The launches follow one another on the stream and share the scratch.
+int launch_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, cudaStream_t st) {
+  const int n_q = (a->k + 1) * (a->k + 1), k1 = a->k + 1;
+  const int per_group = LM_MAX_N / n_q;
+  if (per_group < 1) return SPACE_E_UNSUPPORTED;
+  for (int b0 = 0; b0 < a->batch; b0 += per_group) {
+    space_lmhead_args g = *a;
+    g.batch = a->batch - b0 < per_group ? a->batch - b0 : per_group;
+    g.hidden = static_cast<const __nv_bfloat16*>(a->hidden) + (int64_t)b0 * n_q * a->hidden_row_stride;
+    g.cand = a->cand + (int64_t)b0 * a->k;
+    if (a->cand_prob) g.cand_prob = a->cand_prob + (int64_t)b0 * a->k;
+    if (a->seq_id) g.seq_id = a->seq_id + b0;
+    if (a->kv_len) g.kv_len = a->kv_len + b0;
+    g.n_accept = a->n_accept + b0; g.out_tokens = a->out_tokens + (int64_t)b0 * k1; g.n_out = a->n_out + b0;
+    g.next_cand = a->next_cand + (int64_t)b0 * a->k; g.next_cand_prob = a->next_cand_prob + (int64_t)b0 * a->k;
+    g.finished = a->finished + b0;
+    if (a->status) g.status = a->status + b0;
+    if (a->row_max) g.row_max = a->row_max + (int64_t)b0 * n_q;
+    if (a->row_argmax) g.row_argmax = a->row_argmax + (int64_t)b0 * n_q;
+    const int rc = launch_group(ctx, &g, (uint32_t)b0, st);
+    if (rc != SPACE_OK) return rc;
+  }
+  return SPACE_OK;
 }

@@ -50,7 +50,8 @@ Carve carve(const space_config* c, int sm_count) {
   v.vrow = off; off += align_up((size_t)c->max_batch * (c->k_max + 1) * sizeof(VerifyRow), 256);
   v.status = off; off += align_up((size_t)c->max_batch * sizeof(int32_t), 256);
   v.lm_part = off; off += align_up(lmhead_partial_bytes(sm_count), 256);
-  v.lm_counter = off; off += 256 + 256 * sizeof(unsigned long long);   // counter, error word; one arg-max key per block row
+  // counter, error word; one arg-max key per block row; one candidate logit per block row
+  v.lm_counter = off; off += 256 + 256 * sizeof(unsigned long long) + 256 * sizeof(float);
   v.stage = off;
   if (c->host_staging) {
     const size_t n_q = (size_t)(c->k_max + 1) * (c->k_max + 1);
@@ -319,7 +320,12 @@ int space_lmhead_verify(space_ctx* ctx, const space_lmhead_args* a, void* stream
       ((uintptr_t)a->hidden & 15) || ((uintptr_t)a->weight & 15))
     return SPACE_E_ALIGNMENT;
   if (a->hidden_row_stride < a->hidden_dim || a->weight_row_stride < a->hidden_dim) return SPACE_E_INVALID_ARG;
-  if (a->batch * (a->k + 1) * (a->k + 1) > SPACE_LMHEAD_MAX_ROWS) return SPACE_E_UNSUPPORTED;
+  if (a->mode != SPACE_MODE_GREEDY && a->mode != SPACE_MODE_SAMPLE) return SPACE_E_INVALID_ARG;
+  if (a->mode == SPACE_MODE_SAMPLE) {
+    if (!(a->temperature > 0.f) || !a->cand_prob) return SPACE_E_INVALID_ARG;
+    if (a->resample != SPACE_RESAMPLE_RESIDUAL_POINTMASS && a->resample != SPACE_RESAMPLE_PAPER_LITERAL)
+      return SPACE_E_INVALID_ARG;
+  }
   if (!use_device(ctx)) return SPACE_E_CUDA;
   return launch_lmhead_verify(ctx, a, (cudaStream_t)stream);
 }

@@ -30,6 +30,7 @@ constexpr int64_t SPACE_FUSED_MAX_BYTES = 64ll << 20;
 
 struct VerifyParams {
   int B, k, V, n_q, n_chunks, chunk;
+  int n_chunks_g, chunk_g;   // the row with Gumbel noise is cut finer (several times the work per logit)
   int mode, resample, eos_id;
   float c_t;                 // log2(e) / T   (target rows, sampled rows)
   float inv_t;               // 1 / T
@@ -61,24 +62,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-}
-
-// Gumbel noise in units of log 2:  -log2(-log2 u)  for u = (m + 1/2) 2^-23.
-// arg-max_x (z_x/T - log(-log u_x)) = arg-max_x (z_x*log2(e)/T - log2(-log2 u_x)):
-// the two scores differ by the factor log 2 and a constant, so the hardware
-// base-2 logarithm serves without rescaling.  Near u = 1 the inner logarithm is
-// taken from its series in d = 1 - u (exact in binary32); the error of the result
-// stays below 3e-5, inside the 1e-4 band within which two scores count as tied.
-__device__ __forceinline__ float fast_log2(float x) {
-  float y;
-  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float gumbel2_from_uniform(float u) {
-  const float d = 1.0f - u;
-  const float t = (d < 0.0078125f) ? d * (1.0f + d * (0.5f + d * 0.33333334f)) * 1.4426950408889634f
-                                   : -fast_log2(u);
-  return -fast_log2(t);
 }
 
 struct Stat {                // running statistics of a set of logits
@@ -128,17 +111,23 @@ template <> struct Vec<__nv_bfloat16> {
 };
 
 // One logit (the ragged ends of a chunk and unaligned rows).
-template <bool GUMBEL, bool STATS>
+// What a scan keeps of its logits: nothing (the noisy arg-max alone), the maximum with its
+// lowest-index arg-max, or those and the sum of exp((z - max) c).
+enum { STAT_NONE = 0, STAT_MAX = 1, STAT_SUM = 2 };
+
+template <bool GUMBEL, int STATS>
 __device__ __forceinline__ void fold_one(Stat& st, float v, int x, float c, int exclude,
                                          uint32_t key0, uint32_t key1, uint32_t purpose,
                                          uint32_t seq, uint32_t pos) {
-  if (STATS) {
+  if (STATS == STAT_SUM) {
     if (v > st.m) {
       st.s = (st.m > -CUDART_INF_F) ? st.s * fast_exp2((st.m - v) * c) : 0.f;
       st.idx = x;
       st.m = v;
     }
     if (st.m > -CUDART_INF_F) st.s += fast_exp2(fmaf(v, c, -st.m * c));
+  } else if (STATS == STAT_MAX) {
+    if (v > st.m) { st.idx = x; st.m = v; }
   }
   if (GUMBEL) {
     // noise of token x: lane x&3 of the Philox block with counter word x>>2
@@ -154,7 +143,7 @@ __device__ __forceinline__ void fold_one(Stat& st, float v, int x, float c, int 
 // call, then independent exponentials and tree sums.  -inf entries (slots past the
 // end of the chunk) change neither the maximum nor the sum.  st.idx is left at the first
 // index of the vector that holds the maximum (see scan_chunk).
-template <int U, int N>
+template <int U, int N, bool SUMS>
 __device__ __forceinline__ void fold_stats(Stat& st, const float (&v)[U][N], int x0, int stride, float c) {
   float vm[U];
 #pragma unroll
@@ -172,7 +161,7 @@ __device__ __forceinline__ void fold_stats(Stat& st, const float (&v)[U][N], int
 #pragma unroll
   for (int u = 1; u < U; ++u) vmax = fmaxf(vmax, vm[u]);
   if (vmax > st.m) {
-    st.s = (st.m > -CUDART_INF_F) ? st.s * fast_exp2((st.m - vmax) * c) : 0.f;
+    if (SUMS) st.s = (st.m > -CUDART_INF_F) ? st.s * fast_exp2((st.m - vmax) * c) : 0.f;
     // first vector that holds the new maximum (walk backwards, the last hit wins); which of
     // its N logits it is gets settled once, at the end of the chunk (this branch is taken in
     // almost every sweep of a short chunk, so it stays small)
@@ -181,7 +170,7 @@ __device__ __forceinline__ void fold_stats(Stat& st, const float (&v)[U][N], int
       if (vm[u] == vmax) st.idx = x0 + u * stride;
     st.m = vmax;
   }
-  if (st.m > -CUDART_INF_F) {
+  if (SUMS && st.m > -CUDART_INF_F) {
     const float nmc = -st.m * c;                            // exp2(z*c - m*c): exponent error below 1e-5
     float su[U];
 #pragma unroll
@@ -228,7 +217,7 @@ __device__ __forceinline__ void fold_gumbel(Stat& st, const float* v, int x0, fl
 // Statistics of logits [begin, end) of one row.  STATS: maximum, arg-max and sum;
 // GUMBEL: the best noisy score (token `exclude` left out).  With VECTOR, `begin`
 // is a multiple of the vector length and the row is 16-byte aligned.
-template <typename T, bool VECTOR, bool GUMBEL, bool STATS>
+template <typename T, bool VECTOR, bool GUMBEL, int STATS>
 __device__ Stat scan_chunk(const T* row, int begin, int end, float c, int exclude,
                            uint32_t key0, uint32_t key1, uint32_t purpose, uint32_t seq,
                            uint32_t pos) {
@@ -255,7 +244,7 @@ __device__ Stat scan_chunk(const T* row, int begin, int end, float c, int exclud
       float v[U][N];
 #pragma unroll
       for (int u = 0; u < U; ++u) Vec<T>::convert(cur[u], v[u]);
-      if (STATS) fold_stats<U, N>(st, v, x, stride, c);
+      if (STATS) fold_stats<U, N, STATS == STAT_SUM>(st, v, x, stride, c);
       if (GUMBEL) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -419,7 +408,7 @@ verify_target_kernel(const VerifyParams p) {
   const int k1 = p.k + 1;
   const T* row = reinterpret_cast<const T*>(p.logits) + ((int64_t)b * p.n_q + (int64_t)t * k1) * p.row_stride;
   const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
-  Stat st = scan_chunk<T, VECTOR, false, true>(row, begin, end, p.c_t, -1, 0, 0, 0, 0, 0);
+  Stat st = scan_chunk<T, VECTOR, false, STAT_SUM>(row, begin, end, p.c_t, -1, 0, 0, 0, 0, 0);
   st = block_reduce_plain(st, p.c_t);
   VerifyPartial* part = p.part + ((int64_t)b * (p.k + 2) + t) * p.n_chunks;
   if (threadIdx.x == 0) store_partial(part + ch, st);
@@ -478,16 +467,27 @@ __global__ void __launch_bounds__(SPACE_VERIFY_THREADS, 3)   // 80 registers, no
 verify_emit_kernel(const VerifyParams p) {
   pdl_launch_dependents();
   pdl_wait();
-  const int b = blockIdx.y, ch = blockIdx.x;
   const int k1 = p.k + 1;
-  const int i_star = p.n_accept[b];
   const bool sample = p.mode == SPACE_MODE_SAMPLE;
-  // Slot is the slowest grid dimension and the rows with Gumbel noise (several times
-  // the work of a plain row) come first in it: the long blocks of every sequence
-  // start before any short one, so none is left for the tail of the launch.
-  const int slot = sample ? (blockIdx.z == 0 ? p.k : (int)blockIdx.z - 1) : (int)blockIdx.z;
+  // One-dimensional grid.  In sampling mode the first B * n_chunks_g blocks are the chunks of the
+  // extra-token rows: a logit there costs a Philox block and two logarithms, several times a plain
+  // one, so those rows are cut finer (their work spreads over every SM) and start first (no long
+  // block is left for the tail of the launch).  Then the mask rows: chunk, sequence, slot.
+  const int n_g = sample ? p.B * p.n_chunks_g : 0;
+  int b, ch, slot, chunk_len, n_ch;
+  if ((int)blockIdx.x < n_g) {
+    slot = p.k; b = blockIdx.x / p.n_chunks_g; ch = blockIdx.x - b * p.n_chunks_g;
+    chunk_len = p.chunk_g; n_ch = p.n_chunks_g;
+  } else {
+    int r = blockIdx.x - n_g;
+    ch = r % p.n_chunks; r /= p.n_chunks;
+    b = r % p.B; slot = r / p.B;
+    chunk_len = p.chunk; n_ch = p.n_chunks;
+  }
+  const int i_star = p.n_accept[b];
   const bool literal = sample && p.resample == SPACE_RESAMPLE_PAPER_LITERAL;
-  const int n_slots = sample ? k1 : p.k;
+  const int blocks_per_seq = p.k * p.n_chunks + (sample ? p.n_chunks_g : 0);
+  const int part_id = (slot == p.k) ? ch : (sample ? p.n_chunks_g : 0) + slot * p.n_chunks + ch;
   const uint32_t seq = p.seq_id ? p.seq_id[b] : (uint32_t)b;
   const int L = p.kv_len ? p.kv_len[b] : 0;
   const T* base = reinterpret_cast<const T*>(p.logits) + (int64_t)b * p.n_q * p.row_stride;
@@ -497,13 +497,12 @@ verify_emit_kernel(const VerifyParams p) {
   if (p.do_commit) {
     Lc = p.cm.kv_len[b];
     if (commit_fits(p.cm, Lc))
-      commit_rows(p.cm, b, Lc, max(0, min(i_star, p.k)), slot * p.n_chunks + ch, n_slots * p.n_chunks,
-                  threadIdx.x, blockDim.x);
+      commit_rows(p.cm, b, Lc, max(0, min(i_star, p.k)), part_id, blocks_per_seq, threadIdx.x, blockDim.x);
   }
   // slot o < k: mask row (i*, o+1); slot k: target row i* (extra token, sampling)
   const int brow = (slot < p.k) ? i_star * k1 + slot + 1 : i_star * k1;
   const T* row = base + (int64_t)brow * p.row_stride;
-  const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
+  const int begin = ch * chunk_len, end = min(p.V, begin + chunk_len);
   const float c = sample ? p.c_t : 1.4426950408889634f;
   Stat st;
   if (slot == p.k) {
@@ -512,27 +511,31 @@ verify_emit_kernel(const VerifyParams p) {
     // with any other P_c (Algorithm 1 starts from P_c = +inf) was no point mass: a ~ Q.
     if (!literal && i_star < p.k && p.cand_prob[b * p.k + i_star] == 1.0f) exclude = p.cand[b * p.k + i_star];
     // the extra token needs the noisy arg-max alone: the row's sums are known
-    st = scan_chunk<T, VECTOR, true, false>(row, begin, end, c, exclude, p.key0, p.key1, PURPOSE_TOKEN,
+    st = scan_chunk<T, VECTOR, true, STAT_NONE>(row, begin, end, c, exclude, p.key0, p.key1, PURPOSE_TOKEN,
                                             seq, (uint32_t)(L + i_star + 1));
   } else if (literal) {
-    st = scan_chunk<T, VECTOR, true, true>(row, begin, end, c, -1, p.key0, p.key1, PURPOSE_DRAFT, seq,
+    st = scan_chunk<T, VECTOR, true, STAT_SUM>(row, begin, end, c, -1, p.key0, p.key1, PURPOSE_DRAFT, seq,
                                            (uint32_t)(L + i_star + 1 + slot + 1));
+  } else if (sample) {
+    // point-mass drafts: the new candidates are the rows' arg-maxes with P_c = 1, no sums needed
+    st = scan_chunk<T, VECTOR, false, STAT_MAX>(row, begin, end, c, -1, 0, 0, 0, 0, 0);
   } else {
-    st = scan_chunk<T, VECTOR, false, true>(row, begin, end, c, -1, 0, 0, 0, 0, 0);
+    st = scan_chunk<T, VECTOR, false, STAT_SUM>(row, begin, end, c, -1, 0, 0, 0, 0, 0);
   }
   st = block_reduce(st, c);
-  VerifyPartial* part = p.part + ((int64_t)b * (p.k + 2) + slot) * p.n_chunks;
+  // (chunk results of the emit kernel: SPACE_VERIFY_MAX_CHUNKS slots per row, whatever its cut)
+  VerifyPartial* part = p.part + ((int64_t)b * (p.k + 2) + slot) * SPACE_VERIFY_MAX_CHUNKS;
   if (threadIdx.x == 0) store_partial(part + ch, st);
-  if (!arrive_last(p.counter_b + b, n_slots * p.n_chunks)) return;
+  if (!arrive_last(p.counter_b + b, blocks_per_seq)) return;
 
   // ---- last block of sequence b: emitted tokens and new candidates -------
   // Warp o combines mask row o (next candidate o+1); warp k the extra-token row.
   __shared__ int sh_bonus;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  VerifyPartial* pb = p.part + (int64_t)b * (p.k + 2) * p.n_chunks;
+  VerifyPartial* pb = p.part + (int64_t)b * (p.k + 2) * SPACE_VERIFY_MAX_CHUNKS;
   if (warp < p.k) {
     const int o = warp;
-    const Stat r = gather_row(pb + (int64_t)o * p.n_chunks, p.n_chunks, c);
+    const Stat r = gather_row(pb + (int64_t)o * SPACE_VERIFY_MAX_CHUNKS, p.n_chunks, c);
     if (lane == 0) {
       int tok; float pr;
       if (!sample)      { tok = r.idx;  pr = 1.f / r.s; }          // softmax at T = 1 of its own maximum
@@ -547,7 +550,7 @@ verify_emit_kernel(const VerifyParams p) {
     }
   } else if (warp == p.k) {
     int bonus;
-    if (sample) bonus = gather_row(pb + (int64_t)p.k * p.n_chunks, p.n_chunks, c).gidx;
+    if (sample) bonus = gather_row(pb + (int64_t)p.k * SPACE_VERIFY_MAX_CHUNKS, p.n_chunks_g, c).gidx;
     else bonus = p.rows[b * k1 + i_star].idx;
     if (lane == 0) sh_bonus = bonus;
   }
@@ -586,7 +589,7 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
   int Lc = 0;
   if (p.do_commit) Lc = p.cm.kv_len[b];                     // in flight during the scan
-  Stat st = scan_chunk<T, VECTOR, false, true>(row, begin, end, C1, -1, 0, 0, 0, 0, 0);
+  Stat st = scan_chunk<T, VECTOR, false, STAT_SUM>(row, begin, end, C1, -1, 0, 0, 0, 0, 0);
   // KV commit on board: which candidates are accepted is known only to the last block, at the very
   // end, so every block moves its slice of ALL k candidate rows now, while the logits stream.
   // Rows L+1 .. L+i* end up exactly as the plain commit leaves them; rows L+i*+1 .. L+k, which lie
@@ -665,7 +668,8 @@ void launch_fused(space_ctx* ctx, const VerifyParams& p, cudaStream_t st) {
 
 template <typename T, bool VECTOR>
 void launch_both(space_ctx* ctx, const VerifyParams& p, int n_slots_b, cudaStream_t st) {
-  dim3 ga(p.n_chunks, p.k + 1, p.B), gb(p.n_chunks, p.B, n_slots_b);
+  dim3 ga(p.n_chunks, p.k + 1, p.B);
+  const dim3 gb(p.B * (p.k * p.n_chunks + (p.mode == SPACE_MODE_SAMPLE ? p.n_chunks_g : 0)));
   {
     ProfScope ps(ctx, SPACE_K_VERIFY_TARGET, st);
     launch_pdl(verify_target_kernel<T, VECTOR>, ga, dim3(SPACE_VERIFY_THREADS), 0, st, p);
@@ -721,7 +725,7 @@ int launch_verify(space_ctx* ctx, const space_verify_args* a, const space_commit
     int chunk = (a->vocab + nc - 1) / nc;
     chunk = ((chunk + vec - 1) / vec) * vec;
     nc = (a->vocab + chunk - 1) / chunk;
-    p.n_chunks = nc; p.chunk = chunk;
+    p.n_chunks = nc; p.chunk = chunk; p.n_chunks_g = 0; p.chunk_g = 0;
     if (a->logits_dtype == SPACE_DTYPE_F32) {
       if (vector) launch_fused<float, true>(ctx, p, st); else launch_fused<float, false>(ctx, p, st);
     } else {
@@ -745,6 +749,18 @@ int launch_verify(space_ctx* ctx, const space_verify_args* a, const space_commit
   nc = (a->vocab + chunk - 1) / chunk;
   p.n_chunks = nc; p.chunk = chunk;
   const int n_slots_b = (a->mode == SPACE_MODE_SAMPLE) ? a->k + 1 : a->k;
+  // the extra-token row has a cut of its own (its logits cost several times a plain row's)
+  {
+    int ncg = nc;                                           // (measured: a finer cut of this row, up to 8x, is no faster)
+    const int min_chunk_g = SPACE_VERIFY_THREADS * vec * 4;
+    const int max_ncg = (a->vocab + min_chunk_g - 1) / min_chunk_g;
+    if (ncg > max_ncg) ncg = max_ncg;
+    if (ncg > SPACE_VERIFY_MAX_CHUNKS) ncg = SPACE_VERIFY_MAX_CHUNKS;
+    if (ncg < 1) ncg = 1;
+    int cg = (a->vocab + ncg - 1) / ncg;
+    cg = ((cg + vec - 1) / vec) * vec;
+    p.n_chunks_g = (a->vocab + cg - 1) / cg; p.chunk_g = cg;
+  }
 
   if (a->logits_dtype == SPACE_DTYPE_F32) {
     if (vector) launch_both<float, true>(ctx, p, n_slots_b, st); else launch_both<float, false>(ctx, p, n_slots_b, st);

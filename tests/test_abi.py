@@ -86,9 +86,9 @@ def test_struct_sizes_match_c(binding):
     src = r'''
 #include <stdio.h>
 #include "space.h"
-int main(void){ printf("%zu %zu %zu %zu %zu %zu %zu %zu\n", sizeof(space_config), sizeof(space_layout_t),
+int main(void){ printf("%zu %zu %zu %zu %zu %zu %zu %zu %zu\n", sizeof(space_config), sizeof(space_layout_t),
   sizeof(space_attn_args), sizeof(space_verify_args), sizeof(space_commit_args), sizeof(space_host_step_args),
-  sizeof(space_lmhead_args), sizeof(space_decode_state)); return 0; }
+  sizeof(space_lmhead_args), sizeof(space_decode_state), sizeof(space_sar_args)); return 0; }
 '''
     with tempfile.TemporaryDirectory() as d:
         open(os.path.join(d, "t.c"), "w").write(src)
@@ -97,5 +97,5 @@ int main(void){ printf("%zu %zu %zu %zu %zu %zu %zu %zu\n", sizeof(space_config)
         out = subprocess.check_output([os.path.join(d, "t")]).decode().split()
     want = [ctypes.sizeof(x) for x in (binding.Config, binding.Layout, binding.AttnArgs,
                                        binding.VerifyArgs, binding.CommitArgs, binding.HostStepArgs,
-                                       binding.LmHeadArgs, binding.DecodeState)]
+                                       binding.LmHeadArgs, binding.DecodeState, binding.SarArgs)]
     assert [int(x) for x in out] == want

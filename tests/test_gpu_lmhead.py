@@ -1,5 +1,5 @@
-"""GPU parity of space_lmhead_verify (output projection fused with greedy
-verification) against the float64 oracle, through the C ABI.
+"""GPU parity of space_lmhead_verify (output projection fused with verification,
+greedy and sampling) against the float64 oracle, through the C ABI.
 
 Integers (accepted count, emitted tokens, next candidates, row arg-maxes) must
 match exactly.  The arg-max of a row is decided on fp32 accumulators of bf16
@@ -29,7 +29,8 @@ def H():
     return gpu_harness
 
 
-def _run(H, cfg, x, eos_id=-1, ctx=None, pad=0):
+def _run(H, cfg, x, eos_id=-1, ctx=None, pad=0, sample=None):
+    """sample: None (greedy) or dict(temperature, seed, resample, kv_len, seq_id)."""
     from paper_2402_11809_b200 import binding as B
     Bn, k, V, D = cfg["B"], cfg["k"], cfg["V"], cfg["D"]
     n_q = x["n_q"]
@@ -58,13 +59,22 @@ def _run(H, cfg, x, eos_id=-1, ctx=None, pad=0):
         row_max=torch.full((Bn, n_q), float("nan"), device=dev),
         row_argmax=torch.full((Bn, n_q), -7, dtype=torch.int32, device=dev),
     )
+    extra = {}
+    if sample is not None:
+        extra = dict(mode=B.MODE_SAMPLE, temperature=sample["temperature"], seed=sample["seed"],
+                     resample=B.RESAMPLE_PAPER_LITERAL if sample["resample"] == "paper_literal"
+                     else B.RESAMPLE_RESIDUAL_POINTMASS,
+                     cand_prob=H.to_dev(x["cand_prob"].astype(np.float32)),
+                     kv_len=H.to_dev(sample["kv_len"].astype(np.int32)),
+                     seq_id=H.to_dev(sample["seq_id"].astype(np.uint32)) if sample.get("seq_id") is not None else None)
     a = ctx.lmhead_args(hidden, weight, H.to_dev(x["cand"]), o["n_accept"], o["out_tokens"], o["n_out"],
                         o["next_cand"], o["next_cand_prob"], o["finished"], k, eos_id=eos_id,
-                        status=o["status"], row_max=o["row_max"], row_argmax=o["row_argmax"])
+                        status=o["status"], row_max=o["row_max"], row_argmax=o["row_argmax"], **extra)
     n0 = ctx.launch_count
     ctx.space_lmhead_verify(a)
     torch.cuda.synchronize()
-    assert ctx.launch_count == n0 + 1
+    per_group = B.LMHEAD_MAX_ROWS // n_q                     # one launch per group of sequences
+    assert ctx.launch_count == n0 + (Bn + per_group - 1) // per_group
     got = {key: v.cpu().numpy() for key, v in o.items()}
     if own:
         ctx.close()
@@ -182,10 +192,91 @@ def test_lmhead_repeated_calls_and_argument_checks(H):
     a = good(); a.weight = a.weight + 2
     assert B.lib.space_lmhead_verify(ctx._h, a, None) == B.E_ALIGNMENT
     ctx.close()
-    big = B.Context(device=0, max_batch=8, n_q_heads=8, n_kv_heads=8, head_dim=64, k_max=7, vocab=9000, s_cap=256)
-    a = big.lmhead_args(hidden, weight, z, z, z, z, z, f, u, 7); a.batch = 5   # 5 * 64 rows > 256
-    assert B.lib.space_lmhead_verify(big._h, a, None) == B.E_UNSUPPORTED
-    big.close()
+    ctx = B.Context(device=0, max_batch=2, n_q_heads=8, n_kv_heads=8, head_dim=64, k_max=5, vocab=9000, s_cap=256)
+    a = good(); a.mode = 7
+    assert B.lib.space_lmhead_verify(ctx._h, a, None) == B.E_INVALID_ARG
+    a = good(); a.mode = B.MODE_SAMPLE; a.temperature = 0.7           # sampling needs P_c
+    assert B.lib.space_lmhead_verify(ctx._h, a, None) == B.E_INVALID_ARG
+    a = good(mode=B.MODE_SAMPLE, temperature=0.0, cand_prob=f)
+    assert B.lib.space_lmhead_verify(ctx._h, a, None) == B.E_INVALID_ARG
+    ctx.close()
+
+
+def test_lmhead_wide_batch_goes_group_by_group(H):
+    # 16 sequences of 36 block rows: 576 rows, three launches of at most 256 rows each
+    cfg = workloads.resolve_lmhead("lmhead_tiny", V=20000, D=256, k=5, B=16, p_accept=(0.3, 0.9))
+    x = workloads.make_lmhead_inputs(cfg)
+    got = _run(H, cfg, x)
+    r = _compare(cfg, x, got, what="B16 k5")
+    assert len(set(r["n_accept"].tolist())) > 2
+
+
+ACCEPT_BAND = 1e-3      # relative distance of r P_c from Q(c) below which an acceptance is a tie
+NOISY_BAND = 1e-3       # top-two gap of the Gumbel-perturbed scores below which a draw is a tie
+
+
+def _compare_sampling(cfg, x, got, sp, what=""):
+    """Sampling mode against the oracle.  Excluded (and printed): sequences whose acceptance test,
+    Gumbel draw or arg-max sits inside a tie band -- the kernel takes those decisions on fp32
+    accumulators of bf16 products, the oracle in float64."""
+    k = cfg["k"]
+    r = lmhead_verify_step(x["hidden"], x["weight"], x["cand"], x["cand_prob"], k, mode="sample",
+                           temperature=sp["temperature"], seed=sp["seed"], seq_id=sp.get("seq_id"),
+                           kv_len=sp["kv_len"], resample=sp["resample"])
+    ref_max = r["logits"].max(axis=-1)
+    assert np.abs(got["row_max"] - ref_max).max() <= MAX_TOL, what
+    tie = r["row_gap"] <= GAP_BAND
+    excl = (r["accept_margin"] <= ACCEPT_BAND).any(axis=1) | (r["bonus_gap"] <= NOISY_BAND) | \
+        (r["draft_gap"] <= NOISY_BAND).any(axis=1)
+    for b in range(cfg["B"]):
+        i = int(r["n_accept"][b])
+        if sp["resample"] != "paper_literal" and tie[b, [i * (k + 1) + o for o in range(1, k + 1)]].any():
+            excl[b] = True                                   # point-mass drafts are arg-maxes of the mask rows
+    keep = ~excl
+    if excl.any():
+        print(f"{what}: excluded sequences {np.nonzero(excl)[0].tolist()}")
+    assert excl.sum() <= max(1, cfg["B"] // 8), what
+    for name in ("n_accept", "out_tokens", "n_out", "next_cand", "finished"):
+        assert np.array_equal(got[name][keep], r[name][keep]), (what, name)
+    assert np.allclose(got["next_cand_prob"][keep], r["next_cand_prob"][keep], rtol=PROB_RTOL, atol=0), what
+    return r
+
+
+@pytest.mark.parametrize("resample", ["residual_pointmass", "paper_literal"])
+@pytest.mark.parametrize("V,D,k,Bn,T", [(1000, 256, 4, 3, 1.0), (40000, 192, 2, 5, 0.8), (33000, 128, 7, 4, 0.7),
+                                        (20000, 256, 5, 16, 0.9)])
+def test_lmhead_sampling_small_shapes(H, resample, V, D, k, Bn, T):
+    from paper_2402_11809_b200 import binding as B
+    cfg = workloads.resolve_lmhead("lmhead_tiny", V=V, D=D, k=k, B=Bn, p_accept=(0.5, 0.9), sigma=2.0)
+    rng = np.random.default_rng(V + k)
+    for s in range(2):
+        x = workloads.make_lmhead_inputs(cfg, set_index=s)
+        # planted candidates score about 30 (accepted almost surely); give some rows a mid-range
+        # candidate as well: the runner-up of its target row
+        if resample == "paper_literal":
+            x["cand_prob"] = rng.uniform(0.05, 1.0, size=x["cand_prob"].shape).astype(np.float32)
+        x["cand_prob"][0, :] = np.inf                        # Algorithm 1's initial state
+        x["cand"][-1, -1] = V + 9                            # out of range: rejected, flagged
+        sp = dict(temperature=T, seed=0xC0FFEE + s, resample=resample,
+                  kv_len=rng.integers(0, 3000, size=Bn), seq_id=np.arange(Bn) * 3 + 1)
+        got = _run(H, cfg, x, sample=sp)
+        r = _compare_sampling(cfg, x, got, sp, what=f"{resample} V{V} k{k} B{Bn} set{s}")
+        assert r["n_accept"][0] == 0 and got["n_accept"][0] == 0
+        assert got["status"][-1] & B.ST_BAD_CANDIDATE and not got["status"][:-1].any()
+    # without sequence ids the batch index keys the draws, also across the groups of a wide batch
+    sp = dict(temperature=T, seed=5, resample=resample, kv_len=np.zeros(Bn, dtype=np.int64), seq_id=None)
+    got = _run(H, cfg, x, sample=sp)
+    _compare_sampling(cfg, x, got, sp, what="no seq ids")
+
+
+def test_lmhead_sampling_vocab128k(H):
+    # the vocabulary of the 64-sequence sampling configuration at T = 0.8
+    cfg = workloads.resolve_lmhead("lmhead_vocab128k", D=1024, B=2, k=4)
+    x = workloads.make_lmhead_inputs(cfg)
+    sp = dict(temperature=0.8, seed=4, resample="residual_pointmass", kv_len=np.array([1500, 16000]), seq_id=None)
+    got = _run(H, cfg, x, sample=sp)
+    r = _compare_sampling(cfg, x, got, sp, what="vocab128k sampling")
+    assert r["n_accept"].max() > 0
 
 
 @pytest.mark.parametrize("name", ["lmhead_llama7b", "lmhead_batch4", "lmhead_vocab128k"])

@@ -90,3 +90,29 @@ def test_planted_candidates_are_accepted_as_a_prefix():
 def test_top_two_gap():
     z = np.array([[[1.0, 5.0, 3.0, 5.0], [0.0, -1.0, 4.0, 1.5]]])
     assert np.array_equal(top_two_gap(z), np.array([[0.0, 2.5]]))
+
+
+def test_identity_embedding_reduces_to_verify_step_in_sampling_mode_too():
+    # W = identity: the logits are the hidden rows themselves, so the step from hidden states must
+    # be verify_step on those rows -- same acceptance draws, same extra token, same new candidates --
+    # for both resampling readings, with candidates that get accepted, rejected and are out of range
+    rng = np.random.default_rng(11)
+    k, V, Bn = 3, 24, 40
+    n_q = (k + 1) ** 2
+    h = rng.standard_normal((Bn, n_q, V)) * 2.0
+    cand = rng.integers(0, V, size=(Bn, k))
+    cand[:10, 0] = np.argmax(h[:10, 0], axis=-1)               # likely accepted
+    cand[10, 1] = V + 3                                        # out of range
+    P_c = np.ones((Bn, k))
+    P_c[11, :] = np.inf                                        # Algorithm 1's initial state
+    for resample in ("residual_pointmass", "paper_literal"):
+        if resample == "paper_literal":
+            P_c = np.where(np.isinf(P_c), P_c, rng.uniform(0.2, 1.0, size=P_c.shape))
+        kw = dict(temperature=0.7, seed=99, seq_id=np.arange(Bn) + 5, kv_len=rng.integers(0, 50, size=Bn),
+                  resample=resample)
+        r = lmhead_verify_step(h, np.eye(V), cand, P_c, k, mode="sample", **kw)
+        ref = verify_step(h, cand, P_c, k, "sample", **kw)
+        for key in ("n_accept", "out_tokens", "n_out", "next_cand", "next_cand_prob", "finished",
+                    "accept_margin", "bonus_gap", "draft_gap"):
+            assert np.array_equal(r[key], ref[key]), (resample, key)
+        assert r["n_accept"].max() > 0 and r["n_accept"][11] == 0
