@@ -308,6 +308,9 @@ int space_lmhead_verify(space_ctx* ctx, const space_lmhead_args* args, void* str
 int space_kv_commit(space_ctx* ctx, const space_commit_args* args, void* stream);
 
 /* The three stages from host buffers; synchronises `stream` before returning.
+ * (The logits go up and the attention output comes down on a second stream of the
+ * context, ordered against `stream` by events, so that both copies overlap the kernels;
+ * when the call returns everything it enqueued on either stream has finished.)
  * Needs cfg.host_staging.  Only sequence prefixes in use are copied (with
  * cache_resident: only the block's rows, see the field).  The call stages the
  * small per-sequence arrays in a pinned buffer of the context: one call at a

@@ -97,6 +97,8 @@ struct space_ctx {
   // staging for space_step_host
   char* stage;
   char* host_small;        // pinned host mirror of the staging area's small per-sequence arrays (host_staging only)
+  cudaStream_t aux_stream; // space_step_host: second stream, so that the logits upload and the download of the
+  cudaEvent_t aux_ev[4];   //   attention output overlap the kernels (host_staging only)
   size_t stage_bytes;
   // per-kernel event timing (space_profile_*)
   int prof_on;

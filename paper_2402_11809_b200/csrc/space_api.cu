@@ -214,6 +214,17 @@ int space_create(space_ctx** out, const space_config* cfg) {
     delete ctx;
     return SPACE_E_CUDA;
   }
+  if (cfg->host_staging) {
+    bool ok = cudaStreamCreateWithFlags(&ctx->aux_stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; i < 4 && ok; ++i) ok = cudaEventCreateWithFlags(&ctx->aux_ev[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      cudaGetLastError();
+      if (ctx->host_small) cudaFreeHost(ctx->host_small);
+      cudaFree(ctx->ws);
+      delete ctx;
+      return SPACE_E_CUDA;
+    }
+  }
   // counters and status start at zero; the kernels restore them after use
   if (cudaMemset(ctx->ws + cv.counters, 0, cv.stage - cv.counters) != cudaSuccess) {
     if (ctx->host_small) cudaFreeHost(ctx->host_small);
@@ -234,6 +245,10 @@ void space_destroy(space_ctx* ctx) {
     free(ctx->prof_ev[w]);
   }
   if (ctx->host_small) cudaFreeHost(ctx->host_small);
+  if (ctx->aux_stream) {
+    for (int i = 0; i < 4; ++i) if (ctx->aux_ev[i]) cudaEventDestroy(ctx->aux_ev[i]);
+    cudaStreamDestroy(ctx->aux_stream);
+  }
   cudaFree(ctx->ws);
   delete ctx;
 }
@@ -377,16 +392,15 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* a, void* stream)
     h2d += (int64_t)n;
     return cudaMemcpyAsync(dst, src, n, cudaMemcpyHostToDevice, st) == cudaSuccess;
   };
-  auto down = [&](void* dst, const void* src, size_t n) {
-    d2h += (int64_t)n;
-    return cudaMemcpyAsync(dst, src, n, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  };
   bool ok = true;
   const size_t row_b = (size_t)d * 2, head_pitch = (size_t)c.s_cap * row_b;
   const size_t seq_b = (size_t)c.n_kv_heads * head_pitch;
   const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;
+  // Two streams: what attention needs (q, the K/V rows, the lengths) goes up first on `st`; the logits
+  // follow on the second stream while attention already runs; the attention output comes down on the
+  // second stream while verification runs.  Events order the two; the call ends with everything done.
+  cudaStream_t sb = ctx->aux_stream;
   ok = ok && up(d_q, a->q, (size_t)B * n_q * c.n_q_heads * d * 2);
-  ok = ok && up(d_logits, a->logits, (size_t)B * n_q * a->vocab * esz);
   // the small per-sequence arrays travel as one block each way through a pinned mirror of their slots
   char* hsm = ctx->host_small;
   memcpy(hsm, a->kv_len, (size_t)B * 4);
@@ -407,6 +421,11 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* a, void* stream)
     h2d += 2 * (int64_t)w * c.n_kv_heads;
   }
   ok = ok && cudaMemsetAsync(d_status, 0, (size_t)B * 4, st) == cudaSuccess;
+  ok = ok && cudaEventRecord(ctx->aux_ev[0], st) == cudaSuccess;          // attention's inputs are on their way
+  ok = ok && cudaStreamWaitEvent(sb, ctx->aux_ev[0], 0) == cudaSuccess;
+  h2d += (int64_t)((size_t)B * n_q * a->vocab * esz);
+  ok = ok && cudaMemcpyAsync(d_logits, a->logits, (size_t)B * n_q * a->vocab * esz, cudaMemcpyHostToDevice, sb) == cudaSuccess;
+  ok = ok && cudaEventRecord(ctx->aux_ev[1], sb) == cudaSuccess;          // logits uploaded
   if (!ok) { cudaGetLastError(); return SPACE_E_CUDA; }
 
   space_attn_args at{};
@@ -417,6 +436,14 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* a, void* stream)
   at.kv_len = d_kvlen; at.out = d_out; at.lse = nullptr; at.status = d_status;
   int rc = space_attn_step(ctx, &at, stream);
   if (rc != SPACE_OK) return rc;
+  // the attention output leaves on the second stream, under the verification kernels
+  ok = ok && cudaEventRecord(ctx->aux_ev[2], st) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(sb, ctx->aux_ev[2], 0) == cudaSuccess;
+  d2h += (int64_t)((size_t)B * n_q * c.n_q_heads * d * 4);
+  ok = ok && cudaMemcpyAsync(a->out, d_out, (size_t)B * n_q * c.n_q_heads * d * 4, cudaMemcpyDeviceToHost, sb) == cudaSuccess;
+  ok = ok && cudaEventRecord(ctx->aux_ev[3], sb) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(st, ctx->aux_ev[1], 0) == cudaSuccess;   // verification needs the logits
+  if (!ok) { cudaGetLastError(); return SPACE_E_CUDA; }
   space_verify_args ve{};
   ve.batch = B; ve.k = k; ve.vocab = a->vocab; ve.logits_dtype = a->logits_dtype; ve.mode = a->mode;
   ve.resample = a->resample; ve.eos_id = a->eos_id; ve.temperature = a->temperature; ve.seed = a->seed;
@@ -430,7 +457,6 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* a, void* stream)
   rc = space_verify_commit(ctx, &ve, &cm, stream);
   if (rc != SPACE_OK) return rc;
 
-  ok = ok && down(a->out, d_out, (size_t)B * n_q * c.n_q_heads * d * 4);
   ok = ok && cudaMemcpyAsync(hsm + 3 * slot, d_small + 3 * slot, 8 * slot, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   d2h += (int64_t)B * (4 + k1 * 4 + 4 + k * 4 + k * 4 + 1 + 4 + 4);
   for (int b = 0; b < B && ok; ++b) {                    // rows L .. L+k: the compacted rows
@@ -443,6 +469,7 @@ int space_step_host(space_ctx* ctx, const space_host_step_args* a, void* stream)
                                  cudaMemcpyDeviceToHost, st) == cudaSuccess;
     d2h += 2 * (int64_t)w * c.n_kv_heads;
   }
+  ok = ok && cudaStreamWaitEvent(st, ctx->aux_ev[3], 0) == cudaSuccess;   // ... and the output has arrived
   if (!ok) { cudaGetLastError(); return SPACE_E_CUDA; }
   if (cudaStreamSynchronize(st) != cudaSuccess) return SPACE_E_CUDA;
   memcpy(a->n_accept, hsm + 3 * slot, (size_t)B * 4);
