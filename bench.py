@@ -38,10 +38,10 @@ L2_BYTES = 126 * 1024 * 1024
 # summarised under profiles/: (bytes, kernel source file, first 12 hex digits of that file's sha256 when
 # the capture was taken).  The figure is reported only while the source still has that hash; once the
 # kernel has changed the bench line carries null until the capture is taken again.
-ATTN_TRAFFIC = {"llama7b": (34518272, "attn_tc.cu", "000000000000"),
-                "gqa70b": (293366272, "attn_rows.cu", "000000000000")}
-LMHEAD_TRAFFIC = {"lmhead_llama7b": (266427264, "lmhead.cu", "000000000000"),
-                  "lmhead_vocab128k": (1071626000, "lmhead.cu", "000000000000")}
+ATTN_TRAFFIC = {"llama7b": (34521600, "attn_tc.cu", "78e14be6371c"),
+                "gqa70b": (292651392, "attn_rows.cu", "de4dcfd5fc39")}
+LMHEAD_TRAFFIC = {"lmhead_llama7b": (266501000, "lmhead.cu", "d9399b3ecf84"),
+                  "lmhead_vocab128k": (1088925000, "lmhead.cu", "d9399b3ecf84")}
 METRIC = "auto-correct steps/sec"
 UNIT = "steps/s"
 
@@ -229,7 +229,9 @@ def run_ours(args):
     torch.cuda.set_device(local)
     replicas.init("nccl", local)
 
-    cfg = workloads.resolve(args.config)
+    cfg = workloads.resolve(args.config, **({"B": args.batch} if args.batch else {}))
+    if args.batch:
+        cfg["name"] = f"{args.config}@batch{args.batch}"   # a reduced copy of the workload (profiler captures)
     k, n_q = cfg["k"], workloads.n_block_rows(cfg["k"])
     sample = cfg["mode"] == "sample"
     mode = B.MODE_SAMPLE if sample else B.MODE_GREEDY
@@ -647,6 +649,9 @@ def main():
     ap.add_argument("--config", default="llama7b",
                     choices=sorted(workloads.CONFIGS) + sorted(workloads.LMHEAD_CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the workload's batch size (a smaller copy of a large workload for profiler "
+                         "captures; the bench line then names the workload NAME@batchN)")
     ap.add_argument("--separate-commit", action="store_true",
                     help="three calls per step (space_verify, then space_kv_commit) instead of space_verify_commit")
     ap.add_argument("--attn-impl", default="tensor", choices=["tensor", "rows"],

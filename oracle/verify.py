@@ -38,6 +38,13 @@ the test r*P_c <= Q by accident).
         token's probability.
 Greedy mode is the zero-temperature limit: accept iff c_i is the arg-max of Q,
 a = argmax Q, new candidates are the mask rows' arg-maxes.
+
+Filtered sampling (App. A.4 runs random sampling with top-k = 10 and top-p = 0.95): with
+top_k > 0 every distribution that is sampled from or tested against -- Q of the target rows,
+and the mask rows' distributions when candidates are sampled -- is softmax(z / T) restricted
+to its top_k largest logits (lowest index first on ties), then to the shortest prefix of
+those, in descending order, whose probability reaches top_p, and renormalised.  The
+auto-correct step is then lossless with respect to that filtered distribution.
 """
 import numpy as np
 
@@ -53,6 +60,34 @@ def softmax_rows(z, T=1.0):
     z = z - z.max(axis=-1, keepdims=True)
     e = np.exp(z)
     return e / e.sum(axis=-1, keepdims=True)
+
+
+def filter_top_k_top_p(z, T, top_k, top_p):
+    """z [..., V] logits -> (filtered, renormalised probabilities [..., V], nucleus_margin [...]).
+
+    Temperature, then top-k, then top-p, in that order: keep the top_k largest z (ties: lower
+    index first); p = softmax(z / T) over them; in descending order keep token j while the
+    probability of the tokens before it is below top_p (the first one is always kept).
+    nucleus_margin: smallest |that cumulative probability - top_p| over the top-k tokens after the
+    first -- how close the floating-point decision "before it is below top_p" came to a tie."""
+    z = np.asarray(z, dtype=np.float64)
+    shape, V = z.shape[:-1], z.shape[-1]
+    z2 = z.reshape(-1, V)
+    K = min(int(top_k), V) if top_k > 0 else V
+    order = np.argsort(-z2, axis=1, kind="stable")[:, :K]    # descending, lowest index first on ties
+    s = np.take_along_axis(z2, order, axis=1) / T
+    p = np.exp(s - s[:, :1])
+    p /= p.sum(axis=1, keepdims=True)
+    cum = np.cumsum(p, axis=1)
+    before = np.concatenate((np.zeros((z2.shape[0], 1)), cum[:, :-1]), axis=1)   # probability of the tokens before j
+    keep = before < top_p
+    keep[:, 0] = True
+    margin = np.abs(before[:, 1:] - top_p).min(axis=1) if K > 1 else np.full(z2.shape[0], np.inf)
+    pk = np.where(keep, p, 0.0)
+    pk /= pk.sum(axis=1, keepdims=True)
+    out = np.zeros_like(z2)
+    np.put_along_axis(out, order, pk, axis=1)
+    return out.reshape(shape + (V,)), margin.reshape(shape)
 
 
 def gumbel_noise(seed, purpose, seq_id, position, V):
@@ -84,14 +119,15 @@ def _top2_gap(score):
 
 
 def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed=0,
-                seq_id=None, kv_len=None, resample="residual_pointmass", eos_id=-1):
+                seq_id=None, kv_len=None, resample="residual_pointmass", eos_id=-1, top_k=0, top_p=1.0):
     """logits [B, n_q, V]; cand (L_c) [B, k] ints; cand_prob (P_c) [B, k].
 
     Returns a dict: n_accept (i*), out_tokens [B, k+1] (-1 padded), n_out,
     next_cand, next_cand_prob, finished, and tie diagnostics
     (accept_margin [B, k] relative distance of the acceptance test from
     equality, bonus_gap [B], draft_gap [B, k] Gumbel top-two gaps; inf when
-    no floating-point decision was taken).
+    no floating-point decision was taken; nucleus_margin [B] likewise for the top-p cuts of
+    the rows that were read).
     """
     logits = np.asarray(logits)
     B, n_q, V = logits.shape
@@ -110,6 +146,8 @@ def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed
 
     if greedy:
         top = np.argmax(z_t, axis=-1)                        # lowest index on ties
+    elif top_k > 0:
+        Qrows, q_margin = filter_top_k_top_p(z_t, T, top_k, top_p)   # [B, k+1, V], [B, k+1]
     else:
         Qrows = softmax_rows(z_t, T)                         # [B, k+1, V]
 
@@ -168,6 +206,11 @@ def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed
     next_cand = np.zeros((B, k), dtype=np.int64)
     next_cand_prob = np.zeros((B, k), dtype=np.float64)
     draft_gap = np.full((B, k), np.inf)
+    nucleus_margin = np.full(B, np.inf)
+    if not greedy and top_k > 0:
+        # target rows 0 .. i* are the ones whose filtered distribution was used
+        used = np.arange(k + 1)[None, :] <= i_star[:, None]
+        nucleus_margin = np.where(used, q_margin, np.inf).min(axis=1)
     rows = np.array([mask_group_rows(k, g) for g in range(k + 1)])   # [k+1, k]
     for o in range(1, k + 1):
         z = as_f64(logits[bi, rows[i_star, o - 1], :])       # [B, V]
@@ -178,8 +221,13 @@ def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed
             next_cand[:, o - 1] = np.argmax(z, axis=-1)
             next_cand_prob[:, o - 1] = 1.0
         else:
-            p = softmax_rows(z, T)
-            score = np.log(p) + gumbel_noise(seed, PURPOSE_DRAFT, seq_id, L + i_star + 1 + o, V)
+            if top_k > 0:
+                p, m_o = filter_top_k_top_p(z, T, top_k, top_p)
+                nucleus_margin = np.minimum(nucleus_margin, m_o)
+            else:
+                p = softmax_rows(z, T)
+            with np.errstate(divide="ignore"):
+                score = np.log(p) + gumbel_noise(seed, PURPOSE_DRAFT, seq_id, L + i_star + 1 + o, V)
             best, gap = _top2_gap(score)
             next_cand[:, o - 1] = best
             next_cand_prob[:, o - 1] = p[bi, best]
@@ -187,4 +235,5 @@ def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed
 
     return dict(n_accept=i_star, out_tokens=out_tokens, n_out=n_out, next_cand=next_cand,
                 next_cand_prob=next_cand_prob, finished=finished,
-                accept_margin=accept_margin, bonus_gap=bonus_gap, draft_gap=draft_gap)
+                accept_margin=accept_margin, bonus_gap=bonus_gap, draft_gap=draft_gap,
+                nucleus_margin=nucleus_margin)

@@ -592,7 +592,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           if (g >= (uint32_t)n_st)
             ok = mbar_wait(BAR(b_empty + s), ((g / n_st) - 1) & 1, abort_flag, p.err, is_k ? 1 : 2);
           if (!ok) break;
-          if (v_hold) {
+          if (v_hold || (is_k && g == 1)) {                 // (the second K tile holds back as well)
             ok = mbar_wait(BAR(B_KFULL), 0, abort_flag, p.err, 14);
             v_hold = false;
             if (!ok) break;

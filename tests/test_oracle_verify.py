@@ -291,3 +291,67 @@ def test_acceptance_needs_a_positive_probability_and_an_in_range_token():
             r = verify_step(z, np.full((8, k), c0), np.full((8, k), bad_p), k, "sample",
                             seed=3, seq_id=np.arange(8))
             assert np.all(r["n_accept"] == 0), (bad_p, c0)
+
+
+# ------------------------------------------------ filtered sampling (top-k, then top-p)
+def test_filter_on_a_hand_written_row():
+    from oracle.verify import filter_top_k_top_p
+    z = np.log(np.array([[0.05, 0.5, 0.15, 0.2, 0.1]]))
+    # top-k = 4 drops token 0; renormalised 0.5, 0.2, 0.15, 0.1 -> 10/19, 4/19, 3/19, 2/19
+    p, m = filter_top_k_top_p(z, 1.0, 4, 1.0)
+    assert np.allclose(p[0], np.array([0, 10, 3, 4, 2]) / 19.0)
+    # top-p = 0.7 on top of it: 10/19 = 0.526 < 0.7 -> token 3 (4/19) is kept too, 14/19 >= 0.7 -> stop
+    p, m = filter_top_k_top_p(z, 1.0, 4, 0.7)
+    assert np.allclose(p[0], np.array([0, 10, 0, 4, 0]) / 14.0)
+    assert abs(m[0] - min(abs(10 / 19 - 0.7), abs(14 / 19 - 0.7), abs(17 / 19 - 0.7))) < 1e-12
+    # the first token is always kept; top_k beyond the vocabulary and top_p = 1 change nothing
+    p, _ = filter_top_k_top_p(z, 1.0, 4, 0.01)
+    assert p[0].tolist() == [0, 1, 0, 0, 0]
+    p, _ = filter_top_k_top_p(z, 0.5, 99, 1.0)
+    assert np.allclose(p[0], softmax_rows(z, 0.5)[0])
+    # a tie at the top-k boundary goes to the lower token; temperature acts before the cut
+    zt = np.array([[1.0, 3.0, 1.0, 1.0]])
+    p, _ = filter_top_k_top_p(zt, 2.0, 2, 1.0)
+    e = np.exp(-1.0)
+    assert np.allclose(p[0], np.array([e, 1, 0, 0]) / (1 + e))
+
+
+def test_filtered_sampling_is_lossless_for_the_filtered_law():
+    # point-mass drafts, top-k = 5 and top-p = 0.9: the first emitted token follows the filtered Q of
+    # row 0, a token outside the filter is never emitted, and a candidate outside it is never accepted
+    from oracle.verify import filter_top_k_top_p
+    k, T, seed, tk, tp = 2, 0.8, 77, 5, 0.9
+    z = _fixed_logits(k, 5)
+    qf, _ = filter_top_k_top_p(z[0, layout.target_rows(k)], T, tk, tp)       # [k+1, V]
+    inside = int(np.argsort(qf[0])[-2])                                      # second most likely kept token
+    outside = int(np.argmin(qf[0]))
+    assert qf[0, outside] == 0.0 and 0.0 < qf[0, inside] < 1.0
+    for c0 in (inside, outside):
+        cand = np.broadcast_to(np.array([c0, int(np.argmax(qf[1]))]), (N, k))
+        r = verify_step(z, cand, np.ones((N, k)), k, "sample", temperature=T, seed=seed, seq_id=np.arange(N),
+                        kv_len=np.full(N, 2), top_k=tk, top_p=tp)
+        acc = (r["n_accept"] >= 1).mean()
+        assert abs(acc - qf[0, c0]) < 5 * np.sqrt(max(qf[0, c0] * (1 - qf[0, c0]), 1e-9) / N) + 1e-12
+        counts = np.bincount(r["out_tokens"][:, 0], minlength=V16)
+        chi, _ = _chi2(counts, qf[0])                                        # also asserts: nothing outside the filter
+        assert chi < 55.0, chi
+        sel = r["n_accept"] >= 1
+        if sel.any():
+            chi, _ = _chi2(np.bincount(r["out_tokens"][sel, 1], minlength=V16), qf[1])
+            assert chi < 55.0, chi
+    # without a filter the same call does emit tokens outside it
+    r = verify_step(z, cand, np.ones((N, k)), k, "sample", temperature=T, seed=seed, seq_id=np.arange(N))
+    assert np.bincount(r["out_tokens"][:, 0], minlength=V16)[qf[0] == 0].sum() > 0
+
+
+def test_filtered_literal_reading_samples_candidates_from_the_filtered_rows():
+    from oracle.verify import filter_top_k_top_p
+    k, T, tk, tp = 1, 1.0, 4, 0.95
+    z = _fixed_logits(k, 6)
+    r = verify_step(z, np.zeros((N, k), dtype=int), np.full((N, k), INF), k, "sample", temperature=T, seed=3,
+                    seq_id=np.arange(N), resample="paper_literal", top_k=tk, top_p=tp)
+    pm, _ = filter_top_k_top_p(z[0, layout.mask_group_rows(k, 0)[0]], T, tk, tp)
+    chi, _ = _chi2(np.bincount(r["next_cand"][:, 0], minlength=V16), pm)
+    assert chi < 55.0, chi
+    assert np.allclose(r["next_cand_prob"][:, 0], pm[r["next_cand"][:, 0]])
+    assert np.isfinite(r["nucleus_margin"]).all()
