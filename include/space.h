@@ -137,6 +137,12 @@ typedef struct {
   float*   next_cand_prob;     /* device [B, k]                                */
   uint8_t* finished;           /* device [B]       1 once <EOS> was emitted    */
   int32_t* status;             /* device [B] or NULL                           */
+  int32_t top_k;               /* sampling mode: 0 = unfiltered; 1..32 = every distribution that is tested
+                                  against or sampled from is softmax(z/T) over its top_k largest logits
+                                  (lowest token first on ties), cut to the shortest prefix, in descending
+                                  order, whose probability reaches top_p, and renormalised (App. A.4 runs
+                                  sampling with top-k = 10, top-p = 0.95); ignored in greedy mode        */
+  float   top_p;               /* in (0, 1] when top_k > 0 (1 = no nucleus cut)                         */
 } space_verify_args;
 
 /* Output projection fused with verification: the end of the model call P = M(I) of

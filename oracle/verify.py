@@ -67,7 +67,8 @@ def filter_top_k_top_p(z, T, top_k, top_p):
 
     Temperature, then top-k, then top-p, in that order: keep the top_k largest z (ties: lower
     index first); p = softmax(z / T) over them; in descending order keep token j while the
-    probability of the tokens before it is below top_p (the first one is always kept).
+    probability of the tokens before it is below top_p (the first one is always kept; top_p >= 1
+    keeps all of them).
     nucleus_margin: smallest |that cumulative probability - top_p| over the top-k tokens after the
     first -- how close the floating-point decision "before it is below top_p" came to a tie."""
     z = np.asarray(z, dtype=np.float64)
@@ -80,9 +81,13 @@ def filter_top_k_top_p(z, T, top_k, top_p):
     p /= p.sum(axis=1, keepdims=True)
     cum = np.cumsum(p, axis=1)
     before = np.concatenate((np.zeros((z2.shape[0], 1)), cum[:, :-1]), axis=1)   # probability of the tokens before j
-    keep = before < top_p
-    keep[:, 0] = True
-    margin = np.abs(before[:, 1:] - top_p).min(axis=1) if K > 1 else np.full(z2.shape[0], np.inf)
+    if top_p >= 1.0:                                         # no nucleus cut at all
+        keep = np.ones_like(before, dtype=bool)
+        margin = np.full(z2.shape[0], np.inf)
+    else:
+        keep = before < top_p
+        keep[:, 0] = True
+        margin = np.abs(before[:, 1:] - top_p).min(axis=1) if K > 1 else np.full(z2.shape[0], np.inf)
     pk = np.where(keep, p, 0.0)
     pk /= pk.sum(axis=1, keepdims=True)
     out = np.zeros_like(z2)

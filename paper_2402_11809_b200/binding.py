@@ -69,7 +69,8 @@ class VerifyArgs(C.Structure):
                 ("cand", C.c_void_p), ("cand_prob", C.c_void_p), ("seq_id", C.c_void_p),
                 ("kv_len", C.c_void_p), ("n_accept", C.c_void_p), ("out_tokens", C.c_void_p),
                 ("n_out", C.c_void_p), ("next_cand", C.c_void_p), ("next_cand_prob", C.c_void_p),
-                ("finished", C.c_void_p), ("status", C.c_void_p)]
+                ("finished", C.c_void_p), ("status", C.c_void_p),
+                ("top_k", C.c_int32), ("top_p", C.c_float)]
 
 
 class CommitArgs(C.Structure):
@@ -268,7 +269,8 @@ class Context:
     # -- space_verify -----------------------------------------------------
     def verify_args(self, logits, cand, cand_prob, kv_len, n_accept, out_tokens, n_out, next_cand,
                     next_cand_prob, finished, k, mode=MODE_GREEDY, temperature=1.0, seed=0,
-                    resample=RESAMPLE_RESIDUAL_POINTMASS, eos_id=-1, seq_id=None, status=None):
+                    resample=RESAMPLE_RESIDUAL_POINTMASS, eos_id=-1, seq_id=None, status=None,
+                    top_k=0, top_p=1.0):
         import torch
         assert logits.stride(2) == 1 and logits.stride(0) == logits.shape[1] * logits.stride(1)
         return VerifyArgs(batch=logits.shape[0], k=k, vocab=logits.shape[2],
@@ -279,7 +281,7 @@ class Context:
                           kv_len=_ptr(kv_len), n_accept=_ptr(n_accept), out_tokens=_ptr(out_tokens),
                           n_out=_ptr(n_out), next_cand=_ptr(next_cand),
                           next_cand_prob=_ptr(next_cand_prob), finished=_ptr(finished),
-                          status=_ptr(status))
+                          status=_ptr(status), top_k=top_k, top_p=top_p)
 
     def space_verify(self, args):
         _check(lib.space_verify(self._h, C.byref(args), _stream()))

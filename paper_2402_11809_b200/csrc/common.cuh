@@ -91,6 +91,7 @@ struct space_ctx {
   VerifyPartial* vpart;    // [max_batch][k_max+2][SPACE_VERIFY_MAX_CHUNKS]
   VerifyRow* vrow;         // [max_batch][k_max+1]
   VerifyPartial* vfused;   // [max_batch][SPACE_MAX_ROWS][16] single-launch greedy path
+  char* vtopk;             // filtered sampling: top-k lists per (sequence, row, chunk)
   int32_t* scratch_status; // [max_batch] used when the caller passes no status array
   char* lm_part;           // output-projection statistics [256 block rows][sm_count] x 16 bytes
   int* lm_counter;         // {arrival counter, first timeout site}
@@ -183,6 +184,8 @@ __device__ __forceinline__ void commit_tables(const CommitParams& p, int b, int 
 // ---- per-stage launchers (defined next to their kernels) -------------------
 // cm != nullptr: the verify kernels also carry out the commit described by cm (one launch less)
 int launch_verify(space_ctx* ctx, const space_verify_args* a, const space_commit_args* cm, cudaStream_t st);
+int launch_verify_filtered(space_ctx* ctx, const space_verify_args* a, cudaStream_t st);
+size_t verify_filter_scratch_bytes(int max_batch, int k_max);
 void fill_commit_params(const space_ctx* ctx, const space_commit_args* a, CommitParams* p);
 int launch_verify_noalloc(const space_verify_args* a, cudaStream_t st);
 int launch_commit(space_ctx* ctx, const space_commit_args* a, cudaStream_t st);

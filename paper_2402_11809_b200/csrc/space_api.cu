@@ -28,7 +28,7 @@ int config_supported(const space_config* c) {
 }
 
 struct Carve {
-  size_t attn_part, counters, merge_cnt, vpart, vfused, vrow, status, lm_part, lm_counter, stage, total;
+  size_t attn_part, counters, merge_cnt, vtopk, vpart, vfused, vrow, status, lm_part, lm_counter, stage, total;
   size_t part_slots;
   // staging sub-offsets (relative to stage)
   size_t st_q, st_k, st_v, st_logits, st_small;
@@ -43,6 +43,7 @@ Carve carve(const space_config* c, int sm_count) {
   v.merge_cnt = off;
   // up to 8 row blocks, one {first, count} pair each; then one word per thread block of the attention grid
   off += align_up((size_t)c->max_batch * c->n_kv_heads * 8 * sizeof(int2) + (size_t)(sm_count + 8) * sizeof(int), 256);
+  v.vtopk = off; off += align_up(verify_filter_scratch_bytes(c->max_batch, c->k_max), 256);
   v.vpart = off;
   off += align_up((size_t)c->max_batch * (c->k_max + 2) * SPACE_VERIFY_MAX_CHUNKS * sizeof(VerifyPartial), 256);
   static_assert(SPACE_FUSED_MAX_CHUNKS <= 16, "the single-launch verify reduces a row's chunks with 16 lanes");
@@ -119,6 +120,9 @@ int check_verify_args(const space_ctx* ctx, const space_verify_args* a) {
   if (a->resample != SPACE_RESAMPLE_RESIDUAL_POINTMASS && a->resample != SPACE_RESAMPLE_PAPER_LITERAL)
     return SPACE_E_INVALID_ARG;
   if (a->mode == SPACE_MODE_SAMPLE && !(a->temperature > 0.f)) return SPACE_E_INVALID_ARG;
+  if (a->mode == SPACE_MODE_SAMPLE && a->top_k != 0 &&
+      (a->top_k < 0 || a->top_k > 32 || !(a->top_p > 0.f) || a->top_p > 1.f))
+    return SPACE_E_INVALID_ARG;
   if (a->logits_row_stride < a->vocab) return SPACE_E_INVALID_ARG;
   const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;
   if ((uintptr_t)a->logits % esz) return SPACE_E_ALIGNMENT;
@@ -199,6 +203,7 @@ int space_create(space_ctx** out, const space_config* cfg) {
   ctx->counters = (int*)(ctx->ws + cv.counters);
   ctx->merge_cnt = (int*)(ctx->ws + cv.merge_cnt);
   ctx->vpart = (VerifyPartial*)(ctx->ws + cv.vpart);
+  ctx->vtopk = ctx->ws + cv.vtopk;
   ctx->vrow = (VerifyRow*)(ctx->ws + cv.vrow);
   ctx->vfused = (VerifyPartial*)(ctx->ws + cv.vfused);
   ctx->scratch_status = (int32_t*)(ctx->ws + cv.status);

@@ -692,6 +692,12 @@ __global__ void philox_debug_kernel(uint32_t k0, uint32_t k1, int64_t n, const u
 }  // namespace
 
 int launch_verify(space_ctx* ctx, const space_verify_args* a, const space_commit_args* cm, cudaStream_t st) {
+  if (a->mode == SPACE_MODE_SAMPLE && a->top_k > 0) {
+    // filtered target distributions: kernels of their own (verify_filter.cu); the commit follows as its own launch
+    const int rc = launch_verify_filtered(ctx, a, st);
+    if (rc != SPACE_OK || !cm) return rc;
+    return launch_commit(ctx, cm, st);
+  }
   VerifyParams p;
   p.do_commit = cm != nullptr;
   if (cm) fill_commit_params(ctx, cm, &p.cm); else memset(&p.cm, 0, sizeof(p.cm));

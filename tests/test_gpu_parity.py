@@ -483,3 +483,66 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable(B, H):
     ref, _ = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], 3, x["scale"])
     _check_attention(H, ds.out.cpu().numpy().astype(np.float64), ref, "after a time-out")
     assert int(ds.status.abs().sum()) == 0
+
+
+# ------------------------------------------------- filtered sampling (top-k, top-p)
+NUCLEUS_BAND = 1e-5     # distance of a cumulative probability from top_p below which the nucleus cut is a tie
+
+
+@pytest.mark.parametrize("resample", ["residual_pointmass", "paper_literal"])
+@pytest.mark.parametrize("k,V,Bn,T,top_k,top_p,dtype", [
+    (2, 16, 48, 1.0, 5, 0.9, "f32"),          # tiny vocabulary
+    (4, 5000, 16, 0.8, 10, 0.95, "bf16"),     # the paper's setting (App. A.4)
+    (3, 128256, 4, 0.8, 10, 0.95, "bf16"),    # full vocabulary, several chunks per row
+    (5, 9, 6, 0.7, 32, 1.0, "f32"),           # top_k beyond the vocabulary, no nucleus cut: unfiltered
+    (1, 40000, 7, 1.3, 1, 0.5, "bf16"),       # top-1: deterministic
+])
+def test_verify_filtered_sampling(B, H, resample, k, V, Bn, T, top_k, top_p, dtype):
+    cfg = workloads.resolve("sampling64", B=Bn, H_q=1, H_kv=1, d=64, L=(5, 600), k=k, V=V, temperature=T,
+                            logits_dtype=dtype, seed=400 + k)
+    x = workloads.make_step_inputs(cfg)
+    rng = np.random.default_rng(k)
+    if resample == "paper_literal":
+        x["cand_prob"] = rng.uniform(0.2, 1.0, size=x["cand_prob"].shape).astype(np.float32)
+    x["cand_prob"][0, :] = np.inf
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    code = B.RESAMPLE_RESIDUAL_POINTMASS if resample == "residual_pointmass" else B.RESAMPLE_PAPER_LITERAL
+    kept_outside = 0
+    for seed in (1, 0xABCDEF0123):
+        a = ctx.verify_args(ds.logits, ds.cand, ds.cand_prob, ds.kv_len, ds.n_accept, ds.out_tokens, ds.n_out,
+                            ds.next_cand, ds.next_cand_prob, ds.finished, k, mode=B.MODE_SAMPLE, temperature=T,
+                            seed=seed, resample=code, seq_id=ds.seq_id, status=ds.status, top_k=top_k, top_p=top_p)
+        ctx.space_verify(a)
+        r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "sample", temperature=T, seed=seed,
+                        seq_id=x["seq_id"], kv_len=x["kv_len"], resample=resample, top_k=top_k, top_p=top_p)
+        nuc = r["nucleus_margin"] <= NUCLEUS_BAND
+        r["accept_margin"] = np.where(nuc[:, None], 0.0, r["accept_margin"])    # a nucleus tie excludes the sequence
+        _check_verify(ds, r, k, sample=True)
+        assert r["n_accept"][0] == 0
+        kept_outside += int((r["out_tokens"][:, 0] >= 0).sum())
+    assert kept_outside > 0
+    # the same call through space_verify_commit moves the accepted rows as well
+    ds2 = H.DeviceStep(cfg, x)
+    v = ctx.verify_args(ds2.logits, ds2.cand, ds2.cand_prob, ds2.kv_len, ds2.n_accept, ds2.out_tokens, ds2.n_out,
+                        ds2.next_cand, ds2.next_cand_prob, ds2.finished, k, mode=B.MODE_SAMPLE, temperature=T,
+                        seed=seed, resample=code, seq_id=ds2.seq_id, status=ds2.status, top_k=top_k, top_p=top_p)
+    c = ctx.commit_args(ds2.k_cache, ds2.v_cache, ds2.n_accept, ds2.kv_len, k, kv_len_out=ds2.kv_len_out)
+    ctx.space_verify_commit(v, c)
+    _check_verify(ds2, r, k, sample=True)
+    Kc, Vc = x["k_cache"].copy(), x["v_cache"].copy()
+    new_len, _, _ = commit_step(Kc, Vc, x["kv_len"], ds2.n_accept.cpu().numpy(), k)
+    assert np.array_equal(H.bf16_to_bits(ds2.k_cache), Kc) and np.array_equal(ds2.kv_len_out.cpu().numpy(), new_len)
+
+
+def test_verify_filter_arguments(B, H):
+    import ctypes as C
+    cfg = workloads.resolve("sampling64", B=2, H_q=1, H_kv=1, d=64, L=(5, 50), k=2, V=100, seed=1)
+    x = workloads.make_step_inputs(cfg)
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    mk = lambda **kw: ctx.verify_args(ds.logits, ds.cand, ds.cand_prob, ds.kv_len, ds.n_accept, ds.out_tokens, ds.n_out,
+                                      ds.next_cand, ds.next_cand_prob, ds.finished, 2, mode=B.MODE_SAMPLE, temperature=1.0, **kw)
+    for bad in (dict(top_k=33, top_p=0.9), dict(top_k=-1, top_p=0.9), dict(top_k=5, top_p=0.0), dict(top_k=5, top_p=1.5)):
+        assert B.lib.space_verify(ctx._h, C.byref(mk(**bad)), None) == B.E_INVALID_ARG, bad
+    torch.cuda.synchronize()
