@@ -326,6 +326,8 @@ __device__ __noinline__ void piece_rescale(uint32_t taddr, const float* fq) {
 
 // Warp roles
 constexpr int WARP_K = 0, WARP_MMA = 1, WARP_V = 2, WARP_PV = 3, WARP_SOFTMAX0 = 4;
+constexpr int L2_AHEAD_TILES = 1;      // tiles per operand a block asks L2 for before its dependency wait (more of them
+                                       // crowd out the kernels that still run: measured slower)
 constexpr float OVER_THRESHOLD = 60.f;   // re-reference a query row when a score exceeds its reference by 2^60
 
 // The tile products are taken transposed: S^T = K Q^T (128 keys x N query rows)
@@ -390,12 +392,35 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     const int j = threadIdx.x - WARP_SOFTMAX0 * 32;
     visq[j] = p.visq[mb][j];
   }
+  // single-sequence partition (explained where the tables are built, below)
+  const int sp_base = max(p.n_groups / p.H_kv, 1), sp_extra = p.n_groups - sp_base * p.H_kv;
+  const bool sp_helper = group >= sp_base * p.H_kv;
+  const int sp_h = sp_helper ? group - sp_base * p.H_kv : group / sp_base;
+  const int sp_piece = sp_helper ? 0 : group - sp_h * sp_base;
+  const bool early = p.spec && !sp_helper;                 // this group requests Q and its first K tile at once
   if (warp == WARP_K && lane == 0)
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_k) : "memory");
   if (warp == WARP_V && lane == 0)
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_v) : "memory");
   if (warp == WARP_MMA && lane == 0)
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_q) : "memory");
+  if (early && lane == 0 && (warp == WARP_K || warp == WARP_V)) {
+    // A regular group's tiles (sp_piece, sp_piece + sp_base, ...) of head sp_h do not depend on the
+    // length, so L2 is asked for them now, while the kernel before this one may still be running:
+    // with a programmatic launch this block is resident long before its dependency wait returns,
+    // and the tile loads after the wait then find their lines in L2 instead of paying the DRAM
+    // latency in a burst of all blocks at once.  Only a request to the cache: whatever the earlier
+    // kernel still writes is what the loads will see.  The length is read here as a hint for how
+    // many tiles are worth asking for (a stale value costs or saves a request, never an error).
+    const uint64_t pol = l2_evict_first_policy();
+    const int Lh = *reinterpret_cast<const volatile int*>(p.kv_len);
+    const int Th = (Lh >= 0 && (int64_t)Lh + p.n_q <= p.s_cap) ? (Lh + p.n_q) / TILE_N : 0;   // whole tiles
+    const CUtensorMap* tm = warp == WARP_K ? &p.tm_k : &p.tm_v;
+    for (int j = 0, t = sp_piece; j < L2_AHEAD_TILES && t < Th; ++j, t += sp_base) {
+#pragma unroll
+      for (int hf = 0; hf < S::HALVES; ++hf) tma_prefetch_l2_4d(tm, hf * 64, t * TILE_N, sp_h, 0, pol);
+    }
+  }
   // barriers and the TMEM allocation are visible to every warp before the first
   // global access (with a programmatic launch this part runs under the previous kernel)
   tc_fence_before();
@@ -410,11 +435,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   // left over are helpers that each take the last tile of some heads -- the one with the block's
   // own keys, whose Eq. 5 mask makes it the slowest -- so that no regular piece carries it on top
   // of its share of the full tiles.
-  const int sp_base = max(p.n_groups / p.H_kv, 1), sp_extra = p.n_groups - sp_base * p.H_kv;
-  const bool sp_helper = group >= sp_base * p.H_kv;
-  const int sp_h = sp_helper ? group - sp_base * p.H_kv : group / sp_base;
-  const int sp_piece = sp_helper ? 0 : group - sp_h * sp_base;
-  const bool early = p.spec && !sp_helper;                 // this group requests Q and its first K tile at once
   if (early && warp == WARP_K && lane == 0 && !*abort_flag) {
     // Which head and which first tile a regular group works on does not depend on the length,
     // so its query rows and its first K tile are requested before the length is even read (one
@@ -440,12 +460,34 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     if (!okL && blockIdx.x == 0 && threadIdx.x == 0 && p.status) atomicOr(p.status, SPACE_ST_CAPACITY);
     const int L = okL ? L0 : -1;
     const int T = okL ? (L + p.n_q + TILE_N - 1) / TILE_N : 0;
+    if (threadIdx.x == 0 && L0 != 0x7FFFFFFF) TL(14);
     seq_len[0] = L; prefix[0] = 0; prefix[1] = okL ? (T + SHARE_COST) * p.H_kv : 0;
     int ag = -1, spec_ok = 0;
     const int W = T * p.H_kv;
-    if (W > 0 && W < 8 * p.n_groups && p.H_kv <= p.n_groups) {
+    const bool cut_aligned = W > 0 && W < 8 * p.n_groups && p.H_kv <= p.n_groups;
+    const bool helpers = cut_aligned && sp_extra > 0 && T > sp_base;   // the last tile goes to a helper group
+    if (p.spec && sp_helper && helpers) {
+      // A helper knows its first share as soon as it has the length: the last tile of head sp_h.
+      // Its query rows and that tile are requested here, ahead of the tables and the producer's
+      // own start-up, which would come a microsecond later.
+      spec_ok = 1;
+      if (warp == WARP_K && lane == 0 && !*abort_flag) {
+        const int n_keys = L + p.n_q;
+        const int kt = (T * TILE_N <= n_keys) ? (T - 1) * TILE_N : n_keys - TILE_N;
+        mbar_expect_tx(BAR(B_QFULL), (uint32_t)n_pad * DH * 2);
+#pragma unroll
+        for (int hf = 0; hf < S::HALVES; ++hf)
+          tma_load_4d(sm_base + S::Q_OFF + hf * (n_pad * 128), &p.tm_q, BAR(B_QFULL), hf * 64, sp_h * p.G, i0, 0);
+        mbar_expect_tx(BAR(B_KFULL), S::TILE_BYTES);
+#pragma unroll
+        for (int hf = 0; hf < S::HALVES; ++hf)
+          tma_load_4d_hint(sm_base + S::K_OFF + hf * (TILE_N * 128), &p.tm_k, BAR(B_KFULL), hf * 64, kt, sp_h, 0,
+                           l2_evict_first_policy());
+        TL(3);
+      }
+    }
+    if (cut_aligned) {
       ag = p.n_groups;
-      const bool helpers = sp_extra > 0 && T > sp_base;    // the last tile goes to a helper group
       const int Treg = helpers ? T - 1 : T;                // tiles cut among the regular pieces
       const int dn = helpers ? sp_base + 1 : min(sp_base, T);
       if (!sp_helper) {
@@ -557,8 +599,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       // Early requests (one sequence): when this share's first tile is the requested one, the K
       // producer skips the query rows and that tile; when it is not, the two buffers are given
       // back by the S^T issuer and the rings start one slot further.
+      if (is_k) TL(15);
       const uint64_t kv_policy = l2_evict_first_policy();
-      bool pre = early && is_k && seg0[9] != 0;
+      bool pre = p.spec && is_k && seg0[9] != 0;           // Q and the first K tile of the first share are on their way
       const uint32_t koff = (early && is_k && !pre) ? 1u : 0u;
       uint32_t gt = 0, seg = koff;
       bool ok = true;
@@ -638,6 +681,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       }
       while (ok && part.next(sg)) {
         const uint32_t qb = seg % S::Q_BUFS, use = seg / S::Q_BUFS;
+        if (gt == 0) TL(12);
         ok = mbar_wait(BAR(B_QFULL + qb), use & 1, abort_flag, p.err, 6);
         const uint64_t qd = qdesc0 + (uint64_t)((qb * S::Q_BYTES) >> 4);
         const int n = sg.n;
@@ -1040,7 +1084,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
   // ---- teardown -----------------------------------------------------------
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0) TL(12);
   if (warp == WARP_MMA) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");

@@ -89,6 +89,14 @@ __device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap
       " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
       ::"r"(dst), "l"((uint64_t)tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol) : "memory");
 }
+// Asks L2 for one box of a 4-D tensor map without waiting for it and without a destination in
+// shared memory.  L2 is the point of coherence for global memory, so the request may be made
+// while an earlier kernel can still write the tensor: the later load sees the final bytes.
+__device__ __forceinline__ void tma_prefetch_l2_4d(const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.prefetch.tensor.4d.L2.global.tile.L2::cache_hint [%0, {%1, %2, %3, %4}], %5;"
+      ::"l"((uint64_t)tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol) : "memory");
+}
 // Policy for data that is read once per step: its lines are evicted first and leave the cache to
 // what is read again (kernel code, lengths, partials).
 __device__ __forceinline__ uint64_t l2_evict_first_policy() {

@@ -581,12 +581,12 @@ template <typename T, bool VECTOR>
 __global__ void __launch_bounds__(SPACE_VERIFY_THREADS)
 verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   pdl_launch_dependents();
-  pdl_wait();
   const int b = blockIdx.z, row_i = blockIdx.y, ch = blockIdx.x;
   const int k1 = p.k + 1;
   constexpr float C1 = 1.4426950408889634f;                 // T = 1
   const T* row = reinterpret_cast<const T*>(p.logits) + ((int64_t)b * p.n_q + row_i) * p.row_stride;
   const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
+  pdl_wait();
   int Lc = 0;
   if (p.do_commit) Lc = p.cm.kv_len[b];                     // in flight during the scan
   Stat st = scan_chunk<T, VECTOR, false, STAT_SUM>(row, begin, end, C1, -1, 0, 0, 0, 0, 0);
