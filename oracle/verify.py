@@ -36,6 +36,15 @@ the test r*P_c <= Q by accident).
   "paper_literal"       Algorithm 1 as printed: a ~ Q also after a rejection,
         new candidates are sampled from their mask rows and P_c is the sampled
         token's probability.
+  "residual_draft"      sampled candidates made lossless (needs top_k > 0): candidate o of the
+        next step is drawn from the filtered distribution D_o of its mask row, and the step hands
+        D_o on as a compact list (at most top_k tokens with their probabilities, descending) beside
+        L_c and P_c = D_o(L_c[o]).  The next step accepts c_i with probability min(1, Q(c_i)/P_c[i])
+        as Algorithm 1 does, and after rejecting c_i draws the extra token from the residual
+        norm(max(0, Q - D_i)), the rule of speculative sampling that Sec. 3.2's claim of an
+        unchanged output distribution rests on; after k acceptances, and in Algorithm 1's initial
+        state (empty lists), a ~ Q.  Should the residual have no mass (Q <= D_i everywhere, where a
+        rejection has probability zero) Q itself is used.
 Greedy mode is the zero-temperature limit: accept iff c_i is the arg-max of Q,
 a = argmax Q, new candidates are the mask rows' arg-maxes.
 
@@ -62,8 +71,10 @@ def softmax_rows(z, T=1.0):
     return e / e.sum(axis=-1, keepdims=True)
 
 
-def filter_top_k_top_p(z, T, top_k, top_p):
-    """z [..., V] logits -> (filtered, renormalised probabilities [..., V], nucleus_margin [...]).
+def filter_top_k_top_p(z, T, top_k, top_p, as_list=False):
+    """z [..., V] logits -> (filtered, renormalised probabilities [..., V], nucleus_margin [...]);
+    with as_list the distribution comes as (tokens [..., K], probabilities [..., K], margin) in
+    descending order, K = min(top_k, V), dropped entries as token -1 with probability 0.
 
     Temperature, then top-k, then top-p, in that order: keep the top_k largest z (ties: lower
     index first); p = softmax(z / T) over them; in descending order keep token j while the
@@ -92,7 +103,22 @@ def filter_top_k_top_p(z, T, top_k, top_p):
     pk /= pk.sum(axis=1, keepdims=True)
     out = np.zeros_like(z2)
     np.put_along_axis(out, order, pk, axis=1)
+    if as_list:
+        tok = np.where(keep, order, -1)
+        return tok.reshape(shape + (K,)), pk.reshape(shape + (K,)), margin.reshape(shape)
     return out.reshape(shape + (V,)), margin.reshape(shape)
+
+
+def compact_to_dense(tok, prob, V):
+    """Compact distribution lists tok, prob [B, K] -> dense [B, V]; entries with a token outside
+    [0, V) or a probability that is not a positive finite number do not count."""
+    tok = np.asarray(tok, dtype=np.int64)
+    prob = np.asarray(prob, dtype=np.float64)
+    ok = (tok >= 0) & (tok < V) & np.isfinite(prob) & (prob > 0)
+    out = np.zeros((tok.shape[0], V))
+    b = np.broadcast_to(np.arange(tok.shape[0])[:, None], tok.shape)
+    np.add.at(out, (b[ok], tok[ok]), prob[ok])
+    return out
 
 
 def gumbel_noise(seed, purpose, seq_id, position, V):
@@ -124,8 +150,14 @@ def _top2_gap(score):
 
 
 def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed=0,
-                seq_id=None, kv_len=None, resample="residual_pointmass", eos_id=-1, top_k=0, top_p=1.0):
-    """logits [B, n_q, V]; cand (L_c) [B, k] ints; cand_prob (P_c) [B, k].
+                seq_id=None, kv_len=None, resample="residual_pointmass", eos_id=-1, top_k=0, top_p=1.0,
+                draft_tok=None, draft_prob=None):
+    """logits [B, n_q, V]; cand (L_c) [B, k] ints; cand_prob (P_c) [B, k];
+    draft_tok, draft_prob [B, k, K_d] ("residual_draft" only): the compact distributions the
+    candidates were drawn from (None = empty lists, Algorithm 1's initial state).  That reading
+    also returns next_draft_tok, next_draft_prob [B, k, min(top_k, V)] and bonus_cond [B], the
+    condition number max(Q, D) / (Q - D) of the residual weight of the winning token or of its
+    runner-up, whichever is larger (1 when no subtraction took place).
 
     Returns a dict: n_accept (i*), out_tokens [B, k+1] (-1 padded), n_out,
     next_cand, next_cand_prob, finished, and tie diagnostics
@@ -177,6 +209,7 @@ def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed
 
     # ---- extra token a from the last accepted row ------------------------
     bonus_gap = np.full(B, np.inf)
+    bonus_cond = np.ones(B)
     if greedy:
         a = top[bi, i_star]
     else:
@@ -187,9 +220,29 @@ def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed
             rej = rej & in_range[bi, np.minimum(i_star, k - 1)]
             rej = rej & (P_c[bi, np.minimum(i_star, k - 1)] == 1.0)   # a point-mass draft only
             w[bi[rej], c_rej[rej]] = 0.0
+        if resample == "residual_draft":
+            assert top_k > 0, "compact draft distributions need top_k > 0"
+            Qw = w.copy()
+            D = np.zeros((B, V))
+            if draft_tok is not None:
+                dt = np.asarray(draft_tok)[bi, np.minimum(i_star, k - 1)]     # list of the rejected candidate
+                dp = np.asarray(draft_prob)[bi, np.minimum(i_star, k - 1)]
+                D = compact_to_dense(dt, dp, V)
+            D[i_star >= k] = 0.0                             # nothing was rejected
+            res = np.maximum(Qw - D, 0.0)
+            empty = res.sum(axis=1) <= 0.0
+            w = np.where(empty[:, None], Qw, res)
+            D[empty] = 0.0
         with np.errstate(divide="ignore"):
             score = np.log(w) + gumbel_noise(seed, PURPOSE_TOKEN, seq_id, L + i_star + 1, V)
         a, bonus_gap = _top2_gap(score)
+        if resample == "residual_draft":
+            s2 = score.copy()
+            s2[bi, a] = -np.inf
+            for t in (a, np.argmax(s2, axis=-1)):
+                ok_t = w[bi, t] > 0
+                cond = np.where(ok_t, np.maximum(Qw[bi, t], D[bi, t]) / np.where(ok_t, w[bi, t], 1.0), 1.0)
+                bonus_cond = np.maximum(bonus_cond, cond)
 
     out_tokens = np.full((B, k + 1), -1, dtype=np.int64)
     for j in range(k + 1):
@@ -216,6 +269,9 @@ def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed
         # target rows 0 .. i* are the ones whose filtered distribution was used
         used = np.arange(k + 1)[None, :] <= i_star[:, None]
         nucleus_margin = np.where(used, q_margin, np.inf).min(axis=1)
+    K_d = min(int(top_k), V) if top_k > 0 else 0
+    next_draft_tok = np.full((B, k, K_d), -1, dtype=np.int64)
+    next_draft_prob = np.zeros((B, k, K_d))
     rows = np.array([mask_group_rows(k, g) for g in range(k + 1)])   # [k+1, k]
     for o in range(1, k + 1):
         z = as_f64(logits[bi, rows[i_star, o - 1], :])       # [B, V]
@@ -229,6 +285,8 @@ def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed
             if top_k > 0:
                 p, m_o = filter_top_k_top_p(z, T, top_k, top_p)
                 nucleus_margin = np.minimum(nucleus_margin, m_o)
+                if resample == "residual_draft":
+                    next_draft_tok[:, o - 1], next_draft_prob[:, o - 1], _ = filter_top_k_top_p(z, T, top_k, top_p, as_list=True)
             else:
                 p = softmax_rows(z, T)
             with np.errstate(divide="ignore"):
@@ -241,4 +299,5 @@ def verify_step(logits, cand, cand_prob, k, mode="greedy", temperature=1.0, seed
     return dict(n_accept=i_star, out_tokens=out_tokens, n_out=n_out, next_cand=next_cand,
                 next_cand_prob=next_cand_prob, finished=finished,
                 accept_margin=accept_margin, bonus_gap=bonus_gap, draft_gap=draft_gap,
-                nucleus_margin=nucleus_margin)
+                nucleus_margin=nucleus_margin, bonus_cond=bonus_cond,
+                next_draft_tok=next_draft_tok, next_draft_prob=next_draft_prob)

@@ -355,3 +355,100 @@ def test_filtered_literal_reading_samples_candidates_from_the_filtered_rows():
     assert chi < 55.0, chi
     assert np.allclose(r["next_cand_prob"][:, 0], pm[r["next_cand"][:, 0]])
     assert np.isfinite(r["nucleus_margin"]).all()
+
+
+# ------------------------------------------------ compact draft distributions, full residual resampling
+def test_compact_draft_residual_on_hand_written_rows():
+    from oracle.verify import compact_to_dense
+    k, V = 1, 4
+    z = np.full((1, layout.n_block_rows(k), V), -50.0)
+    z[0, 0] = np.log(np.array([0.5, 0.3, 0.2, 1e-30]))       # Q of the root row; top-k = 3 drops token 3
+    n = 4000
+    zz = np.broadcast_to(z, (n,) + z.shape[1:])
+    tok = np.broadcast_to(np.array([[[0, 2, -1]]]), (n, 1, 3))
+    prob = np.broadcast_to(np.array([[[0.8, 0.2, 0.0]]]), (n, 1, 3))
+    r = verify_step(zz, np.zeros((n, 1), dtype=int), np.full((n, 1), 0.8), k, "sample", seed=5, seq_id=np.arange(n),
+                    resample="residual_draft", top_k=3, top_p=1.0, draft_tok=tok, draft_prob=prob)
+    acc = r["n_accept"] == 1
+    assert abs(acc.mean() - 0.5 / 0.8) < 5 * np.sqrt(0.625 * 0.375 / n)
+    # residual max(0, Q - D) = (0, 0.3, 0, 0): after a rejection the extra token is token 1, always
+    assert (r["out_tokens"][~acc, 0] == 1).all() and (~acc).sum() > 1000
+    assert (r["out_tokens"][acc, 0] == 0).all()
+    # Q(1) = 0.3, D(1) = 0: no subtraction for the winner; the runner-up has no mass
+    assert np.allclose(r["bonus_cond"][~acc], 1.0)
+    # a residual without mass (Q <= D everywhere) falls back to Q; here forced by P_c = +inf
+    prob_q = np.broadcast_to(np.array([[[0.5, 0.2, 0.3]]]), (n, 1, 3))
+    tok_q = np.broadcast_to(np.array([[[0, 2, 1]]]), (n, 1, 3))
+    r = verify_step(zz, np.zeros((n, 1), dtype=int), np.full((n, 1), INF), k, "sample", seed=6, seq_id=np.arange(n),
+                    resample="residual_draft", top_k=3, top_p=1.0, draft_tok=tok_q, draft_prob=prob_q)
+    assert (r["n_accept"] == 0).all()
+    f = np.bincount(r["out_tokens"][:, 0], minlength=V) / n
+    assert np.abs(f - np.array([0.5, 0.3, 0.2, 0.0])).max() < 5 * np.sqrt(0.25 / n)
+    # entries that are no distribution entries do not count
+    d = compact_to_dense(np.array([[1, -1, 7, 2, 2]]), np.array([[0.5, 0.9, 0.9, np.nan, 0.25]]), 4)
+    assert d.tolist() == [[0.0, 0.5, 0.25, 0.0]]
+    # cancellation is reported: Q = (0.5, 0.3, 0.2), D = (0.499, 0, 0) -> the weight of token 0 is 0.001
+    prob_c = np.broadcast_to(np.array([[[0.499, 0.0, 0.0]]]), (n, 1, 3))
+    r = verify_step(zz, np.zeros((n, 1), dtype=int), np.full((n, 1), INF), k, "sample", seed=7, seq_id=np.arange(n),
+                    resample="residual_draft", top_k=3, top_p=1.0, draft_tok=tok, draft_prob=prob_c)
+    top_two_has_0 = (r["out_tokens"][:, 0] == 0) | (r["bonus_cond"] > 1.0)
+    assert np.allclose(r["bonus_cond"][top_two_has_0], 0.5 / 0.001, rtol=1e-6) and top_two_has_0.any()
+
+
+def test_compact_draft_lists_are_the_filtered_mask_rows():
+    from oracle.verify import filter_top_k_top_p
+    k, T, tk, tp = 2, 0.7, 5, 0.9
+    z = _fixed_logits(k, 8)[:1000]
+    n = z.shape[0]
+    r = verify_step(z, np.zeros((n, k), dtype=int), np.full((n, k), INF), k, "sample", temperature=T, seed=9,
+                    seq_id=np.arange(n), resample="residual_draft", top_k=tk, top_p=tp)
+    for o in range(k):
+        pm, _ = filter_top_k_top_p(z[0, layout.mask_group_rows(k, 0)[o]], T, tk, tp)
+        t, p = r["next_draft_tok"][0, o], r["next_draft_prob"][0, o]
+        kept = t >= 0
+        assert abs(p.sum() - 1.0) < 1e-12 and (p[~kept] == 0).all() and (np.diff(p[kept]) <= 0).all()
+        assert np.allclose(pm[t[kept]], p[kept]) and np.count_nonzero(pm) == kept.sum()
+        # P_c is the list's probability of the drawn token
+        c = r["next_cand"][:, o]
+        assert np.allclose(r["next_cand_prob"][:, o], pm[c]) and (pm[c] > 0).all()
+
+
+def test_compact_draft_residual_is_lossless_where_algorithm_1_as_printed_is_not():
+    # Step A draws the candidates from the filtered mask rows of one set of logits; step B verifies them
+    # against other logits.  With the residual rule the first emitted token follows the filtered Q of the
+    # root row exactly, and the token after an accepted candidate the filtered Q of that candidate's row;
+    # with a ~ Q after a rejection (Algorithm 1 as printed) the first token's law is
+    # min(D, Q) + (1 - sum min(D, Q)) Q instead, which the same test tells apart.
+    from oracle.verify import filter_top_k_top_p
+    k, T, tk, tp = 2, 0.9, 5, 0.9
+    zA = _fixed_logits(k, 21)
+    # the verifying model agrees with the drafts in part: its target rows are the mask rows plus noise
+    zb = np.array(_fixed_logits(k, 22)[0])
+    zb[layout.target_rows(k)[0]] = zA[0, layout.mask_group_rows(k, 0)[0]] + 0.6 * zb[layout.target_rows(k)[0]]
+    zB = np.broadcast_to(zb[None], zA.shape)
+    ids = np.arange(N)
+    rA = verify_step(zA, np.zeros((N, k), dtype=int), np.full((N, k), INF), k, "sample", temperature=T, seed=11,
+                     seq_id=ids, resample="residual_draft", top_k=tk, top_p=tp)
+    D1, _ = filter_top_k_top_p(zA[0, layout.mask_group_rows(k, 0)[0]], T, tk, tp)
+    qf, _ = filter_top_k_top_p(zB[0, layout.target_rows(k)], T, tk, tp)
+    assert 0.2 < np.minimum(D1, qf[0]).sum() < 0.9            # a real mix of acceptances and rejections
+    kw = dict(temperature=T, seed=12, seq_id=ids, kv_len=np.full(N, 3), top_k=tk, top_p=tp)
+    r = verify_step(zB, rA["next_cand"], rA["next_cand_prob"], k, "sample", resample="residual_draft",
+                    draft_tok=rA["next_draft_tok"], draft_prob=rA["next_draft_prob"], **kw)
+    acc = (r["n_accept"] >= 1).mean()
+    want = np.minimum(D1, qf[0]).sum()
+    assert abs(acc - want) < 5 * np.sqrt(want * (1 - want) / N)
+    chi, _ = _chi2(np.bincount(r["out_tokens"][:, 0], minlength=V16), qf[0])
+    assert chi < 55.0, chi
+    # second token, by accepted first candidate c: its law is the filtered Q of row 1 (the row depends on c only
+    # through the acceptance, the logits here being fixed)
+    sel = r["n_accept"] >= 1
+    chi, _ = _chi2(np.bincount(r["out_tokens"][sel, 1], minlength=V16), qf[1])
+    assert chi < 55.0, chi
+    # Algorithm 1 as printed on the same candidates
+    rl = verify_step(zB, rA["next_cand"], rA["next_cand_prob"], k, "sample", resample="paper_literal", **kw)
+    mix = np.minimum(D1, qf[0]) + (1 - want) * qf[0]
+    chi_l, _ = _chi2(np.bincount(rl["out_tokens"][:, 0], minlength=V16), mix)
+    assert chi_l < 55.0, chi_l
+    chi_wrong, _ = _chi2(np.bincount(rl["out_tokens"][:, 0], minlength=V16), qf[0])
+    assert chi_wrong > 1000.0, chi_wrong
