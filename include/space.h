@@ -49,7 +49,7 @@ enum {
 
 enum { SPACE_MASK_SAME_GROUP = 0, SPACE_MASK_EQ5_LITERAL = 1 };
 enum { SPACE_MODE_GREEDY = 0, SPACE_MODE_SAMPLE = 1 };
-enum { SPACE_RESAMPLE_RESIDUAL_POINTMASS = 0, SPACE_RESAMPLE_PAPER_LITERAL = 1 };
+enum { SPACE_RESAMPLE_RESIDUAL_POINTMASS = 0, SPACE_RESAMPLE_PAPER_LITERAL = 1, SPACE_RESAMPLE_RESIDUAL_DRAFT = 2 };
 enum { SPACE_DTYPE_BF16 = 0, SPACE_DTYPE_F32 = 1 };
 enum { SPACE_ATTN_TENSOR = 0, SPACE_ATTN_SIMT = 1, SPACE_ATTN_TENSOR_ROWS = 2 };
 
@@ -143,6 +143,18 @@ typedef struct {
                                   order, whose probability reaches top_p, and renormalised (App. A.4 runs
                                   sampling with top-k = 10, top-p = 0.95); ignored in greedy mode        */
   float   top_p;               /* in (0, 1] when top_k > 0 (1 = no nucleus cut)                         */
+  /* SPACE_RESAMPLE_RESIDUAL_DRAFT (sampling mode with top_k > 0 through space_verify / space_verify_commit;
+     ignored otherwise): sampled candidates whose rejection keeps the output distribution unchanged
+     (Sec. 3.2).  Candidate o of the next step is drawn from the filtered distribution D_o of its mask row,
+     P_c = D_o(candidate), and D_o is handed on as a list of top_k (token, probability) pairs in descending
+     order, dropped entries as (-1, 0).  After rejecting candidate i the extra token is drawn from
+     norm(max(0, Q - D_i)) (from Q if that has no mass), after k acceptances from Q.                      */
+  const int32_t* draft_tok;    /* device [B, k, top_k] lists the candidates were drawn from, or NULL together
+                                  with draft_prob (no lists: Algorithm 1's initial state, a ~ Q)          */
+  const float*   draft_prob;   /* device [B, k, top_k]; entries with a token outside [0, vocab) or a
+                                  probability that is not positive and finite do not count              */
+  int32_t* next_draft_tok;     /* device [B, k, top_k]: lists of the next candidates (required)          */
+  float*   next_draft_prob;    /* device [B, k, top_k]                                                   */
 } space_verify_args;
 
 /* Output projection fused with verification: the end of the model call P = M(I) of

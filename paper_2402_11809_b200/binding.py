@@ -19,7 +19,7 @@ NOALLOC_MAX_BATCH = 8
 LMHEAD_MAX_ROWS = 256
 MASK_SAME_GROUP, MASK_EQ5_LITERAL = 0, 1
 MODE_GREEDY, MODE_SAMPLE = 0, 1
-RESAMPLE_RESIDUAL_POINTMASS, RESAMPLE_PAPER_LITERAL = 0, 1
+RESAMPLE_RESIDUAL_POINTMASS, RESAMPLE_PAPER_LITERAL, RESAMPLE_RESIDUAL_DRAFT = 0, 1, 2
 DTYPE_BF16, DTYPE_F32 = 0, 1
 ATTN_TENSOR, ATTN_SIMT, ATTN_TENSOR_ROWS = 0, 1, 2
 ST_CAPACITY, ST_BAD_CANDIDATE, ST_TIMEOUT = 1, 2, 4
@@ -70,7 +70,9 @@ class VerifyArgs(C.Structure):
                 ("kv_len", C.c_void_p), ("n_accept", C.c_void_p), ("out_tokens", C.c_void_p),
                 ("n_out", C.c_void_p), ("next_cand", C.c_void_p), ("next_cand_prob", C.c_void_p),
                 ("finished", C.c_void_p), ("status", C.c_void_p),
-                ("top_k", C.c_int32), ("top_p", C.c_float)]
+                ("top_k", C.c_int32), ("top_p", C.c_float),
+                ("draft_tok", C.c_void_p), ("draft_prob", C.c_void_p),
+                ("next_draft_tok", C.c_void_p), ("next_draft_prob", C.c_void_p)]
 
 
 class CommitArgs(C.Structure):
@@ -270,7 +272,7 @@ class Context:
     def verify_args(self, logits, cand, cand_prob, kv_len, n_accept, out_tokens, n_out, next_cand,
                     next_cand_prob, finished, k, mode=MODE_GREEDY, temperature=1.0, seed=0,
                     resample=RESAMPLE_RESIDUAL_POINTMASS, eos_id=-1, seq_id=None, status=None,
-                    top_k=0, top_p=1.0):
+                    top_k=0, top_p=1.0, draft_tok=None, draft_prob=None, next_draft_tok=None, next_draft_prob=None):
         import torch
         assert logits.stride(2) == 1 and logits.stride(0) == logits.shape[1] * logits.stride(1)
         return VerifyArgs(batch=logits.shape[0], k=k, vocab=logits.shape[2],
@@ -281,7 +283,9 @@ class Context:
                           kv_len=_ptr(kv_len), n_accept=_ptr(n_accept), out_tokens=_ptr(out_tokens),
                           n_out=_ptr(n_out), next_cand=_ptr(next_cand),
                           next_cand_prob=_ptr(next_cand_prob), finished=_ptr(finished),
-                          status=_ptr(status), top_k=top_k, top_p=top_p)
+                          status=_ptr(status), top_k=top_k, top_p=top_p,
+                          draft_tok=_ptr(draft_tok), draft_prob=_ptr(draft_prob),
+                          next_draft_tok=_ptr(next_draft_tok), next_draft_prob=_ptr(next_draft_prob))
 
     def space_verify(self, args):
         _check(lib.space_verify(self._h, C.byref(args), _stream()))

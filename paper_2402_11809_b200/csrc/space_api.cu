@@ -117,8 +117,14 @@ int check_verify_args(const space_ctx* ctx, const space_verify_args* a) {
     return SPACE_E_INVALID_ARG;
   if (a->logits_dtype != SPACE_DTYPE_F32 && a->logits_dtype != SPACE_DTYPE_BF16) return SPACE_E_INVALID_ARG;
   if (a->mode != SPACE_MODE_GREEDY && a->mode != SPACE_MODE_SAMPLE) return SPACE_E_INVALID_ARG;
-  if (a->resample != SPACE_RESAMPLE_RESIDUAL_POINTMASS && a->resample != SPACE_RESAMPLE_PAPER_LITERAL)
+  if (a->resample != SPACE_RESAMPLE_RESIDUAL_POINTMASS && a->resample != SPACE_RESAMPLE_PAPER_LITERAL &&
+      a->resample != SPACE_RESAMPLE_RESIDUAL_DRAFT)
     return SPACE_E_INVALID_ARG;
+  if (a->mode == SPACE_MODE_SAMPLE && a->resample == SPACE_RESAMPLE_RESIDUAL_DRAFT) {
+    // compact draft lists are the filtered mask rows: they need a top-k, a place to go, and come in pairs
+    if (a->top_k < 1 || !a->next_draft_tok || !a->next_draft_prob) return SPACE_E_INVALID_ARG;
+    if ((a->draft_tok == nullptr) != (a->draft_prob == nullptr)) return SPACE_E_INVALID_ARG;
+  }
   if (a->mode == SPACE_MODE_SAMPLE && !(a->temperature > 0.f)) return SPACE_E_INVALID_ARG;
   if (a->mode == SPACE_MODE_SAMPLE && a->top_k != 0 &&
       (a->top_k < 0 || a->top_k > 32 || !(a->top_p > 0.f) || a->top_p > 1.f))

@@ -10,6 +10,11 @@
 // writes the next candidates (their arg-maxes with P_c = 1, or samples from the filtered rows with
 // their probabilities when candidates are sampled).
 //
+// SPACE_RESAMPLE_RESIDUAL_DRAFT keeps sampled candidates lossless (Sec. 3.2 claims an unchanged output
+// distribution): phase 1 also writes every candidate's filtered distribution D as a list of top_k
+// (token, probability) pairs, and phase 0 of the next step, after rejecting candidate i, draws the extra
+// token from norm(max(0, Q - D_i)) -- one warp, its 32 lanes holding Q's kept tokens and D_i's entries.
+//
 // Top-k selection: every warp keeps a sorted list of at most 32 (logit, token) keys, one per lane, and
 // a threshold (its last key); a logit above the threshold is inserted with one ballot and one shuffle.
 // Keys are 64-bit words whose unsigned order is "larger logit, then lower token", so exact ties go to
@@ -33,6 +38,9 @@ struct FiltParams {
   const int32_t* cand; const float* cand_prob; const uint32_t* seq_id; const int32_t* kv_len;
   int32_t* n_accept; int32_t* out_tokens; int32_t* n_out; int32_t* next_cand; float* next_cand_prob;
   uint8_t* finished; int32_t* status;
+  const int32_t* draft_tok; const float* draft_prob;      // [B, k, list_stride] or NULL (no lists)
+  int32_t* next_draft_tok; float* next_draft_prob;        // [B, k, list_stride]
+  int list_stride;
   unsigned long long* part;            // [B][k+1][FILT_MAX_CHUNKS][32]
   int* counter;                        // [B], self-resetting
 };
@@ -127,7 +135,8 @@ __global__ void __launch_bounds__(FILT_THREADS) verify_filter_kernel(const FiltP
   __shared__ int sh_ok[SPACE_MAX_K + 1];
   __shared__ int sh_bits;
   if (threadIdx.x == 0) sh_bits = 0;
-  const bool literal = p.resample == SPACE_RESAMPLE_PAPER_LITERAL;
+  const bool with_lists = p.resample == SPACE_RESAMPLE_RESIDUAL_DRAFT;
+  const bool literal = p.resample == SPACE_RESAMPLE_PAPER_LITERAL || with_lists;   // candidates are sampled
   const uint32_t seq = p.seq_id ? p.seq_id[b] : (uint32_t)b;
   const int L = p.kv_len ? p.kv_len[b] : 0;
   float z = 0.f, q = 0.f; int idx = -1; bool keep = false;
@@ -190,10 +199,32 @@ __global__ void __launch_bounds__(FILT_THREADS) verify_filter_kernel(const FiltP
       int exclude = -1;
       if (!literal && i_star < p.k && p.cand_prob[b * p.k + i_star] == 1.0f) exclude = p.cand[b * p.k + i_star];
       float sc = -CUDART_INF_F;
-      if (keep && idx != exclude) {
+      // compact draft distribution of the rejected candidate: the weight of a kept token is
+      // max(0, Q - D); Q itself when nothing was rejected, there are no lists, or nothing is left
+      float wq = q;
+      bool residual = false;
+      if (with_lists && i_star < p.k && p.draft_tok) {
+        int dt = -1; float dp = 0.f;
+        if (lane < p.list_stride) {
+          dt = p.draft_tok[((int64_t)b * p.k + i_star) * p.list_stride + lane];
+          dp = p.draft_prob[((int64_t)b * p.k + i_star) * p.list_stride + lane];
+          if (dt < 0 || dt >= p.V || !(dp > 0.f) || !(dp < CUDART_INF_F)) { dt = -1; dp = 0.f; }
+        }
+        float d = 0.f;
+        for (int j = 0; j < p.list_stride; ++j) {
+          const int tj = __shfl_sync(0xFFFFFFFFu, dt, j);
+          const float pj2 = __shfl_sync(0xFFFFFFFFu, dp, j);
+          if (tj == idx) d += pj2;
+        }
+        const float res = keep ? fmaxf(q - d, 0.f) : 0.f;
+        residual = __any_sync(0xFFFFFFFFu, res > 0.f);
+        if (residual) wq = res;
+      }
+      if (keep && idx != exclude && (!residual || wq > 0.f)) {
         const Philox4 ph = philox4x32_10((uint32_t)(idx >> 2), PURPOSE_TOKEN, seq, (uint32_t)(L + i_star + 1), p.key0, p.key1);
         const uint32_t w4[4] = {ph.x, ph.y, ph.z, ph.w};
-        sc = fmaf(z, p.c_t, gumbel2_from_uniform(uniform_open(w4[idx & 3])));
+        const float g = gumbel2_from_uniform(uniform_open(w4[idx & 3]));
+        sc = with_lists ? fast_log2(wq) + g : fmaf(z, p.c_t, g);
       }
       int bi = keep ? idx : 0x7FFFFFFF;
 #pragma unroll
@@ -240,6 +271,10 @@ __global__ void __launch_bounds__(FILT_THREADS) verify_filter_kernel(const FiltP
       tok = bi; pr = bq;
     }
     if (lane == 0) { p.next_cand[b * p.k + warp] = tok; p.next_cand_prob[b * p.k + warp] = pr; }
+    if (with_lists && lane < p.list_stride) {               // the row's filtered distribution, descending
+      p.next_draft_tok[((int64_t)b * p.k + warp) * p.list_stride + lane] = keep ? idx : -1;
+      p.next_draft_prob[((int64_t)b * p.k + warp) * p.list_stride + lane] = keep ? q : 0.f;
+    }
   }
 }
 
@@ -262,6 +297,8 @@ int launch_verify_filtered(space_ctx* ctx, const space_verify_args* a, cudaStrea
   p.cand = a->cand; p.cand_prob = a->cand_prob; p.seq_id = a->seq_id; p.kv_len = a->kv_len;
   p.n_accept = a->n_accept; p.out_tokens = a->out_tokens; p.n_out = a->n_out; p.next_cand = a->next_cand;
   p.next_cand_prob = a->next_cand_prob; p.finished = a->finished; p.status = a->status;
+  p.draft_tok = a->draft_tok; p.draft_prob = a->draft_prob;
+  p.next_draft_tok = a->next_draft_tok; p.next_draft_prob = a->next_draft_prob; p.list_stride = a->top_k;
   p.part = reinterpret_cast<unsigned long long*>(ctx->vtopk);
   // about two blocks per SM over the (k+1) rows of every sequence, at least 8192 logits per block
   const int rows = a->batch * (a->k + 1);

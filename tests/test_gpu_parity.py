@@ -535,6 +535,89 @@ def test_verify_filtered_sampling(B, H, resample, k, V, Bn, T, top_k, top_p, dty
     assert np.array_equal(H.bf16_to_bits(ds2.k_cache), Kc) and np.array_equal(ds2.kv_len_out.cpu().numpy(), new_len)
 
 
+@pytest.mark.parametrize("k,V,Bn,T,top_k,top_p,dtype", [
+    (2, 5000, 24, 0.9, 10, 0.95, "bf16"),     # App. A.4's setting
+    (4, 32000, 8, 1.0, 10, 0.95, "f32"),
+    (3, 300, 16, 0.7, 32, 1.0, "f32"),        # the longest lists, no nucleus cut
+    (1, 40, 6, 1.2, 5, 0.6, "bf16"),
+])
+def test_verify_compact_draft_residual(B, H, k, V, Bn, T, top_k, top_p, dtype):
+    """SPACE_RESAMPLE_RESIDUAL_DRAFT over two steps: the first step starts from Algorithm 1's initial
+    state and hands on candidates with their compact distributions; the second verifies them against
+    logits whose target rows agree with the drafts in part, so that acceptances, rejections with a
+    non-trivial residual max(0, Q - D) and full acceptances all occur."""
+    from oracle.layout import mask_group_rows, target_rows
+    cfg = workloads.resolve("sampling64", B=Bn, H_q=1, H_kv=1, d=64, L=(5, 600), k=k, V=V, temperature=T,
+                            logits_dtype=dtype, seed=900 + k)
+    x = workloads.make_step_inputs(cfg)
+    x["cand"][:] = 0
+    x["cand_prob"][:] = np.inf
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    Kl = top_k
+    nd_tok = torch.full((Bn, k, Kl), -7, dtype=torch.int32, device="cuda")
+    nd_prob = torch.full((Bn, k, Kl), float("nan"), dtype=torch.float32, device="cuda")
+
+    def run(ds_, seed, draft=None):
+        a = ctx.verify_args(ds_.logits, ds_.cand, ds_.cand_prob, ds_.kv_len, ds_.n_accept, ds_.out_tokens, ds_.n_out,
+                            ds_.next_cand, ds_.next_cand_prob, ds_.finished, k, mode=B.MODE_SAMPLE, temperature=T,
+                            seed=seed, resample=B.RESAMPLE_RESIDUAL_DRAFT, seq_id=ds_.seq_id, status=ds_.status,
+                            top_k=top_k, top_p=top_p, next_draft_tok=nd_tok, next_draft_prob=nd_prob,
+                            draft_tok=None if draft is None else draft[0], draft_prob=None if draft is None else draft[1])
+        ctx.space_verify(a)
+        torch.cuda.synchronize()
+
+    def check(ds_, r):
+        nuc = r["nucleus_margin"] <= NUCLEUS_BAND
+        r["accept_margin"] = np.where(nuc[:, None], 0.0, r["accept_margin"])
+        r["bonus_gap"] = r["bonus_gap"] / r["bonus_cond"]                    # cancellation in Q - D widens the band
+        excl = _check_verify(ds_, r, k, sample=True)
+        keep = ~excl
+        assert np.array_equal(nd_tok.cpu().numpy()[keep], r["next_draft_tok"][keep])
+        np.testing.assert_allclose(nd_prob.cpu().numpy()[keep], r["next_draft_prob"][keep], rtol=1e-4, atol=1e-30)
+        return keep
+
+    # ---- step A: initial state, no lists ----
+    run(ds, 11)
+    rA = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "sample", temperature=T, seed=11, seq_id=x["seq_id"],
+                     kv_len=x["kv_len"], resample="residual_draft", top_k=top_k, top_p=top_p)
+    check(ds, rA)
+    assert (rA["n_accept"] == 0).all()
+    # ---- step B: the oracle's candidates and lists, target rows that partly agree with the drafts ----
+    x2 = dict(x)
+    lg = x["logits"].copy()
+    rng = np.random.default_rng(5)
+    for i in range(k):
+        take = rng.random((Bn, V)) < 0.8
+        lg[:, target_rows(k)[i], :] = np.where(take, x["logits"][:, mask_group_rows(k, 0)[i], :], lg[:, target_rows(k)[i], :])
+    x2["logits"] = lg
+    x2["cand"] = rA["next_cand"].astype(np.int32)
+    x2["cand_prob"] = rA["next_cand_prob"].astype(np.float32)
+    dtok = rA["next_draft_tok"].astype(np.int32)
+    dprob = rA["next_draft_prob"].astype(np.float32)
+    ds2 = H.DeviceStep(cfg, x2)
+    seen = np.zeros(3, dtype=int)
+    for seed in (12, 13, 14):
+        run(ds2, seed, draft=(H.to_dev(dtok), H.to_dev(dprob)))
+        rB = verify_step(lg, x2["cand"], x2["cand_prob"].astype(np.float64), k, "sample", temperature=T, seed=seed,
+                         seq_id=x["seq_id"], kv_len=x["kv_len"], resample="residual_draft", top_k=top_k, top_p=top_p,
+                         draft_tok=dtok, draft_prob=dprob.astype(np.float64))
+        check(ds2, rB)
+        seen += np.array([(rB["n_accept"] == 0).sum(), ((rB["n_accept"] > 0) & (rB["n_accept"] < k)).sum() if k > 1 else 0,
+                          (rB["n_accept"] == k).sum()])
+    assert seen[0] > 0 and (seen[1] + seen[2] > 0 or Bn < 8), seen   # rejections at once and after acceptances
+    # the reading needs a top-k, both list inputs or none, and a place for the new lists
+    import ctypes as C
+    mk = lambda **kw: ctx.verify_args(ds.logits, ds.cand, ds.cand_prob, ds.kv_len, ds.n_accept, ds.out_tokens, ds.n_out,
+                                      ds.next_cand, ds.next_cand_prob, ds.finished, k, mode=B.MODE_SAMPLE, temperature=T,
+                                      resample=B.RESAMPLE_RESIDUAL_DRAFT, **kw)
+    assert B.lib.space_verify(ctx._h, C.byref(mk(top_k=0, next_draft_tok=nd_tok, next_draft_prob=nd_prob)), None) == B.E_INVALID_ARG
+    assert B.lib.space_verify(ctx._h, C.byref(mk(top_k=top_k, top_p=top_p)), None) == B.E_INVALID_ARG
+    assert B.lib.space_verify(ctx._h, C.byref(mk(top_k=top_k, top_p=top_p, next_draft_tok=nd_tok, next_draft_prob=nd_prob,
+                                                 draft_tok=H.to_dev(dtok))), None) == B.E_INVALID_ARG
+    torch.cuda.synchronize()
+
+
 def test_verify_filter_arguments(B, H):
     import ctypes as C
     cfg = workloads.resolve("sampling64", B=2, H_q=1, H_kv=1, d=64, L=(5, 50), k=2, V=100, seed=1)
