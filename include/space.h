@@ -35,6 +35,7 @@ extern "C" {
 
 #define SPACE_MAX_K     7      /* (k+1)^2 <= 64 block rows                    */
 #define SPACE_MAX_ROWS  64
+#define SPACE_PAGE_SIZE 128    /* key rows per page of a paged cache (the kernels' key tile) */
 
 enum {
   SPACE_OK            =  0,
@@ -57,7 +58,10 @@ enum { SPACE_ATTN_TENSOR = 0, SPACE_ATTN_SIMT = 1, SPACE_ATTN_TENSOR_ROWS = 2 };
 enum {
   SPACE_ST_CAPACITY      = 1,  /* kv_len + (k+1)^2 exceeds the cache capacity */
   SPACE_ST_BAD_CANDIDATE = 2,  /* a candidate id outside [0, vocab): rejected */
-  SPACE_ST_TIMEOUT       = 4   /* a bounded on-chip wait expired              */
+  SPACE_ST_TIMEOUT       = 4,  /* a bounded on-chip wait expired              */
+  SPACE_ST_BAD_PAGE      = 8   /* a page-table entry outside [0, n_pages): that page is not
+                                  touched (attention reads zeros in its place, the commit skips
+                                  the row)                                     */
 };
 
 typedef struct space_ctx space_ctx;   /* opaque; owns only its own workspace */
@@ -106,6 +110,18 @@ typedef struct {
   void*          out;       /* device [B, n_q, H_q, d] of out_dtype            */
   float*         lse;       /* device [B, H_q, n_q] natural-log sum-exp, or NULL */
   int32_t*       status;    /* device [B], OR-ed with SPACE_ST_*, or NULL      */
+  /* Paged cache (the serving setting of Sec. 4.3: continuous batching over a pool of pages).
+     page_table == NULL: the contiguous cache described above.  Otherwise k_cache / v_cache are
+     pools of pages of SPACE_PAGE_SIZE key rows, element (page, h, r, :) at
+     page*kv_stride_b + h*kv_stride_h + r*kv_stride_s, and key position s of sequence b (cache
+     rows and the block's own rows L_b .. L_b+n_q-1 alike) is row s % SPACE_PAGE_SIZE of page
+     page_table[b*pages_per_seq + s / SPACE_PAGE_SIZE].  A sequence's capacity is
+     pages_per_seq * SPACE_PAGE_SIZE rows (it replaces s_cap in the SPACE_ST_CAPACITY check, and
+     must not exceed the context's s_cap).  Entries past the pages a sequence needs are
+     ignored.  Rows of its last page beyond L_b+n_q may hold anything, NaN included.            */
+  const int32_t* page_table;   /* device [B, pages_per_seq] or NULL                            */
+  int32_t pages_per_seq;
+  int32_t n_pages;             /* pages in the pool                                            */
 } space_attn_args;
 
 /* Verification and emission (Algorithm 1 after the model call; Sec. 3.2). */
@@ -210,6 +226,9 @@ typedef struct {
   int32_t* commit_src;         /* device [B, k+1] or NULL, -1 padded           */
   int32_t* commit_dst;         /* device [B, k+1] or NULL                      */
   int32_t* status;             /* device [B] or NULL                           */
+  const int32_t* page_table;   /* paged cache as in space_attn_args, or NULL (contiguous)      */
+  int32_t pages_per_seq;
+  int32_t n_pages;
 } space_commit_args;
 
 /* Whole step from host memory (copies in, the three stages, copies out). */

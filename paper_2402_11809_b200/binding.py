@@ -22,7 +22,8 @@ MODE_GREEDY, MODE_SAMPLE = 0, 1
 RESAMPLE_RESIDUAL_POINTMASS, RESAMPLE_PAPER_LITERAL, RESAMPLE_RESIDUAL_DRAFT = 0, 1, 2
 DTYPE_BF16, DTYPE_F32 = 0, 1
 ATTN_TENSOR, ATTN_SIMT, ATTN_TENSOR_ROWS = 0, 1, 2
-ST_CAPACITY, ST_BAD_CANDIDATE, ST_TIMEOUT = 1, 2, 4
+ST_CAPACITY, ST_BAD_CANDIDATE, ST_TIMEOUT, ST_BAD_PAGE = 1, 2, 4, 8
+PAGE_SIZE = 128
 
 EXPORTS = ["space_create", "space_destroy", "space_workspace_bytes", "space_layout",
            "space_attn_step", "space_verify", "space_verify_commit", "space_verify_greedy_noalloc",
@@ -58,7 +59,8 @@ class AttnArgs(C.Structure):
                 ("q", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
                 ("kv_stride_b", C.c_int64), ("kv_stride_h", C.c_int64), ("kv_stride_s", C.c_int64),
                 ("kv_len", C.c_void_p), ("out", C.c_void_p), ("lse", C.c_void_p),
-                ("status", C.c_void_p)]
+                ("status", C.c_void_p), ("page_table", C.c_void_p), ("pages_per_seq", C.c_int32),
+                ("n_pages", C.c_int32)]
 
 
 class VerifyArgs(C.Structure):
@@ -80,7 +82,8 @@ class CommitArgs(C.Structure):
                 ("v_cache", C.c_void_p), ("kv_stride_b", C.c_int64), ("kv_stride_h", C.c_int64),
                 ("kv_stride_s", C.c_int64), ("n_accept", C.c_void_p), ("kv_len", C.c_void_p),
                 ("kv_len_out", C.c_void_p), ("commit_src", C.c_void_p), ("commit_dst", C.c_void_p),
-                ("status", C.c_void_p)]
+                ("status", C.c_void_p), ("page_table", C.c_void_p), ("pages_per_seq", C.c_int32),
+                ("n_pages", C.c_int32)]
 
 
 class LmHeadArgs(C.Structure):
@@ -254,7 +257,8 @@ class Context:
 
     # -- space_attn_step --------------------------------------------------
     def attn_args(self, q, k_cache, v_cache, kv_len, out, k, scale, lse=None, status=None,
-                  mask_variant=MASK_SAME_GROUP, impl=ATTN_TENSOR):
+                  mask_variant=MASK_SAME_GROUP, impl=ATTN_TENSOR, page_table=None):
+        """page_table [B, pages_per_seq] int32: k_cache / v_cache are then pools [n_pages, H_kv, PAGE_SIZE, d]."""
         import torch
         assert q.is_contiguous() and out.is_contiguous()
         assert k_cache.stride() == v_cache.stride() and k_cache.stride(3) == 1
@@ -263,7 +267,9 @@ class Context:
                         impl=impl, scale=scale, q=_ptr(q), k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
                         kv_stride_b=k_cache.stride(0), kv_stride_h=k_cache.stride(1),
                         kv_stride_s=k_cache.stride(2), kv_len=_ptr(kv_len), out=_ptr(out),
-                        lse=_ptr(lse), status=_ptr(status))
+                        lse=_ptr(lse), status=_ptr(status), page_table=_ptr(page_table),
+                        pages_per_seq=0 if page_table is None else page_table.shape[1],
+                        n_pages=0 if page_table is None else k_cache.shape[0])
 
     def space_attn_step(self, args):
         _check(lib.space_attn_step(self._h, C.byref(args), _stream()))
@@ -317,12 +323,14 @@ class Context:
 
     # -- space_kv_commit --------------------------------------------------
     def commit_args(self, k_cache, v_cache, n_accept, kv_len, k, kv_len_out=None, commit_src=None,
-                    commit_dst=None, status=None):
-        return CommitArgs(batch=k_cache.shape[0], k=k, k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
+                    commit_dst=None, status=None, page_table=None):
+        return CommitArgs(batch=n_accept.shape[0], k=k, k_cache=_ptr(k_cache), v_cache=_ptr(v_cache),
                           kv_stride_b=k_cache.stride(0), kv_stride_h=k_cache.stride(1),
                           kv_stride_s=k_cache.stride(2), n_accept=_ptr(n_accept), kv_len=_ptr(kv_len),
                           kv_len_out=_ptr(kv_len_out), commit_src=_ptr(commit_src),
-                          commit_dst=_ptr(commit_dst), status=_ptr(status))
+                          commit_dst=_ptr(commit_dst), status=_ptr(status), page_table=_ptr(page_table),
+                          pages_per_seq=0 if page_table is None else page_table.shape[1],
+                          n_pages=0 if page_table is None else k_cache.shape[0])
 
     def space_kv_commit(self, args):
         _check(lib.space_kv_commit(self._h, C.byref(args), _stream()))

@@ -34,7 +34,11 @@ struct AttnParams {
   int n_mblocks, rows_per_mb;          // query-row blocks per kv head; block rows i per block
   int n_groups;                        // thread-block groups (grid = n_groups * n_mblocks)
   int out_dtype;
-  int64_t s_cap;
+  int64_t s_cap;                       // rows a sequence may hold (paged: pages_per_seq * SPACE_PAGE_SIZE)
+  // Paged cache (page_table != nullptr): tm_k / tm_v describe a pool [n_pages][H_kv][TILE_N][d] and tile t
+  // of sequence b is the whole page page_table[b * pages_per_seq + t]; no tile is shifted back, the
+  // rows of the last page past the last key are masked (S) and cleared in shared memory (V).
+  const int32_t* page_table; int pages_per_seq, n_pages;
   float scale_log2;                    // scale * log2(e)
   const int32_t* kv_len;
   void* out; float* lse; int32_t* status;
@@ -47,6 +51,15 @@ struct AttnParams {
 };
 
 struct Seg { int b, h, t0, t1, T, L; };
+
+// Page of tile t of sequence b (paged cache).  An entry outside the pool is flagged and answered
+// with a page past the pool's end: the TMA load then fills the tile with zeros.
+__device__ __forceinline__ int page_of(const AttnParams& p, int b, int t) {
+  const int pg = t < p.pages_per_seq ? p.page_table[(int64_t)b * p.pages_per_seq + t] : -1;
+  if (pg >= 0 && pg < p.n_pages) return pg;
+  if (p.status) atomicOr(p.status + b, SPACE_ST_BAD_PAGE);
+  return p.n_pages;
+}
 
 // PTX helpers: tc_common.cuh.  Every wait of this kernel is bounded by WAIT_NS.
 using namespace tc;
@@ -295,12 +308,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
           if (!ok) break;
           // the last tile of a sequence is shifted back so that it ends at the
           // last key: rows past the end are never read (they may hold anything)
-          const int kt = ((t + 1) * TILE_N <= n_keys) ? t * TILE_N : n_keys - TILE_N;
+          // (a paged cache has whole pages for tiles instead; see AttnParams)
+          const int kt = p.page_table ? 0 : (((t + 1) * TILE_N <= n_keys) ? t * TILE_N : n_keys - TILE_N);
+          const int kb = p.page_table ? page_of(p, sg.b, t) : sg.b;
           const uint32_t dst = ring + s * S::TILE_BYTES;
           mbar_expect_tx(BAR(b_full + s), S::TILE_BYTES);
 #pragma unroll
           for (int hf = 0; hf < S::HALVES; ++hf)
-            tma_load_4d(dst + hf * (TILE_N * 128), tm, BAR(b_full + s), hf * 64, kt, sg.h, sg.b);
+            tma_load_4d(dst + hf * (TILE_N * 128), tm, BAR(b_full + s), hf * 64, kt, sg.h, kb);
         }
       }
       // drain: every issued copy must have landed before the block may exit
@@ -413,8 +428,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
         for (int cc = 0; cc < HC / 32; ++cc) tmem_ld32(ts + half * HC + cc * 32, sreg + cc * 32);
         tmem_wait_ld();
         const int lo = t * TILE_N;
-        const int kt = ((t + 1) * TILE_N <= n_keys) ? lo : n_keys - TILE_N;
-        const bool masked = (kt + TILE_N > sg.L) || (kt < lo);
+        const int kt = (p.page_table || (t + 1) * TILE_N <= n_keys) ? lo : n_keys - TILE_N;
+        const bool masked = (kt + TILE_N > sg.L) || (kt < lo);   // (rows of a page past the last key: no mask bit names them)
         float tmax = -CUDART_INF_F;
         if (masked) {
           // Visibility of this thread's 64 keys as one 64-bit word (bit c: key k0 + c):
@@ -495,6 +510,22 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
         tmem_st32(ts + half * (HC / 2), sreg);
         tmem_st32(ts + TILE_N / 2 + half * (HC / 2), lreg);
         tmem_wait_st();
+        if (p.page_table && kt + TILE_N > n_keys) {
+          // Paged cache, last tile: the page's rows past the last key may hold anything, and 0 * NaN
+          // would reach the output.  Once the V tile has landed the softmax threads clear those rows
+          // (128 contiguous bytes per row and 64-wide half of d, whatever the swizzle inside them).
+          const uint32_t vs = gt % S::V_STAGES;
+          ok &= mbar_wait(BAR(B_VFULL + vs), (gt / S::V_STAGES) & 1, abort_flag, p.err, 17);
+          const int first_bad = n_keys - kt;
+          for (int it = first_bad * S::HALVES + sidx; it < TILE_N * S::HALVES; it += n_soft) {
+            const int r = it / S::HALVES, hf = it % S::HALVES;
+            const uint32_t vrow = sm_base + S::V_OFF + vs * S::TILE_BYTES + hf * (TILE_N * 128) + r * 128;
+#pragma unroll
+            for (int x = 0; x < 8; ++x)
+              asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vrow + x * 16), "r"(0u) : "memory");
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
         tc_fence_before();
         mbar_arrive(BAR(B_PREADY + buf));
       }
@@ -712,7 +743,9 @@ int launch_attn_rows(space_ctx* ctx, const space_attn_args* a, const uint64_t* m
   p.H_q = cfg.n_q_heads; p.H_kv = cfg.n_kv_heads; p.G = p.H_q / p.H_kv;
   p.n_mblocks = pl.n_mblocks; p.rows_per_mb = pl.rows_per_mblock;
   p.n_groups = pl.n_ctas / pl.n_mblocks;
-  p.out_dtype = a->out_dtype; p.s_cap = cfg.s_cap;
+  p.out_dtype = a->out_dtype;
+  p.s_cap = a->page_table ? (int64_t)a->pages_per_seq * SPACE_PAGE_SIZE : cfg.s_cap;
+  p.page_table = a->page_table; p.pages_per_seq = a->pages_per_seq; p.n_pages = a->n_pages;
   p.scale_log2 = a->scale * 1.4426950408889634f;
   p.kv_len = a->kv_len; p.out = a->out; p.lse = a->lse; p.status = a->status;
   p.part = ctx->attn_part; p.err = ctx->counters + 3 * cfg.max_batch;
@@ -722,10 +755,12 @@ int launch_attn_rows(space_ctx* ctx, const space_attn_args* a, const uint64_t* m
   for (int i = 0; i < SPACE_MAX_ROWS; ++i) p.mask[i] = mask_rows[i];
 
   // TMA descriptors, rebuilt only when a base pointer or a stride changes
-  const int64_t key[8] = {a->kv_stride_b, a->kv_stride_h, a->kv_stride_s, a->batch, p.n_q, -1, 0, 0};
+  const int64_t key[8] = {a->kv_stride_b, a->kv_stride_h, a->kv_stride_s, a->batch, p.n_q, -1,
+                          a->page_table ? a->n_pages : 0, 0};
   if (ctx->tm_q_ptr != a->q || ctx->tm_k_ptr != a->k_cache || ctx->tm_v_ptr != a->v_cache ||
       memcmp(key, ctx->tm_key, sizeof(key)) != 0) {
-    const cuuint64_t kd[4] = {(cuuint64_t)DH, (cuuint64_t)cfg.s_cap, (cuuint64_t)p.H_kv, (cuuint64_t)a->batch};
+    const cuuint64_t kd[4] = {(cuuint64_t)DH, (cuuint64_t)(a->page_table ? TILE_N : cfg.s_cap), (cuuint64_t)p.H_kv,
+                              (cuuint64_t)(a->page_table ? a->n_pages : a->batch)};
     const cuuint64_t ks[3] = {(cuuint64_t)a->kv_stride_s * 2, (cuuint64_t)a->kv_stride_h * 2,
                               (cuuint64_t)a->kv_stride_b * 2};
     const cuuint32_t kb[4] = {64, TILE_N, 1, 1};

@@ -17,6 +17,7 @@ struct SimtParams {
   const int32_t* kv_len;
   void* out; float* lse; int32_t* status;
   uint64_t mask[SPACE_MAX_ROWS];
+  const int32_t* page_table; int pages_per_seq, n_pages;   // paged cache, or page_table == nullptr
 };
 
 constexpr int SIMT_THREADS = 128;
@@ -56,8 +57,16 @@ __global__ void __launch_bounds__(SIMT_THREADS) attn_simt_kernel(const SimtParam
   const __nv_bfloat16* qrow = p.q + (((int64_t)b * p.n_q + i) * p.H_q + h) * p.d;
   for (int c = threadIdx.x; c < p.d; c += SIMT_THREADS) qs[c] = __bfloat162float(qrow[c]);
   __syncthreads();
-  const __nv_bfloat16* kb = p.kc + (int64_t)b * p.sb + (int64_t)hk * p.sh;
-  const __nv_bfloat16* vb = p.vc + (int64_t)b * p.sb + (int64_t)hk * p.sh;
+  // offset of key row j (contiguous cache, or through the page table); a page outside the pool
+  // reads as zeros and is flagged
+  __shared__ int bad_page;
+  if (threadIdx.x == 0) bad_page = 0;
+  __syncthreads();
+  auto row_off = [&](int j) {
+    const int64_t o = kv_row_offset(p.page_table, p.pages_per_seq, p.n_pages, p.sb, p.sh, p.ss, b, hk, j);
+    if (o < 0) bad_page = 1;
+    return o;
+  };
   const int n_keys = L + p.n_q;
   const uint64_t mrow = p.mask[i];
   float mx = -CUDART_INF_F;
@@ -65,9 +74,10 @@ __global__ void __launch_bounds__(SIMT_THREADS) attn_simt_kernel(const SimtParam
     const bool vis = (j < L) || ((mrow >> (j - L)) & 1ull);
     float s = -CUDART_INF_F;
     if (vis) {
-      const __nv_bfloat162* kr = reinterpret_cast<const __nv_bfloat162*>(kb + (int64_t)j * p.ss);
+      const int64_t ko = row_off(j);
+      const __nv_bfloat162* kr = reinterpret_cast<const __nv_bfloat162*>(p.kc + (ko < 0 ? 0 : ko));
       float acc = 0.f;
-      for (int c = 0; c < p.d / 2; ++c) {
+      for (int c = 0; c < (ko < 0 ? 0 : p.d / 2); ++c) {
         const float2 kk = __bfloat1622float2(kr[c]);
         acc = fmaf(qs[2 * c], kk.x, acc);
         acc = fmaf(qs[2 * c + 1], kk.y, acc);
@@ -90,13 +100,18 @@ __global__ void __launch_bounds__(SIMT_THREADS) attn_simt_kernel(const SimtParam
     float acc = 0.f;
     for (int j = 0; j < n_keys; ++j) {
       const float e = sc[j];
-      if (e != 0.f) acc = fmaf(e, __bfloat162float(vb[(int64_t)j * p.ss + c]), acc);
+      if (e != 0.f) {
+        const int64_t vo = row_off(j);
+        if (vo >= 0) acc = fmaf(e, __bfloat162float(p.vc[vo + c]), acc);
+      }
     }
     const int64_t o = (((int64_t)b * p.n_q + i) * p.H_q + h) * p.d + c;
     if (p.out_dtype == SPACE_DTYPE_F32) reinterpret_cast<float*>(p.out)[o] = acc * inv;
     else reinterpret_cast<__nv_bfloat16*>(p.out)[o] = __float2bfloat16_rn(acc * inv);
   }
   if (p.lse && threadIdx.x == 0) p.lse[((int64_t)b * p.H_q + h) * p.n_q + i] = mx + logf(sum);
+  __syncthreads();
+  if (threadIdx.x == 0 && bad_page && p.status) atomicOr(p.status + b, SPACE_ST_BAD_PAGE);
 }
 
 }  // namespace
@@ -106,7 +121,9 @@ int launch_attn_simt(space_ctx* ctx, const space_attn_args* a, const uint64_t* m
   SimtParams p;
   p.B = a->batch; p.k = a->k; p.n_q = (a->k + 1) * (a->k + 1);
   p.H_q = ctx->cfg.n_q_heads; p.H_kv = ctx->cfg.n_kv_heads; p.d = ctx->cfg.head_dim;
-  p.out_dtype = a->out_dtype; p.s_cap = ctx->cfg.s_cap; p.scale = a->scale;
+  p.out_dtype = a->out_dtype; p.scale = a->scale;
+  p.s_cap = a->page_table ? (int64_t)a->pages_per_seq * SPACE_PAGE_SIZE : ctx->cfg.s_cap;
+  p.page_table = a->page_table; p.pages_per_seq = a->pages_per_seq; p.n_pages = a->n_pages;
   p.q = (const __nv_bfloat16*)a->q; p.kc = (const __nv_bfloat16*)a->k_cache;
   p.vc = (const __nv_bfloat16*)a->v_cache;
   p.sb = a->kv_stride_b; p.sh = a->kv_stride_h; p.ss = a->kv_stride_s;

@@ -56,7 +56,12 @@ struct AttnParams {
   int n_groups;                        // thread-block groups (grid = n_groups * n_mblocks)
   int out_dtype;
   int spec;                            // one sequence: every group requests its first K tile before the length is read
-  int64_t s_cap;
+  int64_t s_cap;                       // rows a sequence may hold (paged: pages_per_seq * SPACE_PAGE_SIZE)
+  // Paged cache (page_table != nullptr): tm_k / tm_v describe a pool [n_pages][H_kv][TILE_N][d]; tile t
+  // of sequence b is the whole page page_table[b * pages_per_seq + t].  No tile is shifted back then:
+  // the last one may end in rows that belong to no key, whose scores are masked and whose V rows are
+  // cleared in shared memory before the O^T product reads them.
+  const int32_t* page_table; int pages_per_seq, n_pages;
   float scale_log2;                    // scale * log2(e)
   const int32_t* kv_len;
   void* out; float* lse; int32_t* status;
@@ -70,6 +75,16 @@ struct AttnParams {
   // any of its G heads) sees block key j
   uint64_t visq[2][SPACE_MAX_ROWS];
 };
+
+// Page of tile t of sequence b (paged cache).  An entry outside the pool is flagged and answered
+// with a page past the pool's end: the TMA load then fills the tile with zeros.
+// (flag = false: a request made before the length is known, for a tile the sequence may not have.)
+__device__ __forceinline__ int page_of(const AttnParams& p, int b, int t, bool flag = true) {
+  const int pg = t < p.pages_per_seq ? p.page_table[(int64_t)b * p.pages_per_seq + t] : -1;
+  if (pg >= 0 && pg < p.n_pages) return pg;
+  if (flag && p.status) atomicOr(p.status + b, SPACE_ST_BAD_PAGE);
+  return p.n_pages;
+}
 
 // One share: tiles t0, t0 + step, ... (n of them) of the T tiles of (sequence b, kv head h).
 struct Seg {
@@ -404,7 +419,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_v) : "memory");
   if (warp == WARP_MMA && lane == 0)
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_q) : "memory");
-  if (early && lane == 0 && (warp == WARP_K || warp == WARP_V)) {
+  if (early && !p.page_table && lane == 0 && (warp == WARP_K || warp == WARP_V)) {
     // A regular group's tiles (sp_piece, sp_piece + sp_base, ...) of head sp_h do not depend on the
     // length, so L2 is asked for them now, while the kernel before this one may still be running:
     // with a programmatic launch this block is resident long before its dependency wait returns,
@@ -447,7 +462,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     mbar_expect_tx(BAR(B_KFULL), S::TILE_BYTES);
 #pragma unroll
     for (int hf = 0; hf < S::HALVES; ++hf)
-      tma_load_4d_hint(sm_base + S::K_OFF + hf * (TILE_N * 128), &p.tm_k, BAR(B_KFULL), hf * 64, sp_piece * TILE_N, sp_h, 0,
+      tma_load_4d_hint(sm_base + S::K_OFF + hf * (TILE_N * 128), &p.tm_k, BAR(B_KFULL), hf * 64,
+                       p.page_table ? 0 : sp_piece * TILE_N, sp_h, p.page_table ? page_of(p, 0, sp_piece, false) : 0,
                        l2_evict_first_policy());
     TL(3);
   }
@@ -473,7 +489,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       spec_ok = 1;
       if (warp == WARP_K && lane == 0 && !*abort_flag) {
         const int n_keys = L + p.n_q;
-        const int kt = (T * TILE_N <= n_keys) ? (T - 1) * TILE_N : n_keys - TILE_N;
+        const int kt = p.page_table ? 0 : ((T * TILE_N <= n_keys) ? (T - 1) * TILE_N : n_keys - TILE_N);
+        const int kb = p.page_table ? page_of(p, 0, T - 1) : 0;
         mbar_expect_tx(BAR(B_QFULL), (uint32_t)n_pad * DH * 2);
 #pragma unroll
         for (int hf = 0; hf < S::HALVES; ++hf)
@@ -481,7 +498,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         mbar_expect_tx(BAR(B_KFULL), S::TILE_BYTES);
 #pragma unroll
         for (int hf = 0; hf < S::HALVES; ++hf)
-          tma_load_4d_hint(sm_base + S::K_OFF + hf * (TILE_N * 128), &p.tm_k, BAR(B_KFULL), hf * 64, kt, sp_h, 0,
+          tma_load_4d_hint(sm_base + S::K_OFF + hf * (TILE_N * 128), &p.tm_k, BAR(B_KFULL), hf * 64, kt, sp_h, kb,
                            l2_evict_first_policy());
         TL(3);
       }
@@ -493,6 +510,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       if (!sp_helper) {
         const int n_mine = sp_piece < Treg ? (Treg - sp_piece + sp_base - 1) / sp_base : 0;
         spec_ok = (n_mine > 0 && (sp_piece + 1) * TILE_N <= L + p.n_q) ? 1 : 0;   // the requested tile is this share's first
+        if (spec_ok && p.page_table && warp == WARP_K && lane == 0) (void)page_of(p, 0, sp_piece);   // flags a bad entry
         reinterpret_cast<int4*>(seg0)[0] = make_int4(0, sp_h, sp_piece, n_mine);
         reinterpret_cast<int4*>(seg0)[1] = make_int4(T, L, sp_h * (sp_base + 1), dn);
         seg0[8] = sp_base; seg0[10] = 0; seg0[11] = sp_h * (sp_base + 1) + sp_piece; seg0[12] = n_mine > 0 ? 1 : 0;
@@ -642,12 +660,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           }
           // the last tile of a sequence is shifted back so that it ends at the
           // last key: rows past the end are never read (they may hold anything)
-          const int kt = ((t + 1) * TILE_N <= n_keys) ? t * TILE_N : n_keys - TILE_N;
+          // (a paged cache has whole pages for tiles instead; see AttnParams)
+          const int kt = p.page_table ? 0 : (((t + 1) * TILE_N <= n_keys) ? t * TILE_N : n_keys - TILE_N);
+          const int kb = p.page_table ? page_of(p, sg.b, t) : sg.b;
           const uint32_t dst = ring + s * S::TILE_BYTES;
           mbar_expect_tx(BAR(b_full + s), S::TILE_BYTES);
 #pragma unroll
           for (int hf = 0; hf < S::HALVES; ++hf)
-            tma_load_4d_hint(dst + hf * (TILE_N * 128), tm, BAR(b_full + s), hf * 64, kt, sg.h, sg.b, kv_policy);
+            tma_load_4d_hint(dst + hf * (TILE_N * 128), tm, BAR(b_full + s), hf * 64, kt, sg.h, kb, kv_policy);
           if (is_k) TL(7);
         }
       }
@@ -795,7 +815,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           if (j < np) tmem_ld8(ts + j * 8, reinterpret_cast<uint32_t*>(sv[j]));
         tmem_wait_ld();
         const int lo = t * TILE_N;
-        const int kt = ((t + 1) * TILE_N <= n_keys) ? lo : n_keys - TILE_N;
+        const int kt = (p.page_table || (t + 1) * TILE_N <= n_keys) ? lo : n_keys - TILE_N;
         const int key = kt + kl;
         const int jb = key - sg.L;                         // block key index when >= 0
         // Visibility of this thread's key: keys before `lo` belong to the previous
@@ -804,6 +824,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
         uint64_t vis = ~0ull;
         if (masked) {
           if (key < lo) vis = 0ull;
+          else if (jb >= p.n_q) vis = 0ull;                 // (paged cache) a row of the page past the last key
           else if (jb >= 0) vis = visq[jb] >> col0;         // (bits past this thread's columns are never looked at)
         }
         // ---- first tile of a share: references from scores at hand.  Any reference within
@@ -956,7 +977,21 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
             st_shared_v4(dst + S::P_PART, lw[0], lw[1], lw[2], lw[3]);
           }
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core
+        if (p.page_table && kt + TILE_N > n_keys) {
+          // Paged cache, last tile: the page's rows past the last key may hold anything, and 0 * NaN
+          // would reach O^T.  Once the V tile has landed, the thread of such a row clears it (a row
+          // is 128 contiguous bytes per 64-wide half of d, whatever the swizzle inside them).
+          const uint32_t vs = gt % S::V_STAGES;
+          ok &= mbar_wait(BAR(B_VFULL + vs), (gt / S::V_STAGES) & 1, abort_flag, p.err, 17);
+          if (key >= n_keys) {
+            for (int hf = half; hf < S::HALVES; hf += 2) {
+              const uint32_t vrow = sm_base + S::V_OFF + vs * S::TILE_BYTES + hf * (TILE_N * 128) + kl * 128;
+#pragma unroll
+              for (int i = 0; i < 8; ++i) st_shared_v4(vrow + i * 16, 0u, 0u, 0u, 0u);
+            }
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P (and a cleared V row) is read by the tensor core
         tc_fence_before();
         mbar_arrive(BAR(B_PREADY + buf));
         if (sidx == 0) { if (gt == 0) TL(6); TL(9); }
@@ -1272,7 +1307,9 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   p.n_mblocks = pl.n_mblocks; p.rows_per_mb = pl.rows_per_mblock;
   p.n_groups = pl.n_ctas / pl.n_mblocks;
   p.n_pad = ((pl.rows_per_mblock * p.G + 15) / 16) * 16;
-  p.out_dtype = a->out_dtype; p.s_cap = cfg.s_cap;
+  p.out_dtype = a->out_dtype;
+  p.s_cap = a->page_table ? (int64_t)a->pages_per_seq * SPACE_PAGE_SIZE : cfg.s_cap;
+  p.page_table = a->page_table; p.pages_per_seq = a->pages_per_seq; p.n_pages = a->n_pages;
   p.scale_log2 = a->scale * 1.4426950408889634f;
   p.kv_len = a->kv_len; p.out = a->out; p.lse = a->lse; p.status = a->status;
   p.part = ctx->attn_part; p.err = ctx->counters + 3 * cfg.max_batch;
@@ -1297,10 +1334,12 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   memcpy(p.visq, ctx->visq, sizeof(p.visq));
 
   // TMA descriptors, rebuilt only when a base pointer or a stride changes
-  const int64_t key[8] = {a->kv_stride_b, a->kv_stride_h, a->kv_stride_s, a->batch, p.n_q, p.n_pad, 0, 0};
+  const int64_t key[8] = {a->kv_stride_b, a->kv_stride_h, a->kv_stride_s, a->batch, p.n_q, p.n_pad,
+                          a->page_table ? a->n_pages : 0, 0};
   if (ctx->tm_q_ptr != a->q || ctx->tm_k_ptr != a->k_cache || ctx->tm_v_ptr != a->v_cache ||
       memcmp(key, ctx->tm_key, sizeof(key)) != 0) {
-    const cuuint64_t kd[4] = {(cuuint64_t)DH, (cuuint64_t)cfg.s_cap, (cuuint64_t)p.H_kv, (cuuint64_t)a->batch};
+    const cuuint64_t kd[4] = {(cuuint64_t)DH, (cuuint64_t)(a->page_table ? TILE_N : cfg.s_cap), (cuuint64_t)p.H_kv,
+                              (cuuint64_t)(a->page_table ? a->n_pages : a->batch)};
     const cuuint64_t ks[3] = {(cuuint64_t)a->kv_stride_s * 2, (cuuint64_t)a->kv_stride_h * 2,
                               (cuuint64_t)a->kv_stride_b * 2};
     const cuuint32_t kb[4] = {64, TILE_N, 1, 1};

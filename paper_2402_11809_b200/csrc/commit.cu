@@ -45,7 +45,8 @@ __global__ void __launch_bounds__(256) kv_commit_kernel(const CommitParams p) {
 void fill_commit_params(const space_ctx* ctx, const space_commit_args* a, CommitParams* pp) {
   CommitParams& p = *pp;
   p.B = a->batch; p.k = a->k; p.H_kv = ctx->cfg.n_kv_heads; p.d = ctx->cfg.head_dim;
-  p.s_cap = ctx->cfg.s_cap;
+  p.s_cap = a->page_table ? (int64_t)a->pages_per_seq * SPACE_PAGE_SIZE : ctx->cfg.s_cap;
+  p.page_table = a->page_table; p.pages_per_seq = a->pages_per_seq; p.n_pages = a->n_pages;
   p.kc = (__nv_bfloat16*)a->k_cache; p.vc = (__nv_bfloat16*)a->v_cache;
   p.sb = a->kv_stride_b; p.sh = a->kv_stride_h; p.ss = a->kv_stride_s;
   p.n_accept = a->n_accept; p.kv_len = a->kv_len; p.kv_len_out = a->kv_len_out;

@@ -128,7 +128,18 @@ struct CommitParams {
   const int32_t* n_accept; const int32_t* kv_len;
   int32_t* kv_len_out; int32_t* src; int32_t* dst; int32_t* status;
   int* counter;
+  const int32_t* page_table; int pages_per_seq, n_pages;   // paged cache (page_table != nullptr): kc / vc are page pools
 };
+
+// Row s of sequence b, head h, of a cache that is contiguous (page_table == nullptr) or paged:
+// offset in elements from the cache base, or -1 for a page-table entry outside the pool.
+__device__ __forceinline__ int64_t kv_row_offset(const int32_t* page_table, int pages_per_seq, int n_pages,
+                                                 int64_t sb, int64_t sh, int64_t ss, int b, int h, int s) {
+  if (!page_table) return (int64_t)b * sb + (int64_t)h * sh + (int64_t)s * ss;
+  const int pg = page_table[(int64_t)b * pages_per_seq + s / SPACE_PAGE_SIZE];
+  if (pg < 0 || pg >= n_pages) return -1;
+  return (int64_t)pg * sb + (int64_t)h * sh + (int64_t)(s % SPACE_PAGE_SIZE) * ss;
+}
 
 __device__ __forceinline__ bool commit_fits(const CommitParams& p, int L) {
   return L >= 0 && (int64_t)L + (int64_t)(p.k + 1) * (p.k + 1) <= p.s_cap;
@@ -156,9 +167,15 @@ __device__ __forceinline__ void commit_rows(const CommitParams& p, int b, int L,
         const int which = r % 2;       r /= 2;
         const int h = r % p.H_kv;      r /= p.H_kv;
         const int g = r + 1;                            // accepted candidate g = 1..i*
-        __nv_bfloat16* base = (which ? p.vc : p.kc) + (int64_t)b * p.sb + (int64_t)h * p.sh;
-        val[u] = *(reinterpret_cast<const uint4*>(base + (int64_t)(L + g * k1) * p.ss) + v);
-        dd[u] = reinterpret_cast<uint4*>(base + (int64_t)(L + g) * p.ss) + v;
+        __nv_bfloat16* base = which ? p.vc : p.kc;
+        const int64_t so = kv_row_offset(p.page_table, p.pages_per_seq, p.n_pages, p.sb, p.sh, p.ss, b, h, L + g * k1);
+        const int64_t dof = kv_row_offset(p.page_table, p.pages_per_seq, p.n_pages, p.sb, p.sh, p.ss, b, h, L + g);
+        if (so >= 0 && dof >= 0) {
+          val[u] = *(reinterpret_cast<const uint4*>(base + so) + v);
+          dd[u] = reinterpret_cast<uint4*>(base + dof) + v;
+        } else if (p.status && v == 0 && which == 0 && h == 0) {
+          atomicOr(p.status + b, SPACE_ST_BAD_PAGE);          // the row stays where it is
+        }
       }
     }
 #pragma unroll

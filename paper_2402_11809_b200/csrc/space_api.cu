@@ -143,6 +143,9 @@ int check_commit_args(const space_ctx* ctx, const space_commit_args* a) {
   if (!aligned16(a->k_cache) || !aligned16(a->v_cache)) return SPACE_E_ALIGNMENT;
   if (a->kv_stride_b % 8 || a->kv_stride_h % 8 || a->kv_stride_s % 8) return SPACE_E_ALIGNMENT;
   if (a->kv_stride_s < ctx->cfg.head_dim) return SPACE_E_INVALID_ARG;
+  if (a->page_table && (a->pages_per_seq < 1 || a->n_pages < 1 ||
+                        (int64_t)a->pages_per_seq * SPACE_PAGE_SIZE > ctx->cfg.s_cap))
+    return SPACE_E_INVALID_ARG;
   return SPACE_OK;
 }
 
@@ -286,6 +289,9 @@ int space_attn_step(space_ctx* ctx, const space_attn_args* a, void* stream) {
     return SPACE_E_ALIGNMENT;
   if (a->kv_stride_s < ctx->cfg.head_dim || a->kv_stride_b < 1 || a->kv_stride_h < 1) return SPACE_E_INVALID_ARG;
   if (a->kv_stride_b % 8 || a->kv_stride_h % 8 || a->kv_stride_s % 8) return SPACE_E_ALIGNMENT;
+  if (a->page_table && (a->pages_per_seq < 1 || a->n_pages < 1 ||
+                        (int64_t)a->pages_per_seq * SPACE_PAGE_SIZE > ctx->cfg.s_cap))
+    return SPACE_E_INVALID_ARG;
   if (!use_device(ctx)) return SPACE_E_CUDA;
   if (ctx->lay_k != a->k || ctx->lay_variant != a->mask_variant) {   // the layout is rebuilt only when k or the reading changes
     space_layout_t lay;

@@ -34,6 +34,8 @@ class DeviceStep:
         self.k_cache = to_dev(x["k_cache"])
         self.v_cache = to_dev(x["v_cache"])
         self.kv_len = to_dev(x["kv_len"])
+        # paged cache (workloads.to_pages): k_cache / v_cache are page pools, found through the table
+        self.page_table = to_dev(x["page_table"]) if "page_table" in x else None
         self.logits = to_dev(x["logits"])
         self.cand = to_dev(x["cand"])
         self.cand_prob = to_dev(x["cand_prob"])
@@ -56,7 +58,7 @@ class DeviceStep:
     def attn(self, ctx, impl=B.ATTN_TENSOR, mask_variant=B.MASK_SAME_GROUP, out=None):
         a = ctx.attn_args(self.q, self.k_cache, self.v_cache, self.kv_len,
                           self.out if out is None else out, self.k, self.scale, lse=self.lse,
-                          status=self.status, mask_variant=mask_variant, impl=impl)
+                          status=self.status, mask_variant=mask_variant, impl=impl, page_table=self.page_table)
         ctx.space_attn_step(a)
         return a
 
@@ -77,13 +79,13 @@ class DeviceStep:
                             resample=resample, eos_id=eos_id, seq_id=self.seq_id, status=self.status)
         c = ctx.commit_args(self.k_cache, self.v_cache, self.n_accept, self.kv_len, self.k,
                             kv_len_out=self.kv_len if in_place else self.kv_len_out,
-                            commit_src=self.commit_src, commit_dst=self.commit_dst, status=self.status)
+                            commit_src=self.commit_src, commit_dst=self.commit_dst, status=self.status, page_table=self.page_table)
         ctx.space_verify_commit(v, c)
         return v, c
 
     def commit(self, ctx):
         a = ctx.commit_args(self.k_cache, self.v_cache, self.n_accept, self.kv_len, self.k,
                             kv_len_out=self.kv_len_out, commit_src=self.commit_src,
-                            commit_dst=self.commit_dst, status=self.status)
+                            commit_dst=self.commit_dst, status=self.status, page_table=self.page_table)
         ctx.space_kv_commit(a)
         return a

@@ -112,6 +112,38 @@ def make_step_inputs(cfg, set_index=0, s_cap=None, poison_tail=False):
                 s_cap=s_cap, n_q=n_q, scale=float(1.0 / np.sqrt(d)))
 
 
+PAGE_SIZE = 128
+
+
+def to_pages(x, seed=0, extra_pages=3, poison=True):
+    """The caches of a step's inputs as page pools (the cache of a serving engine with continuous
+    batching): returns a copy of x whose k_cache / v_cache are pools [n_pages, H_kv, PAGE_SIZE, d]
+    and which carries page_table [B, pages_per_seq] (int32).  Every sequence gets the pages its
+    L_b + n_q rows need plus whatever its capacity (s_cap rounded up to whole pages) allows, pages
+    of all sequences shuffled among `extra_pages` unused ones.  Rows that hold no key -- the tail
+    of a sequence's last page, its spare pages, the unused pages -- are NaN patterns when `poison`
+    is set (zero otherwise): nothing may depend on them."""
+    kc, vc = x["k_cache"], x["v_cache"]
+    B, H, S, d = kc.shape
+    n_q = x["n_q"]
+    pps = (S + PAGE_SIZE - 1) // PAGE_SIZE
+    n_pages = B * pps + extra_pages
+    rng = np.random.Generator(np.random.Philox(key=[seed, 12345]))
+    table = rng.permutation(n_pages)[: B * pps].reshape(B, pps).astype(np.int32)
+    fill = np.uint16(0x7FC0) if poison else np.uint16(0)
+    kp = np.full((n_pages, H, PAGE_SIZE, d), fill, dtype=np.uint16)
+    vp = np.full((n_pages, H, PAGE_SIZE, d), fill, dtype=np.uint16)
+    for b in range(B):
+        n = int(x["kv_len"][b]) + n_q
+        for j in range((n + PAGE_SIZE - 1) // PAGE_SIZE):
+            r = min(PAGE_SIZE, n - j * PAGE_SIZE)
+            kp[table[b, j], :, :r, :] = kc[b, :, j * PAGE_SIZE: j * PAGE_SIZE + r, :]
+            vp[table[b, j], :, :r, :] = vc[b, :, j * PAGE_SIZE: j * PAGE_SIZE + r, :]
+    y = dict(x)
+    y.update(k_cache=kp, v_cache=vp, page_table=table, s_cap=pps * PAGE_SIZE)
+    return y
+
+
 def algorithmic_bytes(cfg, kv_len, n_accept=None):
     """Bytes one step has to move at least once: K and V of the cache and block,
     Q, the attention output (as bf16), 2k+1 logits rows per sequence and the

@@ -1,0 +1,133 @@
+"""GPU parity for the paged KV cache (the serving setting of Sec. 4.3): attention of all three
+implementations and the compaction of accepted rows, through the C ABI, against oracle.paged on
+page pools whose unused rows -- spare pages, pages of no sequence, the tail of every sequence's
+last page -- are NaN patterns.  Same tolerances as the contiguous cache: attention within
+min(2e-2, 1e-2 RMS), log-sum-exp 2e-3, cache bytes and lengths exact."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from oracle.paged import attention_step_paged, commit_step_paged
+from oracle.verify import verify_step
+from oracle.bf16 import bf16_bits_to_f64
+from paper_2402_11809_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2402_11809_b200 import build
+    build.build()
+    from paper_2402_11809_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def H():
+    import gpu_harness
+    return gpu_harness
+
+
+def _cfg(k, L, d=128, H_q=2, H_kv=2, Bn=3, V=777, seed=0):
+    return workloads.resolve("tiny", B=Bn, H_q=H_q, H_kv=H_kv, d=d, L=L, k=k, V=V, logits_dtype="bf16",
+                             sigma=2.0, p_accept=(0.6, 0.6), seed=seed)
+
+
+IMPL = {"tensor": "ATTN_TENSOR", "rows": "ATTN_TENSOR_ROWS", "simt": "ATTN_SIMT"}
+
+
+@pytest.mark.parametrize("impl", ["tensor", "rows", "simt"])
+@pytest.mark.parametrize("k,L,d,H_q,H_kv,Bn", [
+    (1, (0, 0), 64, 2, 2, 3),            # the block's rows only
+    (3, (119, 119), 128, 2, 1, 2),       # L + n_q = 135: the block straddles two pages
+    (4, (103, 103), 64, 8, 8, 2),        # L + n_q = 128: ends exactly on a page boundary
+    (5, (129, 700), 128, 4, 4, 3),
+    (7, (5, 900), 128, 4, 2, 3),
+    (2, (10, 200), 64, 64, 64, 3),       # more (sequence, head) pairs than thread blocks: the flat cut
+    (5, (2048, 2048), 128, 32, 32, 1),   # one sequence: pieces per head, helper groups, early requests
+    (6, (3000, 3300), 128, 8, 1, 1),     # one sequence, grouped heads
+])
+def test_paged_attention(B, H, impl, k, L, d, H_q, H_kv, Bn):
+    cfg = _cfg(k, L, d=d, H_q=H_q, H_kv=H_kv, Bn=Bn, seed=70 + k)
+    x = workloads.to_pages(workloads.make_step_inputs(cfg), seed=k)
+    if impl == "simt" and x["s_cap"] > 3000:
+        pytest.skip("the SIMT cross-check keeps a sequence's scores in shared memory")
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    ds.attn(ctx, impl=getattr(B, IMPL[impl]))
+    torch.cuda.synchronize()
+    ref, ref_lse = attention_step_paged(bf16_bits_to_f64(x["q"]), bf16_bits_to_f64(x["k_cache"]),
+                                        bf16_bits_to_f64(x["v_cache"]), x["page_table"], x["kv_len"], k, x["scale"])
+    H.check_attention(ds.out.cpu().numpy().astype(np.float64), ref, f"paged {impl} k={k} L={L}")
+    np.testing.assert_allclose(ds.lse.cpu().numpy(), ref_lse, rtol=0, atol=2e-3)
+    assert int(ds.status.abs().sum()) == 0
+
+
+def test_paged_commit_and_verify_commit(B, H):
+    for k, L in ((5, (100, 140)), (3, (240, 260)), (7, (0, 70))):      # moved rows on both sides of page boundaries
+        cfg = _cfg(k, L, Bn=6, seed=90 + k)
+        x = workloads.to_pages(workloads.make_step_inputs(cfg), seed=k, poison=False)
+        ctx = H.make_context(cfg, x)
+        r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "greedy")
+        assert r["n_accept"].max() > 0
+        for fused in (False, True):
+            ds = H.DeviceStep(cfg, x)
+            if fused:
+                ds.verify_commit(ctx)
+            else:
+                ds.verify(ctx)
+                ds.commit(ctx)
+            torch.cuda.synchronize()
+            kp, vp = x["k_cache"].copy(), x["v_cache"].copy()
+            new_len = commit_step_paged(kp, vp, x["page_table"], x["kv_len"], r["n_accept"], k)
+            assert np.array_equal(ds.kv_len_out.cpu().numpy(), new_len)
+            gk, gv = H.bf16_to_bits(ds.k_cache), H.bf16_to_bits(ds.v_cache)
+            if fused:
+                # the single-launch form also moves the rejected candidates' rows to L+i*+1 .. L+k,
+                # rows beyond the new length that nobody reads again
+                for b in range(cfg["B"]):
+                    for s in range(int(new_len[b]), int(x["kv_len"][b]) + k + 1):
+                        pg = int(x["page_table"][b, s // 128])
+                        gk[pg, :, s % 128, :] = kp[pg, :, s % 128, :]
+                        gv[pg, :, s % 128, :] = vp[pg, :, s % 128, :]
+            assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
+            assert int(ds.status.abs().sum()) == 0
+
+
+def test_paged_capacity_bad_pages_and_arguments(B, H):
+    k = 3
+    cfg = _cfg(k, (200, 230), Bn=2, seed=5)
+    x = workloads.to_pages(workloads.make_step_inputs(cfg), seed=1, poison=False)
+    ctx = H.make_context(cfg, x)
+    # a table entry outside the pool: flagged, nothing read or written through it
+    bad = dict(x)
+    bad["page_table"] = x["page_table"].copy()
+    bad["page_table"][1, 0] = x["k_cache"].shape[0] + 5
+    for impl in ("tensor", "rows", "simt"):
+        ds = H.DeviceStep(cfg, bad)
+        ds.attn(ctx, impl=getattr(B, IMPL[impl]))
+        torch.cuda.synchronize()
+        st = ds.status.cpu().numpy()
+        assert st[1] & B.ST_BAD_PAGE and not st[0] & B.ST_BAD_PAGE, (impl, st)
+        assert torch.isfinite(ds.out).all()
+    # a length beyond the table's capacity: flagged, output untouched
+    over = dict(x)
+    over["kv_len"] = x["kv_len"].copy()
+    over["kv_len"][0] = x["page_table"].shape[1] * 128 - 3
+    for impl in ("tensor", "rows", "simt"):
+        ds = H.DeviceStep(cfg, over)
+        ds.attn(ctx, impl=getattr(B, IMPL[impl]))
+        torch.cuda.synchronize()
+        assert ds.status.cpu().numpy()[0] & B.ST_CAPACITY
+        assert torch.isnan(ds.out[0]).all() and torch.isfinite(ds.out[1]).all()
+    # arguments: a table needs its sizes, and its capacity must fit the context's
+    ds = H.DeviceStep(cfg, x)
+    a = ctx.attn_args(ds.q, ds.k_cache, ds.v_cache, ds.kv_len, ds.out, k, ds.scale, page_table=ds.page_table)
+    for field, val in (("pages_per_seq", 0), ("n_pages", 0), ("pages_per_seq", 10 ** 6)):
+        b2 = B.AttnArgs.from_buffer_copy(a)
+        setattr(b2, field, val)
+        assert B.lib.space_attn_step(ctx._h, C.byref(b2), None) == B.E_INVALID_ARG, field
+    torch.cuda.synchronize()
