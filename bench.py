@@ -232,6 +232,8 @@ def run_ours(args):
     cfg = workloads.resolve(args.config, **({"B": args.batch} if args.batch else {}))
     if args.batch:
         cfg["name"] = f"{args.config}@batch{args.batch}"   # a reduced copy of the workload (profiler captures)
+    if args.paged:
+        cfg["name"] += "+paged"                            # (no profiler capture of this form: traffic stays null)
     k, n_q = cfg["k"], workloads.n_block_rows(cfg["k"])
     sample = cfg["mode"] == "sample"
     mode = B.MODE_SAMPLE if sample else B.MODE_GREEDY
@@ -243,20 +245,24 @@ def run_ours(args):
     n_sets = min(n_sets, 16)
     sets = [x0] + [workloads.make_step_inputs(cfg, set_index=replicas.set_index(rank, i)) for i in range(1, n_sets)]
 
-    s_cap = max(x["s_cap"] for x in sets)
+    # --paged: the same caches as page pools behind shuffled page tables (the host-buffer leg and the
+    # oracle keep the contiguous form: space_step_host has no paged variant)
+    dev_sets = [workloads.to_pages(x, seed=i, poison=False) for i, x in enumerate(sets)] if args.paged else sets
+    s_cap = max(x["s_cap"] for x in dev_sets + sets)
     ctx = B.Context(device=local, max_batch=cfg["B"], n_q_heads=cfg["H_q"], n_kv_heads=cfg["H_kv"],
                     head_dim=cfg["d"], k_max=k, vocab=cfg["V"], host_staging=1, s_cap=s_cap)
-    steps_dev = [H.DeviceStep(cfg, x) for x in sets]
+    steps_dev = [H.DeviceStep(cfg, x) for x in dev_sets]
     arg_sets = []
     for ds in steps_dev:
         a = ctx.attn_args(ds.q, ds.k_cache, ds.v_cache, ds.kv_len, ds.out, k, ds.scale, status=ds.status,
-                          impl=B.ATTN_TENSOR_ROWS if args.attn_impl == "rows" else B.ATTN_TENSOR)
+                          impl=B.ATTN_TENSOR_ROWS if args.attn_impl == "rows" else B.ATTN_TENSOR,
+                          page_table=ds.page_table)
         v = ctx.verify_args(ds.logits, ds.cand, ds.cand_prob, ds.kv_len, ds.n_accept, ds.out_tokens,
                             ds.n_out, ds.next_cand, ds.next_cand_prob, ds.finished, k, mode=mode,
                             temperature=cfg["temperature"], seed=cfg["seed"], seq_id=ds.seq_id,
                             status=ds.status)
         c = ctx.commit_args(ds.k_cache, ds.v_cache, ds.n_accept, ds.kv_len, k, kv_len_out=ds.kv_len_out,
-                            status=ds.status)
+                            status=ds.status, page_table=ds.page_table)
         arg_sets.append((a, v, c))
 
     def step(i):
@@ -426,6 +432,7 @@ def run_ours(args):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg["name"], "batch": cfg["B"], "k": k, "heads": [cfg["H_q"], cfg["H_kv"]],
                    "head_dim": cfg["d"], "kv_len": list(cfg["L"]), "vocab": cfg["V"], "mode": cfg["mode"],
+                   "cache": "page pools of 128-row pages behind shuffled page tables" if args.paged else "contiguous",
                    "l2": f"{n_sets} distinct input sets rotated ({n_sets * ab['total'] / 1e6:.0f} MB > 2 x L2)",
                    "launch": "CUDA graph replay of the C-ABI calls (" +
                              ("space_attn_step, space_verify, space_kv_commit" if args.separate_commit
@@ -654,6 +661,8 @@ def main():
                          "captures; the bench line then names the workload NAME@batchN)")
     ap.add_argument("--separate-commit", action="store_true",
                     help="three calls per step (space_verify, then space_kv_commit) instead of space_verify_commit")
+    ap.add_argument("--paged", action="store_true",
+                    help="keep the KV caches as page pools behind page tables (attention and commit through the table)")
     ap.add_argument("--attn-impl", default="tensor", choices=["tensor", "rows"],
                     help="tensor: keys on the MMA M extent (default); rows: query rows on M")
     args = ap.parse_args()

@@ -349,7 +349,9 @@ constexpr float OVER_THRESHOLD = 60.f;   // re-reference a query row when a scor
 // and O^T += V^T P^T (head_dim x N), so the MMA N extent is the number of
 // query rows rounded up to 16 instead of a full 128-row tile, and one thread
 // owns one key of the tile (all 128 TMEM lanes carry work).
-template <int DH>
+// PAGED: the cache is a pool of pages behind a page table (see AttnParams); a build of its own, so
+// that the contiguous form carries none of it (registers are at the limit of 384 threads).
+template <int DH, bool PAGED>
 __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_constant__ AttnParams p,
                                                              int max_batch) {
   using S = Smem<DH>;
@@ -419,7 +421,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_v) : "memory");
   if (warp == WARP_MMA && lane == 0)
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&p.tm_q) : "memory");
-  if (early && !p.page_table && lane == 0 && (warp == WARP_K || warp == WARP_V)) {
+  if (early && !PAGED && lane == 0 && (warp == WARP_K || warp == WARP_V)) {
     // A regular group's tiles (sp_piece, sp_piece + sp_base, ...) of head sp_h do not depend on the
     // length, so L2 is asked for them now, while the kernel before this one may still be running:
     // with a programmatic launch this block is resident long before its dependency wait returns,
@@ -463,7 +465,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
 #pragma unroll
     for (int hf = 0; hf < S::HALVES; ++hf)
       tma_load_4d_hint(sm_base + S::K_OFF + hf * (TILE_N * 128), &p.tm_k, BAR(B_KFULL), hf * 64,
-                       p.page_table ? 0 : sp_piece * TILE_N, sp_h, p.page_table ? page_of(p, 0, sp_piece, false) : 0,
+                       PAGED ? 0 : sp_piece * TILE_N, sp_h, PAGED ? page_of(p, 0, sp_piece, false) : 0,
                        l2_evict_first_policy());
     TL(3);
   }
@@ -489,8 +491,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       spec_ok = 1;
       if (warp == WARP_K && lane == 0 && !*abort_flag) {
         const int n_keys = L + p.n_q;
-        const int kt = p.page_table ? 0 : ((T * TILE_N <= n_keys) ? (T - 1) * TILE_N : n_keys - TILE_N);
-        const int kb = p.page_table ? page_of(p, 0, T - 1) : 0;
+        const int kt = PAGED ? 0 : ((T * TILE_N <= n_keys) ? (T - 1) * TILE_N : n_keys - TILE_N);
+        const int kb = PAGED ? page_of(p, 0, T - 1) : 0;
         mbar_expect_tx(BAR(B_QFULL), (uint32_t)n_pad * DH * 2);
 #pragma unroll
         for (int hf = 0; hf < S::HALVES; ++hf)
@@ -510,7 +512,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
       if (!sp_helper) {
         const int n_mine = sp_piece < Treg ? (Treg - sp_piece + sp_base - 1) / sp_base : 0;
         spec_ok = (n_mine > 0 && (sp_piece + 1) * TILE_N <= L + p.n_q) ? 1 : 0;   // the requested tile is this share's first
-        if (spec_ok && p.page_table && warp == WARP_K && lane == 0) (void)page_of(p, 0, sp_piece);   // flags a bad entry
+        if (PAGED && spec_ok && warp == WARP_K && lane == 0) (void)page_of(p, 0, sp_piece);   // flags a bad entry
         reinterpret_cast<int4*>(seg0)[0] = make_int4(0, sp_h, sp_piece, n_mine);
         reinterpret_cast<int4*>(seg0)[1] = make_int4(T, L, sp_h * (sp_base + 1), dn);
         seg0[8] = sp_base; seg0[10] = 0; seg0[11] = sp_h * (sp_base + 1) + sp_piece; seg0[12] = n_mine > 0 ? 1 : 0;
@@ -661,8 +663,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           // the last tile of a sequence is shifted back so that it ends at the
           // last key: rows past the end are never read (they may hold anything)
           // (a paged cache has whole pages for tiles instead; see AttnParams)
-          const int kt = p.page_table ? 0 : (((t + 1) * TILE_N <= n_keys) ? t * TILE_N : n_keys - TILE_N);
-          const int kb = p.page_table ? page_of(p, sg.b, t) : sg.b;
+          const int kt = PAGED ? 0 : (((t + 1) * TILE_N <= n_keys) ? t * TILE_N : n_keys - TILE_N);
+          const int kb = PAGED ? page_of(p, sg.b, t) : sg.b;
           const uint32_t dst = ring + s * S::TILE_BYTES;
           mbar_expect_tx(BAR(b_full + s), S::TILE_BYTES);
 #pragma unroll
@@ -815,7 +817,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
           if (j < np) tmem_ld8(ts + j * 8, reinterpret_cast<uint32_t*>(sv[j]));
         tmem_wait_ld();
         const int lo = t * TILE_N;
-        const int kt = (p.page_table || (t + 1) * TILE_N <= n_keys) ? lo : n_keys - TILE_N;
+        const int kt = (PAGED || (t + 1) * TILE_N <= n_keys) ? lo : n_keys - TILE_N;
         const int key = kt + kl;
         const int jb = key - sg.L;                         // block key index when >= 0
         // Visibility of this thread's key: keys before `lo` belong to the previous
@@ -977,7 +979,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
             st_shared_v4(dst + S::P_PART, lw[0], lw[1], lw[2], lw[3]);
           }
         }
-        if (p.page_table && kt + TILE_N > n_keys) {
+        if (PAGED && kt + TILE_N > n_keys) {
           // Paged cache, last tile: the page's rows past the last key may hold anything, and 0 * NaN
           // would reach O^T.  Once the V tile has landed, the thread of such a row clears it (a row
           // is 128 contiguous bytes per 64-wide half of d, whatever the swizzle inside them).
@@ -1252,19 +1254,19 @@ size_t smem_bytes(int max_batch) {
   return Smem<DH>::TABLE_OFF + (size_t)(2 * max_batch + 1) * sizeof(int);
 }
 
-template <int DH>
+template <int DH, bool PAGED>
 cudaError_t launch_main(const AttnParams& p, int n_ctas, int max_batch, cudaStream_t st) {
   const size_t sm = smem_bytes<DH>(max_batch);
   // the shared-memory limit of the kernel is raised once per device (to the most any batch needs)
-  static unsigned long long done_mask = 0;
+  static unsigned long long done_mask = 0;                 // (one per instantiation)
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 64 || !((done_mask >> dev) & 1ull)) {
-    cudaFuncSetAttribute(attn_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaFuncSetAttribute(attn_tc_kernel<DH, PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          (int)smem_bytes<DH>(128));
     if (dev < 64) done_mask |= 1ull << dev;
   }
-  return launch_pdl(attn_tc_kernel<DH>, dim3(n_ctas), dim3(THREADS), sm, st, p, max_batch);
+  return launch_pdl(attn_tc_kernel<DH, PAGED>, dim3(n_ctas), dim3(THREADS), sm, st, p, max_batch);
 }
 
 }  // namespace
@@ -1361,8 +1363,13 @@ int launch_attn_tensor(space_ctx* ctx, const space_attn_args* a, const uint64_t*
   const dim3 mgrid(p.merge_by_owner ? pl.n_ctas : a->batch * p.H_kv * p.n_mblocks, (m_valid_max * (DH / 4) + 127) / 128);
   {
     ProfScope ps(ctx, SPACE_K_ATTN, st);
-    if (DH == 128) launch_main<128>(p, pl.n_ctas, cfg.max_batch, st);
-    else launch_main<64>(p, pl.n_ctas, cfg.max_batch, st);
+    if (a->page_table) {
+      if (DH == 128) launch_main<128, true>(p, pl.n_ctas, cfg.max_batch, st);
+      else launch_main<64, true>(p, pl.n_ctas, cfg.max_batch, st);
+    } else {
+      if (DH == 128) launch_main<128, false>(p, pl.n_ctas, cfg.max_batch, st);
+      else launch_main<64, false>(p, pl.n_ctas, cfg.max_batch, st);
+    }
   }
   {
     ProfScope ps(ctx, SPACE_K_MERGE, st);

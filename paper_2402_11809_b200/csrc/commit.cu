@@ -17,7 +17,7 @@ __global__ void __launch_bounds__(256) kv_commit_kernel(const CommitParams p) {
   int i_star = p.n_accept[b];
   i_star = max(0, min(i_star, p.k));
   const bool fits = commit_fits(p, L);
-  if (fits) commit_rows(p, b, L, i_star, part, p.blocks_per_seq, threadIdx.x, blockDim.x);
+  if (fits) commit_rows_any(p, b, L, i_star, part, p.blocks_per_seq, threadIdx.x, blockDim.x);
   // New length and index tables.  When the new length goes to its own array no
   // block depends on another and block 0 writes them at once; when it overwrites
   // kv_len itself the other blocks must have read the old value first, so the

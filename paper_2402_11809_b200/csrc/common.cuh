@@ -147,8 +147,9 @@ __device__ __forceinline__ bool commit_fits(const CommitParams& p, int L) {
 
 // Slice `part` of `nparts` of sequence b's move, by `nthreads` threads (this one is `tid`).
 // All loads of a batch are issued before its stores.
-__device__ __forceinline__ void commit_rows(const CommitParams& p, int b, int L, int i_star, int part, int nparts,
-                                            int tid, int nthreads) {
+template <bool PAGED>
+__device__ __forceinline__ void commit_rows_impl(const CommitParams& p, int b, int L, int i_star, int part, int nparts,
+                                                 int tid, int nthreads) {
   const int k1 = p.k + 1;
   const int vec_per_row = p.d / 8;                      // 16-byte pieces per row
   const int total = i_star * p.H_kv * 2 * vec_per_row;
@@ -167,14 +168,20 @@ __device__ __forceinline__ void commit_rows(const CommitParams& p, int b, int L,
         const int which = r % 2;       r /= 2;
         const int h = r % p.H_kv;      r /= p.H_kv;
         const int g = r + 1;                            // accepted candidate g = 1..i*
-        __nv_bfloat16* base = which ? p.vc : p.kc;
-        const int64_t so = kv_row_offset(p.page_table, p.pages_per_seq, p.n_pages, p.sb, p.sh, p.ss, b, h, L + g * k1);
-        const int64_t dof = kv_row_offset(p.page_table, p.pages_per_seq, p.n_pages, p.sb, p.sh, p.ss, b, h, L + g);
-        if (so >= 0 && dof >= 0) {
-          val[u] = *(reinterpret_cast<const uint4*>(base + so) + v);
-          dd[u] = reinterpret_cast<uint4*>(base + dof) + v;
-        } else if (p.status && v == 0 && which == 0 && h == 0) {
-          atomicOr(p.status + b, SPACE_ST_BAD_PAGE);          // the row stays where it is
+        if (!PAGED) {
+          __nv_bfloat16* base = (which ? p.vc : p.kc) + (int64_t)b * p.sb + (int64_t)h * p.sh;
+          val[u] = *(reinterpret_cast<const uint4*>(base + (int64_t)(L + g * k1) * p.ss) + v);
+          dd[u] = reinterpret_cast<uint4*>(base + (int64_t)(L + g) * p.ss) + v;
+        } else {
+          __nv_bfloat16* base = which ? p.vc : p.kc;
+          const int64_t so = kv_row_offset(p.page_table, p.pages_per_seq, p.n_pages, p.sb, p.sh, p.ss, b, h, L + g * k1);
+          const int64_t dof = kv_row_offset(p.page_table, p.pages_per_seq, p.n_pages, p.sb, p.sh, p.ss, b, h, L + g);
+          if (so >= 0 && dof >= 0) {
+            val[u] = *(reinterpret_cast<const uint4*>(base + so) + v);
+            dd[u] = reinterpret_cast<uint4*>(base + dof) + v;
+          } else if (p.status && v == 0 && which == 0 && h == 0) {
+            atomicOr(p.status + b, SPACE_ST_BAD_PAGE);        // the row stays where it is
+          }
         }
       }
     }
@@ -182,6 +189,19 @@ __device__ __forceinline__ void commit_rows(const CommitParams& p, int b, int L,
     for (int u = 0; u < U; ++u)
       if (dd[u]) *dd[u] = val[u];
   }
+}
+
+// Contiguous cache only: the form the verify kernels carry (it sits in their critical path; with a
+// paged cache space_verify_commit runs the commit kernel after them instead).
+__device__ __forceinline__ void commit_rows(const CommitParams& p, int b, int L, int i_star, int part, int nparts,
+                                            int tid, int nthreads) {
+  commit_rows_impl<false>(p, b, L, i_star, part, nparts, tid, nthreads);
+}
+// Either cache form (the commit kernel).
+__device__ __forceinline__ void commit_rows_any(const CommitParams& p, int b, int L, int i_star, int part, int nparts,
+                                                int tid, int nthreads) {
+  if (p.page_table) commit_rows_impl<true>(p, b, L, i_star, part, nparts, tid, nthreads);
+  else commit_rows_impl<false>(p, b, L, i_star, part, nparts, tid, nthreads);
 }
 
 // New length and index tables of sequence b (one thread).

@@ -698,6 +698,12 @@ int launch_verify(space_ctx* ctx, const space_verify_args* a, const space_commit
     if (rc != SPACE_OK || !cm) return rc;
     return launch_commit(ctx, cm, st);
   }
+  if (cm && cm->page_table) {
+    // paged cache: the verify kernels carry the contiguous commit only; the commit kernel follows
+    const int rc = launch_verify(ctx, a, nullptr, st);
+    if (rc != SPACE_OK) return rc;
+    return launch_commit(ctx, cm, st);
+  }
   VerifyParams p;
   p.do_commit = cm != nullptr;
   if (cm) fill_commit_params(ctx, cm, &p.cm); else memset(&p.cm, 0, sizeof(p.cm));
