@@ -463,6 +463,28 @@ int space_debug_philox(space_ctx* ctx, uint64_t seed, int64_t n, const uint32_t*
  * Errors: INVALID_ARG (NULL, limit out of range), CUDA. */
 int space_debug_wait_timeout(space_ctx* ctx, uint64_t limit_ns, int32_t* out4, void* stream);
 
+/* Page bookkeeping for a paged cache shared by sequences that come and go between steps (the
+ * serving setting of Sec. 4.3: continuous batching).  Host-side only: it hands out pages of a pool
+ * and keeps every sequence's page list; the pool's memory and the device copy of a table belong to
+ * the caller.  A sequence occupies a slot from space_pager_admit to space_pager_release; a step's
+ * batch is any list of slots, and space_pager_batch_table writes the table rows of those slots in
+ * that order, the page_table that space_attn_args / space_commit_args take for that batch.
+ * Not thread-safe.  Errors: INVALID_ARG (NULL, slot not in use, sizes out of range), WORKSPACE (no
+ * free slot; not enough free pages, in which case nothing has changed). */
+typedef struct space_pager space_pager;
+int  space_pager_create(int32_t n_pages, int32_t pages_per_seq, int32_t max_slots, space_pager** out);
+void space_pager_destroy(space_pager* p);
+int  space_pager_admit(space_pager* p, int32_t* slot);          /* a free slot, holding no page yet     */
+int  space_pager_reserve(space_pager* p, int32_t slot, int32_t n_rows);
+                             /* pages so that cache rows 0 .. n_rows-1 of the slot exist (a sequence
+                                of length L needs L + (k+1)^2 rows before its next step); pages a
+                                slot already holds stay where they are                                */
+int  space_pager_release(space_pager* p, int32_t slot);         /* its pages return to the pool         */
+int32_t space_pager_free_pages(const space_pager* p);
+int32_t space_pager_rows(const space_pager* p, int32_t slot);   /* rows reserved for the slot, -1 if unused */
+int  space_pager_batch_table(const space_pager* p, const int32_t* slots, int32_t n,
+                             int32_t* table_out);               /* host [n, pages_per_seq]; -1 = no page */
+
 const char* space_strerror(int code);
 
 #ifdef __cplusplus

@@ -31,7 +31,9 @@ EXPORTS = ["space_create", "space_destroy", "space_workspace_bytes", "space_layo
            "space_lmhead_verify", "space_sar_sft_transform", "space_decode_begin", "space_decode_advance",
            "space_step_host",
            "space_launch_count", "space_profile_enable", "space_profile_read",
-           "space_debug_philox", "space_debug_wait_timeout", "space_strerror"]
+           "space_debug_philox", "space_debug_wait_timeout", "space_strerror",
+           "space_pager_create", "space_pager_destroy", "space_pager_admit", "space_pager_reserve",
+           "space_pager_release", "space_pager_free_pages", "space_pager_rows", "space_pager_batch_table"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -165,6 +167,22 @@ lib.space_debug_wait_timeout.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.c
 lib.space_debug_wait_timeout.restype = C.c_int
 lib.space_strerror.argtypes = [C.c_int]
 lib.space_strerror.restype = C.c_char_p
+lib.space_pager_create.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_void_p)]
+lib.space_pager_create.restype = C.c_int
+lib.space_pager_destroy.argtypes = [C.c_void_p]
+lib.space_pager_destroy.restype = None
+lib.space_pager_admit.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
+lib.space_pager_admit.restype = C.c_int
+lib.space_pager_reserve.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+lib.space_pager_reserve.restype = C.c_int
+lib.space_pager_release.argtypes = [C.c_void_p, C.c_int32]
+lib.space_pager_release.restype = C.c_int
+lib.space_pager_free_pages.argtypes = [C.c_void_p]
+lib.space_pager_free_pages.restype = C.c_int32
+lib.space_pager_rows.argtypes = [C.c_void_p, C.c_int32]
+lib.space_pager_rows.restype = C.c_int32
+lib.space_pager_batch_table.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+lib.space_pager_batch_table.restype = C.c_int
 
 
 class SpaceError(RuntimeError):
@@ -362,3 +380,45 @@ class Context:
     def space_debug_philox(self, seed, c0, c1, c2, c3, out):
         _check(lib.space_debug_philox(self._h, seed, c0.numel(), _ptr(c0), _ptr(c1), _ptr(c2),
                                       _ptr(c3), _ptr(out), _stream()))
+
+
+class Pager:
+    """Page bookkeeping of a paged cache (space_pager_*): slots, pages, batch tables.  Host only."""
+
+    def __init__(self, n_pages, pages_per_seq, max_slots):
+        h = C.c_void_p()
+        _check(lib.space_pager_create(n_pages, pages_per_seq, max_slots, C.byref(h)))
+        self._h, self.pages_per_seq = h, pages_per_seq
+
+    def close(self):
+        if self._h:
+            lib.space_pager_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def admit(self):
+        s = C.c_int32(-1)
+        _check(lib.space_pager_admit(self._h, C.byref(s)))
+        return s.value
+
+    def reserve(self, slot, n_rows):
+        _check(lib.space_pager_reserve(self._h, slot, n_rows))
+
+    def release(self, slot):
+        _check(lib.space_pager_release(self._h, slot))
+
+    @property
+    def free_pages(self):
+        return lib.space_pager_free_pages(self._h)
+
+    def rows(self, slot):
+        return lib.space_pager_rows(self._h, slot)
+
+    def batch_table(self, slots):
+        import numpy as np
+        sl = np.ascontiguousarray(slots, dtype=np.int32)
+        out = np.empty((len(sl), self.pages_per_seq), dtype=np.int32)
+        _check(lib.space_pager_batch_table(self._h, sl.ctypes.data_as(C.c_void_p), len(sl),
+                                           out.ctypes.data_as(C.c_void_p)))
+        return out

@@ -10,7 +10,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libspace.so")
-SOURCES = ["space_api.cu", "attn_tc.cu", "attn_rows.cu", "attn_simt.cu", "verify.cu", "commit.cu", "lmhead.cu", "decode.cu", "sar_sft.cu", "verify_filter.cu"]
+SOURCES = ["space_api.cu", "attn_tc.cu", "attn_rows.cu", "attn_simt.cu", "verify.cu", "commit.cu", "lmhead.cu", "decode.cu", "sar_sft.cu", "verify_filter.cu", "pager.cu"]
 
 
 def _nvcc():

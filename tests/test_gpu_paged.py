@@ -131,3 +131,92 @@ def test_paged_capacity_bad_pages_and_arguments(B, H):
         setattr(b2, field, val)
         assert B.lib.space_attn_step(ctx._h, C.byref(b2), None) == B.E_INVALID_ARG, field
     torch.cuda.synchronize()
+
+
+def test_continuous_batching_over_a_shared_pool(B, H):
+    """Sequences join and leave between steps; the pager hands their pages out of one pool and the
+    step's batch is whatever slots are active.  Every step: the model's block rows go into the pool
+    through the table, attention, greedy verification and the paged commit run on the GPU, and all of
+    it -- attention output, accepted counts, the whole pool bit for bit, the lengths -- is compared
+    with the oracle working on a host mirror of the pool."""
+    k, Hh, d, V, P = 3, 2, 64, 500, 128
+    n_q = (k + 1) ** 2
+    n_pages, pps, slots = 9, 3, 3
+    rng = np.random.default_rng(2024)
+    bits = lambda shape: workloads.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+    pager = B.Pager(n_pages, pps, slots)
+    ctx = B.Context(device=0, max_batch=slots, n_q_heads=Hh, n_kv_heads=Hh, head_dim=d, k_max=k, vocab=V, s_cap=pps * P)
+    kp = np.full((n_pages, Hh, P, d), 0x7FC0, dtype=np.uint16)     # host mirror, NaN wherever no row lives
+    vp = kp.copy()
+    length = {}
+
+    def write_rows(slot, s0, n):
+        t = pager.batch_table([slot])[0]
+        for s in range(s0, s0 + n):
+            kp[t[s // P], :, s % P, :] = bits((Hh, d))
+            vp[t[s // P], :, s % P, :] = bits((Hh, d))
+
+    def admit(L):
+        s = pager.admit()
+        pager.reserve(s, L)
+        write_rows(s, 0, L)                                        # the prompt's rows
+        length[s] = L
+        return s
+
+    a, b_ = admit(120), admit(5)
+    events = {3: ("admit", 250), 5: ("release", a), 6: ("admit", 100)}
+    accepted_total, reused = 0, False
+    for step in range(9):
+        if step in events:
+            kind, arg = events[step]
+            if kind == "admit":
+                s_new = admit(arg)
+                reused |= step == 6 and s_new == a
+            else:
+                pager.release(arg)
+                del length[arg]
+        batch = sorted(length)
+        Bn = len(batch)
+        for s in batch:
+            pager.reserve(s, length[s] + n_q)
+            write_rows(s, length[s], n_q)                          # the model's K / V rows of this step's block
+        table = pager.batch_table(batch)
+        L = np.array([length[s] for s in batch], dtype=np.int32)
+        q = bits((Bn, n_q, Hh, d))
+        logits = (rng.standard_normal((Bn, n_q, V)) * 2).astype(np.float32)
+        cand = rng.integers(0, V, size=(Bn, k)).astype(np.int32)
+        for i in range(Bn):
+            for j in range(k):
+                if rng.random() < 0.7:
+                    logits[i, j * (k + 1), cand[i, j]] = 30.0      # the model agrees with this candidate
+        dev = dict(kp=H.to_dev(kp), vp=H.to_dev(vp), table=H.to_dev(table), L=H.to_dev(L), q=H.to_dev(q),
+                   logits=H.to_dev(logits), cand=H.to_dev(cand), cprob=torch.ones((Bn, k), device="cuda"))
+        out = torch.full((Bn, n_q, Hh, d), float("nan"), device="cuda")
+        status = torch.zeros(Bn, dtype=torch.int32, device="cuda")
+        i32 = lambda *sh: torch.full(sh, -7, dtype=torch.int32, device="cuda")
+        n_acc, toks, n_out, ncand, L_out = i32(Bn), i32(Bn, k + 1), i32(Bn), i32(Bn, k), i32(Bn)
+        nprob = torch.zeros((Bn, k), device="cuda")
+        fin = torch.zeros(Bn, dtype=torch.uint8, device="cuda")
+        ctx.space_attn_step(ctx.attn_args(dev["q"], dev["kp"], dev["vp"], dev["L"], out, k, 0.125, status=status,
+                                          page_table=dev["table"]))
+        v = ctx.verify_args(dev["logits"], dev["cand"], dev["cprob"], dev["L"], n_acc, toks, n_out, ncand, nprob, fin, k,
+                            status=status)
+        c = ctx.commit_args(dev["kp"], dev["vp"], n_acc, dev["L"], k, kv_len_out=L_out, status=status,
+                            page_table=dev["table"])
+        ctx.space_verify_commit(v, c)
+        torch.cuda.synchronize()
+        # ---- the same step in the oracle, on the mirror ----
+        ref, _ = attention_step_paged(q, kp, vp, table, L, k, 0.125)
+        H.check_attention(out.cpu().numpy().astype(np.float64), ref, f"step {step}")
+        r = verify_step(logits, cand, np.ones((Bn, k)), k, "greedy")
+        assert np.array_equal(n_acc.cpu().numpy(), r["n_accept"])
+        new_len = commit_step_paged(kp, vp, table, L, r["n_accept"], k)
+        assert np.array_equal(L_out.cpu().numpy(), new_len)
+        assert np.array_equal(H.bf16_to_bits(dev["kp"]), kp) and np.array_equal(H.bf16_to_bits(dev["vp"]), vp)
+        assert int(status.abs().sum()) == 0
+        for i, s in enumerate(batch):
+            length[s] = int(new_len[i])
+        accepted_total += int(r["n_accept"].sum())
+    assert accepted_total > 5 and reused          # pages and the slot of the sequence that left were used again
+    assert max(length.values()) > P               # at least one sequence grew across a page boundary
+    pager.close()
