@@ -589,6 +589,8 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   pdl_wait();
   int Lc = 0;
   if (p.do_commit) Lc = p.cm.kv_len[b];                     // in flight during the scan
+  // (the candidates too: the block that finishes the sequence must not start a memory round trip for them)
+  const int my_cand = threadIdx.x < p.k ? p.cand[b * p.k + threadIdx.x] : 0;
   Stat st = scan_chunk<T, VECTOR, false, STAT_SUM>(row, begin, end, C1, -1, 0, 0, 0, 0, 0);
   // KV commit on board: which candidates are accepted is known only to the last block, at the very
   // end, so every block moves its slice of ALL k candidate rows now, while the logits stream.
@@ -597,33 +599,70 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   // candidates' rows instead.
   if (p.do_commit && commit_fits(p.cm, Lc))
     commit_rows(p.cm, b, Lc, p.k, row_i * p.n_chunks + ch, p.n_q * p.n_chunks, threadIdx.x, blockDim.x);
-  st = block_reduce_plain(st, C1);
+  // ---- block result and arrival: two block barriers in all.  Every warp reduces its own
+  // (maximum, arg-max, sum); eight lanes of warp 0 combine the warps, and lane 0 publishes the
+  // chunk's result, fences it and counts the block in.
+  constexpr int NW = SPACE_VERIFY_THREADS / 32;
+  __shared__ float wm[NW], ws[NW];
+  __shared__ int wi[NW];
+  __shared__ int sh_last;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  {
+    float m = st.m; int idx = st.idx;
+    warp_max_idx(m, idx);
+    float sv = (st.m > -CUDART_INF_F) ? st.s * fast_exp2((st.m - m) * C1) : 0.f;
+    sv = warp_sum(sv);
+    if (lane == 0) { wm[warp] = m; wi[warp] = idx; ws[warp] = sv; }
+  }
+  __syncthreads();
   VerifyPartial* pb = fpart + (int64_t)b * SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS;
-  if (threadIdx.x == 0) store_partial(pb + row_i * p.n_chunks + ch, st);
-  if (!arrive_last(p.counter_a + b, p.n_q * p.n_chunks)) return;
+  if (warp == 0) {
+    float m = lane < NW ? wm[lane] : -CUDART_INF_F;
+    int idx = lane < NW ? wi[lane] : 0x7FFFFFFF;
+    const float own = m;
+    warp_max_idx(m, idx, NW);
+    float sv = (lane < NW && own > -CUDART_INF_F) ? ws[lane] * fast_exp2((own - m) * C1) : 0.f;
+    sv = warp_sum(sv, NW);
+    if (lane == 0) {
+      Stat r = stat_empty();
+      r.m = m; r.idx = idx; r.s = sv;
+      store_partial(pb + row_i * p.n_chunks + ch, r);
+      __threadfence();
+      const int prev = atomicAdd(p.counter_a + b, 1);
+      const int last = prev == p.n_q * p.n_chunks - 1;
+      if (last) p.counter_a[b] = 0;                         // ready for the next launch
+      sh_last = last;
+    }
+  }
+  __syncthreads();                                          // (also: every thread's read of the old length precedes the arrival)
+  if (!sh_last) return;
+  __threadfence();
 
   // ---- last block of sequence b -------------------------------------------
-  __shared__ float sh_m[SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS];
-  __shared__ float sh_s[SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS];
-  __shared__ int sh_i[SPACE_MAX_ROWS * SPACE_FUSED_MAX_CHUNKS];
   __shared__ float row_s[SPACE_MAX_ROWS];
   __shared__ int row_idx[SPACE_MAX_ROWS];
   __shared__ int sh_cand[SPACE_MAX_K];
-  const int total = p.n_q * p.n_chunks;
-  for (int t = threadIdx.x; t < total; t += blockDim.x) {   // every chunk result, one round trip
-    sh_m[t] = __ldcg(&pb[t].m); sh_s[t] = __ldcg(&pb[t].s); sh_i[t] = __ldcg(&pb[t].idx);
+  if (threadIdx.x < p.k) sh_cand[threadIdx.x] = my_cand;
+  // two rows per warp at a time: lanes 0..15 and 16..31 each fetch and reduce one row's chunk results
+  // (all fetches of a warp are in flight together)
+  constexpr int RPW = (SPACE_MAX_ROWS + 2 * NW - 1) / (2 * NW);   // row pairs per warp at most
+  float pm[RPW], ps[RPW]; int pi[RPW];
+  const int cl = lane & 15;
+#pragma unroll
+  for (int it = 0; it < RPW; ++it) {
+    const int r = (warp + it * NW) * 2 + (lane >> 4);
+    pm[it] = -CUDART_INF_F; ps[it] = 0.f; pi[it] = 0x7FFFFFFF;
+    if (r < p.n_q && cl < p.n_chunks) {
+      const VerifyPartial* q = pb + r * p.n_chunks + cl;
+      pm[it] = __ldcg(&q->m); ps[it] = __ldcg(&q->s); pi[it] = __ldcg(&q->idx);
+    }
   }
-  if (threadIdx.x < p.k) sh_cand[threadIdx.x] = p.cand[b * p.k + threadIdx.x];
-  __syncthreads();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // two rows per warp at a time: lanes 0..15 and 16..31 each reduce one row's chunks
-  for (int r0 = warp * 2; r0 < p.n_q; r0 += 2 * (SPACE_VERIFY_THREADS / 32)) {
-    const int r = r0 + (lane >> 4), cl = lane & 15;
-    float m = -CUDART_INF_F, sv = 0.f; int idx = 0x7FFFFFFF;
-    if (r < p.n_q && cl < p.n_chunks) { m = sh_m[r * p.n_chunks + cl]; sv = sh_s[r * p.n_chunks + cl]; idx = sh_i[r * p.n_chunks + cl]; }
-    float bm = m; int bi = idx;
+#pragma unroll
+  for (int it = 0; it < RPW; ++it) {
+    const int r = (warp + it * NW) * 2 + (lane >> 4);
+    float bm = pm[it]; int bi = pi[it];
     warp_max_idx(bm, bi, 16);
-    sv = (m > -CUDART_INF_F) ? sv * fast_exp2((m - bm) * C1) : 0.f;
+    float sv = (pm[it] > -CUDART_INF_F) ? ps[it] * fast_exp2((pm[it] - bm) * C1) : 0.f;
     sv = warp_sum(sv, 16);
     if (cl == 0 && r < p.n_q) { row_s[r] = sv; row_idx[r] = bi; }
   }
