@@ -514,7 +514,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_rows_kernel(const __grid_cons
           // Paged cache, last tile: the page's rows past the last key may hold anything, and 0 * NaN
           // would reach the output.  Once the V tile has landed the softmax threads clear those rows
           // (128 contiguous bytes per row and 64-wide half of d, whatever the swizzle inside them).
+          // The softmax may run up to NS tiles ahead of the O product, the V ring has fewer stages:
+          // first make sure that the stage's previous tile has been consumed, so that the wait below
+          // looks at the barrier phase of THIS tile and the stores cannot hit the tile before it.
           const uint32_t vs = gt % S::V_STAGES;
+          if (gt >= (uint32_t)S::V_STAGES) {
+            const uint32_t pg = gt - S::V_STAGES;
+            ok &= mbar_wait(BAR(B_PVDONE + pg % NS), (pg / NS) & 1, abort_flag, p.err, 18);
+          }
           ok &= mbar_wait(BAR(B_VFULL + vs), (gt / S::V_STAGES) & 1, abort_flag, p.err, 17);
           const int first_bad = n_keys - kt;
           for (int it = first_bad * S::HALVES + sidx; it < TILE_N * S::HALVES; it += n_soft) {

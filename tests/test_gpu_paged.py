@@ -220,3 +220,45 @@ def test_continuous_batching_over_a_shared_pool(B, H):
     assert accepted_total > 5 and reused          # pages and the slot of the sequence that left were used again
     assert max(length.values()) > P               # at least one sequence grew across a page boundary
     pager.close()
+
+
+@pytest.mark.parametrize("name,over,heads_per_seq", [
+    ("ragged16", {}, 4),                       # the transposed kernel at full size, 16 ragged sequences
+    ("sampling64", {"B": 8}, 2),               # grouped heads: the row kernel, eight of the 64 sequences
+])
+def test_paged_step_at_full_size(B, H, name, over, heads_per_seq):
+    """A whole step of a full-size configuration on a paged cache: attention on seeded (sequence, head)
+    pairs against the oracle over the rows the table names, the verify + commit call's lengths and the
+    whole pools after the commit against oracle.paged."""
+    from oracle.attention import attention_head
+    from oracle.paged import gather_cache
+    cfg = workloads.resolve(name, **over)
+    x = workloads.to_pages(workloads.make_step_inputs(cfg), seed=3)
+    ctx = H.make_context(cfg, x)
+    ds = H.DeviceStep(cfg, x)
+    k = cfg["k"]
+    sample = cfg["mode"] == "sample"
+    ds.attn(ctx)
+    ds.verify_commit(ctx, mode=B.MODE_SAMPLE if sample else B.MODE_GREEDY, temperature=cfg["temperature"], seed=cfg["seed"])
+    torch.cuda.synchronize()
+    assert int(ds.status.abs().sum()) == 0
+    out = ds.out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(out).all()
+    G = cfg["H_q"] // cfg["H_kv"]
+    rng = np.random.default_rng(cfg["seed"])
+    n_rows = x["kv_len"].astype(np.int64) + x["n_q"]
+    for b in range(cfg["B"]):
+        heads = sorted(rng.choice(cfg["H_q"], size=heads_per_seq, replace=False).tolist())
+        L = int(x["kv_len"][b])
+        kb = gather_cache(x["k_cache"], x["page_table"][b:b + 1], n_rows[b:b + 1])[0]      # [H_kv, rows, d]
+        vb = gather_cache(x["v_cache"], x["page_table"][b:b + 1], n_rows[b:b + 1])[0]
+        refs = np.stack([attention_head(x["q"][b, :, h], kb[h // G], vb[h // G], L, k, x["scale"])[0] for h in heads])
+        H.check_attention(out[b][:, heads].transpose(1, 0, 2)[None], refs[None], f"{name} paged b={b}")
+    n_acc = ds.n_accept.cpu().numpy()
+    kp, vp = x["k_cache"].copy(), x["v_cache"].copy()
+    new_len = commit_step_paged(kp, vp, x["page_table"], x["kv_len"], n_acc, k)
+    assert np.array_equal(ds.kv_len_out.cpu().numpy(), new_len)
+    assert np.array_equal(H.bf16_to_bits(ds.k_cache), kp) and np.array_equal(H.bf16_to_bits(ds.v_cache), vp)
+    if not sample:
+        r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "greedy")
+        assert np.array_equal(n_acc, r["n_accept"])
