@@ -3,7 +3,8 @@ head counts, GQA group, head_dim, k and ragged lengths drawn at random (fixed
 seeds), each case against the fp64 oracle.  The shapes are chosen to cross the
 boundaries of the work partition: one tile per sequence, more (sequence, head)
 pairs than thread blocks, a single long sequence cut over every block, query
-blocks of one or several 64/128-row pieces."""
+blocks of one or several 64/128-row pieces.  Every case runs on the contiguous cache and on
+the same cache cut into pages."""
 import numpy as np
 import pytest
 import torch
@@ -50,11 +51,16 @@ def test_attention_shape_sweep(B, seed):
                             logits_dtype="f32", sigma=2.0, p_accept=(0.5, 0.5), seed=c["seed"])
     x = workloads.make_step_inputs(cfg, poison_tail=True)
     ref, ref_lse = attention_step(x["q"], x["k_cache"], x["v_cache"], x["kv_len"], c["k"], x["scale"])
-    ctx = H.make_context(cfg, x)
-    for impl in (B.ATTN_TENSOR, B.ATTN_TENSOR_ROWS):
-        ds = H.DeviceStep(cfg, x)
-        ds.attn(ctx, impl=impl)
-        torch.cuda.synchronize()
-        assert int(ds.status.abs().sum()) == 0, (c, impl)
-        H.check_attention(ds.out.cpu().numpy().astype(np.float64), ref, f"sweep {c} impl {impl}")
-        np.testing.assert_allclose(ds.lse.cpu().numpy(), ref_lse, rtol=0, atol=2e-3)
+    # the same caches once more as page pools behind a shuffled table, NaN wherever no key lives: the
+    # result must not change (the oracle's paged form is pinned to the contiguous one on the CPU)
+    xp = workloads.to_pages(x, seed=seed)
+    for xi, what in ((x, "contiguous"), (xp, "paged")):
+        ctx = H.make_context(cfg, xi)
+        for impl in (B.ATTN_TENSOR, B.ATTN_TENSOR_ROWS):
+            for rep in range(2 if what == "paged" else 1):    # (a second launch meets other timings)
+                ds = H.DeviceStep(cfg, xi)
+                ds.attn(ctx, impl=impl)
+                torch.cuda.synchronize()
+                assert int(ds.status.abs().sum()) == 0, (c, impl, what)
+                H.check_attention(ds.out.cpu().numpy().astype(np.float64), ref, f"sweep {c} impl {impl} {what}")
+                np.testing.assert_allclose(ds.lse.cpu().numpy(), ref_lse, rtol=0, atol=2e-3)
