@@ -120,6 +120,14 @@ class ClockSampler:
             nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
             nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
         }
+        # further reasons, recorded when the binding knows them (a clock below the maximum then has a name:
+        # a short timed region catches the clocks between idle and load)
+        for attr, name in (("nvmlClocksThrottleReasonGpuIdle", "gpu_idle"),
+                           ("nvmlClocksThrottleReasonApplicationsClocksSetting", "applications_clocks_setting"),
+                           ("nvmlClocksThrottleReasonHwPowerBrakeSlowdown", "hw_power_brake_slowdown"),
+                           ("nvmlClocksThrottleReasonSyncBoost", "sync_boost")):
+            if hasattr(nv, attr):
+                names[getattr(nv, attr)] = name
         while not self._stop.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
