@@ -100,7 +100,7 @@ class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU through NVML while running."""
 
     def __init__(self, index):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.reasons, self.other, self.max_mhz = [], set(), set(), None
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -120,14 +120,15 @@ class ClockSampler:
             nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
             nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
         }
-        # further reasons, recorded when the binding knows them (a clock below the maximum then has a name:
-        # a short timed region catches the clocks between idle and load)
+        # further clock-event reasons, kept apart ("other_reasons"): a clock below the maximum then has a
+        # name (a short timed region catches the clocks between idle and load)
+        others = {}
         for attr, name in (("nvmlClocksThrottleReasonGpuIdle", "gpu_idle"),
                            ("nvmlClocksThrottleReasonApplicationsClocksSetting", "applications_clocks_setting"),
                            ("nvmlClocksThrottleReasonHwPowerBrakeSlowdown", "hw_power_brake_slowdown"),
                            ("nvmlClocksThrottleReasonSyncBoost", "sync_boost")):
             if hasattr(nv, attr):
-                names[getattr(nv, attr)] = name
+                others[getattr(nv, attr)] = name
         while not self._stop.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
@@ -135,6 +136,9 @@ class ClockSampler:
                 for bit, name in names.items():
                     if r & bit:
                         self.reasons.add(name)
+                for bit, name in others.items():
+                    if r & bit:
+                        self.other.add(name)
             except Exception:
                 pass
             self._stop.wait(0.005)
@@ -150,7 +154,7 @@ class ClockSampler:
             self._thread.join()
         med = float(np.median(self.samples)) if self.samples else None
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                "other_reasons": sorted(self.other), "samples": len(self.samples)}
 
 
 # ------------------------------------------------------------------- CPU oracle
