@@ -76,7 +76,19 @@ __device__ __forceinline__ void list_insert(unsigned long long& mine, unsigned l
 __device__ __forceinline__ float ld_logit(const float* p) { return *p; }
 __device__ __forceinline__ float ld_logit(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 
-template <typename T>
+// 16 bytes of logits as floats
+__device__ __forceinline__ void unpack16(const uint4& v, float (&f)[4], const float*) {
+  f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+}
+__device__ __forceinline__ void unpack16(const uint4& v, float (&f)[8], const __nv_bfloat16*) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
+}
+
+// VECTOR: the row and the chunk start are 16-byte aligned (the launcher checks): every lane fetches four
+// 16-byte pieces per sweep, all in flight together, instead of one logit at a time.
+template <typename T, bool VECTOR>
 __global__ void __launch_bounds__(FILT_THREADS) verify_filter_kernel(const FiltParams p) {
   pdl_launch_dependents();
   pdl_wait();
@@ -91,7 +103,40 @@ __global__ void __launch_bounds__(FILT_THREADS) verify_filter_kernel(const FiltP
 
   // ---- this warp's top-K of its share of the chunk ------------------------------------
   unsigned long long mine = 0ull;
-  for (int x0 = begin + warp * 32; x0 < end; x0 += FILT_THREADS) {
+  int scalar_from = begin;                                  // what the one-by-one loop below still has to look at
+  if (VECTOR) {
+    constexpr int N = 16 / (int)sizeof(T), U = 4;
+    const int full_end = begin + ((end - begin) / N) * N;
+    constexpr int stride = FILT_THREADS * N;
+    unsigned long long tau = 0ull;                          // the warp's K-th key so far (0: fewer than K keys)
+    for (int xw = begin + warp * 32 * N; xw < full_end; xw += U * stride) {   // (the same trip count in every lane)
+      uint4 v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int x = xw + lane * N + u * stride;
+        v[u] = x < full_end ? __ldg(reinterpret_cast<const uint4*>(row + x)) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int x = xw + lane * N + u * stride;
+        float f[N];
+        unpack16(v[u], f, (const T*)nullptr);
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+          const unsigned long long key = x < full_end ? make_key(f[i], x + i) : 0ull;
+          unsigned pass = __ballot_sync(0xFFFFFFFFu, key > tau);
+          while (pass) {
+            const int src = __ffs(pass) - 1;
+            pass &= pass - 1;
+            list_insert(mine, shfl64(key, src), K, lane);
+            tau = shfl64(mine, K - 1);
+          }
+        }
+      }
+    }
+    scalar_from = full_end;                                 // (fewer than N logits, looked at by every warp: keys are unique, a
+  }                                                         //  second look at one changes nothing -- but only warp 0 does it)
+  for (int x0 = scalar_from + (VECTOR ? 0 : warp * 32); x0 < end && (!VECTOR || warp == 0); x0 += VECTOR ? 32 : FILT_THREADS) {
     const int x = x0 + lane;
     const unsigned long long key = x < end ? make_key(ld_logit(row + x), x) : 0ull;
     const unsigned long long tau = shfl64(mine, K - 1);
@@ -302,20 +347,27 @@ int launch_verify_filtered(space_ctx* ctx, const space_verify_args* a, cudaStrea
   p.part = reinterpret_cast<unsigned long long*>(ctx->vtopk);
   // about two blocks per SM over the (k+1) rows of every sequence, at least 8192 logits per block
   const int rows = a->batch * (a->k + 1);
-  int nc = (2 * ctx->sm_count + rows - 1) / rows;
+  int nc = (2 * ctx->sm_count + rows - 1) / rows;   // (4, 8, 16 per SM measured slower: every block starts from an empty list)
   const int max_nc = (a->vocab + 8191) / 8192;
   if (nc > max_nc) nc = max_nc;
   if (nc > FILT_MAX_CHUNKS) nc = FILT_MAX_CHUNKS;
   if (nc < 1) nc = 1;
-  p.chunk = (a->vocab + nc - 1) / nc;
+  p.chunk = (((a->vocab + nc - 1) / nc + 7) / 8) * 8;       // chunk starts stay 16-byte aligned
   p.n_chunks = (a->vocab + p.chunk - 1) / p.chunk;
+  const int esz = a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2;
+  const bool vector = ((uintptr_t)a->logits % 16 == 0) && ((a->logits_row_stride * esz) % 16 == 0);
   for (int phase = 0; phase < 2; ++phase) {
     p.phase = phase;
     p.counter = ctx->counters + (phase == 0 ? 0 : ctx->cfg.max_batch);
     const dim3 grid(p.n_chunks, phase == 0 ? a->k + 1 : a->k, a->batch);
     ProfScope ps(ctx, phase == 0 ? SPACE_K_VERIFY_TARGET : SPACE_K_VERIFY_EMIT, st);
-    if (a->logits_dtype == SPACE_DTYPE_F32) launch_pdl(verify_filter_kernel<float>, grid, dim3(FILT_THREADS), 0, st, p);
-    else launch_pdl(verify_filter_kernel<__nv_bfloat16>, grid, dim3(FILT_THREADS), 0, st, p);
+    if (a->logits_dtype == SPACE_DTYPE_F32) {
+      if (vector) launch_pdl(verify_filter_kernel<float, true>, grid, dim3(FILT_THREADS), 0, st, p);
+      else launch_pdl(verify_filter_kernel<float, false>, grid, dim3(FILT_THREADS), 0, st, p);
+    } else {
+      if (vector) launch_pdl(verify_filter_kernel<__nv_bfloat16, true>, grid, dim3(FILT_THREADS), 0, st, p);
+      else launch_pdl(verify_filter_kernel<__nv_bfloat16, false>, grid, dim3(FILT_THREADS), 0, st, p);
+    }
   }
   ctx->launches += 2;
   return cuda_ok(cudaGetLastError());
