@@ -241,9 +241,16 @@ def run_ours(args):
     torch.cuda.set_device(local)
     replicas.init("nccl", local)
 
-    cfg = workloads.resolve(args.config, **({"B": args.batch} if args.batch else {}))
+    over = {}
+    if args.batch:
+        over["B"] = args.batch
+    if args.k:
+        over["k"] = args.k
+    cfg = workloads.resolve(args.config, **over)
     if args.batch:
         cfg["name"] = f"{args.config}@batch{args.batch}"   # a reduced copy of the workload (profiler captures)
+    if args.k:
+        cfg["name"] += f"@k{args.k}"                       # another number of mask tokens (Sec. 4.3: k = 2 beats k = 5 from batch 8)
     if args.paged:
         cfg["name"] += "+paged"                            # (no profiler capture of this form: traffic stays null)
     k, n_q = cfg["k"], workloads.n_block_rows(cfg["k"])
@@ -673,6 +680,7 @@ def main():
                          "captures; the bench line then names the workload NAME@batchN)")
     ap.add_argument("--separate-commit", action="store_true",
                     help="three calls per step (space_verify, then space_kv_commit) instead of space_verify_commit")
+    ap.add_argument("--k", type=int, default=0, help="number of mask tokens k instead of the workload's own")
     ap.add_argument("--paged", action="store_true",
                     help="keep the KV caches as page pools behind page tables (attention and commit through the table)")
     ap.add_argument("--attn-impl", default="tensor", choices=["tensor", "rows"],
