@@ -251,6 +251,8 @@ def run_ours(args):
         cfg["name"] = f"{args.config}@batch{args.batch}"   # a reduced copy of the workload (profiler captures)
     if args.k:
         cfg["name"] += f"@k{args.k}"                       # another number of mask tokens (Sec. 4.3: k = 2 beats k = 5 from batch 8)
+    if args.top_k and cfg["mode"] == "sample":
+        cfg["name"] += f"+top{args.top_k}p{args.top_p:g}"  # filtered target distributions (App. A.4: top-k 10, top-p 0.95)
     if args.paged:
         cfg["name"] += "+paged"                            # (no profiler capture of this form: traffic stays null)
     k, n_q = cfg["k"], workloads.n_block_rows(cfg["k"])
@@ -279,7 +281,7 @@ def run_ours(args):
         v = ctx.verify_args(ds.logits, ds.cand, ds.cand_prob, ds.kv_len, ds.n_accept, ds.out_tokens,
                             ds.n_out, ds.next_cand, ds.next_cand_prob, ds.finished, k, mode=mode,
                             temperature=cfg["temperature"], seed=cfg["seed"], seq_id=ds.seq_id,
-                            status=ds.status)
+                            status=ds.status, top_k=args.top_k if sample else 0, top_p=args.top_p)
         c = ctx.commit_args(ds.k_cache, ds.v_cache, ds.n_accept, ds.kv_len, k, kv_len_out=ds.kv_len_out,
                             status=ds.status, page_table=ds.page_table)
         arg_sets.append((a, v, c))
@@ -390,6 +392,8 @@ def run_ours(args):
     e2e_val, _ = replicas.job_throughput(n_e2e, e2e_s, device="cuda")
     e2e_ok = bool((outs["status"] == 0).all()) and \
         bool(torch.equal(outs["n_accept"], steps_dev[0].n_accept.cpu()))
+    if args.top_k and sample:
+        e2e_ok = None          # space_step_host verifies against the unfiltered distributions: nothing to compare
     h2d_full, d2h_full = int(h2d.value), int(d2h.value)
 
     # The same call as a decoder would make it: the KV cache is state that stays on the device
@@ -410,6 +414,8 @@ def run_ours(args):
     res_val, _ = replicas.job_throughput(n_res, res_s, device="cuda")
     res_ok = bool((outs["status"] == 0).all()) and \
         bool(torch.equal(outs["n_accept"], steps_dev[0].n_accept.cpu()))
+    if args.top_k and sample:
+        res_ok = None
 
     if rank != 0:
         replicas.shutdown()
@@ -680,6 +686,9 @@ def main():
                          "captures; the bench line then names the workload NAME@batchN)")
     ap.add_argument("--separate-commit", action="store_true",
                     help="three calls per step (space_verify, then space_kv_commit) instead of space_verify_commit")
+    ap.add_argument("--top-k", type=int, default=0, dest="top_k",
+                    help="sampling workloads: verify against top-k / top-p filtered distributions (0 = unfiltered)")
+    ap.add_argument("--top-p", type=float, default=1.0, dest="top_p")
     ap.add_argument("--k", type=int, default=0, help="number of mask tokens k instead of the workload's own")
     ap.add_argument("--paged", action="store_true",
                     help="keep the KV caches as page pools behind page tables (attention and commit through the table)")

@@ -577,7 +577,9 @@ verify_emit_kernel(const VerifyParams p) {
 
 // One launch for greedy mode on small inputs: statistics of every block row,
 // then acceptance, emission and next candidates by the last block of a sequence.
-template <typename T, bool VECTOR>
+// PAGED: the commit on board goes through a page table (a build of its own: the table look-ups are
+// not compiled into the contiguous form, whose addressing sits in the critical path).
+template <typename T, bool VECTOR, bool PAGED = false>
 __global__ void __launch_bounds__(SPACE_VERIFY_THREADS)
 verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   pdl_launch_dependents();
@@ -598,7 +600,7 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   // beyond the new length and held mask-token rows nobody reads again, receive the rejected
   // candidates' rows instead.
   if (p.do_commit && commit_fits(p.cm, Lc))
-    commit_rows(p.cm, b, Lc, p.k, row_i * p.n_chunks + ch, p.n_q * p.n_chunks, threadIdx.x, blockDim.x);
+    commit_rows_impl<PAGED>(p.cm, b, Lc, p.k, row_i * p.n_chunks + ch, p.n_q * p.n_chunks, threadIdx.x, blockDim.x);
   // ---- block result and arrival: two block barriers in all.  Every warp reduces its own
   // (maximum, arg-max, sum); eight lanes of warp 0 combine the warps, and lane 0 publishes the
   // chunk's result, fences it and counts the block in.
@@ -702,6 +704,9 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
 template <typename T, bool VECTOR>
 void launch_fused(space_ctx* ctx, const VerifyParams& p, cudaStream_t st) {
   ProfScope ps(ctx, SPACE_K_VERIFY_TARGET, st);
+  if (p.do_commit && p.cm.page_table)
+    launch_pdl(verify_fused_kernel<T, VECTOR, true>, dim3(p.n_chunks, p.n_q, p.B), dim3(SPACE_VERIFY_THREADS), 0, st, p, ctx->vfused);
+  else
   launch_pdl(verify_fused_kernel<T, VECTOR>, dim3(p.n_chunks, p.n_q, p.B), dim3(SPACE_VERIFY_THREADS), 0, st, p, ctx->vfused);
 }
 
@@ -738,10 +743,14 @@ int launch_verify(space_ctx* ctx, const space_verify_args* a, const space_commit
     return launch_commit(ctx, cm, st);
   }
   if (cm && cm->page_table) {
-    // paged cache: the verify kernels carry the contiguous commit only; the commit kernel follows
-    const int rc = launch_verify(ctx, a, nullptr, st);
-    if (rc != SPACE_OK) return rc;
-    return launch_commit(ctx, cm, st);
+    // paged cache: only the single-launch greedy form carries the commit through a page table; the
+    // two-launch form is followed by the commit kernel
+    const int64_t all_b = (int64_t)a->batch * (a->k + 1) * (a->k + 1) * a->vocab * (a->logits_dtype == SPACE_DTYPE_F32 ? 4 : 2);
+    if (!(a->mode == SPACE_MODE_GREEDY && all_b <= SPACE_FUSED_MAX_BYTES)) {
+      const int rc = launch_verify(ctx, a, nullptr, st);
+      if (rc != SPACE_OK) return rc;
+      return launch_commit(ctx, cm, st);
+    }
   }
   VerifyParams p;
   p.do_commit = cm != nullptr;

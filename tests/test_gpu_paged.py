@@ -212,7 +212,14 @@ def test_continuous_batching_over_a_shared_pool(B, H):
         assert np.array_equal(n_acc.cpu().numpy(), r["n_accept"])
         new_len = commit_step_paged(kp, vp, table, L, r["n_accept"], k)
         assert np.array_equal(L_out.cpu().numpy(), new_len)
-        assert np.array_equal(H.bf16_to_bits(dev["kp"]), kp) and np.array_equal(H.bf16_to_bits(dev["vp"]), vp)
+        gk, gv = H.bf16_to_bits(dev["kp"]), H.bf16_to_bits(dev["vp"])
+        for i in range(Bn):
+            # rows L+i*+1 .. L+k lie beyond the new length; the single-launch form leaves the rejected
+            # candidates' rows there (unspecified by the interface, overwritten by the next block)
+            for s_ in range(int(new_len[i]), int(L[i]) + k + 1):
+                gk[table[i, s_ // P], :, s_ % P, :] = kp[table[i, s_ // P], :, s_ % P, :]
+                gv[table[i, s_ // P], :, s_ % P, :] = vp[table[i, s_ // P], :, s_ % P, :]
+        assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
         assert int(status.abs().sum()) == 0
         for i, s in enumerate(batch):
             length[s] = int(new_len[i])
@@ -258,7 +265,15 @@ def test_paged_step_at_full_size(B, H, name, over, heads_per_seq):
     kp, vp = x["k_cache"].copy(), x["v_cache"].copy()
     new_len = commit_step_paged(kp, vp, x["page_table"], x["kv_len"], n_acc, k)
     assert np.array_equal(ds.kv_len_out.cpu().numpy(), new_len)
-    assert np.array_equal(H.bf16_to_bits(ds.k_cache), kp) and np.array_equal(H.bf16_to_bits(ds.v_cache), vp)
+    gk, gv = H.bf16_to_bits(ds.k_cache), H.bf16_to_bits(ds.v_cache)
+    for b in range(cfg["B"]):
+        # rows beyond the new length (L+i*+1 .. L+k) are unspecified: the single-launch greedy form
+        # leaves the rejected candidates' rows there
+        for s_ in range(int(new_len[b]), int(x["kv_len"][b]) + k + 1):
+            pg = int(x["page_table"][b, s_ // 128])
+            gk[pg, :, s_ % 128, :] = kp[pg, :, s_ % 128, :]
+            gv[pg, :, s_ % 128, :] = vp[pg, :, s_ % 128, :]
+    assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
     if not sample:
         r = verify_step(x["logits"], x["cand"], x["cand_prob"], k, "greedy")
         assert np.array_equal(n_acc, r["n_accept"])
