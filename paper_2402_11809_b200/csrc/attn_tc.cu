@@ -99,8 +99,15 @@ struct Seg {
 __device__ unsigned long long g_timeline[256 * TL_POINTS];
 #define TL(i) do { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); \
                    g_timeline[blockIdx.x * TL_POINTS + (i)] = t_; } while (0)
+// the same for the merge kernel: four points per thread block (entry, dependency wait returned,
+// descriptor in registers, output stored), written by thread 0
+__device__ unsigned long long g_timeline_merge[4096 * 4];
+#define TLM(i) do { if (threadIdx.x == 0 && blockIdx.y * gridDim.x + blockIdx.x < 4096) { unsigned long long t_; \
+                   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); \
+                   g_timeline_merge[(blockIdx.y * gridDim.x + blockIdx.x) * 4 + (i)] = t_; } } while (0)
 #else
 #define TL(i) do { } while (0)
+#define TLM(i) do { } while (0)
 #endif   // slot: partial slot; dfirst/dn: cut (aligned mode)
 
 // PTX helpers: tc_common.cuh.  Every wait of this kernel is bounded by WAIT_NS.
@@ -1137,8 +1144,10 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tc_kernel(const __grid_consta
 // grid = (B*H_kv*n_mblocks, ceil(rows*DH/4 / 128)), 128 threads.
 template <int DH>
 __global__ void __launch_bounds__(128) attn_merge_kernel(const AttnParams p) {
+  TLM(0);
   pdl_launch_dependents();
   pdl_wait();
+  TLM(1);
   constexpr int C4 = DH / 4;
   // Large batches: one grid column per attention thread block (each holds the last
   // piece of at most one cut); small ones: one per (sequence, head, row block).
@@ -1154,6 +1163,7 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(const AttnParams p) {
   const int2 d = __ldcg(p.desc + (size_t)item * p.n_mblocks + mb);
   if (L < 0 || (int64_t)L + p.n_q > p.s_cap) return;
   const int n = d.y;
+  TLM(2);
   if (n <= 1) return;                                       // written directly by the main kernel
   const int i0 = mb * p.rows_per_mb;
   const int m_valid = min(p.rows_per_mb, p.n_q - i0) * p.G;
@@ -1206,6 +1216,7 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(const AttnParams p) {
   }
   if (p.lse && c4 == 0)
     p.lse[((size_t)b * p.H_q + hq) * p.n_q + ri] = (mx + log2f(den)) * 0.6931471805599453f;
+  TLM(3);
 }
 
 // ------------------------------------------------------------------ host side
@@ -1288,6 +1299,9 @@ size_t attn_tensor_partial_floats(const space_config* cfg, int sm_count, size_t*
 #ifdef SPACE_TIMELINE
 extern "C" int space_debug_timeline_read(unsigned long long* host_dst, int n_blocks) {
   return cuda_ok(cudaMemcpyFromSymbol(host_dst, g_timeline, sizeof(unsigned long long) * TL_POINTS * n_blocks));
+}
+extern "C" int space_debug_timeline_read_merge(unsigned long long* host_dst, int n_blocks) {
+  return cuda_ok(cudaMemcpyFromSymbol(host_dst, g_timeline_merge, sizeof(unsigned long long) * 4 * n_blocks));
 }
 #endif
 

@@ -577,11 +577,24 @@ verify_emit_kernel(const VerifyParams p) {
 
 // One launch for greedy mode on small inputs: statistics of every block row,
 // then acceptance, emission and next candidates by the last block of a sequence.
+// Optional per-block timeline of the single-launch kernel (compiled in with -DSPACE_TIMELINE, as in
+// attn_tc.cu): entry, dependency wait returned, logits in registers, counted in, (finishing block) rows
+// reduced, done.  Written by thread 0.
+#ifdef SPACE_TIMELINE
+__device__ unsigned long long g_timeline_verify[4096 * 8];
+#define TLV(i) do { const int b_ = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x; \
+                    if (threadIdx.x == 0 && b_ < 4096) { unsigned long long t_; \
+                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_timeline_verify[b_ * 8 + (i)] = t_; } } while (0)
+#else
+#define TLV(i) do { } while (0)
+#endif
+
 // PAGED: the commit on board goes through a page table (a build of its own: the table look-ups are
 // not compiled into the contiguous form, whose addressing sits in the critical path).
 template <typename T, bool VECTOR, bool PAGED = false>
 __global__ void __launch_bounds__(SPACE_VERIFY_THREADS)
 verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
+  TLV(0);
   pdl_launch_dependents();
   const int b = blockIdx.z, row_i = blockIdx.y, ch = blockIdx.x;
   const int k1 = p.k + 1;
@@ -589,11 +602,15 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   const T* row = reinterpret_cast<const T*>(p.logits) + ((int64_t)b * p.n_q + row_i) * p.row_stride;
   const int begin = ch * p.chunk, end = min(p.V, begin + p.chunk);
   pdl_wait();
+  TLV(1);
   int Lc = 0;
   if (p.do_commit) Lc = p.cm.kv_len[b];                     // in flight during the scan
   // (the candidates too: the block that finishes the sequence must not start a memory round trip for them)
   const int my_cand = threadIdx.x < p.k ? p.cand[b * p.k + threadIdx.x] : 0;
   Stat st = scan_chunk<T, VECTOR, false, STAT_SUM>(row, begin, end, C1, -1, 0, 0, 0, 0, 0);
+#ifdef SPACE_TIMELINE
+  if (st.m != 12345.f) TLV(2);                              // (a use of the result: the stamp follows the loads)
+#endif
   // KV commit on board: which candidates are accepted is known only to the last block, at the very
   // end, so every block moves its slice of ALL k candidate rows now, while the logits stream.
   // Rows L+1 .. L+i* end up exactly as the plain commit leaves them; rows L+i*+1 .. L+k, which lie
@@ -637,6 +654,7 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
     }
   }
   __syncthreads();                                          // (also: every thread's read of the old length precedes the arrival)
+  TLV(3);
   if (!sh_last) return;
   __threadfence();
 
@@ -669,6 +687,7 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
     if (cl == 0 && r < p.n_q) { row_s[r] = sv; row_idx[r] = bi; }
   }
   __syncthreads();
+  TLV(4);
   if (threadIdx.x >= 32) return;
   // acceptance: longest prefix of candidates equal to the arg-max chain
   int i_star = 0, bits = 0;
@@ -697,6 +716,7 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
       if (p.status && bits) atomicOr(p.status + b, bits);
       // new length and index tables; every block of the sequence read the old length before it arrived
       if (p.do_commit) commit_tables(p.cm, b, Lc, i_star, commit_fits(p.cm, Lc));
+      TLV(5);
     }
   }
 }
@@ -734,6 +754,12 @@ __global__ void philox_debug_kernel(uint32_t k0, uint32_t k1, int64_t n, const u
 }
 
 }  // namespace
+
+#ifdef SPACE_TIMELINE
+extern "C" int space_debug_timeline_read_verify(unsigned long long* host_dst, int n_blocks) {
+  return cuda_ok(cudaMemcpyFromSymbol(host_dst, g_timeline_verify, sizeof(unsigned long long) * 8 * n_blocks));
+}
+#endif
 
 int launch_verify(space_ctx* ctx, const space_verify_args* a, const space_commit_args* cm, cudaStream_t st) {
   if (a->mode == SPACE_MODE_SAMPLE && a->top_k > 0) {
