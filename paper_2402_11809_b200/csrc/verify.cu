@@ -656,7 +656,9 @@ verify_fused_kernel(const VerifyParams p, VerifyPartial* fpart) {
   __syncthreads();                                          // (also: every thread's read of the old length precedes the arrival)
   TLV(3);
   if (!sh_last) return;
-  __threadfence();
+  // (No fence on this side: every chunk result was fenced by its writer before that block's count, the
+  // counts are ordered in L2, and the loads below go to L2 -- after the barrier that followed lane 0's own
+  // count.  A fence here would also wait for this thread's row stores of the commit.)
 
   // ---- last block of sequence b -------------------------------------------
   __shared__ float row_s[SPACE_MAX_ROWS];
