@@ -6,7 +6,7 @@ the regular one, replays a graph of eight steps of a single-sequence workload an
 after the attention kernel's dependency wait of the last step: when the attention blocks pass their stages
 (regular groups and helper groups apart), when the merge and verify blocks become resident, when their
 dependency waits return and when they finish.  What a kernel boundary costs and where a launch spends its
-time cannot be seen from outside the kernels; this is the tool the figures in the design doc come from.
+time cannot be seen from outside the kernels: a profiler serialises the launches.
 
 Usage: python -m paper_2402_11809_b200.timeline [workload]      (default llama7b; needs a B200)
 """
